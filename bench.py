@@ -1,0 +1,357 @@
+#!/usr/bin/env python
+"""Benchmark of the UBTree draft+verify hot path: drafted-and-verified trees per second.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3] [--impl ours|reference]
+
+A step is one pass of the whole path over one synthetic batch: ubt_draft_tree (vocabulary log-softmax +
+top-k, pair normalisation, tree expansion, mask/positions) followed by ubt_verify_tree (per-node target
+pick over [B,N,V] logits and the acceptance walk).  Prints ONE JSON line.  With torchrun (N > 1) every
+rank runs the same step on its own batch (weak scaling, no data-path collective) and rank 0 reports the
+aggregate; timing is CUDA events, max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+sys.path.insert(0, os.path.join(ROOT, "tests"))
+
+import numpy as np
+import torch
+
+import ubt_synth as synth
+
+NOMINAL_HBM_GBS = 8000.0          # the north-star's "~8 TB/s"
+FALLBACK_HBM_GBS = 6650.0         # earlier measurement on this machine, used only without MEASURED_PEAKS.json
+
+
+def algorithmic_bytes_per_tree(cfg: synth.Config) -> dict:
+    """Bytes the method must move per tree: every logit once, the selector scores, every output."""
+    e = 2 if cfg.dtype == "bf16" else 4
+    mw = (cfg.N + 31) // 32
+    draft = cfg.L * cfg.V * e
+    target = cfg.N * cfg.V * e
+    small = (max(cfg.L - 1, 0) * cfg.k * cfg.k * 4            # bigram scores
+             + cfg.L * cfg.k * 8                               # candidates out
+             + cfg.N * (6 * 4 + mw * 4) + 4                    # tree arrays + mask + n_nodes
+             + (2 * (cfg.L + 1) + 2) * 4)                      # verify outputs
+    return {"draft_logits": draft, "target_logits": target, "other": small, "total": draft + target + small}
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def recorded_traffic(kernel: str, workload: str):
+    """DRAM bytes per launch of `kernel` from the committed ncu summary, if one exists (else None)."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        with open(path) as f:
+            return json.load(f).get(kernel, {}).get(workload)
+    except Exception:
+        return None
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        rows = [r for t, r in self.rows if t0 - 0.05 <= t <= t1 + 0.15 and len(r) >= 9] or [r for _, r in self.rows if len(r) >= 9]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        num = lambda s: float(s) if s.replace(".", "", 1).isdigit() else None
+        sm = [num(r[1]) for r in rows if num(r[1]) is not None]
+        reasons = set()
+        for r in rows:
+            for name, col in (("hw_slowdown", 5), ("hw_thermal_slowdown", 6), ("sw_thermal_slowdown", 7),
+                              ("sw_power_cap", 8)):
+                if r[col].lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": num(rows[0][2]),
+                "power_w_max": max((num(r[3]) or 0.0) for r in rows), "samples": len(rows),
+                "reasons": sorted(reasons)}
+
+
+def dist_setup(n_gpus: int):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl" if torch.cuda.is_available() else "gloo")
+    return world, rank, local
+
+
+def max_over_ranks(value: float, world: int, device) -> float:
+    if world == 1:
+        return value
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def barrier(world: int):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def oracle_pass(cfg, uh, bh, zh, seed):
+    """One oracle draft+verify pass on host arrays; returns (tree, verdict, seconds)."""
+    import oracle
+    t0 = time.perf_counter()
+    tr = oracle.draft_tree(uh, bh, cfg.k, cfg.N)
+    v = oracle.verify(tr.token_ids, tr.parents, tr.n_nodes, cfg.L, zh, cfg.mode, seed=seed)
+    return tr, v, time.perf_counter() - t0
+
+
+def run_reference(args, cfg, world, rank):
+    """The reference arm: the CPU oracle as it stands, on the host cores, on a bounded sample per step."""
+    if rank != 0:
+        return
+    import oracle
+    sample = max(1, min(cfg.B, args.ref_trees))
+    sub = cfg.replace(B=sample)
+    di = synth.draft_inputs(sub, 0)
+    z = synth.target_logits(sub, 0)
+    for _ in range(args.warmup):
+        oracle_pass(sub, di.unigram_logits, di.bigram_scores, z, 0)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_pass(sub, di.unigram_logits, di.bigram_scores, z, 0)
+    dt = time.perf_counter() - t0
+    value = sample * args.steps / dt
+    line = {"impl": "reference", "metric": "draft+verify trees/sec", "value": value, "unit": "trees/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "B": cfg.B, "L": cfg.L, "V": cfg.V, "k": cfg.k, "node_budget": cfg.N,
+                       "verify": cfg.mode, "logits": cfg.dtype},
+            "cpu_baseline": {"value": value, "unit": "trees/s", "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": f"{sample} of {cfg.B} sequences per step"},
+            "e2e": {"value": value, "unit": "trees/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c3", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--ref-trees", type=int, default=4, help="sequences per step of the reference arm")
+    ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time budget of the oracle baseline")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    cfg = synth.CONFIGS[args.workload]
+    world, rank, local = dist_setup(args.gpus)
+
+    if args.impl == "reference":
+        run_reference(args, cfg, world, rank)
+        return
+
+    import paper_2609_39972_b200 as ubt          # fails loudly if libubt.so is missing: no CPU fallback
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    ubt.load()
+
+    # ---- inputs: enough distinct batches that one rotation exceeds twice the 126 MB L2
+    bpt = algorithmic_bytes_per_tree(cfg)
+    batch_bytes = bpt["total"] * cfg.B
+    n_sets = max(2, min(16, -(-4 * 126_000_000 // max(batch_bytes, 1))))
+    sets = []
+    for s in range(n_sets):
+        ud, bd, zd = synth.device_inputs(cfg, 1000 * rank + s, dev)
+        sets.append((ud, bd, zd))
+    tree = ubt.Tree.empty(cfg.B, cfg.N, cfg.L, cfg.k, dev)
+    res = ubt.VerifyResult.empty(cfg.B, cfg.L, dev)
+    ws_d = ubt.workspace(ubt.ubt_draft_workspace_bytes(cfg.B, cfg.L, cfg.V, cfg.k, cfg.N), dev)
+    ws_v = ubt.workspace(ubt.ubt_verify_workspace_bytes(cfg.B, cfg.N, cfg.V, cfg.mode), dev)
+    stream = torch.cuda.current_stream()
+
+    ev_pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                for _ in range(args.steps)]
+    for a, b in ev_pairs:           # create the underlying cudaEvent_t handles
+        a.record(stream); b.record(stream)
+
+    def step(i, events=None):
+        ud, bd, zd = sets[i % n_sets]
+        ubt.ubt_draft_tree(ud, bd, cfg.k, cfg.N, tree=tree, ws=ws_d, stream=stream)
+        ubt.ubt_verify_tree(tree, zd, cfg.mode, seed=i, temperature=1.0, result=res, ws=ws_v, stream=stream,
+                            event_before=events[0] if events else None, event_after=events[1] if events else None)
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    barrier(world)
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)
+    t_wall0 = time.time()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        step(args.warmup + i, ev_pairs[i])
+    e1.record(stream)
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    barrier(world)
+    clocks = sampler.stop(t_wall0, t_wall1)
+    elapsed_ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
+    kern_ms = statistics.mean(a.elapsed_time(b) for a, b in ev_pairs)
+    trees_per_s = cfg.B * args.steps * world / (elapsed_ms * 1e-3)
+
+    # ---- draft / verify split (separate untimed pass, for the record)
+    ea, eb, ec = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+    td, tv = [], []
+    for i in range(min(args.steps, 20)):
+        ud, bd, zd = sets[i % n_sets]
+        ea.record(stream)
+        ubt.ubt_draft_tree(ud, bd, cfg.k, cfg.N, tree=tree, ws=ws_d, stream=stream)
+        eb.record(stream)
+        ubt.ubt_verify_tree(tree, zd, cfg.mode, seed=i, result=res, ws=ws_v, stream=stream)
+        ec.record(stream)
+        torch.cuda.synchronize()
+        td.append(ea.elapsed_time(eb)); tv.append(eb.elapsed_time(ec))
+
+    peak, peak_kind = measured_peak()
+    e = 2 if cfg.dtype == "bf16" else 4
+    kern_name = "k_row_argmax" if cfg.mode == "greedy" else "k_row_sample"
+    kern_bytes = cfg.B * cfg.N * cfg.V * e
+    achieved = kern_bytes / (kern_ms * 1e-3) / 1e9
+    step_gbs = batch_bytes * args.steps / (elapsed_ms * 1e-3) / 1e9 if world == 1 else \
+        batch_bytes * args.steps * world / (elapsed_ms * 1e-3) / 1e9
+
+    line = {
+        "metric": "draft+verify trees/sec", "value": trees_per_s, "unit": "trees/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": cfg.name, "B": cfg.B, "L": cfg.L, "V": cfg.V, "k": cfg.k, "node_budget": cfg.N,
+                   "verify": cfg.mode, "logits": cfg.dtype, "input_sets": n_sets,
+                   "l2": "inputs larger than L2 (rotation of %d MB)" % (batch_bytes * n_sets // 1_000_000)},
+        "hbm": {"bytes_per_tree": bpt["total"], "step_gbs_per_gpu": step_gbs / world,
+                "frac_of_%s_peak" % peak_kind: step_gbs / world / peak,
+                "frac_of_nominal_8tbs": step_gbs / world / NOMINAL_HBM_GBS,
+                "draft_ms": statistics.median(td), "verify_ms": statistics.median(tv)},
+        "roofline": {"bound": "hbm", "kernel": kern_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_source": f"of {peak_kind}",
+                     "traffic": recorded_traffic(kern_name, cfg.name), "bytes_per_launch": kern_bytes,
+                     "avg_launch_ms": kern_ms},
+        "clocks": clocks,
+        "gpu_launches": 5 * args.steps,
+    }
+
+    # ---- end to end through the host-buffer entry points (pinned host inputs, results read back)
+    if not args.no_e2e:
+        ud, bd, zd = sets[0]
+        uh, bh, zh = ud.cpu().pin_memory(), bd.cpu().pin_memory(), zd.cpu().pin_memory()
+        tree_h = ubt.Tree.empty(cfg.B, cfg.N, cfg.L, cfg.k, dev, pin=True)
+        res_h = ubt.VerifyResult.empty(cfg.B, cfg.L, dev, pin=True)
+        code = 1 if cfg.dtype == "bf16" else 0
+        dbuf = ubt.workspace(ubt.ubt_draft_host_buffer_bytes(cfg.B, cfg.L, cfg.V, cfg.k, cfg.N, code), dev)
+        vbuf = ubt.workspace(ubt.ubt_verify_host_buffer_bytes(cfg.B, cfg.L, cfg.N, cfg.V, code, cfg.mode), dev)
+
+        def e2e_step(i):
+            ubt.ubt_draft_tree_host(uh, bh, cfg.k, cfg.N, tree_h, dbuf, stream=stream)
+            ubt.ubt_verify_tree_host(tree_h, zh, res_h, vbuf, cfg.mode, seed=i, stream=stream)
+
+        k_e2e = max(3, min(args.steps, 10))
+        for i in range(3):
+            e2e_step(i)
+        torch.cuda.synchronize(); barrier(world)
+        t0 = time.perf_counter()
+        for i in range(k_e2e):
+            e2e_step(i)
+        torch.cuda.synchronize()
+        dt = max_over_ranks(time.perf_counter() - t0, world, dev)
+        mw = (cfg.N + 31) // 32
+        h2d = uh.numel() * uh.element_size() + bh.numel() * 4 + zh.numel() * zh.element_size() + cfg.B * (2 * cfg.N + 1) * 4
+        d2h = cfg.B * (cfg.N * (6 + mw) * 4 + 4 + cfg.L * cfg.k * 8) + cfg.B * (2 * (cfg.L + 1) + 2) * 4
+        line["e2e"] = {"value": cfg.B * k_e2e * world / dt, "unit": "trees/s", "h2d_bytes_per_step": h2d,
+                       "d2h_bytes_per_step": d2h, "steps": k_e2e, "gpu_launches": 5 * k_e2e}
+        line["gpu_launches"] += 5 * k_e2e
+        del uh, bh, zh
+
+    # ---- CPU baseline: the oracle as it stands on the host cores, on a bounded sample; doubles as a parity check
+    if rank == 0 and not args.no_cpu_baseline:
+        import oracle
+        from parity import compare_draft, compare_verify, tree_to_numpy
+        ud, bd, zd = sets[0]
+        sample = max(1, min(cfg.B, 8))
+        uh, bh, zh = (synth.to_host_bits(t[:sample]) for t in (ud, bd, zd))
+        done, spent, tr = 0, 0.0, None
+        while spent < args.cpu_seconds:
+            tr, ov, dt = oracle_pass(cfg, uh, bh, zh, 0)
+            done += sample; spent += dt
+        line["cpu_baseline"] = {"value": done / spent, "unit": "trees/s", "cores": oracle.num_threads(),
+                                "kind": "oracle", "sample": f"first {sample} of {cfg.B} sequences, repeated for "
+                                                            f"{spent:.1f} s ({done} trees)"}
+        # live parity of the bench configuration on that sample
+        ubt.ubt_draft_tree(ud, bd, cfg.k, cfg.N, tree=tree, ws=ws_d, stream=stream)
+        pick = torch.empty((cfg.B, cfg.N), dtype=torch.int32, device=dev)
+        ubt.ubt_verify_tree(tree, zd, cfg.mode, seed=0, result=res, ws=ws_v, stream=stream, node_pick=pick)
+        torch.cuda.synchronize()
+        try:
+            g = tree_to_numpy(tree)
+            swaps = compare_draft(g, tr, cfg.L, cfg.k, cfg.N, rows=list(range(sample)))
+            if not swaps:
+                compare_verify(res, ov, pick, rows=slice(0, sample))
+            line["parity"] = {"checked_trees": sample, "near_tie_swaps": len(swaps), "ok": True}
+        except AssertionError as ex:
+            line["parity"] = {"checked_trees": sample, "ok": False, "error": str(ex)[:200]}
+
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,174 @@
+/*
+ * ubt.h -- C ABI of the UBTree draft-tree + verification hot path on NVIDIA B200 (sm_100a).
+ *
+ * The library computes, for a batch of B independent sequences:
+ *   a1  per-position vocabulary log-softmax and top-k candidates          (paper eq. 3, "Candidate Sets")
+ *   a2  combine with bigram transition scores, normalise over candidates  (eq. 5, eq. 9)
+ *   a3  best-path expansion into a node-budgeted draft tree               (eq. 10-12, Algorithm 1)
+ *   a3b tree-attention inputs: position ids and packed ancestor bitmask   (Section 3.1.3, Appendix A)
+ *   a4  acceptance walk against target logits, plus the bonus token       (Appendix A, verification)
+ *
+ * Conventions that hold for every entry point unless it says otherwise
+ *   - Pointers named in a struct or argument list are DEVICE pointers owned by the caller; the
+ *     library never allocates, frees or synchronises.  All work is enqueued on `cuda_stream`
+ *     (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *   - Tensors are dense, row-major, in the shapes given; base pointers must be 16-byte aligned.
+ *   - Inputs are read-only.  Outputs and the workspace are overwritten; workspace content on entry
+ *     is irrelevant.
+ *   - Argument errors are detected on the host and returned before anything is launched.
+ *     A failed launch returns UBT_ERR_CUDA.  Nothing in the library traps or spins on the device.
+ *   - Logits must be free of NaN; each row must hold at least k entries greater than -inf.
+ *
+ * Sizes: B sequences, L draft positions (the paper's gamma), V vocabulary, k candidates per position
+ * (the paper's K), N = node budget = tree slots INCLUDING the root (the paper's budget B counts
+ * non-root nodes only, so its B equals N - 1).
+ * Limits (else UBT_ERR_UNSUPPORTED): 1 <= k <= 64, k <= V < 2^31, 1 <= N <= 256, 1 <= L <= 64,
+ * and the per-sequence pair table L*k*k*5 bytes must fit in 160 KiB of shared memory.
+ */
+#ifndef UBT_H_
+#define UBT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  UBT_OK = 0,
+  UBT_ERR_INVALID_ARG = 1, /* NULL / misaligned pointer, size out of range, k > V, zeta > 0 ... */
+  UBT_ERR_UNSUPPORTED = 2, /* valid request beyond the compiled limits above */
+  UBT_ERR_WORKSPACE = 3,   /* workspace NULL or smaller than ubt_*_workspace_bytes() */
+  UBT_ERR_CUDA = 4         /* a CUDA call or kernel launch failed */
+} ubt_status;
+
+typedef enum { UBT_F32 = 0, UBT_BF16 = 1 } ubt_dtype;
+typedef enum { UBT_VERIFY_GREEDY = 0, UBT_VERIFY_SAMPLE = 1 } ubt_verify_mode;
+
+/*
+ * A batch of draft trees.  Slot 0 of every sequence is the root (the empty draft prefix; Appendix A,
+ * "Path Scores").  Slots 1..n_nodes-1 hold the selected nodes ordered by (depth, parent slot,
+ * candidate rank), so parents[i] < i and the children of one parent are contiguous.  Unused slots
+ * n_nodes..N-1 hold -1 (scores: -inf; mask rows: zero).
+ */
+typedef struct ubt_tree {
+  int32_t B, N, L, k, mask_words; /* mask_words = ceil(N / 32) */
+  int32_t *token_ids;             /* [B,N]  token of the node; root: anchor token or -1 */
+  int32_t *parents;               /* [B,N]  slot of the parent; root: -1 */
+  int32_t *depths;                /* [B,N]  root: 0 */
+  int32_t *position_ids;          /* [B,N]  pos_offset[b] + depth */
+  int32_t *cand_rank;             /* [B,N]  rank of the node's token inside its position's candidates */
+  float *scores;                  /* [B,N]  cumulative log-probability ell_zeta (eq. 9-10); root: 0 */
+  uint32_t *mask;                 /* [B,N,mask_words]  bit j of row i (word j>>5, bit j&31) set iff
+                                     slot j is slot i or an ancestor of it */
+  int32_t *n_nodes;               /* [B]    used slots, root included */
+  int32_t *cand_ids;              /* [B,L,k] candidate token ids, best first (logit desc, id asc) */
+  float *cand_logprob;            /* [B,L,k] their vocabulary log-softmax values */
+} ubt_tree;
+
+/* Options of the tree construction; pass NULL for the defaults written beside each field. */
+typedef struct ubt_draft_opts {
+  int32_t search_width;         /* W of eq. 11; 0 = unbounded (default).  The paper runs W = 12. */
+  float depth_bonus;            /* zeta of eq. 10, must be <= 0; default 0 */
+  const float *alpha;           /* [L] depth calibration of eq. 5; NULL = 1 */
+  const float *lambda;          /* [L] depth calibration of eq. 5; NULL = 1 */
+  const float *anchor_bigram;   /* [B,k] selector score of the anchor -> depth-1 transition; NULL = 0 */
+  const int32_t *anchor_tokens; /* [B] token stored in the root slot; NULL = -1 */
+  const int32_t *pos_offset;    /* [B] position id of the root; NULL = 0 */
+} ubt_draft_opts;
+
+typedef struct ubt_verify_opts {
+  uint64_t seed;       /* Philox4x32-10 key (low word, high word); sampling mode only */
+  float temperature;   /* > 0; sampling mode only; default 1 */
+  int32_t *node_pick;  /* optional [B,N]: the target's pick at EVERY row, visited or not */
+  void *event_before;  /* optional cudaEvent_t recorded on the stream just before the V-wide */
+  void *event_after;   /* per-node kernel and just after it (for timing that kernel alone)    */
+} ubt_verify_opts;
+
+typedef struct ubt_verify_result {
+  int32_t *accepted_len;   /* [B]     accepted draft tokens; the paper's tau = accepted_len + 1 */
+  int32_t *bonus_token;    /* [B]     first unmatched target pick */
+  int32_t *accepted_nodes; /* [B,L+1] slots on the accepted path, root first; padded with -1 */
+  int32_t *out_tokens;     /* [B,L+1] accepted tokens followed by the bonus token; padded with -1 */
+} ubt_verify_result;
+
+int ubt_version(void);
+const char *ubt_status_string(int status);
+
+/* Bytes of device workspace the calls below need for the given shape (0 on invalid shapes). */
+size_t ubt_draft_workspace_bytes(int B, int L, int V, int k, int node_budget);
+size_t ubt_verify_workspace_bytes(int B, int node_budget, int V, int mode);
+
+/*
+ * Step a1 alone (eq. 3 and "Candidate Sets", Section 3.1.1).  For each of `rows` logit rows of
+ * length V: the k largest logits ordered (value descending, token id ascending; -0 equals +0),
+ * and cand_logprob[r] = logit[cand_ids[r]] - log(sum_v exp logit[v]) in fp32.
+ * Workspace: ubt_draft_workspace_bytes(rows, 1, V, k, 1).
+ */
+int ubt_topk_logprob(const void *logits, int dtype, int64_t rows, int V, int k, int32_t *cand_ids,
+                     float *cand_logprob, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Steps a2, a3, a3b from candidates that are already in out->cand_ids / out->cand_logprob
+ * (eq. 5, eq. 9-12, Algorithm 1).  bigram_scores[b,j,ra,rb] is the selector score delta of the
+ * transition from the rank-ra candidate of position j to the rank-rb candidate of position j+1.
+ * s = alpha*logprob + lambda*delta is normalised over the k successor candidates of each
+ * predecessor; a node's score is the sum of those log-probabilities along its prefix plus
+ * zeta*depth.  The search keeps, per depth, the W best extensions of the retained nodes and
+ * finally the N-1 best retained nodes overall; ties prefer the shallower node, then the lower
+ * token id, then the lower candidate rank, then the lexicographically smaller rank path.
+ * Scores are computed in fp32.
+ */
+int ubt_build_tree(const float *bigram_scores, int B, int L, int k, int node_budget,
+                   const ubt_draft_opts *opts, ubt_tree *out, void *cuda_stream);
+
+/*
+ * Step a3b alone: position ids and the ancestor bitmask from parents / depths / n_nodes of `tree`
+ * (for callers that edit a tree).  Overwrites tree->position_ids and tree->mask.
+ */
+int ubt_build_mask(ubt_tree *tree, const int32_t *pos_offset /* [B] or NULL */, void *cuda_stream);
+
+/*
+ * Steps a1 -> a3b in one call: unigram_logits[B,L,V] (fp32 or bf16) and bigram_scores[B,L-1,k,k]
+ * (fp32) -> *out.  Equivalent to ubt_topk_logprob followed by ubt_build_tree.
+ */
+int ubt_draft_tree(const void *unigram_logits, int dtype, const float *bigram_scores, int B, int L,
+                   int V, int k, int node_budget, const ubt_draft_opts *opts, ubt_tree *out,
+                   void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Step a4 (Appendix A, "Verification via Tree-attention").  target_logits[B,N,V] holds one row per
+ * tree slot.  The target's pick at a row is, in greedy mode, the smallest token id attaining the
+ * row maximum; in sampling mode, a draw from softmax(row / temperature) defined by integer
+ * weights w_v = trunc(2^(40 + fma(z_v, a, c))) (a = log2(e)/T, c = -max*a, a fixed fp32 degree-5
+ * routine for 2^x), theta = floor(R * sum(w) / 2^64) with R the first two words of
+ * Philox4x32-10(counter = (slot, b, 0, 0), key = seed), pick = first token whose inclusive prefix
+ * sum exceeds theta.  The walk starts at the root and follows the child whose token equals the pick
+ * of the current slot until none matches; that pick is the bonus token.
+ */
+int ubt_verify_tree(const ubt_tree *tree, const void *target_logits, int dtype, int V, int mode,
+                    const ubt_verify_opts *opts, ubt_verify_result *out, void *workspace,
+                    size_t workspace_bytes, void *cuda_stream);
+
+/*
+ * Host-buffer forms.  Every pointer inside `tree`, `opts` (alpha ... pos_offset, node_pick) and
+ * `out`, and the logits / bigram arguments, are HOST pointers (pinned memory makes the copies
+ * asynchronous).  `device_buffer` is caller-owned DEVICE memory of at least
+ * ubt_*_host_buffer_bytes(); the call copies inputs into it, runs the device path on
+ * `cuda_stream`, copies the results back and waits for the stream before returning.
+ */
+size_t ubt_draft_host_buffer_bytes(int B, int L, int V, int k, int node_budget, int dtype);
+size_t ubt_verify_host_buffer_bytes(int B, int L, int node_budget, int V, int dtype, int mode);
+int ubt_draft_tree_host(const void *unigram_logits, int dtype, const float *bigram_scores, int B,
+                        int L, int V, int k, int node_budget, const ubt_draft_opts *opts,
+                        ubt_tree *out, void *device_buffer, size_t device_buffer_bytes,
+                        void *cuda_stream);
+int ubt_verify_tree_host(const ubt_tree *tree, const void *target_logits, int dtype, int V, int mode,
+                         const ubt_verify_opts *opts, ubt_verify_result *out, void *device_buffer,
+                         size_t device_buffer_bytes, void *cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* UBT_H_ */

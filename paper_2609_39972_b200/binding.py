@@ -1,0 +1,308 @@
+"""ctypes binding of ``libubt.so``: argument marshalling only, every step runs in the CUDA kernels.
+
+The functions carry the names of the C ABI (``include/ubt.h``).  Tensors are ``torch`` CUDA tensors
+(device memory and streams are all PyTorch is used for); the host-buffer forms take pinned CPU
+tensors.  There is no CPU fallback: a missing library or a non-CUDA tensor raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+from . import _build
+
+UBT_OK = 0
+UBT_F32, UBT_BF16 = 0, 1
+UBT_VERIFY_GREEDY, UBT_VERIFY_SAMPLE = 0, 1
+_MODES = {"greedy": UBT_VERIFY_GREEDY, "sample": UBT_VERIFY_SAMPLE}
+
+
+class UbtError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+class _Tree(C.Structure):
+    _fields_ = [("B", C.c_int32), ("N", C.c_int32), ("L", C.c_int32), ("k", C.c_int32), ("mask_words", C.c_int32),
+                ("token_ids", C.c_void_p), ("parents", C.c_void_p), ("depths", C.c_void_p),
+                ("position_ids", C.c_void_p), ("cand_rank", C.c_void_p), ("scores", C.c_void_p),
+                ("mask", C.c_void_p), ("n_nodes", C.c_void_p), ("cand_ids", C.c_void_p),
+                ("cand_logprob", C.c_void_p)]
+
+
+class _DraftOpts(C.Structure):
+    _fields_ = [("search_width", C.c_int32), ("depth_bonus", C.c_float), ("alpha", C.c_void_p),
+                ("lambda_", C.c_void_p), ("anchor_bigram", C.c_void_p), ("anchor_tokens", C.c_void_p),
+                ("pos_offset", C.c_void_p)]
+
+
+class _VerifyOpts(C.Structure):
+    _fields_ = [("seed", C.c_uint64), ("temperature", C.c_float), ("node_pick", C.c_void_p),
+                ("event_before", C.c_void_p), ("event_after", C.c_void_p)]
+
+
+class _VerifyResult(C.Structure):
+    _fields_ = [("accepted_len", C.c_void_p), ("bonus_token", C.c_void_p), ("accepted_nodes", C.c_void_p),
+                ("out_tokens", C.c_void_p)]
+
+
+EXPORTS = ["ubt_version", "ubt_status_string", "ubt_draft_workspace_bytes", "ubt_verify_workspace_bytes",
+           "ubt_topk_logprob", "ubt_build_tree", "ubt_build_mask", "ubt_draft_tree", "ubt_verify_tree",
+           "ubt_draft_host_buffer_bytes", "ubt_verify_host_buffer_bytes", "ubt_draft_tree_host",
+           "ubt_verify_tree_host"]
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def load() -> C.CDLL:
+    """Load ``libubt.so`` (built in-tree by ``_build.build``); raises if it is missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = lib_path()
+    if not os.path.exists(path):
+        raise ImportError(f"{path} is missing: build it with paper_2609_39972_b200._build.build() "
+                          "(needs nvcc); there is no CPU fallback")
+    L = C.CDLL(path)
+    L.ubt_version.restype = C.c_int
+    L.ubt_status_string.restype = C.c_char_p
+    L.ubt_status_string.argtypes = [C.c_int]
+    for name in ("ubt_draft_workspace_bytes", "ubt_verify_workspace_bytes", "ubt_draft_host_buffer_bytes",
+                 "ubt_verify_host_buffer_bytes"):
+        getattr(L, name).restype = C.c_size_t
+    L.ubt_draft_workspace_bytes.argtypes = [C.c_int] * 5
+    L.ubt_verify_workspace_bytes.argtypes = [C.c_int] * 4
+    L.ubt_draft_host_buffer_bytes.argtypes = [C.c_int] * 6
+    L.ubt_verify_host_buffer_bytes.argtypes = [C.c_int] * 6
+    L.ubt_topk_logprob.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
+                                   C.c_void_p, C.c_size_t, C.c_void_p]
+    L.ubt_build_tree.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.ubt_build_mask.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+    L.ubt_draft_tree.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    L.ubt_verify_tree.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
+                                  C.c_void_p, C.c_size_t, C.c_void_p]
+    L.ubt_draft_tree_host.argtypes = L.ubt_draft_tree.argtypes
+    L.ubt_verify_tree_host.argtypes = L.ubt_verify_tree.argtypes
+    _lib = L
+    return L
+
+
+def ubt_version() -> int:
+    return int(load().ubt_version())
+
+
+def status_string(status: int) -> str:
+    return load().ubt_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != UBT_OK:
+        raise UbtError(status, where)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return UBT_BF16
+    if t.dtype == torch.float32:
+        return UBT_F32
+    raise TypeError("logits must be torch.float32 or torch.bfloat16")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _need(t: torch.Tensor, name: str, cuda: bool = True) -> torch.Tensor:
+    if cuda and not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor (no CPU fallback)")
+    if not cuda and t.is_cuda:
+        raise ValueError(f"{name} must be a host tensor")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    return t
+
+
+def _stream(stream) -> C.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+@dataclass
+class Tree:
+    """Storage of a batch of draft trees (see ``ubt_tree`` in include/ubt.h)."""
+    B: int
+    N: int
+    L: int
+    k: int
+    token_ids: torch.Tensor
+    parents: torch.Tensor
+    depths: torch.Tensor
+    position_ids: torch.Tensor
+    cand_rank: torch.Tensor
+    scores: torch.Tensor
+    mask: torch.Tensor
+    n_nodes: torch.Tensor
+    cand_ids: torch.Tensor
+    cand_logprob: torch.Tensor
+
+    @staticmethod
+    def empty(B: int, N: int, L: int, k: int, device, pin: bool = False) -> "Tree":
+        kw = dict(device=device)
+        if pin:
+            kw = dict(device="cpu", pin_memory=True)
+        i32 = lambda *s: torch.empty(s, dtype=torch.int32, **kw)
+        return Tree(B, N, L, k, i32(B, N), i32(B, N), i32(B, N), i32(B, N), i32(B, N),
+                    torch.empty((B, N), dtype=torch.float32, **kw), i32(B, N, (N + 31) // 32), i32(B),
+                    i32(B, L, k), torch.empty((B, L, k), dtype=torch.float32, **kw))
+
+    def c_struct(self) -> _Tree:
+        return _Tree(self.B, self.N, self.L, self.k, (self.N + 31) // 32, self.token_ids.data_ptr(),
+                     self.parents.data_ptr(), self.depths.data_ptr(), self.position_ids.data_ptr(),
+                     self.cand_rank.data_ptr(), self.scores.data_ptr(), self.mask.data_ptr(),
+                     self.n_nodes.data_ptr(), self.cand_ids.data_ptr(), self.cand_logprob.data_ptr())
+
+
+@dataclass
+class VerifyResult:
+    accepted_len: torch.Tensor
+    bonus_token: torch.Tensor
+    accepted_nodes: torch.Tensor
+    out_tokens: torch.Tensor
+    node_pick: Optional[torch.Tensor] = None
+
+    @staticmethod
+    def empty(B: int, L: int, device, pin: bool = False) -> "VerifyResult":
+        kw = dict(device="cpu", pin_memory=True) if pin else dict(device=device)
+        i32 = lambda *s: torch.empty(s, dtype=torch.int32, **kw)
+        return VerifyResult(i32(B), i32(B), i32(B, L + 1), i32(B, L + 1))
+
+    def c_struct(self) -> _VerifyResult:
+        return _VerifyResult(self.accepted_len.data_ptr(), self.bonus_token.data_ptr(),
+                             self.accepted_nodes.data_ptr(), self.out_tokens.data_ptr())
+
+
+def _draft_opts(search_width=0, depth_bonus=0.0, alpha=None, lam=None, anchor_bigram=None, anchor_tokens=None,
+                pos_offset=None) -> _DraftOpts:
+    p = lambda t: None if t is None else t.data_ptr()
+    return _DraftOpts(int(search_width), float(depth_bonus), p(alpha), p(lam), p(anchor_bigram), p(anchor_tokens),
+                      p(pos_offset))
+
+
+def ubt_draft_workspace_bytes(B: int, L: int, V: int, k: int, node_budget: int) -> int:
+    return int(load().ubt_draft_workspace_bytes(B, L, V, k, node_budget))
+
+
+def ubt_verify_workspace_bytes(B: int, node_budget: int, V: int, mode="greedy") -> int:
+    return int(load().ubt_verify_workspace_bytes(B, node_budget, V, _MODES.get(mode, mode)))
+
+
+def workspace(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def ubt_topk_logprob(logits: torch.Tensor, k: int, cand_ids: torch.Tensor, cand_logprob: torch.Tensor,
+                     ws: torch.Tensor, stream=None) -> None:
+    _need(logits, "logits")
+    V = logits.shape[-1]
+    rows = logits.numel() // V
+    _check(load().ubt_topk_logprob(_ptr(logits), _dtype_code(logits), rows, V, k, _ptr(_need(cand_ids, "cand_ids")),
+                                   _ptr(_need(cand_logprob, "cand_logprob")), _ptr(ws), ws.numel(), _stream(stream)),
+           "ubt_topk_logprob")
+
+
+def ubt_build_tree(bigram_scores: Optional[torch.Tensor], tree: Tree, stream=None, **opts) -> None:
+    o = _draft_opts(**opts)
+    t = tree.c_struct()
+    _check(load().ubt_build_tree(_ptr(bigram_scores), tree.B, tree.L, tree.k, tree.N, C.byref(o), C.byref(t),
+                                 _stream(stream)), "ubt_build_tree")
+
+
+def ubt_build_mask(tree: Tree, pos_offset: Optional[torch.Tensor] = None, stream=None) -> None:
+    t = tree.c_struct()
+    _check(load().ubt_build_mask(C.byref(t), _ptr(pos_offset), _stream(stream)), "ubt_build_mask")
+
+
+def ubt_draft_tree(unigram_logits: torch.Tensor, bigram_scores: Optional[torch.Tensor], k: int, node_budget: int,
+                   tree: Optional[Tree] = None, ws: Optional[torch.Tensor] = None, stream=None, **opts) -> Tree:
+    """``unigram_logits[B,L,V]``, ``bigram_scores[B,L-1,k,k]`` -> draft trees (steps a1-a3b)."""
+    _need(unigram_logits, "unigram_logits")
+    B, L, V = unigram_logits.shape
+    if tree is None:
+        tree = Tree.empty(B, node_budget, L, k, unigram_logits.device)
+    if ws is None:
+        ws = workspace(ubt_draft_workspace_bytes(B, L, V, k, node_budget), unigram_logits.device)
+    o = _draft_opts(**opts)
+    t = tree.c_struct()
+    _check(load().ubt_draft_tree(_ptr(unigram_logits), _dtype_code(unigram_logits), _ptr(bigram_scores), B, L, V, k,
+                                 node_budget, C.byref(o), C.byref(t), _ptr(ws), ws.numel(), _stream(stream)),
+           "ubt_draft_tree")
+    return tree
+
+
+def ubt_verify_tree(tree: Tree, target_logits: torch.Tensor, mode="greedy", seed: int = 0, temperature: float = 1.0,
+                    node_pick: Optional[torch.Tensor] = None, result: Optional[VerifyResult] = None,
+                    ws: Optional[torch.Tensor] = None, stream=None, event_before=None,
+                    event_after=None) -> VerifyResult:
+    """Walk ``tree`` against ``target_logits[B,N,V]`` (step a4)."""
+    _need(target_logits, "target_logits")
+    B, N, V = target_logits.shape
+    m = _MODES.get(mode, mode)
+    if result is None:
+        result = VerifyResult.empty(B, tree.L, target_logits.device)
+    if ws is None:
+        ws = workspace(ubt_verify_workspace_bytes(B, N, V, m), target_logits.device)
+    ev = lambda e: None if e is None else C.c_void_p(e.cuda_event)
+    o = _VerifyOpts(int(seed), float(temperature), None if node_pick is None else node_pick.data_ptr(),
+                    ev(event_before), ev(event_after))
+    t = tree.c_struct()
+    r = result.c_struct()
+    _check(load().ubt_verify_tree(C.byref(t), _ptr(target_logits), _dtype_code(target_logits), V, m, C.byref(o),
+                                  C.byref(r), _ptr(ws), ws.numel(), _stream(stream)), "ubt_verify_tree")
+    result.node_pick = node_pick
+    return result
+
+
+def ubt_draft_host_buffer_bytes(B, L, V, k, node_budget, dtype) -> int:
+    return int(load().ubt_draft_host_buffer_bytes(B, L, V, k, node_budget, dtype))
+
+
+def ubt_verify_host_buffer_bytes(B, L, node_budget, V, dtype, mode="greedy") -> int:
+    return int(load().ubt_verify_host_buffer_bytes(B, L, node_budget, V, dtype, _MODES.get(mode, mode)))
+
+
+def ubt_draft_tree_host(unigram_logits: torch.Tensor, bigram_scores: Optional[torch.Tensor], k: int, node_budget: int,
+                        tree: Tree, device_buffer: torch.Tensor, stream=None, **opts) -> Tree:
+    """Host-buffer form: inputs and ``tree`` live in (pinned) host memory; returns after the stream is idle."""
+    _need(unigram_logits, "unigram_logits", cuda=False)
+    B, L, V = unigram_logits.shape
+    o = _draft_opts(**opts)
+    t = tree.c_struct()
+    _check(load().ubt_draft_tree_host(_ptr(unigram_logits), _dtype_code(unigram_logits), _ptr(bigram_scores), B, L, V,
+                                      k, node_budget, C.byref(o), C.byref(t), _ptr(device_buffer),
+                                      device_buffer.numel(), _stream(stream)), "ubt_draft_tree_host")
+    return tree
+
+
+def ubt_verify_tree_host(tree: Tree, target_logits: torch.Tensor, result: VerifyResult, device_buffer: torch.Tensor,
+                         mode="greedy", seed: int = 0, temperature: float = 1.0,
+                         node_pick: Optional[torch.Tensor] = None, stream=None) -> VerifyResult:
+    _need(target_logits, "target_logits", cuda=False)
+    B, N, V = target_logits.shape
+    o = _VerifyOpts(int(seed), float(temperature), None if node_pick is None else node_pick.data_ptr(), None, None)
+    t = tree.c_struct()
+    r = result.c_struct()
+    _check(load().ubt_verify_tree_host(C.byref(t), _ptr(target_logits), _dtype_code(target_logits), V,
+                                       _MODES.get(mode, mode), C.byref(o), C.byref(r), _ptr(device_buffer),
+                                       device_buffer.numel(), _stream(stream)), "ubt_verify_tree_host")
+    result.node_pick = node_pick
+    return result

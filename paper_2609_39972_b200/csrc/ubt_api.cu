@@ -1,0 +1,349 @@
+// C ABI of libubt: argument validation, workspace carving, launches.  See include/ubt.h.
+#include <cstring>
+#include <mutex>
+
+#include "ubt_internal.h"
+
+namespace ubt {
+
+const DeviceInfo& device_info() {
+  static DeviceInfo info[64];
+  static bool known[64];
+  static std::mutex mu;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev < 0 || dev >= 64) dev = 0;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!known[dev]) {
+    int sms = 0, smem = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+    if (cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess || smem <= 0)
+      smem = 227 * 1024;
+    cudaGetLastError();
+    info[dev].sm_count = sms;
+    info[dev].max_smem_optin = smem;
+    known[dev] = true;
+  }
+  return info[dev];
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static size_t esize(int dtype) { return dtype == UBT_BF16 ? 2 : 4; }
+
+static int check_shape(int B, int L, int V, int k, int N) {
+  if (B < 0 || L < 1 || V < 1 || k < 1 || N < 1 || k > V) return UBT_ERR_INVALID_ARG;
+  if (k > kMaxK || N > kMaxN || L > kMaxL) return UBT_ERR_UNSUPPORTED;
+  if ((size_t)L * k * k * 5 > kTreeTableBytes) return UBT_ERR_UNSUPPORTED;
+  return UBT_OK;
+}
+
+static int check_tree(const ubt_tree* t, bool need_cands) {
+  if (!t) return UBT_ERR_INVALID_ARG;
+  if (t->mask_words != (t->N + 31) / 32) return UBT_ERR_INVALID_ARG;
+  const void* ptrs[] = {t->token_ids, t->parents, t->depths, t->position_ids, t->cand_rank,
+                        t->scores,    t->mask,    t->n_nodes};
+  for (const void* p : ptrs)
+    if (!p || !aligned16(p)) return UBT_ERR_INVALID_ARG;
+  if (need_cands && (!t->cand_ids || !t->cand_logprob || !aligned16(t->cand_ids) || !aligned16(t->cand_logprob)))
+    return UBT_ERR_INVALID_ARG;
+  return UBT_OK;
+}
+
+}  // namespace ubt
+
+using namespace ubt;
+
+extern "C" {
+
+int ubt_version(void) { return 100; }
+
+const char* ubt_status_string(int status) {
+  switch (status) {
+    case UBT_OK: return "ok";
+    case UBT_ERR_INVALID_ARG: return "invalid argument";
+    case UBT_ERR_UNSUPPORTED: return "shape beyond the compiled limits";
+    case UBT_ERR_WORKSPACE: return "workspace missing or too small";
+    case UBT_ERR_CUDA: return "CUDA call or launch failed";
+    default: return "unknown status";
+  }
+}
+
+size_t ubt_draft_workspace_bytes(int B, int L, int V, int k, int N) {
+  if (B < 0 || L < 1 || V < 1 || k < 1 || N < 1 || k > V || k > kMaxK) return 0;
+  return topk_workspace_bytes((int64_t)B * L, V, k) + 256;
+}
+
+size_t ubt_verify_workspace_bytes(int B, int N, int V, int mode) {
+  if (B < 0 || N < 1 || V < 1 || (mode != UBT_VERIFY_GREEDY && mode != UBT_VERIFY_SAMPLE)) return 0;
+  return verify_workspace_bytes((int64_t)B * N, V, mode) + 256;
+}
+
+int ubt_topk_logprob(const void* logits, int dtype, int64_t rows, int V, int k, int32_t* cand_ids,
+                     float* cand_logprob, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!logits || !cand_ids || !cand_logprob || rows < 0 || V < 1 || k < 1 || k > V) return UBT_ERR_INVALID_ARG;
+  if (dtype != UBT_F32 && dtype != UBT_BF16) return UBT_ERR_INVALID_ARG;
+  if (!aligned16(logits) || !aligned16(cand_ids) || !aligned16(cand_logprob)) return UBT_ERR_INVALID_ARG;
+  if (k > kMaxK) return UBT_ERR_UNSUPPORTED;
+  if (rows == 0) return UBT_OK;
+  if (!workspace || !aligned16(workspace) || workspace_bytes < topk_workspace_bytes(rows, V, k))
+    return UBT_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  TopkWorkspace w = carve_topk_workspace(workspace, rows, V, k);
+  if (launch_lse_topk(logits, dtype, rows, V, k, w, st) != cudaSuccess) return UBT_ERR_CUDA;
+  if (launch_merge_topk(rows, V, k, w, cand_ids, cand_logprob, st) != cudaSuccess) return UBT_ERR_CUDA;
+  return UBT_OK;
+}
+
+static int check_draft_opts(const ubt_draft_opts* o) {
+  if (!o) return UBT_OK;
+  if (o->search_width < 0 || !(o->depth_bonus <= 0.0f)) return UBT_ERR_INVALID_ARG;
+  return UBT_OK;
+}
+
+int ubt_build_tree(const float* bigram_scores, int B, int L, int k, int N, const ubt_draft_opts* opts,
+                   ubt_tree* out, void* cuda_stream) {
+  int rc = check_shape(B, L, k, k, N);  // V is not an input here; k stands in for the k <= V check
+  if (rc) return rc;
+  if ((rc = check_tree(out, true))) return rc;
+  if ((rc = check_draft_opts(opts))) return rc;
+  if (L > 1 && (!bigram_scores || !aligned16(bigram_scores))) return UBT_ERR_INVALID_ARG;
+  if (out->B != B || out->N != N || out->L != L || out->k != k) return UBT_ERR_INVALID_ARG;
+  if (tree_smem_bytes(L, k, N) > (size_t)device_info().max_smem_optin) return UBT_ERR_UNSUPPORTED;
+  const ubt_draft_opts d{};
+  const ubt_draft_opts* o = opts ? opts : &d;
+  cudaError_t e = launch_build_tree(bigram_scores, B, L, k, N, o->search_width, o->depth_bonus, o->alpha, o->lambda,
+                                    o->anchor_bigram, o->anchor_tokens, o->pos_offset, *out,
+                                    static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? UBT_OK : UBT_ERR_CUDA;
+}
+
+int ubt_build_mask(ubt_tree* tree, const int32_t* pos_offset, void* cuda_stream) {
+  int rc = check_tree(tree, false);
+  if (rc) return rc;
+  if (tree->B < 0 || tree->N < 1) return UBT_ERR_INVALID_ARG;
+  if (tree->N > kMaxN) return UBT_ERR_UNSUPPORTED;
+  cudaError_t e = launch_build_mask(*tree, pos_offset, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? UBT_OK : UBT_ERR_CUDA;
+}
+
+int ubt_draft_tree(const void* unigram_logits, int dtype, const float* bigram_scores, int B, int L, int V, int k,
+                   int N, const ubt_draft_opts* opts, ubt_tree* out, void* workspace, size_t workspace_bytes,
+                   void* cuda_stream) {
+  int rc = check_shape(B, L, V, k, N);
+  if (rc) return rc;
+  if (dtype != UBT_F32 && dtype != UBT_BF16) return UBT_ERR_INVALID_ARG;
+  if (!unigram_logits || !aligned16(unigram_logits)) return UBT_ERR_INVALID_ARG;
+  if ((rc = check_tree(out, true))) return rc;
+  if ((rc = check_draft_opts(opts))) return rc;
+  if (L > 1 && (!bigram_scores || !aligned16(bigram_scores))) return UBT_ERR_INVALID_ARG;
+  if (out->B != B || out->N != N || out->L != L || out->k != k) return UBT_ERR_INVALID_ARG;
+  if (tree_smem_bytes(L, k, N) > (size_t)device_info().max_smem_optin) return UBT_ERR_UNSUPPORTED;
+  if (B == 0) return UBT_OK;
+  rc = ubt_topk_logprob(unigram_logits, dtype, (int64_t)B * L, V, k, out->cand_ids, out->cand_logprob, workspace,
+                        workspace_bytes, cuda_stream);
+  if (rc) return rc;
+  return ubt_build_tree(bigram_scores, B, L, k, N, opts, out, cuda_stream);
+}
+
+int ubt_verify_tree(const ubt_tree* tree, const void* target_logits, int dtype, int V, int mode,
+                    const ubt_verify_opts* opts, ubt_verify_result* out, void* workspace, size_t workspace_bytes,
+                    void* cuda_stream) {
+  int rc = check_tree(tree, false);
+  if (rc) return rc;
+  if (!target_logits || !aligned16(target_logits) || !out || V < 1) return UBT_ERR_INVALID_ARG;
+  if (dtype != UBT_F32 && dtype != UBT_BF16) return UBT_ERR_INVALID_ARG;
+  if (mode != UBT_VERIFY_GREEDY && mode != UBT_VERIFY_SAMPLE) return UBT_ERR_INVALID_ARG;
+  if (!out->accepted_len || !out->bonus_token || !out->accepted_nodes || !out->out_tokens) return UBT_ERR_INVALID_ARG;
+  const int B = tree->B, N = tree->N, L = tree->L;
+  if (B < 0 || N < 1 || L < 1) return UBT_ERR_INVALID_ARG;
+  if (N > kMaxN || L > kMaxL) return UBT_ERR_UNSUPPORTED;
+  const ubt_verify_opts d{0, 1.0f, nullptr, nullptr, nullptr};
+  const ubt_verify_opts* o = opts ? opts : &d;
+  if (mode == UBT_VERIFY_SAMPLE) {
+    if (!(o->temperature > 0.0f)) return UBT_ERR_INVALID_ARG;
+    if (V > 2048 * 1024) return UBT_ERR_UNSUPPORTED;
+  }
+  if (B == 0) return UBT_OK;
+  const int64_t rows = (int64_t)B * N;
+  if (!workspace || !aligned16(workspace) || workspace_bytes < verify_workspace_bytes(rows, V, mode))
+    return UBT_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  VerifyWorkspace w = carve_verify_workspace(workspace, rows, V, mode);
+  const int32_t* sampled = nullptr;
+  if (o->event_before && cudaEventRecord(static_cast<cudaEvent_t>(o->event_before), st) != cudaSuccess)
+    return UBT_ERR_CUDA;
+  if (mode == UBT_VERIFY_GREEDY) {
+    if (launch_row_argmax(target_logits, dtype, rows, V, w, st) != cudaSuccess) return UBT_ERR_CUDA;
+  } else {
+    int32_t* pick = o->node_pick ? o->node_pick : w.pick;
+    if (launch_row_sample(target_logits, dtype, B, N, V, o->seed, o->temperature, pick, st) != cudaSuccess)
+      return UBT_ERR_CUDA;
+    sampled = pick;
+  }
+  if (o->event_after && cudaEventRecord(static_cast<cudaEvent_t>(o->event_after), st) != cudaSuccess)
+    return UBT_ERR_CUDA;
+  if (launch_walk(*tree, mode, w, V, sampled, o->node_pick, *out, st) != cudaSuccess) return UBT_ERR_CUDA;
+  return UBT_OK;
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------------------- host-buffer forms
+namespace {
+struct Carver {
+  unsigned char* base;
+  size_t off = 0;
+  template <typename T> T* take(size_t count) {
+    T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+    off += align_up(count * sizeof(T), 256);
+    return p;
+  }
+};
+
+struct DeviceTree {
+  ubt_tree t;
+  void carve(Carver& c, int B, int L, int k, int N, bool cands) {
+    t.B = B; t.N = N; t.L = L; t.k = k; t.mask_words = (N + 31) / 32;
+    const size_t bn = (size_t)B * N;
+    t.token_ids = c.take<int32_t>(bn); t.parents = c.take<int32_t>(bn); t.depths = c.take<int32_t>(bn);
+    t.position_ids = c.take<int32_t>(bn); t.cand_rank = c.take<int32_t>(bn); t.scores = c.take<float>(bn);
+    t.mask = c.take<uint32_t>(bn * t.mask_words); t.n_nodes = c.take<int32_t>((size_t)B);
+    t.cand_ids = cands ? c.take<int32_t>((size_t)B * L * k) : nullptr;
+    t.cand_logprob = cands ? c.take<float>((size_t)B * L * k) : nullptr;
+  }
+};
+
+struct DraftHostLayout {
+  void* logits; float* bigram; float *alpha, *lambda, *anchor_bigram; int32_t *anchor_tokens, *pos_offset;
+  DeviceTree tree; void* ws; size_t ws_bytes; size_t total;
+  DraftHostLayout(void* buf, int B, int L, int V, int k, int N, int dtype) {
+    Carver c{static_cast<unsigned char*>(buf)};
+    logits = c.take<unsigned char>((size_t)B * L * V * esize(dtype));
+    bigram = c.take<float>((size_t)B * (L - 1) * k * k);
+    alpha = c.take<float>((size_t)L); lambda = c.take<float>((size_t)L);
+    anchor_bigram = c.take<float>((size_t)B * k);
+    anchor_tokens = c.take<int32_t>((size_t)B); pos_offset = c.take<int32_t>((size_t)B);
+    tree.carve(c, B, L, k, N, true);
+    ws_bytes = ubt_draft_workspace_bytes(B, L, V, k, N);
+    ws = c.take<unsigned char>(ws_bytes);
+    total = c.off;
+  }
+};
+
+struct VerifyHostLayout {
+  void* logits; DeviceTree tree; int32_t *accepted_len, *bonus, *accepted_nodes, *out_tokens, *node_pick;
+  void* ws; size_t ws_bytes; size_t total;
+  VerifyHostLayout(void* buf, int B, int L, int N, int V, int dtype, int mode) {
+    Carver c{static_cast<unsigned char*>(buf)};
+    logits = c.take<unsigned char>((size_t)B * N * V * esize(dtype));
+    tree.carve(c, B, L, 1, N, false);
+    accepted_len = c.take<int32_t>((size_t)B); bonus = c.take<int32_t>((size_t)B);
+    accepted_nodes = c.take<int32_t>((size_t)B * (L + 1)); out_tokens = c.take<int32_t>((size_t)B * (L + 1));
+    node_pick = c.take<int32_t>((size_t)B * N);
+    ws_bytes = ubt_verify_workspace_bytes(B, N, V, mode);
+    ws = c.take<unsigned char>(ws_bytes);
+    total = c.off;
+  }
+};
+
+#define UBT_CUDA_OK(call) do { if ((call) != cudaSuccess) { cudaGetLastError(); return UBT_ERR_CUDA; } } while (0)
+}  // namespace
+
+extern "C" {
+
+size_t ubt_draft_host_buffer_bytes(int B, int L, int V, int k, int N, int dtype) {
+  if (check_shape(B, L, V, k, N) != UBT_OK || (dtype != UBT_F32 && dtype != UBT_BF16)) return 0;
+  return DraftHostLayout(nullptr, B, L, V, k, N, dtype).total;
+}
+
+size_t ubt_verify_host_buffer_bytes(int B, int L, int N, int V, int dtype, int mode) {
+  if (B < 0 || L < 1 || N < 1 || V < 1 || (dtype != UBT_F32 && dtype != UBT_BF16)) return 0;
+  if (mode != UBT_VERIFY_GREEDY && mode != UBT_VERIFY_SAMPLE) return 0;
+  return VerifyHostLayout(nullptr, B, L, N, V, dtype, mode).total;
+}
+
+int ubt_draft_tree_host(const void* unigram_logits, int dtype, const float* bigram_scores, int B, int L, int V, int k,
+                        int N, const ubt_draft_opts* opts, ubt_tree* out, void* device_buffer,
+                        size_t device_buffer_bytes, void* cuda_stream) {
+  int rc = check_shape(B, L, V, k, N);
+  if (rc) return rc;
+  if (dtype != UBT_F32 && dtype != UBT_BF16) return UBT_ERR_INVALID_ARG;
+  if (!unigram_logits || !out || (L > 1 && !bigram_scores)) return UBT_ERR_INVALID_ARG;
+  if (out->B != B || out->N != N || out->L != L || out->k != k) return UBT_ERR_INVALID_ARG;
+  if ((rc = check_draft_opts(opts))) return rc;
+  if (!device_buffer || !aligned16(device_buffer) ||
+      device_buffer_bytes < ubt_draft_host_buffer_bytes(B, L, V, k, N, dtype))
+    return UBT_ERR_WORKSPACE;
+  if (B == 0) return UBT_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  DraftHostLayout d(device_buffer, B, L, V, k, N, dtype);
+  UBT_CUDA_OK(cudaMemcpyAsync(d.logits, unigram_logits, (size_t)B * L * V * esize(dtype), cudaMemcpyHostToDevice, st));
+  if (L > 1)
+    UBT_CUDA_OK(cudaMemcpyAsync(d.bigram, bigram_scores, sizeof(float) * (size_t)B * (L - 1) * k * k,
+                                cudaMemcpyHostToDevice, st));
+  ubt_draft_opts dev_opts{};
+  if (opts) {
+    dev_opts.search_width = opts->search_width;
+    dev_opts.depth_bonus = opts->depth_bonus;
+    if (opts->alpha) { UBT_CUDA_OK(cudaMemcpyAsync(d.alpha, opts->alpha, sizeof(float) * L, cudaMemcpyHostToDevice, st)); dev_opts.alpha = d.alpha; }
+    if (opts->lambda) { UBT_CUDA_OK(cudaMemcpyAsync(d.lambda, opts->lambda, sizeof(float) * L, cudaMemcpyHostToDevice, st)); dev_opts.lambda = d.lambda; }
+    if (opts->anchor_bigram) { UBT_CUDA_OK(cudaMemcpyAsync(d.anchor_bigram, opts->anchor_bigram, sizeof(float) * (size_t)B * k, cudaMemcpyHostToDevice, st)); dev_opts.anchor_bigram = d.anchor_bigram; }
+    if (opts->anchor_tokens) { UBT_CUDA_OK(cudaMemcpyAsync(d.anchor_tokens, opts->anchor_tokens, sizeof(int32_t) * B, cudaMemcpyHostToDevice, st)); dev_opts.anchor_tokens = d.anchor_tokens; }
+    if (opts->pos_offset) { UBT_CUDA_OK(cudaMemcpyAsync(d.pos_offset, opts->pos_offset, sizeof(int32_t) * B, cudaMemcpyHostToDevice, st)); dev_opts.pos_offset = d.pos_offset; }
+  }
+  rc = ubt_draft_tree(d.logits, dtype, L > 1 ? d.bigram : nullptr, B, L, V, k, N, &dev_opts, &d.tree.t, d.ws,
+                      d.ws_bytes, cuda_stream);
+  if (rc) return rc;
+  const size_t bn = (size_t)B * N;
+  const ubt_tree& t = d.tree.t;
+  struct { void* dst; const void* src; size_t bytes; } copies[] = {
+      {out->token_ids, t.token_ids, bn * 4}, {out->parents, t.parents, bn * 4}, {out->depths, t.depths, bn * 4},
+      {out->position_ids, t.position_ids, bn * 4}, {out->cand_rank, t.cand_rank, bn * 4},
+      {out->scores, t.scores, bn * 4}, {out->mask, t.mask, bn * t.mask_words * 4}, {out->n_nodes, t.n_nodes, (size_t)B * 4},
+      {out->cand_ids, t.cand_ids, (size_t)B * L * k * 4}, {out->cand_logprob, t.cand_logprob, (size_t)B * L * k * 4}};
+  for (auto& c : copies)
+    if (c.dst) UBT_CUDA_OK(cudaMemcpyAsync(c.dst, c.src, c.bytes, cudaMemcpyDeviceToHost, st));
+  UBT_CUDA_OK(cudaStreamSynchronize(st));
+  return UBT_OK;
+}
+
+int ubt_verify_tree_host(const ubt_tree* tree, const void* target_logits, int dtype, int V, int mode,
+                         const ubt_verify_opts* opts, ubt_verify_result* out, void* device_buffer,
+                         size_t device_buffer_bytes, void* cuda_stream) {
+  if (!tree || !target_logits || !out || V < 1) return UBT_ERR_INVALID_ARG;
+  if (dtype != UBT_F32 && dtype != UBT_BF16) return UBT_ERR_INVALID_ARG;
+  if (mode != UBT_VERIFY_GREEDY && mode != UBT_VERIFY_SAMPLE) return UBT_ERR_INVALID_ARG;
+  const int B = tree->B, N = tree->N, L = tree->L;
+  if (B < 0 || N < 1 || L < 1) return UBT_ERR_INVALID_ARG;
+  if (N > kMaxN || L > kMaxL) return UBT_ERR_UNSUPPORTED;
+  if (!tree->token_ids || !tree->parents || !tree->n_nodes) return UBT_ERR_INVALID_ARG;
+  if (!out->accepted_len || !out->bonus_token || !out->accepted_nodes || !out->out_tokens) return UBT_ERR_INVALID_ARG;
+  if (!device_buffer || !aligned16(device_buffer) ||
+      device_buffer_bytes < ubt_verify_host_buffer_bytes(B, L, N, V, dtype, mode))
+    return UBT_ERR_WORKSPACE;
+  if (B == 0) return UBT_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  VerifyHostLayout d(device_buffer, B, L, N, V, dtype, mode);
+  const size_t bn = (size_t)B * N;
+  UBT_CUDA_OK(cudaMemcpyAsync(d.logits, target_logits, bn * V * esize(dtype), cudaMemcpyHostToDevice, st));
+  UBT_CUDA_OK(cudaMemcpyAsync(d.tree.t.token_ids, tree->token_ids, bn * 4, cudaMemcpyHostToDevice, st));
+  UBT_CUDA_OK(cudaMemcpyAsync(d.tree.t.parents, tree->parents, bn * 4, cudaMemcpyHostToDevice, st));
+  UBT_CUDA_OK(cudaMemcpyAsync(d.tree.t.n_nodes, tree->n_nodes, (size_t)B * 4, cudaMemcpyHostToDevice, st));
+  ubt_verify_opts dev_opts{0, 1.0f, nullptr, nullptr, nullptr};
+  if (opts) { dev_opts = *opts; }
+  int32_t* host_pick = dev_opts.node_pick;
+  dev_opts.node_pick = host_pick ? d.node_pick : nullptr;
+  ubt_verify_result r{d.accepted_len, d.bonus, d.accepted_nodes, d.out_tokens};
+  int rc = ubt_verify_tree(&d.tree.t, d.logits, dtype, V, mode, &dev_opts, &r, d.ws, d.ws_bytes, cuda_stream);
+  if (rc) return rc;
+  UBT_CUDA_OK(cudaMemcpyAsync(out->accepted_len, d.accepted_len, (size_t)B * 4, cudaMemcpyDeviceToHost, st));
+  UBT_CUDA_OK(cudaMemcpyAsync(out->bonus_token, d.bonus, (size_t)B * 4, cudaMemcpyDeviceToHost, st));
+  UBT_CUDA_OK(cudaMemcpyAsync(out->accepted_nodes, d.accepted_nodes, (size_t)B * (L + 1) * 4, cudaMemcpyDeviceToHost, st));
+  UBT_CUDA_OK(cudaMemcpyAsync(out->out_tokens, d.out_tokens, (size_t)B * (L + 1) * 4, cudaMemcpyDeviceToHost, st));
+  if (host_pick) UBT_CUDA_OK(cudaMemcpyAsync(host_pick, d.node_pick, bn * 4, cudaMemcpyDeviceToHost, st));
+  UBT_CUDA_OK(cudaStreamSynchronize(st));
+  return UBT_OK;
+}
+
+}  // extern "C"

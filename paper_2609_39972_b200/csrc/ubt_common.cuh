@@ -1,0 +1,93 @@
+// Shared device helpers of the UBTree hot-path kernels (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ubt {
+
+constexpr unsigned FULL = 0xffffffffu;
+constexpr float kLog2e = 1.4426950408889634f;
+
+// ---------------------------------------------------------------- ordering keys
+// Monotone map float -> uint32 (larger float <=> larger key); -0 and +0 share a key.
+// NaN has no place in the order; the callers document NaN-free inputs.
+__device__ __forceinline__ uint32_t f2key(float x) {
+  uint32_t b = __float_as_uint(__fadd_rn(x, 0.0f));  // -0 + 0 = +0
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float key2f(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+// (value desc, index asc) as one descending 64-bit key.
+__device__ __forceinline__ uint64_t make_key(float x, int idx) {
+  return ((uint64_t)f2key(x) << 32) | (uint32_t)(~(uint32_t)idx);
+}
+__device__ __forceinline__ int key_idx(uint64_t k) { return (int)(~(uint32_t)k); }
+__device__ __forceinline__ float key_val(uint64_t k) { return key2f((uint32_t)(k >> 32)); }
+
+// ---------------------------------------------------------------- streaming loads
+__device__ __forceinline__ uint4 ldg_stream(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+// One 16-byte fragment of a logits row as floats.
+template <typename T> struct Frag;
+template <> struct Frag<__nv_bfloat16> {
+  static constexpr int N = 8;
+  float x[8];
+  __device__ __forceinline__ void unpack(const uint4& v) {
+    x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xffff0000u);
+    x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xffff0000u);
+    x[4] = __uint_as_float(v.z << 16); x[5] = __uint_as_float(v.z & 0xffff0000u);
+    x[6] = __uint_as_float(v.w << 16); x[7] = __uint_as_float(v.w & 0xffff0000u);
+  }
+};
+template <> struct Frag<float> {
+  static constexpr int N = 4;
+  float x[4];
+  __device__ __forceinline__ void unpack(const uint4& v) {
+    x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y);
+    x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
+  }
+};
+
+__device__ __forceinline__ float load_elem(const __nv_bfloat16* p, int64_t i) {
+  return __uint_as_float((uint32_t)reinterpret_cast<const unsigned short*>(p)[i] << 16);
+}
+__device__ __forceinline__ float load_elem(const float* p, int64_t i) { return p[i]; }
+
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// ---------------------------------------------------------------- warp / block reductions
+__device__ __forceinline__ uint64_t warp_max_u64(uint64_t v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    uint64_t w = __shfl_xor_sync(FULL, v, o);
+    v = w > v ? w : v;
+  }
+  return v;
+}
+__device__ __forceinline__ uint64_t warp_sum_u64(uint64_t v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
+  return v;
+}
+
+// How a flat range of rows*V elements is cut into per-CTA spans.
+struct SpanPlan {
+  int64_t span;  // elements per CTA (multiple of 256)
+  int grid;      // CTAs
+  int smax;      // partial slots per row: a row meets at most this many spans
+};
+
+}  // namespace ubt

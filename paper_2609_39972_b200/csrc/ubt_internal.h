@@ -1,0 +1,68 @@
+// Launchers shared between the translation units of libubt (host side, not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/ubt.h"
+#include "ubt_common.cuh"
+
+namespace ubt {
+
+constexpr int kMaxK = 64;
+constexpr int kMaxN = 256;
+constexpr int kMaxL = 64;
+constexpr size_t kTreeTableBytes = 160 * 1024;
+
+struct DeviceInfo {
+  int sm_count;
+  int max_smem_optin;
+};
+// Properties of the current device (queried once per device, cached).
+const DeviceInfo& device_info();
+
+// Cut rows*V elements into equal contiguous spans, one per CTA.
+SpanPlan make_span_plan(int64_t rows, int V, int ctas, int64_t min_span);
+
+// ---- a1: per-row (max, sum-exp, top-k) partials, then the per-row merge --------------------
+struct TopkWorkspace {
+  SpanPlan plan;
+  float* part_ms;     // [rows, smax, 2]
+  float* part_val;    // [rows, smax, k]
+  int32_t* part_idx;  // [rows, smax, k]
+  int32_t* part_cnt;  // [rows, smax]
+};
+SpanPlan topk_plan(int64_t rows, int V);
+size_t topk_workspace_bytes(int64_t rows, int V, int k);
+TopkWorkspace carve_topk_workspace(void* ws, int64_t rows, int V, int k);
+cudaError_t launch_lse_topk(const void* logits, int dtype, int64_t rows, int V, int k,
+                            const TopkWorkspace& w, cudaStream_t st);
+cudaError_t launch_merge_topk(int64_t rows, int V, int k, const TopkWorkspace& w, int32_t* cand_ids,
+                              float* cand_lp, cudaStream_t st);
+
+// ---- a2 + a3 + a3b --------------------------------------------------------------------------
+size_t tree_smem_bytes(int L, int k, int N);
+cudaError_t launch_build_tree(const float* bigram, int B, int L, int k, int N, int W, float zeta,
+                              const float* alpha, const float* lambda, const float* anchor_bigram,
+                              const int32_t* anchor_tokens, const int32_t* pos_offset,
+                              const ubt_tree& out, cudaStream_t st);
+cudaError_t launch_build_mask(const ubt_tree& tree, const int32_t* pos_offset, cudaStream_t st);
+
+// ---- a4 ---------------------------------------------------------------------------------------
+struct VerifyWorkspace {
+  SpanPlan plan;                 // greedy: spans of the row-argmax kernel
+  unsigned long long* part_key;  // greedy: [B*N, smax] (value, ~token) keys
+  int32_t* pick;                 // sampling: [B*N] picks when the caller gave no node_pick
+};
+size_t verify_workspace_bytes(int64_t rows, int V, int mode);
+VerifyWorkspace carve_verify_workspace(void* ws, int64_t rows, int V, int mode);
+cudaError_t launch_row_argmax(const void* logits, int dtype, int64_t rows, int V,
+                              const VerifyWorkspace& w, cudaStream_t st);
+cudaError_t launch_row_sample(const void* logits, int dtype, int B, int N, int V, uint64_t seed,
+                              float temperature, int32_t* pick, cudaStream_t st);
+cudaError_t launch_walk(const ubt_tree& tree, int mode, const VerifyWorkspace& w, int V,
+                        const int32_t* sampled_pick, int32_t* node_pick,
+                        const ubt_verify_result& out, cudaStream_t st);
+
+}  // namespace ubt

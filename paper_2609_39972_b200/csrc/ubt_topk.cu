@@ -1,0 +1,377 @@
+// Step a1: per-position vocabulary log-sum-exp and top-k candidates (eq. 3, "Candidate Sets").
+//
+// The rows*V logits are cut into equal contiguous spans, one per CTA, so that every SM streams the
+// same number of bytes whatever rows is.  A span meets a few row segments; for each the CTA emits a
+// partial (max, sum exp, sorted top-k) and a small merge kernel combines the partials of a row.
+//
+// Streaming one segment: every thread keeps an online (max, sum) pair and tests the fragment
+// maximum against a CTA-wide exclusive threshold; elements above it are appended (their column
+// only) to a shared pool.  The threshold starts at a bound obtained by bisecting the per-thread
+// maxima of the first tile and becomes exact whenever the pool is ranked ("flush").  The next tile
+// is prefetched into registers before the current one is processed, so the one barrier per tile
+// does not drain the loads in flight.
+#include "ubt_internal.h"
+
+namespace ubt {
+
+constexpr int G1_T = 512;    // threads per CTA
+constexpr int G1_U = 2;      // 16-byte fragments per thread per tile
+constexpr int G1_RC = 1024;  // pool entries ranked by counting; larger pools use k extraction rounds
+constexpr int G1_SLACK = 4 * kMaxK;  // a tile starts with fewer pool entries than this
+
+template <typename T, int VEC> struct RawFrag { uint4 v; };
+template <typename T> struct RawFrag<T, 1> { float v; };
+
+struct G1Shared {
+  int cnt;     // pool entries
+  int ntop;    // entries of top[]
+  float taux;  // exclusive threshold: x enters the pool iff x > taux
+  int pad;
+  float redf[2 * (G1_T / 32)];
+  unsigned long long red64[G1_T / 32];
+  unsigned long long top[kMaxK];
+  unsigned long long topn[kMaxK];
+  unsigned long long keys[G1_RC + kMaxK];
+};
+
+template <typename T, int VEC>
+__device__ __forceinline__ void load_frag(const T* seg, int nfrag, int i, RawFrag<T, VEC>& r) {
+  if constexpr (VEC == 1) {
+    r.v = i < nfrag ? load_elem(seg, i) : -INFINITY;
+  } else {
+    if (i < nfrag) {
+      r.v = ldg_stream(reinterpret_cast<const uint4*>(seg) + i);
+    } else {
+      const uint32_t ninf = sizeof(T) == 2 ? 0xff80ff80u : 0xff800000u;
+      r.v = make_uint4(ninf, ninf, ninf, ninf);
+    }
+  }
+}
+
+template <typename T, int VEC>
+__device__ __forceinline__ void unpack_frag(const RawFrag<T, VEC>& r, float (&x)[VEC]) {
+  if constexpr (VEC == 1) {
+    x[0] = r.v;
+  } else {
+    Frag<T> f;
+    f.unpack(r.v);
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) x[j] = f.x[j];
+  }
+}
+
+__device__ __forceinline__ unsigned long long block_max_u64(unsigned long long v, unsigned long long* red) {
+  v = warp_max_u64(v);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  unsigned long long r = 0;
+  for (int w = 0; w < (int)(blockDim.x >> 5); ++w) r = red[w] > r ? red[w] : r;
+  return r;
+}
+
+// Rank the pool (and the carried top list) exactly; afterwards top[0..ntop) is sorted best first,
+// the pool is empty and, when k entries exist, taux is the k-th best value (strict from then on:
+// a later element equal to it has a larger column than every kept entry).
+template <typename T>
+__device__ void flush_pool(G1Shared& sh, const int* pool, const T* rowp, int k) {
+  const int tid = threadIdx.x;
+  const int M = sh.cnt, nt = sh.ntop, total = M + nt;
+  const int newn = total < k ? total : k;
+  if (M <= G1_RC) {
+    for (int i = tid; i < M; i += G1_T) {
+      int col = pool[i];
+      sh.keys[i] = make_key(load_elem(rowp, col), col);
+    }
+    for (int i = tid; i < nt; i += G1_T) sh.keys[M + i] = sh.top[i];
+    __syncthreads();
+    for (int i = tid; i < total; i += G1_T) {
+      unsigned long long ki = sh.keys[i];
+      int rank = 0;
+      for (int j = 0; j < total; ++j) rank += sh.keys[j] > ki;
+      if (rank < k) sh.topn[rank] = ki;
+    }
+  } else {
+    unsigned long long last = ~0ull;
+    for (int r = 0; r < newn; ++r) {
+      unsigned long long best = 0;
+      for (int i = tid; i < M; i += G1_T) {
+        int col = pool[i];
+        unsigned long long key = make_key(load_elem(rowp, col), col);
+        if (key < last && key > best) best = key;
+      }
+      for (int i = tid; i < nt; i += G1_T) {
+        unsigned long long key = sh.top[i];
+        if (key < last && key > best) best = key;
+      }
+      best = block_max_u64(best, sh.red64);
+      if (tid == 0) sh.topn[r] = best;
+      last = best;
+    }
+  }
+  __syncthreads();
+  if (tid < newn) sh.top[tid] = sh.topn[tid];
+  if (tid == 0) {
+    sh.ntop = newn;
+    sh.cnt = 0;
+    if (newn == k) sh.taux = key_val(sh.topn[k - 1]);
+  }
+  __syncthreads();
+}
+
+template <typename T, int VEC>
+__global__ void __launch_bounds__(G1_T, VEC == 1 ? 1 : 2)
+k_lse_topk(const T* __restrict__ logits, int64_t total, int V, int k, SpanPlan plan,
+           float* __restrict__ part_ms, float* __restrict__ part_val, int32_t* __restrict__ part_idx,
+           int32_t* __restrict__ part_cnt) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  G1Shared& sh = *reinterpret_cast<G1Shared*>(smem_raw);
+  int* pool = reinterpret_cast<int*>(smem_raw + sizeof(G1Shared));
+  constexpr int TILE_FRAGS = G1_T * G1_U;
+
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int64_t lo = (int64_t)blockIdx.x * plan.span;
+  const int64_t hi = lo + plan.span < total ? lo + plan.span : total;
+
+  for (int64_t e = lo; e < hi;) {
+    const int64_t row = e / V;
+    const int c0 = (int)(e - row * V);
+    const int c1 = (int)((int64_t)V - c0 < hi - e ? V : c0 + (hi - e));
+    const T* rowp = logits + row * V;
+    const T* seg = rowp + c0;
+    const int nfrag = (c1 - c0) / VEC;  // spans and V are multiples of VEC on this path
+    e += c1 - c0;
+
+    if (tid == 0) { sh.cnt = 0; sh.ntop = 0; sh.taux = -INFINITY; }
+
+    float m_t = -3.0e38f, s_t = 0.f, negml = 3.0e38f * kLog2e;
+    RawFrag<T, VEC> cur[G1_U], nxt[G1_U];
+#pragma unroll
+    for (int u = 0; u < G1_U; ++u) load_frag<T, VEC>(seg, nfrag, u * G1_T + tid, cur[u]);
+
+    // Bound for the k-th largest element from the per-thread maxima of the first tile: bisect the
+    // top 16 key bits with CTA-wide counts; the result never exceeds the k-th largest maximum.
+    {
+      float tmax = -INFINITY;
+      bool has = false;
+#pragma unroll
+      for (int u = 0; u < G1_U; ++u) {
+        float x[VEC];
+        unpack_frag<T, VEC>(cur[u], x);
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) tmax = fmaxf(tmax, x[j]);
+        has = has || (u * G1_T + tid < nfrag);
+      }
+      const uint32_t mykey = has ? f2key(tmax) : 0u;
+      uint32_t lob = 0;
+      for (int bit = 31; bit >= 16; --bit) {
+        uint32_t cand = lob | (1u << bit);
+        if (__syncthreads_count(mykey >= cand) >= k) lob = cand;
+      }
+      if (tid == 0 && lob != 0) {
+        uint32_t below = lob - 1;
+        if (below == 0x7fffffffu) below = 0x7ffffffeu;  // skip -0: it equals +0
+        float t = key2f(below);
+        sh.taux = (t != t) ? -INFINITY : t;
+      }
+      __syncthreads();
+    }
+
+    for (int base = 0; base < nfrag; base += TILE_FRAGS) {
+      const float taux = sh.taux;
+      if (base + TILE_FRAGS < nfrag) {
+#pragma unroll
+        for (int u = 0; u < G1_U; ++u)
+          load_frag<T, VEC>(seg, nfrag, base + TILE_FRAGS + u * G1_T + tid, nxt[u]);
+      }
+#pragma unroll
+      for (int u = 0; u < G1_U; ++u) {
+        float x[VEC];
+        unpack_frag<T, VEC>(cur[u], x);
+        float vmax = x[0];
+#pragma unroll
+        for (int j = 1; j < VEC; ++j) vmax = fmaxf(vmax, x[j]);
+        if (vmax > m_t) {  // online rescale; rare after the first fragments
+          s_t *= ex2_approx(fmaf(m_t, kLog2e, -vmax * kLog2e));
+          m_t = vmax;
+          negml = -vmax * kLog2e;
+        }
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) s_t += ex2_approx(fmaf(x[j], kLog2e, negml));
+        if (__any_sync(FULL, vmax > taux)) {
+          const int col0 = c0 + (base + u * G1_T + tid) * VEC;
+#pragma unroll
+          for (int j = 0; j < VEC; ++j) {
+            const bool hit = x[j] > taux;
+            const unsigned mask = __ballot_sync(FULL, hit);
+            if (mask) {
+              const int leader = __ffs(mask) - 1;
+              int at = 0;
+              if (lane == leader) at = atomicAdd(&sh.cnt, __popc(mask));
+              at = __shfl_sync(FULL, at, leader);
+              if (hit) pool[at + __popc(mask & ((1u << lane) - 1))] = col0 + j;
+            }
+          }
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < G1_U; ++u) cur[u] = nxt[u];
+      __syncthreads();
+      if (sh.cnt >= 4 * k) flush_pool<T>(sh, pool, rowp, k);  // tighten the threshold early
+    }
+    flush_pool<T>(sh, pool, rowp, k);
+
+    // partial (max, sum exp) of the segment
+    float mw = m_t;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mw = fmaxf(mw, __shfl_xor_sync(FULL, mw, o));
+    if (lane == 0) sh.redf[tid >> 5] = mw;
+    __syncthreads();
+    float M = sh.redf[0];
+    for (int w = 1; w < G1_T / 32; ++w) M = fmaxf(M, sh.redf[w]);
+    float sw = s_t * ex2_approx((m_t - M) * kLog2e);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sw += __shfl_xor_sync(FULL, sw, o);
+    if (lane == 0) sh.redf[G1_T / 32 + (tid >> 5)] = sw;
+    __syncthreads();
+
+    const int64_t c_first = (row * (int64_t)V) / plan.span;
+    const int64_t slot = row * plan.smax + ((int64_t)blockIdx.x - c_first);
+    if (tid == 0) {
+      float S = 0.f;
+      for (int w = 0; w < G1_T / 32; ++w) S += sh.redf[G1_T / 32 + w];
+      part_ms[slot * 2] = M;
+      part_ms[slot * 2 + 1] = S;
+      part_cnt[slot] = sh.ntop;
+    }
+    if (tid < sh.ntop) {
+      part_val[slot * k + tid] = key_val(sh.top[tid]);
+      part_idx[slot * k + tid] = key_idx(sh.top[tid]);
+    }
+    __syncthreads();
+  }
+}
+
+// One warp per row: combine the partials of the row's segments.
+__global__ void __launch_bounds__(128)
+k_merge_topk(const float* __restrict__ part_ms, const float* __restrict__ part_val,
+             const int32_t* __restrict__ part_idx, const int32_t* __restrict__ part_cnt, int64_t rows,
+             int V, int k, SpanPlan plan, int32_t* __restrict__ cand_ids, float* __restrict__ cand_lp) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const int64_t c_first = (row * (int64_t)V) / plan.span;
+  const int64_t c_last = ((row + 1) * (int64_t)V - 1) / plan.span;
+  const int nseg = (int)(c_last - c_first + 1);
+  const int64_t base = row * plan.smax;
+
+  float M = -3.0e38f;
+  for (int j = lane; j < nseg; j += 32) M = fmaxf(M, part_ms[(base + j) * 2]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(FULL, M, o));
+  float S = 0.f;
+  for (int j = lane; j < nseg; j += 32)
+    S += part_ms[(base + j) * 2 + 1] * exp2f((part_ms[(base + j) * 2] - M) * kLog2e);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) S += __shfl_xor_sync(FULL, S, o);
+  const float lse = M + logf(S);
+
+  int found = 0;
+  const int nq = nseg * k;
+  for (int q = lane; q < nq; q += 32) {
+    const int j = q / k, i = q - j * k;
+    if (i >= part_cnt[base + j]) continue;
+    const float val = part_val[(base + j) * k + i];
+    const int idx = part_idx[(base + j) * k + i];
+    const uint64_t key = make_key(val, idx);
+    int rank = 0;
+    for (int j2 = 0; j2 < nseg; ++j2) {
+      const int c2 = part_cnt[base + j2];
+      for (int i2 = 0; i2 < c2; ++i2)
+        rank += make_key(part_val[(base + j2) * k + i2], part_idx[(base + j2) * k + i2]) > key;
+    }
+    if (rank < k) {
+      cand_ids[row * k + rank] = idx;
+      cand_lp[row * k + rank] = val - lse;
+    }
+  }
+  for (int j = lane; j < nseg; j += 32) found += part_cnt[base + j];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) found += __shfl_xor_sync(FULL, found, o);
+  for (int r = found + lane; r < k; r += 32) {  // fewer than k entries above -inf: documented as unsupported
+    cand_ids[row * k + r] = -1;
+    cand_lp[row * k + r] = -INFINITY;
+  }
+}
+
+// ------------------------------------------------------------------------------------ host side
+SpanPlan make_span_plan(int64_t rows, int V, int ctas, int64_t min_span) {
+  SpanPlan p;
+  const int64_t total = rows * (int64_t)V;
+  int64_t span = (total + ctas - 1) / ctas;
+  if (span < min_span) span = min_span;
+  span = (span + 255) / 256 * 256;
+  p.span = span;
+  p.grid = (int)((total + span - 1) / span);
+  if (p.grid < 1) p.grid = 1;
+  p.smax = (int)(((int64_t)V + span - 1) / span) + 1;
+  return p;
+}
+
+SpanPlan topk_plan(int64_t rows, int V) {
+  return make_span_plan(rows, V, device_info().sm_count * 2, 32768);
+}
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+size_t topk_workspace_bytes(int64_t rows, int V, int k) {
+  const SpanPlan p = topk_plan(rows, V);
+  const size_t slots = (size_t)rows * p.smax;
+  return align_up(slots * 2 * sizeof(float), 256) + align_up(slots * k * sizeof(float), 256) +
+         align_up(slots * k * sizeof(int32_t), 256) + align_up(slots * sizeof(int32_t), 256);
+}
+
+TopkWorkspace carve_topk_workspace(void* ws, int64_t rows, int V, int k) {
+  TopkWorkspace w;
+  w.plan = topk_plan(rows, V);
+  const size_t slots = (size_t)rows * w.plan.smax;
+  unsigned char* p = static_cast<unsigned char*>(ws);
+  w.part_ms = reinterpret_cast<float*>(p); p += align_up(slots * 2 * sizeof(float), 256);
+  w.part_val = reinterpret_cast<float*>(p); p += align_up(slots * k * sizeof(float), 256);
+  w.part_idx = reinterpret_cast<int32_t*>(p); p += align_up(slots * k * sizeof(int32_t), 256);
+  w.part_cnt = reinterpret_cast<int32_t*>(p);
+  return w;
+}
+
+template <typename T, int VEC>
+static cudaError_t launch_lse_topk_t(const void* logits, int64_t rows, int V, int k,
+                                     const TopkWorkspace& w, cudaStream_t st) {
+  const size_t smem = sizeof(G1Shared) + sizeof(int) * (size_t)(G1_T * G1_U * VEC + G1_SLACK);
+  auto kern = k_lse_topk<T, VEC>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  kern<<<w.plan.grid, G1_T, smem, st>>>(static_cast<const T*>(logits), rows * (int64_t)V, V, k, w.plan,
+                                        w.part_ms, w.part_val, w.part_idx, w.part_cnt);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_lse_topk(const void* logits, int dtype, int64_t rows, int V, int k,
+                            const TopkWorkspace& w, cudaStream_t st) {
+  if (dtype == UBT_BF16) {
+    if (V % 8 == 0) return launch_lse_topk_t<__nv_bfloat16, 8>(logits, rows, V, k, w, st);
+    return launch_lse_topk_t<__nv_bfloat16, 1>(logits, rows, V, k, w, st);
+  }
+  if (V % 4 == 0) return launch_lse_topk_t<float, 4>(logits, rows, V, k, w, st);
+  return launch_lse_topk_t<float, 1>(logits, rows, V, k, w, st);
+}
+
+cudaError_t launch_merge_topk(int64_t rows, int V, int k, const TopkWorkspace& w, int32_t* cand_ids,
+                              float* cand_lp, cudaStream_t st) {
+  const int warps = 4;
+  const int grid = (int)((rows + warps - 1) / warps);
+  k_merge_topk<<<grid, warps * 32, 0, st>>>(w.part_ms, w.part_val, w.part_idx, w.part_cnt, rows, V, k,
+                                            w.plan, cand_ids, cand_lp);
+  return cudaGetLastError();
+}
+
+}  // namespace ubt

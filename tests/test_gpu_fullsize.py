@@ -1,0 +1,100 @@
+"""Full-size configurations in the launch configuration the benchmark times; the oracle checks a sample.
+
+Inputs of 0.8-5.6 GB are drawn on the device (seeded torch generator); the sequences the oracle checks
+are copied back bit for bit, so both sides read the same bytes.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import ubt_synth as synth
+from parity import compare_draft, compare_verify, tree_to_numpy
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _run_full(name, sample, seeds=(0,)):
+    import paper_2609_39972_b200 as u
+    cfg = synth.CONFIGS[name]
+    ud, bd, zd = synth.device_inputs(cfg, 11, DEV)
+    gtree = u.ubt_draft_tree(ud, bd, cfg.k, cfg.N)
+    torch.cuda.synchronize()
+    g = tree_to_numpy(gtree)
+    rows = sorted(sample)
+    uh = synth.to_host_bits(ud[rows]); bh = synth.to_host_bits(bd[rows]); zh = synth.to_host_bits(zd[rows])
+    otree = oracle.draft_tree(uh, bh, cfg.k, cfg.N)
+    swaps = compare_draft(g, otree, cfg.L, cfg.k, cfg.N, rows=rows)
+    print(f"{name}: near-tie swaps on the sampled sequences: {swaps}")
+    pick = torch.empty((cfg.B, cfg.N), dtype=torch.int32, device=DEV)
+    sub = lambda a: a[rows]
+    for s in seeds:
+        res = u.ubt_verify_tree(gtree, zd, cfg.mode, seed=s, node_pick=pick)
+        torch.cuda.synchronize()
+        if cfg.mode == "greedy":
+            ov = oracle.verify(sub(g.token_ids), sub(g.parents), sub(g.n_nodes), cfg.L, zh, "greedy")
+        else:   # the Philox counter holds the true batch index b
+            ov = _oracle_sample_rows(g, zh, rows, cfg, s)
+        compare_verify(res, ov, pick, rows=rows)
+    # properties that hold at any size, on the whole batch
+    n = g.n_nodes
+    assert np.all(n >= 1) and np.all(n <= cfg.N)
+    par = g.parents
+    idx = np.arange(cfg.N)[None, :]
+    assert np.all((par < idx) | (idx >= n[:, None]))
+    acc = res.accepted_len.cpu().numpy()
+    assert np.all(acc >= 0) and np.all(acc <= cfg.L)
+    pk = pick.cpu().numpy()
+    assert pk.min() >= 0 and pk.max() < cfg.V
+    if cfg.mode == "greedy":
+        # sampled rows of the full batch against a library argmax on the device copy
+        rr = np.random.default_rng(0).integers(0, cfg.B * cfg.N, 64)
+        flat = zd.view(cfg.B * cfg.N, cfg.V)
+        for r in rr:
+            assert int(torch.argmax(flat[r].float())) == pk.reshape(-1)[r] or \
+                flat[r, pk.reshape(-1)[r]] == flat[r].max()
+
+
+_CDF_CACHE = {}
+
+
+def _oracle_sample_rows(g, zh, rows, cfg, seed):
+    """Oracle sampling verdicts for sampled sequences, each under its TRUE batch index.
+
+    The draw is keyed by (seed, b, n) and the oracle's whole-batch call numbers sequences by their
+    position in the array it is given, so the sampled sequences go through its row-level primitives:
+    row CDF, threshold of (seed, b, n), first token whose prefix sum exceeds it, then the walk.
+    """
+    acc, bonus, nodes, toks, picks = [], [], [], [], []
+    for j, b in enumerate(rows):
+        if (id(zh), j) not in _CDF_CACHE:
+            _CDF_CACHE[(id(zh), j)] = np.stack([oracle.row_cdf(zh[j], n) for n in range(cfg.N)])
+        cdf = _CDF_CACHE[(id(zh), j)]
+        pk = np.array([int(np.searchsorted(cdf[n], oracle.threshold(seed, b, n, int(cdf[n, -1])), side="right"))
+                       for n in range(cfg.N)], np.int32)
+        a, bo = oracle.walks_from_cdf(g.token_ids[b], g.parents[b], int(g.n_nodes[b]), cdf, b,
+                                      np.array([seed], np.uint64))
+        cur, an, ot = 0, [0], []
+        for _ in range(int(a[0])):
+            x = pk[cur]
+            cur = [c for c in range(1, int(g.n_nodes[b])) if g.parents[b, c] == cur and g.token_ids[b, c] == x][0]
+            an.append(cur); ot.append(int(x))
+        ot.append(int(bo[0]))
+        pad = lambda v: v + [-1] * (cfg.L + 1 - len(v))
+        acc.append(int(a[0])); bonus.append(int(bo[0])); nodes.append(pad(an)); toks.append(pad(ot)); picks.append(pk)
+    return oracle.Verdict(np.array(acc, np.int32), np.array(nodes, np.int32), np.array(toks, np.int32),
+                          np.array(bonus, np.int32), np.stack(picks))
+
+
+def test_c3_full_batch():
+    _run_full("c3", sample=range(32))          # every sequence
+
+
+def test_c4_full_batch_sampled():
+    _run_full("c4", sample=[0, 17, 63])
+
+
+def test_c5_full_batch_sampled():
+    _run_full("c5", sample=[0, 64, 127], seeds=(0, 12345))
+    _CDF_CACHE.clear()

@@ -1,0 +1,240 @@
+"""CUDA path vs oracle through the C ABI, element by element on the same seeded inputs (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import ubt_synth as synth
+from parity import compare_draft, compare_verify, tree_to_numpy
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def ubt():
+    import paper_2609_39972_b200 as u
+    return u
+
+
+def run_case(cfg, seed, targets="plant", W=0, zeta=0.0, use_opts=False, seeds_sample=(0,)):
+    """Draft + verify one synthetic batch on the GPU and against the oracle; returns logged swaps."""
+    u = ubt()
+    di = synth.draft_inputs(cfg, seed)
+    rng = np.random.default_rng(seed + 1000)
+    kw_np = {}
+    if use_opts:
+        kw_np = dict(alpha=rng.uniform(0.5, 1.5, cfg.L).astype(np.float32),
+                     lam=rng.uniform(0.5, 2.0, cfg.L).astype(np.float32),
+                     anchor_bigram=rng.standard_normal((cfg.B, cfg.k)).astype(np.float32),
+                     anchor_tokens=rng.integers(0, cfg.V, cfg.B).astype(np.int32),
+                     pos_offset=rng.integers(0, 200000, cfg.B).astype(np.int32))
+    otree = oracle.draft_tree(di.unigram_logits, di.bigram_scores, cfg.k, cfg.N, W=W, zeta=zeta, **kw_np)
+    kw_t = {n: torch.from_numpy(v).to(DEV) for n, v in kw_np.items()}
+    ud = synth.to_device(di.unigram_logits, cfg.dtype, DEV)
+    bd = torch.from_numpy(di.bigram_scores).to(DEV)
+    gtree = u.ubt_draft_tree(ud, bd, cfg.k, cfg.N, search_width=W, depth_bonus=zeta, **kw_t)
+    torch.cuda.synchronize()
+    g = tree_to_numpy(gtree)
+    swaps = compare_draft(g, otree, cfg.L, cfg.k, cfg.N, W, zeta, kw_np.get("anchor_tokens"), kw_np.get("pos_offset"))
+    # targets are built from the GPU's tree arrays (identical to the oracle's unless a swap was logged)
+    if targets == "plant":
+        z = synth.target_logits(cfg, seed)
+        synth.plant_path(z, cfg.dtype, g.token_ids, g.parents, g.n_nodes, seed)
+    elif targets == "agree":
+        z = synth.agree_targets(cfg, di.unigram_logits, g.token_ids, g.parents, g.depths, g.n_nodes, seed)
+    else:
+        z = synth.target_logits(cfg, seed)
+    zd = synth.to_device(z, cfg.dtype, DEV)
+    pick = torch.empty((cfg.B, cfg.N), dtype=torch.int32, device=DEV)
+    if cfg.mode == "greedy":
+        res = u.ubt_verify_tree(gtree, zd, "greedy", node_pick=pick)
+        torch.cuda.synchronize()
+        ov = oracle.verify(g.token_ids, g.parents, g.n_nodes, cfg.L, z, "greedy")
+        compare_verify(res, ov, pick)
+        res2 = u.ubt_verify_tree(gtree, zd, "greedy")          # without node_pick
+        torch.cuda.synchronize()
+        compare_verify(res2, ov)
+    for s in (seeds_sample if cfg.mode == "sample" else ()):
+        res = u.ubt_verify_tree(gtree, zd, "sample", seed=s, temperature=1.0, node_pick=pick)
+        torch.cuda.synchronize()
+        ov = oracle.verify(g.token_ids, g.parents, g.n_nodes, cfg.L, z, "sample", seed=s, temperature=1.0)
+        compare_verify(res, ov, pick)
+    return swaps
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_c1_tiny_fp32_exact(seed):
+    assert run_case(synth.CONFIGS["c1"], seed) == []
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_c1_options_width_bonus(seed):
+    cfg = synth.CONFIGS["c1"]
+    run_case(cfg, seed, use_opts=True)
+    run_case(cfg, seed, W=3, zeta=-0.25, use_opts=True)
+    run_case(cfg, seed, W=1)
+
+
+def test_c1_sampling_modes():
+    cfg = synth.CONFIGS["c1"].replace(mode="sample")
+    run_case(cfg, 0, targets="agree", seeds_sample=range(12))
+
+
+def test_c2_single_stream():
+    swaps = run_case(synth.CONFIGS["c2"], 0)
+    print("c2 near-tie swaps:", swaps)
+
+
+def test_c2_agree_targets():
+    run_case(synth.CONFIGS["c2"], 1, targets="agree")
+
+
+def test_c3_batched():
+    swaps = run_case(synth.CONFIGS["c3"], 0, targets="plant")
+    print("c3 near-tie swaps:", swaps)
+
+
+def test_c4_reduced_batch_wide_tree():
+    cfg = synth.CONFIGS["c4"].replace(B=4)
+    swaps = run_case(cfg, 0, targets="plant")
+    print("c4(B=4) near-tie swaps:", swaps)
+    assert cfg.N == 256 and (cfg.N + 31) // 32 == 8          # 256 mask bits per node
+
+
+def test_c5_reduced_batch_sampling():
+    cfg = synth.CONFIGS["c5"].replace(B=3)
+    run_case(cfg, 0, targets="agree", seeds_sample=(0, 7))
+
+
+def test_paper_search_configuration_k64_w12():
+    # the paper's academic setup (Appendix B): K = 64, W = 12, 64 non-root nodes, 15 future positions;
+    # the pair table must fit shared memory, so L*k*k*5 <= 160 KiB caps L at 8 here
+    cfg = synth.Config("paper", 2, 8, 4096, 64, 65, "bf16", "pos_uniform:0.5,4", 1.0, 0.0, "greedy")
+    run_case(cfg, 0, W=12)
+    run_case(cfg, 1, W=0)
+
+
+@pytest.mark.parametrize("V,k,L,N,dtype", [
+    (1000, 4, 4, 16, "bf16"),     # aligned bf16, tiny
+    (1001, 4, 3, 9, "bf16"),      # V not a multiple of 8: scalar path
+    (1003, 5, 3, 9, "f32"),       # V not a multiple of 4: scalar path
+    (37, 8, 2, 5, "f32"),         # V smaller than a tile
+    (64, 64, 2, 33, "f32"),       # k == V == 64
+    (3000, 1, 5, 4, "bf16"),      # k = 1: a chain
+    (2048, 3, 1, 4, "f32"),       # L = 1: no bigram tensor
+    (500, 4, 4, 1, "f32"),        # N = 1: root only
+    (70001, 16, 6, 200, "bf16"),  # several spans per row, ragged tail, scalar path
+    (70000, 16, 6, 256, "bf16"),  # several spans per row, vector path
+])
+def test_edge_shapes(V, k, L, N, dtype):
+    cfg = synth.Config("edge", 3, L, V, k, N, dtype, "pos_uniform:0.5,3", 1.0, 0.0, "greedy")
+    run_case(cfg, 5, targets="plant")
+    run_case(cfg.replace(mode="sample"), 5, targets="agree", seeds_sample=(3,))
+
+
+def test_rows_full_of_ties():
+    # bf16 rows quantised to a handful of values, rows with +-0 at the top, a constant row
+    u = ubt()
+    rng = np.random.default_rng(0)
+    V, k = 4096, 8
+    x = np.round(rng.standard_normal((6, V)) * 2).astype(np.float32)
+    x[1, :] = 0.75
+    x[2] = -np.abs(x[2]); x[2, 100] = 0.0; x[2, 50] = -0.0
+    x[3, ::3] = x[3].max()
+    for dtype in ("bf16", "f32"):
+        host = synth.f32_to_bf16_bits(x) if dtype == "bf16" else x
+        ids, lp, _ = oracle.topk_logprob(host, k)
+        d = synth.to_device(host, dtype, DEV)
+        cid = torch.empty((6, k), dtype=torch.int32, device=DEV)
+        clp = torch.empty((6, k), dtype=torch.float32, device=DEV)
+        ws = u.workspace(u.ubt_draft_workspace_bytes(6, 1, V, k, 1), DEV)
+        u.ubt_topk_logprob(d, k, cid, clp, ws)
+        torch.cuda.synchronize()
+        assert cid.cpu().numpy().tolist() == ids.tolist()
+        np.testing.assert_allclose(clp.cpu().numpy(), lp, rtol=1e-5, atol=1e-5)
+        # greedy picks on the same rows: lowest token among the maxima
+        tree = u.Tree.empty(1, 6, 1, 1, DEV)
+        for t in (tree.token_ids, tree.parents):
+            t.fill_(-1)
+        tree.n_nodes.fill_(1)
+        pick = torch.empty((1, 6), dtype=torch.int32, device=DEV)
+        u.ubt_verify_tree(tree, d.view(1, 6, V), "greedy", node_pick=pick)
+        torch.cuda.synchronize()
+        assert pick.cpu().numpy()[0].tolist() == np.argmax(synth.as_f32(host, dtype), -1).tolist()
+
+
+def test_exact_score_ties_follow_total_order():
+    # integer-valued inputs with lambda = 0: many node scores are exactly equal in fp32 and in double
+    u = ubt()
+    rng = np.random.default_rng(3)
+    B, L, V, k, N = 4, 4, 64, 3, 12
+    x = np.round(rng.standard_normal((B, L, V)) * 2).astype(np.float32)
+    big = np.zeros((B, L - 1, k, k), np.float32)
+    lam = np.zeros(L, np.float32)
+    otree = oracle.draft_tree(x, big, k, N, lam=lam)
+    gtree = u.ubt_draft_tree(torch.from_numpy(x).to(DEV), torch.from_numpy(big).to(DEV), k, N,
+                             lam=torch.from_numpy(lam).to(DEV))
+    torch.cuda.synchronize()
+    compare_draft(tree_to_numpy(gtree), otree, L, k, N)
+
+
+def test_split_entry_points_match_fused_call():
+    u = ubt()
+    cfg = synth.CONFIGS["c2"].replace(V=20000)
+    di = synth.draft_inputs(cfg, 2)
+    ud = synth.to_device(di.unigram_logits, cfg.dtype, DEV)
+    bd = torch.from_numpy(di.bigram_scores).to(DEV)
+    fused = u.ubt_draft_tree(ud, bd, cfg.k, cfg.N)
+    split = u.Tree.empty(cfg.B, cfg.N, cfg.L, cfg.k, DEV)
+    ws = u.workspace(u.ubt_draft_workspace_bytes(cfg.B, cfg.L, cfg.V, cfg.k, cfg.N), DEV)
+    u.ubt_topk_logprob(ud, cfg.k, split.cand_ids, split.cand_logprob, ws)
+    u.ubt_build_tree(bd, split)
+    torch.cuda.synchronize()
+    for name in ("token_ids", "parents", "depths", "position_ids", "cand_rank", "mask", "n_nodes", "cand_ids"):
+        assert torch.equal(getattr(fused, name), getattr(split, name)), name
+    assert torch.equal(fused.scores, split.scores)
+    # the standalone mask builder reproduces mask and position ids from parents/depths
+    off = torch.arange(cfg.B, dtype=torch.int32, device=DEV) * 1000 + 17
+    want_mask = split.mask.clone()
+    split.mask.zero_(); split.position_ids.zero_()
+    u.ubt_build_mask(split, off)
+    torch.cuda.synchronize()
+    assert torch.equal(split.mask, want_mask)
+    want_pos = torch.where(fused.depths >= 0, fused.depths + off[:, None], torch.full_like(fused.depths, -1))
+    assert torch.equal(split.position_ids, want_pos)
+
+
+def test_host_buffer_entry_points():
+    u = ubt()
+    cfg = synth.CONFIGS["c1"].replace(B=3, V=5000, dtype="bf16")
+    di = synth.draft_inputs(cfg, 4)
+    uh = synth.to_device(di.unigram_logits, cfg.dtype, "cpu").pin_memory()
+    bh = torch.from_numpy(di.bigram_scores).pin_memory()
+    tree_h = u.Tree.empty(cfg.B, cfg.N, cfg.L, cfg.k, DEV, pin=True)
+    buf = u.workspace(u.ubt_draft_host_buffer_bytes(cfg.B, cfg.L, cfg.V, cfg.k, cfg.N, 1), DEV)
+    u.ubt_draft_tree_host(uh, bh, cfg.k, cfg.N, tree_h, buf)
+    otree = oracle.draft_tree(di.unigram_logits, di.bigram_scores, cfg.k, cfg.N)
+    g = tree_to_numpy(tree_h)
+    compare_draft(g, otree, cfg.L, cfg.k, cfg.N)
+    z = synth.target_logits(cfg, 4)
+    synth.plant_path(z, cfg.dtype, g.token_ids, g.parents, g.n_nodes, 4)
+    zh = synth.to_device(z, cfg.dtype, "cpu").pin_memory()
+    res = u.VerifyResult.empty(cfg.B, cfg.L, DEV, pin=True)
+    pick = torch.empty((cfg.B, cfg.N), dtype=torch.int32).pin_memory()
+    vbuf = u.workspace(u.ubt_verify_host_buffer_bytes(cfg.B, cfg.L, cfg.N, cfg.V, 1, "greedy"), DEV)
+    u.ubt_verify_tree_host(tree_h, zh, res, vbuf, "greedy", node_pick=pick)
+    compare_verify(res, oracle.verify(g.token_ids, g.parents, g.n_nodes, cfg.L, z, "greedy"), pick)
+
+
+def test_repeat_calls_are_deterministic():
+    u = ubt()
+    cfg = synth.CONFIGS["c3"].replace(B=4)
+    ud, bd, zd = synth.device_inputs(cfg, 3, DEV)
+    a = u.ubt_draft_tree(ud, bd, cfg.k, cfg.N)
+    ra = u.ubt_verify_tree(a, zd, "sample", seed=5)
+    b = u.ubt_draft_tree(ud, bd, cfg.k, cfg.N)
+    rb = u.ubt_verify_tree(b, zd, "sample", seed=5)
+    torch.cuda.synchronize()
+    for name in ("token_ids", "parents", "mask", "scores", "cand_logprob"):
+        assert torch.equal(getattr(a, name), getattr(b, name)), name
+    assert torch.equal(ra.accepted_len, rb.accepted_len) and torch.equal(ra.out_tokens, rb.out_tokens)
