@@ -8,6 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libubt.so")
+CHECKED_LIB = os.path.join(HERE, "libubt_checked.so")   # -DUBT_BOUNDS_CHECK debug build
 SOURCES = ["ubt_api.cu", "ubt_topk.cu", "ubt_tree.cu", "ubt_verify.cu"]
 HEADERS = ["ubt_common.cuh", "ubt_internal.h", os.path.join("..", "..", "include", "ubt.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
@@ -29,15 +30,20 @@ def is_stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every kernel for sm_100a and link the shared library; returns its path."""
-    if not force and not is_stale():
+def build(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    """Compile every kernel for sm_100a and link the shared library; returns its path.
+
+    ``checked=True`` builds ``libubt_checked.so`` with range-checked array views (a debugging aid).
+    """
+    target = CHECKED_LIB if checked else LIB
+    if not checked and not force and not is_stale():
         return LIB
     objs = []
     procs = []
     for s in SOURCES:
-        obj = os.path.join(CSRC, s.replace(".cu", ".o"))
-        cmd = [_nvcc(), *NVCC_FLAGS, "-c", os.path.join(CSRC, s), "-o", obj]
+        obj = os.path.join(CSRC, s.replace(".cu", ".chk.o" if checked else ".o"))
+        cmd = [_nvcc(), *NVCC_FLAGS, *(["-DUBT_BOUNDS_CHECK"] if checked else []), "-c", os.path.join(CSRC, s),
+               "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas=-v")
         procs.append((s, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
@@ -50,12 +56,12 @@ def build(force: bool = False, verbose: bool = False) -> str:
         failed = failed or p.returncode != 0
     if failed:
         raise RuntimeError("nvcc failed building libubt")
-    tmp = LIB + f".{os.getpid()}.tmp"
+    tmp = target + f".{os.getpid()}.tmp"
     subprocess.check_call([_nvcc(), "-shared", "-o", tmp, *objs, "-gencode", "arch=compute_100a,code=sm_100a",
                            "-lcudart"])
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, target)
+    return target
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, checked="--checked" in sys.argv))

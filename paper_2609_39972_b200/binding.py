@@ -60,7 +60,8 @@ _lib = None
 
 
 def lib_path() -> str:
-    return _build.LIB
+    """``libubt.so`` beside this file; UBT_LIB=checked selects the range-checked debug build."""
+    return _build.CHECKED_LIB if os.environ.get("UBT_LIB") == "checked" else _build.LIB
 
 
 def load() -> C.CDLL:

@@ -346,4 +346,19 @@ int ubt_verify_tree_host(const ubt_tree* tree, const void* target_logits, int dt
   return UBT_OK;
 }
 
+#ifdef UBT_BOUNDS_CHECK
+}  // extern "C"
+namespace ubt {
+cudaError_t bounds_report_topk(long long out[4]);
+cudaError_t bounds_report_tree(long long out[4]);
+cudaError_t bounds_report_verify(long long out[4]);
+}  // namespace ubt
+extern "C" {
+// Debug builds only (-DUBT_BOUNDS_CHECK): which = 0 top-k, 1 tree, 2 verify; out = flag, site, index, limit.
+int ubt_debug_bounds_report(int which, long long out[4]) {
+  cudaError_t e = which == 0 ? bounds_report_topk(out) : which == 1 ? bounds_report_tree(out) : bounds_report_verify(out);
+  return e == cudaSuccess ? UBT_OK : UBT_ERR_CUDA;
+}
+#endif
+
 }  // extern "C"

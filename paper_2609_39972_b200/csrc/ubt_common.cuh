@@ -83,6 +83,41 @@ __device__ __forceinline__ uint64_t warp_sum_u64(uint64_t v) {
   return v;
 }
 
+// ---------------------------------------------------------------- checked array views
+// With -DUBT_BOUNDS_CHECK every indexed access through a Span is range-checked; the first violation is
+// recorded (site, index, limit) in a per-translation-unit device word and the access is redirected to
+// element 0, so a wrong index is reported instead of faulting.  Without the flag a Span is a bare pointer.
+#ifdef UBT_BOUNDS_CHECK
+struct BoundsReport { unsigned int flag; int site; long long index; long long limit; };
+static __device__ BoundsReport g_bounds_report;
+static __device__ __noinline__ void bounds_violation(int site, long long i, long long n) {
+  if (atomicCAS(&g_bounds_report.flag, 0u, 1u) == 0u) {
+    g_bounds_report.site = site; g_bounds_report.index = i; g_bounds_report.limit = n;
+  }
+}
+template <typename T> struct Span {
+  T* p; long long n; int site;
+  __host__ __device__ Span() : p(nullptr), n(0), site(0) {}
+  __host__ __device__ Span(T* p_, long long n_, int site_) : p(p_), n(n_), site(site_) {}
+  __device__ __forceinline__ T& operator[](long long i) const {
+    if (i < 0 || i >= n) { bounds_violation(site, i, n); return p[0]; }
+    return p[i];
+  }
+  __device__ __forceinline__ T* ptr(long long i, long long count) const {  // checked sub-range
+    if (i < 0 || i + count > n) { bounds_violation(site, i, n); return p; }
+    return p + i;
+  }
+};
+#else
+template <typename T> struct Span {
+  T* p;
+  __host__ __device__ Span() : p(nullptr) {}
+  __host__ __device__ Span(T* p_, long long, int) : p(p_) {}
+  __device__ __forceinline__ T& operator[](long long i) const { return p[i]; }
+  __device__ __forceinline__ T* ptr(long long i, long long) const { return p + i; }
+};
+#endif
+
 // How a flat range of rows*V elements is cut into per-CTA spans.
 struct SpanPlan {
   int64_t span;  // elements per CTA (multiple of 256)

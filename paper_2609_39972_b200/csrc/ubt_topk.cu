@@ -74,22 +74,24 @@ __device__ __forceinline__ unsigned long long block_max_u64(unsigned long long v
 // the pool is empty and, when k entries exist, taux is the k-th best value (strict from then on:
 // a later element equal to it has a larger column than every kept entry).
 template <typename T>
-__device__ void flush_pool(G1Shared& sh, const int* pool, const T* rowp, int k) {
+__device__ void flush_pool(G1Shared& sh, Span<int> pool, const T* rowp_raw, int V, int k) {
   const int tid = threadIdx.x;
+  const Span<const T> rowp(rowp_raw, V, 303);
+  const Span<unsigned long long> keys(sh.keys, G1_RC + kMaxK, 304), top(sh.top, kMaxK, 305), topn(sh.topn, kMaxK, 306);
   const int M = sh.cnt, nt = sh.ntop, total = M + nt;
   const int newn = total < k ? total : k;
   if (M <= G1_RC) {
     for (int i = tid; i < M; i += G1_T) {
       int col = pool[i];
-      sh.keys[i] = make_key(load_elem(rowp, col), col);
+      keys[i] = make_key(load_elem(rowp.ptr(col, 1), 0), col);
     }
-    for (int i = tid; i < nt; i += G1_T) sh.keys[M + i] = sh.top[i];
+    for (int i = tid; i < nt; i += G1_T) keys[M + i] = top[i];
     __syncthreads();
     for (int i = tid; i < total; i += G1_T) {
-      unsigned long long ki = sh.keys[i];
+      unsigned long long ki = keys[i];
       int rank = 0;
-      for (int j = 0; j < total; ++j) rank += sh.keys[j] > ki;
-      if (rank < k) sh.topn[rank] = ki;
+      for (int j = 0; j < total; ++j) rank += keys[j] > ki;
+      if (rank < k) topn[rank] = ki;
     }
   } else {
     unsigned long long last = ~0ull;
@@ -97,24 +99,24 @@ __device__ void flush_pool(G1Shared& sh, const int* pool, const T* rowp, int k) 
       unsigned long long best = 0;
       for (int i = tid; i < M; i += G1_T) {
         int col = pool[i];
-        unsigned long long key = make_key(load_elem(rowp, col), col);
+        unsigned long long key = make_key(load_elem(rowp.ptr(col, 1), 0), col);
         if (key < last && key > best) best = key;
       }
       for (int i = tid; i < nt; i += G1_T) {
-        unsigned long long key = sh.top[i];
+        unsigned long long key = top[i];
         if (key < last && key > best) best = key;
       }
       best = block_max_u64(best, sh.red64);
-      if (tid == 0) sh.topn[r] = best;
+      if (tid == 0) topn[r] = best;
       last = best;
     }
   }
   __syncthreads();
-  if (tid < newn) sh.top[tid] = sh.topn[tid];
+  if (tid < newn) top[tid] = topn[tid];
   if (tid == 0) {
     sh.ntop = newn;
     sh.cnt = 0;
-    if (newn == k) sh.taux = key_val(sh.topn[k - 1]);
+    if (newn == k) sh.taux = key_val(topn[k - 1]);
   }
   __syncthreads();
 }
@@ -126,8 +128,12 @@ k_lse_topk(const T* __restrict__ logits, int64_t total, int V, int k, SpanPlan p
            int32_t* __restrict__ part_cnt) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   G1Shared& sh = *reinterpret_cast<G1Shared*>(smem_raw);
-  int* pool = reinterpret_cast<int*>(smem_raw + sizeof(G1Shared));
   constexpr int TILE_FRAGS = G1_T * G1_U;
+  const Span<int> pool(reinterpret_cast<int*>(smem_raw + sizeof(G1Shared)), TILE_FRAGS * VEC + G1_SLACK, 301);
+  const long long nslots = (total / V) * plan.smax;
+  const Span<float> g_ms(part_ms, nslots * 2, 311), g_val(part_val, nslots * k, 312);
+  const Span<int32_t> g_idx(part_idx, nslots * k, 313), g_cnt(part_cnt, nslots, 314);
+  const Span<const T> g_logits(logits, total, 302);
 
   const int tid = threadIdx.x, lane = tid & 31;
   const int64_t lo = (int64_t)blockIdx.x * plan.span;
@@ -137,14 +143,15 @@ k_lse_topk(const T* __restrict__ logits, int64_t total, int V, int k, SpanPlan p
     const int64_t row = e / V;
     const int c0 = (int)(e - row * V);
     const int c1 = (int)((int64_t)V - c0 < hi - e ? V : c0 + (hi - e));
-    const T* rowp = logits + row * V;
-    const T* seg = rowp + c0;
+    const T* rowp = g_logits.ptr(row * V, V);
+    const T* seg = g_logits.ptr(row * V + c0, c1 - c0);
     const int nfrag = (c1 - c0) / VEC;  // spans and V are multiples of VEC on this path
     e += c1 - c0;
 
     if (tid == 0) { sh.cnt = 0; sh.ntop = 0; sh.taux = -INFINITY; }
 
-    float m_t = -3.0e38f, s_t = 0.f, negml = 3.0e38f * kLog2e;
+    // Running (max, sum) start at a finite floor so that -inf padding gives exp2(-inf) = 0, never inf - inf.
+    float m_t = -1.0e30f, s_t = 0.f, negml = 1.0e30f * kLog2e;
     RawFrag<T, VEC> cur[G1_U], nxt[G1_U];
 #pragma unroll
     for (int u = 0; u < G1_U; ++u) load_frag<T, VEC>(seg, nfrag, u * G1_T + tid, cur[u]);
@@ -216,10 +223,13 @@ k_lse_topk(const T* __restrict__ logits, int64_t total, int V, int k, SpanPlan p
       }
 #pragma unroll
       for (int u = 0; u < G1_U; ++u) cur[u] = nxt[u];
-      __syncthreads();
-      if (sh.cnt >= 4 * k) flush_pool<T>(sh, pool, rowp, k);  // tighten the threshold early
+      // One barrier that also takes the decision: a warp may not re-read the counter after the barrier,
+      // because faster warps are already appending hits of the next tile.  The last warp to arrive has
+      // seen every append of this tile and counts only grow, so the OR is the decision on the final count.
+      if (__syncthreads_or(*reinterpret_cast<volatile int*>(&sh.cnt) >= 4 * k))
+        flush_pool<T>(sh, pool, rowp, V, k);  // tighten the threshold early
     }
-    flush_pool<T>(sh, pool, rowp, k);
+    flush_pool<T>(sh, pool, rowp, V, k);
 
     // partial (max, sum exp) of the segment
     float mw = m_t;
@@ -240,13 +250,13 @@ k_lse_topk(const T* __restrict__ logits, int64_t total, int V, int k, SpanPlan p
     if (tid == 0) {
       float S = 0.f;
       for (int w = 0; w < G1_T / 32; ++w) S += sh.redf[G1_T / 32 + w];
-      part_ms[slot * 2] = M;
-      part_ms[slot * 2 + 1] = S;
-      part_cnt[slot] = sh.ntop;
+      g_ms[slot * 2] = M;
+      g_ms[slot * 2 + 1] = S;
+      g_cnt[slot] = sh.ntop;
     }
     if (tid < sh.ntop) {
-      part_val[slot * k + tid] = key_val(sh.top[tid]);
-      part_idx[slot * k + tid] = key_idx(sh.top[tid]);
+      g_val[slot * k + tid] = key_val(sh.top[tid]);
+      g_idx[slot * k + tid] = key_idx(sh.top[tid]);
     }
     __syncthreads();
   }
@@ -254,18 +264,23 @@ k_lse_topk(const T* __restrict__ logits, int64_t total, int V, int k, SpanPlan p
 
 // One warp per row: combine the partials of the row's segments.
 __global__ void __launch_bounds__(128)
-k_merge_topk(const float* __restrict__ part_ms, const float* __restrict__ part_val,
-             const int32_t* __restrict__ part_idx, const int32_t* __restrict__ part_cnt, int64_t rows,
-             int V, int k, SpanPlan plan, int32_t* __restrict__ cand_ids, float* __restrict__ cand_lp) {
+k_merge_topk(const float* __restrict__ part_ms_, const float* __restrict__ part_val_,
+             const int32_t* __restrict__ part_idx_, const int32_t* __restrict__ part_cnt_, int64_t rows,
+             int V, int k, SpanPlan plan, int32_t* __restrict__ cand_ids_, float* __restrict__ cand_lp_) {
   const int lane = threadIdx.x & 31;
   const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (row >= rows) return;
+  const long long nslots = rows * plan.smax;
+  const Span<const float> part_ms(part_ms_, nslots * 2, 321), part_val(part_val_, nslots * k, 322);
+  const Span<const int32_t> part_idx(part_idx_, nslots * k, 323), part_cnt(part_cnt_, nslots, 324);
+  const Span<int32_t> cand_ids(cand_ids_, rows * k, 325);
+  const Span<float> cand_lp(cand_lp_, rows * k, 326);
   const int64_t c_first = (row * (int64_t)V) / plan.span;
   const int64_t c_last = ((row + 1) * (int64_t)V - 1) / plan.span;
   const int nseg = (int)(c_last - c_first + 1);
   const int64_t base = row * plan.smax;
 
-  float M = -3.0e38f;
+  float M = -1.0e30f;
   for (int j = lane; j < nseg; j += 32) M = fmaxf(M, part_ms[(base + j) * 2]);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(FULL, M, o));
@@ -373,5 +388,15 @@ cudaError_t launch_merge_topk(int64_t rows, int V, int k, const TopkWorkspace& w
                                             w.plan, cand_ids, cand_lp);
   return cudaGetLastError();
 }
+
+#ifdef UBT_BOUNDS_CHECK
+// Debug builds only: first out-of-range index seen by the kernels of this file (flag, site, index, limit).
+cudaError_t bounds_report_topk(long long out[4]) {
+  BoundsReport r;
+  cudaError_t e = cudaMemcpyFromSymbol(&r, g_bounds_report, sizeof r);
+  out[0] = r.flag; out[1] = r.site; out[2] = r.index; out[3] = r.limit;
+  return e;
+}
+#endif
 
 }  // namespace ubt

@@ -15,25 +15,25 @@ namespace ubt {
 constexpr int G2_T = 256;
 
 struct TreeSmem {
-  float* t;            // [L,k,k]
-  unsigned char* ord;  // [L,k,k]  successor ranks sorted by (t desc, token asc)
-  float* lp;           // [L,k]
-  int* tok;            // [L,k]
-  uint32_t* f_key;     // frontier, <= N entries
-  float* f_score;
-  short* f_parent;     // accepted-node index of the parent, -1 = root
-  unsigned char* f_sib;  // position in the parent's sorted successor list
-  short* nd_parent;    // accepted nodes in pop order, <= N-1
-  unsigned char* nd_depth;
-  unsigned char* nd_rank;
-  float* nd_score;
-  short* nd_slot;
-  short* bkt;          // nodes grouped by depth
-  int* kk;             // per-depth sort keys
-  int* depth_cnt;      // [L+2]
-  int* depth_off;      // [L+2]
-  uint32_t* maskrow;   // [N, mask_words]
-  int* scalars;        // [0] = accepted count
+  Span<float> t;            // [L,k,k]
+  Span<unsigned char> ord;  // [L,k,k]  successor ranks sorted by (t desc, token asc)
+  Span<float> lp;           // [L,k]
+  Span<int> tok;            // [L,k]
+  Span<uint32_t> f_key;     // frontier, <= N entries
+  Span<float> f_score;
+  Span<short> f_parent;     // accepted-node index of the parent, -1 = root
+  Span<unsigned char> f_sib;  // position in the parent's sorted successor list
+  Span<short> nd_parent;    // accepted nodes in pop order, <= N-1
+  Span<unsigned char> nd_depth;
+  Span<unsigned char> nd_rank;
+  Span<float> nd_score;
+  Span<short> nd_slot;
+  Span<short> bkt;          // nodes grouped by depth
+  Span<int> kk;             // per-depth sort keys
+  Span<int> depth_cnt;      // [L+2]
+  Span<int> depth_off;      // [L+2]
+  Span<uint32_t> maskrow;   // [N, mask_words]
+  Span<int> scalars;        // [0] = accepted count
 };
 
 __host__ __device__ inline size_t tree_carve(TreeSmem* s, unsigned char* base, int L, int k, int N) {
@@ -44,8 +44,9 @@ __host__ __device__ inline size_t tree_carve(TreeSmem* s, unsigned char* base, i
     return at;
   };
   const int mw = (N + 31) / 32;
-  size_t o_t = take(sizeof(float) * L * k * k), o_ord = take((size_t)L * k * k);
-  size_t o_lp = take(sizeof(float) * L * k), o_tok = take(sizeof(int) * L * k);
+  const long long lkk = (long long)L * k * k, lk = (long long)L * k;
+  size_t o_t = take(sizeof(float) * lkk), o_ord = take((size_t)lkk);
+  size_t o_lp = take(sizeof(float) * lk), o_tok = take(sizeof(int) * lk);
   size_t o_fk = take(sizeof(uint32_t) * (N + 1)), o_fs = take(sizeof(float) * (N + 1));
   size_t o_fp = take(sizeof(short) * (N + 1)), o_fb = take(N + 1);
   size_t o_np = take(sizeof(short) * N), o_nd = take(N), o_nr = take(N);
@@ -54,13 +55,25 @@ __host__ __device__ inline size_t tree_carve(TreeSmem* s, unsigned char* base, i
   size_t o_dc = take(sizeof(int) * (L + 2)), o_do = take(sizeof(int) * (L + 2));
   size_t o_mk = take(sizeof(uint32_t) * N * mw), o_sc = take(sizeof(int) * 4);
   if (s) {
-    s->t = (float*)(base + o_t); s->ord = base + o_ord; s->lp = (float*)(base + o_lp);
-    s->tok = (int*)(base + o_tok); s->f_key = (uint32_t*)(base + o_fk); s->f_score = (float*)(base + o_fs);
-    s->f_parent = (short*)(base + o_fp); s->f_sib = base + o_fb; s->nd_parent = (short*)(base + o_np);
-    s->nd_depth = base + o_nd; s->nd_rank = base + o_nr; s->nd_score = (float*)(base + o_ns);
-    s->nd_slot = (short*)(base + o_nl); s->bkt = (short*)(base + o_bk); s->kk = (int*)(base + o_kk);
-    s->depth_cnt = (int*)(base + o_dc); s->depth_off = (int*)(base + o_do);
-    s->maskrow = (uint32_t*)(base + o_mk); s->scalars = (int*)(base + o_sc);
+    s->t = Span<float>((float*)(base + o_t), lkk, 101);
+    s->ord = Span<unsigned char>(base + o_ord, lkk, 102);
+    s->lp = Span<float>((float*)(base + o_lp), lk, 103);
+    s->tok = Span<int>((int*)(base + o_tok), lk, 104);
+    s->f_key = Span<uint32_t>((uint32_t*)(base + o_fk), N + 1, 105);
+    s->f_score = Span<float>((float*)(base + o_fs), N + 1, 106);
+    s->f_parent = Span<short>((short*)(base + o_fp), N + 1, 107);
+    s->f_sib = Span<unsigned char>(base + o_fb, N + 1, 108);
+    s->nd_parent = Span<short>((short*)(base + o_np), N, 109);
+    s->nd_depth = Span<unsigned char>(base + o_nd, N, 110);
+    s->nd_rank = Span<unsigned char>(base + o_nr, N, 111);
+    s->nd_score = Span<float>((float*)(base + o_ns), N, 112);
+    s->nd_slot = Span<short>((short*)(base + o_nl), N, 113);
+    s->bkt = Span<short>((short*)(base + o_bk), N, 114);
+    s->kk = Span<int>((int*)(base + o_kk), N, 115);
+    s->depth_cnt = Span<int>((int*)(base + o_dc), L + 2, 116);
+    s->depth_off = Span<int>((int*)(base + o_do), L + 2, 117);
+    s->maskrow = Span<uint32_t>((uint32_t*)(base + o_mk), (long long)N * mw, 118);
+    s->scalars = Span<int>((int*)(base + o_sc), 4, 119);
   }
   return off;
 }
@@ -77,18 +90,25 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   tree_carve(&s, smem_raw, L, k, N);
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
   const int kk2 = k * k, mw = (N + 31) / 32, budget = N - 1;
+  const long long nB = gridDim.x;
+  const Span<const float> g_lp(out.cand_logprob, nB * L * k, 201), g_big(bigram, nB * (L - 1) * kk2, 203);
+  const Span<const int32_t> g_ids(out.cand_ids, nB * L * k, 202);
+  const Span<int32_t> g_tok(out.token_ids, nB * N, 211), g_par(out.parents, nB * N, 212), g_dep(out.depths, nB * N, 213);
+  const Span<int32_t> g_rk(out.cand_rank, nB * N, 214), g_pos(out.position_ids, nB * N, 215), g_nn(out.n_nodes, nB, 216);
+  const Span<float> g_sc(out.scores, nB * N, 217);
+  const Span<uint32_t> g_mask(out.mask, nB * N * mw, 218);
 
   // ---- stage candidates and raw selector scores
   for (int i = tid; i < L * k; i += G2_T) {
-    s.lp[i] = out.cand_logprob[(int64_t)b * L * k + i];
-    s.tok[i] = out.cand_ids[(int64_t)b * L * k + i];
+    s.lp[i] = g_lp[(int64_t)b * L * k + i];
+    s.tok[i] = g_ids[(int64_t)b * L * k + i];
   }
   for (int i = tid; i < L * kk2; i += G2_T) {
     float d = 0.f;
     if (i < kk2) {
       if (i < k && anchor_bigram) d = anchor_bigram[(int64_t)b * k + i];  // only predecessor row 0 exists
     } else {
-      d = bigram[(int64_t)b * (L - 1) * kk2 + (i - kk2)];
+      d = g_big[(int64_t)b * (L - 1) * kk2 + (i - kk2)];
     }
     s.t[i] = d;
   }
@@ -101,7 +121,7 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   for (int r = tid; r < nrows; r += G2_T) {
     const int i = r == 0 ? 0 : 1 + (r - 1) / k;
     const int ra = r == 0 ? 0 : (r - 1) % k;
-    float* row = s.t + ((size_t)i * k + ra) * k;
+    float* row = s.t.ptr(((long long)i * k + ra) * k, k);
     const float al = alpha ? alpha[i] : 1.f, la = lambda ? lambda[i] : 1.f;
     float mx = -INFINITY;
     for (int rb = 0; rb < k; ++rb) {
@@ -120,11 +140,15 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
     const int r = q / k, rb = q - r * k;
     const int i = r == 0 ? 0 : 1 + (r - 1) / k;
     const int ra = r == 0 ? 0 : (r - 1) % k;
-    const float* row = s.t + ((size_t)i * k + ra) * k;
-    const int* tk = s.tok + i * k;
-    const float v = row[rb];
+    const float* row = s.t.ptr(((long long)i * k + ra) * k, k);
+    const int* tk = s.tok.ptr((long long)i * k, k);
+    // integer keys and a final index tie-break keep this a permutation whatever the values are (even NaN)
+    const uint32_t kv = f2key(row[rb]);
     int rank = 0;
-    for (int j = 0; j < k; ++j) rank += (row[j] > v) || (row[j] == v && tk[j] < tk[rb]);
+    for (int j = 0; j < k; ++j) {
+      const uint32_t kj = f2key(row[j]);
+      rank += (kj > kv) || (kj == kv && (tk[j] < tk[rb] || (tk[j] == tk[rb] && j < rb)));
+    }
     s.ord[((size_t)i * k + ra) * k + rank] = (unsigned char)rb;
   }
   __syncthreads();
@@ -258,18 +282,18 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   const int64_t o = (int64_t)b * N;
   const int poff = pos_offset ? pos_offset[b] : 0;
   if (tid == 0) {
-    out.token_ids[o] = anchor_tokens ? anchor_tokens[b] : -1;
-    out.parents[o] = -1; out.depths[o] = 0; out.cand_rank[o] = -1; out.position_ids[o] = poff;
-    out.scores[o] = 0.f; out.n_nodes[b] = n_acc + 1;
+    g_tok[o] = anchor_tokens ? anchor_tokens[b] : -1;
+    g_par[o] = -1; g_dep[o] = 0; g_rk[o] = -1; g_pos[o] = poff;
+    g_sc[o] = 0.f; g_nn[b] = n_acc + 1;
     s.maskrow[0] = 1u;
   }
   if (tid < n_acc) {
     const int sl = s.nd_slot[tid], p = s.nd_parent[tid], d = s.nd_depth[tid], r = s.nd_rank[tid];
-    out.token_ids[o + sl] = s.tok[(d - 1) * k + r];
-    out.parents[o + sl] = p < 0 ? 0 : s.nd_slot[p];
-    out.depths[o + sl] = d; out.cand_rank[o + sl] = r; out.position_ids[o + sl] = poff + d;
-    out.scores[o + sl] = s.nd_score[tid];
-    uint32_t* row = s.maskrow + (size_t)sl * mw;
+    g_tok[o + sl] = s.tok[(d - 1) * k + r];
+    g_par[o + sl] = p < 0 ? 0 : s.nd_slot[p];
+    g_dep[o + sl] = d; g_rk[o + sl] = r; g_pos[o + sl] = poff + d;
+    g_sc[o + sl] = s.nd_score[tid];
+    uint32_t* row = s.maskrow.ptr((long long)sl * mw, mw);
     row[0] |= 1u;  // the root
     for (int a = tid; a >= 0; a = s.nd_parent[a]) {
       const int as = s.nd_slot[a];
@@ -277,11 +301,11 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
     }
   }
   for (int i = n_acc + 1 + tid; i < N; i += G2_T) {
-    out.token_ids[o + i] = -1; out.parents[o + i] = -1; out.depths[o + i] = -1;
-    out.cand_rank[o + i] = -1; out.position_ids[o + i] = -1; out.scores[o + i] = -INFINITY;
+    g_tok[o + i] = -1; g_par[o + i] = -1; g_dep[o + i] = -1;
+    g_rk[o + i] = -1; g_pos[o + i] = -1; g_sc[o + i] = -INFINITY;
   }
   __syncthreads();
-  for (int i = tid; i < N * mw; i += G2_T) out.mask[(int64_t)b * N * mw + i] = s.maskrow[i];
+  for (int i = tid; i < N * mw; i += G2_T) g_mask[(int64_t)b * N * mw + i] = s.maskrow[i];
 }
 
 // Step a3b alone: one CTA per sequence, one thread per slot.
@@ -330,5 +354,15 @@ cudaError_t launch_build_mask(const ubt_tree& tree, const int32_t* pos_offset, c
   k_build_mask<<<tree.B, G2_T, smem, st>>>(tree, pos_offset);
   return cudaGetLastError();
 }
+
+#ifdef UBT_BOUNDS_CHECK
+// Debug builds only: first out-of-range index seen by the kernels of this file (flag, site, index, limit).
+cudaError_t bounds_report_tree(long long out[4]) {
+  BoundsReport r;
+  cudaError_t e = cudaMemcpyFromSymbol(&r, g_bounds_report, sizeof r);
+  out[0] = r.flag; out[1] = r.site; out[2] = r.index; out[3] = r.limit;
+  return e;
+}
+#endif
 
 }  // namespace ubt

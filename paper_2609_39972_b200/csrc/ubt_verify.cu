@@ -391,4 +391,14 @@ cudaError_t launch_walk(const ubt_tree& tree, int mode, const VerifyWorkspace& w
   return cudaGetLastError();
 }
 
+#ifdef UBT_BOUNDS_CHECK
+// Debug builds only: first out-of-range index seen by the kernels of this file (flag, site, index, limit).
+cudaError_t bounds_report_verify(long long out[4]) {
+  BoundsReport r;
+  cudaError_t e = cudaMemcpyFromSymbol(&r, g_bounds_report, sizeof r);
+  out[0] = r.flag; out[1] = r.site; out[2] = r.index; out[3] = r.limit;
+  return e;
+}
+#endif
+
 }  // namespace ubt

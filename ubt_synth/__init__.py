@@ -184,7 +184,7 @@ def target_logits(cfg: Config, seed: int = 0) -> np.ndarray:
 
 def _set(z: np.ndarray, dtype: str, idx, value: np.ndarray) -> None:
     if dtype == "bf16":
-        z[idx] = f32_to_bf16_bits(np.asarray(value, np.float32))
+        z[idx] = f32_to_bf16_bits(np.asarray(value, np.float32).reshape(1))[0]
     else:
         z[idx] = np.asarray(value, np.float32)
 
