@@ -40,7 +40,8 @@ typedef enum {
   UBT_ERR_INVALID_ARG = 1, /* NULL / misaligned pointer, size out of range, k > V, zeta > 0 ... */
   UBT_ERR_UNSUPPORTED = 2, /* valid request beyond the compiled limits above */
   UBT_ERR_WORKSPACE = 3,   /* workspace NULL or smaller than ubt_*_workspace_bytes() */
-  UBT_ERR_CUDA = 4         /* a CUDA call or kernel launch failed */
+  UBT_ERR_CUDA = 4,        /* a CUDA call or kernel launch failed */
+  UBT_ERR_STATIC_SCRATCH = 5 /* request larger than the built-in scratch of ubt_verify_tree_static */
 } ubt_status;
 
 typedef enum { UBT_F32 = 0, UBT_BF16 = 1 } ubt_dtype;
@@ -167,6 +168,31 @@ int ubt_draft_tree_host(const void *unigram_logits, int dtype, const float *bigr
 int ubt_verify_tree_host(const ubt_tree *tree, const void *target_logits, int dtype, int V, int mode,
                          const ubt_verify_opts *opts, ubt_verify_result *out, void *device_buffer,
                          size_t device_buffer_bytes, void *cuda_stream);
+
+/*
+ * Greedy verification for callers that cannot allocate device memory (the paper has no counterpart: this
+ * is a packaging variant of ubt_verify_tree in UBT_VERIFY_GREEDY mode).  Such callers are, for example,
+ * code running after a memory pool has handed out all of the device, a plugin that only ever receives its
+ * input and output buffers, or a latency-critical loop that must not hit cudaMalloc's implicit
+ * synchronisation.  The call takes no workspace: its scratch (one 8-byte key per row and span) lives in a
+ * 512 KiB array compiled into the library, which every GPU that loads the library holds until the process
+ * ends.  It allocates nothing, frees nothing and calls no allocating routine.
+ *
+ * Same arguments, outputs and results as ubt_verify_tree(tree, target_logits, dtype, V, GREEDY, ...);
+ * node_pick ([B,N] device, may be NULL) receives the pick of every row.
+ * Limit: B*N*spans_per_row <= ubt_verify_static_capacity() keys (65,536), where spans_per_row =
+ * ceil(V/span)+1 and span = max(65,536, B*N*V / (2 * SM count)) elements: 2 for large batches (32,768
+ * keys for B*N = 16,384 rows), 4 for a single 64-slot tree over V = 151,936.  A larger request returns
+ * UBT_ERR_STATIC_SCRATCH before anything is launched.
+ * The first call on a device looks up the array's device address (once per device, with that device
+ * current); make that first call outside any stream capture.
+ * All calls on a device share the one array and it keeps the previous call's contents (every key that is
+ * read is written first, so nothing needs clearing): two calls whose kernels overlap on the GPU -- different
+ * streams, or different host threads -- race on it and must be serialised by the caller.
+ */
+int ubt_verify_tree_static(const ubt_tree *tree, const void *target_logits, int dtype, int V,
+                           int32_t *node_pick, ubt_verify_result *out, void *cuda_stream);
+long long ubt_verify_static_capacity(void);
 
 #ifdef __cplusplus
 }

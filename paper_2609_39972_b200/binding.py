@@ -54,7 +54,7 @@ class _VerifyResult(C.Structure):
 EXPORTS = ["ubt_version", "ubt_status_string", "ubt_draft_workspace_bytes", "ubt_verify_workspace_bytes",
            "ubt_topk_logprob", "ubt_build_tree", "ubt_build_mask", "ubt_draft_tree", "ubt_verify_tree",
            "ubt_draft_host_buffer_bytes", "ubt_verify_host_buffer_bytes", "ubt_draft_tree_host",
-           "ubt_verify_tree_host"]
+           "ubt_verify_tree_host", "ubt_verify_tree_static", "ubt_verify_static_capacity"]
 
 _lib = None
 
@@ -92,6 +92,8 @@ def load() -> C.CDLL:
                                  C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
     L.ubt_verify_tree.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
                                   C.c_void_p, C.c_size_t, C.c_void_p]
+    L.ubt_verify_tree_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.ubt_verify_static_capacity.restype = C.c_longlong
     L.ubt_draft_tree_host.argtypes = L.ubt_draft_tree.argtypes
     L.ubt_verify_tree_host.argtypes = L.ubt_verify_tree.argtypes
     _lib = L
@@ -305,5 +307,30 @@ def ubt_verify_tree_host(tree: Tree, target_logits: torch.Tensor, result: Verify
     _check(load().ubt_verify_tree_host(C.byref(t), _ptr(target_logits), _dtype_code(target_logits), V,
                                        _MODES.get(mode, mode), C.byref(o), C.byref(r), _ptr(device_buffer),
                                        device_buffer.numel(), _stream(stream)), "ubt_verify_tree_host")
+    result.node_pick = node_pick
+    return result
+
+
+def ubt_verify_static_capacity() -> int:
+    """Keys (one per target row and span) the built-in scratch of ``ubt_verify_tree_static`` holds."""
+    return int(load().ubt_verify_static_capacity())
+
+
+def ubt_verify_tree_static(tree: Tree, target_logits: torch.Tensor, node_pick: Optional[torch.Tensor] = None,
+                           result: Optional[VerifyResult] = None, stream=None) -> VerifyResult:
+    """Greedy ``ubt_verify_tree`` for callers that cannot allocate device memory.
+
+    The library call takes no workspace and allocates nothing: its scratch is a fixed 512 KiB array inside
+    ``libubt.so``.  Pass ``result`` (and ``node_pick``) preallocated if this wrapper, too, must not allocate.
+    Calls share that one array, so calls that may overlap on the GPU have to be serialised by the caller.
+    """
+    _need(target_logits, "target_logits")
+    B, N, V = target_logits.shape
+    if result is None:
+        result = VerifyResult.empty(B, tree.L, target_logits.device)
+    t = tree.c_struct()
+    r = result.c_struct()
+    _check(load().ubt_verify_tree_static(C.byref(t), _ptr(target_logits), _dtype_code(target_logits), V,
+                                         _ptr(node_pick), C.byref(r), _stream(stream)), "ubt_verify_tree_static")
     result.node_pick = node_pick
     return result

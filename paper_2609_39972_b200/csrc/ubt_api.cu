@@ -65,6 +65,7 @@ const char* ubt_status_string(int status) {
     case UBT_ERR_UNSUPPORTED: return "shape beyond the compiled limits";
     case UBT_ERR_WORKSPACE: return "workspace missing or too small";
     case UBT_ERR_CUDA: return "CUDA call or launch failed";
+    case UBT_ERR_STATIC_SCRATCH: return "request exceeds the built-in scratch of ubt_verify_tree_static";
     default: return "unknown status";
   }
 }
