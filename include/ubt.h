@@ -16,7 +16,8 @@
  *   - Inputs are read-only.  Outputs and the workspace are overwritten; workspace content on entry
  *     is irrelevant.
  *   - Argument errors are detected on the host and returned before anything is launched.
- *     A failed launch returns UBT_ERR_CUDA.  Nothing in the library traps or spins on the device.
+ *     A failed launch returns UBT_ERR_CUDA.  Nothing in the library traps; the only device-side waits
+ *     (for a bulk copy to land) are bounded and counted by ubt_debug_ring_timeouts().
  *   - Logits must be free of NaN; each row must hold at least k entries greater than -inf.
  *
  * Sizes: B sequences, L draft positions (the paper's gamma), V vocabulary, k candidates per position
@@ -96,6 +97,10 @@ typedef struct ubt_verify_result {
 
 int ubt_version(void);
 const char *ubt_status_string(int status);
+/* Diagnostics: how many bounded device-side waits (on a bulk copy's completion) gave up since the library
+ * was loaded on the current device.  0 in a healthy process; -1 if the counter cannot be read.  Results of a
+ * call during which a wait gave up are undefined (but the call returned and nothing hung). */
+long long ubt_debug_ring_timeouts(void);
 
 /* Bytes of device workspace the calls below need for the given shape (0 on invalid shapes). */
 size_t ubt_draft_workspace_bytes(int B, int L, int V, int k, int node_budget);

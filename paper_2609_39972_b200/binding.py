@@ -51,7 +51,7 @@ class _VerifyResult(C.Structure):
                 ("out_tokens", C.c_void_p)]
 
 
-EXPORTS = ["ubt_version", "ubt_status_string", "ubt_draft_workspace_bytes", "ubt_verify_workspace_bytes",
+EXPORTS = ["ubt_version", "ubt_status_string", "ubt_debug_ring_timeouts", "ubt_draft_workspace_bytes", "ubt_verify_workspace_bytes",
            "ubt_topk_logprob", "ubt_build_tree", "ubt_build_mask", "ubt_draft_tree", "ubt_verify_tree",
            "ubt_draft_host_buffer_bytes", "ubt_verify_host_buffer_bytes", "ubt_draft_tree_host",
            "ubt_verify_tree_host", "ubt_verify_tree_static", "ubt_verify_static_capacity"]
@@ -94,6 +94,7 @@ def load() -> C.CDLL:
                                   C.c_void_p, C.c_size_t, C.c_void_p]
     L.ubt_verify_tree_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
     L.ubt_verify_static_capacity.restype = C.c_longlong
+    L.ubt_debug_ring_timeouts.restype = C.c_longlong
     L.ubt_draft_tree_host.argtypes = L.ubt_draft_tree.argtypes
     L.ubt_verify_tree_host.argtypes = L.ubt_verify_tree.argtypes
     _lib = L
@@ -334,3 +335,8 @@ def ubt_verify_tree_static(tree: Tree, target_logits: torch.Tensor, node_pick: O
                                          _ptr(node_pick), C.byref(r), _stream(stream)), "ubt_verify_tree_static")
     result.node_pick = node_pick
     return result
+
+
+def ubt_debug_ring_timeouts() -> int:
+    """Bounded device-side waits that gave up since the library was loaded (0 in a healthy process)."""
+    return int(load().ubt_debug_ring_timeouts())

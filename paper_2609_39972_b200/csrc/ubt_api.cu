@@ -347,6 +347,18 @@ int ubt_verify_tree_host(const ubt_tree* tree, const void* target_logits, int dt
   return UBT_OK;
 }
 
+}  // extern "C"
+namespace ubt {
+cudaError_t ring_timeouts_verify(unsigned int* out);
+cudaError_t ring_timeouts_topk(unsigned int* out);
+}  // namespace ubt
+extern "C" {
+long long ubt_debug_ring_timeouts(void) {
+  unsigned int a = 0, b = 0;
+  if (ring_timeouts_verify(&a) != cudaSuccess || ring_timeouts_topk(&b) != cudaSuccess) return -1;
+  return (long long)a + b;
+}
+
 #ifdef UBT_BOUNDS_CHECK
 }  // extern "C"
 namespace ubt {

@@ -11,6 +11,7 @@
 // is prefetched into registers before the current one is processed, so the one barrier per tile
 // does not drain the loads in flight.
 #include "ubt_internal.h"
+#include "ubt_ring.cuh"
 
 namespace ubt {
 
@@ -388,6 +389,9 @@ cudaError_t launch_merge_topk(int64_t rows, int V, int k, const TopkWorkspace& w
                                             w.plan, cand_ids, cand_lp);
   return cudaGetLastError();
 }
+
+// Number of bounded waits that gave up in this file's kernels (0 in a healthy run).
+cudaError_t ring_timeouts_topk(unsigned int* out) { return cudaMemcpyFromSymbol(out, g_ring_timeouts, sizeof *out); }
 
 #ifdef UBT_BOUNDS_CHECK
 // Debug builds only: first out-of-range index seen by the kernels of this file (flag, site, index, limit).

@@ -28,16 +28,21 @@ def pytest_collection_modifyitems(config, items):
 
 @pytest.fixture(autouse=True)
 def _bounds_report(request):
-    """With UBT_LIB=checked (the range-checked debug build) fail a GPU test that indexed out of range."""
+    """Fail a GPU test during which a device-side wait gave up or (UBT_LIB=checked) an index was out of range."""
     yield
-    if os.environ.get("UBT_LIB") != "checked" or "gpu" not in request.keywords:
+    if "gpu" not in request.keywords:
         return
     import ctypes as C
 
     import torch
 
     import paper_2609_39972_b200 as u
+    if not torch.cuda.is_available():
+        return
     torch.cuda.synchronize()
+    assert u.ubt_debug_ring_timeouts() == 0, "a bounded device-side wait gave up"
+    if os.environ.get("UBT_LIB") != "checked":
+        return
     lib = u.load()
     for which, name in enumerate(("top-k", "tree", "verify")):
         out = (C.c_longlong * 4)()
