@@ -74,7 +74,7 @@ __device__ __forceinline__ unsigned long long block_max_u64(unsigned long long v
 // Rank the pool (and the carried top list) exactly; afterwards top[0..ntop) is sorted best first,
 // the pool is empty and, when k entries exist, taux is the k-th best value (strict from then on:
 // a later element equal to it has a larger column than every kept entry).
-template <typename T>
+template <typename T, int THREADS>
 __device__ void flush_pool(G1Shared& sh, Span<int> pool, const T* rowp_raw, int V, int k) {
   const int tid = threadIdx.x;
   const Span<const T> rowp(rowp_raw, V, 303);
@@ -82,13 +82,13 @@ __device__ void flush_pool(G1Shared& sh, Span<int> pool, const T* rowp_raw, int 
   const int M = sh.cnt, nt = sh.ntop, total = M + nt;
   const int newn = total < k ? total : k;
   if (M <= G1_RC) {
-    for (int i = tid; i < M; i += G1_T) {
+    for (int i = tid; i < M; i += THREADS) {
       int col = pool[i];
       keys[i] = make_key(load_elem(rowp.ptr(col, 1), 0), col);
     }
-    for (int i = tid; i < nt; i += G1_T) keys[M + i] = top[i];
+    for (int i = tid; i < nt; i += THREADS) keys[M + i] = top[i];
     __syncthreads();
-    for (int i = tid; i < total; i += G1_T) {
+    for (int i = tid; i < total; i += THREADS) {
       unsigned long long ki = keys[i];
       int rank = 0;
       for (int j = 0; j < total; ++j) rank += keys[j] > ki;
@@ -98,12 +98,12 @@ __device__ void flush_pool(G1Shared& sh, Span<int> pool, const T* rowp_raw, int 
     unsigned long long last = ~0ull;
     for (int r = 0; r < newn; ++r) {
       unsigned long long best = 0;
-      for (int i = tid; i < M; i += G1_T) {
+      for (int i = tid; i < M; i += THREADS) {
         int col = pool[i];
         unsigned long long key = make_key(load_elem(rowp.ptr(col, 1), 0), col);
         if (key < last && key > best) best = key;
       }
-      for (int i = tid; i < nt; i += G1_T) {
+      for (int i = tid; i < nt; i += THREADS) {
         unsigned long long key = top[i];
         if (key < last && key > best) best = key;
       }
@@ -127,7 +127,7 @@ __global__ void __launch_bounds__(G1_T, VEC == 1 ? 1 : 2)
 k_lse_topk(const T* __restrict__ logits, int64_t total, int V, int k, SpanPlan plan,
            float* __restrict__ part_ms, float* __restrict__ part_val, int32_t* __restrict__ part_idx,
            int32_t* __restrict__ part_cnt) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+  extern __shared__ __align__(128) unsigned char smem_raw[];
   G1Shared& sh = *reinterpret_cast<G1Shared*>(smem_raw);
   constexpr int TILE_FRAGS = G1_T * G1_U;
   const Span<int> pool(reinterpret_cast<int*>(smem_raw + sizeof(G1Shared)), TILE_FRAGS * VEC + G1_SLACK, 301);
@@ -228,9 +228,9 @@ k_lse_topk(const T* __restrict__ logits, int64_t total, int V, int k, SpanPlan p
       // because faster warps are already appending hits of the next tile.  The last warp to arrive has
       // seen every append of this tile and counts only grow, so the OR is the decision on the final count.
       if (__syncthreads_or(*reinterpret_cast<volatile int*>(&sh.cnt) >= 4 * k))
-        flush_pool<T>(sh, pool, rowp, V, k);  // tighten the threshold early
+        flush_pool<T, G1_T>(sh, pool, rowp, V, k);  // tighten the threshold early
     }
-    flush_pool<T>(sh, pool, rowp, V, k);
+    flush_pool<T, G1_T>(sh, pool, rowp, V, k);
 
     // partial (max, sum exp) of the segment
     float mw = m_t;
@@ -261,6 +261,195 @@ k_lse_topk(const T* __restrict__ logits, int64_t total, int V, int k, SpanPlan p
     }
     __syncthreads();
   }
+}
+
+// ------------------------------------------------------------------------------- ring-fed version
+// Same algorithm with the logits arriving through the bulk-copy ring (ubt_ring.cuh), two CTAs per SM so
+// that one CTA's barriers (threshold bisection, pool ranking) overlap the other's streaming.
+//
+// Log-sum-exp without a running maximum in the common path: every thread fixes a reference ref >= tau0 (the
+// bisected bound, which the exclusive threshold taux never falls below) and accumulates 2^((x-ref)*log2 e).
+// An element <= taux cannot overflow that; an element > taux takes the rare hit path anyway, where the
+// thread moves its reference up if the element is more than 60 above it.
+constexpr int G1R_T = 256, G1R_STAGES = 4, G1R_STAGE_BYTES = 16384, G1R_CTAS = 2;
+
+template <typename T>
+__global__ void __launch_bounds__(G1R_T, G1R_CTAS)
+k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanPlan plan,
+                float* __restrict__ part_ms, float* __restrict__ part_val, int32_t* __restrict__ part_idx,
+                int32_t* __restrict__ part_cnt) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  constexpr int VEC = 16 / (int)sizeof(T);
+  constexpr int STAGE_ELEMS = G1R_STAGE_BYTES / (int)sizeof(T);
+  constexpr int RING_BYTES = G1R_STAGES * G1R_STAGE_BYTES;
+  constexpr int NW = G1R_T / 32;
+  unsigned char* ring = smem_raw;
+  G1Shared& sh = *reinterpret_cast<G1Shared*>(smem_raw + RING_BYTES);
+  const Span<int> pool(reinterpret_cast<int*>(smem_raw + RING_BYTES + sizeof(G1Shared)), STAGE_ELEMS + G1_SLACK, 331);
+  __shared__ uint64_t full[G1R_STAGES];
+  __shared__ int s_fail;
+
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int64_t lo = (int64_t)blockIdx.x * plan.span;
+  const int64_t hi = lo + plan.span < total ? lo + plan.span : total;
+  if (lo >= hi) return;
+  const long long nslots = (total / V) * plan.smax;
+  const Span<float> g_ms(part_ms, nslots * 2, 341), g_val(part_val, nslots * k, 342);
+  const Span<int32_t> g_idx(part_idx, nslots * k, 343), g_cnt(part_cnt, nslots, 344);
+
+  if (tid == 0) {
+    for (int s = 0; s < G1R_STAGES; ++s) mbar_init(&full[s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    s_fail = 0;
+  }
+  __syncthreads();
+  RingProducer<T, G1R_STAGES, G1R_STAGE_BYTES> prod;
+  if (tid == 0) {
+    prod.init(lo, hi, V);
+    for (int i = 0; i < G1R_STAGES - 1; ++i) prod.issue_one(logits, ring, full);
+  }
+  RingPos<G1R_STAGES> rp;
+  rp.init();
+  int consumed = 0;
+  bool failed = false;
+
+  for (int64_t pos = lo; pos < hi && !failed;) {
+    Segment sg;
+    sg.at(pos, hi, V);
+    const T* rowp = logits + sg.row * V;
+    if (tid == 0) { sh.cnt = 0; sh.ntop = 0; sh.taux = -INFINITY; }
+    float ref = -1.0e30f, negref = 1.0e30f * kLog2e, s_t = 0.f;  // ref = -1e30: not fixed yet
+
+    for (int c = 0; c < sg.len; c += STAGE_ELEMS) {
+      const int l = sg.len - c < STAGE_ELEMS ? sg.len - c : STAGE_ELEMS;
+      if (*reinterpret_cast<volatile int*>(&s_fail)) { failed = true; break; }
+      if (tid == 0) prod.issue_one(logits, ring, full);
+      const bool ok = mbar_wait(&full[rp.stage], rp.parity);
+      if (!ok) s_fail = 1;
+      const uint4* stage = reinterpret_cast<const uint4*>(ring + (size_t)rp.stage * G1R_STAGE_BYTES);
+      const int nfrag = l / VEC;
+      const int nround = (nfrag + G1R_T - 1) / G1R_T;
+
+      if (c == 0) {
+        // Bound for the k-th largest element: bisect the top 16 key bits of the per-thread maxima of the
+        // first chunk with CTA-wide counts; the result never exceeds the k-th largest maximum.
+        float tmax = -INFINITY;
+        bool has = false;
+        if (ok) {
+          for (int r = 0; r < nround; ++r) {
+            const int f = r * G1R_T + tid;
+            if (f < nfrag) {
+              Frag<T> x;
+              x.unpack(stage[f]);
+#pragma unroll
+              for (int j = 0; j < VEC; ++j) tmax = fmaxf(tmax, x.x[j]);
+              has = true;
+            }
+          }
+        }
+        const uint32_t mykey = has ? f2key(tmax) : 0u;
+        uint32_t lob = 0;
+        for (int bit = 31; bit >= 16; --bit) {
+          const uint32_t cand = lob | (1u << bit);
+          if (__syncthreads_count(mykey >= cand) >= k) lob = cand;
+        }
+        float tau0 = -INFINITY;
+        if (lob != 0u) {
+          uint32_t below = lob - 1;
+          if (below == 0x7fffffffu) below = 0x7ffffffeu;  // skip -0: it equals +0
+          const float t = key2f(below), t0 = key2f(lob);
+          if (t == t && t0 == t0) {
+            tau0 = t0;
+            if (tid == 0) sh.taux = t;
+          }
+        }
+        const float r0 = fmaxf(tau0, has ? tmax : -INFINITY);
+        if (r0 > -1.0e29f && r0 < 1.0e30f) { ref = r0; negref = -r0 * kLog2e; }
+        __syncthreads();
+      }
+
+      const float taux = sh.taux;
+      if (ok) {
+        for (int r = 0; r < nround; ++r) {  // warp-uniform trip count: the votes need every lane
+          const int f = r * G1R_T + tid;
+          float x[VEC];
+          if (f < nfrag) {
+            Frag<T> fr;
+            fr.unpack(stage[f]);
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) x[j] = fr.x[j];
+          } else {
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) x[j] = -INFINITY;
+          }
+          float vmax = x[0];
+#pragma unroll
+          for (int j = 1; j < VEC; ++j) vmax = fmaxf(vmax, x[j]);
+          if (__any_sync(FULL, vmax > taux)) {
+            if (vmax > ref + 60.f || (ref < -1.0e29f && vmax > -INFINITY)) {  // move the reference up
+              s_t *= ex2_approx(fmaf(ref, kLog2e, -vmax * kLog2e));
+              ref = vmax;
+              negref = -vmax * kLog2e;
+            }
+            const int col0 = sg.col0 + c + f * VEC;
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) {
+              const bool hit = x[j] > taux;
+              const unsigned mask = __ballot_sync(FULL, hit);
+              if (mask) {
+                const int leader = __ffs(mask) - 1;
+                int at = 0;
+                if (lane == leader) at = atomicAdd(&sh.cnt, __popc(mask));
+                at = __shfl_sync(FULL, at, leader);
+                if (hit) pool[at + __popc(mask & ((1u << lane) - 1))] = col0 + j;
+              }
+            }
+          }
+#pragma unroll
+          for (int j = 0; j < VEC; ++j) s_t += ex2_approx(fmaf(x[j], kLog2e, negref));
+        }
+      }
+      // One barrier frees the stage and takes the flush decision on the final hit count (see the comment
+      // in k_lse_topk); a failed wait skips the flush and is seen by everybody at the next chunk.
+      const bool want = *reinterpret_cast<volatile int*>(&sh.cnt) >= 4 * k;
+      if (__syncthreads_or(want)) flush_pool<T, G1R_T>(sh, pool, rowp, V, k);
+      rp.next();
+      ++consumed;
+    }
+    if (failed) break;
+    flush_pool<T, G1R_T>(sh, pool, rowp, V, k);
+
+    // partial (max, sum exp) of the segment from the per-thread (reference, sum) pairs
+    float mw = ref;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mw = fmaxf(mw, __shfl_xor_sync(FULL, mw, o));
+    if (lane == 0) sh.redf[tid >> 5] = mw;
+    __syncthreads();
+    float M = sh.redf[0];
+    for (int w = 1; w < NW; ++w) M = fmaxf(M, sh.redf[w]);
+    float sw = s_t * ex2_approx((ref - M) * kLog2e);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sw += __shfl_xor_sync(FULL, sw, o);
+    if (lane == 0) sh.redf[G1_T / 32 + (tid >> 5)] = sw;
+    __syncthreads();
+    const int64_t c_first = (sg.row * (int64_t)V) / plan.span;
+    const int64_t slot = sg.row * plan.smax + ((int64_t)blockIdx.x - c_first);
+    if (tid == 0) {
+      float S = 0.f;
+      for (int w = 0; w < NW; ++w) S += sh.redf[G1_T / 32 + w];
+      g_ms[slot * 2] = M;
+      g_ms[slot * 2 + 1] = S;
+      g_cnt[slot] = sh.ntop;
+    }
+    if (tid < sh.ntop) {
+      g_val[slot * k + tid] = key_val(sh.top[tid]);
+      g_idx[slot * k + tid] = key_idx(sh.top[tid]);
+    }
+    __syncthreads();
+    pos += sg.len;
+  }
+  __syncthreads();
+  if (tid == 0 && *reinterpret_cast<volatile int*>(&s_fail)) prod.drain(consumed > 0 ? consumed - 1 : 0, full);
 }
 
 // One warp per row: combine the partials of the row's segments.
@@ -371,13 +560,31 @@ static cudaError_t launch_lse_topk_t(const void* logits, int64_t rows, int V, in
   return cudaGetLastError();
 }
 
+template <typename T>
+static cudaError_t launch_lse_topk_ring_t(const void* logits, int64_t rows, int V, int k, const TopkWorkspace& w,
+                                          cudaStream_t st) {
+  constexpr int kStageElems = G1R_STAGE_BYTES / (int)sizeof(T);
+  const size_t smem = (size_t)G1R_STAGES * G1R_STAGE_BYTES + sizeof(G1Shared) + sizeof(int) * (size_t)(kStageElems + G1_SLACK);
+  auto kern = k_lse_topk_ring<T>;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  kern<<<w.plan.grid, G1R_T, smem, st>>>(static_cast<const T*>(logits), rows * (int64_t)V, V, k, w.plan, w.part_ms,
+                                         w.part_val, w.part_idx, w.part_cnt);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_lse_topk(const void* logits, int dtype, int64_t rows, int V, int k,
                             const TopkWorkspace& w, cudaStream_t st) {
+  // rows that are whole 16-byte fragments go through the bulk-copy ring; other V use plain scalar loads
   if (dtype == UBT_BF16) {
-    if (V % 8 == 0) return launch_lse_topk_t<__nv_bfloat16, 8>(logits, rows, V, k, w, st);
+    if (V % 8 == 0) return launch_lse_topk_ring_t<__nv_bfloat16>(logits, rows, V, k, w, st);
     return launch_lse_topk_t<__nv_bfloat16, 1>(logits, rows, V, k, w, st);
   }
-  if (V % 4 == 0) return launch_lse_topk_t<float, 4>(logits, rows, V, k, w, st);
+  if (V % 4 == 0) return launch_lse_topk_ring_t<float>(logits, rows, V, k, w, st);
   return launch_lse_topk_t<float, 1>(logits, rows, V, k, w, st);
 }
 
