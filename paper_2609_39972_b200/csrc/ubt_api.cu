@@ -114,7 +114,7 @@ int ubt_build_tree(const float* bigram_scores, int B, int L, int k, int N, const
   const ubt_draft_opts d{};
   const ubt_draft_opts* o = opts ? opts : &d;
   cudaError_t e = launch_build_tree(bigram_scores, B, L, k, N, o->search_width, o->depth_bonus, o->alpha, o->lambda,
-                                    o->anchor_bigram, o->anchor_tokens, o->pos_offset, *out,
+                                    o->anchor_bigram, o->anchor_tokens, o->pos_offset, *out, no_merge_parts(), 0,
                                     static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? UBT_OK : UBT_ERR_CUDA;
 }
@@ -141,10 +141,18 @@ int ubt_draft_tree(const void* unigram_logits, int dtype, const float* bigram_sc
   if (out->B != B || out->N != N || out->L != L || out->k != k) return UBT_ERR_INVALID_ARG;
   if (tree_smem_bytes(L, k, N) > (size_t)device_info().max_smem_optin) return UBT_ERR_UNSUPPORTED;
   if (B == 0) return UBT_OK;
-  rc = ubt_topk_logprob(unigram_logits, dtype, (int64_t)B * L, V, k, out->cand_ids, out->cand_logprob, workspace,
-                        workspace_bytes, cuda_stream);
-  if (rc) return rc;
-  return ubt_build_tree(bigram_scores, B, L, k, N, opts, out, cuda_stream);
+  const int64_t rows = (int64_t)B * L;
+  if (!workspace || !aligned16(workspace) || workspace_bytes < topk_workspace_bytes(rows, V, k))
+    return UBT_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  TopkWorkspace w = carve_topk_workspace(workspace, rows, V, k);
+  if (launch_lse_topk(unigram_logits, dtype, rows, V, k, w, st) != cudaSuccess) return UBT_ERR_CUDA;
+  // the tree kernel merges the row partials in its prologue: one launch less than topk + merge + tree
+  const ubt_draft_opts d{};
+  const ubt_draft_opts* o = opts ? opts : &d;
+  cudaError_t e = launch_build_tree(bigram_scores, B, L, k, N, o->search_width, o->depth_bonus, o->alpha, o->lambda,
+                                    o->anchor_bigram, o->anchor_tokens, o->pos_offset, *out, merge_parts(w), V, st);
+  return e == cudaSuccess ? UBT_OK : UBT_ERR_CUDA;
 }
 
 int ubt_verify_tree(const ubt_tree* tree, const void* target_logits, int dtype, int V, int mode,

@@ -68,6 +68,14 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// A kernel launched with the programmatic-stream-serialization attribute may start while the kernel before
+// it in the stream is still running, once every CTA of that kernel has called pdl_launch_dependents() (or
+// exited); pdl_wait() blocks until the earlier kernel has completed and its writes are visible.  Both are
+// no-ops for a kernel that was launched without the attribute / has no such successor.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---------------------------------------------------------------- warp / block reductions
 __device__ __forceinline__ uint64_t warp_max_u64(uint64_t v) {
 #pragma unroll

@@ -7,6 +7,7 @@
 
 #include "../../include/ubt.h"
 #include "ubt_common.cuh"
+#include "ubt_merge.cuh"
 
 namespace ubt {
 
@@ -14,6 +15,23 @@ constexpr int kMaxK = 64;
 constexpr int kMaxN = 256;
 constexpr int kMaxL = 64;
 constexpr size_t kTreeTableBytes = 160 * 1024;
+
+// Kernel launch with or without programmatic dependent launch (see pdl_wait in ubt_common.cuh).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                 bool programmatic, Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = programmatic ? attr : nullptr;
+  cfg.numAttrs = programmatic ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
 
 struct DeviceInfo {
   int sm_count;
@@ -40,13 +58,19 @@ cudaError_t launch_lse_topk(const void* logits, int dtype, int64_t rows, int V, 
                             const TopkWorkspace& w, cudaStream_t st);
 cudaError_t launch_merge_topk(int64_t rows, int V, int k, const TopkWorkspace& w, int32_t* cand_ids,
                               float* cand_lp, cudaStream_t st);
+inline MergeParts merge_parts(const TopkWorkspace& w) {
+  return MergeParts{w.plan, w.part_ms, w.part_val, w.part_idx, w.part_cnt};
+}
+inline MergeParts no_merge_parts() { return MergeParts{SpanPlan{0, 0, 0}, nullptr, nullptr, nullptr, nullptr}; }
 
 // ---- a2 + a3 + a3b --------------------------------------------------------------------------
 size_t tree_smem_bytes(int L, int k, int N);
+// `parts` with a non-null part_ms makes the kernel merge the step-a1 partials itself (V is then the row
+// length they were cut from) and write out.cand_ids / out.cand_logprob; otherwise it reads them.
 cudaError_t launch_build_tree(const float* bigram, int B, int L, int k, int N, int W, float zeta,
                               const float* alpha, const float* lambda, const float* anchor_bigram,
                               const int32_t* anchor_tokens, const int32_t* pos_offset,
-                              const ubt_tree& out, cudaStream_t st);
+                              const ubt_tree& out, const MergeParts& parts, int V, cudaStream_t st);
 cudaError_t launch_build_mask(const ubt_tree& tree, const int32_t* pos_offset, cudaStream_t st);
 
 // ---- a4 ---------------------------------------------------------------------------------------

@@ -1,0 +1,72 @@
+// Merge of the per-segment partials of step a1 into a row's candidates (one warp per row).
+// Used by the standalone merge kernel and by the prologue of the tree kernel.
+#pragma once
+
+#include "ubt_common.cuh"
+
+namespace ubt {
+
+// The partial arrays the streaming kernel wrote (see TopkWorkspace); parts.part_ms == nullptr means "none".
+struct MergeParts {
+  SpanPlan plan;
+  const float* part_ms;     // [rows, smax, 2]  (max, sum of exp relative to it)
+  const float* part_val;    // [rows, smax, k]
+  const int32_t* part_idx;  // [rows, smax, k]
+  const int32_t* part_cnt;  // [rows, smax]
+};
+
+// Every lane of one warp calls this for the same row.  Writes cand_ids[row, 0..k) (best first) and
+// cand_lp[row, r] = value - log-sum-exp of the whole row.
+__device__ __forceinline__ void merge_row_warp(const MergeParts& p, int64_t rows, int64_t row, int V, int k,
+                                               int32_t* __restrict__ cand_ids_, float* __restrict__ cand_lp_,
+                                               int lane) {
+  const long long nslots = rows * p.plan.smax;
+  const Span<const float> part_ms(p.part_ms, nslots * 2, 321), part_val(p.part_val, nslots * k, 322);
+  const Span<const int32_t> part_idx(p.part_idx, nslots * k, 323), part_cnt(p.part_cnt, nslots, 324);
+  const Span<int32_t> cand_ids(cand_ids_, rows * k, 325);
+  const Span<float> cand_lp(cand_lp_, rows * k, 326);
+  const int64_t c_first = (row * (int64_t)V) / p.plan.span;
+  const int64_t c_last = ((row + 1) * (int64_t)V - 1) / p.plan.span;
+  const int nseg = (int)(c_last - c_first + 1);
+  const int64_t base = row * p.plan.smax;
+
+  float M = -1.0e30f;
+  for (int j = lane; j < nseg; j += 32) M = fmaxf(M, part_ms[(base + j) * 2]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(FULL, M, o));
+  float S = 0.f;
+  for (int j = lane; j < nseg; j += 32)
+    S += part_ms[(base + j) * 2 + 1] * exp2f((part_ms[(base + j) * 2] - M) * kLog2e);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) S += __shfl_xor_sync(FULL, S, o);
+  const float lse = M + logf(S);
+
+  int found = 0;
+  const int nq = nseg * k;
+  for (int q = lane; q < nq; q += 32) {
+    const int j = q / k, i = q - j * k;
+    if (i >= part_cnt[base + j]) continue;
+    const float val = part_val[(base + j) * k + i];
+    const int idx = part_idx[(base + j) * k + i];
+    const uint64_t key = make_key(val, idx);
+    int rank = 0;
+    for (int j2 = 0; j2 < nseg; ++j2) {
+      const int c2 = part_cnt[base + j2];
+      for (int i2 = 0; i2 < c2; ++i2)
+        rank += make_key(part_val[(base + j2) * k + i2], part_idx[(base + j2) * k + i2]) > key;
+    }
+    if (rank < k) {
+      cand_ids[row * k + rank] = idx;
+      cand_lp[row * k + rank] = val - lse;
+    }
+  }
+  for (int j = lane; j < nseg; j += 32) found += part_cnt[base + j];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) found += __shfl_xor_sync(FULL, found, o);
+  for (int r = found + lane; r < k; r += 32) {  // fewer than k entries above -inf: documented as unsupported
+    cand_ids[row * k + r] = -1;
+    cand_lp[row * k + r] = -INFINITY;
+  }
+}
+
+}  // namespace ubt

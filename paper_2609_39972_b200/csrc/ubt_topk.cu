@@ -11,6 +11,7 @@
 // is prefetched into registers before the current one is processed, so the one barrier per tile
 // does not drain the loads in flight.
 #include "ubt_internal.h"
+#include "ubt_merge.cuh"
 #include "ubt_ring.cuh"
 
 namespace ubt {
@@ -292,6 +293,7 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
   const int tid = threadIdx.x, lane = tid & 31;
   const int64_t lo = (int64_t)blockIdx.x * plan.span;
   const int64_t hi = lo + plan.span < total ? lo + plan.span : total;
+  pdl_launch_dependents();  // the tree kernel may be scheduled; it waits for this grid before reading
   if (lo >= hi) return;
   const long long nslots = (total / V) * plan.smax;
   const Span<float> g_ms(part_ms, nslots * 2, 341), g_val(part_val, nslots * k, 342);
@@ -452,61 +454,13 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
   if (tid == 0 && *reinterpret_cast<volatile int*>(&s_fail)) prod.drain(consumed > 0 ? consumed - 1 : 0, full);
 }
 
-// One warp per row: combine the partials of the row's segments.
+// One warp per row: combine the partials of the row's segments (see merge_row_warp in ubt_merge.cuh).
 __global__ void __launch_bounds__(128)
-k_merge_topk(const float* __restrict__ part_ms_, const float* __restrict__ part_val_,
-             const int32_t* __restrict__ part_idx_, const int32_t* __restrict__ part_cnt_, int64_t rows,
-             int V, int k, SpanPlan plan, int32_t* __restrict__ cand_ids_, float* __restrict__ cand_lp_) {
-  const int lane = threadIdx.x & 31;
+k_merge_topk(MergeParts parts, int64_t rows, int V, int k, int32_t* __restrict__ cand_ids,
+             float* __restrict__ cand_lp) {
   const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (row >= rows) return;
-  const long long nslots = rows * plan.smax;
-  const Span<const float> part_ms(part_ms_, nslots * 2, 321), part_val(part_val_, nslots * k, 322);
-  const Span<const int32_t> part_idx(part_idx_, nslots * k, 323), part_cnt(part_cnt_, nslots, 324);
-  const Span<int32_t> cand_ids(cand_ids_, rows * k, 325);
-  const Span<float> cand_lp(cand_lp_, rows * k, 326);
-  const int64_t c_first = (row * (int64_t)V) / plan.span;
-  const int64_t c_last = ((row + 1) * (int64_t)V - 1) / plan.span;
-  const int nseg = (int)(c_last - c_first + 1);
-  const int64_t base = row * plan.smax;
-
-  float M = -1.0e30f;
-  for (int j = lane; j < nseg; j += 32) M = fmaxf(M, part_ms[(base + j) * 2]);
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(FULL, M, o));
-  float S = 0.f;
-  for (int j = lane; j < nseg; j += 32)
-    S += part_ms[(base + j) * 2 + 1] * exp2f((part_ms[(base + j) * 2] - M) * kLog2e);
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) S += __shfl_xor_sync(FULL, S, o);
-  const float lse = M + logf(S);
-
-  int found = 0;
-  const int nq = nseg * k;
-  for (int q = lane; q < nq; q += 32) {
-    const int j = q / k, i = q - j * k;
-    if (i >= part_cnt[base + j]) continue;
-    const float val = part_val[(base + j) * k + i];
-    const int idx = part_idx[(base + j) * k + i];
-    const uint64_t key = make_key(val, idx);
-    int rank = 0;
-    for (int j2 = 0; j2 < nseg; ++j2) {
-      const int c2 = part_cnt[base + j2];
-      for (int i2 = 0; i2 < c2; ++i2)
-        rank += make_key(part_val[(base + j2) * k + i2], part_idx[(base + j2) * k + i2]) > key;
-    }
-    if (rank < k) {
-      cand_ids[row * k + rank] = idx;
-      cand_lp[row * k + rank] = val - lse;
-    }
-  }
-  for (int j = lane; j < nseg; j += 32) found += part_cnt[base + j];
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) found += __shfl_xor_sync(FULL, found, o);
-  for (int r = found + lane; r < k; r += 32) {  // fewer than k entries above -inf: documented as unsupported
-    cand_ids[row * k + r] = -1;
-    cand_lp[row * k + r] = -INFINITY;
-  }
+  merge_row_warp(parts, rows, row, V, k, cand_ids, cand_lp, threadIdx.x & 31);
 }
 
 // ------------------------------------------------------------------------------------ host side
@@ -592,8 +546,7 @@ cudaError_t launch_merge_topk(int64_t rows, int V, int k, const TopkWorkspace& w
                               float* cand_lp, cudaStream_t st) {
   const int warps = 4;
   const int grid = (int)((rows + warps - 1) / warps);
-  k_merge_topk<<<grid, warps * 32, 0, st>>>(w.part_ms, w.part_val, w.part_idx, w.part_cnt, rows, V, k,
-                                            w.plan, cand_ids, cand_lp);
+  k_merge_topk<<<grid, warps * 32, 0, st>>>(merge_parts(w), rows, V, k, cand_ids, cand_lp);
   return cudaGetLastError();
 }
 

@@ -1,35 +1,44 @@
 // Steps a2, a3, a3b: candidate-pair log-probabilities, budgeted tree expansion, tree-attention inputs.
 //
-// One CTA per sequence.  The pair table t[i][ra][rb] = log q^bi (eq. 5 + eq. 9) lives in shared
-// memory with, for every (i, ra), the successors sorted best first.  Algorithm 1 is run as a
-// best-first search: the frontier holds, per expanded node, its best not-yet-taken child; a pop
-// takes the best frontier entry under the total order (score desc, depth asc, token asc, rank path
-// asc), replaces it by its next sibling and adds its own first child.  Because every pair
-// log-probability is <= 0 and zeta <= 0, scores never increase along a path, so pops come out in
-// the global order; a node popped when its depth already holds W nodes is outside Top_W(E_d) and is
-// dropped with its later siblings.  N-1 accepted pops give Top_B of the supertree (eq. 11-12).
+// One CTA per sequence.  The pair table t[i][ra][.] = log q^bi (eq. 5 + eq. 9) lives in shared memory,
+// every row sorted best first, next to the permutation that sorted it.  Algorithm 1 is run as a best-first
+// search: the frontier holds, per expanded node, its best not-yet-taken child; a pop takes the best
+// frontier entry under the total order (score desc, depth asc, token asc, rank path asc), replaces it by its
+// next sibling and adds its own first child.  Because every pair log-probability is <= 0 and zeta <= 0,
+// scores never increase along a path, so pops come out in the global order; a node popped when its depth
+// already holds W nodes is outside Top_W(E_d) and is dropped with its later siblings.  N-1 accepted pops
+// give Top_B of the supertree (eq. 11-12).
+//
+// The search is a chain of N-1 dependent pops, so its latency is what counts: the frontier lives in the
+// registers of one warp (entry i in lane i&31, slot i>>5; the score is recovered from its ordering key and
+// everything a pop needs is packed in one word), a pop is a register scan, one warp-wide max, two shuffles
+// and one round of independent shared-memory loads.
 #include "ubt_internal.h"
+#ifdef UBT_TREE_TIMING
+#include <cstdio>
+#define TT(i) do { if (b == 0 && tid == 0) tt[i] = clock64(); } while (0)
+#else
+#define TT(i) do {} while (0)
+#endif
 
 namespace ubt {
 
 constexpr int G2_T = 256;
 
 struct TreeSmem {
-  Span<float> t;            // [L,k,k]
-  Span<unsigned char> ord;  // [L,k,k]  successor ranks sorted by (t desc, token asc)
+  Span<float> t;            // [L,k,k]  pair log-probabilities, each row sorted descending after set-up
+  Span<unsigned char> ord;  // [L,k,k]  ord[row][j] = candidate rank of the j-th best successor
   Span<float> lp;           // [L,k]
   Span<int> tok;            // [L,k]
-  Span<uint32_t> f_key;     // frontier, <= N entries
-  Span<float> f_score;
-  Span<short> f_parent;     // accepted-node index of the parent, -1 = root
-  Span<unsigned char> f_sib;  // position in the parent's sorted successor list
-  Span<short> nd_parent;    // accepted nodes in pop order, <= N-1
+  Span<uint32_t> f_key;     // mirror of the frontier (for exact score ties only), <= N entries
+  Span<uint32_t> f_info;
+  Span<short> nd_parent;    // accepted nodes in pop order, <= N-1; -1 = child of the root
   Span<unsigned char> nd_depth;
   Span<unsigned char> nd_rank;
   Span<float> nd_score;
   Span<short> nd_slot;
-  Span<short> bkt;          // nodes grouped by depth
-  Span<int> kk;             // per-depth sort keys
+  Span<unsigned long long> nd_pk;  // [N,2] rank path packed big-endian (hi, lo): lexicographic = numeric
+  Span<int> kk;             // per-depth sort keys (fallback slot assignment)
   Span<int> depth_cnt;      // [L+2]
   Span<int> depth_off;      // [L+2]
   Span<uint32_t> maskrow;   // [N, mask_words]
@@ -47,11 +56,10 @@ __host__ __device__ inline size_t tree_carve(TreeSmem* s, unsigned char* base, i
   const long long lkk = (long long)L * k * k, lk = (long long)L * k;
   size_t o_t = take(sizeof(float) * lkk), o_ord = take((size_t)lkk);
   size_t o_lp = take(sizeof(float) * lk), o_tok = take(sizeof(int) * lk);
-  size_t o_fk = take(sizeof(uint32_t) * (N + 1)), o_fs = take(sizeof(float) * (N + 1));
-  size_t o_fp = take(sizeof(short) * (N + 1)), o_fb = take(N + 1);
+  size_t o_fk = take(sizeof(uint32_t) * (N + 1)), o_fi = take(sizeof(uint32_t) * (N + 1));
   size_t o_np = take(sizeof(short) * N), o_nd = take(N), o_nr = take(N);
-  size_t o_ns = take(sizeof(float) * N), o_nl = take(sizeof(short) * N), o_bk = take(sizeof(short) * N);
-  size_t o_kk = take(sizeof(int) * N);
+  size_t o_ns = take(sizeof(float) * N), o_nl = take(sizeof(short) * N);
+  size_t o_pk = take(sizeof(unsigned long long) * 2 * N), o_kk = take(sizeof(int) * N);
   size_t o_dc = take(sizeof(int) * (L + 2)), o_do = take(sizeof(int) * (L + 2));
   size_t o_mk = take(sizeof(uint32_t) * N * mw), o_sc = take(sizeof(int) * 4);
   if (s) {
@@ -60,15 +68,13 @@ __host__ __device__ inline size_t tree_carve(TreeSmem* s, unsigned char* base, i
     s->lp = Span<float>((float*)(base + o_lp), lk, 103);
     s->tok = Span<int>((int*)(base + o_tok), lk, 104);
     s->f_key = Span<uint32_t>((uint32_t*)(base + o_fk), N + 1, 105);
-    s->f_score = Span<float>((float*)(base + o_fs), N + 1, 106);
-    s->f_parent = Span<short>((short*)(base + o_fp), N + 1, 107);
-    s->f_sib = Span<unsigned char>(base + o_fb, N + 1, 108);
+    s->f_info = Span<uint32_t>((uint32_t*)(base + o_fi), N + 1, 106);
     s->nd_parent = Span<short>((short*)(base + o_np), N, 109);
     s->nd_depth = Span<unsigned char>(base + o_nd, N, 110);
     s->nd_rank = Span<unsigned char>(base + o_nr, N, 111);
     s->nd_score = Span<float>((float*)(base + o_ns), N, 112);
     s->nd_slot = Span<short>((short*)(base + o_nl), N, 113);
-    s->bkt = Span<short>((short*)(base + o_bk), N, 114);
+    s->nd_pk = Span<unsigned long long>((unsigned long long*)(base + o_pk), 2LL * N, 114);
     s->kk = Span<int>((int*)(base + o_kk), N, 115);
     s->depth_cnt = Span<int>((int*)(base + o_dc), L + 2, 116);
     s->depth_off = Span<int>((int*)(base + o_do), L + 2, 117);
@@ -80,11 +86,129 @@ __host__ __device__ inline size_t tree_carve(TreeSmem* s, unsigned char* base, i
 
 size_t tree_smem_bytes(int L, int k, int N) { return tree_carve(nullptr, nullptr, L, k, N); }
 
+// Frontier entry word: parent node (8 bits, 255 = the root), sibling position j in the parent's sorted
+// successor list (6), depth - 1 (6), candidate rank of the parent (6), own candidate rank (6).
+__device__ __forceinline__ uint32_t pack_info(int p, int j, int d, int pr, int r) {
+  return (uint32_t)p | ((uint32_t)j << 8) | ((uint32_t)(d - 1) << 14) | ((uint32_t)pr << 20) | ((uint32_t)r << 26);
+}
+
+// Best-first expansion by one warp; returns the number of accepted nodes (all lanes agree).
+template <int SLOTS>
+__device__ int expand_tree(TreeSmem& s, int L, int k, int budget, int W, float zeta, int bits, bool use_pk,
+                           int lane) {
+  uint32_t fk[SLOTS], fi[SLOTS];
+#pragma unroll
+  for (int q = 0; q < SLOTS; ++q) { fk[q] = 0u; fi[q] = 0u; }
+  int f_cnt = 0, n_acc = 0;
+  // entry idx <- (key, info); every lane calls, the owner keeps it in registers and mirrors it to shared
+  auto put = [&](int idx, uint32_t key, uint32_t info) {
+    const int ol = idx & 31, os = idx >> 5;
+#pragma unroll
+    for (int q = 0; q < SLOTS; ++q)
+      if (q == os && lane == ol) { fk[q] = key; fi[q] = info; }
+    if (lane == ol) { s.f_key[idx] = key; s.f_info[idx] = info; }
+  };
+  if (budget > 0) {
+    const int r0 = s.ord[0];
+    put(0, f2key(s.t[0] + zeta), pack_info(255, 0, 1, 0, r0));
+    f_cnt = 1;
+  }
+  __syncwarp();
+  while (n_acc < budget) {
+    uint32_t bk = fk[0];
+    int bs = 0;
+    bool dup = false;
+#pragma unroll
+    for (int q = 1; q < SLOTS; ++q) {
+      if (fk[q] > bk) { bk = fk[q]; bs = q; dup = false; }
+      else if (fk[q] == bk && bk != 0u) dup = true;
+    }
+    const uint32_t maxk = __reduce_max_sync(FULL, bk);
+    if (maxk == 0u) break;  // frontier exhausted
+    const unsigned holders = __ballot_sync(FULL, bk == maxk);
+    const bool tie = __any_sync(FULL, bk == maxk && dup) || __popc(holders) > 1;
+    int widx;
+    uint32_t winfo;
+    if (!tie) {
+      const int wl = __ffs(holders) - 1;
+      uint32_t mine = fi[0];
+#pragma unroll
+      for (int q = 1; q < SLOTS; ++q) mine = q == bs ? fi[q] : mine;
+      winfo = __shfl_sync(FULL, mine, wl);
+      widx = __shfl_sync(FULL, bs, wl) * 32 + wl;
+    } else {
+      int best = -1;
+      if (lane == 0) {  // exact score ties: depth asc, token asc, then rank path lexicographic
+        int bd = 0, bt = 0;
+        for (int i = 0; i < f_cnt; ++i) {
+          if (s.f_key[i] != maxk) continue;
+          const uint32_t inf = s.f_info[i];
+          const int d = (int)((inf >> 14) & 63u) + 1, r = (int)(inf >> 26);
+          const int tkn = s.tok[(d - 1) * k + r];
+          bool better;
+          if (best < 0) better = true;
+          else if (d != bd) better = d < bd;
+          else if (tkn != bt) better = tkn < bt;
+          else {  // same depth and token: the shallowest level where the two prefixes differ decides
+            int pa = (int)(inf & 255u), pb = (int)(s.f_info[best] & 255u), ra = 0, rb = 0;
+            pa = pa == 255 ? -1 : pa; pb = pb == 255 ? -1 : pb;
+            while (pa != pb) {
+              ra = s.nd_rank[pa]; rb = s.nd_rank[pb];
+              pa = s.nd_parent[pa]; pb = s.nd_parent[pb];
+            }
+            better = ra < rb;
+          }
+          if (better) { best = i; bd = d; bt = tkn; }
+        }
+      }
+      widx = __shfl_sync(FULL, best, 0);
+      winfo = s.f_info[widx];
+    }
+    const int p = (int)(winfo & 255u), j = (int)((winfo >> 8) & 63u), d = (int)((winfo >> 14) & 63u) + 1;
+    const int pr = (int)((winfo >> 20) & 63u), r = (int)(winfo >> 26);
+    const float score = key2f(maxk);
+    const int prev = ((d - 1) * k + pr) * k;
+    const int dc = s.depth_cnt[d];
+    if (W > 0 && dc >= W) {  // outside Top_W(E_d); so are its later siblings
+      put(widx, 0u, 0u);
+      __syncwarp();
+      continue;
+    }
+    // one round of independent loads: next sibling, first child, parent score
+    const bool has_sib = j + 1 < k, has_child = d < L;
+    const int child = (d * k + r) * k;
+    const float t_sib = has_sib ? s.t[prev + j + 1] : 0.f;
+    const int r_sib = has_sib ? s.ord[prev + j + 1] : 0;
+    const float t_child = has_child ? s.t[child] : 0.f;
+    const int r_child = has_child ? s.ord[child] : 0;
+    const float ps = p == 255 ? 0.f : s.nd_score[p];
+    const int n = n_acc++;
+    if (lane == 0) {
+      s.nd_parent[n] = (short)(p == 255 ? -1 : p);
+      s.nd_depth[n] = (unsigned char)d;
+      s.nd_rank[n] = (unsigned char)r;
+      s.nd_score[n] = score;
+      s.depth_cnt[d] = dc + 1;
+      if (use_pk) {
+        unsigned long long hi = p == 255 ? 0ull : s.nd_pk[2 * p], lo = p == 255 ? 0ull : s.nd_pk[2 * p + 1];
+        const int sh = 128 - bits * d;
+        if (sh >= 64) hi |= (unsigned long long)r << (sh - 64); else lo |= (unsigned long long)r << sh;
+        s.nd_pk[2 * n] = hi; s.nd_pk[2 * n + 1] = lo;
+      }
+    }
+    if (has_sib) put(widx, f2key(ps + t_sib + zeta), pack_info(p, j + 1, d, pr, r_sib));
+    else put(widx, 0u, 0u);
+    if (has_child) { put(f_cnt, f2key(score + t_child + zeta), pack_info(n, 0, d + 1, r, r_child)); ++f_cnt; }
+    __syncwarp();
+  }
+  return n_acc;
+}
+
 __global__ void __launch_bounds__(G2_T)
 k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float zeta,
              const float* __restrict__ alpha, const float* __restrict__ lambda,
              const float* __restrict__ anchor_bigram, const int32_t* __restrict__ anchor_tokens,
-             const int32_t* __restrict__ pos_offset, ubt_tree out) {
+             const int32_t* __restrict__ pos_offset, ubt_tree out, MergeParts parts, int V) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   TreeSmem s;
   tree_carve(&s, smem_raw, L, k, N);
@@ -97,7 +221,20 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   const Span<int32_t> g_rk(out.cand_rank, nB * N, 214), g_pos(out.position_ids, nB * N, 215), g_nn(out.n_nodes, nB, 216);
   const Span<float> g_sc(out.scores, nB * N, 217);
   const Span<uint32_t> g_mask(out.mask, nB * N * mw, 218);
+#ifdef UBT_TREE_TIMING
+  long long tt[10];
+#endif
+  TT(0);
+  pdl_wait();  // the partials / candidates come from the kernel before this one
 
+  // ---- step a1's last part when fused: merge the row partials of this sequence's L rows
+  if (parts.part_ms != nullptr) {
+    for (int i = tid >> 5; i < L; i += G2_T / 32)
+      merge_row_warp(parts, nB * L, (int64_t)b * L + i, V, k, out.cand_ids, out.cand_logprob, lane);
+    __syncthreads();  // the candidates were written by this CTA; the barrier orders them before the reads below
+  }
+
+  TT(1);
   // ---- stage candidates and raw selector scores
   for (int i = tid; i < L * k; i += G2_T) {
     s.lp[i] = g_lp[(int64_t)b * L * k + i];
@@ -112,10 +249,17 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
     }
     s.t[i] = d;
   }
+  // Every read of memory an earlier kernel produced (row partials in the caller's workspace, candidates,
+  // selector scores) has been issued; from here on only this kernel's own outputs are touched, so the next
+  // kernel in the stream -- typically the V-wide pass of ubt_verify_tree, which needs none of them -- may
+  // start.  It waits for this grid before it exits, so stream order still holds for whatever follows it.
+  __syncthreads();
+  pdl_launch_dependents();
   for (int i = tid; i < L + 2; i += G2_T) s.depth_cnt[i] = 0;
   for (int i = tid; i < N * mw; i += G2_T) s.maskrow[i] = 0u;
   __syncthreads();
 
+  TT(2);
   // ---- eq. 5 and eq. 9: one thread per (position, predecessor) row
   const int nrows = 1 + (L - 1) * k;
   for (int r = tid; r < nrows; r += G2_T) {
@@ -135,117 +279,51 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
     for (int rb = 0; rb < k; ++rb) row[rb] -= lse;
   }
   __syncthreads();
-  // successors of every row sorted by (t desc, token asc)
-  for (int q = tid; q < nrows * k; q += G2_T) {
-    const int r = q / k, rb = q - r * k;
-    const int i = r == 0 ? 0 : 1 + (r - 1) / k;
-    const int ra = r == 0 ? 0 : (r - 1) % k;
-    const float* row = s.t.ptr(((long long)i * k + ra) * k, k);
-    const int* tk = s.tok.ptr((long long)i * k, k);
-    // integer keys and a final index tie-break keep this a permutation whatever the values are (even NaN)
-    const uint32_t kv = f2key(row[rb]);
-    int rank = 0;
-    for (int j = 0; j < k; ++j) {
-      const uint32_t kj = f2key(row[j]);
-      rank += (kj > kv) || (kj == kv && (tk[j] < tk[rb] || (tk[j] == tk[rb] && j < rb)));
+  TT(3);
+  // every row sorted by (t desc, token asc), in place; integer keys and a final index tie-break keep the
+  // ranks a permutation whatever the values are (even NaN)
+  const int rows_per_batch = G2_T / k;  // whole rows per batch: a row is read completely before it is rewritten
+  for (int row0 = 0; row0 < nrows; row0 += rows_per_batch) {
+    const int r = row0 + tid / k, rb = tid % k;
+    const bool active = tid < rows_per_batch * k && r < nrows;
+    float v = 0.f;
+    int rank = 0, at = 0;
+    if (active) {
+      const int i = r == 0 ? 0 : 1 + (r - 1) / k;
+      const int ra = r == 0 ? 0 : (r - 1) % k;
+      at = (i * k + ra) * k;
+      const float* row = s.t.ptr(at, k);
+      const int* tk = s.tok.ptr((long long)i * k, k);
+      v = row[rb];
+      const uint32_t kv = f2key(v);
+      for (int j = 0; j < k; ++j) {
+        const uint32_t kj = f2key(row[j]);
+        rank += (kj > kv) || (kj == kv && (tk[j] < tk[rb] || (tk[j] == tk[rb] && j < rb)));
+      }
     }
-    s.ord[((size_t)i * k + ra) * k + rank] = (unsigned char)rb;
+    __syncthreads();  // all reads of this batch of rows precede the in-place writes
+    if (active) {
+      s.t[at + rank] = v;
+      s.ord[at + rank] = (unsigned char)rb;
+    }
+    __syncthreads();
   }
-  __syncthreads();
 
+  TT(4);
   // ---- best-first expansion (warp 0)
+  int bits = 1;
+  while ((1 << bits) < k) ++bits;
+  const bool use_pk = bits * L <= 128;
   if (tid < 32) {
-    int f_cnt = 0, n_acc = 0;
-    if (budget > 0) {
-      const int r0 = s.ord[0];
-      const float sc = s.t[r0] + zeta;
-      if (lane == 0) {
-        s.f_key[0] = f2key(sc); s.f_score[0] = sc; s.f_parent[0] = -1; s.f_sib[0] = 0;
-      }
-      f_cnt = 1;
-    }
-    __syncwarp();
-    while (n_acc < budget) {
-      uint32_t bk = 0; int bi = -1; bool dup = false;
-      for (int i = lane; i < f_cnt; i += 32) {
-        const uint32_t key = s.f_key[i];
-        if (key > bk) { bk = key; bi = i; dup = false; }
-        else if (key == bk && key != 0) dup = true;
-      }
-      const uint32_t maxk = __reduce_max_sync(FULL, bk);
-      if (maxk == 0) break;  // frontier exhausted
-      const unsigned holders = __ballot_sync(FULL, bk == maxk);
-      const bool tie = __any_sync(FULL, bk == maxk && dup) || __popc(holders) > 1;
-      int wi;
-      if (!tie) {
-        wi = __shfl_sync(FULL, bi, __ffs(holders) - 1);
-      } else {
-        int best = -1;
-        if (lane == 0) {  // exact ties: depth asc, token asc, then rank path lexicographic
-          int bd = 0, bt = 0;
-          for (int i = 0; i < f_cnt; ++i) {
-            if (s.f_key[i] != maxk) continue;
-            const int p = s.f_parent[i];
-            const int d = p < 0 ? 1 : s.nd_depth[p] + 1;
-            const int pr = p < 0 ? 0 : s.nd_rank[p];
-            const int tkn = s.tok[(d - 1) * k + s.ord[((size_t)(d - 1) * k + pr) * k + s.f_sib[i]]];
-            bool better;
-            if (best < 0) better = true;
-            else if (d != bd) better = d < bd;
-            else if (tkn != bt) better = tkn < bt;
-            else {
-              int pa = p, pb = s.f_parent[best], ra = 0, rb = 0;
-              while (pa != pb) {
-                ra = s.nd_rank[pa]; rb = s.nd_rank[pb];
-                pa = s.nd_parent[pa]; pb = s.nd_parent[pb];
-              }
-              better = ra < rb;
-            }
-            if (better) { best = i; bd = d; bt = tkn; }
-          }
-        }
-        wi = __shfl_sync(FULL, best, 0);
-      }
-      const int p = s.f_parent[wi], j = s.f_sib[wi];
-      const int d = p < 0 ? 1 : s.nd_depth[p] + 1;
-      const int pr = p < 0 ? 0 : s.nd_rank[p];
-      const float score = s.f_score[wi];
-      const int r = s.ord[((size_t)(d - 1) * k + pr) * k + j];
-      const int dc = s.depth_cnt[d];
-      __syncwarp();
-      if (W > 0 && dc >= W) {  // outside Top_W(E_d); so are its later siblings
-        if (lane == 0) s.f_key[wi] = 0u;
-        __syncwarp();
-        continue;
-      }
-      const int n = n_acc++;
-      if (lane == 0) {
-        s.nd_parent[n] = (short)p; s.nd_depth[n] = (unsigned char)d; s.nd_rank[n] = (unsigned char)r;
-        s.nd_score[n] = score;
-        s.bkt[n] = (short)dc;  // position inside its depth, in pop order (re-bucketed below)
-        s.depth_cnt[d] = dc + 1;
-        if (j + 1 < k) {
-          const int r2 = s.ord[((size_t)(d - 1) * k + pr) * k + j + 1];
-          const float ps = p < 0 ? 0.f : s.nd_score[p];
-          const float s2 = ps + s.t[((size_t)(d - 1) * k + pr) * k + r2] + zeta;
-          s.f_score[wi] = s2; s.f_key[wi] = f2key(s2); s.f_sib[wi] = (unsigned char)(j + 1);
-        } else {
-          s.f_key[wi] = 0u;
-        }
-        if (d < L) {
-          const int r3 = s.ord[((size_t)d * k + r) * k];
-          const float s3 = score + s.t[((size_t)d * k + r) * k + r3] + zeta;
-          s.f_score[f_cnt] = s3; s.f_key[f_cnt] = f2key(s3);
-          s.f_parent[f_cnt] = (short)n; s.f_sib[f_cnt] = 0;
-        }
-      }
-      if (d < L) ++f_cnt;
-      __syncwarp();
-    }
-    if (lane == 0) s.scalars[0] = n_acc;
+    int n;
+    if (N <= 64) n = expand_tree<2>(s, L, k, budget, W, zeta, bits, use_pk, lane);
+    else if (N <= 128) n = expand_tree<4>(s, L, k, budget, W, zeta, bits, use_pk, lane);
+    else n = expand_tree<8>(s, L, k, budget, W, zeta, bits, use_pk, lane);
+    if (lane == 0) s.scalars[0] = n;
   }
   __syncthreads();
 
+  TT(5);
   // ---- canonical slots: root 0, then depth by depth ordered by (parent slot, rank)
   const int n_acc = s.scalars[0];
   if (tid == 0) {
@@ -253,31 +331,39 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
     for (int d = 1; d <= L; ++d) { s.depth_off[d] = off; off += s.depth_cnt[d]; }
   }
   __syncthreads();
-  short mynode_dpos = -1;
-  if (tid < n_acc) mynode_dpos = s.bkt[tid];
-  __syncthreads();
-  if (tid < n_acc) s.bkt[s.depth_off[s.nd_depth[tid]] - 1 + mynode_dpos] = (short)tid;
-  __syncthreads();
-  for (int d = 1; d <= L; ++d) {
-    const int cnt = s.depth_cnt[d];
-    if (cnt == 0) break;  // prefix-closed: deeper levels are empty too
-    const int off = s.depth_off[d];
-    int node = -1, key = 0;
-    if (tid < cnt) {
-      node = s.bkt[off - 1 + tid];
-      const int p = s.nd_parent[node];
-      key = (p < 0 ? 0 : s.nd_slot[p]) * k + s.nd_rank[node];
-      s.kk[tid] = key;
-    }
-    __syncthreads();
-    if (tid < cnt) {
+  if (use_pk) {
+    // inside a depth, (parent slot, rank) order is the lexicographic order of the rank paths
+    if (tid < n_acc) {
+      const int d = s.nd_depth[tid];
+      const unsigned long long hi = s.nd_pk[2 * tid], lo = s.nd_pk[2 * tid + 1];
       int c = 0;
-      for (int j = 0; j < cnt; ++j) c += s.kk[j] < key;
-      s.nd_slot[node] = (short)(off + c);
+      for (int j = 0; j < n_acc; ++j) {
+        const unsigned long long hj = s.nd_pk[2 * j], lj = s.nd_pk[2 * j + 1];
+        c += (s.nd_depth[j] == d) && (hj < hi || (hj == hi && lj < lo));
+      }
+      s.nd_slot[tid] = (short)(s.depth_off[d] + c);
     }
     __syncthreads();
+  } else {
+    for (int d = 1; d <= L; ++d) {  // paths too long to pack: one depth at a time
+      if (s.depth_cnt[d] == 0) break;  // prefix-closed: deeper levels are empty too
+      const bool mine = tid < n_acc && s.nd_depth[tid] == d;
+      if (tid < n_acc) {
+        const int p = s.nd_parent[tid];
+        s.kk[tid] = mine ? (p < 0 ? 0 : s.nd_slot[p]) * k + s.nd_rank[tid] : -1;
+      }
+      __syncthreads();
+      if (mine) {
+        const int key = s.kk[tid];
+        int c = 0;
+        for (int j = 0; j < n_acc; ++j) c += s.kk[j] >= 0 && s.kk[j] < key;
+        s.nd_slot[tid] = (short)(s.depth_off[d] + c);
+      }
+      __syncthreads();
+    }
   }
 
+  TT(6);
   // ---- outputs
   const int64_t o = (int64_t)b * N;
   const int poff = pos_offset ? pos_offset[b] : 0;
@@ -306,6 +392,12 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   }
   __syncthreads();
   for (int i = tid; i < N * mw; i += G2_T) g_mask[(int64_t)b * N * mw + i] = s.maskrow[i];
+  TT(7);
+#ifdef UBT_TREE_TIMING
+  if (b == 0 && tid == 0)
+    printf("tree cycles: merge %lld stage %lld rows %lld sort %lld expand %lld slots %lld out %lld total %lld\n", tt[1] - tt[0],
+           tt[2] - tt[1], tt[3] - tt[2], tt[4] - tt[3], tt[5] - tt[4], tt[6] - tt[5], tt[7] - tt[6], tt[7] - tt[0]);
+#endif
 }
 
 // Step a3b alone: one CTA per sequence, one thread per slot.
@@ -338,14 +430,14 @@ k_build_mask(ubt_tree tree, const int32_t* __restrict__ pos_offset) {
 cudaError_t launch_build_tree(const float* bigram, int B, int L, int k, int N, int W, float zeta,
                               const float* alpha, const float* lambda, const float* anchor_bigram,
                               const int32_t* anchor_tokens, const int32_t* pos_offset,
-                              const ubt_tree& out, cudaStream_t st) {
+                              const ubt_tree& out, const MergeParts& parts, int V, cudaStream_t st) {
   if (B == 0) return cudaSuccess;
   const size_t smem = tree_smem_bytes(L, k, N);
   cudaError_t e = cudaFuncSetAttribute(k_build_tree, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
-  k_build_tree<<<B, G2_T, smem, st>>>(bigram, L, k, N, W, zeta, alpha, lambda, anchor_bigram,
-                                      anchor_tokens, pos_offset, out);
-  return cudaGetLastError();
+  // programmatic launch only when the kernel before it is this library's own streaming kernel
+  return launch_kernel(k_build_tree, dim3(B), dim3(G2_T), smem, st, parts.part_ms != nullptr, bigram, L, k, N, W,
+                       zeta, alpha, lambda, anchor_bigram, anchor_tokens, pos_offset, out, parts, V);
 }
 
 cudaError_t launch_build_mask(const ubt_tree& tree, const int32_t* pos_offset, cudaStream_t st) {

@@ -145,6 +145,7 @@ k_row_argmax_ring(const T* __restrict__ logits, int64_t total, int V, SpanPlan p
   const int64_t lo = (int64_t)blockIdx.x * plan.span;
   const int64_t hi = lo + plan.span < total ? lo + plan.span : total;
   const Span<unsigned long long> part_key(part_key_, (total / V) * plan.smax, 401);
+  pdl_launch_dependents();  // the walk kernel may be scheduled; it waits for this grid before reading
   if (lo >= hi) return;
 
   if (tid == 0) {
@@ -238,6 +239,10 @@ k_row_argmax_ring(const T* __restrict__ logits, int64_t total, int V, SpanPlan p
   }
   __syncthreads();
   if (tid == 0 && *reinterpret_cast<volatile int*>(&s_fail)) prod.drain(consumed > 0 ? consumed - 1 : 0, full);
+  // This kernel reads only the target logits, so it may have started before the kernel in front of it (the
+  // tree builder) finished; it must not complete before that kernel does, or the walk behind it could run
+  // on an unfinished tree.
+  if (tid == 0) pdl_wait();
 }
 
 // ---------------------------------------------------------------------------- sampling picks
@@ -403,6 +408,7 @@ k_walk(ubt_tree tree, int mode, SpanPlan plan, const unsigned long long* __restr
   __shared__ int s_pick[kMaxN], s_tok[kMaxN], s_par[kMaxN];
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, N = tree.N, L = tree.L;
   const int64_t o = (int64_t)b * N;
+  pdl_wait();  // picks and tree come from the kernels before this one
   for (int n = tid; n < N; n += blockDim.x) {
     int p;
     if (mode == UBT_VERIFY_GREEDY) {
@@ -501,9 +507,8 @@ static cudaError_t launch_row_argmax_ring_t(const void* logits, int64_t rows, in
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  kern<<<w.plan.grid, kArgmaxThreads, kBytes, st>>>(static_cast<const T*>(logits), rows * (int64_t)V, V, w.plan,
-                                                    w.part_key);
-  return cudaGetLastError();
+  return launch_kernel(kern, dim3(w.plan.grid), dim3(kArgmaxThreads), kBytes, st, true, static_cast<const T*>(logits),
+                       rows * (int64_t)V, V, w.plan, w.part_key);
 }
 
 cudaError_t launch_row_argmax(const void* logits, int dtype, int64_t rows, int V, const VerifyWorkspace& w,
@@ -546,8 +551,8 @@ cudaError_t launch_walk(const ubt_tree& tree, int mode, const VerifyWorkspace& w
                         const int32_t* sampled_pick, int32_t* node_pick, const ubt_verify_result& out,
                         cudaStream_t st) {
   if (tree.B == 0) return cudaSuccess;
-  k_walk<<<tree.B, 128, 0, st>>>(tree, mode, w.plan, w.part_key, V, sampled_pick, node_pick, out);
-  return cudaGetLastError();
+  return launch_kernel(k_walk, dim3(tree.B), dim3(128), 0, st, true, tree, mode, w.plan,
+                       (const unsigned long long*)w.part_key, V, sampled_pick, node_pick, out);
 }
 
 // Number of bounded waits that gave up in this file's kernels (0 in a healthy run).
