@@ -20,6 +20,12 @@ __device__ __forceinline__ uint32_t f2key(float x) {
 __device__ __forceinline__ float key2f(uint32_t k) {
   return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
+// Largest float strictly below x in the numeric order (x finite or +inf; -0 and +0 are one value).
+__device__ __forceinline__ float next_below(float x) {
+  uint32_t k = f2key(x) - 1u;
+  if (k == 0x7fffffffu) k = 0x7ffffffeu;  // the key of -0 is never produced; step over it
+  return key2f(k);
+}
 // (value desc, index asc) as one descending 64-bit key.
 __device__ __forceinline__ uint64_t make_key(float x, int idx) {
   return ((uint64_t)f2key(x) << 32) | (uint32_t)(~(uint32_t)idx);

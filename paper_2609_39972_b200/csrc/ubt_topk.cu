@@ -13,6 +13,12 @@
 #include "ubt_internal.h"
 #include "ubt_merge.cuh"
 #include "ubt_ring.cuh"
+#ifdef UBT_G1_TIMING
+#include <cstdio>
+#define GT(i) do { long long now_ = clock64(); tt[i] += now_ - tlast; tlast = now_; } while (0)
+#else
+#define GT(i) do {} while (0)
+#endif
 
 namespace ubt {
 
@@ -265,14 +271,67 @@ k_lse_topk(const T* __restrict__ logits, int64_t total, int V, int k, SpanPlan p
 }
 
 // ------------------------------------------------------------------------------- ring-fed version
-// Same algorithm with the logits arriving through the bulk-copy ring (ubt_ring.cuh), two CTAs per SM so
-// that one CTA's barriers (threshold bisection, pool ranking) overlap the other's streaming.
+// Same algorithm with the logits arriving through the bulk-copy ring (ubt_ring.cuh), three CTAs per SM so
+// that one CTA's barriers (threshold bisection, pool ranking) overlap the others' streaming.
 //
 // Log-sum-exp without a running maximum in the common path: every thread fixes a reference ref >= tau0 (the
 // bisected bound, which the exclusive threshold taux never falls below) and accumulates 2^((x-ref)*log2 e).
 // An element <= taux cannot overflow that; an element > taux takes the rare hit path anyway, where the
 // thread moves its reference up if the element is more than 60 above it.
-constexpr int G1R_T = 256, G1R_STAGES = 4, G1R_STAGE_BYTES = 16384, G1R_CTAS = 2;
+//
+// Hits go to a small pool of (value, column) keys, so ranking the pool touches shared memory only.  A chunk
+// that overflows the pool (possible only for pathological rows, e.g. long runs of equal values before the
+// threshold turns strict) has its hits discarded and is walked again in slices that cannot overflow.
+constexpr int G1R_T = 256, G1R_STAGES = 4, G1R_STAGE_BYTES = 16384, G1R_CTAS = 3;
+constexpr int G1R_POOL = 1024;  // hit pool entries
+constexpr int G1R_GROUP = 4;    // fragments per vote
+
+struct G1RShared {
+  int cnt;     // pool entries (may exceed G1R_POOL while a chunk overflows)
+  int ntop;    // entries of top[]
+  float taux;  // exclusive threshold: x enters the pool iff x > taux
+  int fail;    // a bounded wait gave up
+  float redf[2 * (G1R_T / 32)];
+  unsigned long long top[kMaxK];
+  unsigned long long topn[kMaxK];
+  unsigned long long pool[G1R_POOL];
+};
+
+// Rank pool + carried list exactly (keys are unique); afterwards top[0..ntop) is sorted best first, the
+// pool is empty and, when k entries exist, taux is the k-th best value (strict from then on).
+__device__ void flush_keyed(G1RShared& sh, int k) {
+  const int tid = threadIdx.x;
+  const int M = sh.cnt < G1R_POOL ? sh.cnt : G1R_POOL, nt = sh.ntop, total = M + nt;
+  const int newn = total < k ? total : k;
+  for (int i = tid; i < total; i += G1R_T) {
+    const unsigned long long ki = i < M ? sh.pool[i] : sh.top[i - M];
+    int rank = 0;
+    for (int j = 0; j < M; ++j) rank += sh.pool[j] > ki;
+    for (int j = 0; j < nt; ++j) rank += sh.top[j] > ki;
+    if (rank < k) sh.topn[rank] = ki;
+  }
+  __syncthreads();
+  if (tid < newn) sh.top[tid] = sh.topn[tid];
+  if (tid == 0) {
+    sh.ntop = newn;
+    sh.cnt = 0;
+    if (newn == k) sh.taux = key_val(sh.topn[k - 1]);
+  }
+  __syncthreads();
+}
+
+// Append the elements of one fragment that beat the threshold.  Hits are rare, so each hit lane reserves its
+// own pool entry; the other lanes fall through.
+template <int VEC>
+__device__ __forceinline__ void append_hits(G1RShared& sh, const float (&x)[VEC], float taux, int col0) {
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) {
+    if (x[j] > taux) {
+      const int at = atomicAdd(&sh.cnt, 1);
+      if (at < G1R_POOL) sh.pool[at] = make_key(x[j], col0 + j);
+    }
+  }
+}
 
 template <typename T>
 __global__ void __launch_bounds__(G1R_T, G1R_CTAS)
@@ -285,10 +344,8 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
   constexpr int RING_BYTES = G1R_STAGES * G1R_STAGE_BYTES;
   constexpr int NW = G1R_T / 32;
   unsigned char* ring = smem_raw;
-  G1Shared& sh = *reinterpret_cast<G1Shared*>(smem_raw + RING_BYTES);
-  const Span<int> pool(reinterpret_cast<int*>(smem_raw + RING_BYTES + sizeof(G1Shared)), STAGE_ELEMS + G1_SLACK, 331);
+  G1RShared& sh = *reinterpret_cast<G1RShared*>(smem_raw + RING_BYTES);
   __shared__ uint64_t full[G1R_STAGES];
-  __shared__ int s_fail;
 
   const int tid = threadIdx.x, lane = tid & 31;
   const int64_t lo = (int64_t)blockIdx.x * plan.span;
@@ -302,7 +359,7 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
   if (tid == 0) {
     for (int s = 0; s < G1R_STAGES; ++s) mbar_init(&full[s], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    s_fail = 0;
+    sh.fail = 0;
   }
   __syncthreads();
   RingProducer<T, G1R_STAGES, G1R_STAGE_BYTES> prod;
@@ -310,6 +367,10 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
     prod.init(lo, hi, V);
     for (int i = 0; i < G1R_STAGES - 1; ++i) prod.issue_one(logits, ring, full);
   }
+#ifdef UBT_G1_TIMING
+  long long tt[8] = {0, 0, 0, 0, 0, 0, 0, 0}, tlast = clock64();
+  int nflush = 0;
+#endif
   RingPos<G1R_STAGES> rp;
   rp.init();
   int consumed = 0;
@@ -318,36 +379,36 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
   for (int64_t pos = lo; pos < hi && !failed;) {
     Segment sg;
     sg.at(pos, hi, V);
-    const T* rowp = logits + sg.row * V;
     if (tid == 0) { sh.cnt = 0; sh.ntop = 0; sh.taux = -INFINITY; }
-    float ref = -1.0e30f, negref = 1.0e30f * kLog2e, s_t = 0.f;  // ref = -1e30: not fixed yet
+    float ref = -1.0e30f, negref = 1.0e30f * kLog2e;  // ref = -1e30: not fixed yet
+    float acc[G1R_GROUP];
+#pragma unroll
+    for (int u = 0; u < G1R_GROUP; ++u) acc[u] = 0.f;
 
     for (int c = 0; c < sg.len; c += STAGE_ELEMS) {
       const int l = sg.len - c < STAGE_ELEMS ? sg.len - c : STAGE_ELEMS;
-      if (*reinterpret_cast<volatile int*>(&s_fail)) { failed = true; break; }
+      if (*reinterpret_cast<volatile int*>(&sh.fail)) { failed = true; break; }
+      GT(0);
       if (tid == 0) prod.issue_one(logits, ring, full);
+      GT(1);
       const bool ok = mbar_wait(&full[rp.stage], rp.parity);
-      if (!ok) s_fail = 1;
-      const uint4* stage = reinterpret_cast<const uint4*>(ring + (size_t)rp.stage * G1R_STAGE_BYTES);
-      const int nfrag = l / VEC;
-      const int nround = (nfrag + G1R_T - 1) / G1R_T;
+      GT(2);
+      if (!ok) sh.fail = 1;
+      const uint4* stage = reinterpret_cast<const uint4*>(ring + (size_t)rp.stage * G1R_STAGE_BYTES) + tid;
+      const int nfrag = ok ? l / VEC : 0;
+      const int colbase = sg.col0 + c + tid * VEC;
 
       if (c == 0) {
         // Bound for the k-th largest element: bisect the top 16 key bits of the per-thread maxima of the
         // first chunk with CTA-wide counts; the result never exceeds the k-th largest maximum.
         float tmax = -INFINITY;
         bool has = false;
-        if (ok) {
-          for (int r = 0; r < nround; ++r) {
-            const int f = r * G1R_T + tid;
-            if (f < nfrag) {
-              Frag<T> x;
-              x.unpack(stage[f]);
+        for (int f0 = 0; f0 + tid < nfrag; f0 += G1R_T) {
+          Frag<T> x;
+          x.unpack(stage[f0]);
 #pragma unroll
-              for (int j = 0; j < VEC; ++j) tmax = fmaxf(tmax, x.x[j]);
-              has = true;
-            }
-          }
+          for (int j = 0; j < VEC; ++j) tmax = fmaxf(tmax, x.x[j]);
+          has = true;
         }
         const uint32_t mykey = has ? f2key(tmax) : 0u;
         uint32_t lob = 0;
@@ -370,58 +431,123 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
         __syncthreads();
       }
 
+      GT(3);
       const float taux = sh.taux;
-      if (ok) {
-        for (int r = 0; r < nround; ++r) {  // warp-uniform trip count: the votes need every lane
-          const int f = r * G1R_T + tid;
-          float x[VEC];
-          if (f < nfrag) {
-            Frag<T> fr;
-            fr.unpack(stage[f]);
+      int f0 = 0;
+      for (; f0 + G1R_GROUP * G1R_T <= nfrag; f0 += G1R_GROUP * G1R_T) {  // full groups: no bounds checks
+        float x[G1R_GROUP][VEC];
+        float vmax[G1R_GROUP];
 #pragma unroll
-            for (int j = 0; j < VEC; ++j) x[j] = fr.x[j];
-          } else {
+        for (int u = 0; u < G1R_GROUP; ++u) {
+          Frag<T> fr;
+          fr.unpack(stage[f0 + u * G1R_T]);
+          vmax[u] = fr.x[0];
 #pragma unroll
-            for (int j = 0; j < VEC; ++j) x[j] = -INFINITY;
-          }
-          float vmax = x[0];
+          for (int j = 0; j < VEC; ++j) { x[u][j] = fr.x[j]; vmax[u] = fmaxf(vmax[u], fr.x[j]); }
+        }
+        const float gmax = fmaxf(fmaxf(vmax[0], vmax[1]), fmaxf(vmax[2], vmax[3]));
+        if (__any_sync(FULL, gmax > taux)) {  // rare: a candidate somewhere in the warp's 4 fragments
+          if (gmax > ref + 60.f || (ref < -1.0e29f && gmax > -INFINITY)) {  // move the reference up
+            const float sc = ex2_approx(fmaf(ref, kLog2e, -gmax * kLog2e));
 #pragma unroll
-          for (int j = 1; j < VEC; ++j) vmax = fmaxf(vmax, x[j]);
-          if (__any_sync(FULL, vmax > taux)) {
-            if (vmax > ref + 60.f || (ref < -1.0e29f && vmax > -INFINITY)) {  // move the reference up
-              s_t *= ex2_approx(fmaf(ref, kLog2e, -vmax * kLog2e));
-              ref = vmax;
-              negref = -vmax * kLog2e;
-            }
-            const int col0 = sg.col0 + c + f * VEC;
-#pragma unroll
-            for (int j = 0; j < VEC; ++j) {
-              const bool hit = x[j] > taux;
-              const unsigned mask = __ballot_sync(FULL, hit);
-              if (mask) {
-                const int leader = __ffs(mask) - 1;
-                int at = 0;
-                if (lane == leader) at = atomicAdd(&sh.cnt, __popc(mask));
-                at = __shfl_sync(FULL, at, leader);
-                if (hit) pool[at + __popc(mask & ((1u << lane) - 1))] = col0 + j;
-              }
-            }
+            for (int u = 0; u < G1R_GROUP; ++u) acc[u] *= sc;
+            ref = gmax;
+            negref = -gmax * kLog2e;
           }
 #pragma unroll
-          for (int j = 0; j < VEC; ++j) s_t += ex2_approx(fmaf(x[j], kLog2e, negref));
+          for (int u = 0; u < G1R_GROUP; ++u)
+            if (vmax[u] > taux) append_hits<VEC>(sh, x[u], taux, colbase + (f0 + u * G1R_T) * VEC);
+        }
+#pragma unroll
+        for (int u = 0; u < G1R_GROUP; ++u) {
+#pragma unroll
+          for (int j = 0; j < VEC; ++j) acc[u] += ex2_approx(fmaf(x[u][j], kLog2e, negref));
         }
       }
-      // One barrier frees the stage and takes the flush decision on the final hit count (see the comment
-      // in k_lse_topk); a failed wait skips the flush and is seen by everybody at the next chunk.
-      const bool want = *reinterpret_cast<volatile int*>(&sh.cnt) >= 4 * k;
-      if (__syncthreads_or(want)) flush_pool<T, G1R_T>(sh, pool, rowp, V, k);
+      for (; f0 < nfrag; f0 += G1R_T) {  // ragged end of a chunk, one fragment per vote
+        float x[VEC];
+        if (f0 + tid < nfrag) {
+          Frag<T> fr;
+          fr.unpack(stage[f0]);
+#pragma unroll
+          for (int j = 0; j < VEC; ++j) x[j] = fr.x[j];
+        } else {
+#pragma unroll
+          for (int j = 0; j < VEC; ++j) x[j] = -INFINITY;
+        }
+        float vm = x[0];
+#pragma unroll
+        for (int j = 1; j < VEC; ++j) vm = fmaxf(vm, x[j]);
+        if (__any_sync(FULL, vm > taux)) {
+          if (vm > ref + 60.f || (ref < -1.0e29f && vm > -INFINITY)) {
+            const float sc = ex2_approx(fmaf(ref, kLog2e, -vm * kLog2e));
+#pragma unroll
+            for (int u = 0; u < G1R_GROUP; ++u) acc[u] *= sc;
+            ref = vm;
+            negref = -vm * kLog2e;
+          }
+          if (vm > taux) append_hits<VEC>(sh, x, taux, colbase + f0 * VEC);
+        }
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) acc[0] += ex2_approx(fmaf(x[j], kLog2e, negref));
+      }
+
+      GT(4);
+      // One barrier takes the decision on the final hit count (see the comment in k_lse_topk): rank the pool
+      // now?  Inside the branch nobody is ahead in the next chunk, so the counter can be read plainly.
+      if (__syncthreads_or(*reinterpret_cast<volatile int*>(&sh.cnt) >= k)) {
+        GT(5);
+#ifdef UBT_G1_TIMING
+        ++nflush;
+#endif
+        const bool overflow = sh.cnt > G1R_POOL;
+        flush_keyed(sh, k);  // ranks what the pool holds; tightens the threshold
+        if (overflow) {
+          // The chunk produced more hits than the pool holds and the surplus was dropped.  Walk the chunk
+          // again in slices of 64 fragments, ranking after each slice so that the pool cannot overflow; a
+          // hit that already sits in the carried list (it was ranked above) is not added twice.  The walk
+          // admits elements EQUAL to the current k-th value too: a dropped one may have the lower column.
+          const uint4* st0 = stage - tid;
+          for (int g0 = 0; g0 < nfrag; g0 += 64) {
+            const float tx = next_below(sh.taux);
+            if (tid < 64) {  // two whole warps
+              float x[VEC];
+              const int f = g0 + tid;
+              if (f < nfrag) {
+                Frag<T> fr;
+                fr.unpack(st0[f]);
+#pragma unroll
+                for (int j = 0; j < VEC; ++j) x[j] = fr.x[j];
+              } else {
+#pragma unroll
+                for (int j = 0; j < VEC; ++j) x[j] = -INFINITY;
+              }
+              const int col0 = sg.col0 + c + f * VEC;
+              const int nt = sh.ntop;
+#pragma unroll
+              for (int j = 0; j < VEC; ++j) {
+                if (x[j] > tx) {
+                  const unsigned long long key = make_key(x[j], col0 + j);
+                  for (int q = 0; q < nt; ++q)
+                    if (sh.top[q] == key) x[j] = -INFINITY;  // already ranked
+                }
+              }
+              append_hits<VEC>(sh, x, tx, col0);
+            }
+            __syncthreads();
+            flush_keyed(sh, k);
+          }
+        }
+      }
+      GT(6);
       rp.next();
       ++consumed;
     }
     if (failed) break;
-    flush_pool<T, G1R_T>(sh, pool, rowp, V, k);
+    flush_keyed(sh, k);
 
     // partial (max, sum exp) of the segment from the per-thread (reference, sum) pairs
+    const float s_t = (acc[0] + acc[1]) + (acc[2] + acc[3]);
     float mw = ref;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mw = fmaxf(mw, __shfl_xor_sync(FULL, mw, o));
@@ -432,13 +558,13 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
     float sw = s_t * ex2_approx((ref - M) * kLog2e);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sw += __shfl_xor_sync(FULL, sw, o);
-    if (lane == 0) sh.redf[G1_T / 32 + (tid >> 5)] = sw;
+    if (lane == 0) sh.redf[NW + (tid >> 5)] = sw;
     __syncthreads();
     const int64_t c_first = (sg.row * (int64_t)V) / plan.span;
     const int64_t slot = sg.row * plan.smax + ((int64_t)blockIdx.x - c_first);
     if (tid == 0) {
       float S = 0.f;
-      for (int w = 0; w < NW; ++w) S += sh.redf[G1_T / 32 + w];
+      for (int w = 0; w < NW; ++w) S += sh.redf[NW + w];
       g_ms[slot * 2] = M;
       g_ms[slot * 2 + 1] = S;
       g_cnt[slot] = sh.ntop;
@@ -449,9 +575,15 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
     }
     __syncthreads();
     pos += sg.len;
+    GT(7);
   }
   __syncthreads();
-  if (tid == 0 && *reinterpret_cast<volatile int*>(&s_fail)) prod.drain(consumed > 0 ? consumed - 1 : 0, full);
+  if (tid == 0 && *reinterpret_cast<volatile int*>(&sh.fail)) prod.drain(consumed > 0 ? consumed - 1 : 0, full);
+#ifdef UBT_G1_TIMING
+  if (tid == 32 && (blockIdx.x == 0 || blockIdx.x == 100 || blockIdx.x == 300))
+    printf("g1 cta %d chunks %d flushes %d cycles: top %lld issue %lld wait %lld bisect %lld process %lld vote %lld flush %lld segend %lld\n", blockIdx.x,
+           consumed, nflush, tt[0], tt[1], tt[2], tt[3], tt[4], tt[5], tt[6], tt[7]);
+#endif
 }
 
 // One warp per row: combine the partials of the row's segments (see merge_row_warp in ubt_merge.cuh).
@@ -478,7 +610,7 @@ SpanPlan make_span_plan(int64_t rows, int V, int ctas, int64_t min_span) {
 }
 
 SpanPlan topk_plan(int64_t rows, int V) {
-  return make_span_plan(rows, V, device_info().sm_count * 2, 32768);
+  return make_span_plan(rows, V, device_info().sm_count * G1R_CTAS, 32768);
 }
 
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -517,8 +649,7 @@ static cudaError_t launch_lse_topk_t(const void* logits, int64_t rows, int V, in
 template <typename T>
 static cudaError_t launch_lse_topk_ring_t(const void* logits, int64_t rows, int V, int k, const TopkWorkspace& w,
                                           cudaStream_t st) {
-  constexpr int kStageElems = G1R_STAGE_BYTES / (int)sizeof(T);
-  const size_t smem = (size_t)G1R_STAGES * G1R_STAGE_BYTES + sizeof(G1Shared) + sizeof(int) * (size_t)(kStageElems + G1_SLACK);
+  const size_t smem = (size_t)G1R_STAGES * G1R_STAGE_BYTES + sizeof(G1RShared);
   auto kern = k_lse_topk_ring<T>;
   static bool configured = false;
   if (!configured) {
