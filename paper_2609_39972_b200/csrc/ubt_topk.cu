@@ -282,7 +282,7 @@ k_lse_topk(const T* __restrict__ logits, int64_t total, int V, int k, SpanPlan p
 // Hits go to a small pool of (value, column) keys, so ranking the pool touches shared memory only.  A chunk
 // that overflows the pool (possible only for pathological rows, e.g. long runs of equal values before the
 // threshold turns strict) has its hits discarded and is walked again in slices that cannot overflow.
-constexpr int G1R_T = 256, G1R_STAGES = 4, G1R_STAGE_BYTES = 16384, G1R_CTAS = 3;
+constexpr int G1R_T = 256, G1R_STAGES = 2, G1R_STAGE_BYTES = 32768, G1R_CTAS = 3;
 constexpr int G1R_POOL = 1024;  // hit pool entries
 constexpr int G1R_GROUP = 4;    // fragments per vote
 
