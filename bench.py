@@ -183,10 +183,13 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time budget of the oracle baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override B of the workload (profiling captures only)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
     cfg = synth.CONFIGS[args.workload]
+    if args.batch > 0:
+        cfg = cfg.replace(B=args.batch, name=f"{cfg.name}-B{args.batch}")
     world, rank, local = dist_setup(args.gpus)
 
     if args.impl == "reference":

@@ -186,7 +186,7 @@ int ubt_verify_tree(const ubt_tree* tree, const void* target_logits, int dtype, 
     if (launch_row_argmax(target_logits, dtype, rows, V, w, st) != cudaSuccess) return UBT_ERR_CUDA;
   } else {
     int32_t* pick = o->node_pick ? o->node_pick : w.pick;
-    if (launch_row_sample(target_logits, dtype, B, N, V, o->seed, o->temperature, pick, st) != cudaSuccess)
+    if (launch_row_sample(target_logits, dtype, B, N, V, o->seed, o->temperature, pick, w, st) != cudaSuccess)
       return UBT_ERR_CUDA;
     sampled = pick;
   }

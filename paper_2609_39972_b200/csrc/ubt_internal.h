@@ -78,13 +78,16 @@ struct VerifyWorkspace {
   SpanPlan plan;                 // greedy: spans of the row-argmax kernel
   unsigned long long* part_key;  // greedy: [B*N, smax] (value, ~token) keys
   int32_t* pick;                 // sampling: [B*N] picks when the caller gave no node_pick
+  float* row_ac;                 // sampling: [B*N, 2] per-row constants (a, c) of the weight routine
+  unsigned long long* block_sum; // sampling: [B*N, nblocks] sums of the integer weights per 1024 tokens
+  int nblocks;
 };
 size_t verify_workspace_bytes(int64_t rows, int V, int mode);
 VerifyWorkspace carve_verify_workspace(void* ws, int64_t rows, int V, int mode);
 cudaError_t launch_row_argmax(const void* logits, int dtype, int64_t rows, int V,
                               const VerifyWorkspace& w, cudaStream_t st);
 cudaError_t launch_row_sample(const void* logits, int dtype, int B, int N, int V, uint64_t seed,
-                              float temperature, int32_t* pick, cudaStream_t st);
+                              float temperature, int32_t* pick, const VerifyWorkspace& w, cudaStream_t st);
 cudaError_t launch_walk(const ubt_tree& tree, int mode, const VerifyWorkspace& w, int V,
                         const int32_t* sampled_pick, int32_t* node_pick,
                         const ubt_verify_result& out, cudaStream_t st);

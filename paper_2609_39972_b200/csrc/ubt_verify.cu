@@ -280,8 +280,218 @@ __device__ __forceinline__ unsigned long long weight_of(float z, float a, float 
   return __float2ull_rz(__uint_as_float(e));
 }
 
+constexpr int G5_CHUNK = 1024;  // tokens per partial sum
+
+// One warp: from the per-1024-token sums of a row's integer weights to the sampled token.  total = sum of
+// the sums; theta = floor(R * total / 2^64) with R from Philox4x32-10(counter = (slot, b, 0, 0), key = seed);
+// the pick is the first token whose inclusive prefix sum exceeds theta.  All lanes return the pick.
+template <typename T>
+__device__ int locate_pick(const T* rowp, int V, float a, float c, const unsigned long long* csum, int nchunks,
+                           uint64_t seed, uint32_t b, uint32_t slot, int lane) {
+  unsigned long long run = 0;
+  for (int ch = lane; ch < nchunks; ch += 32) run += csum[ch];
+  const unsigned long long total = warp_sum_u64(run);
+  uint32_t x[4];
+  philox4x32_10(slot, b, 0u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), x);
+  const unsigned long long R = (unsigned long long)x[0] | ((unsigned long long)x[1] << 32);
+  unsigned long long theta = __umul64hi(R, total);
+  // sequential over groups of 32 chunks, warp scan inside a group
+  int found_chunk = nchunks - 1;
+  unsigned long long before = 0;
+  bool done = false;
+  for (int g = 0; g < nchunks && !done; g += 32) {
+    const unsigned long long v = (g + lane < nchunks) ? csum[g + lane] : 0ull;
+    unsigned long long inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      unsigned long long up = __shfl_up_sync(FULL, inc, o);
+      if (lane >= o) inc += up;
+    }
+    const unsigned hit = __ballot_sync(FULL, before + inc > theta && g + lane < nchunks);
+    if (hit) {
+      const int l = __ffs(hit) - 1;
+      found_chunk = g + l;
+      before += __shfl_sync(FULL, inc - v, l);
+      done = true;
+    } else {
+      before += __shfl_sync(FULL, inc, 31);
+    }
+  }
+  theta -= before;  // threshold relative to the chunk start
+  // every lane takes 32 consecutive tokens of the chunk
+  const int t0 = found_chunk * G5_CHUNK + lane * (G5_CHUNK / 32);
+  unsigned long long lsum = 0;
+  for (int j = 0; j < G5_CHUNK / 32; ++j) {
+    const int tkn = t0 + j;
+    lsum += tkn < V ? weight_of(load_elem(rowp, tkn), a, c) : 0ull;
+  }
+  unsigned long long inc = lsum;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    unsigned long long up = __shfl_up_sync(FULL, inc, o);
+    if (lane >= o) inc += up;
+  }
+  const unsigned hit = __ballot_sync(FULL, inc > theta);
+  const int l = hit ? __ffs(hit) - 1 : 31;
+  int ans = t0 + G5_CHUNK / 32 - 1;
+  if (lane == l) {
+    unsigned long long run2 = inc - lsum;
+    for (int j = 0; j < G5_CHUNK / 32; ++j) {
+      const int tkn = t0 + j;
+      run2 += tkn < V ? weight_of(load_elem(rowp, tkn), a, c) : 0ull;
+      if (run2 > theta) { ans = tkn; break; }
+    }
+    ans = ans < V ? ans : V - 1;
+  }
+  return __shfl_sync(FULL, ans, l);
+}
+
+// ---------------------------------------------------------------------------- sampling picks, ring-fed
+// Every CTA owns whole rows and walks each of them twice through the bulk-copy ring: first for the row
+// maximum, then (served by L2: a row is 0.3 MB and only one row per SM is in flight) for the integer weights,
+// of which it stores one sum per 1024 tokens.  A second small kernel, one warp per row, turns the sums into
+// the pick.  HBM traffic stays at one read of every logit; the weight arithmetic is what bounds this kernel.
+constexpr int G5R_T = 512, G5R_STAGES = 3, G5R_STAGE_BYTES = 65536;
+
+template <typename T>
+struct RowTwiceProducer {  // thread 0: chunks of row r (pass 0), the same chunks again (pass 1), then row r+1
+  static constexpr int kStageElems = G5R_STAGE_BYTES / (int)sizeof(T);
+  int64_t row, row_end;
+  int V, col, pass, stage, issued;
+  __device__ __forceinline__ void init(int64_t r0, int64_t r1, int V_) {
+    row = r0; row_end = r1; V = V_; col = 0; pass = 0; stage = 0; issued = 0;
+  }
+  __device__ __forceinline__ void issue_one(const T* base, unsigned char* ring, uint64_t* full) {
+    if (row >= row_end) return;
+    const int l = V - col < kStageElems ? V - col : kStageElems;
+    mbar_expect_tx(&full[stage], (uint32_t)(l * sizeof(T)));
+    bulk_load(ring + (size_t)stage * G5R_STAGE_BYTES, base + row * V + col, (uint32_t)(l * sizeof(T)), &full[stage]);
+    col += l;
+    if (col == V) { col = 0; if (pass == 0) pass = 1; else { pass = 0; ++row; } }
+    if (++stage == G5R_STAGES) stage = 0;
+    ++issued;
+  }
+  __device__ __forceinline__ void drain(int consumed, uint64_t* full) {
+    for (int i = consumed; i < issued; ++i) mbar_wait(&full[i % G5R_STAGES], (uint32_t)(i / G5R_STAGES) & 1u);
+  }
+};
+
+template <typename T>
+__global__ void __launch_bounds__(G5R_T, 1)
+k_row_weights_ring(const T* __restrict__ logits, int64_t rows, int V, float temperature,
+                   float* __restrict__ row_ac, unsigned long long* __restrict__ block_sum, int nblocks) {
+  extern __shared__ __align__(128) unsigned char ring[];
+  __shared__ uint64_t full[G5R_STAGES];
+  __shared__ float redf[G5R_T / 32];
+  __shared__ int s_fail;
+  constexpr int VEC = 16 / (int)sizeof(T);
+  constexpr int STAGE_ELEMS = G5R_STAGE_BYTES / (int)sizeof(T);
+  constexpr int BF = G5_CHUNK / VEC;  // fragments per 1024-token block
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int64_t r0 = rows * blockIdx.x / gridDim.x, r1 = rows * (blockIdx.x + 1) / gridDim.x;
+  pdl_launch_dependents();
+  if (r0 >= r1) return;
+  if (tid == 0) {
+    for (int s = 0; s < G5R_STAGES; ++s) mbar_init(&full[s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    s_fail = 0;
+  }
+  __syncthreads();
+  RowTwiceProducer<T> prod;
+  if (tid == 0) {
+    prod.init(r0, r1, V);
+    for (int i = 0; i < G5R_STAGES - 1; ++i) prod.issue_one(logits, ring, full);
+  }
+  RingPos<G5R_STAGES> rp;
+  rp.init();
+  int consumed = 0;
+  bool failed = false;
+  const float inv_t = __fdiv_rn(1.0f, temperature);
+  const float a = __fmul_rn(0x1.715476p+0f, inv_t);
+
+  for (int64_t row = r0; row < r1 && !failed; ++row) {
+    // ---- pass 1: the row maximum
+    float m = -INFINITY;
+    for (int c0 = 0; c0 < V; c0 += STAGE_ELEMS) {
+      const int l = V - c0 < STAGE_ELEMS ? V - c0 : STAGE_ELEMS;
+      if (*reinterpret_cast<volatile int*>(&s_fail)) { failed = true; break; }
+      if (tid == 0) prod.issue_one(logits, ring, full);
+      if (mbar_wait(&full[rp.stage], rp.parity)) {
+        const uint4* stage = reinterpret_cast<const uint4*>(ring + (size_t)rp.stage * G5R_STAGE_BYTES);
+        const int nfrag = l / VEC;
+#pragma unroll 4
+        for (int f = tid; f < nfrag; f += G5R_T) m = fmaxf(m, frag_max(stage[f], (const T*)nullptr));
+      } else {
+        s_fail = 1;
+      }
+      __syncthreads();
+      rp.next();
+      ++consumed;
+    }
+    if (failed) break;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(FULL, m, o));
+    if (lane == 0) redf[warp] = m;
+    __syncthreads();
+    m = redf[0];
+    for (int w = 1; w < G5R_T / 32; ++w) m = fmaxf(m, redf[w]);
+    const float c = -__fmul_rn(m, a);
+    if (tid == 0) { row_ac[row * 2] = a; row_ac[row * 2 + 1] = c; }
+    // ---- pass 2: integer weights, one sum per 1024-token block (a warp owns a block)
+    for (int c0 = 0; c0 < V; c0 += STAGE_ELEMS) {
+      const int l = V - c0 < STAGE_ELEMS ? V - c0 : STAGE_ELEMS;
+      if (*reinterpret_cast<volatile int*>(&s_fail)) { failed = true; break; }
+      if (tid == 0) prod.issue_one(logits, ring, full);
+      if (mbar_wait(&full[rp.stage], rp.parity)) {
+        const uint4* stage = reinterpret_cast<const uint4*>(ring + (size_t)rp.stage * G5R_STAGE_BYTES);
+        const int nfrag = l / VEC;
+        const int nblk = (nfrag + BF - 1) / BF;
+        for (int blk = warp; blk < nblk; blk += G5R_T / 32) {
+          unsigned long long acc = 0;
+#pragma unroll
+          for (int q = 0; q < BF / 32; ++q) {
+            const int f = blk * BF + q * 32 + lane;
+            if (f < nfrag) {
+              Frag<T> x;
+              x.unpack(stage[f]);
+#pragma unroll
+              for (int j = 0; j < VEC; ++j) acc += weight_of(x.x[j], a, c);
+            }
+          }
+          acc = warp_sum_u64(acc);
+          if (lane == 0) block_sum[row * nblocks + c0 / G5_CHUNK + blk] = acc;
+        }
+      } else {
+        s_fail = 1;
+      }
+      __syncthreads();  // frees the stage; also separates redf's use in consecutive rows
+      rp.next();
+      ++consumed;
+    }
+  }
+  __syncthreads();
+  if (tid == 0 && *reinterpret_cast<volatile int*>(&s_fail)) prod.drain(consumed > 0 ? consumed - 1 : 0, full);
+  if (tid == 0) pdl_wait();  // started early, like the greedy kernel: do not complete before the tree builder
+}
+
+// One warp per row: block sums -> pick.
+template <typename T>
+__global__ void __launch_bounds__(128)
+k_row_pick(const T* __restrict__ logits, int64_t rows, int N, int V, uint64_t seed,
+           const float* __restrict__ row_ac, const unsigned long long* __restrict__ block_sum, int nblocks,
+           int32_t* __restrict__ pick) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  pdl_wait();
+  pdl_launch_dependents();
+  if (row >= rows) return;
+  const int ans = locate_pick<T>(logits + row * V, V, row_ac[row * 2], row_ac[row * 2 + 1],
+                                 block_sum + row * nblocks, nblocks, seed, (uint32_t)(row / N), (uint32_t)(row % N), lane);
+  if (lane == 0) pick[row] = ans;
+}
+
 constexpr int G5_T = 512;
-constexpr int G5_CHUNK = 1024;     // tokens per partial sum
+
 constexpr int G5_MAXCHUNKS = 2048;  // V <= 2M
 
 template <typename T, int VEC>
@@ -340,61 +550,8 @@ k_row_sample(const T* __restrict__ logits, int64_t rows, int N, int V, uint64_t 
 
     // locate the chunk that holds the threshold, then the token inside it (warp 0)
     if (warp == 0) {
-      unsigned long long run = 0;
-      for (int ch = lane; ch < nchunks; ch += 32) run += csum[ch];
-      const unsigned long long total = warp_sum_u64(run);
-      uint32_t x[4];
-      philox4x32_10((uint32_t)(row % N), (uint32_t)(row / N), 0u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), x);
-      const unsigned long long R = (unsigned long long)x[0] | ((unsigned long long)x[1] << 32);
-      unsigned long long theta = __umul64hi(R, total);
-      // sequential over groups of 32 chunks, warp scan inside a group
-      int found_chunk = nchunks - 1;
-      unsigned long long before = 0;
-      bool done = false;
-      for (int g = 0; g < nchunks && !done; g += 32) {
-        const unsigned long long v = (g + lane < nchunks) ? csum[g + lane] : 0ull;
-        unsigned long long inc = v;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          unsigned long long up = __shfl_up_sync(FULL, inc, o);
-          if (lane >= o) inc += up;
-        }
-        const unsigned hit = __ballot_sync(FULL, before + inc > theta && g + lane < nchunks);
-        if (hit) {
-          const int l = __ffs(hit) - 1;
-          found_chunk = g + l;
-          before += __shfl_sync(FULL, inc - v, l);
-          done = true;
-        } else {
-          before += __shfl_sync(FULL, inc, 31);
-        }
-      }
-      theta -= before;  // threshold relative to the chunk start
-      // every lane takes 32 consecutive tokens of the chunk
-      const int t0 = found_chunk * G5_CHUNK + lane * (G5_CHUNK / 32);
-      unsigned long long lsum = 0;
-      for (int j = 0; j < G5_CHUNK / 32; ++j) {
-        const int tkn = t0 + j;
-        lsum += tkn < V ? weight_of(load_elem(rowp, tkn), a, c) : 0ull;
-      }
-      unsigned long long inc = lsum;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        unsigned long long up = __shfl_up_sync(FULL, inc, o);
-        if (lane >= o) inc += up;
-      }
-      const unsigned hit = __ballot_sync(FULL, inc > theta);
-      const int l = hit ? __ffs(hit) - 1 : 31;
-      if (lane == l) {
-        unsigned long long run2 = inc - lsum;
-        int ans = t0 + G5_CHUNK / 32 - 1;
-        for (int j = 0; j < G5_CHUNK / 32; ++j) {
-          const int tkn = t0 + j;
-          run2 += tkn < V ? weight_of(load_elem(rowp, tkn), a, c) : 0ull;
-          if (run2 > theta) { ans = tkn; break; }
-        }
-        pick[row] = ans < V ? ans : V - 1;
-      }
+      const int ans = locate_pick<T>(rowp, V, a, c, csum, nchunks, seed, (uint32_t)(row / N), (uint32_t)(row % N), lane);
+      if (lane == 0) pick[row] = ans;
     }
     __syncthreads();
   }
@@ -469,7 +626,9 @@ size_t verify_workspace_bytes(int64_t rows, int V, int mode) {
     const SpanPlan p = argmax_plan(rows, V);
     return align_up((size_t)rows * p.smax * sizeof(unsigned long long), 256);
   }
-  return align_up((size_t)rows * sizeof(int32_t), 256);
+  const size_t nblocks = ((size_t)V + G5_CHUNK - 1) / G5_CHUNK;
+  return align_up((size_t)rows * sizeof(int32_t), 256) + align_up((size_t)rows * 2 * sizeof(float), 256) +
+         align_up((size_t)rows * nblocks * sizeof(unsigned long long), 256);
 }
 
 VerifyWorkspace carve_verify_workspace(void* ws, int64_t rows, int V, int mode) {
@@ -479,7 +638,11 @@ VerifyWorkspace carve_verify_workspace(void* ws, int64_t rows, int V, int mode) 
     w.part_key = static_cast<unsigned long long*>(ws);
   } else {
     w.plan = SpanPlan{0, 0, 0};
-    w.pick = static_cast<int32_t*>(ws);
+    unsigned char* p = static_cast<unsigned char*>(ws);
+    w.pick = reinterpret_cast<int32_t*>(p); p += align_up((size_t)rows * sizeof(int32_t), 256);
+    w.row_ac = reinterpret_cast<float*>(p); p += align_up((size_t)rows * 2 * sizeof(float), 256);
+    w.block_sum = reinterpret_cast<unsigned long long*>(p);
+    w.nblocks = (V + G5_CHUNK - 1) / G5_CHUNK;
   }
   return w;
 }
@@ -535,10 +698,38 @@ static cudaError_t launch_row_sample_t(const void* logits, int64_t rows, int N, 
   return cudaGetLastError();
 }
 
+template <typename T>
+static cudaError_t launch_row_sample_ring_t(const void* logits, int64_t rows, int N, int V, uint64_t seed,
+                                            float temperature, int32_t* pick, const VerifyWorkspace& w,
+                                            cudaStream_t st) {
+  auto kern = k_row_weights_ring<T>;
+  constexpr int kBytes = G5R_STAGES * G5R_STAGE_BYTES;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBytes);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  int grid = device_info().sm_count;
+  if ((int64_t)grid > rows) grid = (int)rows;
+  cudaError_t e = launch_kernel(kern, dim3(grid), dim3(G5R_T), kBytes, st, true, static_cast<const T*>(logits), rows, V,
+                                temperature, w.row_ac, w.block_sum, w.nblocks);
+  if (e != cudaSuccess) return e;
+  const int warps = 4;
+  return launch_kernel(k_row_pick<T>, dim3((unsigned)((rows + warps - 1) / warps)), dim3(warps * 32), 0, st, true,
+                       static_cast<const T*>(logits), rows, N, V, seed, (const float*)w.row_ac,
+                       (const unsigned long long*)w.block_sum, w.nblocks, pick);
+}
+
 cudaError_t launch_row_sample(const void* logits, int dtype, int B, int N, int V, uint64_t seed,
-                              float temperature, int32_t* pick, cudaStream_t st) {
+                              float temperature, int32_t* pick, const VerifyWorkspace& w, cudaStream_t st) {
   const int64_t rows = (int64_t)B * N;
   if (rows == 0) return cudaSuccess;
+  // rows that are whole 16-byte fragments go through the bulk-copy ring; other V use plain loads
+  if (dtype == UBT_BF16 && V % 8 == 0)
+    return launch_row_sample_ring_t<__nv_bfloat16>(logits, rows, N, V, seed, temperature, pick, w, st);
+  if (dtype == UBT_F32 && V % 4 == 0)
+    return launch_row_sample_ring_t<float>(logits, rows, N, V, seed, temperature, pick, w, st);
   if (dtype == UBT_BF16) {
     if (V % 8 == 0) return launch_row_sample_t<__nv_bfloat16, 8>(logits, rows, N, V, seed, temperature, pick, st);
     return launch_row_sample_t<__nv_bfloat16, 1>(logits, rows, N, V, seed, temperature, pick, st);
