@@ -280,6 +280,57 @@ __device__ __forceinline__ unsigned long long weight_of(float z, float a, float 
   return __float2ull_rz(__uint_as_float(e));
 }
 
+// Two weights at once with the packed fp32 instructions of sm_100 (fma/add .f32x2): the same IEEE operations
+// per component as weight_of, half the issue slots for the arithmetic part.
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+struct WeightConsts2 {  // the routine's constants, duplicated into both halves
+  unsigned long long a, c, big, nbig, none, c5, c4, c3, c2, c1, one;
+  __device__ __forceinline__ void init(float a_, float c_) {
+    a = pack2(a_, a_); c = pack2(c_, c_);
+    big = pack2(12582912.0f, 12582912.0f); nbig = pack2(-12582912.0f, -12582912.0f);
+    none = pack2(-1.0f, -1.0f);
+    c5 = pack2(0x1.5c7746p-10f, 0x1.5c7746p-10f); c4 = pack2(0x1.3cea8p-7f, 0x1.3cea8p-7f);
+    c3 = pack2(0x1.c6b54ap-5f, 0x1.c6b54ap-5f); c2 = pack2(0x1.ebf9bcp-3f, 0x1.ebf9bcp-3f);
+    c1 = pack2(0x1.62e42cp-1f, 0x1.62e42cp-1f); one = pack2(1.0f, 1.0f);
+  }
+};
+__device__ __forceinline__ unsigned long long weight_pair_sum(float z0, float z1, const WeightConsts2& k) {
+  float y0, y1;
+  unpack2(fma2(pack2(z0, z1), k.a, k.c), y0, y1);
+  const unsigned long long y = pack2(fmaxf(y0, -42.0f), fmaxf(y1, -42.0f));
+  const unsigned long long tmp = add2(y, k.big);
+  const unsigned long long nf = add2(tmp, k.nbig);  // tmp - big
+  const unsigned long long f = fma2(nf, k.none, y);  // y - nf, exact like the scalar subtraction
+  unsigned long long p = fma2(k.c5, f, k.c4);
+  p = fma2(p, f, k.c3);
+  p = fma2(p, f, k.c2);
+  p = fma2(p, f, k.c1);
+  p = fma2(p, f, k.one);
+  float p0, p1, t0, t1;
+  unpack2(p, p0, p1);
+  unpack2(tmp, t0, t1);
+  const uint32_t e0 = __float_as_uint(p0) + ((__float_as_uint(t0) + 40u) << 23);
+  const uint32_t e1 = __float_as_uint(p1) + ((__float_as_uint(t1) + 40u) << 23);
+  return __float2ull_rz(__uint_as_float(e0)) + __float2ull_rz(__uint_as_float(e1));
+}
+
 constexpr int G5_CHUNK = 1024;  // tokens per partial sum
 
 // One warp: from the per-1024-token sums of a row's integer weights to the sampled token.  total = sum of
@@ -351,7 +402,7 @@ __device__ int locate_pick(const T* rowp, int V, float a, float c, const unsigne
 // maximum, then (served by L2: a row is 0.3 MB and only one row per SM is in flight) for the integer weights,
 // of which it stores one sum per 1024 tokens.  A second small kernel, one warp per row, turns the sums into
 // the pick.  HBM traffic stays at one read of every logit; the weight arithmetic is what bounds this kernel.
-constexpr int G5R_T = 512, G5R_STAGES = 3, G5R_STAGE_BYTES = 65536;
+constexpr int G5R_T = 512, G5R_STAGES = 3, G5R_STAGE_BYTES = 32768, G5R_CTAS = 2;
 
 template <typename T>
 struct RowTwiceProducer {  // thread 0: chunks of row r (pass 0), the same chunks again (pass 1), then row r+1
@@ -377,7 +428,7 @@ struct RowTwiceProducer {  // thread 0: chunks of row r (pass 0), the same chunk
 };
 
 template <typename T>
-__global__ void __launch_bounds__(G5R_T, 1)
+__global__ void __launch_bounds__(G5R_T, G5R_CTAS)
 k_row_weights_ring(const T* __restrict__ logits, int64_t rows, int V, float temperature,
                    float* __restrict__ row_ac, unsigned long long* __restrict__ block_sum, int nblocks) {
   extern __shared__ __align__(128) unsigned char ring[];
@@ -437,6 +488,8 @@ k_row_weights_ring(const T* __restrict__ logits, int64_t rows, int V, float temp
     for (int w = 1; w < G5R_T / 32; ++w) m = fmaxf(m, redf[w]);
     const float c = -__fmul_rn(m, a);
     if (tid == 0) { row_ac[row * 2] = a; row_ac[row * 2 + 1] = c; }
+    WeightConsts2 wc;
+    wc.init(a, c);
     // ---- pass 2: integer weights, one sum per 1024-token block (a warp owns a block)
     for (int c0 = 0; c0 < V; c0 += STAGE_ELEMS) {
       const int l = V - c0 < STAGE_ELEMS ? V - c0 : STAGE_ELEMS;
@@ -455,7 +508,7 @@ k_row_weights_ring(const T* __restrict__ logits, int64_t rows, int V, float temp
               Frag<T> x;
               x.unpack(stage[f]);
 #pragma unroll
-              for (int j = 0; j < VEC; ++j) acc += weight_of(x.x[j], a, c);
+              for (int j = 0; j < VEC; j += 2) acc += weight_pair_sum(x.x[j], x.x[j + 1], wc);
             }
           }
           acc = warp_sum_u64(acc);
@@ -710,7 +763,7 @@ static cudaError_t launch_row_sample_ring_t(const void* logits, int64_t rows, in
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  int grid = device_info().sm_count;
+  int grid = device_info().sm_count * G5R_CTAS;
   if ((int64_t)grid > rows) grid = (int)rows;
   cudaError_t e = launch_kernel(kern, dim3(grid), dim3(G5R_T), kBytes, st, true, static_cast<const T*>(logits), rows, V,
                                 temperature, w.row_ac, w.block_sum, w.nblocks);
