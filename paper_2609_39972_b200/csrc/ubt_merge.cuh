@@ -43,21 +43,55 @@ __device__ __forceinline__ void merge_row_warp(const MergeParts& p, int64_t rows
 
   int found = 0;
   const int nq = nseg * k;
-  for (int q = lane; q < nq; q += 32) {
-    const int j = q / k, i = q - j * k;
-    if (i >= part_cnt[base + j]) continue;
-    const float val = part_val[(base + j) * k + i];
-    const int idx = part_idx[(base + j) * k + i];
-    const uint64_t key = make_key(val, idx);
-    int rank = 0;
-    for (int j2 = 0; j2 < nseg; ++j2) {
-      const int c2 = part_cnt[base + j2];
-      for (int i2 = 0; i2 < c2; ++i2)
-        rank += make_key(part_val[(base + j2) * k + i2], part_idx[(base + j2) * k + i2]) > key;
+  if (nq <= 64) {
+    // The usual case (a row is cut into a few segments): every lane takes up to two entries into registers
+    // with independent loads, and the exact ranks are counted by exchanging keys with shuffles.
+    uint64_t key[2];
+    float val[2];
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      const int q = lane + 32 * c;
+      const int j = q / k, i = q - j * k;
+      key[c] = 0ull;
+      val[c] = 0.f;
+      if (q < nq && i < part_cnt[base + j]) {
+        val[c] = part_val[(base + j) * k + i];
+        key[c] = make_key(val[c], part_idx[(base + j) * k + i]);
+      }
     }
-    if (rank < k) {
-      cand_ids[row * k + rank] = idx;
-      cand_lp[row * k + rank] = val - lse;
+    int rank[2] = {0, 0};
+#pragma unroll
+    for (int c2 = 0; c2 < 2; ++c2) {
+      const int n2 = nq - 32 * c2 < 32 ? nq - 32 * c2 : 32;
+      for (int l2 = 0; l2 < n2; ++l2) {
+        const uint64_t other = __shfl_sync(FULL, key[c2], l2);
+        rank[0] += other > key[0];
+        rank[1] += other > key[1];
+      }
+    }
+#pragma unroll
+    for (int c = 0; c < 2; ++c)
+      if (key[c] != 0ull && rank[c] < k) {
+        cand_ids[row * k + rank[c]] = key_idx(key[c]);
+        cand_lp[row * k + rank[c]] = val[c] - lse;
+      }
+  } else {
+    for (int q = lane; q < nq; q += 32) {
+      const int j = q / k, i = q - j * k;
+      if (i >= part_cnt[base + j]) continue;
+      const float val = part_val[(base + j) * k + i];
+      const int idx = part_idx[(base + j) * k + i];
+      const uint64_t key = make_key(val, idx);
+      int rank = 0;
+      for (int j2 = 0; j2 < nseg; ++j2) {
+        const int c2 = part_cnt[base + j2];
+        for (int i2 = 0; i2 < c2; ++i2)
+          rank += make_key(part_val[(base + j2) * k + i2], part_idx[(base + j2) * k + i2]) > key;
+      }
+      if (rank < k) {
+        cand_ids[row * k + rank] = idx;
+        cand_lp[row * k + rank] = val - lse;
+      }
     }
   }
   for (int j = lane; j < nseg; j += 32) found += part_cnt[base + j];

@@ -23,15 +23,15 @@
 
 namespace ubt {
 
-constexpr int G2_T = 256;
+constexpr int G2_T = 512;
 
 struct TreeSmem {
   Span<float> t;            // [L,k,k]  pair log-probabilities, each row sorted descending after set-up
   Span<unsigned char> ord;  // [L,k,k]  ord[row][j] = candidate rank of the j-th best successor
   Span<float> lp;           // [L,k]
   Span<int> tok;            // [L,k]
-  Span<uint32_t> f_key;     // mirror of the frontier (for exact score ties only), <= N entries
-  Span<uint32_t> f_info;
+  Span<float> al;           // [L]    eq. 5 weight of the base log-probability per position
+  Span<uint4> ent;          // [N+1]  frontier records of the expansion
   Span<short> nd_parent;    // accepted nodes in pop order, <= N-1; -1 = child of the root
   Span<unsigned char> nd_depth;
   Span<unsigned char> nd_rank;
@@ -56,7 +56,7 @@ __host__ __device__ inline size_t tree_carve(TreeSmem* s, unsigned char* base, i
   const long long lkk = (long long)L * k * k, lk = (long long)L * k;
   size_t o_t = take(sizeof(float) * lkk), o_ord = take((size_t)lkk);
   size_t o_lp = take(sizeof(float) * lk), o_tok = take(sizeof(int) * lk);
-  size_t o_fk = take(sizeof(uint32_t) * (N + 1)), o_fi = take(sizeof(uint32_t) * (N + 1));
+  size_t o_al = take(sizeof(float) * L), o_en = take(sizeof(uint4) * (N + 1));
   size_t o_np = take(sizeof(short) * N), o_nd = take(N), o_nr = take(N);
   size_t o_ns = take(sizeof(float) * N), o_nl = take(sizeof(short) * N);
   size_t o_pk = take(sizeof(unsigned long long) * 2 * N), o_kk = take(sizeof(int) * N);
@@ -67,8 +67,8 @@ __host__ __device__ inline size_t tree_carve(TreeSmem* s, unsigned char* base, i
     s->ord = Span<unsigned char>(base + o_ord, lkk, 102);
     s->lp = Span<float>((float*)(base + o_lp), lk, 103);
     s->tok = Span<int>((int*)(base + o_tok), lk, 104);
-    s->f_key = Span<uint32_t>((uint32_t*)(base + o_fk), N + 1, 105);
-    s->f_info = Span<uint32_t>((uint32_t*)(base + o_fi), N + 1, 106);
+    s->al = Span<float>((float*)(base + o_al), L, 105);
+    s->ent = Span<uint4>((uint4*)(base + o_en), N + 1, 106);
     s->nd_parent = Span<short>((short*)(base + o_np), N, 109);
     s->nd_depth = Span<unsigned char>(base + o_nd, N, 110);
     s->nd_rank = Span<unsigned char>(base + o_nr, N, 111);
@@ -86,31 +86,29 @@ __host__ __device__ inline size_t tree_carve(TreeSmem* s, unsigned char* base, i
 
 size_t tree_smem_bytes(int L, int k, int N) { return tree_carve(nullptr, nullptr, L, k, N); }
 
-// Frontier entry word: parent node (8 bits, 255 = the root), sibling position j in the parent's sorted
-// successor list (6), depth - 1 (6), candidate rank of the parent (6), own candidate rank (6).
-__device__ __forceinline__ uint32_t pack_info(int p, int j, int d, int pr, int r) {
-  return (uint32_t)p | ((uint32_t)j << 8) | ((uint32_t)(d - 1) << 14) | ((uint32_t)pr << 20) | ((uint32_t)r << 26);
+// A frontier entry is one 16-byte record in shared memory (entry i belongs to lane i & 31, slot i >> 5); only
+// its ordering key is mirrored in a register of the owner lane, so that finding the best entry is a register
+// scan and one warp-wide maximum.  The record holds all a pop needs:
+//   x: parent node (8 bits, 255 = the root) | sibling position j (6) | depth - 1 (6) | own candidate rank (6)
+//   y: index of its value in the sorted pair table (15 bits) | index of its first child's row (15 bits)
+//   z: score of its parent (float bits)     w: ordering key of its own score, 0 = dead
+__device__ __forceinline__ uint32_t pack_lo(int p, int j, int d, int r) {
+  return (uint32_t)p | ((uint32_t)j << 8) | ((uint32_t)(d - 1) << 14) | ((uint32_t)r << 20);
 }
 
 // Best-first expansion by one warp; returns the number of accepted nodes (all lanes agree).
+// Writes the accepted nodes in pop order: nd_parent, nd_depth, nd_rank, nd_score.
 template <int SLOTS>
-__device__ int expand_tree(TreeSmem& s, int L, int k, int budget, int W, float zeta, int bits, bool use_pk,
-                           int lane) {
-  uint32_t fk[SLOTS], fi[SLOTS];
+__device__ int expand_tree(TreeSmem& s, int L, int k, int budget, int W, float zeta, int lane) {
+  uint32_t fk[SLOTS];
 #pragma unroll
-  for (int q = 0; q < SLOTS; ++q) { fk[q] = 0u; fi[q] = 0u; }
+  for (int q = 0; q < SLOTS; ++q) fk[q] = 0u;
   int f_cnt = 0, n_acc = 0;
-  // entry idx <- (key, info); every lane calls, the owner keeps it in registers and mirrors it to shared
-  auto put = [&](int idx, uint32_t key, uint32_t info) {
-    const int ol = idx & 31, os = idx >> 5;
-#pragma unroll
-    for (int q = 0; q < SLOTS; ++q)
-      if (q == os && lane == ol) { fk[q] = key; fi[q] = info; }
-    if (lane == ol) { s.f_key[idx] = key; s.f_info[idx] = info; }
-  };
   if (budget > 0) {
     const int r0 = s.ord[0];
-    put(0, f2key(s.t[0] + zeta), pack_info(255, 0, 1, 0, r0));
+    const uint32_t key0 = f2key(s.t[0] + zeta);
+    if (lane == 0) fk[0] = key0;
+    s.ent[0] = make_uint4(pack_lo(255, 0, 1, r0), (uint32_t)((k + r0) * k) << 15, __float_as_uint(0.f), key0);
     f_cnt = 1;
   }
   __syncwarp();
@@ -120,87 +118,95 @@ __device__ int expand_tree(TreeSmem& s, int L, int k, int budget, int W, float z
     bool dup = false;
 #pragma unroll
     for (int q = 1; q < SLOTS; ++q) {
-      if (fk[q] > bk) { bk = fk[q]; bs = q; dup = false; }
-      else if (fk[q] == bk && bk != 0u) dup = true;
+      dup = fk[q] > bk ? false : (dup || (fk[q] == bk && bk != 0u));
+      bs = fk[q] > bk ? q : bs;
+      bk = fk[q] > bk ? fk[q] : bk;
     }
     const uint32_t maxk = __reduce_max_sync(FULL, bk);
     if (maxk == 0u) break;  // frontier exhausted
-    const unsigned holders = __ballot_sync(FULL, bk == maxk);
-    const bool tie = __any_sync(FULL, bk == maxk && dup) || __popc(holders) > 1;
-    int widx;
-    uint32_t winfo;
-    if (!tie) {
-      const int wl = __ffs(holders) - 1;
-      uint32_t mine = fi[0];
-#pragma unroll
-      for (int q = 1; q < SLOTS; ++q) mine = q == bs ? fi[q] : mine;
-      winfo = __shfl_sync(FULL, mine, wl);
-      widx = __shfl_sync(FULL, bs, wl) * 32 + wl;
-    } else {
-      int best = -1;
-      if (lane == 0) {  // exact score ties: depth asc, token asc, then rank path lexicographic
-        int bd = 0, bt = 0;
-        for (int i = 0; i < f_cnt; ++i) {
-          if (s.f_key[i] != maxk) continue;
-          const uint32_t inf = s.f_info[i];
-          const int d = (int)((inf >> 14) & 63u) + 1, r = (int)(inf >> 26);
-          const int tkn = s.tok[(d - 1) * k + r];
-          bool better;
-          if (best < 0) better = true;
-          else if (d != bd) better = d < bd;
-          else if (tkn != bt) better = tkn < bt;
-          else {  // same depth and token: the shallowest level where the two prefixes differ decides
-            int pa = (int)(inf & 255u), pb = (int)(s.f_info[best] & 255u), ra = 0, rb = 0;
-            pa = pa == 255 ? -1 : pa; pb = pb == 255 ? -1 : pb;
-            while (pa != pb) {
-              ra = s.nd_rank[pa]; rb = s.nd_rank[pb];
-              pa = s.nd_parent[pa]; pb = s.nd_parent[pb];
-            }
-            better = ra < rb;
+    // who holds it: lane | slot << 5 | (two equal keys in that lane) << 8; minimum and maximum over the
+    // holders agree iff there is one holder
+    const uint32_t code = (uint32_t)lane | ((uint32_t)bs << 5) | (dup ? 256u : 0u);
+    const uint32_t cmin = __reduce_min_sync(FULL, bk == maxk ? code : 0xffffffffu);
+    const uint32_t cmax = __reduce_max_sync(FULL, bk == maxk ? code : 0u);
+    int wl = (int)(cmin & 31u), ws = (int)((cmin >> 5) & 7u);
+    if (cmin != cmax || (cmin & 256u)) {
+      // Exact score ties (rare): depth asc, token asc, then rank path lexicographic, decided redundantly
+      // on all lanes from the records in shared memory.
+      int best = -1, bd = 0, bt = 0;
+      uint32_t best_lo = 0;
+      for (int i = 0; i < f_cnt; ++i) {
+        const uint4 e = s.ent[i];
+        if (e.w != maxk) continue;
+        const uint32_t el = e.x;
+        const int d = (int)((el >> 14) & 63u) + 1, r = (int)((el >> 20) & 63u);
+        const int tkn = s.tok[(d - 1) * k + r];
+        bool better;
+        if (best < 0) better = true;
+        else if (d != bd) better = d < bd;
+        else if (tkn != bt) better = tkn < bt;
+        else {  // same depth and token: the shallowest level where the two prefixes differ decides
+          int pa = (int)(el & 255u), pb = (int)(best_lo & 255u), ra = 0, rb = 0;
+          pa = pa == 255 ? -1 : pa; pb = pb == 255 ? -1 : pb;
+          while (pa != pb) {
+            ra = s.nd_rank[pa]; rb = s.nd_rank[pb];
+            pa = s.nd_parent[pa]; pb = s.nd_parent[pb];
           }
-          if (better) { best = i; bd = d; bt = tkn; }
+          better = ra < rb;
         }
+        if (better) { best = i; bd = d; bt = tkn; best_lo = el; }
       }
-      widx = __shfl_sync(FULL, best, 0);
-      winfo = s.f_info[widx];
+      wl = best & 31;
+      ws = best >> 5;
     }
-    const int p = (int)(winfo & 255u), j = (int)((winfo >> 8) & 63u), d = (int)((winfo >> 14) & 63u) + 1;
-    const int pr = (int)((winfo >> 20) & 63u), r = (int)(winfo >> 26);
+    const int e_idx = ws * 32 + wl;
+    const uint4 ent = s.ent[e_idx];
+    const uint32_t lo = ent.x, hi = ent.y;
+    const float ps = __uint_as_float(ent.z);
+    const int p = (int)(lo & 255u), j = (int)((lo >> 8) & 63u), d = (int)((lo >> 14) & 63u) + 1;
+    const int r = (int)((lo >> 20) & 63u), at = (int)(hi & 0x7fffu), cb = (int)((hi >> 15) & 0x7fffu);
     const float score = key2f(maxk);
-    const int prev = ((d - 1) * k + pr) * k;
-    const int dc = s.depth_cnt[d];
-    if (W > 0 && dc >= W) {  // outside Top_W(E_d); so are its later siblings
-      put(widx, 0u, 0u);
-      __syncwarp();
-      continue;
-    }
-    // one round of independent loads: next sibling, first child, parent score
-    const bool has_sib = j + 1 < k, has_child = d < L;
-    const int child = (d * k + r) * k;
-    const float t_sib = has_sib ? s.t[prev + j + 1] : 0.f;
-    const int r_sib = has_sib ? s.ord[prev + j + 1] : 0;
-    const float t_child = has_child ? s.t[child] : 0.f;
-    const int r_child = has_child ? s.ord[child] : 0;
-    const float ps = p == 255 ? 0.f : s.nd_score[p];
-    const int n = n_acc++;
-    if (lane == 0) {
-      s.nd_parent[n] = (short)(p == 255 ? -1 : p);
-      s.nd_depth[n] = (unsigned char)d;
-      s.nd_rank[n] = (unsigned char)r;
-      s.nd_score[n] = score;
-      s.depth_cnt[d] = dc + 1;
-      if (use_pk) {
-        unsigned long long hi = p == 255 ? 0ull : s.nd_pk[2 * p], lo = p == 255 ? 0ull : s.nd_pk[2 * p + 1];
-        const int sh = 128 - bits * d;
-        if (sh >= 64) hi |= (unsigned long long)r << (sh - 64); else lo |= (unsigned long long)r << sh;
-        s.nd_pk[2 * n] = hi; s.nd_pk[2 * n + 1] = lo;
+    if (W > 0) {
+      const int dc = s.depth_cnt[d];
+      if (dc >= W) {  // outside Top_W(E_d); so are its later siblings
+#pragma unroll
+        for (int q = 0; q < SLOTS; ++q) fk[q] = (lane == wl && q == ws) ? 0u : fk[q];
+        s.ent[e_idx] = make_uint4(0u, 0u, 0u, 0u);
+        __syncwarp();
+        continue;
       }
+      s.depth_cnt[d] = dc + 1;
     }
-    if (has_sib) put(widx, f2key(ps + t_sib + zeta), pack_info(p, j + 1, d, pr, r_sib));
-    else put(widx, 0u, 0u);
-    if (has_child) { put(f_cnt, f2key(score + t_child + zeta), pack_info(n, 0, d + 1, r, r_child)); ++f_cnt; }
+    // one round of independent loads: next sibling and first child
+    const bool has_sib = j + 1 < k, has_child = d < L;
+    const int i_sib = has_sib ? at + 1 : 0, i_child = has_child ? cb : 0;
+    const float t_sib = s.t[i_sib], t_child = s.t[i_child];
+    const int r_sib = s.ord[i_sib], r_child = s.ord[i_child];
+    // Every store below is executed by all lanes with the same address and value: a divergent single-lane
+    // block costs more than the whole rest of the pop.
+    const int n = n_acc++;
+    s.nd_parent[n] = (short)(p == 255 ? -1 : p);
+    s.nd_depth[n] = (unsigned char)d;
+    s.nd_rank[n] = (unsigned char)r;
+    s.nd_score[n] = score;
+    const uint32_t k_sib = has_sib ? f2key(ps + t_sib + zeta) : 0u;
+    const uint32_t k_child = has_child ? f2key(score + t_child + zeta) : 0u;
+    const int cl = f_cnt & 31, cs = f_cnt >> 5;
+    s.ent[e_idx] = make_uint4(pack_lo(p, j + 1, d, r_sib), (uint32_t)i_sib | ((uint32_t)((d * k + r_sib) * k) << 15),
+                              ent.z, k_sib);
+    // without a child the record is dead (key 0) and its place is taken by the next one
+    s.ent[f_cnt] = make_uint4(pack_lo(n, 0, d + 1, r_child),
+                              (uint32_t)i_child | ((uint32_t)(((d + 1) * k + r_child) * k) << 15),
+                              __float_as_uint(score), k_child);
+#pragma unroll
+    for (int q = 0; q < SLOTS; ++q) {
+      fk[q] = (lane == wl && q == ws) ? k_sib : fk[q];
+      fk[q] = (has_child && lane == cl && q == cs) ? k_child : fk[q];
+    }
+    f_cnt += has_child ? 1 : 0;
     __syncwarp();
   }
+  __syncwarp();
   return n_acc;
 }
 
@@ -225,6 +231,30 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   long long tt[10];
 #endif
   TT(0);
+  // ---- the selector's scores, scaled by eq. 5's lambda, go to shared memory first.  They are an input of
+  // the call, complete before the streaming kernel ahead of this one was launched, so they may be read
+  // while that kernel is still running: their DRAM latency hides behind its tail.
+  const int nrows = 1 + (L - 1) * k;
+  {
+    const int n_big = (L - 1) * kk2;
+    constexpr int U = 8;
+    for (int i0 = 0; i0 < n_big; i0 += G2_T * U) {
+      float d[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int i = i0 + u * G2_T + tid;
+        d[u] = i < n_big ? g_big[(int64_t)b * n_big + i] : 0.f;
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int i = i0 + u * G2_T + tid;
+        if (i < n_big) s.t[kk2 + i] = (lambda ? lambda[1 + i / kk2] : 1.f) * d[u];
+      }
+    }
+    for (int i = tid; i < kk2; i += G2_T)  // position 0: only predecessor row 0 exists
+      s.t[i] = (i < k && anchor_bigram) ? (lambda ? lambda[0] : 1.f) * anchor_bigram[(int64_t)b * k + i] : 0.f;
+    for (int i = tid; i < L; i += G2_T) s.al[i] = alpha ? alpha[i] : 1.f;
+  }
   pdl_wait();  // the partials / candidates come from the kernel before this one
 
   // ---- step a1's last part when fused: merge the row partials of this sequence's L rows
@@ -240,15 +270,105 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
     s.lp[i] = g_lp[(int64_t)b * L * k + i];
     s.tok[i] = g_ids[(int64_t)b * L * k + i];
   }
-  for (int i = tid; i < L * kk2; i += G2_T) {
-    float d = 0.f;
-    if (i < kk2) {
-      if (i < k && anchor_bigram) d = anchor_bigram[(int64_t)b * k + i];  // only predecessor row 0 exists
-    } else {
-      d = g_big[(int64_t)b * (L - 1) * kk2 + (i - kk2)];
+  TT(2);
+  int kp = 1;
+  while (kp < k) kp <<= 1;
+  if (k <= 32) {
+    // ---- eq. 5 and eq. 9, then every row sorted by (t desc, token asc): a group of kp = 2^ceil(log2 k)
+    // lanes per (position, predecessor) row, the row's values in registers, reductions and exact ranks by
+    // shuffles inside the group; integer keys and a final index tie-break keep the ranks a permutation
+    // whatever the values are (even NaN).  Several rows are in flight per warp and no CTA barrier is needed.
+    __syncthreads();  // s.lp, s.tok
+    const int gpw = 32 / kp, rb = lane & (kp - 1);
+    const int gid = (tid >> 5) * gpw + lane / kp, ngroups = (G2_T / 32) * gpw;
+    for (int r0 = 0; r0 < nrows; r0 += ngroups) {
+      const int r = r0 + gid;
+      const bool active = r < nrows && rb < k;
+      const int i = r <= 0 ? 0 : 1 + (r - 1) / k;
+      const int ra = r <= 0 ? 0 : (r - 1) % k;
+      float v = -INFINITY;
+      int tk = 0;
+      const int at = (i * k + ra) * k;
+      if (active) {
+        v = fmaf(s.al[i], s.lp[i * k + rb], s.t[at + rb]);
+        tk = s.tok[i * k + rb];
+      }
+      float mx = v;
+      for (int o = kp >> 1; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, o));
+      float sum = active ? expf(v - mx) : 0.f;
+      for (int o = kp >> 1; o > 0; o >>= 1) sum += __shfl_xor_sync(FULL, sum, o);
+      const float tv = v - (mx + logf(sum));
+      const uint32_t kv = f2key(tv);
+      int rank = 0;
+      bool tie = false;
+#pragma unroll 4
+      for (int j = 0; j < k; ++j) {
+        const uint32_t kj = __shfl_sync(FULL, kv, j, kp);
+        rank += kj > kv;
+        tie |= kj == kv && j != rb;
+      }
+      if (__any_sync(FULL, tie && active)) {  // equal values in one row (rare): token, then index, decide
+        rank = 0;
+        for (int j = 0; j < k; ++j) {
+          const uint32_t kj = __shfl_sync(FULL, kv, j, kp);
+          const int tj = __shfl_sync(FULL, tk, j, kp);
+          rank += (kj > kv) || (kj == kv && (tj < tk || (tj == tk && j < rb)));
+        }
+      }
+      if (active) {
+        s.t[at + rank] = tv;
+        s.ord[at + rank] = (unsigned char)rb;
+      }
     }
-    s.t[i] = d;
+  } else {
+    __syncthreads();
+    // eq. 5 and eq. 9: one thread per (position, predecessor) row
+    for (int r = tid; r < nrows; r += G2_T) {
+      const int i = r == 0 ? 0 : 1 + (r - 1) / k;
+      const int ra = r == 0 ? 0 : (r - 1) % k;
+      float* row = s.t.ptr(((long long)i * k + ra) * k, k);
+      const float al = s.al[i];
+      float mx = -INFINITY;
+      for (int rb = 0; rb < k; ++rb) {
+        float v = fmaf(al, s.lp[i * k + rb], row[rb]);
+        row[rb] = v;
+        mx = fmaxf(mx, v);
+      }
+      float sum = 0.f;
+      for (int rb = 0; rb < k; ++rb) sum += expf(row[rb] - mx);
+      const float lse = mx + logf(sum);
+      for (int rb = 0; rb < k; ++rb) row[rb] -= lse;
+    }
+    __syncthreads();
+    // in-place sort, whole rows per batch: a row is read completely before it is rewritten
+    const int rows_per_batch = G2_T / k;
+    for (int row0 = 0; row0 < nrows; row0 += rows_per_batch) {
+      const int r = row0 + tid / k, rb = tid % k;
+      const bool active = tid < rows_per_batch * k && r < nrows;
+      float v = 0.f;
+      int rank = 0, at = 0;
+      if (active) {
+        const int i = r == 0 ? 0 : 1 + (r - 1) / k;
+        const int ra = r == 0 ? 0 : (r - 1) % k;
+        at = (i * k + ra) * k;
+        const float* row = s.t.ptr(at, k);
+        const int* tk = s.tok.ptr((long long)i * k, k);
+        v = row[rb];
+        const uint32_t kv = f2key(v);
+        for (int j = 0; j < k; ++j) {
+          const uint32_t kj = f2key(row[j]);
+          rank += (kj > kv) || (kj == kv && (tk[j] < tk[rb] || (tk[j] == tk[rb] && j < rb)));
+        }
+      }
+      __syncthreads();  // all reads of this batch of rows precede the in-place writes
+      if (active) {
+        s.t[at + rank] = v;
+        s.ord[at + rank] = (unsigned char)rb;
+      }
+      __syncthreads();
+    }
   }
+  TT(3);
   // Every read of memory an earlier kernel produced (row partials in the caller's workspace, candidates,
   // selector scores) has been issued; from here on only this kernel's own outputs are touched, so the next
   // kernel in the stream -- typically the V-wide pass of ubt_verify_tree, which needs none of them -- may
@@ -259,56 +379,6 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   for (int i = tid; i < N * mw; i += G2_T) s.maskrow[i] = 0u;
   __syncthreads();
 
-  TT(2);
-  // ---- eq. 5 and eq. 9: one thread per (position, predecessor) row
-  const int nrows = 1 + (L - 1) * k;
-  for (int r = tid; r < nrows; r += G2_T) {
-    const int i = r == 0 ? 0 : 1 + (r - 1) / k;
-    const int ra = r == 0 ? 0 : (r - 1) % k;
-    float* row = s.t.ptr(((long long)i * k + ra) * k, k);
-    const float al = alpha ? alpha[i] : 1.f, la = lambda ? lambda[i] : 1.f;
-    float mx = -INFINITY;
-    for (int rb = 0; rb < k; ++rb) {
-      float v = al * s.lp[i * k + rb] + la * row[rb];
-      row[rb] = v;
-      mx = fmaxf(mx, v);
-    }
-    float sum = 0.f;
-    for (int rb = 0; rb < k; ++rb) sum += expf(row[rb] - mx);
-    const float lse = mx + logf(sum);
-    for (int rb = 0; rb < k; ++rb) row[rb] -= lse;
-  }
-  __syncthreads();
-  TT(3);
-  // every row sorted by (t desc, token asc), in place; integer keys and a final index tie-break keep the
-  // ranks a permutation whatever the values are (even NaN)
-  const int rows_per_batch = G2_T / k;  // whole rows per batch: a row is read completely before it is rewritten
-  for (int row0 = 0; row0 < nrows; row0 += rows_per_batch) {
-    const int r = row0 + tid / k, rb = tid % k;
-    const bool active = tid < rows_per_batch * k && r < nrows;
-    float v = 0.f;
-    int rank = 0, at = 0;
-    if (active) {
-      const int i = r == 0 ? 0 : 1 + (r - 1) / k;
-      const int ra = r == 0 ? 0 : (r - 1) % k;
-      at = (i * k + ra) * k;
-      const float* row = s.t.ptr(at, k);
-      const int* tk = s.tok.ptr((long long)i * k, k);
-      v = row[rb];
-      const uint32_t kv = f2key(v);
-      for (int j = 0; j < k; ++j) {
-        const uint32_t kj = f2key(row[j]);
-        rank += (kj > kv) || (kj == kv && (tk[j] < tk[rb] || (tk[j] == tk[rb] && j < rb)));
-      }
-    }
-    __syncthreads();  // all reads of this batch of rows precede the in-place writes
-    if (active) {
-      s.t[at + rank] = v;
-      s.ord[at + rank] = (unsigned char)rb;
-    }
-    __syncthreads();
-  }
-
   TT(4);
   // ---- best-first expansion (warp 0)
   int bits = 1;
@@ -316,9 +386,9 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   const bool use_pk = bits * L <= 128;
   if (tid < 32) {
     int n;
-    if (N <= 64) n = expand_tree<2>(s, L, k, budget, W, zeta, bits, use_pk, lane);
-    else if (N <= 128) n = expand_tree<4>(s, L, k, budget, W, zeta, bits, use_pk, lane);
-    else n = expand_tree<8>(s, L, k, budget, W, zeta, bits, use_pk, lane);
+    if (N <= 64) n = expand_tree<2>(s, L, k, budget, W, zeta, lane);
+    else if (N <= 128) n = expand_tree<4>(s, L, k, budget, W, zeta, lane);
+    else n = expand_tree<8>(s, L, k, budget, W, zeta, lane);
     if (lane == 0) s.scalars[0] = n;
   }
   __syncthreads();
@@ -326,23 +396,43 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   TT(5);
   // ---- canonical slots: root 0, then depth by depth ordered by (parent slot, rank)
   const int n_acc = s.scalars[0];
+  for (int i = tid; i < L + 2; i += G2_T) s.depth_cnt[i] = 0;
+  __syncthreads();
+  if (tid < n_acc) {
+    atomicAdd(&s.depth_cnt[s.nd_depth[tid]], 1);
+    if (use_pk) {  // rank path packed big-endian: walk up to the root
+      unsigned long long hi = 0ull, lo = 0ull;
+      for (int a = tid; a >= 0; a = s.nd_parent[a]) {
+        const int sh = 128 - bits * (int)s.nd_depth[a];
+        const unsigned long long r = s.nd_rank[a];
+        if (sh >= 64) hi |= r << (sh - 64); else lo |= r << sh;
+      }
+      s.nd_pk[2 * tid] = hi; s.nd_pk[2 * tid + 1] = lo;
+    }
+  }
+  __syncthreads();
   if (tid == 0) {
     int off = 1;
     for (int d = 1; d <= L; ++d) { s.depth_off[d] = off; off += s.depth_cnt[d]; }
   }
   __syncthreads();
   if (use_pk) {
-    // inside a depth, (parent slot, rank) order is the lexicographic order of the rank paths
-    if (tid < n_acc) {
-      const int d = s.nd_depth[tid];
-      const unsigned long long hi = s.nd_pk[2 * tid], lo = s.nd_pk[2 * tid + 1];
-      int c = 0;
-      for (int j = 0; j < n_acc; ++j) {
+    // inside a depth, (parent slot, rank) order is the lexicographic order of the rank paths; the count for
+    // one node is shared by `sp` neighbouring lanes
+    int sp = 1;
+    while (sp < 32 && sp * 2 * N <= G2_T) sp <<= 1;
+    const int node = tid / sp, q = tid & (sp - 1);
+    const bool mine = node < n_acc;
+    const int d = mine ? s.nd_depth[node] : 0;
+    const unsigned long long hi = mine ? s.nd_pk[2 * node] : 0ull, lo = mine ? s.nd_pk[2 * node + 1] : 0ull;
+    int c = 0;
+    if (mine)
+      for (int j = q; j < n_acc; j += sp) {
         const unsigned long long hj = s.nd_pk[2 * j], lj = s.nd_pk[2 * j + 1];
         c += (s.nd_depth[j] == d) && (hj < hi || (hj == hi && lj < lo));
       }
-      s.nd_slot[tid] = (short)(s.depth_off[d] + c);
-    }
+    for (int o = sp >> 1; o > 0; o >>= 1) c += __shfl_xor_sync(FULL, c, o);
+    if (mine && q == 0) s.nd_slot[node] = (short)(s.depth_off[d] + c);
     __syncthreads();
   } else {
     for (int d = 1; d <= L; ++d) {  // paths too long to pack: one depth at a time
