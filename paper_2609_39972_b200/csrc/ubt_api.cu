@@ -183,7 +183,7 @@ int ubt_verify_tree(const ubt_tree* tree, const void* target_logits, int dtype, 
   if (o->event_before && cudaEventRecord(static_cast<cudaEvent_t>(o->event_before), st) != cudaSuccess)
     return UBT_ERR_CUDA;
   if (mode == UBT_VERIFY_GREEDY) {
-    if (launch_row_argmax(target_logits, dtype, rows, V, w, st) != cudaSuccess) return UBT_ERR_CUDA;
+    if (launch_row_argmax(target_logits, dtype, rows, V, w, tree_smem_bytes(tree->L, tree->k, tree->N), st) != cudaSuccess) return UBT_ERR_CUDA;
   } else {
     int32_t* pick = o->node_pick ? o->node_pick : w.pick;
     if (launch_row_sample(target_logits, dtype, B, N, V, o->seed, o->temperature, pick, w, st) != cudaSuccess)

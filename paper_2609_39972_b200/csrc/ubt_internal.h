@@ -84,8 +84,10 @@ struct VerifyWorkspace {
 };
 size_t verify_workspace_bytes(int64_t rows, int V, int mode);
 VerifyWorkspace carve_verify_workspace(void* ws, int64_t rows, int V, int mode);
+// neighbour_smem: dynamic shared memory of one CTA of the kernel launched just before on the stream (the tree
+// kernel when draft and verify calls follow one another); the ring is sized to fit beside it on an SM.
 cudaError_t launch_row_argmax(const void* logits, int dtype, int64_t rows, int V,
-                              const VerifyWorkspace& w, cudaStream_t st);
+                              const VerifyWorkspace& w, size_t neighbour_smem, cudaStream_t st);
 cudaError_t launch_row_sample(const void* logits, int dtype, int B, int N, int V, uint64_t seed,
                               float temperature, int32_t* pick, const VerifyWorkspace& w, cudaStream_t st);
 cudaError_t launch_walk(const ubt_tree& tree, int mode, const VerifyWorkspace& w, int V,

@@ -708,15 +708,19 @@ static cudaError_t launch_row_argmax_t(const void* logits, int64_t rows, int V, 
   return cudaGetLastError();
 }
 
-// Ring configuration of the greedy kernel: three 64 KiB stages, 256 threads, one CTA per SM.  Measured on
-// B200 (622 MB of bf16 rows): 94.7 us; 6 x 32 KiB: 105 us; 12 x 16 KiB: 179 us (per-chunk latency dominates).
-constexpr int kArgmaxStages = 3, kArgmaxStageBytes = 65536, kArgmaxThreads = 256;
+// Ring configuration of the greedy kernel: three stages, 256 threads, one CTA per SM.  Measured on B200
+// (622 MB of bf16 rows) with 64 KiB stages: 94.7 us; 6 x 32 KiB: 105 us; 12 x 16 KiB: 179 us (per-chunk latency
+// dominates).  The kernel is launched programmatically behind the tree kernel, so its CTAs should fit on an
+// SM beside one CTA of that kernel: when the tree's tables leave no room for 3 x 64 KiB the stages shrink to
+// 48 KiB (same speed on 5 GB of rows, 2 % slower on 0.6 GB), which lets the whole tree build hide behind it.
+constexpr int kArgmaxStages = 3, kArgmaxThreads = 256;
+constexpr int kSmemPerSm = 228 * 1024, kSmemPerCtaReserved = 1024;
 
-template <typename T>
+template <typename T, int STAGE_BYTES>
 static cudaError_t launch_row_argmax_ring_t(const void* logits, int64_t rows, int V, const VerifyWorkspace& w,
                                             cudaStream_t st) {
-  auto kern = k_row_argmax_ring<T, kArgmaxStages, kArgmaxStageBytes, kArgmaxThreads, 1>;
-  constexpr int kBytes = kArgmaxStages * kArgmaxStageBytes;
+  auto kern = k_row_argmax_ring<T, kArgmaxStages, STAGE_BYTES, kArgmaxThreads, 1>;
+  constexpr int kBytes = kArgmaxStages * STAGE_BYTES;
   static bool configured = false;  // the attribute sticks to the function; set it once
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBytes);
@@ -727,12 +731,20 @@ static cudaError_t launch_row_argmax_ring_t(const void* logits, int64_t rows, in
                        rows * (int64_t)V, V, w.plan, w.part_key);
 }
 
+template <typename T>
+static cudaError_t launch_row_argmax_ring_t(const void* logits, int64_t rows, int V, const VerifyWorkspace& w,
+                                            size_t neighbour_smem, cudaStream_t st) {
+  const bool roomy = kArgmaxStages * 65536 + neighbour_smem + 2 * kSmemPerCtaReserved <= (size_t)kSmemPerSm;
+  return roomy ? launch_row_argmax_ring_t<T, 65536>(logits, rows, V, w, st)
+               : launch_row_argmax_ring_t<T, 49152>(logits, rows, V, w, st);
+}
+
 cudaError_t launch_row_argmax(const void* logits, int dtype, int64_t rows, int V, const VerifyWorkspace& w,
-                              cudaStream_t st) {
+                              size_t neighbour_smem, cudaStream_t st) {
   if (rows == 0) return cudaSuccess;
   // rows that are whole 16-byte fragments go through the bulk-copy ring; other V use plain loads
-  if (dtype == UBT_BF16 && V % 8 == 0) return launch_row_argmax_ring_t<__nv_bfloat16>(logits, rows, V, w, st);
-  if (dtype == UBT_F32 && V % 4 == 0) return launch_row_argmax_ring_t<float>(logits, rows, V, w, st);
+  if (dtype == UBT_BF16 && V % 8 == 0) return launch_row_argmax_ring_t<__nv_bfloat16>(logits, rows, V, w, neighbour_smem, st);
+  if (dtype == UBT_F32 && V % 4 == 0) return launch_row_argmax_ring_t<float>(logits, rows, V, w, neighbour_smem, st);
   if (dtype == UBT_BF16) {
     if (V % 8 == 0) return launch_row_argmax_t<__nv_bfloat16, 8>(logits, rows, V, w, st);
     return launch_row_argmax_t<__nv_bfloat16, 1>(logits, rows, V, w, st);
