@@ -38,10 +38,28 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// The same poll, but the hardware may keep the thread suspended for up to `hint_ns` while the phase is
+// incomplete: a waiting warp then takes (almost) no issue slots from the warps that share its scheduler.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint64_t* bar, uint32_t parity, uint32_t hint_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3; selp.u32 %0, 1, 0, p; }"
+      : "=r"(ok)
+      : "r"(smem_addr(bar)), "r"(parity), "r"(hint_ns)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_hint(uint64_t* bar, uint32_t parity, uint32_t hint_ns);
 // Bounded wait; false = gave up.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
   for (int spins = 0; spins < kRingSpinLimit; ++spins)
     if (mbar_try_wait(bar, parity)) return true;
+  atomicAdd(&g_ring_timeouts, 1u);
+  return false;
+}
+__device__ __forceinline__ bool mbar_wait_hint(uint64_t* bar, uint32_t parity, uint32_t hint_ns) {
+  for (int spins = 0; spins < kRingSpinLimit; ++spins)
+    if (mbar_try_wait_hint(bar, parity, hint_ns)) return true;
   atomicAdd(&g_ring_timeouts, 1u);
   return false;
 }
@@ -95,6 +113,20 @@ struct RingProducer {
     const int l = rem < kStageElems ? rem : kStageElems;
     mbar_expect_tx(&full[stage], (uint32_t)(l * sizeof(T)));
     bulk_load(ring + (size_t)stage * STAGE_BYTES, base + pos, (uint32_t)(l * sizeof(T)), &full[stage]);
+    pos += l;
+    rem -= l;
+    if (rem == 0 && pos < hi) {
+      Segment sg;
+      sg.at(pos, hi, V);
+      rem = sg.len;
+    }
+    if (++stage == STAGES) stage = 0;
+    ++issued;
+  }
+  // Advance past one chunk without copying it (for a thread that follows the sequence another one issues).
+  __device__ __forceinline__ void skip_one() {
+    if (rem == 0) return;
+    const int l = rem < kStageElems ? rem : kStageElems;
     pos += l;
     rem -= l;
     if (rem == 0 && pos < hi) {

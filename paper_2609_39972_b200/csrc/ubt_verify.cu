@@ -282,24 +282,6 @@ __device__ __forceinline__ unsigned long long weight_of(float z, float a, float 
 
 // Two weights at once with the packed fp32 instructions of sm_100 (fma/add .f32x2): the same IEEE operations
 // per component as weight_of, half the issue slots for the arithmetic part.
-__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
-  unsigned long long r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
-  unsigned long long d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
-  unsigned long long d;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
 struct WeightConsts2 {  // the routine's constants, duplicated into both halves
   unsigned long long a, c, big, nbig, none, c5, c4, c3, c2, c1, one;
   __device__ __forceinline__ void init(float a_, float c_) {
