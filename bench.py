@@ -108,6 +108,11 @@ class ClockSampler:
                 "reasons": sorted(reasons)}
 
 
+def input_seed(rank: int, s: int) -> int:
+    """Seed of input set ``s`` on rank ``rank``: every rank streams its own batches (weak scaling)."""
+    return 1000 * rank + s
+
+
 def dist_setup(n_gpus: int):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -209,7 +214,7 @@ def main():
     n_sets = max(2, min(16, -(-4 * 126_000_000 // max(batch_bytes, 1))))
     sets = []
     for s in range(n_sets):
-        ud, bd, zd = synth.device_inputs(cfg, 1000 * rank + s, dev)
+        ud, bd, zd = synth.device_inputs(cfg, input_seed(rank, s), dev)
         sets.append((ud, bd, zd))
     tree = ubt.Tree.empty(cfg.B, cfg.N, cfg.L, cfg.k, dev)
     res = ubt.VerifyResult.empty(cfg.B, cfg.L, dev)
@@ -275,7 +280,8 @@ def main():
 
     peak, peak_kind = measured_peak()
     e = 2 if cfg.dtype == "bf16" else 4
-    kern_name = "k_row_argmax" if cfg.mode == "greedy" else "k_row_sample"
+    kern_name = "k_row_argmax_ring" if cfg.mode == "greedy" else "k_row_weights_ring+k_row_pick"
+    launches_per_step = 2 + (2 if cfg.mode == "greedy" else 3)   # top-k, tree | argmax or weights+pick, walk
     kern_bytes = cfg.B * cfg.N * cfg.V * e
     achieved = kern_bytes / (kern_ms * 1e-3) / 1e9
     step_gbs = batch_bytes * args.steps / (elapsed_ms * 1e-3) / 1e9 if world == 1 else \
@@ -300,7 +306,7 @@ def main():
                      "timed": "second pass of the same %d steps with an event pair around this kernel "
                               "(%.4f ms/step in that pass)" % (args.steps, elapsed_ev_ms / args.steps)},
         "clocks": clocks,
-        "gpu_launches": 4 * 2 * args.steps,
+        "gpu_launches": launches_per_step * args.steps,
     }
 
     # ---- end to end through the host-buffer entry points (pinned host inputs, results read back)
@@ -330,8 +336,7 @@ def main():
         h2d = uh.numel() * uh.element_size() + bh.numel() * 4 + zh.numel() * zh.element_size() + cfg.B * (2 * cfg.N + 1) * 4
         d2h = cfg.B * (cfg.N * (6 + mw) * 4 + 4 + cfg.L * cfg.k * 8) + cfg.B * (2 * (cfg.L + 1) + 2) * 4
         line["e2e"] = {"value": cfg.B * k_e2e * world / dt, "unit": "trees/s", "h2d_bytes_per_step": h2d,
-                       "d2h_bytes_per_step": d2h, "steps": k_e2e, "gpu_launches": 4 * k_e2e}
-        line["gpu_launches"] += 4 * k_e2e
+                       "d2h_bytes_per_step": d2h, "steps": k_e2e, "gpu_launches": launches_per_step * k_e2e}
         del uh, bh, zh
 
     # ---- CPU baseline: the oracle as it stands on the host cores, on a bounded sample; doubles as a parity check

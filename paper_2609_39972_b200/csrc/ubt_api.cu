@@ -50,6 +50,74 @@ static int check_tree(const ubt_tree* t, bool need_cands) {
   return UBT_OK;
 }
 
+// ---- which memory a draft call on a stream may still be using when the next call starts
+//
+// The tree kernel lets the kernel behind it on the stream start at once (programmatic dependent launch), so the
+// V-wide pass of a verify call streams while the draft call's kernels are still running.  That is only sound
+// if nothing the early kernel WRITES overlaps anything the draft call reads or writes; plain stream order
+// would allow such reuse (say, the draft logits' buffer as the verify workspace).  Every draft call therefore
+// records its buffers per stream, and a verify call whose written buffers touch them launches its first
+// kernel without the attribute, i.e. strictly after the draft.
+struct ByteRange {
+  const char* lo;
+  const char* hi;
+};
+struct DraftRecord {
+  cudaStream_t stream;
+  bool valid;
+  int n;
+  ByteRange r[24];
+};
+static std::mutex g_draft_mu;
+static DraftRecord g_drafts[16];
+static unsigned g_draft_next;
+
+static void add_range(DraftRecord& d, const void* p, size_t bytes) {
+  if (p && bytes && d.n < 24) d.r[d.n++] = ByteRange{static_cast<const char*>(p), static_cast<const char*>(p) + bytes};
+}
+
+static void remember_draft(cudaStream_t st, const void* logits, size_t logits_bytes, const float* bigram, int B, int L,
+                           int k, int N, const ubt_draft_opts* o, const ubt_tree& t, const void* ws, size_t ws_bytes) {
+  DraftRecord d{};
+  d.stream = st;
+  d.valid = true;
+  const size_t bn = (size_t)B * N, blk = (size_t)B * L * k;
+  add_range(d, logits, logits_bytes);
+  add_range(d, bigram, (size_t)B * (L > 1 ? L - 1 : 0) * k * k * 4);
+  add_range(d, ws, ws_bytes);
+  if (o) {
+    add_range(d, o->alpha, (size_t)L * 4);
+    add_range(d, o->lambda, (size_t)L * 4);
+    add_range(d, o->anchor_bigram, (size_t)B * k * 4);
+    add_range(d, o->anchor_tokens, (size_t)B * 4);
+    add_range(d, o->pos_offset, (size_t)B * 4);
+  }
+  const void* per_node[] = {t.token_ids, t.parents, t.depths, t.position_ids, t.cand_rank, t.scores};
+  for (const void* p : per_node) add_range(d, p, bn * 4);
+  add_range(d, t.mask, bn * t.mask_words * 4);
+  add_range(d, t.n_nodes, (size_t)B * 4);
+  add_range(d, t.cand_ids, blk * 4);
+  add_range(d, t.cand_logprob, blk * 4);
+  std::lock_guard<std::mutex> lock(g_draft_mu);
+  for (DraftRecord& e : g_drafts)
+    if (e.valid && e.stream == st) { e = d; return; }
+  g_drafts[g_draft_next++ % 16] = d;
+}
+
+// May a kernel that writes [p, p + bytes) start while the last draft call on `st` is still running?
+static bool clear_of_last_draft(cudaStream_t st, const void* p, size_t bytes) {
+  if (!p || !bytes) return true;
+  const char* lo = static_cast<const char*>(p);
+  const char* hi = lo + bytes;
+  std::lock_guard<std::mutex> lock(g_draft_mu);
+  for (const DraftRecord& e : g_drafts) {
+    if (!e.valid || e.stream != st) continue;
+    for (int i = 0; i < e.n; ++i)
+      if (lo < e.r[i].hi && e.r[i].lo < hi) return false;
+  }
+  return true;
+}
+
 }  // namespace ubt
 
 using namespace ubt;
@@ -113,6 +181,7 @@ int ubt_build_tree(const float* bigram_scores, int B, int L, int k, int N, const
   if (tree_smem_bytes(L, k, N) > (size_t)device_info().max_smem_optin) return UBT_ERR_UNSUPPORTED;
   const ubt_draft_opts d{};
   const ubt_draft_opts* o = opts ? opts : &d;
+  remember_draft(static_cast<cudaStream_t>(cuda_stream), nullptr, 0, bigram_scores, B, L, k, N, o, *out, nullptr, 0);
   cudaError_t e = launch_build_tree(bigram_scores, B, L, k, N, o->search_width, o->depth_bonus, o->alpha, o->lambda,
                                     o->anchor_bigram, o->anchor_tokens, o->pos_offset, *out, no_merge_parts(), 0,
                                     static_cast<cudaStream_t>(cuda_stream));
@@ -150,6 +219,8 @@ int ubt_draft_tree(const void* unigram_logits, int dtype, const float* bigram_sc
   // the tree kernel merges the row partials in its prologue: one launch less than topk + merge + tree
   const ubt_draft_opts d{};
   const ubt_draft_opts* o = opts ? opts : &d;
+  remember_draft(st, unigram_logits, (size_t)rows * V * esize(dtype), bigram_scores, B, L, k, N, o, *out, workspace,
+                 topk_workspace_bytes(rows, V, k));
   cudaError_t e = launch_build_tree(bigram_scores, B, L, k, N, o->search_width, o->depth_bonus, o->alpha, o->lambda,
                                     o->anchor_bigram, o->anchor_tokens, o->pos_offset, *out, merge_parts(w), V, st);
   return e == cudaSuccess ? UBT_OK : UBT_ERR_CUDA;
@@ -182,11 +253,17 @@ int ubt_verify_tree(const ubt_tree* tree, const void* target_logits, int dtype, 
   const int32_t* sampled = nullptr;
   if (o->event_before && cudaEventRecord(static_cast<cudaEvent_t>(o->event_before), st) != cudaSuccess)
     return UBT_ERR_CUDA;
+  // the V-wide kernels may start while a draft call in front of them on this stream is still running, unless
+  // what they write touches that call's buffers
+  bool early = clear_of_last_draft(st, workspace, verify_workspace_bytes(rows, V, mode));
   if (mode == UBT_VERIFY_GREEDY) {
-    if (launch_row_argmax(target_logits, dtype, rows, V, w, tree_smem_bytes(tree->L, tree->k, tree->N), st) != cudaSuccess) return UBT_ERR_CUDA;
+    if (launch_row_argmax(target_logits, dtype, rows, V, w, tree_smem_bytes(tree->L, tree->k, tree->N), early, st) !=
+        cudaSuccess)
+      return UBT_ERR_CUDA;
   } else {
     int32_t* pick = o->node_pick ? o->node_pick : w.pick;
-    if (launch_row_sample(target_logits, dtype, B, N, V, o->seed, o->temperature, pick, w, st) != cudaSuccess)
+    early = early && clear_of_last_draft(st, o->node_pick, (size_t)rows * 4);
+    if (launch_row_sample(target_logits, dtype, B, N, V, o->seed, o->temperature, pick, w, early, st) != cudaSuccess)
       return UBT_ERR_CUDA;
     sampled = pick;
   }

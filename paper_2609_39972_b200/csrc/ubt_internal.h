@@ -86,10 +86,13 @@ size_t verify_workspace_bytes(int64_t rows, int V, int mode);
 VerifyWorkspace carve_verify_workspace(void* ws, int64_t rows, int V, int mode);
 // neighbour_smem: dynamic shared memory of one CTA of the kernel launched just before on the stream (the tree
 // kernel when draft and verify calls follow one another); the ring is sized to fit beside it on an SM.
+// early: the kernel may start before the kernel in front of it on the stream has completed (programmatic
+// dependent launch); the caller has checked that nothing it writes is still in use there.
 cudaError_t launch_row_argmax(const void* logits, int dtype, int64_t rows, int V,
-                              const VerifyWorkspace& w, size_t neighbour_smem, cudaStream_t st);
+                              const VerifyWorkspace& w, size_t neighbour_smem, bool early, cudaStream_t st);
 cudaError_t launch_row_sample(const void* logits, int dtype, int B, int N, int V, uint64_t seed,
-                              float temperature, int32_t* pick, const VerifyWorkspace& w, cudaStream_t st);
+                              float temperature, int32_t* pick, const VerifyWorkspace& w, bool early,
+                              cudaStream_t st);
 cudaError_t launch_walk(const ubt_tree& tree, int mode, const VerifyWorkspace& w, int V,
                         const int32_t* sampled_pick, int32_t* node_pick,
                         const ubt_verify_result& out, cudaStream_t st);

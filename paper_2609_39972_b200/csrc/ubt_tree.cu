@@ -231,6 +231,12 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   long long tt[10];
 #endif
   TT(0);
+  // The next kernel in the stream may start right away.  When that is the V-wide pass of ubt_verify_tree it
+  // reads target logits only and streams while this kernel (and the tail of the top-k kernel in front of it)
+  // is still running; it waits for this grid before it exits, so stream order still holds for whatever follows.
+  // The host side launches it that way only if nothing it writes touches a buffer of this draft call; any
+  // other kernel is launched normally and starts after this grid has completed, whatever is signalled here.
+  pdl_launch_dependents();
   // ---- the selector's scores, scaled by eq. 5's lambda, go to shared memory first.  They are an input of
   // the call, complete before the streaming kernel ahead of this one was launched, so they may be read
   // while that kernel is still running: their DRAM latency hides behind its tail.
@@ -369,12 +375,7 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
     }
   }
   TT(3);
-  // Every read of memory an earlier kernel produced (row partials in the caller's workspace, candidates,
-  // selector scores) has been issued; from here on only this kernel's own outputs are touched, so the next
-  // kernel in the stream -- typically the V-wide pass of ubt_verify_tree, which needs none of them -- may
-  // start.  It waits for this grid before it exits, so stream order still holds for whatever follows it.
   __syncthreads();
-  pdl_launch_dependents();
   for (int i = tid; i < L + 2; i += G2_T) s.depth_cnt[i] = 0;
   for (int i = tid; i < N * mw; i += G2_T) s.maskrow[i] = 0u;
   __syncthreads();

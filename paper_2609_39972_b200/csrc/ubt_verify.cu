@@ -700,7 +700,7 @@ constexpr int kSmemPerSm = 228 * 1024, kSmemPerCtaReserved = 1024;
 
 template <typename T, int STAGE_BYTES>
 static cudaError_t launch_row_argmax_ring_t(const void* logits, int64_t rows, int V, const VerifyWorkspace& w,
-                                            cudaStream_t st) {
+                                            bool early, cudaStream_t st) {
   auto kern = k_row_argmax_ring<T, kArgmaxStages, STAGE_BYTES, kArgmaxThreads, 1>;
   constexpr int kBytes = kArgmaxStages * STAGE_BYTES;
   static bool configured = false;  // the attribute sticks to the function; set it once
@@ -709,24 +709,24 @@ static cudaError_t launch_row_argmax_ring_t(const void* logits, int64_t rows, in
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  return launch_kernel(kern, dim3(w.plan.grid), dim3(kArgmaxThreads), kBytes, st, true, static_cast<const T*>(logits),
+  return launch_kernel(kern, dim3(w.plan.grid), dim3(kArgmaxThreads), kBytes, st, early, static_cast<const T*>(logits),
                        rows * (int64_t)V, V, w.plan, w.part_key);
 }
 
 template <typename T>
 static cudaError_t launch_row_argmax_ring_t(const void* logits, int64_t rows, int V, const VerifyWorkspace& w,
-                                            size_t neighbour_smem, cudaStream_t st) {
+                                            size_t neighbour_smem, bool early, cudaStream_t st) {
   const bool roomy = kArgmaxStages * 65536 + neighbour_smem + 2 * kSmemPerCtaReserved <= (size_t)kSmemPerSm;
-  return roomy ? launch_row_argmax_ring_t<T, 65536>(logits, rows, V, w, st)
-               : launch_row_argmax_ring_t<T, 49152>(logits, rows, V, w, st);
+  return roomy ? launch_row_argmax_ring_t<T, 65536>(logits, rows, V, w, early, st)
+               : launch_row_argmax_ring_t<T, 49152>(logits, rows, V, w, early, st);
 }
 
 cudaError_t launch_row_argmax(const void* logits, int dtype, int64_t rows, int V, const VerifyWorkspace& w,
-                              size_t neighbour_smem, cudaStream_t st) {
+                              size_t neighbour_smem, bool early, cudaStream_t st) {
   if (rows == 0) return cudaSuccess;
   // rows that are whole 16-byte fragments go through the bulk-copy ring; other V use plain loads
-  if (dtype == UBT_BF16 && V % 8 == 0) return launch_row_argmax_ring_t<__nv_bfloat16>(logits, rows, V, w, neighbour_smem, st);
-  if (dtype == UBT_F32 && V % 4 == 0) return launch_row_argmax_ring_t<float>(logits, rows, V, w, neighbour_smem, st);
+  if (dtype == UBT_BF16 && V % 8 == 0) return launch_row_argmax_ring_t<__nv_bfloat16>(logits, rows, V, w, neighbour_smem, early, st);
+  if (dtype == UBT_F32 && V % 4 == 0) return launch_row_argmax_ring_t<float>(logits, rows, V, w, neighbour_smem, early, st);
   if (dtype == UBT_BF16) {
     if (V % 8 == 0) return launch_row_argmax_t<__nv_bfloat16, 8>(logits, rows, V, w, st);
     return launch_row_argmax_t<__nv_bfloat16, 1>(logits, rows, V, w, st);
@@ -748,7 +748,7 @@ static cudaError_t launch_row_sample_t(const void* logits, int64_t rows, int N, 
 template <typename T>
 static cudaError_t launch_row_sample_ring_t(const void* logits, int64_t rows, int N, int V, uint64_t seed,
                                             float temperature, int32_t* pick, const VerifyWorkspace& w,
-                                            cudaStream_t st) {
+                                            bool early, cudaStream_t st) {
   auto kern = k_row_weights_ring<T>;
   constexpr int kBytes = G5R_STAGES * G5R_STAGE_BYTES;
   static bool configured = false;
@@ -759,7 +759,7 @@ static cudaError_t launch_row_sample_ring_t(const void* logits, int64_t rows, in
   }
   int grid = device_info().sm_count * G5R_CTAS;
   if ((int64_t)grid > rows) grid = (int)rows;
-  cudaError_t e = launch_kernel(kern, dim3(grid), dim3(G5R_T), kBytes, st, true, static_cast<const T*>(logits), rows, V,
+  cudaError_t e = launch_kernel(kern, dim3(grid), dim3(G5R_T), kBytes, st, early, static_cast<const T*>(logits), rows, V,
                                 temperature, w.row_ac, w.block_sum, w.nblocks);
   if (e != cudaSuccess) return e;
   const int warps = 4;
@@ -769,14 +769,15 @@ static cudaError_t launch_row_sample_ring_t(const void* logits, int64_t rows, in
 }
 
 cudaError_t launch_row_sample(const void* logits, int dtype, int B, int N, int V, uint64_t seed,
-                              float temperature, int32_t* pick, const VerifyWorkspace& w, cudaStream_t st) {
+                              float temperature, int32_t* pick, const VerifyWorkspace& w, bool early,
+                              cudaStream_t st) {
   const int64_t rows = (int64_t)B * N;
   if (rows == 0) return cudaSuccess;
   // rows that are whole 16-byte fragments go through the bulk-copy ring; other V use plain loads
   if (dtype == UBT_BF16 && V % 8 == 0)
-    return launch_row_sample_ring_t<__nv_bfloat16>(logits, rows, N, V, seed, temperature, pick, w, st);
+    return launch_row_sample_ring_t<__nv_bfloat16>(logits, rows, N, V, seed, temperature, pick, w, early, st);
   if (dtype == UBT_F32 && V % 4 == 0)
-    return launch_row_sample_ring_t<float>(logits, rows, N, V, seed, temperature, pick, w, st);
+    return launch_row_sample_ring_t<float>(logits, rows, N, V, seed, temperature, pick, w, early, st);
   if (dtype == UBT_BF16) {
     if (V % 8 == 0) return launch_row_sample_t<__nv_bfloat16, 8>(logits, rows, N, V, seed, temperature, pick, st);
     return launch_row_sample_t<__nv_bfloat16, 1>(logits, rows, N, V, seed, temperature, pick, st);

@@ -1,0 +1,78 @@
+"""Host-side logic of the multi-GPU benchmark path, run as two gloo ranks on CPU.
+
+The hot path shards by sequence with no data-path collective (weak scaling): every rank runs the same step
+on its own batch, and the only exchanges are the barrier around the timed region and the max-over-ranks of
+the measured time.  These tests cover exactly that plumbing plus the reference arm under a two-rank launch.
+"""
+import json
+import os
+import socket
+import subprocess
+import sys
+
+import pytest
+import torch
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _rank_main(rank: int, world: int, port: int, out_dir: str):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    sys.path.insert(0, ROOT)
+    import bench
+    w, r, local = bench.dist_setup(world)
+    assert (w, r, local) == (world, rank, rank)
+    bench.barrier(w)
+    # every rank times its own steps; the job's time is the slowest rank's
+    mine = 10.0 + 2.5 * rank
+    job = bench.max_over_ranks(mine, w, torch.device("cpu"))
+    # whole-job throughput = units of all ranks / that time
+    trees = 32 * 4 * w / (job * 1e-3)
+    with open(os.path.join(out_dir, f"rank{rank}.json"), "w") as f:
+        json.dump({"job_ms": job, "trees_per_s": trees}, f)
+    bench.barrier(w)
+    import torch.distributed as dist
+    dist.destroy_process_group()
+
+
+@pytest.mark.timeout(180)
+def test_max_over_ranks_and_barrier_two_gloo_ranks(tmp_path):
+    port = _free_port()
+    mp.spawn(_rank_main, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    got = [json.load(open(tmp_path / f"rank{r}.json")) for r in range(2)]
+    assert got[0] == got[1]
+    assert got[0]["job_ms"] == 12.5
+    assert got[0]["trees_per_s"] == pytest.approx(32 * 4 * 2 / 12.5e-3)
+
+
+@pytest.mark.timeout(300)
+def test_reference_arm_under_a_two_rank_launch_prints_one_line():
+    port = _free_port()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.join(ROOT, "bench.py"),
+           "--impl", "reference", "--gpus", "2", "--steps", "1", "--warmup", "3", "--workload", "c1"]
+    env = dict(os.environ, CUDA_VISIBLE_DEVICES="")
+    p = subprocess.run(cmd, capture_output=True, text=True, cwd=ROOT, env=env, timeout=280)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [json.loads(l) for l in p.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    line = lines[0]
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+    assert line["config"]["workload"] == "c1"
+
+
+def test_ranks_draw_different_batches():
+    """Weak scaling: rank r's input set s is seeded 1000 r + s, so no two ranks stream the same bytes."""
+    sys.path.insert(0, ROOT)
+    import bench
+    seeds = {bench.input_seed(r, s) for r in range(8) for s in range(16)}
+    assert len(seeds) == 8 * 16

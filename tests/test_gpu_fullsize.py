@@ -98,3 +98,56 @@ def test_c4_full_batch_sampled():
 def test_c5_full_batch_sampled():
     _run_full("c5", sample=[0, 64, 127], seeds=(0, 12345))
     _CDF_CACHE.clear()
+
+
+def _same_tree(a, b):
+    for name in ("token_ids", "parents", "depths", "position_ids", "cand_rank", "scores", "mask", "n_nodes",
+                 "cand_ids", "cand_logprob"):
+        assert torch.equal(getattr(a, name), getattr(b, name)), name
+
+
+def _same_result(a, b):
+    for name in ("accepted_len", "bonus_token", "accepted_nodes", "out_tokens"):
+        assert torch.equal(getattr(a, name), getattr(b, name)), name
+
+
+@pytest.mark.parametrize("name", ["c3", "c5"])
+def test_back_to_back_calls_equal_separated_calls(name):
+    """Draft and verify enqueued with nothing between them run overlapped on the device (the verify call's
+    V-wide kernel starts while the draft's kernels are still running); the outcome must be bit-identical to the
+    same calls separated by a synchronisation, which the tests above check against the oracle."""
+    import paper_2609_39972_b200 as u
+    cfg = synth.CONFIGS[name].replace(B=32)
+    ud, bd, zd = synth.device_inputs(cfg, 5, DEV)
+    t_ref = u.ubt_draft_tree(ud, bd, cfg.k, cfg.N)
+    torch.cuda.synchronize()
+    r_ref = u.ubt_verify_tree(t_ref, zd, cfg.mode, seed=3)
+    torch.cuda.synchronize()
+    for _ in range(3):
+        t = u.ubt_draft_tree(ud, bd, cfg.k, cfg.N)
+        r = u.ubt_verify_tree(t, zd, cfg.mode, seed=3)
+        torch.cuda.synchronize()
+        _same_tree(t, t_ref)
+        _same_result(r, r_ref)
+
+
+def test_verify_scratch_that_reuses_a_draft_buffer_is_not_started_early():
+    """Stream order allows a caller to hand the draft call's logits buffer to the verify call as scratch.  The
+    library must then keep the verify kernel behind the draft instead of overlapping them."""
+    import paper_2609_39972_b200 as u
+    cfg = synth.CONFIGS["c3"]
+    ud, bd, zd = synth.device_inputs(cfg, 6, DEV)
+    t_ref = u.ubt_draft_tree(ud, bd, cfg.k, cfg.N)
+    torch.cuda.synchronize()
+    r_ref = u.ubt_verify_tree(t_ref, zd, "greedy")
+    torch.cuda.synchronize()
+    need = u.ubt_verify_workspace_bytes(cfg.B, cfg.N, cfg.V, "greedy")
+    for _ in range(3):
+        scratch = ud.clone()
+        ws = scratch.view(torch.uint8).reshape(-1)
+        assert ws.numel() >= need
+        t = u.ubt_draft_tree(scratch, bd, cfg.k, cfg.N)
+        r = u.ubt_verify_tree(t, zd, "greedy", ws=ws)        # overwrites the draft's logits
+        torch.cuda.synchronize()
+        _same_tree(t, t_ref)
+        _same_result(r, r_ref)

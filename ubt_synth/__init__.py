@@ -292,6 +292,23 @@ def device_inputs(cfg: Config, seed: int, device, want_target: bool = True):
     return u, big.contiguous(), z
 
 
+def boost_children_on_device(z, token_ids, parents, n_nodes, boost: float) -> None:
+    """Make device-resident target logits agree with a tree: in the row of every parent slot, the logit of
+    each child's token is raised by ``boost`` (in place, rounded to the tensor's dtype).  With boost near
+    log(V) a child is then picked with a probability of order one, so acceptance lengths are non-trivial.
+    """
+    import torch
+
+    B, N = token_ids.shape
+    slot = torch.arange(N, device=z.device)[None, :].expand(B, N)
+    live = (slot >= 1) & (slot < n_nodes[:, None].to(z.device))
+    b = torch.arange(B, device=z.device)[:, None].expand(B, N)[live]
+    par = parents.to(z.device)[live].long()
+    tok = token_ids.to(z.device)[live].long()
+    cur = z[b, par, tok].float() + float(boost)
+    z[b, par, tok] = cur.to(z.dtype)
+
+
 def to_host_bits(t) -> np.ndarray:
     """Host copy of a torch tensor in this module's host representation."""
     import torch
