@@ -350,7 +350,11 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
   const int tid = threadIdx.x, lane = tid & 31;
   const int64_t lo = (int64_t)blockIdx.x * plan.span;
   const int64_t hi = lo + plan.span < total ? lo + plan.span : total;
-  pdl_launch_dependents();  // the tree kernel may be scheduled; it waits for this grid before reading
+  // Launched programmatically: the CTAs may become resident while the kernel in front is still running.  Nothing
+  // is read or written before that kernel has completed; only then may the tree kernel behind this one be
+  // scheduled (it waits for this grid before it reads the partials).
+  pdl_wait();
+  pdl_launch_dependents();
   if (lo >= hi) return;
   const long long nslots = (total / V) * plan.smax;
   const Span<float> g_ms(part_ms, nslots * 2, 341), g_val(part_val, nslots * k, 342);
@@ -657,9 +661,8 @@ static cudaError_t launch_lse_topk_ring_t(const void* logits, int64_t rows, int 
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  kern<<<w.plan.grid, G1R_T, smem, st>>>(static_cast<const T*>(logits), rows * (int64_t)V, V, k, w.plan, w.part_ms,
-                                         w.part_val, w.part_idx, w.part_cnt);
-  return cudaGetLastError();
+  return launch_kernel(kern, dim3(w.plan.grid), dim3(G1R_T), smem, st, true, static_cast<const T*>(logits),
+                       rows * (int64_t)V, V, k, w.plan, w.part_ms, w.part_val, w.part_idx, w.part_cnt);
 }
 
 cudaError_t launch_lse_topk(const void* logits, int dtype, int64_t rows, int V, int k,

@@ -601,6 +601,7 @@ k_walk(ubt_tree tree, int mode, SpanPlan plan, const unsigned long long* __restr
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, N = tree.N, L = tree.L;
   const int64_t o = (int64_t)b * N;
   pdl_wait();  // picks and tree come from the kernels before this one
+  pdl_launch_dependents();  // a kernel behind this one may become resident; it has to wait for this grid itself
   for (int n = tid; n < N; n += blockDim.x) {
     int p;
     if (mode == UBT_VERIFY_GREEDY) {
