@@ -385,9 +385,10 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
     sg.at(pos, hi, V);
     if (tid == 0) { sh.cnt = 0; sh.ntop = 0; sh.taux = -INFINITY; }
     float ref = -1.0e30f, negref = 1.0e30f * kLog2e;  // ref = -1e30: not fixed yet
-    float acc[G1R_GROUP];
+    unsigned long long acc[G1R_GROUP];  // packed pairs of partial sums (one FADD2 adds two exponentials)
 #pragma unroll
-    for (int u = 0; u < G1R_GROUP; ++u) acc[u] = 0.f;
+    for (int u = 0; u < G1R_GROUP; ++u) acc[u] = 0ull;
+    const unsigned long long l2e2 = pack2(kLog2e, kLog2e);
 
     for (int c = 0; c < sg.len; c += STAGE_ELEMS) {
       const int l = sg.len - c < STAGE_ELEMS ? sg.len - c : STAGE_ELEMS;
@@ -454,7 +455,7 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
           if (gmax > ref + 60.f || (ref < -1.0e29f && gmax > -INFINITY)) {  // move the reference up
             const float sc = ex2_approx(fmaf(ref, kLog2e, -gmax * kLog2e));
 #pragma unroll
-            for (int u = 0; u < G1R_GROUP; ++u) acc[u] *= sc;
+            for (int u = 0; u < G1R_GROUP; ++u) acc[u] = fma2(acc[u], pack2(sc, sc), 0ull);
             ref = gmax;
             negref = -gmax * kLog2e;
           }
@@ -465,7 +466,11 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
 #pragma unroll
         for (int u = 0; u < G1R_GROUP; ++u) {
 #pragma unroll
-          for (int j = 0; j < VEC; ++j) acc[u] += ex2_approx(fmaf(x[u][j], kLog2e, negref));
+          for (int j = 0; j < VEC; j += 2) {
+            float y0, y1;
+            unpack2(fma2(pack2(x[u][j], x[u][j + 1]), l2e2, pack2(negref, negref)), y0, y1);
+            acc[u] = add2(acc[u], pack2(ex2_approx(y0), ex2_approx(y1)));
+          }
         }
       }
       for (; f0 < nfrag; f0 += G1R_T) {  // ragged end of a chunk, one fragment per vote
@@ -486,14 +491,18 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
           if (vm > ref + 60.f || (ref < -1.0e29f && vm > -INFINITY)) {
             const float sc = ex2_approx(fmaf(ref, kLog2e, -vm * kLog2e));
 #pragma unroll
-            for (int u = 0; u < G1R_GROUP; ++u) acc[u] *= sc;
+            for (int u = 0; u < G1R_GROUP; ++u) acc[u] = fma2(acc[u], pack2(sc, sc), 0ull);
             ref = vm;
             negref = -vm * kLog2e;
           }
           if (vm > taux) append_hits<VEC>(sh, x, taux, colbase + f0 * VEC);
         }
 #pragma unroll
-        for (int j = 0; j < VEC; ++j) acc[0] += ex2_approx(fmaf(x[j], kLog2e, negref));
+        for (int j = 0; j < VEC; j += 2) {
+          float y0, y1;
+          unpack2(fma2(pack2(x[j], x[j + 1]), l2e2, pack2(negref, negref)), y0, y1);
+          acc[0] = add2(acc[0], pack2(ex2_approx(y0), ex2_approx(y1)));
+        }
       }
 
       GT(4);
@@ -551,7 +560,12 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
     flush_keyed(sh, k);
 
     // partial (max, sum exp) of the segment from the per-thread (reference, sum) pairs
-    const float s_t = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+    float s_t;
+    {
+      float a0, a1;
+      unpack2(add2(add2(acc[0], acc[1]), add2(acc[2], acc[3])), a0, a1);
+      s_t = a0 + a1;
+    }
     float mw = ref;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mw = fmaxf(mw, __shfl_xor_sync(FULL, mw, o));
