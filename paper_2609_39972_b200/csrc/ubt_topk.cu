@@ -451,7 +451,9 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
           for (int j = 0; j < VEC; ++j) { x[u][j] = fr.x[j]; vmax[u] = fmaxf(vmax[u], fr.x[j]); }
         }
         const float gmax = fmaxf(fmaxf(vmax[0], vmax[1]), fmaxf(vmax[2], vmax[3]));
-        if (__any_sync(FULL, gmax > taux)) {  // rare: a candidate somewhere in the warp's 4 fragments
+        // rare: a candidate somewhere in the warp's 4 fragments, or an element far above a lane's reference (the
+        // bound rises with what OTHER warps have seen, so a non-candidate can still overflow 2^((x - ref) log2 e))
+        if (__any_sync(FULL, gmax > fminf(taux, ref + 60.f))) {
           if (gmax > ref + 60.f || (ref < -1.0e29f && gmax > -INFINITY)) {  // move the reference up
             const float sc = ex2_approx(fmaf(ref, kLog2e, -gmax * kLog2e));
 #pragma unroll
@@ -487,7 +489,7 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
         float vm = x[0];
 #pragma unroll
         for (int j = 1; j < VEC; ++j) vm = fmaxf(vm, x[j]);
-        if (__any_sync(FULL, vm > taux)) {
+        if (__any_sync(FULL, vm > fminf(taux, ref + 60.f))) {
           if (vm > ref + 60.f || (ref < -1.0e29f && vm > -INFINITY)) {
             const float sc = ex2_approx(fmaf(ref, kLog2e, -vm * kLog2e));
 #pragma unroll

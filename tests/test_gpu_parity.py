@@ -163,6 +163,33 @@ def test_rows_full_of_ties():
         assert pick.cpu().numpy()[0].tolist() == np.argmax(synth.as_f32(host, dtype), -1).tolist()
 
 
+def test_rows_whose_level_jumps_inside_one_warps_share():
+    """Rows built against the streaming kernel's layout: a chunk of zeros, then a chunk in which only the
+    elements that one warp reads are at 100 (so the CTA-wide bound rises to 100 without the other warps ever
+    seeing a candidate), then a chunk of 95s, which are no candidates but lie far above those warps' exponent
+    reference.  The sum of exponentials must survive that."""
+    u = ubt()
+    V, k, rows = 65536, 8, 512
+    chunk, frag = 16384, 8
+    e = np.arange(V)
+    row = np.zeros(V, np.float32)
+    in1 = (e >= chunk) & (e < 2 * chunk)
+    row[in1 & (((e % chunk) // frag) % 256 < 32)] = 100.0
+    row[(e >= 2 * chunk) & (e < 3 * chunk)] = 95.0
+    rng = np.random.default_rng(3)
+    x = np.tile(row, (rows, 1)) + rng.integers(0, 4, (rows, V)).astype(np.float32) * 0.25
+    host = synth.f32_to_bf16_bits(x)
+    ids, lp, _ = oracle.topk_logprob(host, k)
+    d = synth.to_device(host, "bf16", DEV)
+    cid = torch.empty((rows, k), dtype=torch.int32, device=DEV)
+    clp = torch.empty((rows, k), dtype=torch.float32, device=DEV)
+    ws = u.workspace(u.ubt_draft_workspace_bytes(rows, 1, V, k, 1), DEV)
+    u.ubt_topk_logprob(d, k, cid, clp, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(cid.cpu().numpy(), ids)
+    np.testing.assert_allclose(clp.cpu().numpy(), lp, rtol=1e-5, atol=1e-5)
+
+
 def test_exact_score_ties_follow_total_order():
     # integer-valued inputs with lambda = 0: many node scores are exactly equal in fp32 and in double
     u = ubt()
