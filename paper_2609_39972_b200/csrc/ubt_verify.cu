@@ -283,14 +283,17 @@ __device__ __forceinline__ unsigned long long weight_of(float z, float a, float 
 // Two weights at once with the packed fp32 instructions of sm_100 (fma/add .f32x2): the same IEEE operations
 // per component as weight_of, half the issue slots for the arithmetic part.
 struct WeightConsts2 {  // the routine's constants, duplicated into both halves
-  unsigned long long a, c, big, nbig, none, c5, c4, c3, c2, c1, one;
+  // The polynomial's coefficients carry the factor 2^40 of the weight: scaling every Horner step by a power of
+  // two changes no rounding, so the mantissa bits are those of weight_of and the exponent insert is one add.
+  unsigned long long a, c, big, nbig, none, c5, c4, c3, c2, c1, c0;
   __device__ __forceinline__ void init(float a_, float c_) {
+    const float s = 0x1p+40f;
     a = pack2(a_, a_); c = pack2(c_, c_);
     big = pack2(12582912.0f, 12582912.0f); nbig = pack2(-12582912.0f, -12582912.0f);
     none = pack2(-1.0f, -1.0f);
-    c5 = pack2(0x1.5c7746p-10f, 0x1.5c7746p-10f); c4 = pack2(0x1.3cea8p-7f, 0x1.3cea8p-7f);
-    c3 = pack2(0x1.c6b54ap-5f, 0x1.c6b54ap-5f); c2 = pack2(0x1.ebf9bcp-3f, 0x1.ebf9bcp-3f);
-    c1 = pack2(0x1.62e42cp-1f, 0x1.62e42cp-1f); one = pack2(1.0f, 1.0f);
+    c5 = pack2(0x1.5c7746p-10f * s, 0x1.5c7746p-10f * s); c4 = pack2(0x1.3cea8p-7f * s, 0x1.3cea8p-7f * s);
+    c3 = pack2(0x1.c6b54ap-5f * s, 0x1.c6b54ap-5f * s); c2 = pack2(0x1.ebf9bcp-3f * s, 0x1.ebf9bcp-3f * s);
+    c1 = pack2(0x1.62e42cp-1f * s, 0x1.62e42cp-1f * s); c0 = pack2(s, s);
   }
 };
 __device__ __forceinline__ unsigned long long weight_pair_sum(float z0, float z1, const WeightConsts2& k) {
@@ -304,13 +307,20 @@ __device__ __forceinline__ unsigned long long weight_pair_sum(float z0, float z1
   p = fma2(p, f, k.c3);
   p = fma2(p, f, k.c2);
   p = fma2(p, f, k.c1);
-  p = fma2(p, f, k.one);
+  p = fma2(p, f, k.c0);
   float p0, p1, t0, t1;
   unpack2(p, p0, p1);
   unpack2(tmp, t0, t1);
-  const uint32_t e0 = __float_as_uint(p0) + ((__float_as_uint(t0) + 40u) << 23);
-  const uint32_t e1 = __float_as_uint(p1) + ((__float_as_uint(t1) + 40u) << 23);
+  // the low mantissa bits of tmp hold n; shifted into the exponent field (the higher bits fall off the word)
+  const uint32_t e0 = __float_as_uint(p0) + (__float_as_uint(t0) << 23);
+  const uint32_t e1 = __float_as_uint(p1) + (__float_as_uint(t1) << 23);
   return __float2ull_rz(__uint_as_float(e0)) + __float2ull_rz(__uint_as_float(e1));
+}
+// Sum over the warp of per-lane sums below 2^46 (32 weights below 2^41 each): two 23-bit pieces, each summed
+// by one warp-wide integer reduction.
+__device__ __forceinline__ unsigned long long warp_sum_below_2p46(unsigned long long v) {
+  const unsigned lo = (unsigned)v & 0x7fffffu, hi = (unsigned)(v >> 23);
+  return (unsigned long long)__reduce_add_sync(FULL, lo) + ((unsigned long long)__reduce_add_sync(FULL, hi) << 23);
 }
 
 constexpr int G5_CHUNK = 1024;  // tokens per partial sum
@@ -483,17 +493,27 @@ k_row_weights_ring(const T* __restrict__ logits, int64_t rows, int V, float temp
         const int nblk = (nfrag + BF - 1) / BF;
         for (int blk = warp; blk < nblk; blk += G5R_T / 32) {
           unsigned long long acc = 0;
+          if ((blk + 1) * BF <= nfrag) {  // whole block: no bounds checks
 #pragma unroll
-          for (int q = 0; q < BF / 32; ++q) {
-            const int f = blk * BF + q * 32 + lane;
-            if (f < nfrag) {
+            for (int q = 0; q < BF / 32; ++q) {
               Frag<T> x;
-              x.unpack(stage[f]);
+              x.unpack(stage[blk * BF + q * 32 + lane]);
 #pragma unroll
               for (int j = 0; j < VEC; j += 2) acc += weight_pair_sum(x.x[j], x.x[j + 1], wc);
             }
+          } else {
+            for (int q = 0; q < BF / 32; ++q) {
+              const int f = blk * BF + q * 32 + lane;
+              if (f < nfrag) {
+                Frag<T> x;
+                x.unpack(stage[f]);
+#pragma unroll
+                for (int j = 0; j < VEC; j += 2) acc += weight_pair_sum(x.x[j], x.x[j + 1], wc);
+              }
+            }
           }
-          acc = warp_sum_u64(acc);
+          static_assert((BF / 32) * VEC == 32, "a lane sums 32 weights per block");
+          acc = warp_sum_below_2p46(acc);
           if (lane == 0) block_sum[row * nblocks + c0 / G5_CHUNK + blk] = acc;
         }
       } else {
