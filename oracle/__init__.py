@@ -52,6 +52,9 @@ def lib() -> C.CDLL:
         _lib.ubt_oracle_walks_from_cdf.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p,
                                                    C.c_uint32, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         _lib.ubt_oracle_weight_consts.argtypes = [C.c_float, C.c_float, C.c_void_p, C.c_void_p]
+        _lib.ubt_oracle_selector_scores.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int, C.c_void_p,
+                                                    C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p,
+                                                    C.c_void_p]
     return _lib
 
 
@@ -91,6 +94,32 @@ def topk_logprob(logits: np.ndarray, k: int):
     if rc:
         raise ValueError("oracle topk_logprob rejected its arguments")
     return ids, lp, lse
+
+
+def selector_scores(phi: np.ndarray, psi: np.ndarray, gate: np.ndarray, cand_ids: np.ndarray,
+                    anchor_tokens: Optional[np.ndarray] = None):
+    """Selector scores of all candidate pairs (Section 3.1.2, "Parallel Computation").
+
+    ``phi``, ``psi``: codebook tables ``[V, R]`` (fp32, or bf16 bit patterns as uint16); ``gate[B, L, R]`` fp32 is
+    the projected proposer state of each position; ``cand_ids[B, L, k]``.  Returns ``(bigram[B, L-1, k, k] f64,
+    anchor_bigram[B, k] f64 or None)``.
+    """
+    phi = np.ascontiguousarray(phi); psi = np.ascontiguousarray(psi)
+    gate = np.ascontiguousarray(gate, np.float32); cand_ids = np.ascontiguousarray(cand_ids, np.int32)
+    V, R = phi.shape
+    B, L, k = cand_ids.shape
+    assert psi.shape == (V, R) and gate.shape == (B, L, R) and phi.dtype == psi.dtype
+    big = np.zeros((B, max(L - 1, 0), k, k), np.float64)
+    anc = None
+    if anchor_tokens is not None:
+        anchor_tokens = np.ascontiguousarray(anchor_tokens, np.int32)
+        anc = np.zeros((B, k), np.float64)
+    rc = lib().ubt_oracle_selector_scores(_p(phi), _p(psi), _dtype_code(phi), V, R, _p(gate), _p(cand_ids),
+                                          _p(anchor_tokens) if anchor_tokens is not None else None, B, L, k,
+                                          _p(big), _p(anc) if anc is not None else None)
+    if rc:
+        raise ValueError("oracle selector_scores rejected its arguments")
+    return big, anc
 
 
 @dataclass

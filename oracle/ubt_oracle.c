@@ -94,6 +94,49 @@ int ubt_oracle_topk_logprob(const void *logits, int dtype, int64_t rows, int V, 
 }
 
 /* ---------------------------------------------------------------------- */
+/* Selector scores (Section 3.1.2, "Parallel Computation", the edge-matrix   */
+/* equation; the score of one pair is the low-rank bigram selector of        */
+/* Section 2): for predecessor token a and successor token b at position i,  */
+/*   delta_i(a, b) = sum_r g_i[r] * phi[a][r] * psi[b][r],                   */
+/* g_i = P(h_i) being the projected proposer state of the SUCCESSOR position */
+/* and phi, psi the vocabulary-wide codebook tables.  Predecessors are the   */
+/* candidates of position i-1; for the first position the only predecessor   */
+/* is the anchor token.  Outputs: bigram[b][j][ra][rb] = delta between the   */
+/* rank-ra candidate of position j and the rank-rb candidate of position j+1 */
+/* (gate of position j+1); anchor_bigram[b][rb] = delta between the anchor   */
+/* and the rank-rb candidate of position 0 (gate of position 0).  The sum    */
+/* runs over r in index order, in double.                                    */
+/* ---------------------------------------------------------------------- */
+int ubt_oracle_selector_scores(const void *phi, const void *psi, int dtype, int64_t V, int R, const float *gate,
+                               const int32_t *cand_ids, const int32_t *anchor_tokens, int B, int L, int k,
+                               double *bigram, double *anchor_bigram) {
+  if (!phi || !psi || !gate || !cand_ids || B < 0 || L < 1 || k < 1 || R < 1 || V < 1) return 1;
+  if (anchor_bigram && !anchor_tokens) return 1;
+  int bad = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int b = 0; b < B; ++b) {
+    for (int i = 0; i < L; ++i) {
+      const float *g = gate + ((int64_t)b * L + i) * R;
+      const int npred = i == 0 ? 1 : k;
+      if (i == 0 && !anchor_bigram) continue;
+      for (int ra = 0; ra < npred; ++ra) {
+        const int64_t a = i == 0 ? anchor_tokens[b] : cand_ids[((int64_t)b * L + i - 1) * k + ra];
+        for (int rb = 0; rb < k; ++rb) {
+          const int64_t t = cand_ids[((int64_t)b * L + i) * k + rb];
+          if (a < 0 || a >= V || t < 0 || t >= V) { bad = 1; continue; }
+          double sum = 0.0;
+          for (int r = 0; r < R; ++r)
+            sum += (double)g[r] * (double)load_f32(phi, dtype, a * R + r) * (double)load_f32(psi, dtype, t * R + r);
+          if (i == 0) anchor_bigram[(int64_t)b * k + rb] = sum;
+          else bigram[(((int64_t)b * (L - 1) + i - 1) * k + ra) * k + rb] = sum;
+        }
+      }
+    }
+  }
+  return bad;
+}
+
+/* ---------------------------------------------------------------------- */
 /* Steps 2-3.  Tree construction (Appendix A, Algorithm 1).                 */
 /* ---------------------------------------------------------------------- */
 typedef struct {

@@ -292,6 +292,22 @@ def device_inputs(cfg: Config, seed: int, device, want_target: bool = True):
     return u, big.contiguous(), z
 
 
+def selector_tables(V: int, R: int, B: int, L: int, seed: int, dtype: str = "bf16"):
+    """Synthetic stand-ins for the selector's precomputed codebook tables and gate vectors.
+
+    Returns ``(phi[V,R], psi[V,R], gate[B,L,R] fp32)``; tables are N(0,1) in the given dtype (bf16 as bit
+    patterns), gates N(0, 1/R), so that a pair score, a sum of R products, has unit scale like the
+    configurations' bigram scores.
+    """
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, 0x5E1EC7])))
+    phi = rng.standard_normal((V, R), dtype=np.float32)
+    psi = rng.standard_normal((V, R), dtype=np.float32)
+    gate = (rng.standard_normal((B, L, R), dtype=np.float32) / np.sqrt(np.float32(R))).astype(np.float32)
+    if dtype == "bf16":
+        phi, psi = f32_to_bf16_bits(phi), f32_to_bf16_bits(psi)
+    return phi, psi, gate
+
+
 def boost_children_on_device(z, token_ids, parents, n_nodes, boost: float) -> None:
     """Make device-resident target logits agree with a tree: in the row of every parent slot, the logit of
     each child's token is raised by ``boost`` (in place, rounded to the tensor's dtype).  With boost near
