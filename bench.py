@@ -139,11 +139,18 @@ def barrier(world: int):
         dist.barrier()
 
 
-def oracle_pass(cfg, uh, bh, zh, seed):
-    """One oracle draft+verify pass on host arrays; returns (tree, verdict, seconds)."""
+def oracle_pass(cfg, uh, bh, zh, seed, phi=None, psi=None, gate=None, anchor=None, W=0):
+    """One oracle draft+verify pass on host arrays; returns (tree, verdict, seconds).  With selector tables the
+    bigram scores come from the oracle's selector (the paper's data flow) instead of ``bh``."""
     import oracle
     t0 = time.perf_counter()
-    tr = oracle.draft_tree(uh, bh, cfg.k, cfg.N)
+    if phi is not None:
+        ids, _, _ = oracle.topk_logprob(uh, cfg.k)
+        big, anc = oracle.selector_scores(phi, psi, gate, ids, anchor)
+        tr = oracle.draft_tree(uh, big.astype(np.float32), cfg.k, cfg.N, W=W, anchor_bigram=anc.astype(np.float32),
+                               anchor_tokens=anchor)
+    else:
+        tr = oracle.draft_tree(uh, bh, cfg.k, cfg.N)
     v = oracle.verify(tr.token_ids, tr.parents, tr.n_nodes, cfg.L, zh, cfg.mode, seed=seed)
     return tr, v, time.perf_counter() - t0
 
@@ -183,7 +190,7 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c3", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--workload", default="c3", choices=sorted(synth.CONFIGS) + sorted(synth.NEXT_CONFIGS))
     ap.add_argument("--ref-trees", type=int, default=4, help="sequences per step of the reference arm")
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time budget of the oracle baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -192,7 +199,11 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    cfg = synth.CONFIGS[args.workload]
+    cfg = synth.CONFIGS.get(args.workload) or synth.NEXT_CONFIGS[args.workload]
+    # the paper's own configuration goes through the split entry points, selector scores computed on the device
+    paper_flow = args.workload in synth.NEXT_CONFIGS
+    if paper_flow:
+        args.no_e2e = True          # the host-buffer forms cover the fused call only
     if args.batch > 0:
         cfg = cfg.replace(B=args.batch, name=f"{cfg.name}-B{args.batch}")
     world, rank, local = dist_setup(args.gpus)
@@ -227,9 +238,25 @@ def main():
     for a, b in ev_pairs:           # create the underlying cudaEvent_t handles
         a.record(stream); b.record(stream)
 
+    if paper_flow:
+        R, W = synth.SELECTOR_RANK, synth.PAPER_SEARCH_WIDTH
+        phi, psi, gate, anchor = synth.device_selector_tables(cfg.V, R, cfg.B, cfg.L, input_seed(rank, 99), dev)
+        sel_big = torch.empty((cfg.B, cfg.L - 1, cfg.k, cfg.k), dtype=torch.float32, device=dev)
+        sel_anc = torch.empty((cfg.B, cfg.k), dtype=torch.float32, device=dev)
+
+    def draft(ud, bd):
+        if paper_flow:
+            ubt.ubt_topk_logprob(ud, cfg.k, tree.cand_ids, tree.cand_logprob, ws_d, stream=stream)
+            ubt.ubt_selector_scores(phi, psi, gate, tree.cand_ids, anchor, bigram_scores=sel_big,
+                                    anchor_bigram=sel_anc, stream=stream)
+            ubt.ubt_build_tree(sel_big, tree, stream=stream, search_width=W, anchor_bigram=sel_anc,
+                               anchor_tokens=anchor)
+        else:
+            ubt.ubt_draft_tree(ud, bd, cfg.k, cfg.N, tree=tree, ws=ws_d, stream=stream)
+
     def step(i, events=None):
         ud, bd, zd = sets[i % n_sets]
-        ubt.ubt_draft_tree(ud, bd, cfg.k, cfg.N, tree=tree, ws=ws_d, stream=stream)
+        draft(ud, bd)
         ubt.ubt_verify_tree(tree, zd, cfg.mode, seed=i, temperature=1.0, result=res, ws=ws_v, stream=stream,
                             event_before=events[0] if events else None, event_after=events[1] if events else None)
 
@@ -271,7 +298,7 @@ def main():
     for i in range(min(args.steps, 20)):
         ud, bd, zd = sets[i % n_sets]
         ea.record(stream)
-        ubt.ubt_draft_tree(ud, bd, cfg.k, cfg.N, tree=tree, ws=ws_d, stream=stream)
+        draft(ud, bd)
         eb.record(stream)
         ubt.ubt_verify_tree(tree, zd, cfg.mode, seed=i, result=res, ws=ws_v, stream=stream)
         ec.record(stream)
@@ -281,6 +308,8 @@ def main():
     peak, peak_kind = measured_peak()
     e = 2 if cfg.dtype == "bf16" else 4
     launches_per_step = 2 + (2 if cfg.mode == "greedy" else 3)   # top-k, tree | argmax or weights+pick, walk
+    if paper_flow:
+        launches_per_step += 2                                   # separate merge kernel, selector scores
     kern_bytes = cfg.B * cfg.N * cfg.V * e
     if cfg.mode == "greedy":
         # HBM-bound: one read of every target logit
@@ -316,6 +345,9 @@ def main():
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": cfg.name, "B": cfg.B, "L": cfg.L, "V": cfg.V, "k": cfg.k, "node_budget": cfg.N,
                    "verify": cfg.mode, "logits": cfg.dtype, "input_sets": n_sets,
+                   **({"search_width": synth.PAPER_SEARCH_WIDTH, "selector_rank": synth.SELECTOR_RANK,
+                       "flow": "ubt_topk_logprob -> ubt_selector_scores -> ubt_build_tree -> ubt_verify_tree"}
+                      if paper_flow else {}),
                    "l2": "inputs larger than L2 (rotation of %d MB)" % (batch_bytes * n_sets // 1_000_000)},
         "hbm": {"bytes_per_tree": bpt["total"], "step_gbs_per_gpu": step_gbs / world,
                 "frac_of_%s_peak" % peak_kind: step_gbs / world / peak,
@@ -367,20 +399,27 @@ def main():
         sample = max(1, min(cfg.B, 8))
         uh, bh, zh = (synth.to_host_bits(t[:sample]) for t in (ud, bd, zd))
         done, spent, tr = 0, 0.0, None
+        kw = {}
+        if paper_flow:
+            sample = max(1, min(cfg.B, 2))
+            uh, zh = (synth.to_host_bits(t[:sample]) for t in (ud, zd))
+            kw = dict(phi=synth.to_host_bits(phi), psi=synth.to_host_bits(psi), gate=gate[:sample].cpu().numpy(),
+                      anchor=anchor[:sample].cpu().numpy(), W=synth.PAPER_SEARCH_WIDTH)
         while spent < args.cpu_seconds:
-            tr, ov, dt = oracle_pass(cfg, uh, bh, zh, 0)
+            tr, ov, dt = oracle_pass(cfg, uh, bh, zh, 0, **kw)
             done += sample; spent += dt
         line["cpu_baseline"] = {"value": done / spent, "unit": "trees/s", "cores": oracle.num_threads(),
                                 "kind": "oracle", "sample": f"first {sample} of {cfg.B} sequences, repeated for "
                                                             f"{spent:.1f} s ({done} trees)"}
         # live parity of the bench configuration on that sample
-        ubt.ubt_draft_tree(ud, bd, cfg.k, cfg.N, tree=tree, ws=ws_d, stream=stream)
+        draft(ud, bd)
         pick = torch.empty((cfg.B, cfg.N), dtype=torch.int32, device=dev)
         ubt.ubt_verify_tree(tree, zd, cfg.mode, seed=0, result=res, ws=ws_v, stream=stream, node_pick=pick)
         torch.cuda.synchronize()
         try:
             g = tree_to_numpy(tree)
-            swaps = compare_draft(g, tr, cfg.L, cfg.k, cfg.N, rows=list(range(sample)))
+            swaps = compare_draft(g, tr, cfg.L, cfg.k, cfg.N, synth.PAPER_SEARCH_WIDTH if paper_flow else 0, 0.0,
+                                  kw.get("anchor"), None, rows=list(range(sample)))
             if not swaps:
                 compare_verify(res, ov, pick, rows=slice(0, sample))
             line["parity"] = {"checked_trees": sample, "near_tie_swaps": len(swaps), "ok": True}

@@ -23,8 +23,10 @@
  * Sizes: B sequences, L draft positions (the paper's gamma), V vocabulary, k candidates per position
  * (the paper's K), N = node budget = tree slots INCLUDING the root (the paper's budget B counts
  * non-root nodes only, so its B equals N - 1).
- * Limits (else UBT_ERR_UNSUPPORTED): 1 <= k <= 64, k <= V < 2^31, 1 <= N <= 256, 1 <= L <= 64,
- * and the per-sequence pair table L*k*k*5 bytes must fit in 160 KiB of shared memory.
+ * Limits (else UBT_ERR_UNSUPPORTED): 1 <= k <= 64, k <= V < 2^31, 1 <= N <= 256, 1 <= L <= 64.
+ * While the per-sequence pair table (L*k*k*5 bytes) fits in 160 KiB of shared memory all its rows are
+ * prepared in parallel; larger shapes (the paper's K = 64 with 15 positions is one) are served from a
+ * cache of the rows the search touches, each prepared when first needed -- same result, more latency.
  */
 #ifndef UBT_H_
 #define UBT_H_
@@ -128,6 +130,28 @@ int ubt_topk_logprob(const void *logits, int dtype, int64_t rows, int V, int k, 
  */
 int ubt_build_tree(const float *bigram_scores, int B, int L, int k, int node_budget,
                    const ubt_draft_opts *opts, ubt_tree *out, void *cuda_stream);
+
+/*
+ * The step between a1 and a2 in the paper's data flow (Section 3.1.2, "Parallel Computation": the
+ * edge matrix Delta_i = Phi_{i-1} diag(P(h_i)) Psi_i^T): the selector score of every
+ * (predecessor candidate, successor candidate) pair from the precomputed codebook tables,
+ *   delta_i(a, b) = sum_r gate[b, i, r] * phi[a, r] * psi[b, r].
+ * phi, psi: [V, R] row-major device tables of `table_dtype` (ubt_dtype), 16-byte aligned, R a
+ * multiple of 8 (bf16) / 4 (fp32), R <= 8192; gate: [B, L, R] fp32, the projected proposer
+ * state P(h_i) of each position; cand_ids: [B, L, k] as written by ubt_topk_logprob (every id in
+ * [0, V); ids outside give unspecified but memory-safe scores).  Writes
+ *   bigram_scores[b, j, ra, rb] (j < L-1): rank-ra candidate of position j -> rank-rb candidate of
+ *     position j+1, gate of position j+1                              ([B, L-1, k, k] fp32), and,
+ *   if anchor_tokens and anchor_bigram are both non-NULL, anchor_bigram[b, rb]: anchor token ->
+ *     rank-rb candidate of position 0, gate of position 0             ([B, k] fp32),
+ * i.e. exactly the selector inputs of ubt_build_tree.  Products and sums are fp32 (fma) in the
+ * order of r; results agree with a double-precision sum to about 1e-6 * sum_r |term|.  No workspace.  Errors as for the other calls.
+ */
+int ubt_selector_scores(const void *phi, const void *psi, int table_dtype, int V, int R,
+                        const float *gate, const int32_t *cand_ids,
+                        const int32_t *anchor_tokens /* [B] or NULL */, int B, int L, int k,
+                        float *bigram_scores, float *anchor_bigram /* [B,k] or NULL */,
+                        void *cuda_stream);
 
 /*
  * Step a3b alone: position ids and the ancestor bitmask from parents / depths / n_nodes of `tree`

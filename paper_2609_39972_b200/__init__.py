@@ -3,7 +3,7 @@
 ``binding`` holds thin ctypes wrappers with the names of the C entry points; the CUDA library itself
 is ``libubt.so`` next to this file, built by ``_build.build()``.
 """
-from .binding import (Tree, ubt_debug_ring_timeouts, UbtError, VerifyResult, load, status_string, ubt_build_mask, ubt_build_tree,
+from .binding import (Tree, ubt_debug_ring_timeouts, UbtError, VerifyResult, load, status_string, ubt_build_mask, ubt_build_tree, ubt_selector_scores,
                       ubt_draft_host_buffer_bytes, ubt_draft_tree, ubt_draft_tree_host, ubt_draft_workspace_bytes,
                       ubt_topk_logprob, ubt_verify_host_buffer_bytes, ubt_verify_tree, ubt_verify_tree_host, ubt_verify_tree_static, ubt_verify_static_capacity,
                       ubt_verify_workspace_bytes, ubt_version, workspace)

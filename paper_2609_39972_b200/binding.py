@@ -52,7 +52,7 @@ class _VerifyResult(C.Structure):
 
 
 EXPORTS = ["ubt_version", "ubt_status_string", "ubt_debug_ring_timeouts", "ubt_draft_workspace_bytes", "ubt_verify_workspace_bytes",
-           "ubt_topk_logprob", "ubt_build_tree", "ubt_build_mask", "ubt_draft_tree", "ubt_verify_tree",
+           "ubt_topk_logprob", "ubt_selector_scores", "ubt_build_tree", "ubt_build_mask", "ubt_draft_tree", "ubt_verify_tree",
            "ubt_draft_host_buffer_bytes", "ubt_verify_host_buffer_bytes", "ubt_draft_tree_host",
            "ubt_verify_tree_host", "ubt_verify_tree_static", "ubt_verify_static_capacity"]
 
@@ -88,6 +88,8 @@ def load() -> C.CDLL:
                                    C.c_void_p, C.c_size_t, C.c_void_p]
     L.ubt_build_tree.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
     L.ubt_build_mask.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+    L.ubt_selector_scores.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
+                                      C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
     L.ubt_draft_tree.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                  C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
     L.ubt_verify_tree.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
@@ -229,6 +231,28 @@ def ubt_build_tree(bigram_scores: Optional[torch.Tensor], tree: Tree, stream=Non
     t = tree.c_struct()
     _check(load().ubt_build_tree(_ptr(bigram_scores), tree.B, tree.L, tree.k, tree.N, C.byref(o), C.byref(t),
                                  _stream(stream)), "ubt_build_tree")
+
+
+def ubt_selector_scores(phi: torch.Tensor, psi: torch.Tensor, gate: torch.Tensor, cand_ids: torch.Tensor,
+                        anchor_tokens: Optional[torch.Tensor] = None, bigram_scores: Optional[torch.Tensor] = None,
+                        anchor_bigram: Optional[torch.Tensor] = None, stream=None):
+    """Selector scores of all candidate pairs from the codebook tables ``phi``, ``psi`` ``[V,R]`` and the gate
+    vectors ``gate[B,L,R]`` (the step between ``ubt_topk_logprob`` and ``ubt_build_tree``).
+
+    Returns ``(bigram_scores[B,L-1,k,k], anchor_bigram[B,k] or None)``.
+    """
+    for t, n in ((phi, "phi"), (psi, "psi"), (gate, "gate"), (cand_ids, "cand_ids")):
+        _need(t, n)
+    V, R = phi.shape
+    B, L, k = cand_ids.shape
+    if bigram_scores is None:
+        bigram_scores = torch.empty((B, max(L - 1, 0), k, k), dtype=torch.float32, device=phi.device)
+    if anchor_tokens is not None and anchor_bigram is None:
+        anchor_bigram = torch.empty((B, k), dtype=torch.float32, device=phi.device)
+    _check(load().ubt_selector_scores(_ptr(phi), _ptr(psi), _dtype_code(phi), V, R, _ptr(gate), _ptr(cand_ids),
+                                      _ptr(anchor_tokens), B, L, k, _ptr(bigram_scores), _ptr(anchor_bigram),
+                                      _stream(stream)), "ubt_selector_scores")
+    return bigram_scores, anchor_bigram
 
 
 def ubt_build_mask(tree: Tree, pos_offset: Optional[torch.Tensor] = None, stream=None) -> None:

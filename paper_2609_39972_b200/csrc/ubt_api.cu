@@ -34,7 +34,6 @@ static size_t esize(int dtype) { return dtype == UBT_BF16 ? 2 : 4; }
 static int check_shape(int B, int L, int V, int k, int N) {
   if (B < 0 || L < 1 || V < 1 || k < 1 || N < 1 || k > V) return UBT_ERR_INVALID_ARG;
   if (k > kMaxK || N > kMaxN || L > kMaxL) return UBT_ERR_UNSUPPORTED;
-  if ((size_t)L * k * k * 5 > kTreeTableBytes) return UBT_ERR_UNSUPPORTED;
   return UBT_OK;
 }
 
@@ -185,6 +184,21 @@ int ubt_build_tree(const float* bigram_scores, int B, int L, int k, int N, const
   cudaError_t e = launch_build_tree(bigram_scores, B, L, k, N, o->search_width, o->depth_bonus, o->alpha, o->lambda,
                                     o->anchor_bigram, o->anchor_tokens, o->pos_offset, *out, no_merge_parts(), 0,
                                     static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? UBT_OK : UBT_ERR_CUDA;
+}
+
+int ubt_selector_scores(const void* phi, const void* psi, int table_dtype, int V, int R, const float* gate,
+                        const int32_t* cand_ids, const int32_t* anchor_tokens, int B, int L, int k,
+                        float* bigram_scores, float* anchor_bigram, void* cuda_stream) {
+  if (B < 0 || L < 1 || V < 1 || k < 1 || R < 1) return UBT_ERR_INVALID_ARG;
+  if (table_dtype != UBT_F32 && table_dtype != UBT_BF16) return UBT_ERR_INVALID_ARG;
+  if (!phi || !psi || !gate || !cand_ids || !aligned16(phi) || !aligned16(psi)) return UBT_ERR_INVALID_ARG;
+  if (L > 1 && !bigram_scores) return UBT_ERR_INVALID_ARG;
+  if ((anchor_bigram != nullptr) != (anchor_tokens != nullptr)) return UBT_ERR_INVALID_ARG;
+  if (R % (table_dtype == UBT_BF16 ? 8 : 4) != 0) return UBT_ERR_INVALID_ARG;
+  if (k > kMaxK || L > kMaxL || R > kMaxSelectorRank) return UBT_ERR_UNSUPPORTED;
+  cudaError_t e = launch_selector_scores(phi, psi, table_dtype, V, R, gate, cand_ids, anchor_tokens, B, L, k,
+                                         bigram_scores, anchor_bigram, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? UBT_OK : UBT_ERR_CUDA;
 }
 

@@ -63,6 +63,12 @@ inline MergeParts merge_parts(const TopkWorkspace& w) {
 }
 inline MergeParts no_merge_parts() { return MergeParts{SpanPlan{0, 0, 0}, nullptr, nullptr, nullptr, nullptr}; }
 
+// ---- selector scores (between a1 and a2)
+constexpr int kMaxSelectorRank = 8192;
+cudaError_t launch_selector_scores(const void* phi, const void* psi, int dtype, int V, int R, const float* gate,
+                                   const int32_t* cand_ids, const int32_t* anchor_tokens, int B, int L, int k,
+                                   float* bigram, float* anchor_bigram, cudaStream_t st);
+
 // ---- a2 + a3 + a3b --------------------------------------------------------------------------
 size_t tree_smem_bytes(int L, int k, int N);
 // `parts` with a non-null part_ms makes the kernel merge the step-a1 partials itself (V is then the row

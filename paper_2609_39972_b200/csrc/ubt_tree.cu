@@ -26,8 +26,14 @@ namespace ubt {
 constexpr int G2_T = 512;
 
 struct TreeSmem {
-  Span<float> t;            // [L,k,k]  pair log-probabilities, each row sorted descending after set-up
-  Span<unsigned char> ord;  // [L,k,k]  ord[row][j] = candidate rank of the j-th best successor
+  // Pair log-probabilities, one row per (position, predecessor rank), each row sorted descending, next to the
+  // permutation that sorted it (ord[row][j] = candidate rank of the j-th best successor).  Whole table [L,k,k]
+  // when it fits; otherwise a cache of the rows the search touches ([N,k]: a pop opens at most one new row),
+  // filled on demand and found through `rowmap`.
+  Span<float> t;
+  Span<unsigned char> ord;
+  Span<short> rowmap;       // lazy mode: [L*k + 1] cache slot of row (position * k + predecessor rank), -1 = not yet
+  Span<float> la;           // [L]    eq. 5 weight of the selector score per position
   Span<float> lp;           // [L,k]
   Span<int> tok;            // [L,k]
   Span<float> al;           // [L]    eq. 5 weight of the base log-probability per position
@@ -45,6 +51,9 @@ struct TreeSmem {
   Span<int> scalars;        // [0] = accepted count
 };
 
+// Rows of the pair table are computed on demand when the whole table would not fit.
+__host__ __device__ inline bool tree_lazy(int L, int k) { return (size_t)L * k * k * 5 > kTreeTableBytes; }
+
 __host__ __device__ inline size_t tree_carve(TreeSmem* s, unsigned char* base, int L, int k, int N) {
   size_t off = 0;
   auto take = [&](size_t bytes) {
@@ -53,8 +62,10 @@ __host__ __device__ inline size_t tree_carve(TreeSmem* s, unsigned char* base, i
     return at;
   };
   const int mw = (N + 31) / 32;
-  const long long lkk = (long long)L * k * k, lk = (long long)L * k;
+  const bool lazy = tree_lazy(L, k);
+  const long long lkk = lazy ? (long long)N * k : (long long)L * k * k, lk = (long long)L * k;
   size_t o_t = take(sizeof(float) * lkk), o_ord = take((size_t)lkk);
+  size_t o_rm = take(lazy ? sizeof(short) * (lk + 1) : 0), o_la = take(sizeof(float) * L);
   size_t o_lp = take(sizeof(float) * lk), o_tok = take(sizeof(int) * lk);
   size_t o_al = take(sizeof(float) * L), o_en = take(sizeof(uint4) * (N + 1));
   size_t o_np = take(sizeof(short) * N), o_nd = take(N), o_nr = take(N);
@@ -65,6 +76,8 @@ __host__ __device__ inline size_t tree_carve(TreeSmem* s, unsigned char* base, i
   if (s) {
     s->t = Span<float>((float*)(base + o_t), lkk, 101);
     s->ord = Span<unsigned char>(base + o_ord, lkk, 102);
+    s->rowmap = Span<short>((short*)(base + o_rm), lazy ? lk + 1 : 0, 107);
+    s->la = Span<float>((float*)(base + o_la), L, 108);
     s->lp = Span<float>((float*)(base + o_lp), lk, 103);
     s->tok = Span<int>((int*)(base + o_tok), lk, 104);
     s->al = Span<float>((float*)(base + o_al), L, 105);
@@ -96,19 +109,81 @@ __device__ __forceinline__ uint32_t pack_lo(int p, int j, int d, int r) {
   return (uint32_t)p | ((uint32_t)j << 8) | ((uint32_t)(d - 1) << 14) | ((uint32_t)r << 20);
 }
 
+// Lazy mode, one warp: eq. 5 and eq. 9 for the row of (position i, predecessor rank ra), sorted by
+// (t desc, token asc), into cache slot `slot`.  k <= 64: a lane holds successors lane and lane + 32.
+struct RowSource {
+  const float* bigram;         // this sequence's [L-1,k,k] selector scores
+  const float* anchor_bigram;  // this sequence's [k] or nullptr
+};
+__device__ __noinline__ void lazy_row(TreeSmem& s, const RowSource& src, int q, int slot, int k, int lane) {
+  const int i = q / k, ra = q - i * k;
+  const float al = s.al[i], la = s.la[i];
+  float v[2];
+  uint32_t key[2];
+  int tok[2];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int rb = lane + 32 * h;
+    v[h] = -INFINITY;
+    tok[h] = 0;
+    if (rb < k) {
+      float d = 0.f;
+      if (i == 0) d = src.anchor_bigram ? src.anchor_bigram[rb] : 0.f;
+      else d = src.bigram[((size_t)(i - 1) * k + ra) * k + rb];
+      v[h] = fmaf(al, s.lp[i * k + rb], la * d);
+      tok[h] = s.tok[i * k + rb];
+    }
+  }
+  float mx = fmaxf(v[0], v[1]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, o));
+  float sum = (lane < k ? expf(v[0] - mx) : 0.f) + (lane + 32 < k ? expf(v[1] - mx) : 0.f);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(FULL, sum, o);
+  const float lse = mx + logf(sum);
+#pragma unroll
+  for (int h = 0; h < 2; ++h) { v[h] -= lse; key[h] = f2key(v[h]); }
+  int rank[2] = {0, 0};
+  for (int j = 0; j < k; ++j) {  // integer keys and a final index tie-break: the ranks are a permutation
+    const uint32_t kj = __shfl_sync(FULL, j < 32 ? key[0] : key[1], j & 31);
+    const int tj = __shfl_sync(FULL, j < 32 ? tok[0] : tok[1], j & 31);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int rb = lane + 32 * h;
+      rank[h] += (kj > key[h]) || (kj == key[h] && (tj < tok[h] || (tj == tok[h] && j < rb)));
+    }
+  }
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int rb = lane + 32 * h;
+    if (rb < k) {
+      s.t[(long long)slot * k + rank[h]] = v[h];
+      s.ord[(long long)slot * k + rank[h]] = (unsigned char)rb;
+    }
+  }
+  __syncwarp();
+}
+
 // Best-first expansion by one warp; returns the number of accepted nodes (all lanes agree).
 // Writes the accepted nodes in pop order: nd_parent, nd_depth, nd_rank, nd_score.
-template <int SLOTS>
-__device__ int expand_tree(TreeSmem& s, int L, int k, int budget, int W, float zeta, int lane) {
+// A record's y word holds the index of its value in the table (15 bits) and the row number q = depth * k + rank
+// of its node's children (13 bits); with the whole table resident that row starts at q * k, in lazy mode at
+// rowmap[q] * k, computed when the node is popped for the first time.
+template <int SLOTS, bool LAZY>
+__device__ int expand_tree(TreeSmem& s, const RowSource& src, int L, int k, int budget, int W, float zeta, int lane) {
   uint32_t fk[SLOTS];
 #pragma unroll
   for (int q = 0; q < SLOTS; ++q) fk[q] = 0u;
-  int f_cnt = 0, n_acc = 0;
+  int f_cnt = 0, n_acc = 0, n_rows = 0;
   if (budget > 0) {
+    if (LAZY) {
+      lazy_row(s, src, 0, 0, k, lane);
+      n_rows = 1;
+    }
     const int r0 = s.ord[0];
     const uint32_t key0 = f2key(s.t[0] + zeta);
     if (lane == 0) fk[0] = key0;
-    s.ent[0] = make_uint4(pack_lo(255, 0, 1, r0), (uint32_t)((k + r0) * k) << 15, __float_as_uint(0.f), key0);
+    s.ent[0] = make_uint4(pack_lo(255, 0, 1, r0), (uint32_t)(k + r0) << 15, __float_as_uint(0.f), key0);
     f_cnt = 1;
   }
   __syncwarp();
@@ -164,7 +239,7 @@ __device__ int expand_tree(TreeSmem& s, int L, int k, int budget, int W, float z
     const uint32_t lo = ent.x, hi = ent.y;
     const float ps = __uint_as_float(ent.z);
     const int p = (int)(lo & 255u), j = (int)((lo >> 8) & 63u), d = (int)((lo >> 14) & 63u) + 1;
-    const int r = (int)((lo >> 20) & 63u), at = (int)(hi & 0x7fffu), cb = (int)((hi >> 15) & 0x7fffu);
+    const int r = (int)((lo >> 20) & 63u), at = (int)(hi & 0x7fffu), qrow = (int)((hi >> 15) & 0x1fffu);
     const float score = key2f(maxk);
     if (W > 0) {
       const int dc = s.depth_cnt[d];
@@ -179,6 +254,17 @@ __device__ int expand_tree(TreeSmem& s, int L, int k, int budget, int W, float z
     }
     // one round of independent loads: next sibling and first child
     const bool has_sib = j + 1 < k, has_child = d < L;
+    int cb = qrow * k;
+    if (LAZY && has_child) {  // the row of this node's children: open it on first use
+      int slot = s.rowmap[qrow];
+      if (slot < 0) {
+        slot = n_rows++;
+        lazy_row(s, src, qrow, slot, k, lane);
+        if (lane == 0) s.rowmap[qrow] = (short)slot;
+        __syncwarp();
+      }
+      cb = slot * k;
+    }
     const int i_sib = has_sib ? at + 1 : 0, i_child = has_child ? cb : 0;
     const float t_sib = s.t[i_sib], t_child = s.t[i_child];
     const int r_sib = s.ord[i_sib], r_child = s.ord[i_child];
@@ -192,11 +278,11 @@ __device__ int expand_tree(TreeSmem& s, int L, int k, int budget, int W, float z
     const uint32_t k_sib = has_sib ? f2key(ps + t_sib + zeta) : 0u;
     const uint32_t k_child = has_child ? f2key(score + t_child + zeta) : 0u;
     const int cl = f_cnt & 31, cs = f_cnt >> 5;
-    s.ent[e_idx] = make_uint4(pack_lo(p, j + 1, d, r_sib), (uint32_t)i_sib | ((uint32_t)((d * k + r_sib) * k) << 15),
+    s.ent[e_idx] = make_uint4(pack_lo(p, j + 1, d, r_sib), (uint32_t)i_sib | ((uint32_t)(d * k + r_sib) << 15),
                               ent.z, k_sib);
     // without a child the record is dead (key 0) and its place is taken by the next one
     s.ent[f_cnt] = make_uint4(pack_lo(n, 0, d + 1, r_child),
-                              (uint32_t)i_child | ((uint32_t)(((d + 1) * k + r_child) * k) << 15),
+                              (uint32_t)i_child | ((uint32_t)((d + 1) * k + r_child) << 15),
                               __float_as_uint(score), k_child);
 #pragma unroll
     for (int q = 0; q < SLOTS; ++q) {
@@ -210,6 +296,7 @@ __device__ int expand_tree(TreeSmem& s, int L, int k, int budget, int W, float z
   return n_acc;
 }
 
+template <bool LAZY>  // LAZY: the rows of the pair table are computed on demand (see TreeSmem)
 __global__ void __launch_bounds__(G2_T)
 k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float zeta,
              const float* __restrict__ alpha, const float* __restrict__ lambda,
@@ -241,7 +328,14 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   // the call, complete before the streaming kernel ahead of this one was launched, so they may be read
   // while that kernel is still running: their DRAM latency hides behind its tail.
   const int nrows = 1 + (L - 1) * k;
-  {
+  constexpr bool lazy = LAZY;
+  for (int i = tid; i < L; i += G2_T) {
+    s.al[i] = alpha ? alpha[i] : 1.f;
+    s.la[i] = lambda ? lambda[i] : 1.f;
+  }
+  if constexpr (lazy) {
+    for (int i = tid; i < L * k + 1; i += G2_T) s.rowmap[i] = (short)-1;
+  } else {
     const int n_big = (L - 1) * kk2;
     constexpr int U = 8;
     for (int i0 = 0; i0 < n_big; i0 += G2_T * U) {
@@ -259,7 +353,6 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
     }
     for (int i = tid; i < kk2; i += G2_T)  // position 0: only predecessor row 0 exists
       s.t[i] = (i < k && anchor_bigram) ? (lambda ? lambda[0] : 1.f) * anchor_bigram[(int64_t)b * k + i] : 0.f;
-    for (int i = tid; i < L; i += G2_T) s.al[i] = alpha ? alpha[i] : 1.f;
   }
   pdl_wait();  // the partials / candidates come from the kernel before this one
 
@@ -279,7 +372,9 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   TT(2);
   int kp = 1;
   while (kp < k) kp <<= 1;
-  if (k <= 32) {
+  if constexpr (lazy) {
+    // rows are normalised and sorted by the expanding warp, one at a time, when the search first needs them
+  } else if (k <= 32) {
     // ---- eq. 5 and eq. 9, then every row sorted by (t desc, token asc): a group of kp = 2^ceil(log2 k)
     // lanes per (position, predecessor) row, the row's values in registers, reductions and exact ranks by
     // shuffles inside the group; integer keys and a final index tie-break keep the ranks a permutation
@@ -387,9 +482,12 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   const bool use_pk = bits * L <= 128;
   if (tid < 32) {
     int n;
-    if (N <= 64) n = expand_tree<2>(s, L, k, budget, W, zeta, lane);
-    else if (N <= 128) n = expand_tree<4>(s, L, k, budget, W, zeta, lane);
-    else n = expand_tree<8>(s, L, k, budget, W, zeta, lane);
+    RowSource src;
+    src.bigram = L > 1 ? bigram + (size_t)b * (L - 1) * kk2 : nullptr;
+    src.anchor_bigram = anchor_bigram ? anchor_bigram + (size_t)b * k : nullptr;
+    if (N <= 64) n = expand_tree<2, LAZY>(s, src, L, k, budget, W, zeta, lane);
+    else if (N <= 128) n = expand_tree<4, LAZY>(s, src, L, k, budget, W, zeta, lane);
+    else n = expand_tree<8, LAZY>(s, src, L, k, budget, W, zeta, lane);
     if (lane == 0) s.scalars[0] = n;
   }
   __syncthreads();
@@ -524,10 +622,11 @@ cudaError_t launch_build_tree(const float* bigram, int B, int L, int k, int N, i
                               const ubt_tree& out, const MergeParts& parts, int V, cudaStream_t st) {
   if (B == 0) return cudaSuccess;
   const size_t smem = tree_smem_bytes(L, k, N);
-  cudaError_t e = cudaFuncSetAttribute(k_build_tree, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  auto kern = tree_lazy(L, k) ? k_build_tree<true> : k_build_tree<false>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   // programmatic launch only when the kernel before it is this library's own streaming kernel
-  return launch_kernel(k_build_tree, dim3(B), dim3(G2_T), smem, st, parts.part_ms != nullptr, bigram, L, k, N, W,
+  return launch_kernel(kern, dim3(B), dim3(G2_T), smem, st, parts.part_ms != nullptr, bigram, L, k, N, W,
                        zeta, alpha, lambda, anchor_bigram, anchor_tokens, pos_offset, out, parts, V);
 }
 

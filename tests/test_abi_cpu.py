@@ -59,7 +59,7 @@ def test_argument_errors_are_returned_before_any_launch():
     assert call(k=65, V=100000) == 2                             # beyond the compiled limit
     assert call(N=257) == 2
     assert call(L=65) == 2
-    assert call(k=64, L=9, V=100000) == 2                        # pair table too large for shared memory
+    assert call(k=64, L=64, V=100000, N=256, tree=_fake_tree(N=256, L=64, k=64)) == 3   # largest shape: accepted
     assert call(dtype=7) == 1
     assert call(tree=_fake_tree(null="mask")) == 1
     assert call(tree=_fake_tree(N=8)) == 1                       # tree shape does not match the call
@@ -71,6 +71,19 @@ def test_argument_errors_are_returned_before_any_launch():
     assert call(ws_bytes=0) == 3                                 # workspace too small
     assert call(ws=None, ws_bytes=1 << 20) == 3
     assert call(B=0, tree=_fake_tree(B=0)) == 0                                        # empty batch: nothing to do
+
+    sel = lambda **kw: lib.ubt_selector_scores(kw.get("phi", p), kw.get("psi", p), kw.get("dtype", 1),
+                                               kw.get("V", 1000), kw.get("R", 256), kw.get("gate", p),
+                                               kw.get("cand", p), kw.get("anchor", None), kw.get("B", 1),
+                                               kw.get("L", 4), kw.get("k", 8), kw.get("big", p),
+                                               kw.get("abig", None), None)
+    assert sel(phi=None) == 1
+    assert sel(R=100) == 1                                       # bf16 rows are whole 16-byte fragments
+    assert sel(anchor=p) == 1                                    # anchor tokens without an output for them
+    assert sel(big=None) == 1
+    assert sel(R=16384) == 2                                     # beyond the supported rank
+    assert sel(k=65) == 2
+    assert sel(B=0) == 0
 
     res = binding._VerifyResult(0x1000, 0x1000, 0x1000, 0x1000)
     vcall = lambda **kw: lib.ubt_verify_tree(C.byref(kw.get("tree", tree)), kw.get("z", p), kw.get("dtype", 1),

@@ -107,11 +107,17 @@ def test_c5_reduced_batch_sampling():
 
 
 def test_paper_search_configuration_k64_w12():
-    # the paper's academic setup (Appendix B): K = 64, W = 12, 64 non-root nodes, 15 future positions;
-    # the pair table must fit shared memory, so L*k*k*5 <= 160 KiB caps L at 8 here
-    cfg = synth.Config("paper", 2, 8, 4096, 64, 65, "bf16", "pos_uniform:0.5,4", 1.0, 0.0, "greedy")
-    run_case(cfg, 0, W=12)
-    run_case(cfg, 1, W=0)
+    # the paper's academic setup (Appendix B): K = 64, W = 12, 64 non-root nodes, 15 future positions.
+    # L = 8 keeps the whole pair table in shared memory, L = 15 goes through the on-demand row cache.
+    for L in (8, 15):
+        cfg = synth.Config("paper", 2, L, 4096, 64, 65, "bf16", "pos_uniform:0.5,4", 1.0, 0.0, "greedy")
+        run_case(cfg, 0, W=12)
+        run_case(cfg, 1, W=0)
+        run_case(cfg, 2, W=12, zeta=-0.125, use_opts=True)
+    # the largest shape of the interface: every limit at its maximum
+    cfg = synth.Config("max", 1, 64, 4096, 64, 256, "bf16", "pos_uniform:0.5,4", 1.0, 0.0, "greedy")
+    run_case(cfg, 3, W=0)
+    run_case(cfg, 4, W=5)
 
 
 @pytest.mark.parametrize("V,k,L,N,dtype", [

@@ -66,6 +66,17 @@ CONFIGS = {
 }
 
 
+# The paper's own search configuration (Appendix B, "Training and Inference Configuration"): K = 64 candidates,
+# search width 12, 64 non-root nodes, 15 future positions, selector rank 256; run through the split entry points
+# with the selector scores computed on the device.  B = 32 concurrent streams, as in the serving experiments.
+SELECTOR_RANK = 256
+PAPER_SEARCH_WIDTH = 12
+NEXT_CONFIGS = {
+    "p1": Config("p1", 32, 15, V_QWEN3, 64, 65, "bf16", "pos_uniform:0.5,8", 1.0, 4.0, "greedy"),
+    "p1-b1": Config("p1-b1", 1, 15, V_QWEN3, 64, 65, "bf16", "pos_uniform:0.5,8", 1.0, 4.0, "greedy"),
+}
+
+
 # --------------------------------------------------------------------------
 # bf16 helpers (bit-level, no arithmetic of the method)
 # --------------------------------------------------------------------------
@@ -306,6 +317,20 @@ def selector_tables(V: int, R: int, B: int, L: int, seed: int, dtype: str = "bf1
     if dtype == "bf16":
         phi, psi = f32_to_bf16_bits(phi), f32_to_bf16_bits(psi)
     return phi, psi, gate
+
+
+def device_selector_tables(V: int, R: int, B: int, L: int, seed: int, device):
+    """Device-resident stand-ins for the selector's tables: ``(phi[V,R] bf16, psi[V,R] bf16, gate[B,L,R] fp32,
+    anchor_tokens[B] i32)``, same distributions as ``selector_tables``, drawn with a seeded torch generator."""
+    import torch
+
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed) * 1_000_003 + 0x5E1)
+    phi = torch.randn((V, R), generator=g, device=device, dtype=torch.float32).to(torch.bfloat16)
+    psi = torch.randn((V, R), generator=g, device=device, dtype=torch.float32).to(torch.bfloat16)
+    gate = torch.randn((B, L, R), generator=g, device=device, dtype=torch.float32) / float(np.sqrt(R))
+    anchor = torch.randint(0, V, (B,), generator=g, device=device, dtype=torch.int32)
+    return phi, psi, gate.contiguous(), anchor
 
 
 def boost_children_on_device(z, token_ids, parents, n_nodes, boost: float) -> None:
