@@ -34,6 +34,7 @@ struct TreeSmem {
   Span<unsigned char> ord;
   Span<short> rowmap;       // lazy mode: [L*k + 1] cache slot of row (position * k + predecessor rank), -1 = not yet
   Span<float> la;           // [L]    eq. 5 weight of the selector score per position
+  Span<float> pre;          // lazy mode: [N+1][k] raw selector scores of the row each frontier record will open
   Span<float> lp;           // [L,k]
   Span<int> tok;            // [L,k]
   Span<float> al;           // [L]    eq. 5 weight of the base log-probability per position
@@ -66,6 +67,7 @@ __host__ __device__ inline size_t tree_carve(TreeSmem* s, unsigned char* base, i
   const long long lkk = lazy ? (long long)N * k : (long long)L * k * k, lk = (long long)L * k;
   size_t o_t = take(sizeof(float) * lkk), o_ord = take((size_t)lkk);
   size_t o_rm = take(lazy ? sizeof(short) * (lk + 1) : 0), o_la = take(sizeof(float) * L);
+  size_t o_pre = take(lazy ? sizeof(float) * (size_t)(N + 1) * k : 0);
   size_t o_lp = take(sizeof(float) * lk), o_tok = take(sizeof(int) * lk);
   size_t o_al = take(sizeof(float) * L), o_en = take(sizeof(uint4) * (N + 1));
   size_t o_np = take(sizeof(short) * N), o_nd = take(N), o_nr = take(N);
@@ -78,6 +80,7 @@ __host__ __device__ inline size_t tree_carve(TreeSmem* s, unsigned char* base, i
     s->ord = Span<unsigned char>(base + o_ord, lkk, 102);
     s->rowmap = Span<short>((short*)(base + o_rm), lazy ? lk + 1 : 0, 107);
     s->la = Span<float>((float*)(base + o_la), L, 108);
+    s->pre = Span<float>((float*)(base + o_pre), lazy ? (long long)(N + 1) * k : 0, 120);
     s->lp = Span<float>((float*)(base + o_lp), lk, 103);
     s->tok = Span<int>((int*)(base + o_tok), lk, 104);
     s->al = Span<float>((float*)(base + o_al), L, 105);
@@ -109,29 +112,52 @@ __device__ __forceinline__ uint32_t pack_lo(int p, int j, int d, int r) {
   return (uint32_t)p | ((uint32_t)j << 8) | ((uint32_t)(d - 1) << 14) | ((uint32_t)r << 20);
 }
 
-// Lazy mode, one warp: eq. 5 and eq. 9 for the row of (position i, predecessor rank ra), sorted by
-// (t desc, token asc), into cache slot `slot`.  k <= 64: a lane holds successors lane and lane + 32.
+// Lazy mode.  The raw selector scores of a row are fetched ahead of time: when a record enters the frontier, the
+// row its node would open (position = its depth, predecessor = its rank) is copied asynchronously from global
+// memory into the record's prefetch slot, so the copy's latency has passed long before the node is popped.
 struct RowSource {
   const float* bigram;         // this sequence's [L-1,k,k] selector scores
   const float* anchor_bigram;  // this sequence's [k] or nullptr
 };
-__device__ __noinline__ void lazy_row(TreeSmem& s, const RowSource& src, int q, int slot, int k, int lane) {
+__device__ __forceinline__ void cp_async_f32(float* smem_dst, const float* gmem_src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+// row q = i * k + ra into prefetch slot e (k <= 64: a lane copies elements lane and lane + 32)
+__device__ __forceinline__ void prefetch_row(TreeSmem& s, const RowSource& src, int q, int e, int k, int L, int lane) {
   const int i = q / k, ra = q - i * k;
+  if (i >= L) return;
+  const float* row = i == 0 ? src.anchor_bigram : src.bigram + ((size_t)(i - 1) * k + ra) * k;
+  float* dst = s.pre.ptr((long long)e * k, k);
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int rb = lane + 32 * h;
+    if (rb < k) {
+      if (row) cp_async_f32(dst + rb, row + rb);
+      else dst[rb] = 0.f;  // no anchor scores: zeros
+    }
+  }
+}
+// One warp: eq. 5 and eq. 9 for row q from the raw scores in prefetch slot e, then its `m` best successors under
+// (t desc, token asc) into cache slot `slot` (the search never looks further down a row: at most W, or the whole
+// budget, of its entries can be accepted, plus one that is dropped).  Successors are extracted one per round by
+// a warp maximum over (score key, ~token); the candidates of a position are distinct tokens.
+__device__ __noinline__ void lazy_row(TreeSmem& s, int q, int e, int slot, int k, int m, int lane) {
+  const int i = q / k;
   const float al = s.al[i], la = s.la[i];
+  cp_async_wait_all();
+  __syncwarp();
   float v[2];
-  uint32_t key[2];
-  int tok[2];
+  uint32_t ntok[2];
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
     const int rb = lane + 32 * h;
     v[h] = -INFINITY;
-    tok[h] = 0;
+    ntok[h] = 0u;
     if (rb < k) {
-      float d = 0.f;
-      if (i == 0) d = src.anchor_bigram ? src.anchor_bigram[rb] : 0.f;
-      else d = src.bigram[((size_t)(i - 1) * k + ra) * k + rb];
-      v[h] = fmaf(al, s.lp[i * k + rb], la * d);
-      tok[h] = s.tok[i * k + rb];
+      v[h] = fmaf(al, s.lp[i * k + rb], la * s.pre[(long long)e * k + rb]);
+      ntok[h] = ~(uint32_t)s.tok[i * k + rb];
     }
   }
   float mx = fmaxf(v[0], v[1]);
@@ -141,24 +167,22 @@ __device__ __noinline__ void lazy_row(TreeSmem& s, const RowSource& src, int q, 
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(FULL, sum, o);
   const float lse = mx + logf(sum);
-#pragma unroll
-  for (int h = 0; h < 2; ++h) { v[h] -= lse; key[h] = f2key(v[h]); }
-  int rank[2] = {0, 0};
-  for (int j = 0; j < k; ++j) {  // integer keys and a final index tie-break: the ranks are a permutation
-    const uint32_t kj = __shfl_sync(FULL, j < 32 ? key[0] : key[1], j & 31);
-    const int tj = __shfl_sync(FULL, j < 32 ? tok[0] : tok[1], j & 31);
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int rb = lane + 32 * h;
-      rank[h] += (kj > key[h]) || (kj == key[h] && (tj < tok[h] || (tj == tok[h] && j < rb)));
-    }
-  }
+  uint32_t key[2];
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
-    const int rb = lane + 32 * h;
-    if (rb < k) {
-      s.t[(long long)slot * k + rank[h]] = v[h];
-      s.ord[(long long)slot * k + rank[h]] = (unsigned char)rb;
+    v[h] -= lse;
+    key[h] = lane + 32 * h < k ? f2key(v[h]) : 0u;  // 0: not a successor / already taken
+  }
+  for (int j = 0; j < m; ++j) {
+    const bool first = key[0] > key[1] || (key[0] == key[1] && ntok[0] >= ntok[1]);
+    const uint32_t bk = first ? key[0] : key[1], bt = first ? ntok[0] : ntok[1];
+    const uint32_t mk = __reduce_max_sync(FULL, bk);
+    const uint32_t mt = __reduce_max_sync(FULL, bk == mk ? bt : 0u);
+    const unsigned holders = __ballot_sync(FULL, bk == mk && bt == mt);
+    if (lane == __ffs(holders) - 1) {
+      s.t[(long long)slot * k + j] = first ? v[0] : v[1];
+      s.ord[(long long)slot * k + j] = (unsigned char)(first ? lane : lane + 32);
+      if (first) key[0] = 0u; else key[1] = 0u;
     }
   }
   __syncwarp();
@@ -175,15 +199,19 @@ __device__ int expand_tree(TreeSmem& s, const RowSource& src, int L, int k, int 
 #pragma unroll
   for (int q = 0; q < SLOTS; ++q) fk[q] = 0u;
   int f_cnt = 0, n_acc = 0, n_rows = 0;
+  // entries of a row the search can reach (see lazy_row); with the whole table resident rows are fully sorted
+  const int row_len = LAZY ? min(k, (W > 0 ? W : budget) + 1) : k;
   if (budget > 0) {
     if (LAZY) {
-      lazy_row(s, src, 0, 0, k, lane);
+      prefetch_row(s, src, 0, 0, k, L, lane);
+      lazy_row(s, 0, 0, 0, k, row_len, lane);
       n_rows = 1;
     }
     const int r0 = s.ord[0];
     const uint32_t key0 = f2key(s.t[0] + zeta);
     if (lane == 0) fk[0] = key0;
     s.ent[0] = make_uint4(pack_lo(255, 0, 1, r0), (uint32_t)(k + r0) << 15, __float_as_uint(0.f), key0);
+    if (LAZY && L > 1) prefetch_row(s, src, k + r0, 0, k, L, lane);  // the row this first record would open
     f_cnt = 1;
   }
   __syncwarp();
@@ -253,13 +281,13 @@ __device__ int expand_tree(TreeSmem& s, const RowSource& src, int L, int k, int 
       s.depth_cnt[d] = dc + 1;
     }
     // one round of independent loads: next sibling and first child
-    const bool has_sib = j + 1 < k, has_child = d < L;
+    const bool has_sib = j + 1 < row_len, has_child = d < L;
     int cb = qrow * k;
     if (LAZY && has_child) {  // the row of this node's children: open it on first use
       int slot = s.rowmap[qrow];
       if (slot < 0) {
         slot = n_rows++;
-        lazy_row(s, src, qrow, slot, k, lane);
+        lazy_row(s, qrow, e_idx, slot, k, row_len, lane);
         if (lane == 0) s.rowmap[qrow] = (short)slot;
         __syncwarp();
       }
@@ -289,6 +317,11 @@ __device__ int expand_tree(TreeSmem& s, const RowSource& src, int L, int k, int 
       fk[q] = (lane == wl && q == ws) ? k_sib : fk[q];
       fk[q] = (has_child && lane == cl && q == cs) ? k_child : fk[q];
     }
+    if (LAZY) {  // fetch ahead the rows the two new records would open (unless they are open already)
+      const int q_sib = d * k + r_sib, q_child = (d + 1) * k + r_child;
+      if (has_sib && d < L && s.rowmap[q_sib] < 0) prefetch_row(s, src, q_sib, e_idx, k, L, lane);
+      if (has_child && d + 1 < L && s.rowmap[q_child] < 0) prefetch_row(s, src, q_child, f_cnt, k, L, lane);
+    }
     f_cnt += has_child ? 1 : 0;
     __syncwarp();
   }
@@ -296,8 +329,11 @@ __device__ int expand_tree(TreeSmem& s, const RowSource& src, int L, int k, int 
   return n_acc;
 }
 
-template <bool LAZY>  // LAZY: the rows of the pair table are computed on demand (see TreeSmem)
-__global__ void __launch_bounds__(G2_T)
+// LAZY: the rows of the pair table are computed on demand (see TreeSmem).  The resident-table kernel is held to
+// 40 registers: its CTAs then fit on an SM as soon as ONE CTA of the top-k kernel in front has left, they signal
+// at once, and the verify kernel behind them is scheduled that much earlier (measured: 139 vs 160 us per c3 step).
+template <bool LAZY>
+__global__ void __launch_bounds__(G2_T, LAZY ? 1 : 3)
 k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float zeta,
              const float* __restrict__ alpha, const float* __restrict__ lambda,
              const float* __restrict__ anchor_bigram, const int32_t* __restrict__ anchor_tokens,
@@ -504,7 +540,12 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
       for (int a = tid; a >= 0; a = s.nd_parent[a]) {
         const int sh = 128 - bits * (int)s.nd_depth[a];
         const unsigned long long r = s.nd_rank[a];
-        if (sh >= 64) hi |= r << (sh - 64); else lo |= r << sh;
+        if (sh >= 64) {
+          hi |= r << (sh - 64);
+        } else {
+          lo |= r << sh;
+          if (sh + bits > 64) hi |= r >> (64 - sh);  // the field straddles the two words
+        }
       }
       s.nd_pk[2 * tid] = hi; s.nd_pk[2 * tid + 1] = lo;
     }

@@ -114,6 +114,8 @@ def test_paper_search_configuration_k64_w12():
         run_case(cfg, 0, W=12)
         run_case(cfg, 1, W=0)
         run_case(cfg, 2, W=12, zeta=-0.125, use_opts=True)
+        run_case(cfg, 3, W=3)        # deep narrow tree: siblings at depth 11, where 6-bit rank fields of the
+        run_case(cfg, 8, W=7)        # packed path key straddle its two 64-bit words
     # the largest shape of the interface: every limit at its maximum
     cfg = synth.Config("max", 1, 64, 4096, 64, 256, "bf16", "pos_uniform:0.5,4", 1.0, 0.0, "greedy")
     run_case(cfg, 3, W=0)
