@@ -76,17 +76,25 @@ __device__ __forceinline__ void merge_row_warp(const MergeParts& p, int64_t rows
         cand_lp[row * k + rank[c]] = val[c] - lse;
       }
   } else {
+    // Many entries (large k, or a row cut into many segments): every segment's list is sorted best first, so an
+    // entry's rank is its place in its own list plus, per other segment, the number of better keys there,
+    // found by binary search.
     for (int q = lane; q < nq; q += 32) {
       const int j = q / k, i = q - j * k;
       if (i >= part_cnt[base + j]) continue;
       const float val = part_val[(base + j) * k + i];
       const int idx = part_idx[(base + j) * k + i];
       const uint64_t key = make_key(val, idx);
-      int rank = 0;
-      for (int j2 = 0; j2 < nseg; ++j2) {
-        const int c2 = part_cnt[base + j2];
-        for (int i2 = 0; i2 < c2; ++i2)
-          rank += make_key(part_val[(base + j2) * k + i2], part_idx[(base + j2) * k + i2]) > key;
+      int rank = i;
+      for (int j2 = 0; j2 < nseg && rank < k; ++j2) {
+        if (j2 == j) continue;
+        int lo = 0, hi = part_cnt[base + j2];  // list[0..lo) > key, list[hi..) < key
+        while (lo < hi) {
+          const int mid = (lo + hi) >> 1;
+          if (make_key(part_val[(base + j2) * k + mid], part_idx[(base + j2) * k + mid]) > key) lo = mid + 1;
+          else hi = mid;
+        }
+        rank += lo;
       }
       if (rank < k) {
         cand_ids[row * k + rank] = idx;
