@@ -140,6 +140,29 @@ def test_edge_shapes(V, k, L, N, dtype):
     run_case(cfg.replace(mode="sample"), 5, targets="agree", seeds_sample=(3,))
 
 
+@pytest.mark.parametrize("block", range(12))
+def test_random_shapes_both_table_modes(block):
+    """Shapes drawn over the whole range of the interface (k <= 64, L <= 64, N <= 256, any W), so that bit
+    fields, table modes (resident / on-demand rows), slot counts and sub-warp group sizes meet in combinations
+    no hand-picked case covers."""
+    rng = np.random.default_rng(1000 + block)
+    for _ in range(7):
+        k = int(rng.choice([1, 2, 3, 5, 8, 13, 16, 24, 32, 33, 47, 64]))
+        L = int(rng.choice([1, 2, 3, 7, 11, 16, 23, 32, 48, 64]))
+        N = int(rng.choice([1, 2, 5, 16, 33, 64, 65, 100, 129, 256]))
+        W = int(rng.choice([0, 0, 1, 2, 5, 12, 40]))
+        V = max(int(rng.choice([64, 264, 999, 1001, 1000, 4096, 40000])), k + 3)   # odd V: plain-load kernels
+        dtype = "bf16" if rng.random() < 0.5 else "f32"
+        zeta = float(rng.choice([0.0, 0.0, -0.05]))
+        cfg = synth.Config("rnd", int(rng.integers(1, 4)), L, V, k, N, dtype, "pos_uniform:0.5,4", 1.0, 0.0,
+                           "greedy" if rng.random() < 0.7 else "sample")
+        try:
+            run_case(cfg, int(rng.integers(0, 1 << 20)), targets="agree" if rng.random() < 0.5 else "plant",
+                     W=W, zeta=zeta, use_opts=bool(rng.random() < 0.5))
+        except AssertionError as e:
+            raise AssertionError(f"shape k={k} L={L} N={N} W={W} V={V} {dtype} zeta={zeta} {cfg.mode}: {e}") from e
+
+
 def test_rows_full_of_ties():
     # bf16 rows quantised to a handful of values, rows with +-0 at the top, a constant row
     u = ubt()
