@@ -4,12 +4,14 @@
 // same number of bytes whatever rows is.  A span meets a few row segments; for each the CTA emits a
 // partial (max, sum exp, sorted top-k) and a small merge kernel combines the partials of a row.
 //
-// Streaming one segment: every thread keeps an online (max, sum) pair and tests the fragment
-// maximum against a CTA-wide exclusive threshold; elements above it are appended (their column
-// only) to a shared pool.  The threshold starts at a bound obtained by bisecting the per-thread
-// maxima of the first tile and becomes exact whenever the pool is ranked ("flush").  The next tile
-// is prefetched into registers before the current one is processed, so the one barrier per tile
-// does not drain the loads in flight.
+// Streaming one segment (k_lse_topk_ring, rows made of whole 16-byte fragments): chunks of the span arrive in a
+// shared-memory ring through bulk asynchronous copies; every thread sums 2^((x - ref) log2 e) relative to a
+// reference of its own that moves up when an element exceeds it by 60, and a group of four fragments per lane is
+// tested against a CTA-wide exclusive threshold by one warp vote; elements above it are appended as 64-bit
+// (value, ~column) keys to a shared pool.  The threshold starts at the k-th largest per-thread maximum of the
+// first chunk (bisection with CTA-wide counts) and becomes exact whenever the pool holds k entries and is
+// ranked ("flush").  k_lse_topk is the plain-load form for other vocabularies (online max per thread, columns
+// in the pool, the next tile prefetched into registers).
 #include "ubt_internal.h"
 #include "ubt_merge.cuh"
 #include "ubt_ring.cuh"

@@ -9,10 +9,12 @@
 // already holds W nodes is outside Top_W(E_d) and is dropped with its later siblings.  N-1 accepted pops
 // give Top_B of the supertree (eq. 11-12).
 //
-// The search is a chain of N-1 dependent pops, so its latency is what counts: the frontier lives in the
-// registers of one warp (entry i in lane i&31, slot i>>5; the score is recovered from its ordering key and
-// everything a pop needs is packed in one word), a pop is a register scan, one warp-wide max, two shuffles
-// and one round of independent shared-memory loads.
+// The search is a chain of N-1 dependent pops by one warp, so its latency is what counts: the ordering keys of
+// the frontier live in registers (entry i in lane i&31, slot i>>5), the 16-byte records in shared memory; a pop
+// is a register scan, three warp reductions, one 16-byte and four scalar shared-memory loads, and stores that all
+// lanes execute alike (see expand_tree).  Everything around it -- merging the top-k partials, eq. 5 / eq. 9 and
+// the row sorts, slot assignment, masks -- is spread over the CTA's 16 warps.  When the pair table does not fit
+// in shared memory its rows are prepared on demand (k_build_tree<true>, see TreeSmem and lazy_row).
 #include "ubt_internal.h"
 #ifdef UBT_TREE_TIMING
 #include <cstdio>

@@ -2,11 +2,16 @@
 //
 // Greedy: B*N*V target logits are cut into equal contiguous spans, one per CTA; each CTA emits, for
 // every row segment it meets, the (value, lowest token) maximum as one 64-bit key.  The walk kernel
-// reduces a row's few keys, so no atomics and no zero-initialised scratch are needed.
-// Sampling: one CTA per row; pass 1 finds the row maximum, pass 2 (served from L2) turns every logit
-// into an integer weight with a fixed sequence of IEEE operations and sums them per 1024-token chunk;
-// the chunk holding the Philox threshold is rescanned to find the token.  Integer sums make the pick
-// independent of the order of addition.
+// reduces a row's few keys, so no atomics and no zero-initialised scratch are needed.  Rows made of whole
+// 16-byte fragments stream through a shared-memory ring fed by bulk asynchronous copies
+// (k_row_argmax_ring); other vocabularies use the plain-load kernel k_row_argmax.
+// Sampling: k_row_weights_ring passes over every row twice through the same kind of ring -- pass 1 finds the
+// row maximum, pass 2 (partly served from L2) turns every logit into an integer weight with a fixed sequence
+// of IEEE operations and sums them per 1024-token block -- and k_row_pick finds the block, then the token,
+// that holds the row's Philox threshold.  Integer sums make the pick independent of the order of addition.
+// k_row_sample is the plain-load form for other vocabularies.
+// The V-wide kernels are launched programmatically: they start while the kernels of a draft call in front of
+// them are still running and wait for them at their very end (see launch_kernel in ubt_internal.h).
 #include "ubt_internal.h"
 #include "ubt_ring.cuh"
 
