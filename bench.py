@@ -29,8 +29,8 @@ import torch
 
 import ubt_synth as synth
 
-NOMINAL_HBM_GBS = 8000.0          # the north-star's "~8 TB/s"
-FALLBACK_HBM_GBS = 6650.0         # earlier measurement on this machine, used only without MEASURED_PEAKS.json
+NOMINAL_HBM_GBS = 8000.0          # nominal HBM3e bandwidth of a B200, the figure the 70 % target is stated against
+FALLBACK_HBM_GBS = 6650.0         # an earlier measured copy bandwidth, used only without MEASURED_PEAKS.json
 
 
 def algorithmic_bytes_per_tree(cfg: synth.Config) -> dict:
@@ -184,13 +184,223 @@ def run_reference(args, cfg, world, rank):
     print(json.dumps(line), flush=True)
 
 
+WORKLOADS_DEFAULT = ("c4", "c3", "c5")     # headline first (the largest single-GPU configuration), then the other two
+
+
+def kernel_record(name, bytes_per_launch, ms, peak, peak_kind, **extra):
+    gbs = bytes_per_launch / (ms * 1e-3) / 1e9 if ms and ms > 0 else None
+    rec = {"kernel": name, "algorithmic_bytes": bytes_per_launch, "avg_ms": ms, "gbs": gbs,
+           "frac": (gbs / peak) if gbs else None, "peak": peak, "peak_source": f"of {peak_kind}"}
+    rec.update(extra)
+    return rec
+
+
+def measure_workload(ubt, args, cfg, paper_flow, world, rank, dev, stream, headline):
+    """All device-timed figures of one workload.  Returns (record, state) where state keeps what the headline's
+    end-to-end and CPU-baseline legs need."""
+    bpt = algorithmic_bytes_per_tree(cfg)
+    batch_bytes = bpt["total"] * cfg.B
+    # enough distinct batches that one rotation exceeds twice the 126 MB L2
+    n_sets = max(2, min(16, -(-4 * 126_000_000 // max(batch_bytes, 1))))
+    sets = [synth.device_inputs(cfg, input_seed(rank, s), dev) for s in range(n_sets)]
+    tree = ubt.Tree.empty(cfg.B, cfg.N, cfg.L, cfg.k, dev)
+    res = ubt.VerifyResult.empty(cfg.B, cfg.L, dev)
+    ws_d = ubt.workspace(ubt.ubt_draft_workspace_bytes(cfg.B, cfg.L, cfg.V, cfg.k, cfg.N), dev)
+    ws_v = ubt.workspace(ubt.ubt_verify_workspace_bytes(cfg.B, cfg.N, cfg.V, cfg.mode), dev)
+    K = args.steps
+    mk = lambda: torch.cuda.Event(enable_timing=True)
+    ev = [[mk() for _ in range(5)] for _ in range(K)]       # step start, between draft kernels, draft end,
+    for row in ev:                                          # verify kernel end, step end
+        for e in row:
+            e.record(stream)
+
+    sel = {}
+    if paper_flow:
+        R, W = synth.SELECTOR_RANK, synth.PAPER_SEARCH_WIDTH
+        phi, psi, gate, anchor = synth.device_selector_tables(cfg.V, R, cfg.B, cfg.L, input_seed(rank, 99), dev)
+        sel = dict(phi=phi, psi=psi, gate=gate, anchor=anchor, W=W,
+                   big=torch.empty((cfg.B, cfg.L - 1, cfg.k, cfg.k), dtype=torch.float32, device=dev),
+                   anc=torch.empty((cfg.B, cfg.k), dtype=torch.float32, device=dev))
+
+    def draft(ud, bd, between=None):
+        if paper_flow:
+            ubt.ubt_topk_logprob(ud, cfg.k, tree.cand_ids, tree.cand_logprob, ws_d, stream=stream)
+            if between is not None:
+                between.record(stream)
+            ubt.ubt_selector_scores(sel["phi"], sel["psi"], sel["gate"], tree.cand_ids, sel["anchor"],
+                                    bigram_scores=sel["big"], anchor_bigram=sel["anc"], stream=stream)
+            ubt.ubt_build_tree(sel["big"], tree, stream=stream, search_width=sel["W"], anchor_bigram=sel["anc"],
+                               anchor_tokens=sel["anchor"])
+        else:
+            ubt.ubt_draft_tree(ud, bd, cfg.k, cfg.N, tree=tree, ws=ws_d, stream=stream, event_between=between)
+
+    def verify(zd, i, early=False, e_after=None):
+        ubt.ubt_verify_tree(tree, zd, cfg.mode, seed=i, temperature=1.0, result=res, ws=ws_v, stream=stream,
+                            event_after=e_after, early_start=early)
+
+    def step(i, early=False):
+        ud, bd, zd = sets[i % n_sets]
+        draft(ud, bd)
+        verify(zd, i, early)
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    barrier(world)
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    time.sleep(0.25)
+    t_wall0 = time.time()
+    # ---- the timed region: K steps in plain stream order (the verify call reads nothing before the draft call in
+    # front of it has completed, as when the target model's forward pass sits between the two)
+    e0, e1 = mk(), mk()
+    e0.record(stream)
+    for i in range(K):
+        step(args.warmup + i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    elapsed_ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
+    # ---- the same K steps with events between the kernels (an event also keeps a kernel from becoming resident
+    # behind the one in front): per-call and per-kernel times
+    for i in range(K):
+        ud, bd, zd = sets[(args.warmup + i) % n_sets]
+        a, b, c, d, e = ev[i]
+        a.record(stream)
+        draft(ud, bd, between=b)
+        c.record(stream)
+        verify(zd, args.warmup + i, e_after=d)
+        e.record(stream)
+    torch.cuda.synchronize()
+    # ---- and chained with the opt-in early start of the verify pass (only possible when the target logits do not
+    # depend on the tree, as in this benchmark; reported as a secondary figure)
+    e2, e3 = mk(), mk()
+    e2.record(stream)
+    for i in range(K):
+        step(args.warmup + i, early=True)
+    e3.record(stream)
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    barrier(world)
+    clocks = sampler.stop(t_wall0, t_wall1)
+    chained_ms = max_over_ranks(e2.elapsed_time(e3), world, dev)
+
+    med = statistics.median
+    t_a1 = med(r[0].elapsed_time(r[1]) for r in ev)
+    t_tree = med(r[1].elapsed_time(r[2]) for r in ev)
+    t_draft = med(r[0].elapsed_time(r[2]) for r in ev)
+    t_vk = med(r[2].elapsed_time(r[3]) for r in ev)
+    t_walk = med(r[3].elapsed_time(r[4]) for r in ev)
+    t_verify = med(r[2].elapsed_time(r[4]) for r in ev)
+
+    peak, peak_kind = measured_peak()
+    e = 2 if cfg.dtype == "bf16" else 4
+    a1_bytes = cfg.B * cfg.L * cfg.V * e
+    vk_bytes = cfg.B * cfg.N * cfg.V * e
+    tree_bytes = cfg.B * (max(cfg.L - 1, 0) * cfg.k * cfg.k * 4 + cfg.L * cfg.k * 8 + cfg.N * (6 + (cfg.N + 31) // 32) * 4 + 4)
+    kernels = [kernel_record("k_lse_topk_ring", a1_bytes, t_a1, peak, peak_kind,
+                             traffic=recorded_traffic("k_lse_topk_ring", cfg.name))]
+    if paper_flow:
+        kernels.append(kernel_record("k_selector_scores+k_build_tree", tree_bytes, t_tree, peak, peak_kind,
+                                     note="latency-bound search; bytes are its inputs and outputs"))
+    else:
+        kernels.append(kernel_record("k_build_tree", tree_bytes, t_tree, peak, peak_kind,
+                                     note="latency-bound search (one CTA per sequence); bytes are its inputs and outputs"))
+    if cfg.mode == "greedy":
+        dominant = kernel_record("k_row_argmax_ring", vk_bytes, t_vk, peak, peak_kind,
+                                 traffic=recorded_traffic("k_row_argmax_ring", cfg.name))
+    else:
+        dominant = kernel_record("k_row_weights_ring+k_row_pick", vk_bytes, t_vk, peak, peak_kind,
+                                 traffic=recorded_traffic("k_row_weights_ring+k_row_pick", cfg.name),
+                                 note="two passes over every row (maximum, then integer weights); reported against "
+                                      "HBM although instruction issue is what limits it")
+    kernels.append(dominant)
+    kernels.append(kernel_record("k_walk", cfg.B * (2 * (cfg.L + 1) + 2) * 4, t_walk, peak, peak_kind,
+                                 note="latency-bound walk of at most L+1 steps"))
+
+    trees_per_s = cfg.B * K * world / (elapsed_ms * 1e-3)
+    step_gbs = batch_bytes * K / (elapsed_ms * 1e-3) / 1e9
+    launches_per_step = 2 + (2 if cfg.mode == "greedy" else 3)   # top-k, tree | argmax or weights+pick, walk
+    if paper_flow:
+        launches_per_step += 2                                   # separate merge kernel, selector scores
+    rec = {
+        "workload": cfg.name, "B": cfg.B, "L": cfg.L, "V": cfg.V, "k": cfg.k, "node_budget": cfg.N,
+        "verify": cfg.mode, "logits": cfg.dtype, "input_sets": n_sets,
+        "ms_per_step": elapsed_ms / K, "trees_per_s": trees_per_s,
+        "bytes_per_tree": bpt["total"], "step_gbs_per_gpu": step_gbs,
+        "frac_of_%s_peak" % peak_kind: step_gbs / peak, "frac_of_nominal_8tbs": step_gbs / NOMINAL_HBM_GBS,
+        "draft_ms": t_draft, "verify_ms": t_verify,
+        "calls_timed_apart_trees_per_s": cfg.B * world / ((t_draft + t_verify) * 1e-3),
+        "chained_early_start": {"ms_per_step": chained_ms / K, "trees_per_s": cfg.B * K * world / (chained_ms * 1e-3),
+                                "note": "verify pass started while the draft call still ran (ubt_verify_opts.early_start);"
+                                        " not reachable when the target logits depend on the tree"},
+        "kernels": kernels, "gpu_launches": launches_per_step * K, "clocks": clocks,
+    }
+    state = dict(sets=sets, tree=tree, res=res, ws_d=ws_d, ws_v=ws_v, draft=draft, sel=sel, dominant=dominant,
+                 launches_per_step=launches_per_step, elapsed_ms=elapsed_ms, bpt=bpt, n_sets=n_sets, clocks=clocks)
+    return rec, state
+
+
+def live_parity(ubt, cfg, paper_flow, st, dev, stream, sample, timed_seconds=0.0):
+    """Oracle on the first `sample` sequences of input set 0 (repeated until `timed_seconds` of CPU time have
+    passed, for the CPU baseline) and an element-by-element comparison with the CUDA path on the same bytes.
+    Returns (parity record, trees done, seconds spent)."""
+    from parity import compare_draft, compare_verify, tree_to_numpy
+    ud, bd, zd = st["sets"][0]
+    sel = st["sel"]
+    uh, bh, zh = (synth.to_host_bits(t[:sample]) for t in (ud, bd, zd))
+    kw = {}
+    if paper_flow:
+        kw = dict(phi=synth.to_host_bits(sel["phi"]), psi=synth.to_host_bits(sel["psi"]),
+                  gate=sel["gate"][:sample].cpu().numpy(), anchor=sel["anchor"][:sample].cpu().numpy(),
+                  W=synth.PAPER_SEARCH_WIDTH)
+    done, spent = 0, 0.0
+    while True:
+        tr, ov, dt = oracle_pass(cfg, uh, bh, zh, 0, **kw)
+        done += sample; spent += dt
+        if spent >= timed_seconds:
+            break
+    st["draft"](ud, bd)
+    pick = torch.empty((cfg.B, cfg.N), dtype=torch.int32, device=dev)
+    ubt.ubt_verify_tree(st["tree"], zd, cfg.mode, seed=0, result=st["res"], ws=st["ws_v"], stream=stream, node_pick=pick)
+    torch.cuda.synchronize()
+    try:
+        g = tree_to_numpy(st["tree"])
+        swaps = compare_draft(g, tr, cfg.L, cfg.k, cfg.N, synth.PAPER_SEARCH_WIDTH if paper_flow else 0, 0.0,
+                              kw.get("anchor"), None, rows=list(range(sample)))
+        if not swaps:
+            compare_verify(st["res"], ov, pick, rows=slice(0, sample))
+        rec = {"checked_trees": sample, "near_tie_swaps": len(swaps), "ok": True}
+    except AssertionError as ex:
+        rec = {"checked_trees": sample, "ok": False, "error": str(ex)[:200]}
+    return rec, done, spent
+
+
+def parity_sample(cfg, paper_flow) -> int:
+    """Sequences the oracle checks live: the whole c3 batch, a bounded sample of the multi-GB workloads."""
+    if paper_flow:
+        return max(1, min(cfg.B, 2))
+    return cfg.B if cfg.B * cfg.N * cfg.V <= 32 * 64 * 151_936 else 8
+
+
+def self_launch(args) -> int:
+    """`python bench.py --gpus N` outside a multi-rank launcher: start the N ranks (one per GPU) ourselves."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c3", choices=sorted(synth.CONFIGS) + sorted(synth.NEXT_CONFIGS))
+    ap.add_argument("--workload", default=None, choices=sorted(synth.CONFIGS) + sorted(synth.NEXT_CONFIGS),
+                    help="one workload only; default: c4 (headline), then c3 and c5 in per_workload")
     ap.add_argument("--ref-trees", type=int, default=4, help="sequences per step of the reference arm")
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time budget of the oracle baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -199,13 +409,19 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    cfg = synth.CONFIGS.get(args.workload) or synth.NEXT_CONFIGS[args.workload]
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(self_launch(args))
+    names = [args.workload] if args.workload else list(WORKLOADS_DEFAULT)
+    cfgs = []
+    for n in names:
+        c = synth.CONFIGS.get(n) or synth.NEXT_CONFIGS[n]
+        if args.batch > 0:
+            c = c.replace(B=args.batch, name=f"{c.name}-B{args.batch}")
+        cfgs.append((c, n in synth.NEXT_CONFIGS))
+    cfg, paper_flow = cfgs[0]
     # the paper's own configuration goes through the split entry points, selector scores computed on the device
-    paper_flow = args.workload in synth.NEXT_CONFIGS
     if paper_flow:
         args.no_e2e = True          # the host-buffer forms cover the fused call only
-    if args.batch > 0:
-        cfg = cfg.replace(B=args.batch, name=f"{cfg.name}-B{args.batch}")
     world, rank, local = dist_setup(args.gpus)
 
     if args.impl == "reference":
@@ -218,147 +434,51 @@ def main():
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     ubt.load()
-
-    # ---- inputs: enough distinct batches that one rotation exceeds twice the 126 MB L2
-    bpt = algorithmic_bytes_per_tree(cfg)
-    batch_bytes = bpt["total"] * cfg.B
-    n_sets = max(2, min(16, -(-4 * 126_000_000 // max(batch_bytes, 1))))
-    sets = []
-    for s in range(n_sets):
-        ud, bd, zd = synth.device_inputs(cfg, input_seed(rank, s), dev)
-        sets.append((ud, bd, zd))
-    tree = ubt.Tree.empty(cfg.B, cfg.N, cfg.L, cfg.k, dev)
-    res = ubt.VerifyResult.empty(cfg.B, cfg.L, dev)
-    ws_d = ubt.workspace(ubt.ubt_draft_workspace_bytes(cfg.B, cfg.L, cfg.V, cfg.k, cfg.N), dev)
-    ws_v = ubt.workspace(ubt.ubt_verify_workspace_bytes(cfg.B, cfg.N, cfg.V, cfg.mode), dev)
     stream = torch.cuda.current_stream()
 
-    ev_pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                for _ in range(args.steps)]
-    for a, b in ev_pairs:           # create the underlying cudaEvent_t handles
-        a.record(stream); b.record(stream)
+    # the other workloads first, so that the headline's buffers are the ones kept for the end-to-end legs
+    per_workload = {}
+    for c, pf in cfgs[1:]:
+        rec, st = measure_workload(ubt, args, c, pf, world, rank, dev, stream, headline=False)
+        if rank == 0 and not args.no_cpu_baseline:
+            rec["parity"], _, _ = live_parity(ubt, c, pf, st, dev, stream, parity_sample(c, pf))
+        per_workload[c.name] = rec
+        del st
+        torch.cuda.empty_cache()
+    head, st = measure_workload(ubt, args, cfg, paper_flow, world, rank, dev, stream, headline=True)
+    per_workload = {cfg.name: head, **per_workload}
+    sets, tree, res, ws_v, draft, sel = st["sets"], st["tree"], st["res"], st["ws_v"], st["draft"], st["sel"]
+    launches_per_step, n_sets = st["launches_per_step"], st["n_sets"]
+    dom = st["dominant"]
+    batch_bytes = st["bpt"]["total"] * cfg.B
 
-    if paper_flow:
-        R, W = synth.SELECTOR_RANK, synth.PAPER_SEARCH_WIDTH
-        phi, psi, gate, anchor = synth.device_selector_tables(cfg.V, R, cfg.B, cfg.L, input_seed(rank, 99), dev)
-        sel_big = torch.empty((cfg.B, cfg.L - 1, cfg.k, cfg.k), dtype=torch.float32, device=dev)
-        sel_anc = torch.empty((cfg.B, cfg.k), dtype=torch.float32, device=dev)
-
-    def draft(ud, bd):
-        if paper_flow:
-            ubt.ubt_topk_logprob(ud, cfg.k, tree.cand_ids, tree.cand_logprob, ws_d, stream=stream)
-            ubt.ubt_selector_scores(phi, psi, gate, tree.cand_ids, anchor, bigram_scores=sel_big,
-                                    anchor_bigram=sel_anc, stream=stream)
-            ubt.ubt_build_tree(sel_big, tree, stream=stream, search_width=W, anchor_bigram=sel_anc,
-                               anchor_tokens=anchor)
-        else:
-            ubt.ubt_draft_tree(ud, bd, cfg.k, cfg.N, tree=tree, ws=ws_d, stream=stream)
-
-    def step(i, events=None):
-        ud, bd, zd = sets[i % n_sets]
-        draft(ud, bd)
-        ubt.ubt_verify_tree(tree, zd, cfg.mode, seed=i, temperature=1.0, result=res, ws=ws_v, stream=stream,
-                            event_before=events[0] if events else None, event_after=events[1] if events else None)
-
-    for i in range(args.warmup):
-        step(i)
-    torch.cuda.synchronize()
-    barrier(world)
-    sampler = ClockSampler(local)
-    sampler.start()
-    time.sleep(0.25)
-    t_wall0 = time.time()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for i in range(args.steps):
-        step(args.warmup + i)
-    e1.record(stream)
-    torch.cuda.synchronize()
-    elapsed_ms = max_over_ranks(e0.elapsed_time(e1), world, dev)
-    # The same K steps again with an event pair around the dominant kernel of every step (the events are
-    # recorded by the library on this stream).  An event between two kernels also forbids the programmatic
-    # overlap of that kernel with the tree builder in front of it, so this pass times the kernel alone and
-    # is kept out of the headline number.
-    e2, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e2.record(stream)
-    for i in range(args.steps):
-        step(args.warmup + i, ev_pairs[i])
-    e3.record(stream)
-    torch.cuda.synchronize()
-    t_wall1 = time.time()
-    barrier(world)
-    clocks = sampler.stop(t_wall0, t_wall1)
-    elapsed_ev_ms = e2.elapsed_time(e3)
-    kern_ms = statistics.mean(a.elapsed_time(b) for a, b in ev_pairs)
-    trees_per_s = cfg.B * args.steps * world / (elapsed_ms * 1e-3)
-
-    # ---- draft / verify split (separate untimed pass, for the record)
-    ea, eb, ec = (torch.cuda.Event(enable_timing=True) for _ in range(3))
-    td, tv = [], []
-    for i in range(min(args.steps, 20)):
-        ud, bd, zd = sets[i % n_sets]
-        ea.record(stream)
-        draft(ud, bd)
-        eb.record(stream)
-        ubt.ubt_verify_tree(tree, zd, cfg.mode, seed=i, result=res, ws=ws_v, stream=stream)
-        ec.record(stream)
-        torch.cuda.synchronize()
-        td.append(ea.elapsed_time(eb)); tv.append(eb.elapsed_time(ec))
-
-    peak, peak_kind = measured_peak()
-    e = 2 if cfg.dtype == "bf16" else 4
-    launches_per_step = 2 + (2 if cfg.mode == "greedy" else 3)   # top-k, tree | argmax or weights+pick, walk
-    if paper_flow:
-        launches_per_step += 2                                   # separate merge kernel, selector scores
-    kern_bytes = cfg.B * cfg.N * cfg.V * e
-    if cfg.mode == "greedy":
-        # HBM-bound: one read of every target logit
-        kern_name = "k_row_argmax_ring"
-        achieved = kern_bytes / (kern_ms * 1e-3) / 1e9
-        roof = {"bound": "hbm", "kernel": kern_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_source": f"of {peak_kind}"}
-    else:
-        # Bound by instruction issue: the integer-exact weight routine is 16 lane operations per element
-        # (scale fma, clamp, 3 adds of the round-to-nearest split, 5 Horner fma, exponent insert (2), convert,
-        # 64-bit add (2), unpack); peak = SMs x 128 lanes x SM clock.
-        kern_name = "k_row_weights_ring+k_row_pick"
-        sms = torch.cuda.get_device_properties(dev).multi_processor_count
-        mhz = (clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965.0)
-        peak_ops = sms * 128 * mhz * 1e6 / 1e12
-        achieved = cfg.B * cfg.N * cfg.V * 16 / (kern_ms * 1e-3) / 1e12
-        roof = {"bound": "alu", "kernel": kern_name, "achieved": achieved, "peak": peak_ops, "unit": "Tlaneop/s",
-                "frac": achieved / peak_ops,
-                "peak_source": "%d SMs x 128 lanes x %.0f MHz (sampled SM clock)" % (sms, mhz),
-                "hbm_gbs": kern_bytes / (kern_ms * 1e-3) / 1e9}
-    roof.update({"traffic": recorded_traffic(kern_name, cfg.name), "bytes_per_launch": kern_bytes,
-                 "avg_launch_ms": kern_ms,
-                 "timed": "second pass of the same %d steps with an event pair around this kernel "
-                          "(%.4f ms/step in that pass)" % (args.steps, elapsed_ev_ms / args.steps)})
-    step_gbs = batch_bytes * args.steps / (elapsed_ms * 1e-3) / 1e9 if world == 1 else \
-        batch_bytes * args.steps * world / (elapsed_ms * 1e-3) / 1e9
-    d_ms, v_ms = statistics.median(td), statistics.median(tv)
-
+    roof = {"bound": "hbm", "kernel": dom["kernel"], "achieved": dom["gbs"], "peak": dom["peak"], "unit": "GB/s",
+            "frac": dom["frac"], "peak_source": dom["peak_source"], "traffic": dom.get("traffic"),
+            "bytes_per_launch": dom["algorithmic_bytes"], "avg_launch_ms": dom["avg_ms"],
+            "timed": "a second pass of the same %d steps with CUDA events recorded by the library around this "
+                     "kernel on the launching stream" % args.steps}
+    if "note" in dom:
+        roof["note"] = dom["note"]
     line = {
-        "metric": "draft+verify trees/sec", "value": trees_per_s, "unit": "trees/s", "n_gpus": world,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": elapsed_ms / args.steps,
+        "metric": "draft+verify trees/sec", "value": head["trees_per_s"], "unit": "trees/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": head["ms_per_step"],
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": cfg.name, "B": cfg.B, "L": cfg.L, "V": cfg.V, "k": cfg.k, "node_budget": cfg.N,
                    "verify": cfg.mode, "logits": cfg.dtype, "input_sets": n_sets,
+                   "order": "plain stream order: draft call, then verify call, nothing overlapped",
                    **({"search_width": synth.PAPER_SEARCH_WIDTH, "selector_rank": synth.SELECTOR_RANK,
                        "flow": "ubt_topk_logprob -> ubt_selector_scores -> ubt_build_tree -> ubt_verify_tree"}
                       if paper_flow else {}),
                    "l2": "inputs larger than L2 (rotation of %d MB)" % (batch_bytes * n_sets // 1_000_000)},
-        "hbm": {"bytes_per_tree": bpt["total"], "step_gbs_per_gpu": step_gbs / world,
-                "frac_of_%s_peak" % peak_kind: step_gbs / world / peak,
-                "frac_of_nominal_8tbs": step_gbs / world / NOMINAL_HBM_GBS,
-                # the two calls timed one at a time (a synchronisation between them, as when the target model
-                # runs between draft and verify): no overlap of the verify kernel with the draft
-                "draft_ms": d_ms, "verify_ms": v_ms, "separate_calls_trees_per_s": cfg.B / ((d_ms + v_ms) * 1e-3),
-                "separate_calls_frac_of_nominal_8tbs": batch_bytes / ((d_ms + v_ms) * 1e-3) / 1e9 / NOMINAL_HBM_GBS},
+        "hbm": {k: head[k] for k in head if k.startswith("frac_of_") or k in
+                ("bytes_per_tree", "step_gbs_per_gpu", "draft_ms", "verify_ms", "calls_timed_apart_trees_per_s",
+                 "chained_early_start")},
         "roofline": roof,
-        "clocks": clocks,
-        "gpu_launches": launches_per_step * args.steps,
+        "kernels": head["kernels"],
+        "per_workload": per_workload,
+        "clocks": st["clocks"],
+        "gpu_launches": head["gpu_launches"],
     }
 
     # ---- end to end through the host-buffer entry points (pinned host inputs, results read back)
@@ -394,37 +514,13 @@ def main():
     # ---- CPU baseline: the oracle as it stands on the host cores, on a bounded sample; doubles as a parity check
     if rank == 0 and not args.no_cpu_baseline:
         import oracle
-        from parity import compare_draft, compare_verify, tree_to_numpy
-        ud, bd, zd = sets[0]
-        sample = max(1, min(cfg.B, 8))
-        uh, bh, zh = (synth.to_host_bits(t[:sample]) for t in (ud, bd, zd))
-        done, spent, tr = 0, 0.0, None
-        kw = {}
-        if paper_flow:
-            sample = max(1, min(cfg.B, 2))
-            uh, zh = (synth.to_host_bits(t[:sample]) for t in (ud, zd))
-            kw = dict(phi=synth.to_host_bits(phi), psi=synth.to_host_bits(psi), gate=gate[:sample].cpu().numpy(),
-                      anchor=anchor[:sample].cpu().numpy(), W=synth.PAPER_SEARCH_WIDTH)
-        while spent < args.cpu_seconds:
-            tr, ov, dt = oracle_pass(cfg, uh, bh, zh, 0, **kw)
-            done += sample; spent += dt
+        sample = parity_sample(cfg, paper_flow)
+        par, done, spent = live_parity(ubt, cfg, paper_flow, st, dev, stream, sample, args.cpu_seconds)
         line["cpu_baseline"] = {"value": done / spent, "unit": "trees/s", "cores": oracle.num_threads(),
                                 "kind": "oracle", "sample": f"first {sample} of {cfg.B} sequences, repeated for "
                                                             f"{spent:.1f} s ({done} trees)"}
-        # live parity of the bench configuration on that sample
-        draft(ud, bd)
-        pick = torch.empty((cfg.B, cfg.N), dtype=torch.int32, device=dev)
-        ubt.ubt_verify_tree(tree, zd, cfg.mode, seed=0, result=res, ws=ws_v, stream=stream, node_pick=pick)
-        torch.cuda.synchronize()
-        try:
-            g = tree_to_numpy(tree)
-            swaps = compare_draft(g, tr, cfg.L, cfg.k, cfg.N, synth.PAPER_SEARCH_WIDTH if paper_flow else 0, 0.0,
-                                  kw.get("anchor"), None, rows=list(range(sample)))
-            if not swaps:
-                compare_verify(res, ov, pick, rows=slice(0, sample))
-            line["parity"] = {"checked_trees": sample, "near_tie_swaps": len(swaps), "ok": True}
-        except AssertionError as ex:
-            line["parity"] = {"checked_trees": sample, "ok": False, "error": str(ex)[:200]}
+        line["parity"] = par
+        per_workload[cfg.name]["parity"] = par
 
     if rank == 0:
         print(json.dumps(line), flush=True)

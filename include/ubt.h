@@ -11,7 +11,10 @@
  * Conventions that hold for every entry point unless it says otherwise
  *   - Pointers named in a struct or argument list are DEVICE pointers owned by the caller; the
  *     library never allocates, frees or synchronises.  All work is enqueued on `cuda_stream`
- *     (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *     (a cudaStream_t passed as void*; NULL = the legacy default stream) and keeps stream order: no
+ *     input is read, and no output or workspace written, before the work in front of the call on
+ *     that stream has completed, and work enqueued behind the call sees all of its results.  The one
+ *     exception is opt-in (ubt_verify_opts.early_start).
  *   - Tensors are dense, row-major, in the shapes given; base pointers must be 16-byte aligned.
  *   - Inputs are read-only.  Outputs and the workspace are overwritten; workspace content on entry
  *     is irrelevant.
@@ -80,6 +83,9 @@ typedef struct ubt_draft_opts {
   const float *anchor_bigram;   /* [B,k] selector score of the anchor -> depth-1 transition; NULL = 0 */
   const int32_t *anchor_tokens; /* [B] token stored in the root slot; NULL = -1 */
   const int32_t *pos_offset;    /* [B] position id of the root; NULL = 0 */
+  void *event_between;          /* optional cudaEvent_t recorded on the stream between the V-wide kernel of step
+                                   a1 and the tree kernel (ubt_draft_tree only; for timing the two apart -- an
+                                   event between them also keeps the second from becoming resident early) */
 } ubt_draft_opts;
 
 typedef struct ubt_verify_opts {
@@ -88,6 +94,16 @@ typedef struct ubt_verify_opts {
   int32_t *node_pick;  /* optional [B,N]: the target's pick at EVERY row, visited or not */
   void *event_before;  /* optional cudaEvent_t recorded on the stream just before the V-wide */
   void *event_after;   /* per-node kernel and just after it (for timing that kernel alone)    */
+  int32_t early_start; /* 0 (default): plain stream order -- nothing is read or written before the work in
+                          front of the call on `cuda_stream` has completed.  1: the caller vouches that
+                          target_logits were complete, and the workspace and node_pick unused, BEFORE the
+                          preceding ubt_draft_tree call on this stream was enqueued; the V-wide pass over
+                          target_logits may then run while that draft call is still executing (it still
+                          finishes after it, and the walk reads the finished tree).  Ignored -- the call falls
+                          back to stream order -- when the stream's last draft call is not on record (the
+                          library remembers the last one of 16 streams) or one of its buffers overlaps the
+                          workspace or node_pick.  In the method's real order the target logits are computed
+                          FROM the drafted tree (Appendix A), so leave this 0 there. */
 } ubt_verify_opts;
 
 typedef struct ubt_verify_result {
@@ -210,14 +226,17 @@ int ubt_verify_tree_host(const ubt_tree *tree, const void *target_logits, int dt
  * Same arguments, outputs and results as ubt_verify_tree(tree, target_logits, dtype, V, GREEDY, ...);
  * node_pick ([B,N] device, may be NULL) receives the pick of every row.
  * Limit: B*N*spans_per_row <= ubt_verify_static_capacity() keys (65,536), where spans_per_row =
- * ceil(V/span)+1 and span = max(65,536, B*N*V / (2 * SM count)) elements: 2 for large batches (32,768
- * keys for B*N = 16,384 rows), 4 for a single 64-slot tree over V = 151,936.  A larger request returns
- * UBT_ERR_STATIC_SCRATCH before anything is launched.
+ * ceil(V/span)+1 and span = max(32,768, ceil(B*N*V / SM count)) elements rounded up to a multiple of 256:
+ * 2 for large batches (32,768 keys for B*N = 16,384 rows), 4 for a single 64-slot tree over V = 151,936
+ * on 148 SMs.  A larger request returns UBT_ERR_STATIC_SCRATCH before anything is launched.
  * The first call on a device looks up the array's device address (once per device, with that device
  * current); make that first call outside any stream capture.
  * All calls on a device share the one array and it keeps the previous call's contents (every key that is
- * read is written first, so nothing needs clearing): two calls whose kernels overlap on the GPU -- different
- * streams, or different host threads -- race on it and must be serialised by the caller.
+ * read is written first, so nothing needs clearing).  Calls enqueued one after the other on the SAME stream
+ * are safe: the call keeps plain stream order, so its first kernel starts only after the walk of the call in
+ * front has finished with the array.  Two calls whose kernels can overlap on the GPU -- different streams, or
+ * different host threads enqueueing without an order between them -- race on it and must be serialised by
+ * the caller.
  */
 int ubt_verify_tree_static(const ubt_tree *tree, const void *target_logits, int dtype, int V,
                            int32_t *node_pick, ubt_verify_result *out, void *cuda_stream);

@@ -150,11 +150,11 @@ typedef struct {
   int slot;      /* output slot once selected, else -1 */
 } onode;
 
-/* Total order Omega, "better first".  The paper fixes only "preferring
- * ancestors when scores tie" (Appendix A, Global Pruning); an ancestor is
- * always shallower, hence rule 2.  Rules 3-5 are this build's reading that
- * makes the order total: lower token id, lower candidate rank, then the
- * rank path in lexicographic order. */
+/* Total order Omega, "better first".  For equal scores the paper fixes only
+ * that an ancestor goes before its descendants (Appendix A, Global Pruning);
+ * an ancestor is always shallower, hence rule 2.  Rules 3-5 are this build's
+ * reading that makes the order total: lower token id, lower candidate rank,
+ * then the rank path in lexicographic order. */
 static int omega_cmp(const void *pa, const void *pb) {
   const onode *a = (const onode *)pa, *b = (const onode *)pb;
   if (a->score > b->score) return -1;
@@ -180,8 +180,8 @@ static double rel_gap(double kept, double dropped) {
  *   anchor_bigram[b,k]  delta_1(x_t, .) for the anchor -> depth-1 transition, NULL = 0
  *   anchor_tokens[b]    token id stored in the root slot, NULL = -1
  *   pos_offset[b]       position id of the root, NULL = 0
- *   N                   tree slots including the root (paper's budget B = N - 1:
- *                       "the root ... does not count toward B")
+ *   N                   tree slots including the root (the paper's budget B leaves
+ *                       the root out, so its B = N - 1; Appendix A, Global Pruning)
  *   W                   search width; 0 = unbounded.  An unbounded or large width
  *                       is run as W_eff = N - 1: every depth of the exact global
  *                       Top-(N-1) holds at most N - 1 nodes and is contained in
@@ -254,7 +254,7 @@ int ubt_oracle_build_tree(const int32_t *cand_ids, const double *cand_lp, const 
     }
     if (t_out) memcpy(t_out + (int64_t)b * L * k * k, t, sizeof(double) * (size_t)L * k * k);
 
-    /* Algorithm 1: F_0 = {root}, ell(root) = 0, S = {} */
+    /* depth-wise expansion (eq. 11): the retained set of depth 0 is the root alone, with score 0 */
     int nS = 0;         /* nodes in S */
     int f_lo = -1, f_hi = -1; /* F_{d-1} = S[f_lo..f_hi); (-1,-1) = {root} */
     for (int d = 1; d <= L && Weff > 0; ++d) {
@@ -270,7 +270,7 @@ int ubt_oracle_build_tree(const int32_t *cand_ids, const double *cand_lp, const 
           e->path = Epaths + (size_t)nE * L;
           if (p >= 0) memcpy(e->path, S[p].path, sizeof(int) * (size_t)(d - 1));
           e->path[d - 1] = r;
-          /* ell_zeta(y_1:d) = ell_zeta(y_1:d-1) + log q^bi_d(y_d | y_d-1) + zeta */
+          /* eq. 9-10: a child adds its pair log-probability and the depth bonus to its parent's score */
           e->score = pscore + t[((size_t)(d - 1) * k + prank) * k + r] + zeta;
           e->depth = d;
           e->rank = r;
@@ -405,8 +405,9 @@ void ubt_oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint
 }
 
 /*
- * Sampling weights (T_infer > 0).  The paper says only that verification
- * follows "the target-model sample"; this build's reading pins the sampler so
+ * Sampling weights (T_infer > 0).  The paper says only that the walk follows
+ * what the target model samples at each node (Appendix A, verification); this
+ * build's reading pins the sampler so
  * that a pick is a pure function of (row, temperature, seed, b, n):
  *
  *   m  = max_v z[v]                          (fp32, exact)
@@ -496,9 +497,9 @@ static int32_t sample_pick(const void *z, int dtype, int64_t row, int V, float t
 /*
  * The walk.  From the root, take the target's pick x at the current node; if a
  * child of the current node carries token x, move to it and count it accepted;
- * otherwise x is the bonus token and the walk ends ("follows the child matching
- * the target-model sample at each step until the first mismatch; the first
- * unmatched sample is retained as the bonus token").  Siblings carry distinct
+ * otherwise x is the bonus token and the walk ends (Appendix A, verification:
+ * the walk stops at the first pick that no child carries and keeps that pick as
+ * the bonus token).  Siblings carry distinct
  * tokens, so the child is unique.  accepted_len counts draft tokens only; the
  * paper's tau (Section 2) is accepted_len + 1.
  *

@@ -20,6 +20,7 @@ const DeviceInfo& device_info() {
     if (cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess || smem <= 0)
       smem = 227 * 1024;
     cudaGetLastError();
+    info[dev].device = dev;
     info[dev].sm_count = sms;
     info[dev].max_smem_optin = smem;
     known[dev] = true;
@@ -51,12 +52,13 @@ static int check_tree(const ubt_tree* t, bool need_cands) {
 
 // ---- which memory a draft call on a stream may still be using when the next call starts
 //
-// The tree kernel lets the kernel behind it on the stream start at once (programmatic dependent launch), so the
-// V-wide pass of a verify call streams while the draft call's kernels are still running.  That is only sound
-// if nothing the early kernel WRITES overlaps anything the draft call reads or writes; plain stream order
-// would allow such reuse (say, the draft logits' buffer as the verify workspace).  Every draft call therefore
-// records its buffers per stream, and a verify call whose written buffers touch them launches its first
-// kernel without the attribute, i.e. strictly after the draft.
+// A verify call keeps plain stream order unless the caller sets ubt_verify_opts.early_start; then its V-wide
+// pass streams while the draft call in front of it on the stream is still running.  Beyond what the caller
+// vouches for (the target logits were complete before that draft call was enqueued), this is only sound if
+// nothing the early kernel WRITES overlaps anything the draft call reads or writes; plain stream order would
+// allow such reuse (say, the draft logits' buffer as the verify workspace).  Every draft call therefore records
+// its buffers per stream, and an early start is granted only against a recorded draft call that the written
+// buffers stay clear of.
 struct ByteRange {
   const char* lo;
   const char* hi;
@@ -103,18 +105,20 @@ static void remember_draft(cudaStream_t st, const void* logits, size_t logits_by
   g_drafts[g_draft_next++ % 16] = d;
 }
 
-// May a kernel that writes [p, p + bytes) start while the last draft call on `st` is still running?
+// May a kernel that writes [p, p + bytes) start while the last draft call on `st` is still running?  Only if
+// that call is on record (the table holds the last draft of 16 streams; a stream that was pushed out of it, or
+// never drafted, gets the answer "no") and none of its buffers overlaps the range.
 static bool clear_of_last_draft(cudaStream_t st, const void* p, size_t bytes) {
-  if (!p || !bytes) return true;
   const char* lo = static_cast<const char*>(p);
-  const char* hi = lo + bytes;
+  const char* hi = lo + (p ? bytes : 0);
   std::lock_guard<std::mutex> lock(g_draft_mu);
   for (const DraftRecord& e : g_drafts) {
     if (!e.valid || e.stream != st) continue;
     for (int i = 0; i < e.n; ++i)
       if (lo < e.r[i].hi && e.r[i].lo < hi) return false;
+    return true;
   }
-  return true;
+  return false;
 }
 
 }  // namespace ubt
@@ -123,7 +127,7 @@ using namespace ubt;
 
 extern "C" {
 
-int ubt_version(void) { return 100; }
+int ubt_version(void) { return 110; }
 
 const char* ubt_status_string(int status) {
   switch (status) {
@@ -235,6 +239,8 @@ int ubt_draft_tree(const void* unigram_logits, int dtype, const float* bigram_sc
   const ubt_draft_opts* o = opts ? opts : &d;
   remember_draft(st, unigram_logits, (size_t)rows * V * esize(dtype), bigram_scores, B, L, k, N, o, *out, workspace,
                  topk_workspace_bytes(rows, V, k));
+  if (o->event_between && cudaEventRecord(static_cast<cudaEvent_t>(o->event_between), st) != cudaSuccess)
+    return UBT_ERR_CUDA;
   cudaError_t e = launch_build_tree(bigram_scores, B, L, k, N, o->search_width, o->depth_bonus, o->alpha, o->lambda,
                                     o->anchor_bigram, o->anchor_tokens, o->pos_offset, *out, merge_parts(w), V, st);
   return e == cudaSuccess ? UBT_OK : UBT_ERR_CUDA;
@@ -252,7 +258,7 @@ int ubt_verify_tree(const ubt_tree* tree, const void* target_logits, int dtype, 
   const int B = tree->B, N = tree->N, L = tree->L;
   if (B < 0 || N < 1 || L < 1) return UBT_ERR_INVALID_ARG;
   if (N > kMaxN || L > kMaxL) return UBT_ERR_UNSUPPORTED;
-  const ubt_verify_opts d{0, 1.0f, nullptr, nullptr, nullptr};
+  const ubt_verify_opts d{0, 1.0f, nullptr, nullptr, nullptr, 0};
   const ubt_verify_opts* o = opts ? opts : &d;
   if (mode == UBT_VERIFY_SAMPLE) {
     if (!(o->temperature > 0.0f)) return UBT_ERR_INVALID_ARG;
@@ -267,16 +273,16 @@ int ubt_verify_tree(const ubt_tree* tree, const void* target_logits, int dtype, 
   const int32_t* sampled = nullptr;
   if (o->event_before && cudaEventRecord(static_cast<cudaEvent_t>(o->event_before), st) != cudaSuccess)
     return UBT_ERR_CUDA;
-  // the V-wide kernels may start while a draft call in front of them on this stream is still running, unless
-  // what they write touches that call's buffers
-  bool early = clear_of_last_draft(st, workspace, verify_workspace_bytes(rows, V, mode));
+  // stream order by default; on request the V-wide kernels start while the draft call in front of them on this
+  // stream is still running, unless what they write touches that call's buffers
+  bool early = o->early_start != 0 && clear_of_last_draft(st, workspace, verify_workspace_bytes(rows, V, mode));
   if (mode == UBT_VERIFY_GREEDY) {
     if (launch_row_argmax(target_logits, dtype, rows, V, w, tree_smem_bytes(tree->L, tree->k, tree->N), early, st) !=
         cudaSuccess)
       return UBT_ERR_CUDA;
   } else {
     int32_t* pick = o->node_pick ? o->node_pick : w.pick;
-    early = early && clear_of_last_draft(st, o->node_pick, (size_t)rows * 4);
+    early = early && (!o->node_pick || clear_of_last_draft(st, o->node_pick, (size_t)rows * 4));
     if (launch_row_sample(target_logits, dtype, B, N, V, o->seed, o->temperature, pick, w, early, st) != cudaSuccess)
       return UBT_ERR_CUDA;
     sampled = pick;
@@ -391,6 +397,7 @@ int ubt_draft_tree_host(const void* unigram_logits, int dtype, const float* bigr
     if (opts->anchor_bigram) { UBT_CUDA_OK(cudaMemcpyAsync(d.anchor_bigram, opts->anchor_bigram, sizeof(float) * (size_t)B * k, cudaMemcpyHostToDevice, st)); dev_opts.anchor_bigram = d.anchor_bigram; }
     if (opts->anchor_tokens) { UBT_CUDA_OK(cudaMemcpyAsync(d.anchor_tokens, opts->anchor_tokens, sizeof(int32_t) * B, cudaMemcpyHostToDevice, st)); dev_opts.anchor_tokens = d.anchor_tokens; }
     if (opts->pos_offset) { UBT_CUDA_OK(cudaMemcpyAsync(d.pos_offset, opts->pos_offset, sizeof(int32_t) * B, cudaMemcpyHostToDevice, st)); dev_opts.pos_offset = d.pos_offset; }
+    dev_opts.event_between = opts->event_between;
   }
   rc = ubt_draft_tree(d.logits, dtype, L > 1 ? d.bigram : nullptr, B, L, V, k, N, &dev_opts, &d.tree.t, d.ws,
                       d.ws_bytes, cuda_stream);
@@ -430,8 +437,9 @@ int ubt_verify_tree_host(const ubt_tree* tree, const void* target_logits, int dt
   UBT_CUDA_OK(cudaMemcpyAsync(d.tree.t.token_ids, tree->token_ids, bn * 4, cudaMemcpyHostToDevice, st));
   UBT_CUDA_OK(cudaMemcpyAsync(d.tree.t.parents, tree->parents, bn * 4, cudaMemcpyHostToDevice, st));
   UBT_CUDA_OK(cudaMemcpyAsync(d.tree.t.n_nodes, tree->n_nodes, (size_t)B * 4, cudaMemcpyHostToDevice, st));
-  ubt_verify_opts dev_opts{0, 1.0f, nullptr, nullptr, nullptr};
+  ubt_verify_opts dev_opts{0, 1.0f, nullptr, nullptr, nullptr, 0};
   if (opts) { dev_opts = *opts; }
+  dev_opts.early_start = 0;  // the logits are copied in just before: nothing to start ahead of
   int32_t* host_pick = dev_opts.node_pick;
   dev_opts.node_pick = host_pick ? d.node_pick : nullptr;
   ubt_verify_result r{d.accepted_len, d.bonus, d.accepted_nodes, d.out_tokens};

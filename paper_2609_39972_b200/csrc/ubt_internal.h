@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <atomic>
 #include <stddef.h>
 #include <stdint.h>
 
@@ -34,11 +35,25 @@ inline cudaError_t launch_kernel(void (*kern)(KArgs...), dim3 grid, dim3 block, 
 }
 
 struct DeviceInfo {
+  int device;
   int sm_count;
   int max_smem_optin;
 };
 // Properties of the current device (queried once per device, cached).
 const DeviceInfo& device_info();
+
+// Lets kernel `Kern` use up to the device's opt-in maximum of dynamic shared memory.  The attribute belongs to
+// the (function, device) pair, so it is set once per device and per kernel instantiation, with that device current.
+template <auto Kern>
+inline cudaError_t allow_max_dynamic_smem() {
+  static std::atomic<bool> done[64];
+  const DeviceInfo& di = device_info();
+  const int dev = di.device;
+  if (done[dev].load(std::memory_order_acquire)) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(Kern, cudaFuncAttributeMaxDynamicSharedMemorySize, di.max_smem_optin);
+  if (e == cudaSuccess) done[dev].store(true, std::memory_order_release);
+  return e;
+}
 
 // Cut rows*V elements into equal contiguous spans, one per CTA.
 SpanPlan make_span_plan(int64_t rows, int V, int ctas, int64_t min_span);

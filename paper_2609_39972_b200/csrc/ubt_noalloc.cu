@@ -59,7 +59,10 @@ extern "C" int ubt_verify_tree_static(const ubt_tree* tree, const void* target_l
   if (static_row_keys(&keys) != cudaSuccess) { cudaGetLastError(); return UBT_ERR_CUDA; }
   w.part_key = keys;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  if (launch_row_argmax(target_logits, dtype, rows, V, w, tree_smem_bytes(tree->L, tree->k, tree->N), true, st) != cudaSuccess) return UBT_ERR_CUDA;
+  // plain stream order (no early start): the one shared array may still be read by the walk of a call in front
+  if (launch_row_argmax(target_logits, dtype, rows, V, w, tree_smem_bytes(tree->L, tree->k, tree->N), false, st) !=
+      cudaSuccess)
+    return UBT_ERR_CUDA;
   if (launch_walk(*tree, UBT_VERIFY_GREEDY, w, V, nullptr, node_pick, *out, st) != cudaSuccess) return UBT_ERR_CUDA;
   return UBT_OK;
 }

@@ -4,8 +4,7 @@
 // An elected thread keeps STAGES-1 chunks in flight; every chunk lands in one stage and completes an
 // mbarrier that all threads wait on; the CTA barrier that ends a chunk's processing frees its stage.  The
 // copies keep flowing while the CTA is busy, so the bytes in flight per SM do not depend on how the consumer
-// code is scheduled.  On this B200 the ring sustains 6.9 TB/s on a 622 MB read against 6.7 TB/s for the best
-// register-staged loop.
+// code is scheduled.
 //
 // Every wait is bounded: after kRingSpinLimit failed polls a thread gives up and raises a device-side flag
 // (ubt_debug_ring_timeouts); the CTA barrier that ends the chunk carries that vote, so all threads leave the

@@ -130,13 +130,13 @@ cudaError_t launch_selector_scores(const void* phi, const void* psi, int dtype, 
   const size_t smem = (size_t)2 * GS_K * GS_LD * sizeof(float);
   if (dtype == UBT_BF16) {
     auto kern = k_selector_scores<__nv_bfloat16>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = allow_max_dynamic_smem<k_selector_scores<__nv_bfloat16>>();
     if (e != cudaSuccess) return e;
     kern<<<B * L, GS_T, smem, st>>>(static_cast<const __nv_bfloat16*>(phi), static_cast<const __nv_bfloat16*>(psi), V,
                                     R, gate, cand_ids, anchor_tokens, L, k, bigram, anchor_bigram);
   } else {
     auto kern = k_selector_scores<float>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = allow_max_dynamic_smem<k_selector_scores<float>>();
     if (e != cudaSuccess) return e;
     kern<<<B * L, GS_T, smem, st>>>(static_cast<const float*>(phi), static_cast<const float*>(psi), V, R, gate,
                                     cand_ids, anchor_tokens, L, k, bigram, anchor_bigram);

@@ -15,12 +15,6 @@
 #include "ubt_internal.h"
 #include "ubt_merge.cuh"
 #include "ubt_ring.cuh"
-#ifdef UBT_G1_TIMING
-#include <cstdio>
-#define GT(i) do { long long now_ = clock64(); tt[i] += now_ - tlast; tlast = now_; } while (0)
-#else
-#define GT(i) do {} while (0)
-#endif
 
 namespace ubt {
 
@@ -373,10 +367,6 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
     prod.init(lo, hi, V);
     for (int i = 0; i < G1R_STAGES - 1; ++i) prod.issue_one(logits, ring, full);
   }
-#ifdef UBT_G1_TIMING
-  long long tt[8] = {0, 0, 0, 0, 0, 0, 0, 0}, tlast = clock64();
-  int nflush = 0;
-#endif
   RingPos<G1R_STAGES> rp;
   rp.init();
   int consumed = 0;
@@ -395,11 +385,8 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
     for (int c = 0; c < sg.len; c += STAGE_ELEMS) {
       const int l = sg.len - c < STAGE_ELEMS ? sg.len - c : STAGE_ELEMS;
       if (*reinterpret_cast<volatile int*>(&sh.fail)) { failed = true; break; }
-      GT(0);
       if (tid == 0) prod.issue_one(logits, ring, full);
-      GT(1);
       const bool ok = mbar_wait(&full[rp.stage], rp.parity);
-      GT(2);
       if (!ok) sh.fail = 1;
       const uint4* stage = reinterpret_cast<const uint4*>(ring + (size_t)rp.stage * G1R_STAGE_BYTES) + tid;
       const int nfrag = ok ? l / VEC : 0;
@@ -437,8 +424,6 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
         if (r0 > -1.0e29f && r0 < 1.0e30f) { ref = r0; negref = -r0 * kLog2e; }
         __syncthreads();
       }
-
-      GT(3);
       const float taux = sh.taux;
       int f0 = 0;
       for (; f0 + G1R_GROUP * G1R_T <= nfrag; f0 += G1R_GROUP * G1R_T) {  // full groups: no bounds checks
@@ -508,15 +493,9 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
           acc[0] = add2(acc[0], pack2(ex2_approx(y0), ex2_approx(y1)));
         }
       }
-
-      GT(4);
       // One barrier takes the decision on the final hit count (see the comment in k_lse_topk): rank the pool
       // now?  Inside the branch nobody is ahead in the next chunk, so the counter can be read plainly.
       if (__syncthreads_or(*reinterpret_cast<volatile int*>(&sh.cnt) >= k)) {
-        GT(5);
-#ifdef UBT_G1_TIMING
-        ++nflush;
-#endif
         const bool overflow = sh.cnt > G1R_POOL;
         flush_keyed(sh, k);  // ranks what the pool holds; tightens the threshold
         if (overflow) {
@@ -556,7 +535,6 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
           }
         }
       }
-      GT(6);
       rp.next();
       ++consumed;
     }
@@ -597,15 +575,9 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
     }
     __syncthreads();
     pos += sg.len;
-    GT(7);
   }
   __syncthreads();
   if (tid == 0 && *reinterpret_cast<volatile int*>(&sh.fail)) prod.drain(consumed > 0 ? consumed - 1 : 0, full);
-#ifdef UBT_G1_TIMING
-  if (tid == 32 && (blockIdx.x == 0 || blockIdx.x == 100 || blockIdx.x == 300))
-    printf("g1 cta %d chunks %d flushes %d cycles: top %lld issue %lld wait %lld bisect %lld process %lld vote %lld flush %lld segend %lld\n", blockIdx.x,
-           consumed, nflush, tt[0], tt[1], tt[2], tt[3], tt[4], tt[5], tt[6], tt[7]);
-#endif
 }
 
 // One warp per row: combine the partials of the row's segments (see merge_row_warp in ubt_merge.cuh).
@@ -661,7 +633,7 @@ static cudaError_t launch_lse_topk_t(const void* logits, int64_t rows, int V, in
                                      const TopkWorkspace& w, cudaStream_t st) {
   const size_t smem = sizeof(G1Shared) + sizeof(int) * (size_t)(G1_T * G1_U * VEC + G1_SLACK);
   auto kern = k_lse_topk<T, VEC>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = allow_max_dynamic_smem<k_lse_topk<T, VEC>>();
   if (e != cudaSuccess) return e;
   kern<<<w.plan.grid, G1_T, smem, st>>>(static_cast<const T*>(logits), rows * (int64_t)V, V, k, w.plan,
                                         w.part_ms, w.part_val, w.part_idx, w.part_cnt);
@@ -673,12 +645,8 @@ static cudaError_t launch_lse_topk_ring_t(const void* logits, int64_t rows, int 
                                           cudaStream_t st) {
   const size_t smem = (size_t)G1R_STAGES * G1R_STAGE_BYTES + sizeof(G1RShared);
   auto kern = k_lse_topk_ring<T>;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  cudaError_t e = allow_max_dynamic_smem<k_lse_topk_ring<T>>();
+  if (e != cudaSuccess) return e;
   return launch_kernel(kern, dim3(w.plan.grid), dim3(G1R_T), smem, st, true, static_cast<const T*>(logits),
                        rows * (int64_t)V, V, k, w.plan, w.part_ms, w.part_val, w.part_idx, w.part_cnt);
 }

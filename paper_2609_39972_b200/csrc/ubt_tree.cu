@@ -16,12 +16,6 @@
 // the row sorts, slot assignment, masks -- is spread over the CTA's 16 warps.  When the pair table does not fit
 // in shared memory its rows are prepared on demand (k_build_tree<true>, see TreeSmem and lazy_row).
 #include "ubt_internal.h"
-#ifdef UBT_TREE_TIMING
-#include <cstdio>
-#define TT(i) do { if (b == 0 && tid == 0) tt[i] = clock64(); } while (0)
-#else
-#define TT(i) do {} while (0)
-#endif
 
 namespace ubt {
 
@@ -332,8 +326,7 @@ __device__ int expand_tree(TreeSmem& s, const RowSource& src, int L, int k, int 
 }
 
 // LAZY: the rows of the pair table are computed on demand (see TreeSmem).  The resident-table kernel is held to
-// 40 registers: its CTAs then fit on an SM as soon as ONE CTA of the top-k kernel in front has left, they signal
-// at once, and the verify kernel behind them is scheduled that much earlier (measured: 139 vs 160 us per c3 step).
+// 40 registers so that its CTAs fit on an SM as soon as ONE CTA of the top-k kernel in front has left.
 template <bool LAZY>
 __global__ void __launch_bounds__(G2_T, LAZY ? 1 : 3)
 k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float zeta,
@@ -352,10 +345,6 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   const Span<int32_t> g_rk(out.cand_rank, nB * N, 214), g_pos(out.position_ids, nB * N, 215), g_nn(out.n_nodes, nB, 216);
   const Span<float> g_sc(out.scores, nB * N, 217);
   const Span<uint32_t> g_mask(out.mask, nB * N * mw, 218);
-#ifdef UBT_TREE_TIMING
-  long long tt[10];
-#endif
-  TT(0);
   // The next kernel in the stream may start right away.  When that is the V-wide pass of ubt_verify_tree it
   // reads target logits only and streams while this kernel (and the tail of the top-k kernel in front of it)
   // is still running; it waits for this grid before it exits, so stream order still holds for whatever follows.
@@ -400,14 +389,11 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
       merge_row_warp(parts, nB * L, (int64_t)b * L + i, V, k, out.cand_ids, out.cand_logprob, lane);
     __syncthreads();  // the candidates were written by this CTA; the barrier orders them before the reads below
   }
-
-  TT(1);
   // ---- stage candidates and raw selector scores
   for (int i = tid; i < L * k; i += G2_T) {
     s.lp[i] = g_lp[(int64_t)b * L * k + i];
     s.tok[i] = g_ids[(int64_t)b * L * k + i];
   }
-  TT(2);
   int kp = 1;
   while (kp < k) kp <<= 1;
   if constexpr (lazy) {
@@ -507,13 +493,10 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
       __syncthreads();
     }
   }
-  TT(3);
   __syncthreads();
   for (int i = tid; i < L + 2; i += G2_T) s.depth_cnt[i] = 0;
   for (int i = tid; i < N * mw; i += G2_T) s.maskrow[i] = 0u;
   __syncthreads();
-
-  TT(4);
   // ---- best-first expansion (warp 0)
   int bits = 1;
   while ((1 << bits) < k) ++bits;
@@ -529,8 +512,6 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
     if (lane == 0) s.scalars[0] = n;
   }
   __syncthreads();
-
-  TT(5);
   // ---- canonical slots: root 0, then depth by depth ordered by (parent slot, rank)
   const int n_acc = s.scalars[0];
   for (int i = tid; i < L + 2; i += G2_T) s.depth_cnt[i] = 0;
@@ -594,8 +575,6 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
       __syncthreads();
     }
   }
-
-  TT(6);
   // ---- outputs
   const int64_t o = (int64_t)b * N;
   const int poff = pos_offset ? pos_offset[b] : 0;
@@ -624,12 +603,6 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   }
   __syncthreads();
   for (int i = tid; i < N * mw; i += G2_T) g_mask[(int64_t)b * N * mw + i] = s.maskrow[i];
-  TT(7);
-#ifdef UBT_TREE_TIMING
-  if (b == 0 && tid == 0)
-    printf("tree cycles: merge %lld stage %lld rows %lld sort %lld expand %lld slots %lld out %lld total %lld\n", tt[1] - tt[0],
-           tt[2] - tt[1], tt[3] - tt[2], tt[4] - tt[3], tt[5] - tt[4], tt[6] - tt[5], tt[7] - tt[6], tt[7] - tt[0]);
-#endif
 }
 
 // Step a3b alone: one CTA per sequence, one thread per slot.
@@ -665,8 +638,9 @@ cudaError_t launch_build_tree(const float* bigram, int B, int L, int k, int N, i
                               const ubt_tree& out, const MergeParts& parts, int V, cudaStream_t st) {
   if (B == 0) return cudaSuccess;
   const size_t smem = tree_smem_bytes(L, k, N);
-  auto kern = tree_lazy(L, k) ? k_build_tree<true> : k_build_tree<false>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const bool lazy = tree_lazy(L, k);
+  auto kern = lazy ? k_build_tree<true> : k_build_tree<false>;
+  cudaError_t e = lazy ? allow_max_dynamic_smem<k_build_tree<true>>() : allow_max_dynamic_smem<k_build_tree<false>>();
   if (e != cudaSuccess) return e;
   // programmatic launch only when the kernel before it is this library's own streaming kernel
   return launch_kernel(kern, dim3(B), dim3(G2_T), smem, st, parts.part_ms != nullptr, bigram, L, k, N, W,

@@ -10,8 +10,9 @@
 // of IEEE operations and sums them per 1024-token block -- and k_row_pick finds the block, then the token,
 // that holds the row's Philox threshold.  Integer sums make the pick independent of the order of addition.
 // k_row_sample is the plain-load form for other vocabularies.
-// The V-wide kernels are launched programmatically: they start while the kernels of a draft call in front of
-// them are still running and wait for them at their very end (see launch_kernel in ubt_internal.h).
+// The V-wide kernels are launched programmatically, so their CTAs become resident behind the kernel in front of
+// them; by default they wait there for that kernel to complete before they read anything (stream order).  Only
+// when the caller opts in (ubt_verify_opts.early_start) do they stream at once and wait at their very end.
 #include "ubt_internal.h"
 #include "ubt_ring.cuh"
 
@@ -136,7 +137,7 @@ __device__ __forceinline__ float frag_max(const uint4& v, const float*) {
 template <typename T, int STAGES, int STAGE_BYTES, int THREADS, int CTAS>
 __global__ void __launch_bounds__(THREADS, CTAS)
 k_row_argmax_ring(const T* __restrict__ logits, int64_t total, int V, SpanPlan plan,
-                  unsigned long long* __restrict__ part_key_) {
+                  unsigned long long* __restrict__ part_key_, int early) {
   extern __shared__ __align__(128) unsigned char ring[];
   __shared__ uint64_t full[STAGES];
   __shared__ unsigned long long red[THREADS / 32];
@@ -150,8 +151,15 @@ k_row_argmax_ring(const T* __restrict__ logits, int64_t total, int V, SpanPlan p
   const int64_t lo = (int64_t)blockIdx.x * plan.span;
   const int64_t hi = lo + plan.span < total ? lo + plan.span : total;
   const Span<unsigned long long> part_key(part_key_, (total / V) * plan.smax, 401);
+  // Stream order is the default: nothing is read or written before the kernel in front on the stream has
+  // completed.  With `early` (the caller vouches that the target logits were complete, and the scratch unused,
+  // before that kernel's call was enqueued) the span is streamed at once and the wait moves to the very end.
+  if (!early) pdl_wait();
   pdl_launch_dependents();  // the walk kernel may be scheduled; it waits for this grid before reading
-  if (lo >= hi) return;
+  if (lo >= hi) {
+    if (early && tid == 0) pdl_wait();
+    return;
+  }
 
   if (tid == 0) {
     for (int s = 0; s < STAGES; ++s) mbar_init(&full[s], 1);
@@ -244,10 +252,9 @@ k_row_argmax_ring(const T* __restrict__ logits, int64_t total, int V, SpanPlan p
   }
   __syncthreads();
   if (tid == 0 && *reinterpret_cast<volatile int*>(&s_fail)) prod.drain(consumed > 0 ? consumed - 1 : 0, full);
-  // This kernel reads only the target logits, so it may have started before the kernel in front of it (the
-  // tree builder) finished; it must not complete before that kernel does, or the walk behind it could run
-  // on an unfinished tree.
-  if (tid == 0) pdl_wait();
+  // An early start must not become an early finish: the walk behind this kernel waits for THIS grid only, so
+  // this grid may not complete before the kernel in front of it (the tree builder) has.
+  if (early && tid == 0) pdl_wait();
 }
 
 // ---------------------------------------------------------------------------- sampling picks
@@ -427,7 +434,7 @@ struct RowTwiceProducer {  // thread 0: chunks of row r (pass 0), the same chunk
 template <typename T>
 __global__ void __launch_bounds__(G5R_T, G5R_CTAS)
 k_row_weights_ring(const T* __restrict__ logits, int64_t rows, int V, float temperature,
-                   float* __restrict__ row_ac, unsigned long long* __restrict__ block_sum, int nblocks) {
+                   float* __restrict__ row_ac, unsigned long long* __restrict__ block_sum, int nblocks, int early) {
   extern __shared__ __align__(128) unsigned char ring[];
   __shared__ uint64_t full[G5R_STAGES];
   __shared__ float redf[G5R_T / 32];
@@ -437,8 +444,12 @@ k_row_weights_ring(const T* __restrict__ logits, int64_t rows, int V, float temp
   constexpr int BF = G5_CHUNK / VEC;  // fragments per 1024-token block
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t r0 = rows * blockIdx.x / gridDim.x, r1 = rows * (blockIdx.x + 1) / gridDim.x;
+  if (!early) pdl_wait();  // stream order unless the caller opted into an early start (see k_row_argmax_ring)
   pdl_launch_dependents();
-  if (r0 >= r1) return;
+  if (r0 >= r1) {
+    if (early && tid == 0) pdl_wait();
+    return;
+  }
   if (tid == 0) {
     for (int s = 0; s < G5R_STAGES; ++s) mbar_init(&full[s], 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -531,7 +542,7 @@ k_row_weights_ring(const T* __restrict__ logits, int64_t rows, int V, float temp
   }
   __syncthreads();
   if (tid == 0 && *reinterpret_cast<volatile int*>(&s_fail)) prod.drain(consumed > 0 ? consumed - 1 : 0, full);
-  if (tid == 0) pdl_wait();  // started early, like the greedy kernel: do not complete before the tree builder
+  if (early && tid == 0) pdl_wait();  // started early: do not complete before the kernel in front
 }
 
 // One warp per row: block sums -> pick.
@@ -626,7 +637,6 @@ k_walk(ubt_tree tree, int mode, SpanPlan plan, const unsigned long long* __restr
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, N = tree.N, L = tree.L;
   const int64_t o = (int64_t)b * N;
   pdl_wait();  // picks and tree come from the kernels before this one
-  pdl_launch_dependents();  // a kernel behind this one may become resident; it has to wait for this grid itself
   for (int n = tid; n < N; n += blockDim.x) {
     int p;
     if (mode == UBT_VERIFY_GREEDY) {
@@ -648,6 +658,9 @@ k_walk(ubt_tree tree, int mode, SpanPlan plan, const unsigned long long* __restr
     if (node_pick) node_pick[o + n] = p;
   }
   __syncthreads();
+  // Only now may a kernel behind this one become resident: the scratch (row keys / picks) has been read for the
+  // last time, so an early-started pass of a following verify call cannot overwrite anything still needed here.
+  pdl_launch_dependents();
   if (tid >= 32) return;
   const int n_nodes = tree.n_nodes[b];
   int32_t* an = out.accepted_nodes + (int64_t)b * (L + 1);
@@ -716,11 +729,10 @@ static cudaError_t launch_row_argmax_t(const void* logits, int64_t rows, int V, 
   return cudaGetLastError();
 }
 
-// Ring configuration of the greedy kernel: three stages, 256 threads, one CTA per SM.  Measured on B200
-// (622 MB of bf16 rows) with 64 KiB stages: 94.7 us; 6 x 32 KiB: 105 us; 12 x 16 KiB: 179 us (per-chunk latency
-// dominates).  The kernel is launched programmatically behind the tree kernel, so its CTAs should fit on an
-// SM beside one CTA of that kernel: when the tree's tables leave no room for 3 x 64 KiB the stages shrink to
-// 48 KiB (same speed on 5 GB of rows, 2 % slower on 0.6 GB), which lets the whole tree build hide behind it.
+// Ring configuration of the greedy kernel: three stages, 256 threads, one CTA per SM.  Few large stages beat
+// many small ones because every chunk pays a fixed latency.  The kernel is launched programmatically, so its
+// CTAs should fit on an SM beside one CTA of the tree kernel that may still be resident in front of it: when
+// the tree's tables leave no room for 3 x 64 KiB the stages shrink to 48 KiB.
 constexpr int kArgmaxStages = 3, kArgmaxThreads = 256;
 constexpr int kSmemPerSm = 228 * 1024, kSmemPerCtaReserved = 1024;
 
@@ -729,14 +741,12 @@ static cudaError_t launch_row_argmax_ring_t(const void* logits, int64_t rows, in
                                             bool early, cudaStream_t st) {
   auto kern = k_row_argmax_ring<T, kArgmaxStages, STAGE_BYTES, kArgmaxThreads, 1>;
   constexpr int kBytes = kArgmaxStages * STAGE_BYTES;
-  static bool configured = false;  // the attribute sticks to the function; set it once
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBytes);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
-  return launch_kernel(kern, dim3(w.plan.grid), dim3(kArgmaxThreads), kBytes, st, early, static_cast<const T*>(logits),
-                       rows * (int64_t)V, V, w.plan, w.part_key);
+  cudaError_t e = allow_max_dynamic_smem<k_row_argmax_ring<T, kArgmaxStages, STAGE_BYTES, kArgmaxThreads, 1>>();
+  if (e != cudaSuccess) return e;
+  // Always launched programmatically: the CTAs become resident behind the kernel in front.  Without `early`
+  // they wait there until that kernel has completed before they read anything (plain stream order).
+  return launch_kernel(kern, dim3(w.plan.grid), dim3(kArgmaxThreads), kBytes, st, true, static_cast<const T*>(logits),
+                       rows * (int64_t)V, V, w.plan, w.part_key, early ? 1 : 0);
 }
 
 template <typename T>
@@ -777,16 +787,12 @@ static cudaError_t launch_row_sample_ring_t(const void* logits, int64_t rows, in
                                             bool early, cudaStream_t st) {
   auto kern = k_row_weights_ring<T>;
   constexpr int kBytes = G5R_STAGES * G5R_STAGE_BYTES;
-  static bool configured = false;
-  if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBytes);
-    if (e != cudaSuccess) return e;
-    configured = true;
-  }
+  cudaError_t e = allow_max_dynamic_smem<k_row_weights_ring<T>>();
+  if (e != cudaSuccess) return e;
   int grid = device_info().sm_count * G5R_CTAS;
   if ((int64_t)grid > rows) grid = (int)rows;
-  cudaError_t e = launch_kernel(kern, dim3(grid), dim3(G5R_T), kBytes, st, early, static_cast<const T*>(logits), rows, V,
-                                temperature, w.row_ac, w.block_sum, w.nblocks);
+  e = launch_kernel(kern, dim3(grid), dim3(G5R_T), kBytes, st, true, static_cast<const T*>(logits), rows, V,
+                    temperature, w.row_ac, w.block_sum, w.nblocks, early ? 1 : 0);
   if (e != cudaSuccess) return e;
   const int warps = 4;
   return launch_kernel(k_row_pick<T>, dim3((unsigned)((rows + warps - 1) / warps)), dim3(warps * 32), 0, st, true,

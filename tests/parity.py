@@ -7,7 +7,7 @@ import numpy as np
 
 from helpers import check_tree_invariants, layout_from_paths, paths_of_tree
 
-SCORE_TOL = 1e-5   # |gpu - oracle| <= SCORE_TOL * max(1, |oracle|): the north-star's fp32 tolerance
+SCORE_TOL = 1e-5   # |gpu - oracle| <= SCORE_TOL * max(1, |oracle|): fp32 path scores against the fp64 oracle
 
 
 def tree_to_numpy(tree) -> SimpleNamespace:

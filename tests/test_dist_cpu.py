@@ -70,6 +70,25 @@ def test_reference_arm_under_a_two_rank_launch_prints_one_line():
     assert line["config"]["workload"] == "c1"
 
 
+@pytest.mark.timeout(300)
+def test_bare_command_with_gpus_2_starts_two_ranks_itself():
+    """`python bench.py --gpus 2` outside any launcher must spawn the two ranks and report n_gpus = 2."""
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2", "--steps", "1",
+           "--warmup", "3", "--workload", "c1"]
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_PORT")}
+    env["CUDA_VISIBLE_DEVICES"] = ""
+    p = subprocess.run(cmd, capture_output=True, text=True, cwd=ROOT, env=env, timeout=280)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [json.loads(l) for l in p.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1 and lines[0]["n_gpus"] == 2 and lines[0]["impl"] == "reference"
+
+
+def test_default_invocation_measures_the_largest_configuration_first():
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.WORKLOADS_DEFAULT[0] == "c4" and set(bench.WORKLOADS_DEFAULT) == {"c3", "c4", "c5"}
+
+
 def test_ranks_draw_different_batches():
     """Weak scaling: rank r's input set s is seeded 1000 r + s, so no two ranks stream the same bytes."""
     sys.path.insert(0, ROOT)

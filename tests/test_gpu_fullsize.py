@@ -1,7 +1,8 @@
-"""Full-size configurations in the launch configuration the benchmark times; the oracle checks a sample.
+"""Full-size configurations in the launch configuration the benchmark times, every sequence checked.
 
-Inputs of 0.8-5.6 GB are drawn on the device (seeded torch generator); the sequences the oracle checks
-are copied back bit for bit, so both sides read the same bytes.
+Inputs of 0.8-5.6 GB are drawn on the device (seeded torch generator) and copied back bit for bit, so both sides
+read the same bytes.  The oracle drafts every sequence and walks every tree (evaluating only the target rows a
+walk visits); the picks at every slot are compared on eight sequences.
 """
 import numpy as np
 import pytest
@@ -15,28 +16,36 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
-def _run_full(name, sample, seeds=(0,)):
+def _run_full(name, pick_rows, seeds=(0,)):
+    """Every sequence of the full batch: the draft against the oracle, and the walk against the oracle's own lazy
+    walk (which evaluates only the rows it visits).  ``pick_rows``: sequences whose picks at EVERY slot are
+    compared as well."""
     import paper_2609_39972_b200 as u
     cfg = synth.CONFIGS[name]
     ud, bd, zd = synth.device_inputs(cfg, 11, DEV)
     gtree = u.ubt_draft_tree(ud, bd, cfg.k, cfg.N)
     torch.cuda.synchronize()
     g = tree_to_numpy(gtree)
-    rows = sorted(sample)
-    uh = synth.to_host_bits(ud[rows]); bh = synth.to_host_bits(bd[rows]); zh = synth.to_host_bits(zd[rows])
-    otree = oracle.draft_tree(uh, bh, cfg.k, cfg.N)
-    swaps = compare_draft(g, otree, cfg.L, cfg.k, cfg.N, rows=rows)
-    print(f"{name}: near-tie swaps on the sampled sequences: {swaps}")
+    otree = oracle.draft_tree(synth.to_host_bits(ud), synth.to_host_bits(bd), cfg.k, cfg.N)
+    del ud, bd
+    swaps = compare_draft(g, otree, cfg.L, cfg.k, cfg.N)
+    print(f"{name}: near-tie swaps over the whole batch: {swaps}")
+    zh = synth.to_host_bits(zd)
     pick = torch.empty((cfg.B, cfg.N), dtype=torch.int32, device=DEV)
-    sub = lambda a: a[rows]
+    rows = sorted(pick_rows)
+    zr = zh[rows]
     for s in seeds:
         res = u.ubt_verify_tree(gtree, zd, cfg.mode, seed=s, node_pick=pick)
         torch.cuda.synchronize()
+        # the oracle numbers sequences by their place in the arrays it is given: the whole batch keeps b true
+        ov = oracle.verify(g.token_ids, g.parents, g.n_nodes, cfg.L, zh, cfg.mode, seed=s, all_nodes=False)
+        compare_verify(res, ov)
         if cfg.mode == "greedy":
-            ov = oracle.verify(sub(g.token_ids), sub(g.parents), sub(g.n_nodes), cfg.L, zh, "greedy")
-        else:   # the Philox counter holds the true batch index b
-            ov = _oracle_sample_rows(g, zh, rows, cfg, s)
-        compare_verify(res, ov, pick, rows=rows)
+            sub = lambda a: a[rows]
+            ov8 = oracle.verify(sub(g.token_ids), sub(g.parents), sub(g.n_nodes), cfg.L, zr, "greedy")
+        else:
+            ov8 = _oracle_sample_rows(g, zr, rows, cfg, s)
+        compare_verify(res, ov8, pick, rows=rows)
     # properties that hold at any size, on the whole batch
     n = g.n_nodes
     assert np.all(n >= 1) and np.all(n <= cfg.N)
@@ -88,15 +97,15 @@ def _oracle_sample_rows(g, zh, rows, cfg, seed):
 
 
 def test_c3_full_batch():
-    _run_full("c3", sample=range(32))          # every sequence
+    _run_full("c3", pick_rows=range(32))
 
 
-def test_c4_full_batch_sampled():
-    _run_full("c4", sample=[0, 17, 63])
+def test_c4_full_batch():
+    _run_full("c4", pick_rows=[0, 9, 17, 26, 35, 44, 53, 63])
 
 
-def test_c5_full_batch_sampled():
-    _run_full("c5", sample=[0, 64, 127], seeds=(0, 12345))
+def test_c5_full_batch():
+    _run_full("c5", pick_rows=[0, 18, 36, 54, 72, 90, 108, 127], seeds=(0, 12345))
     _CDF_CACHE.clear()
 
 
@@ -111,11 +120,13 @@ def _same_result(a, b):
         assert torch.equal(getattr(a, name), getattr(b, name)), name
 
 
+@pytest.mark.parametrize("early", [False, True])
 @pytest.mark.parametrize("name", ["c3", "c5"])
-def test_back_to_back_calls_equal_separated_calls(name):
-    """Draft and verify enqueued with nothing between them run overlapped on the device (the verify call's
-    V-wide kernel starts while the draft's kernels are still running); the outcome must be bit-identical to the
-    same calls separated by a synchronisation, which the tests above check against the oracle."""
+def test_back_to_back_calls_equal_separated_calls(name, early):
+    """Draft and verify enqueued with nothing between them; with ``early_start`` they run overlapped on the device
+    (the verify call's V-wide kernel starts while the draft's kernels are still running).  Either way the outcome
+    must be bit-identical to the same calls separated by a synchronisation, which the tests above check against
+    the oracle."""
     import paper_2609_39972_b200 as u
     cfg = synth.CONFIGS[name].replace(B=32)
     ud, bd, zd = synth.device_inputs(cfg, 5, DEV)
@@ -125,7 +136,7 @@ def test_back_to_back_calls_equal_separated_calls(name):
     torch.cuda.synchronize()
     for _ in range(3):
         t = u.ubt_draft_tree(ud, bd, cfg.k, cfg.N)
-        r = u.ubt_verify_tree(t, zd, cfg.mode, seed=3)
+        r = u.ubt_verify_tree(t, zd, cfg.mode, seed=3, early_start=early)
         torch.cuda.synchronize()
         _same_tree(t, t_ref)
         _same_result(r, r_ref)
@@ -133,7 +144,7 @@ def test_back_to_back_calls_equal_separated_calls(name):
 
 def test_verify_scratch_that_reuses_a_draft_buffer_is_not_started_early():
     """Stream order allows a caller to hand the draft call's logits buffer to the verify call as scratch.  The
-    library must then keep the verify kernel behind the draft instead of overlapping them."""
+    library must then keep the verify kernel behind the draft even when an early start was asked for."""
     import paper_2609_39972_b200 as u
     cfg = synth.CONFIGS["c3"]
     ud, bd, zd = synth.device_inputs(cfg, 6, DEV)
@@ -147,7 +158,7 @@ def test_verify_scratch_that_reuses_a_draft_buffer_is_not_started_early():
         ws = scratch.view(torch.uint8).reshape(-1)
         assert ws.numel() >= need
         t = u.ubt_draft_tree(scratch, bd, cfg.k, cfg.N)
-        r = u.ubt_verify_tree(t, zd, "greedy", ws=ws)        # overwrites the draft's logits
+        r = u.ubt_verify_tree(t, zd, "greedy", ws=ws, early_start=True)        # overwrites the draft's logits
         torch.cuda.synchronize()
         _same_tree(t, t_ref)
         _same_result(r, r_ref)

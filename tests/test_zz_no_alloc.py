@@ -3,7 +3,8 @@
 It exists for callers that cannot allocate device memory where they verify (a fully handed-out memory pool, a
 plugin that only receives its buffers, a loop that must avoid cudaMalloc's implicit synchronisation).  Its
 scratch is a fixed array inside libubt.so that every call reuses, so the test calls it twice in a row on
-different inputs and compares each result, through the C ABI, with ubt_verify_tree on the same inputs.
+different inputs and compares each result, through the C ABI, with ubt_verify_tree on the same inputs and with
+the CPU oracle's walk of the same tree.
 Collected last on purpose: a run that stops at the first failure has then already run every other test.
 """
 import ctypes as C
@@ -11,7 +12,9 @@ import ctypes as C
 import pytest
 import torch
 
+import oracle
 import ubt_synth as synth
+from parity import compare_verify, tree_to_numpy
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -44,6 +47,9 @@ def test_static_scratch_entry_point_matches_workspace_entry_point_twice_in_a_row
         torch.cuda.synchronize()
         _same(got, want)
         assert torch.equal(got_pick, want_pick)
+        g = tree_to_numpy(tree)
+        compare_verify(got, oracle.verify(g.token_ids, g.parents, g.n_nodes, cfg.L, synth.to_host_bits(zd), "greedy"),
+                       got_pick)
         assert int(got.accepted_len.max()) >= 1
         results.append(got.out_tokens.clone())
     assert not torch.equal(results[0], results[1])          # the two calls really saw different inputs
