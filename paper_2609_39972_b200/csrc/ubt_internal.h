@@ -50,7 +50,12 @@ inline cudaError_t allow_max_dynamic_smem() {
   const DeviceInfo& di = device_info();
   const int dev = di.device;
   if (done[dev].load(std::memory_order_acquire)) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(Kern, cudaFuncAttributeMaxDynamicSharedMemorySize, di.max_smem_optin);
+  cudaFuncAttributes fa{};
+  cudaError_t e = cudaFuncGetAttributes(&fa, Kern);
+  if (e != cudaSuccess) return e;
+  // the limit covers static and dynamic shared memory together
+  e = cudaFuncSetAttribute(Kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           di.max_smem_optin - (int)fa.sharedSizeBytes);
   if (e == cudaSuccess) done[dev].store(true, std::memory_order_release);
   return e;
 }

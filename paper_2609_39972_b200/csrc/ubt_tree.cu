@@ -45,11 +45,22 @@ struct TreeSmem {
   Span<int> depth_cnt;      // [L+2]
   Span<int> depth_off;      // [L+2]
   Span<uint32_t> maskrow;   // [N, mask_words]
-  Span<int> scalars;        // [0] = accepted count
+  Span<int> scalars;        // [0] = accepted count, [1] = threshold key of a round, [2] = flags
+  // Nodes enumerated by the parallel expansion (resident table only; see expand_rounds): node 0 is the root.
+  int xcap;                 // capacity (0 in lazy mode)
+  Span<short> x_parent;     // [xcap] enumerated parent, -1 for the root
+  Span<unsigned char> x_depth, x_rank, x_next, x_bak;  // [xcap] depth, candidate rank, next child to enumerate (+ its backup)
+  Span<float> x_score;      // [xcap]
+  Span<uint32_t> x_key;     // [xcap] ordering key of the node's best child not yet enumerated, 0 = none
+  Span<short> x_aux;        // [xcap] per-round scratch
+  Span<unsigned long long> x_key64;  // [xcap] ordering keys of the final choice
+  Span<int> x_wsum;         // [32] warp totals of the block scans
 };
 
 // Rows of the pair table are computed on demand when the whole table would not fit.
 __host__ __device__ inline bool tree_lazy(int L, int k) { return (size_t)L * k * k * 5 > kTreeTableBytes; }
+// Nodes the parallel expansion may enumerate before it picks the N - 1 best (root included).
+__host__ __device__ inline int expand_capacity(int N) { return 4 * N < 128 ? 128 : (4 * N > 1024 ? 1024 : 4 * N); }
 
 __host__ __device__ inline size_t tree_carve(TreeSmem* s, unsigned char* base, int L, int k, int N) {
   size_t off = 0;
@@ -71,7 +82,22 @@ __host__ __device__ inline size_t tree_carve(TreeSmem* s, unsigned char* base, i
   size_t o_pk = take(sizeof(unsigned long long) * 2 * N), o_kk = take(sizeof(int) * N);
   size_t o_dc = take(sizeof(int) * (L + 2)), o_do = take(sizeof(int) * (L + 2));
   size_t o_mk = take(sizeof(uint32_t) * N * mw), o_sc = take(sizeof(int) * 4);
+  const int xcap = lazy ? 0 : expand_capacity(N);
+  size_t o_xp = take(sizeof(short) * xcap), o_xd = take(xcap), o_xr = take(xcap), o_xn = take(xcap), o_xb = take(xcap);
+  size_t o_xs = take(sizeof(float) * xcap), o_xk = take(sizeof(uint32_t) * xcap), o_xa = take(sizeof(short) * xcap);
+  size_t o_xw = take(sizeof(int) * 32), o_x6 = take(sizeof(unsigned long long) * xcap);
   if (s) {
+    s->xcap = xcap;
+    s->x_parent = Span<short>((short*)(base + o_xp), xcap, 121);
+    s->x_depth = Span<unsigned char>(base + o_xd, xcap, 122);
+    s->x_rank = Span<unsigned char>(base + o_xr, xcap, 123);
+    s->x_next = Span<unsigned char>(base + o_xn, xcap, 124);
+    s->x_bak = Span<unsigned char>(base + o_xb, xcap, 125);
+    s->x_score = Span<float>((float*)(base + o_xs), xcap, 126);
+    s->x_key = Span<uint32_t>((uint32_t*)(base + o_xk), xcap, 127);
+    s->x_aux = Span<short>((short*)(base + o_xa), xcap, 128);
+    s->x_wsum = Span<int>((int*)(base + o_xw), 32, 129);
+    s->x_key64 = Span<unsigned long long>((unsigned long long*)(base + o_x6), xcap, 130);
     s->t = Span<float>((float*)(base + o_t), lkk, 101);
     s->ord = Span<unsigned char>(base + o_ord, lkk, 102);
     s->rowmap = Span<short>((short*)(base + o_rm), lazy ? lk + 1 : 0, 107);
@@ -325,10 +351,411 @@ __device__ int expand_tree(TreeSmem& s, const RowSource& src, int L, int k, int 
   return n_acc;
 }
 
-// LAZY: the rows of the pair table are computed on demand (see TreeSmem).  The resident-table kernel is held to
-// 40 registers so that its CTAs fit on an SM as soon as ONE CTA of the top-k kernel in front has left.
+// ---------------------------------------------------------------------------- parallel expansion
+// Exclusive prefix sum of one int per thread over the CTA (two barriers); `total` is the sum.
+template <int T>
+__device__ __forceinline__ int block_excl_scan(int v, Span<int> wsum, int& total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int up = __shfl_up_sync(FULL, inc, o);
+    if (lane >= o) inc += up;
+  }
+  if (lane == 31) wsum[warp] = inc;
+  __syncthreads();
+  int base = 0, tot = 0;
+#pragma unroll
+  for (int w = 0; w < T / 32; ++w) {
+    const int x = wsum[w];
+    base += w < warp ? x : 0;
+    tot += x;
+  }
+  __syncthreads();
+  total = tot;
+  return base + inc - v;
+}
+
+// Is enumerated node a before node b in the total order, given equal scores and equal depths?  Token ascending,
+// then the rank paths in lexicographic order (the candidates of a position are distinct tokens, so equal tokens
+// mean equal last ranks and the paths differ higher up).
+__device__ __noinline__ bool tie_before(const TreeSmem& s, int a, int b, int k) {
+  const int d = s.x_depth[a];
+  const int ta = s.tok[(d - 1) * k + s.x_rank[a]], tb = s.tok[(d - 1) * k + s.x_rank[b]];
+  if (ta != tb) return ta < tb;
+  int ra = 0, rb = 0;
+  while (a != b) {
+    ra = s.x_rank[a]; rb = s.x_rank[b];
+    a = s.x_parent[a]; b = s.x_parent[b];
+  }
+  return ra < rb;
+}
+
+// Algorithm 1 without a chain of N - 1 dependent pops: threshold rounds by one warp, then the final choice by
+// the whole CTA.
+//
+// Scores never increase from a node to its children or to its later siblings (rows are sorted), so for any
+// threshold the nodes that reach it form a set closed under "parent" and "earlier sibling" that can be
+// enumerated in parallel: every enumerated node (one per lane) counts how many of its next children reach the
+// threshold and appends them; the appended nodes do the same, wave after wave.  A round picks its threshold
+// among the ordering keys of the nodes' best not-yet-enumerated children -- roughly the m-th best, with m the
+// budget still open but at most half of those children (their keys are spread widely; the worst would pull in
+// far more than the budget has room for) -- so a round adds at least one node and usually about doubles the
+// set.  The threshold only steers how fast the set grows; the result does not depend on it: once at least
+// `budget` nodes are enumerated (or nothing is left), every node outside the set scores below every node
+// inside, the nodes of all rounds but the last beat those of the last, and the best of the last round under the
+// total order fill the remaining places (eq. 12).
+// Finite width (eq. 11): F_d = Top_W(E_d) holds the W best children of F_{d-1}, and nodes of earlier rounds beat
+// those of later rounds, so a round sweeps the depths in order and, where a depth would exceed W, keeps only
+// the best of its new candidates and closes the depth; the set is then F restricted to the threshold.
+//
+// expand_rounds_warp returns the number of enumerated nodes (root included; x_* arrays) and in `n_sure` how
+// many of them precede the last round, or -1 if the set outgrew its capacity even for the smallest step
+// (masses of exactly tied scores): the caller then falls back to the sequential search.
+__device__ int expand_rounds_warp(TreeSmem& s, int L, int k, int budget, int W, float zeta, int lane, int& n_sure) {
+  const bool capped = W > 0 && W < budget;
+  const int cap = s.xcap;
+  if (lane == 0) {
+    s.x_parent[0] = -1; s.x_depth[0] = 0; s.x_rank[0] = 0; s.x_next[0] = 0; s.x_score[0] = 0.f;
+  }
+  __syncwarp();
+  int n = 1, shrink = 0;
+  n_sure = 1;
+  // every round that is not taken back adds a node, and a round is taken back at most a few times
+  for (int guard = 0; budget - (n - 1) > 0; ++guard) {
+    if (guard > 16 * (budget + 16)) return -1;
+    const int remaining = budget - (n - 1);
+    // ---- ordering key of every node's best child not yet enumerated (0 = none)
+    int live = 0;
+    uint32_t kmax = 0u;
+    for (int i = lane; i < n; i += 32) {
+      const int d = s.x_depth[i], j = s.x_next[i];
+      uint32_t key = 0u;
+      if (d < L && j < k && (!capped || s.depth_cnt[d + 1] < W)) {
+        key = f2key(s.x_score[i] + s.t[(d * k + (int)s.x_rank[i]) * k + j] + zeta);
+        key = key == 0u ? 1u : key;
+      }
+      s.x_key[i] = key;
+      s.x_bak[i] = (unsigned char)j;
+      live += key != 0u;
+      kmax = key > kmax ? key : kmax;
+    }
+    live = __reduce_add_sync(FULL, live);
+    kmax = __reduce_max_sync(FULL, kmax);
+    if (live == 0) break;
+    if (capped) for (int i = lane; i < L + 2; i += 32) s.depth_off[i] = s.depth_cnt[i];  // backup for a retry
+    __syncwarp();
+    // ---- threshold: the m-th best key, exactly while the set has at most 32 nodes, from 32 evenly spaced
+    // nodes beyond that
+    const int half = (live + 1) >> 1;
+    int m = (remaining < half ? remaining : half) >> (2 * shrink);
+    m = m < 1 ? 1 : m;
+    uint32_t tau;
+    {
+      const int idx = n <= 32 ? lane : (lane * n) >> 5;
+      const uint32_t mine = idx < n ? s.x_key[idx] : 0u;
+      const int ls = __popc(__ballot_sync(FULL, mine != 0u));
+      int r = 0;
+#pragma unroll 8
+      for (int j = 0; j < 32; ++j) {
+        const uint32_t kj = __shfl_sync(FULL, mine, j);
+        r += (kj > mine) || (kj == mine && j < lane);
+      }
+      int want = ls > 0 ? (int)(((long long)m * ls + live - 1) / live) - 1 : 0;
+      want = want < 0 ? 0 : (want > ls - 1 ? ls - 1 : want);
+      const unsigned holder = __ballot_sync(FULL, mine != 0u && r == want);
+      tau = holder ? __shfl_sync(FULL, mine, __ffs(holder) - 1) : kmax;
+    }
+    const int n_before = n;
+    bool overflow = false;
+    // The qualifying children of node i, then those of the first child appended, and so on down: a chain of
+    // best children costs one wave instead of one per level (the other new children wait for the next wave).
+    // With `one` only node i's own children are taken (the depth sweep needs one depth at a time).
+    auto chain = [&](int i, int at, bool write, bool one) {
+      int d = s.x_depth[i], r = s.x_rank[i], j0 = s.x_next[i], par = i, total = 0;
+      float sc = s.x_score[i];
+      while (d < L) {
+        const int base = (d * k + r) * k;
+        int c = 0;
+        while (j0 + c < k && f2key(sc + s.t[base + j0 + c] + zeta) >= tau) ++c;
+        if (c == 0) break;
+        if (write) {
+          for (int q = 0; q < c; ++q) {
+            const int idx = at + q;
+            s.x_parent[idx] = (short)par; s.x_depth[idx] = (unsigned char)(d + 1);
+            s.x_rank[idx] = s.ord[base + j0 + q]; s.x_score[idx] = sc + s.t[base + j0 + q] + zeta;
+            s.x_next[idx] = 0;
+          }
+          s.x_next[par] = (unsigned char)(j0 + c);
+        }
+        total += c;
+        if (one) break;
+        sc = sc + s.t[base + j0] + zeta; r = s.ord[base + j0];
+        par = at; at += c; d += 1; j0 = 0;
+      }
+      return total;
+    };
+    // one batch of 32 nodes: lane `mine` appends; returns false on overflow
+    auto batch = [&](int i, bool mine, bool one) {
+      const int c = mine ? chain(i, 0, false, one) : 0;
+      int inc = c;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int up = __shfl_up_sync(FULL, inc, o);
+        if (lane >= o) inc += up;
+      }
+      const int total = __shfl_sync(FULL, inc, 31);
+      if (n + total > cap) return false;
+      if (c) chain(i, n + inc - c, true, one);
+      n += total;
+      return true;
+    };
+    if (!capped) {
+      int lo = 0, hi = n;
+      bool first = true;
+      while (true) {
+        const int n_wave = n;
+        for (int i0 = lo; i0 < hi && !overflow; i0 += 32) {
+          const int i = i0 + lane;
+          const bool mine = i < hi && (!first || (s.x_key[i] != 0u && s.x_key[i] >= tau));
+          if (!__any_sync(FULL, mine)) continue;
+          overflow = !batch(i, mine, false);
+        }
+        __syncwarp();  // the appended nodes are visible to every lane
+        if (overflow || n == n_wave) break;
+        lo = n_wave; hi = n; first = false;
+      }
+    } else {
+      for (int d = 1; d <= L && !overflow; ++d) {
+        const int room = W - s.depth_cnt[d];
+        const int n_d = n;  // nodes [0, n_d) are the possible parents; candidates go to [n_d, ...)
+        if (room <= 0) continue;
+        for (int i0 = 0; i0 < n_d && !overflow; i0 += 32) {
+          const int i = i0 + lane;
+          const bool mine = i < n_d && (int)s.x_depth[i] == d - 1;
+          if (!__any_sync(FULL, mine)) continue;
+          overflow = !batch(i, mine, true);
+        }
+        __syncwarp();
+        if (overflow) break;
+        const int total_d = n - n_d;
+        if (total_d > room) {
+          // rank the candidates of this depth among themselves (score desc, token asc, rank path asc)
+          for (int c = n_d + lane; c < n; c += 32) {
+            const uint32_t kc = f2key(s.x_score[c]);
+            int r = 0;
+            for (int j = n_d; j < n; ++j) {
+              const uint32_t kj = f2key(s.x_score[j]);
+              r += (kj > kc) || (kj == kc && j != c && tie_before(s, j, c, k));
+            }
+            s.x_aux[c] = (short)(r < room ? 1 : 0);
+          }
+          __syncwarp();
+          // stable compaction of the kept candidates to [n_d, n_d + room): destinations never pass sources
+          int moved = 0;
+          for (int c0 = n_d; c0 < n; c0 += 32) {
+            const int c = c0 + lane;
+            const int keep = c < n ? (int)s.x_aux[c] : 0;
+            short cp = 0; unsigned char cr = 0; float cs = 0.f;
+            if (keep) { cp = s.x_parent[c]; cr = s.x_rank[c]; cs = s.x_score[c]; }
+            const unsigned kept = __ballot_sync(FULL, keep);
+            __syncwarp();
+            if (keep) {
+              const int dst = n_d + moved + __popc(kept & ((1u << lane) - 1));
+              s.x_parent[dst] = cp; s.x_rank[dst] = cr; s.x_score[dst] = cs;
+              s.x_depth[dst] = (unsigned char)d; s.x_next[dst] = 0;
+            }
+            moved += __popc(kept);
+            __syncwarp();
+          }
+          n = n_d + room;
+          if (lane == 0) s.depth_cnt[d] = W;
+        } else if (lane == 0) {
+          s.depth_cnt[d] += total_d;
+        }
+        __syncwarp();
+      }
+    }
+    if (overflow) {
+      if (m == 1) return -1;
+      for (int i = lane; i < n_before; i += 32) s.x_next[i] = s.x_bak[i];
+      if (capped) for (int i = lane; i < L + 2; i += 32) s.depth_cnt[i] = s.depth_off[i];
+      n = n_before;
+      ++shrink;
+      __syncwarp();
+      continue;
+    }
+    shrink = 0;
+    n_sure = n_before;
+  }
+  return n;
+}
+
+// The same rounds by the whole CTA, for an unbounded width (no depth needs closing, so nodes may be appended in
+// any order): one thread per node, places in the node arrays reserved with a shared counter, one barrier per
+// wave.  The order of the nodes in the arrays then varies from run to run; the result does not (the final
+// choice and the slot layout depend on scores, depths and rank paths only).
+// scalars[1] = node count, scalars[2] = threshold key, scalars[3] = flags (1: nothing left, 2: out of room).
+template <int T>
+__device__ int expand_rounds_cta(TreeSmem& s, int L, int k, int budget, float zeta, int& n_sure) {
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int cap = s.xcap;
+  if (tid == 0) {
+    s.x_parent[0] = -1; s.x_depth[0] = 0; s.x_rank[0] = 0; s.x_next[0] = 0; s.x_score[0] = 0.f;
+    s.scalars[1] = 1;
+  }
+  __syncthreads();
+  int n = 1, shrink = 0;
+  n_sure = 1;
+  for (int guard = 0; budget - (n - 1) > 0; ++guard) {
+    if (guard > 16 * (budget + 16)) return -1;
+    const int remaining = budget - (n - 1);
+    for (int i = tid; i < n; i += T) {
+      const int d = s.x_depth[i], j = s.x_next[i];
+      uint32_t key = 0u;
+      if (d < L && j < k) {
+        key = f2key(s.x_score[i] + s.t[(d * k + (int)s.x_rank[i]) * k + j] + zeta);
+        key = key == 0u ? 1u : key;
+      }
+      s.x_key[i] = key;
+      s.x_bak[i] = (unsigned char)j;
+    }
+    __syncthreads();
+    if (tid < 32) {  // threshold of the round (see expand_rounds_warp)
+      int live = 0;
+      uint32_t kmax = 0u;
+      for (int i = lane; i < n; i += 32) {
+        const uint32_t key = s.x_key[i];
+        live += key != 0u;
+        kmax = key > kmax ? key : kmax;
+      }
+      live = __reduce_add_sync(FULL, live);
+      kmax = __reduce_max_sync(FULL, kmax);
+      const int half = (live + 1) >> 1;
+      int m = (remaining < half ? remaining : half) >> (2 * shrink);
+      m = m < 1 ? 1 : m;
+      const int idx = n <= 32 ? lane : (lane * n) >> 5;
+      const uint32_t mine = idx < n ? s.x_key[idx] : 0u;
+      const int ls = __popc(__ballot_sync(FULL, mine != 0u));
+      int r = 0;
+#pragma unroll 8
+      for (int j = 0; j < 32; ++j) {
+        const uint32_t kj = __shfl_sync(FULL, mine, j);
+        r += (kj > mine) || (kj == mine && j < lane);
+      }
+      int want = ls > 0 ? (int)(((long long)m * ls + live - 1) / (live > 0 ? live : 1)) - 1 : 0;
+      want = want < 0 ? 0 : (want > ls - 1 ? ls - 1 : want);
+      const unsigned holder = __ballot_sync(FULL, mine != 0u && r == want);
+      const uint32_t tau = holder ? __shfl_sync(FULL, mine, __ffs(holder) - 1) : kmax;
+      if (lane == 0) { s.scalars[2] = (int)tau; s.scalars[3] = (live == 0 ? 1 : 0) | (m == 1 ? 4 : 0); }
+    }
+    __syncthreads();
+    if (s.scalars[3] & 1) break;
+    const bool smallest_step = (s.scalars[3] & 4) != 0;
+    const uint32_t tau = (uint32_t)s.scalars[2];
+    const int n_before = n;
+    // The qualifying children of node i, then those of the first child appended, and so on down (a chain of
+    // best children costs one wave); every level reserves its places with the shared counter.
+    auto chain = [&](int i) {
+      int d = s.x_depth[i], r = s.x_rank[i], j0 = s.x_next[i], par = i;
+      float sc = s.x_score[i];
+      while (d < L) {
+        const int base = (d * k + r) * k;
+        int c = 0;
+        while (j0 + c < k && f2key(sc + s.t[base + j0 + c] + zeta) >= tau) ++c;
+        if (c == 0) break;
+        const int at = atomicAdd(&s.scalars[1], c);
+        if (at + c > cap) { atomicOr(&s.scalars[3], 2); break; }
+        for (int q = 0; q < c; ++q) {
+          const int idx = at + q;
+          s.x_parent[idx] = (short)par; s.x_depth[idx] = (unsigned char)(d + 1);
+          s.x_rank[idx] = s.ord[base + j0 + q]; s.x_score[idx] = sc + s.t[base + j0 + q] + zeta;
+          s.x_next[idx] = 0;
+        }
+        s.x_next[par] = (unsigned char)(j0 + c);
+        sc = sc + s.t[base + j0] + zeta; r = s.ord[base + j0];
+        par = at; d += 1; j0 = 0;
+      }
+    };
+    int lo = 0, hi = n;
+    bool first = true, overflow = false;
+    while (true) {
+      for (int i = lo + tid; i < hi; i += T)
+        if (!first || (s.x_key[i] != 0u && s.x_key[i] >= tau)) chain(i);
+      __syncthreads();  // the appended nodes and the counter are final for this wave
+      const int n_now = s.scalars[1];
+      overflow = (s.scalars[3] & 2) != 0;
+      __syncthreads();  // ... and every thread has read them before the next wave moves them on
+      if (overflow || n_now == hi) { n = n_now; break; }
+      lo = hi; hi = n_now; first = false;
+      n = n_now;
+    }
+    if (overflow) {
+      if (smallest_step) return -1;
+      for (int i = tid; i < n_before; i += T) s.x_next[i] = s.x_bak[i];
+      if (tid == 0) { s.scalars[1] = n_before; s.scalars[3] = 0; }
+      n = n_before;
+      ++shrink;
+      __syncthreads();
+      continue;
+    }
+    shrink = 0;
+    n_sure = n_before;
+  }
+  return n;
+}
+
+// The `budget` best of the enumerated nodes under the total order, compacted into nd_*; every thread of the
+// CTA calls it.  Nodes [1, n_sure) come from earlier rounds than [n_sure, n) and beat them all, so only the
+// nodes of the last round compete, for the places the earlier ones leave open.  Returns the number selected.
+template <int T>
+__device__ int select_enumerated(TreeSmem& s, int n, int n_sure, int budget, int k) {
+  const int tid = threadIdx.x;
+  const bool all = n - 1 <= budget;
+  const int places = budget - (n_sure - 1);
+  if (!all) {  // ordering keys of the competitors: (score, depth ascending)
+    for (int i = n_sure + tid; i < n; i += T)
+      s.x_key64[i] = ((uint64_t)f2key(s.x_score[i]) << 32) | (uint32_t)(255 - (int)s.x_depth[i]);
+  }
+  __syncthreads();
+  int n_sel = 0;
+  for (int i0 = 1; i0 < n; i0 += T) {
+    const int i = i0 + tid;
+    int sel = 0;
+    if (i < n) {
+      sel = 1;
+      if (!all && i >= n_sure) {
+        const uint64_t ki = s.x_key64[i];
+        int r = 0;
+        for (int j = n_sure; j < n; ++j) {
+          const uint64_t kj = s.x_key64[j];
+          r += (kj > ki) || (kj == ki && j != i && tie_before(s, j, i, k));
+        }
+        sel = r < places;
+      }
+    }
+    int total;
+    const int off = block_excl_scan<T>(sel, s.x_wsum, total);
+    if (i < n) s.x_aux[i] = (short)(sel ? n_sel + off : -1);
+    n_sel += total;
+  }
+  __syncthreads();
+  for (int i = 1 + tid; i < n; i += T) {
+    const int at = s.x_aux[i];
+    if (at < 0) continue;
+    const int p = s.x_parent[i];
+    s.nd_parent[at] = (short)(p == 0 ? -1 : s.x_aux[p]);
+    s.nd_depth[at] = s.x_depth[i];
+    s.nd_rank[at] = s.x_rank[i];
+    s.nd_score[at] = s.x_score[i];
+  }
+  __syncthreads();
+  return n_sel;
+}
+
+// LAZY: the rows of the pair table are computed on demand (see TreeSmem).
 template <bool LAZY>
-__global__ void __launch_bounds__(G2_T, LAZY ? 1 : 3)
+__global__ void __launch_bounds__(G2_T, LAZY ? 1 : 2)
 k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float zeta,
              const float* __restrict__ alpha, const float* __restrict__ lambda,
              const float* __restrict__ anchor_bigram, const int32_t* __restrict__ anchor_tokens,
@@ -497,11 +924,39 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   for (int i = tid; i < L + 2; i += G2_T) s.depth_cnt[i] = 0;
   for (int i = tid; i < N * mw; i += G2_T) s.maskrow[i] = 0u;
   __syncthreads();
-  // ---- best-first expansion (warp 0)
+  // ---- expansion: by the whole CTA when the table is resident; the sequential best-first search by one warp
+  // serves the lazy mode and the rare inputs the parallel form gives up on
   int bits = 1;
   while ((1 << bits) < k) ++bits;
   const bool use_pk = bits * L <= 128;
-  if (tid < 32) {
+  bool sequential = LAZY;
+  if constexpr (!LAZY) {
+    int n;
+    if (W > 0 && W < budget) {  // a finite width closes depths in order: one warp
+      if (tid < 32) {
+        int n_sure = 1;
+        const int nn = expand_rounds_warp(s, L, k, budget, W, zeta, lane, n_sure);
+        if (lane == 0) { s.scalars[1] = nn; s.scalars[2] = n_sure; }
+      }
+      __syncthreads();
+      n = s.scalars[1];
+    } else {
+      int n_sure = 1;
+      n = expand_rounds_cta<G2_T>(s, L, k, budget, zeta, n_sure);
+      __syncthreads();
+      if (tid == 0) s.scalars[2] = n_sure;
+      __syncthreads();
+    }
+    if (n < 0) {
+      sequential = true;
+      for (int i = tid; i < L + 2; i += G2_T) s.depth_cnt[i] = 0;
+      __syncthreads();
+    } else {
+      const int n_sel = select_enumerated<G2_T>(s, n, s.scalars[2], budget, k);
+      if (tid == 0) s.scalars[0] = n_sel;
+    }
+  }
+  if (sequential && tid < 32) {
     int n;
     RowSource src;
     src.bigram = L > 1 ? bigram + (size_t)b * (L - 1) * kk2 : nullptr;
