@@ -16,10 +16,11 @@ struct MergeParts {
 };
 
 // Every lane of one warp calls this for the same row.  Writes cand_ids[row, 0..k) (best first) and
-// cand_lp[row, r] = value - log-sum-exp of the whole row.
+// cand_lp[row, r] = value - log-sum-exp of the whole row; sm_ids / sm_lp, if given, receive a copy of the row's k
+// entries (the caller's shared-memory staging).
 __device__ __forceinline__ void merge_row_warp(const MergeParts& p, int64_t rows, int64_t row, int V, int k,
                                                int32_t* __restrict__ cand_ids_, float* __restrict__ cand_lp_,
-                                               int lane) {
+                                               int lane, int* sm_ids = nullptr, float* sm_lp = nullptr) {
   const long long nslots = rows * p.plan.smax;
   const Span<const float> part_ms(p.part_ms, nslots * 2, 321), part_val(p.part_val, nslots * k, 322);
   const Span<const int32_t> part_idx(p.part_idx, nslots * k, 323), part_cnt(p.part_cnt, nslots, 324);
@@ -30,35 +31,44 @@ __device__ __forceinline__ void merge_row_warp(const MergeParts& p, int64_t rows
   const int nseg = (int)(c_last - c_first + 1);
   const int64_t base = row * p.plan.smax;
 
-  float M = -1.0e30f;
-  for (int j = lane; j < nseg; j += 32) M = fmaxf(M, part_ms[(base + j) * 2]);
+  // every global load of the common case is issued before anything depends on one: a single round trip
+  const int nq = nseg * k;
+  float my_m = -1.0e30f, my_s = 0.f;
+  if (lane < nseg) { my_m = part_ms[(base + lane) * 2]; my_s = part_ms[(base + lane) * 2 + 1]; }
+  uint64_t key[2] = {0ull, 0ull};
+  float val[2] = {0.f, 0.f};
+  int pidx[2] = {0, 0}, pcnt[2] = {0, 0}, pi[2] = {0, 0};
+  if (nq <= 64) {
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      const int q = lane + 32 * c;
+      const int j = q / k, i = q - j * k;
+      pi[c] = i;
+      if (q < nq) {
+        pcnt[c] = part_cnt[base + j];
+        val[c] = part_val[(base + j) * k + i];   // slots beyond the count hold stale data: masked below
+        pidx[c] = part_idx[(base + j) * k + i];
+      }
+    }
+  }
+  float M = my_m;
+  for (int j = lane + 32; j < nseg; j += 32) M = fmaxf(M, part_ms[(base + j) * 2]);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(FULL, M, o));
-  float S = 0.f;
-  for (int j = lane; j < nseg; j += 32)
+  float S = lane < nseg ? my_s * exp2f((my_m - M) * kLog2e) : 0.f;
+  for (int j = lane + 32; j < nseg; j += 32)
     S += part_ms[(base + j) * 2 + 1] * exp2f((part_ms[(base + j) * 2] - M) * kLog2e);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) S += __shfl_xor_sync(FULL, S, o);
   const float lse = M + logf(S);
 
   int found = 0;
-  const int nq = nseg * k;
   if (nq <= 64) {
-    // The usual case (a row is cut into a few segments): every lane takes up to two entries into registers
-    // with independent loads, and the exact ranks are counted by exchanging keys with shuffles.
-    uint64_t key[2];
-    float val[2];
+    // The usual case (a row is cut into a few segments): every lane holds up to two entries in registers,
+    // and the exact ranks are counted by exchanging keys with shuffles.
 #pragma unroll
-    for (int c = 0; c < 2; ++c) {
-      const int q = lane + 32 * c;
-      const int j = q / k, i = q - j * k;
-      key[c] = 0ull;
-      val[c] = 0.f;
-      if (q < nq && i < part_cnt[base + j]) {
-        val[c] = part_val[(base + j) * k + i];
-        key[c] = make_key(val[c], part_idx[(base + j) * k + i]);
-      }
-    }
+    for (int c = 0; c < 2; ++c)
+      if (lane + 32 * c < nq && pi[c] < pcnt[c]) key[c] = make_key(val[c], pidx[c]);
     int rank[2] = {0, 0};
 #pragma unroll
     for (int c2 = 0; c2 < 2; ++c2) {
@@ -74,6 +84,7 @@ __device__ __forceinline__ void merge_row_warp(const MergeParts& p, int64_t rows
       if (key[c] != 0ull && rank[c] < k) {
         cand_ids[row * k + rank[c]] = key_idx(key[c]);
         cand_lp[row * k + rank[c]] = val[c] - lse;
+        if (sm_ids) { sm_ids[rank[c]] = key_idx(key[c]); sm_lp[rank[c]] = val[c] - lse; }
       }
   } else {
     // Many entries (large k, or a row cut into many segments): every segment's list is sorted best first, so an
@@ -99,6 +110,7 @@ __device__ __forceinline__ void merge_row_warp(const MergeParts& p, int64_t rows
       if (rank < k) {
         cand_ids[row * k + rank] = idx;
         cand_lp[row * k + rank] = val - lse;
+        if (sm_ids) { sm_ids[rank] = idx; sm_lp[rank] = val - lse; }
       }
     }
   }
@@ -108,6 +120,7 @@ __device__ __forceinline__ void merge_row_warp(const MergeParts& p, int64_t rows
   for (int r = found + lane; r < k; r += 32) {  // fewer than k entries above -inf: documented as unsupported
     cand_ids[row * k + r] = -1;
     cand_lp[row * k + r] = -INFINITY;
+    if (sm_ids) { sm_ids[r] = -1; sm_lp[r] = -INFINITY; }
   }
 }
 

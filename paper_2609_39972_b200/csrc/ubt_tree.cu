@@ -44,6 +44,7 @@ struct TreeSmem {
   Span<int> kk;             // per-depth sort keys (fallback slot assignment)
   Span<int> depth_cnt;      // [L+2]
   Span<int> depth_off;      // [L+2]
+  Span<int> x_fill;         // [L+2] fill counters of the grouping by depth
   Span<uint32_t> maskrow;   // [N, mask_words]
   Span<int> scalars;        // [0] = accepted count, [1] = threshold key of a round, [2] = flags
   // Nodes enumerated by the parallel expansion (resident table only; see expand_rounds): node 0 is the root.
@@ -62,67 +63,88 @@ __host__ __device__ inline bool tree_lazy(int L, int k) { return (size_t)L * k *
 // Nodes the parallel expansion may enumerate before it picks the N - 1 best (root included).
 __host__ __device__ inline int expand_capacity(int N) { return 4 * N < 128 ? 128 : (4 * N > 1024 ? 1024 : 4 * N); }
 
-__host__ __device__ inline size_t tree_carve(TreeSmem* s, unsigned char* base, int L, int k, int N) {
+// Byte offsets of the arrays above inside the CTA's dynamic shared memory.  They depend on L, k, N only, so
+// the host computes them once per launch and passes them as a kernel argument: the kernel then forms every
+// address from a constant-bank operand instead of keeping (or re-deriving) thirty pointers in registers.
+struct TreeLayout {
+  uint32_t t, ord, rowmap, la, pre, lp, tok, al, ent, nd_parent, nd_depth, nd_rank, nd_score, nd_slot, nd_pk, kk,
+      depth_cnt, depth_off, x_fill, maskrow, scalars, x_parent, x_depth, x_rank, x_next, x_bak, x_score, x_key, x_aux,
+      x_wsum, x_key64;
+  uint32_t total;
+  int xcap;
+};
+
+inline TreeLayout tree_layout(int L, int k, int N) {
+  TreeLayout o{};
   size_t off = 0;
   auto take = [&](size_t bytes) {
     size_t at = off;
     off = (off + bytes + 15) / 16 * 16;
-    return at;
+    return (uint32_t)at;
   };
   const int mw = (N + 31) / 32;
   const bool lazy = tree_lazy(L, k);
   const long long lkk = lazy ? (long long)N * k : (long long)L * k * k, lk = (long long)L * k;
-  size_t o_t = take(sizeof(float) * lkk), o_ord = take((size_t)lkk);
-  size_t o_rm = take(lazy ? sizeof(short) * (lk + 1) : 0), o_la = take(sizeof(float) * L);
-  size_t o_pre = take(lazy ? sizeof(float) * (size_t)(N + 1) * k : 0);
-  size_t o_lp = take(sizeof(float) * lk), o_tok = take(sizeof(int) * lk);
-  size_t o_al = take(sizeof(float) * L), o_en = take(sizeof(uint4) * (N + 1));
-  size_t o_np = take(sizeof(short) * N), o_nd = take(N), o_nr = take(N);
-  size_t o_ns = take(sizeof(float) * N), o_nl = take(sizeof(short) * N);
-  size_t o_pk = take(sizeof(unsigned long long) * 2 * N), o_kk = take(sizeof(int) * N);
-  size_t o_dc = take(sizeof(int) * (L + 2)), o_do = take(sizeof(int) * (L + 2));
-  size_t o_mk = take(sizeof(uint32_t) * N * mw), o_sc = take(sizeof(int) * 4);
+  o.t = take(sizeof(float) * lkk); o.ord = take((size_t)lkk);
+  o.rowmap = take(lazy ? sizeof(short) * (lk + 1) : 0); o.la = take(sizeof(float) * L);
+  o.pre = take(lazy ? sizeof(float) * (size_t)(N + 1) * k : 0);
+  o.lp = take(sizeof(float) * lk); o.tok = take(sizeof(int) * lk);
+  o.al = take(sizeof(float) * L); o.ent = take(sizeof(uint4) * (N + 1));
+  o.nd_parent = take(sizeof(short) * N); o.nd_depth = take(N); o.nd_rank = take(N);
+  o.nd_score = take(sizeof(float) * N); o.nd_slot = take(sizeof(short) * N);
+  o.nd_pk = take(sizeof(unsigned long long) * 2 * N); o.kk = take(sizeof(int) * N);
+  o.depth_cnt = take(sizeof(int) * (L + 2)); o.depth_off = take(sizeof(int) * (L + 2));
+  o.x_fill = take(sizeof(int) * (L + 2));
+  o.maskrow = take(sizeof(uint32_t) * N * mw); o.scalars = take(sizeof(int) * 4);
   const int xcap = lazy ? 0 : expand_capacity(N);
-  size_t o_xp = take(sizeof(short) * xcap), o_xd = take(xcap), o_xr = take(xcap), o_xn = take(xcap), o_xb = take(xcap);
-  size_t o_xs = take(sizeof(float) * xcap), o_xk = take(sizeof(uint32_t) * xcap), o_xa = take(sizeof(short) * xcap);
-  size_t o_xw = take(sizeof(int) * 32), o_x6 = take(sizeof(unsigned long long) * xcap);
-  if (s) {
-    s->xcap = xcap;
-    s->x_parent = Span<short>((short*)(base + o_xp), xcap, 121);
-    s->x_depth = Span<unsigned char>(base + o_xd, xcap, 122);
-    s->x_rank = Span<unsigned char>(base + o_xr, xcap, 123);
-    s->x_next = Span<unsigned char>(base + o_xn, xcap, 124);
-    s->x_bak = Span<unsigned char>(base + o_xb, xcap, 125);
-    s->x_score = Span<float>((float*)(base + o_xs), xcap, 126);
-    s->x_key = Span<uint32_t>((uint32_t*)(base + o_xk), xcap, 127);
-    s->x_aux = Span<short>((short*)(base + o_xa), xcap, 128);
-    s->x_wsum = Span<int>((int*)(base + o_xw), 32, 129);
-    s->x_key64 = Span<unsigned long long>((unsigned long long*)(base + o_x6), xcap, 130);
-    s->t = Span<float>((float*)(base + o_t), lkk, 101);
-    s->ord = Span<unsigned char>(base + o_ord, lkk, 102);
-    s->rowmap = Span<short>((short*)(base + o_rm), lazy ? lk + 1 : 0, 107);
-    s->la = Span<float>((float*)(base + o_la), L, 108);
-    s->pre = Span<float>((float*)(base + o_pre), lazy ? (long long)(N + 1) * k : 0, 120);
-    s->lp = Span<float>((float*)(base + o_lp), lk, 103);
-    s->tok = Span<int>((int*)(base + o_tok), lk, 104);
-    s->al = Span<float>((float*)(base + o_al), L, 105);
-    s->ent = Span<uint4>((uint4*)(base + o_en), N + 1, 106);
-    s->nd_parent = Span<short>((short*)(base + o_np), N, 109);
-    s->nd_depth = Span<unsigned char>(base + o_nd, N, 110);
-    s->nd_rank = Span<unsigned char>(base + o_nr, N, 111);
-    s->nd_score = Span<float>((float*)(base + o_ns), N, 112);
-    s->nd_slot = Span<short>((short*)(base + o_nl), N, 113);
-    s->nd_pk = Span<unsigned long long>((unsigned long long*)(base + o_pk), 2LL * N, 114);
-    s->kk = Span<int>((int*)(base + o_kk), N, 115);
-    s->depth_cnt = Span<int>((int*)(base + o_dc), L + 2, 116);
-    s->depth_off = Span<int>((int*)(base + o_do), L + 2, 117);
-    s->maskrow = Span<uint32_t>((uint32_t*)(base + o_mk), (long long)N * mw, 118);
-    s->scalars = Span<int>((int*)(base + o_sc), 4, 119);
-  }
-  return off;
+  o.xcap = xcap;
+  o.x_parent = take(sizeof(short) * xcap); o.x_depth = take(xcap); o.x_rank = take(xcap); o.x_next = take(xcap);
+  o.x_bak = take(xcap); o.x_score = take(sizeof(float) * xcap); o.x_key = take(sizeof(uint32_t) * xcap);
+  o.x_aux = take(sizeof(short) * xcap); o.x_wsum = take(sizeof(int) * 32);
+  o.x_key64 = take(sizeof(unsigned long long) * xcap);
+  o.total = (uint32_t)off;
+  return o;
 }
 
-size_t tree_smem_bytes(int L, int k, int N) { return tree_carve(nullptr, nullptr, L, k, N); }
+__device__ __forceinline__ void tree_bind(TreeSmem* s, unsigned char* base, const TreeLayout& o, int L, int k, int N) {
+  const int mw = (N + 31) / 32, xcap = o.xcap;
+  const bool lazy = xcap == 0;
+  const long long lkk = lazy ? (long long)N * k : (long long)L * k * k, lk = (long long)L * k;
+  s->xcap = xcap;
+  s->x_parent = Span<short>((short*)(base + o.x_parent), xcap, 121);
+  s->x_depth = Span<unsigned char>(base + o.x_depth, xcap, 122);
+  s->x_rank = Span<unsigned char>(base + o.x_rank, xcap, 123);
+  s->x_next = Span<unsigned char>(base + o.x_next, xcap, 124);
+  s->x_bak = Span<unsigned char>(base + o.x_bak, xcap, 125);
+  s->x_score = Span<float>((float*)(base + o.x_score), xcap, 126);
+  s->x_key = Span<uint32_t>((uint32_t*)(base + o.x_key), xcap, 127);
+  s->x_aux = Span<short>((short*)(base + o.x_aux), xcap, 128);
+  s->x_wsum = Span<int>((int*)(base + o.x_wsum), 32, 129);
+  s->x_key64 = Span<unsigned long long>((unsigned long long*)(base + o.x_key64), xcap, 130);
+  s->t = Span<float>((float*)(base + o.t), lkk, 101);
+  s->ord = Span<unsigned char>(base + o.ord, lkk, 102);
+  s->rowmap = Span<short>((short*)(base + o.rowmap), lazy ? lk + 1 : 0, 107);
+  s->la = Span<float>((float*)(base + o.la), L, 108);
+  s->pre = Span<float>((float*)(base + o.pre), lazy ? (long long)(N + 1) * k : 0, 120);
+  s->lp = Span<float>((float*)(base + o.lp), lk, 103);
+  s->tok = Span<int>((int*)(base + o.tok), lk, 104);
+  s->al = Span<float>((float*)(base + o.al), L, 105);
+  s->ent = Span<uint4>((uint4*)(base + o.ent), N + 1, 106);
+  s->nd_parent = Span<short>((short*)(base + o.nd_parent), N, 109);
+  s->nd_depth = Span<unsigned char>(base + o.nd_depth, N, 110);
+  s->nd_rank = Span<unsigned char>(base + o.nd_rank, N, 111);
+  s->nd_score = Span<float>((float*)(base + o.nd_score), N, 112);
+  s->nd_slot = Span<short>((short*)(base + o.nd_slot), N, 113);
+  s->nd_pk = Span<unsigned long long>((unsigned long long*)(base + o.nd_pk), 2LL * N, 114);
+  s->kk = Span<int>((int*)(base + o.kk), N, 115);
+  s->depth_cnt = Span<int>((int*)(base + o.depth_cnt), L + 2, 116);
+  s->depth_off = Span<int>((int*)(base + o.depth_off), L + 2, 117);
+  s->x_fill = Span<int>((int*)(base + o.x_fill), L + 2, 131);
+  s->maskrow = Span<uint32_t>((uint32_t*)(base + o.maskrow), (long long)N * mw, 118);
+  s->scalars = Span<int>((int*)(base + o.scalars), 4, 119);
+}
+
+size_t tree_smem_bytes(int L, int k, int N) { return tree_layout(L, k, N).total; }
 
 // A frontier entry is one 16-byte record in shared memory (entry i belongs to lane i & 31, slot i >> 5); only
 // its ordering key is mirrored in a register of the owner lane, so that finding the best entry is a register
@@ -165,7 +187,7 @@ __device__ __forceinline__ void prefetch_row(TreeSmem& s, const RowSource& src, 
 // (t desc, token asc) into cache slot `slot` (the search never looks further down a row: at most W, or the whole
 // budget, of its entries can be accepted, plus one that is dropped).  Successors are extracted one per round by
 // a warp maximum over (score key, ~token); the candidates of a position are distinct tokens.
-__device__ __noinline__ void lazy_row(TreeSmem& s, int q, int e, int slot, int k, int m, int lane) {
+__device__ __forceinline__ void lazy_row(TreeSmem& s, int q, int e, int slot, int k, int m, int lane) {
   const int i = q / k;
   const float al = s.al[i], la = s.la[i];
   cp_async_wait_all();
@@ -216,7 +238,7 @@ __device__ __noinline__ void lazy_row(TreeSmem& s, int q, int e, int slot, int k
 // of its node's children (13 bits); with the whole table resident that row starts at q * k, in lazy mode at
 // rowmap[q] * k, computed when the node is popped for the first time.
 template <int SLOTS, bool LAZY>
-__device__ int expand_tree(TreeSmem& s, const RowSource& src, int L, int k, int budget, int W, float zeta, int lane) {
+__device__ __forceinline__ int expand_tree(TreeSmem& s, const RowSource& src, int L, int k, int budget, int W, float zeta, int lane) {
   uint32_t fk[SLOTS];
 #pragma unroll
   for (int q = 0; q < SLOTS; ++q) fk[q] = 0u;
@@ -379,7 +401,7 @@ __device__ __forceinline__ int block_excl_scan(int v, Span<int> wsum, int& total
 // Is enumerated node a before node b in the total order, given equal scores and equal depths?  Token ascending,
 // then the rank paths in lexicographic order (the candidates of a position are distinct tokens, so equal tokens
 // mean equal last ranks and the paths differ higher up).
-__device__ __noinline__ bool tie_before(const TreeSmem& s, int a, int b, int k) {
+__device__ __forceinline__ bool tie_before(const TreeSmem& s, int a, int b, int k) {
   const int d = s.x_depth[a];
   const int ta = s.tok[(d - 1) * k + s.x_rank[a]], tb = s.tok[(d - 1) * k + s.x_rank[b]];
   if (ta != tb) return ta < tb;
@@ -412,7 +434,7 @@ __device__ __noinline__ bool tie_before(const TreeSmem& s, int a, int b, int k) 
 // expand_rounds_warp returns the number of enumerated nodes (root included; x_* arrays) and in `n_sure` how
 // many of them precede the last round, or -1 if the set outgrew its capacity even for the smallest step
 // (masses of exactly tied scores): the caller then falls back to the sequential search.
-__device__ int expand_rounds_warp(TreeSmem& s, int L, int k, int budget, int W, float zeta, int lane, int& n_sure) {
+__device__ __forceinline__ int expand_rounds_warp(TreeSmem& s, int L, int k, int budget, int W, float zeta, int lane, int& n_sure) {
   const bool capped = W > 0 && W < budget;
   const int cap = s.xcap;
   if (lane == 0) {
@@ -461,7 +483,7 @@ __device__ int expand_rounds_warp(TreeSmem& s, int L, int k, int budget, int W, 
         const uint32_t kj = __shfl_sync(FULL, mine, j);
         r += (kj > mine) || (kj == mine && j < lane);
       }
-      int want = ls > 0 ? (int)(((long long)m * ls + live - 1) / live) - 1 : 0;
+      int want = ls > 0 ? (m * ls + live - 1) / live - 1 : 0;
       want = want < 0 ? 0 : (want > ls - 1 ? ls - 1 : want);
       const unsigned holder = __ballot_sync(FULL, mine != 0u && r == want);
       tau = holder ? __shfl_sync(FULL, mine, __ffs(holder) - 1) : kmax;
@@ -591,65 +613,96 @@ __device__ int expand_rounds_warp(TreeSmem& s, int L, int k, int budget, int W, 
   return n;
 }
 
-// The same rounds by the whole CTA, for an unbounded width (no depth needs closing, so nodes may be appended in
-// any order): one thread per node, places in the node arrays reserved with a shared counter, one barrier per
-// wave.  The order of the nodes in the arrays then varies from run to run; the result does not (the final
-// choice and the slot layout depend on scores, depths and rank paths only).
-// scalars[1] = node count, scalars[2] = threshold key, scalars[3] = flags (1: nothing left, 2: out of room).
-template <int T>
-__device__ int expand_rounds_cta(TreeSmem& s, int L, int k, int budget, float zeta, int& n_sure) {
+// The same rounds by EX_T threads (four warps; the others wait at the CTA barrier behind the call), for an
+// unbounded width: no depth needs closing, so nodes may be appended in any order -- one thread per node, places in
+// the node arrays reserved with a shared counter, two barriers per wave.  The order of the nodes in the arrays
+// then varies from run to run; the result does not (the final choice and the slot layout depend on scores,
+// depths and rank paths only).
+// Threshold of a round: the rank rule of expand_rounds_warp on 32 evenly spaced nodes, lowered further, from the
+// third round on, to where the count of enumerated nodes -- which grows roughly geometrically as the threshold
+// falls -- is expected to pass the budget (a secant step on log(count) over the last two thresholds).  A round
+// that outgrows the node arrays is taken back and repeated with a smaller step.
+// scalars[1] = node count, scalars[2] = threshold key, scalars[3] = flags (1: nothing left, 2: out of room,
+// 4: smallest step).
+constexpr int EX_T = 128;
+__device__ __forceinline__ void ex_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(EX_T) : "memory"); }
+
+__device__ __forceinline__ int expand_rounds_cta(TreeSmem& s, int L, int k, int budget, float zeta, int& n_sure) {
   const int tid = threadIdx.x, lane = tid & 31;
   const int cap = s.xcap;
   if (tid == 0) {
     s.x_parent[0] = -1; s.x_depth[0] = 0; s.x_rank[0] = 0; s.x_next[0] = 0; s.x_score[0] = 0.f;
     s.scalars[1] = 1;
+    s.scalars[3] = 0;
   }
-  __syncthreads();
+  ex_barrier();
   int n = 1, shrink = 0;
   n_sure = 1;
+  // ordering key of node i's best child not yet enumerated, 0 = none
+  auto open_key = [&](int i) -> uint32_t {
+    const int d = s.x_depth[i], j = s.x_next[i];
+    if (d >= L || j >= k) return 0u;
+    const uint32_t key = f2key(s.x_score[i] + s.t[(d * k + (int)s.x_rank[i]) * k + j] + zeta);
+    return key == 0u ? 1u : key;
+  };
+  float t_prev = 0.f, t_prev2 = 0.f;  // thresholds of the last two rounds that stood (warp 0 only)
+  int n_prev = 0, n_prev2 = 0;        // ... and the node counts they led to
   for (int guard = 0; budget - (n - 1) > 0; ++guard) {
     if (guard > 16 * (budget + 16)) return -1;
     const int remaining = budget - (n - 1);
-    for (int i = tid; i < n; i += T) {
-      const int d = s.x_depth[i], j = s.x_next[i];
-      uint32_t key = 0u;
-      if (d < L && j < k) {
-        key = f2key(s.x_score[i] + s.t[(d * k + (int)s.x_rank[i]) * k + j] + zeta);
-        key = key == 0u ? 1u : key;
+    if (tid < 32) {
+      const int idx = n <= 32 ? lane : (lane * n) >> 5;
+      const uint32_t mine = idx < n ? open_key(idx) : 0u;
+      int ls = __popc(__ballot_sync(FULL, mine != 0u));
+      uint32_t kmax = __reduce_max_sync(FULL, mine);
+      int live = n <= 32 ? ls : (ls * n + 31) >> 5;  // beyond 32 nodes an estimate is all the rule needs
+      if (ls == 0 && n > 32) {                       // none in the sample: look at every node
+        int cnt = 0;
+        for (int i = lane; i < n; i += 32) {
+          const uint32_t key = open_key(i);
+          cnt += key != 0u;
+          kmax = key > kmax ? key : kmax;
+        }
+        live = __reduce_add_sync(FULL, cnt);
+        kmax = __reduce_max_sync(FULL, kmax);
       }
-      s.x_key[i] = key;
-      s.x_bak[i] = (unsigned char)j;
-    }
-    __syncthreads();
-    if (tid < 32) {  // threshold of the round (see expand_rounds_warp)
-      int live = 0;
-      uint32_t kmax = 0u;
-      for (int i = lane; i < n; i += 32) {
-        const uint32_t key = s.x_key[i];
-        live += key != 0u;
-        kmax = key > kmax ? key : kmax;
-      }
-      live = __reduce_add_sync(FULL, live);
-      kmax = __reduce_max_sync(FULL, kmax);
       const int half = (live + 1) >> 1;
       int m = (remaining < half ? remaining : half) >> (2 * shrink);
       m = m < 1 ? 1 : m;
-      const int idx = n <= 32 ? lane : (lane * n) >> 5;
-      const uint32_t mine = idx < n ? s.x_key[idx] : 0u;
-      const int ls = __popc(__ballot_sync(FULL, mine != 0u));
       int r = 0;
 #pragma unroll 8
       for (int j = 0; j < 32; ++j) {
         const uint32_t kj = __shfl_sync(FULL, mine, j);
         r += (kj > mine) || (kj == mine && j < lane);
       }
-      int want = ls > 0 ? (int)(((long long)m * ls + live - 1) / (live > 0 ? live : 1)) - 1 : 0;
+      int want = ls > 0 ? (m * ls + live - 1) / (live > 0 ? live : 1) - 1 : 0;
       want = want < 0 ? 0 : (want > ls - 1 ? ls - 1 : want);
       const unsigned holder = __ballot_sync(FULL, mine != 0u && r == want);
-      const uint32_t tau = holder ? __shfl_sync(FULL, mine, __ffs(holder) - 1) : kmax;
-      if (lane == 0) { s.scalars[2] = (int)tau; s.scalars[3] = (live == 0 ? 1 : 0) | (m == 1 ? 4 : 0); }
+      uint32_t tau = holder ? __shfl_sync(FULL, mine, __ffs(holder) - 1) : kmax;
+      if (shrink == 0 && n_prev2 >= 8 && n_prev > n_prev2 && t_prev < t_prev2) {
+        // secant step, never below the key that the rank rule gives for the whole open budget
+        int mf = remaining < live ? remaining : live;
+        int wf = ls > 0 ? (mf * ls + live - 1) / (live > 0 ? live : 1) - 1 : 0;
+        wf = wf < 0 ? 0 : (wf > ls - 1 ? ls - 1 : wf);
+        const unsigned hf = __ballot_sync(FULL, mine != 0u && r == wf);
+        const uint32_t tau_full = hf ? __shfl_sync(FULL, mine, __ffs(hf) - 1) : tau;
+        const float ln1 = __logf((float)n_prev2), ln2 = __logf((float)n_prev);
+        const float slope = (ln2 - ln1) / (t_prev2 - t_prev);
+        const float ts = t_prev - (__logf((float)(budget + 1)) - ln2) / slope;
+        if (ts == ts && ts < 0.f) {
+          uint32_t ks = f2key(ts);
+          ks = ks == 0u ? 1u : ks;
+          ks = ks < tau_full ? tau_full : ks;
+          tau = ks < tau ? ks : tau;
+        }
+      }
+      if (tau > kmax) tau = kmax;  // a round must add at least the best open child
+      if (lane == 0) {
+        s.scalars[2] = (int)tau;
+        s.scalars[3] = (live == 0 || kmax == 0u ? 1 : 0) | (m == 1 && shrink > 0 ? 4 : 0);
+      }
     }
-    __syncthreads();
+    ex_barrier();
     if (s.scalars[3] & 1) break;
     const bool smallest_step = (s.scalars[3] & 4) != 0;
     const uint32_t tau = (uint32_t)s.scalars[2];
@@ -680,27 +733,31 @@ __device__ int expand_rounds_cta(TreeSmem& s, int L, int k, int budget, float ze
     int lo = 0, hi = n;
     bool first = true, overflow = false;
     while (true) {
-      for (int i = lo + tid; i < hi; i += T)
-        if (!first || (s.x_key[i] != 0u && s.x_key[i] >= tau)) chain(i);
-      __syncthreads();  // the appended nodes and the counter are final for this wave
+      for (int i = lo + tid; i < hi; i += EX_T) {
+        if (first) s.x_bak[i] = s.x_next[i];  // for taking the round back
+        chain(i);
+      }
+      ex_barrier();  // the appended nodes and the counter are final for this wave
       const int n_now = s.scalars[1];
       overflow = (s.scalars[3] & 2) != 0;
-      __syncthreads();  // ... and every thread has read them before the next wave moves them on
+      ex_barrier();  // ... and every thread has read them before the next wave moves them on
       if (overflow || n_now == hi) { n = n_now; break; }
       lo = hi; hi = n_now; first = false;
       n = n_now;
     }
     if (overflow) {
       if (smallest_step) return -1;
-      for (int i = tid; i < n_before; i += T) s.x_next[i] = s.x_bak[i];
+      for (int i = tid; i < n_before; i += EX_T) s.x_next[i] = s.x_bak[i];
       if (tid == 0) { s.scalars[1] = n_before; s.scalars[3] = 0; }
       n = n_before;
       ++shrink;
-      __syncthreads();
+      ex_barrier();
       continue;
     }
     shrink = 0;
     n_sure = n_before;
+    t_prev2 = t_prev; n_prev2 = n_prev;
+    t_prev = key2f(tau); n_prev = n;
   }
   return n;
 }
@@ -709,7 +766,7 @@ __device__ int expand_rounds_cta(TreeSmem& s, int L, int k, int budget, float ze
 // CTA calls it.  Nodes [1, n_sure) come from earlier rounds than [n_sure, n) and beat them all, so only the
 // nodes of the last round compete, for the places the earlier ones leave open.  Returns the number selected.
 template <int T>
-__device__ int select_enumerated(TreeSmem& s, int n, int n_sure, int budget, int k) {
+__device__ __forceinline__ int select_enumerated(TreeSmem& s, int n, int n_sure, int budget, int k) {
   const int tid = threadIdx.x;
   const bool all = n - 1 <= budget;
   const int places = budget - (n_sure - 1);
@@ -726,11 +783,15 @@ __device__ int select_enumerated(TreeSmem& s, int n, int n_sure, int budget, int
       sel = 1;
       if (!all && i >= n_sure) {
         const uint64_t ki = s.x_key64[i];
-        int r = 0;
+        int r = 0, eq = 0;
+#pragma unroll 4
         for (int j = n_sure; j < n; ++j) {
           const uint64_t kj = s.x_key64[j];
-          r += (kj > ki) || (kj == ki && j != i && tie_before(s, j, i, k));
+          r += kj > ki;
+          eq += kj == ki;
         }
+        if (eq > 1 && r < places)  // exactly tied scores at one depth (rare): token, then rank path decide
+          for (int j = n_sure; j < n; ++j) r += s.x_key64[j] == ki && j != i && tie_before(s, j, i, k);
         sel = r < places;
       }
     }
@@ -753,16 +814,69 @@ __device__ int select_enumerated(TreeSmem& s, int n, int n_sure, int budget, int
   return n_sel;
 }
 
+// eq. 5 and eq. 9, then the sort by (t desc, token asc), one THREAD per (position, predecessor) row, for k <= KP
+// <= 16: the row lives in registers, nothing is exchanged between lanes and the k^2 comparisons are independent
+// of one another.  Element e of the row is visited in an order that starts at tid % k, so that the lanes of a
+// warp spread over the shared-memory banks.  In place: a thread reads its whole row before it rewrites it.
+template <int KP>
+__device__ __forceinline__ void prepare_rows_by_thread(TreeSmem& s, int k, int nrows, int tid) {
+  const int start = tid % k;
+  for (int r = tid; r < nrows; r += G2_T) {
+    const int i = r == 0 ? 0 : 1 + (r - 1) / k;
+    const int ra = r == 0 ? 0 : (r - 1) % k;
+    const int at = (i * k + ra) * k;
+    const float al = s.al[i];
+    float v[KP];
+    int tk[KP];
+    float mx = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < KP; ++j) {
+      int e = start + j;
+      e = e >= k ? e - k : e;
+      v[j] = -INFINITY;
+      tk[j] = 0;
+      if (j < k) {
+        v[j] = fmaf(al, s.lp[i * k + e], s.t[at + e]);
+        tk[j] = s.tok[i * k + e];
+        mx = fmaxf(mx, v[j]);
+      }
+    }
+    float sum = 0.f;
+#pragma unroll
+    for (int j = 0; j < KP; ++j) sum += j < k ? expf(v[j] - mx) : 0.f;
+    const float lse = mx + logf(sum);
+    unsigned long long key[KP];  // (value desc, token asc) as one descending key
+#pragma unroll
+    for (int j = 0; j < KP; ++j) {
+      v[j] -= lse;
+      key[j] = ((unsigned long long)f2key(v[j]) << 32) | (uint32_t)(~(uint32_t)tk[j]);
+    }
+#pragma unroll
+    for (int a = 0; a < KP; ++a) {
+      if (a >= k) break;
+      int rank = 0;
+#pragma unroll
+      for (int c = 0; c < KP; ++c)
+        if (c < k) rank += (key[c] > key[a]) || (key[c] == key[a] && c < a);  // equal keys: a permutation all the same
+      int e = start + a;
+      e = e >= k ? e - k : e;
+      s.t[at + rank] = v[a];
+      s.ord[at + rank] = (unsigned char)e;
+    }
+  }
+}
+
 // LAZY: the rows of the pair table are computed on demand (see TreeSmem).
 template <bool LAZY>
-__global__ void __launch_bounds__(G2_T, LAZY ? 1 : 2)
+__global__ void __launch_bounds__(G2_T, 1)
 k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float zeta,
              const float* __restrict__ alpha, const float* __restrict__ lambda,
              const float* __restrict__ anchor_bigram, const int32_t* __restrict__ anchor_tokens,
-             const int32_t* __restrict__ pos_offset, ubt_tree out, MergeParts parts, int V) {
+             const int32_t* __restrict__ pos_offset, ubt_tree out, MergeParts parts, int V,
+             const __grid_constant__ TreeLayout lay) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   TreeSmem s;
-  tree_carve(&s, smem_raw, L, k, N);
+  tree_bind(&s, smem_raw, lay, L, k, N);
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
   const int kk2 = k * k, mw = (N + 31) / 32, budget = N - 1;
   const long long nB = gridDim.x;
@@ -810,21 +924,29 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   }
   pdl_wait();  // the partials / candidates come from the kernel before this one
 
-  // ---- step a1's last part when fused: merge the row partials of this sequence's L rows
+  // ---- step a1's last part when fused: merge the row partials of this sequence's L rows (one warp per row; the
+  // candidates go to global memory and to the shared-memory staging at once); otherwise stage the candidates
   if (parts.part_ms != nullptr) {
     for (int i = tid >> 5; i < L; i += G2_T / 32)
-      merge_row_warp(parts, nB * L, (int64_t)b * L + i, V, k, out.cand_ids, out.cand_logprob, lane);
-    __syncthreads();  // the candidates were written by this CTA; the barrier orders them before the reads below
-  }
-  // ---- stage candidates and raw selector scores
-  for (int i = tid; i < L * k; i += G2_T) {
-    s.lp[i] = g_lp[(int64_t)b * L * k + i];
-    s.tok[i] = g_ids[(int64_t)b * L * k + i];
+      merge_row_warp(parts, nB * L, (int64_t)b * L + i, V, k, out.cand_ids, out.cand_logprob, lane,
+                     s.tok.ptr((long long)i * k, k), s.lp.ptr((long long)i * k, k));
+  } else {
+    for (int i = tid; i < L * k; i += G2_T) {
+      s.lp[i] = g_lp[(int64_t)b * L * k + i];
+      s.tok[i] = g_ids[(int64_t)b * L * k + i];
+    }
   }
   int kp = 1;
   while (kp < k) kp <<= 1;
   if constexpr (lazy) {
     // rows are normalised and sorted by the expanding warp, one at a time, when the search first needs them
+  } else if (k <= 16) {
+    __syncthreads();  // s.lp, s.tok
+    if (kp == 1) prepare_rows_by_thread<1>(s, k, nrows, tid);
+    else if (kp == 2) prepare_rows_by_thread<2>(s, k, nrows, tid);
+    else if (kp == 4) prepare_rows_by_thread<4>(s, k, nrows, tid);
+    else if (kp == 8) prepare_rows_by_thread<8>(s, k, nrows, tid);
+    else prepare_rows_by_thread<16>(s, k, nrows, tid);
   } else if (k <= 32) {
     // ---- eq. 5 and eq. 9, then every row sorted by (t desc, token asc): a group of kp = 2^ceil(log2 k)
     // lanes per (position, predecessor) row, the row's values in registers, reductions and exact ranks by
@@ -941,11 +1063,13 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
       __syncthreads();
       n = s.scalars[1];
     } else {
-      int n_sure = 1;
-      n = expand_rounds_cta<G2_T>(s, L, k, budget, zeta, n_sure);
+      if (tid < EX_T) {
+        int n_sure = 1;
+        const int nn = expand_rounds_cta(s, L, k, budget, zeta, n_sure);
+        if (tid == 0) { s.scalars[1] = nn; s.scalars[2] = n_sure; }
+      }
       __syncthreads();
-      if (tid == 0) s.scalars[2] = n_sure;
-      __syncthreads();
+      n = s.scalars[1];
     }
     if (n < 0) {
       sequential = true;
@@ -969,7 +1093,7 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   __syncthreads();
   // ---- canonical slots: root 0, then depth by depth ordered by (parent slot, rank)
   const int n_acc = s.scalars[0];
-  for (int i = tid; i < L + 2; i += G2_T) s.depth_cnt[i] = 0;
+  for (int i = tid; i < L + 2; i += G2_T) { s.depth_cnt[i] = 0; s.x_fill[i] = 0; }
   __syncthreads();
   if (tid < n_acc) {
     atomicAdd(&s.depth_cnt[s.nd_depth[tid]], 1);
@@ -995,20 +1119,30 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   }
   __syncthreads();
   if (use_pk) {
-    // inside a depth, (parent slot, rank) order is the lexicographic order of the rank paths; the count for
-    // one node is shared by `sp` neighbouring lanes
+    // inside a depth, (parent slot, rank) order is the lexicographic order of the rank paths.  The nodes are first
+    // grouped by depth (kk = node indices, depth by depth), so that a node is compared with its own depth only;
+    // the count for one node is shared by `sp` neighbouring lanes
+    if (tid < n_acc) {
+      const int d = s.nd_depth[tid];
+      s.kk[s.depth_off[d] - 1 + atomicAdd(&s.x_fill[d], 1)] = tid;
+    }
+    __syncthreads();
     int sp = 1;
-    while (sp < 32 && sp * 2 * N <= G2_T) sp <<= 1;
+    while (sp < 32 && sp * 2 * n_acc <= 2 * G2_T && sp * 2 * n_acc > 0) sp <<= 1;
+    if (sp * n_acc > G2_T) sp >>= 1;
     const int node = tid / sp, q = tid & (sp - 1);
     const bool mine = node < n_acc;
     const int d = mine ? s.nd_depth[node] : 0;
     const unsigned long long hi = mine ? s.nd_pk[2 * node] : 0ull, lo = mine ? s.nd_pk[2 * node + 1] : 0ull;
     int c = 0;
-    if (mine)
-      for (int j = q; j < n_acc; j += sp) {
+    if (mine) {
+      const int b0 = s.depth_off[d] - 1, b1 = b0 + s.depth_cnt[d];
+      for (int jj = b0 + q; jj < b1; jj += sp) {
+        const int j = s.kk[jj];
         const unsigned long long hj = s.nd_pk[2 * j], lj = s.nd_pk[2 * j + 1];
-        c += (s.nd_depth[j] == d) && (hj < hi || (hj == hi && lj < lo));
+        c += hj < hi || (hj == hi && lj < lo);
       }
+    }
     for (int o = sp >> 1; o > 0; o >>= 1) c += __shfl_xor_sync(FULL, c, o);
     if (mine && q == 0) s.nd_slot[node] = (short)(s.depth_off[d] + c);
     __syncthreads();
@@ -1092,14 +1226,15 @@ cudaError_t launch_build_tree(const float* bigram, int B, int L, int k, int N, i
                               const int32_t* anchor_tokens, const int32_t* pos_offset,
                               const ubt_tree& out, const MergeParts& parts, int V, cudaStream_t st) {
   if (B == 0) return cudaSuccess;
-  const size_t smem = tree_smem_bytes(L, k, N);
+  const TreeLayout lay = tree_layout(L, k, N);
+  const size_t smem = lay.total;
   const bool lazy = tree_lazy(L, k);
   auto kern = lazy ? k_build_tree<true> : k_build_tree<false>;
   cudaError_t e = lazy ? allow_max_dynamic_smem<k_build_tree<true>>() : allow_max_dynamic_smem<k_build_tree<false>>();
   if (e != cudaSuccess) return e;
   // programmatic launch only when the kernel before it is this library's own streaming kernel
   return launch_kernel(kern, dim3(B), dim3(G2_T), smem, st, parts.part_ms != nullptr, bigram, L, k, N, W,
-                       zeta, alpha, lambda, anchor_bigram, anchor_tokens, pos_offset, out, parts, V);
+                       zeta, alpha, lambda, anchor_bigram, anchor_tokens, pos_offset, out, parts, V, lay);
 }
 
 cudaError_t launch_build_mask(const ubt_tree& tree, const int32_t* pos_offset, cudaStream_t st) {
