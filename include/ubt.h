@@ -21,7 +21,10 @@
  *   - Argument errors are detected on the host and returned before anything is launched.
  *     A failed launch returns UBT_ERR_CUDA.  Nothing in the library traps; the only device-side waits
  *     (for a bulk copy to land) are bounded and counted by ubt_debug_ring_timeouts().
- *   - Logits must be free of NaN; each row must hold at least k entries greater than -inf.
+ *   - Logits must be free of NaN and +inf (-inf is allowed; each row must hold at least k entries
+ *     greater than -inf).  Nothing traps on a violation and every result stays memory-safe, but the
+ *     results of the sequence concerned are unspecified.  The calls detect it at no extra pass: pass a
+ *     `status` array in the options to learn which sequences were affected.
  *
  * Sizes: B sequences, L draft positions (the paper's gamma), V vocabulary, k candidates per position
  * (the paper's K), N = node budget = tree slots INCLUDING the root (the paper's budget B counts
@@ -47,8 +50,13 @@ typedef enum {
   UBT_ERR_UNSUPPORTED = 2, /* valid request beyond the compiled limits above */
   UBT_ERR_WORKSPACE = 3,   /* workspace NULL or smaller than ubt_*_workspace_bytes() */
   UBT_ERR_CUDA = 4,        /* a CUDA call or kernel launch failed */
-  UBT_ERR_STATIC_SCRATCH = 5 /* request larger than the built-in scratch of ubt_verify_tree_static */
+  UBT_ERR_STATIC_SCRATCH = 5, /* request larger than the built-in scratch of ubt_verify_tree_static */
+  UBT_ERR_NONFINITE = 6    /* host-buffer forms with validate_finite: a NaN or +inf among the logits */
 } ubt_status;
+
+/* Bits of the per-sequence status words (ubt_draft_opts.status, ubt_verify_opts.status). */
+#define UBT_STATUS_NONFINITE 1    /* a NaN or +inf among the sequence's logits: its results are unspecified */
+#define UBT_STATUS_WAIT_GAVE_UP 2 /* a bounded device-side wait gave up: its results are undefined */
 
 typedef enum { UBT_F32 = 0, UBT_BF16 = 1 } ubt_dtype;
 typedef enum { UBT_VERIFY_GREEDY = 0, UBT_VERIFY_SAMPLE = 1 } ubt_verify_mode;
@@ -86,6 +94,10 @@ typedef struct ubt_draft_opts {
   void *event_between;          /* optional cudaEvent_t recorded on the stream between the V-wide kernel of step
                                    a1 and the tree kernel (ubt_draft_tree only; for timing the two apart -- an
                                    event between them also keeps the second from becoming resident early) */
+  int32_t *status;              /* optional [B] device words, written for every sequence: 0, or UBT_STATUS_* bits
+                                   (ubt_draft_tree: NaN / +inf among the unigram logits; ubt_build_tree: among the
+                                   candidate log-probabilities it is given) */
+  int32_t validate_finite;      /* host-buffer form only: return UBT_ERR_NONFINITE if any sequence was flagged */
 } ubt_draft_opts;
 
 typedef struct ubt_verify_opts {
@@ -104,6 +116,9 @@ typedef struct ubt_verify_opts {
                           library remembers the last one of 16 streams) or one of its buffers overlaps the
                           workspace or node_pick.  In the method's real order the target logits are computed
                           FROM the drafted tree (Appendix A), so leave this 0 there. */
+  int32_t *status;     /* optional [B] device words, written for every sequence: 0, or UBT_STATUS_* bits (a NaN
+                          or +inf in one of the sequence's N target rows, used slot or not) */
+  int32_t validate_finite; /* host-buffer form only: return UBT_ERR_NONFINITE if any sequence was flagged */
 } ubt_verify_opts;
 
 typedef struct ubt_verify_result {
@@ -117,7 +132,8 @@ int ubt_version(void);
 const char *ubt_status_string(int status);
 /* Diagnostics: how many bounded device-side waits (on a bulk copy's completion) gave up since the library
  * was loaded on the current device.  0 in a healthy process; -1 if the counter cannot be read.  Results of a
- * call during which a wait gave up are undefined (but the call returned and nothing hung). */
+ * call during which a wait gave up are undefined (but the call returned and nothing hung); the sequences
+ * concerned carry UBT_STATUS_WAIT_GAVE_UP in the call's status words. */
 long long ubt_debug_ring_timeouts(void);
 
 /* Bytes of device workspace the calls below need for the given shape (0 on invalid shapes). */

@@ -38,12 +38,14 @@ class _Tree(C.Structure):
 class _DraftOpts(C.Structure):
     _fields_ = [("search_width", C.c_int32), ("depth_bonus", C.c_float), ("alpha", C.c_void_p),
                 ("lambda_", C.c_void_p), ("anchor_bigram", C.c_void_p), ("anchor_tokens", C.c_void_p),
-                ("pos_offset", C.c_void_p), ("event_between", C.c_void_p)]
+                ("pos_offset", C.c_void_p), ("event_between", C.c_void_p), ("status", C.c_void_p),
+                ("validate_finite", C.c_int32)]
 
 
 class _VerifyOpts(C.Structure):
     _fields_ = [("seed", C.c_uint64), ("temperature", C.c_float), ("node_pick", C.c_void_p),
-                ("event_before", C.c_void_p), ("event_after", C.c_void_p), ("early_start", C.c_int32)]
+                ("event_before", C.c_void_p), ("event_after", C.c_void_p), ("early_start", C.c_int32),
+                ("status", C.c_void_p), ("validate_finite", C.c_int32)]
 
 
 class _VerifyResult(C.Structure):
@@ -198,10 +200,11 @@ class VerifyResult:
 
 
 def _draft_opts(search_width=0, depth_bonus=0.0, alpha=None, lam=None, anchor_bigram=None, anchor_tokens=None,
-                pos_offset=None, event_between=None) -> _DraftOpts:
+                pos_offset=None, event_between=None, status=None, validate_finite=False) -> _DraftOpts:
     p = lambda t: None if t is None else t.data_ptr()
     return _DraftOpts(int(search_width), float(depth_bonus), p(alpha), p(lam), p(anchor_bigram), p(anchor_tokens),
-                      p(pos_offset), None if event_between is None else event_between.cuda_event)
+                      p(pos_offset), None if event_between is None else event_between.cuda_event, p(status),
+                      int(bool(validate_finite)))
 
 
 def ubt_draft_workspace_bytes(B: int, L: int, V: int, k: int, node_budget: int) -> int:
@@ -280,7 +283,7 @@ def ubt_draft_tree(unigram_logits: torch.Tensor, bigram_scores: Optional[torch.T
 def ubt_verify_tree(tree: Tree, target_logits: torch.Tensor, mode="greedy", seed: int = 0, temperature: float = 1.0,
                     node_pick: Optional[torch.Tensor] = None, result: Optional[VerifyResult] = None,
                     ws: Optional[torch.Tensor] = None, stream=None, event_before=None,
-                    event_after=None, early_start: bool = False) -> VerifyResult:
+                    event_after=None, early_start: bool = False, status: Optional[torch.Tensor] = None) -> VerifyResult:
     """Walk ``tree`` against ``target_logits[B,N,V]`` (step a4).  ``early_start``: see ``ubt_verify_opts``."""
     _need(target_logits, "target_logits")
     B, N, V = target_logits.shape
@@ -291,7 +294,8 @@ def ubt_verify_tree(tree: Tree, target_logits: torch.Tensor, mode="greedy", seed
         ws = workspace(ubt_verify_workspace_bytes(B, N, V, m), target_logits.device)
     ev = lambda e: None if e is None else C.c_void_p(e.cuda_event)
     o = _VerifyOpts(int(seed), float(temperature), None if node_pick is None else node_pick.data_ptr(),
-                    ev(event_before), ev(event_after), int(bool(early_start)))
+                    ev(event_before), ev(event_after), int(bool(early_start)),
+                    None if status is None else status.data_ptr(), 0)
     t = tree.c_struct()
     r = result.c_struct()
     _check(load().ubt_verify_tree(C.byref(t), _ptr(target_logits), _dtype_code(target_logits), V, m, C.byref(o),
@@ -323,10 +327,12 @@ def ubt_draft_tree_host(unigram_logits: torch.Tensor, bigram_scores: Optional[to
 
 def ubt_verify_tree_host(tree: Tree, target_logits: torch.Tensor, result: VerifyResult, device_buffer: torch.Tensor,
                          mode="greedy", seed: int = 0, temperature: float = 1.0,
-                         node_pick: Optional[torch.Tensor] = None, stream=None) -> VerifyResult:
+                         node_pick: Optional[torch.Tensor] = None, stream=None, status: Optional[torch.Tensor] = None,
+                         validate_finite: bool = False) -> VerifyResult:
     _need(target_logits, "target_logits", cuda=False)
     B, N, V = target_logits.shape
-    o = _VerifyOpts(int(seed), float(temperature), None if node_pick is None else node_pick.data_ptr(), None, None, 0)
+    o = _VerifyOpts(int(seed), float(temperature), None if node_pick is None else node_pick.data_ptr(), None, None, 0,
+                    None if status is None else status.data_ptr(), int(bool(validate_finite)))
     t = tree.c_struct()
     r = result.c_struct()
     _check(load().ubt_verify_tree_host(C.byref(t), _ptr(target_logits), _dtype_code(target_logits), V,

@@ -1,6 +1,7 @@
 // C ABI of libubt: argument validation, workspace carving, launches.  See include/ubt.h.
 #include <cstring>
 #include <mutex>
+#include <new>
 
 #include "ubt_internal.h"
 
@@ -92,6 +93,7 @@ static void remember_draft(cudaStream_t st, const void* logits, size_t logits_by
     add_range(d, o->anchor_bigram, (size_t)B * k * 4);
     add_range(d, o->anchor_tokens, (size_t)B * 4);
     add_range(d, o->pos_offset, (size_t)B * 4);
+    add_range(d, o->status, (size_t)B * 4);
   }
   const void* per_node[] = {t.token_ids, t.parents, t.depths, t.position_ids, t.cand_rank, t.scores};
   for (const void* p : per_node) add_range(d, p, bn * 4);
@@ -137,6 +139,7 @@ const char* ubt_status_string(int status) {
     case UBT_ERR_WORKSPACE: return "workspace missing or too small";
     case UBT_ERR_CUDA: return "CUDA call or launch failed";
     case UBT_ERR_STATIC_SCRATCH: return "request exceeds the built-in scratch of ubt_verify_tree_static";
+    case UBT_ERR_NONFINITE: return "NaN or +inf among the logits";
     default: return "unknown status";
   }
 }
@@ -187,7 +190,7 @@ int ubt_build_tree(const float* bigram_scores, int B, int L, int k, int N, const
   remember_draft(static_cast<cudaStream_t>(cuda_stream), nullptr, 0, bigram_scores, B, L, k, N, o, *out, nullptr, 0);
   cudaError_t e = launch_build_tree(bigram_scores, B, L, k, N, o->search_width, o->depth_bonus, o->alpha, o->lambda,
                                     o->anchor_bigram, o->anchor_tokens, o->pos_offset, *out, no_merge_parts(), 0,
-                                    static_cast<cudaStream_t>(cuda_stream));
+                                    o->status, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? UBT_OK : UBT_ERR_CUDA;
 }
 
@@ -242,7 +245,8 @@ int ubt_draft_tree(const void* unigram_logits, int dtype, const float* bigram_sc
   if (o->event_between && cudaEventRecord(static_cast<cudaEvent_t>(o->event_between), st) != cudaSuccess)
     return UBT_ERR_CUDA;
   cudaError_t e = launch_build_tree(bigram_scores, B, L, k, N, o->search_width, o->depth_bonus, o->alpha, o->lambda,
-                                    o->anchor_bigram, o->anchor_tokens, o->pos_offset, *out, merge_parts(w), V, st);
+                                    o->anchor_bigram, o->anchor_tokens, o->pos_offset, *out, merge_parts(w), V,
+                                    o->status, st);
   return e == cudaSuccess ? UBT_OK : UBT_ERR_CUDA;
 }
 
@@ -258,7 +262,7 @@ int ubt_verify_tree(const ubt_tree* tree, const void* target_logits, int dtype, 
   const int B = tree->B, N = tree->N, L = tree->L;
   if (B < 0 || N < 1 || L < 1) return UBT_ERR_INVALID_ARG;
   if (N > kMaxN || L > kMaxL) return UBT_ERR_UNSUPPORTED;
-  const ubt_verify_opts d{0, 1.0f, nullptr, nullptr, nullptr, 0};
+  const ubt_verify_opts d{0, 1.0f, nullptr, nullptr, nullptr, 0, nullptr, 0};
   const ubt_verify_opts* o = opts ? opts : &d;
   if (mode == UBT_VERIFY_SAMPLE) {
     if (!(o->temperature > 0.0f)) return UBT_ERR_INVALID_ARG;
@@ -289,7 +293,7 @@ int ubt_verify_tree(const ubt_tree* tree, const void* target_logits, int dtype, 
   }
   if (o->event_after && cudaEventRecord(static_cast<cudaEvent_t>(o->event_after), st) != cudaSuccess)
     return UBT_ERR_CUDA;
-  if (launch_walk(*tree, mode, w, V, sampled, o->node_pick, *out, st) != cudaSuccess) return UBT_ERR_CUDA;
+  if (launch_walk(*tree, mode, w, V, sampled, o->node_pick, *out, o->status, st) != cudaSuccess) return UBT_ERR_CUDA;
   return UBT_OK;
 }
 
@@ -321,7 +325,7 @@ struct DeviceTree {
 };
 
 struct DraftHostLayout {
-  void* logits; float* bigram; float *alpha, *lambda, *anchor_bigram; int32_t *anchor_tokens, *pos_offset;
+  void* logits; float* bigram; float *alpha, *lambda, *anchor_bigram; int32_t *anchor_tokens, *pos_offset, *status;
   DeviceTree tree; void* ws; size_t ws_bytes; size_t total;
   DraftHostLayout(void* buf, int B, int L, int V, int k, int N, int dtype) {
     Carver c{static_cast<unsigned char*>(buf)};
@@ -330,6 +334,7 @@ struct DraftHostLayout {
     alpha = c.take<float>((size_t)L); lambda = c.take<float>((size_t)L);
     anchor_bigram = c.take<float>((size_t)B * k);
     anchor_tokens = c.take<int32_t>((size_t)B); pos_offset = c.take<int32_t>((size_t)B);
+    status = c.take<int32_t>((size_t)B);
     tree.carve(c, B, L, k, N, true);
     ws_bytes = ubt_draft_workspace_bytes(B, L, V, k, N);
     ws = c.take<unsigned char>(ws_bytes);
@@ -338,7 +343,7 @@ struct DraftHostLayout {
 };
 
 struct VerifyHostLayout {
-  void* logits; DeviceTree tree; int32_t *accepted_len, *bonus, *accepted_nodes, *out_tokens, *node_pick;
+  void* logits; DeviceTree tree; int32_t *accepted_len, *bonus, *accepted_nodes, *out_tokens, *node_pick, *status;
   void* ws; size_t ws_bytes; size_t total;
   VerifyHostLayout(void* buf, int B, int L, int N, int V, int dtype, int mode) {
     Carver c{static_cast<unsigned char*>(buf)};
@@ -347,6 +352,7 @@ struct VerifyHostLayout {
     accepted_len = c.take<int32_t>((size_t)B); bonus = c.take<int32_t>((size_t)B);
     accepted_nodes = c.take<int32_t>((size_t)B * (L + 1)); out_tokens = c.take<int32_t>((size_t)B * (L + 1));
     node_pick = c.take<int32_t>((size_t)B * N);
+    status = c.take<int32_t>((size_t)B);
     ws_bytes = ubt_verify_workspace_bytes(B, N, V, mode);
     ws = c.take<unsigned char>(ws_bytes);
     total = c.off;
@@ -354,6 +360,29 @@ struct VerifyHostLayout {
 };
 
 #define UBT_CUDA_OK(call) do { if ((call) != cudaSuccess) { cudaGetLastError(); return UBT_ERR_CUDA; } } while (0)
+
+// End of a host-buffer call: copy the status words back if anybody wants them, wait for the stream, and turn
+// flagged sequences into a return code when the caller asked for validation.
+int finish_host_call(cudaStream_t st, const int32_t* dev_status, int32_t* host_status, bool validate, int B) {
+  int32_t local[64];
+  int32_t* dst = host_status;
+  int32_t* heap = nullptr;
+  if (!dst && validate) dst = B <= 64 ? local : (heap = new (std::nothrow) int32_t[(size_t)B]);
+  if ((host_status || validate) && !dst) return UBT_ERR_CUDA;
+  int rc = UBT_OK;
+  if (dst && cudaMemcpyAsync(dst, dev_status, sizeof(int32_t) * (size_t)B, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    rc = UBT_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) rc = UBT_ERR_CUDA;
+  if (rc == UBT_OK && validate) {
+    int bits = 0;
+    for (int b = 0; b < B; ++b) bits |= dst[b];
+    if (bits & UBT_STATUS_WAIT_GAVE_UP) rc = UBT_ERR_CUDA;
+    else if (bits & UBT_STATUS_NONFINITE) rc = UBT_ERR_NONFINITE;
+  }
+  delete[] heap;
+  if (rc != UBT_OK) cudaGetLastError();
+  return rc;
+}
 }  // namespace
 
 extern "C" {
@@ -399,6 +428,9 @@ int ubt_draft_tree_host(const void* unigram_logits, int dtype, const float* bigr
     if (opts->pos_offset) { UBT_CUDA_OK(cudaMemcpyAsync(d.pos_offset, opts->pos_offset, sizeof(int32_t) * B, cudaMemcpyHostToDevice, st)); dev_opts.pos_offset = d.pos_offset; }
     dev_opts.event_between = opts->event_between;
   }
+  int32_t* host_status = opts ? opts->status : nullptr;  // a HOST array in this form
+  const bool validate = opts && opts->validate_finite;
+  dev_opts.status = (host_status || validate) ? d.status : nullptr;
   rc = ubt_draft_tree(d.logits, dtype, L > 1 ? d.bigram : nullptr, B, L, V, k, N, &dev_opts, &d.tree.t, d.ws,
                       d.ws_bytes, cuda_stream);
   if (rc) return rc;
@@ -411,8 +443,7 @@ int ubt_draft_tree_host(const void* unigram_logits, int dtype, const float* bigr
       {out->cand_ids, t.cand_ids, (size_t)B * L * k * 4}, {out->cand_logprob, t.cand_logprob, (size_t)B * L * k * 4}};
   for (auto& c : copies)
     if (c.dst) UBT_CUDA_OK(cudaMemcpyAsync(c.dst, c.src, c.bytes, cudaMemcpyDeviceToHost, st));
-  UBT_CUDA_OK(cudaStreamSynchronize(st));
-  return UBT_OK;
+  return finish_host_call(st, d.status, host_status, validate, B);
 }
 
 int ubt_verify_tree_host(const ubt_tree* tree, const void* target_logits, int dtype, int V, int mode,
@@ -437,9 +468,12 @@ int ubt_verify_tree_host(const ubt_tree* tree, const void* target_logits, int dt
   UBT_CUDA_OK(cudaMemcpyAsync(d.tree.t.token_ids, tree->token_ids, bn * 4, cudaMemcpyHostToDevice, st));
   UBT_CUDA_OK(cudaMemcpyAsync(d.tree.t.parents, tree->parents, bn * 4, cudaMemcpyHostToDevice, st));
   UBT_CUDA_OK(cudaMemcpyAsync(d.tree.t.n_nodes, tree->n_nodes, (size_t)B * 4, cudaMemcpyHostToDevice, st));
-  ubt_verify_opts dev_opts{0, 1.0f, nullptr, nullptr, nullptr, 0};
+  ubt_verify_opts dev_opts{0, 1.0f, nullptr, nullptr, nullptr, 0, nullptr, 0};
   if (opts) { dev_opts = *opts; }
   dev_opts.early_start = 0;  // the logits are copied in just before: nothing to start ahead of
+  int32_t* host_status = dev_opts.status;  // a HOST array in this form
+  const bool validate = dev_opts.validate_finite != 0;
+  dev_opts.status = (host_status || validate) ? d.status : nullptr;
   int32_t* host_pick = dev_opts.node_pick;
   dev_opts.node_pick = host_pick ? d.node_pick : nullptr;
   ubt_verify_result r{d.accepted_len, d.bonus, d.accepted_nodes, d.out_tokens};
@@ -450,8 +484,7 @@ int ubt_verify_tree_host(const ubt_tree* tree, const void* target_logits, int dt
   UBT_CUDA_OK(cudaMemcpyAsync(out->accepted_nodes, d.accepted_nodes, (size_t)B * (L + 1) * 4, cudaMemcpyDeviceToHost, st));
   UBT_CUDA_OK(cudaMemcpyAsync(out->out_tokens, d.out_tokens, (size_t)B * (L + 1) * 4, cudaMemcpyDeviceToHost, st));
   if (host_pick) UBT_CUDA_OK(cudaMemcpyAsync(host_pick, d.node_pick, bn * 4, cudaMemcpyDeviceToHost, st));
-  UBT_CUDA_OK(cudaStreamSynchronize(st));
-  return UBT_OK;
+  return finish_host_call(st, d.status, host_status, validate, B);
 }
 
 }  // extern "C"

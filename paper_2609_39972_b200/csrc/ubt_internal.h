@@ -96,7 +96,7 @@ size_t tree_smem_bytes(int L, int k, int N);
 cudaError_t launch_build_tree(const float* bigram, int B, int L, int k, int N, int W, float zeta,
                               const float* alpha, const float* lambda, const float* anchor_bigram,
                               const int32_t* anchor_tokens, const int32_t* pos_offset,
-                              const ubt_tree& out, const MergeParts& parts, int V, cudaStream_t st);
+                              const ubt_tree& out, const MergeParts& parts, int V, int32_t* status, cudaStream_t st);
 cudaError_t launch_build_mask(const ubt_tree& tree, const int32_t* pos_offset, cudaStream_t st);
 
 // ---- a4 ---------------------------------------------------------------------------------------
@@ -121,6 +121,6 @@ cudaError_t launch_row_sample(const void* logits, int dtype, int B, int N, int V
                               cudaStream_t st);
 cudaError_t launch_walk(const ubt_tree& tree, int mode, const VerifyWorkspace& w, int V,
                         const int32_t* sampled_pick, int32_t* node_pick,
-                        const ubt_verify_result& out, cudaStream_t st);
+                        const ubt_verify_result& out, int32_t* status, cudaStream_t st);
 
 }  // namespace ubt

@@ -15,10 +15,16 @@ struct MergeParts {
   const int32_t* part_cnt;  // [rows, smax]
 };
 
-// Every lane of one warp calls this for the same row.  Writes cand_ids[row, 0..k) (best first) and
+// Status bits of a sequence (ubt_draft_opts.status / ubt_verify_opts.status).
+constexpr int kStatusNonFinite = 1;  // a NaN or +inf among the logits
+constexpr int kStatusWaitGaveUp = 2; // a bounded device-side wait gave up: results undefined
+
+// Every lane of one warp calls this for the same row; returns the row's status bits (all lanes agree): the
+// log-sum-exp of a row that holds a NaN or +inf is not finite, and a segment whose streaming CTA gave up a wait
+// carries the count -1.  Writes cand_ids[row, 0..k) (best first) and
 // cand_lp[row, r] = value - log-sum-exp of the whole row; sm_ids / sm_lp, if given, receive a copy of the row's k
 // entries (the caller's shared-memory staging).
-__device__ __forceinline__ void merge_row_warp(const MergeParts& p, int64_t rows, int64_t row, int V, int k,
+__device__ __forceinline__ int merge_row_warp(const MergeParts& p, int64_t rows, int64_t row, int V, int k,
                                                int32_t* __restrict__ cand_ids_, float* __restrict__ cand_lp_,
                                                int lane, int* sm_ids = nullptr, float* sm_lp = nullptr) {
   const long long nslots = rows * p.plan.smax;
@@ -45,7 +51,7 @@ __device__ __forceinline__ void merge_row_warp(const MergeParts& p, int64_t rows
       const int j = q / k, i = q - j * k;
       pi[c] = i;
       if (q < nq) {
-        pcnt[c] = part_cnt[base + j];
+        pcnt[c] = part_cnt[base + j];  // -1: the CTA of this segment gave up (no entry passes the mask below)
         val[c] = part_val[(base + j) * k + i];   // slots beyond the count hold stale data: masked below
         pidx[c] = part_idx[(base + j) * k + i];
       }
@@ -92,7 +98,7 @@ __device__ __forceinline__ void merge_row_warp(const MergeParts& p, int64_t rows
     // found by binary search.
     for (int q = lane; q < nq; q += 32) {
       const int j = q / k, i = q - j * k;
-      if (i >= part_cnt[base + j]) continue;
+      if (i >= part_cnt[base + j]) continue;  // also skips a segment that gave up (count -1)
       const float val = part_val[(base + j) * k + i];
       const int idx = part_idx[(base + j) * k + i];
       const uint64_t key = make_key(val, idx);
@@ -100,6 +106,7 @@ __device__ __forceinline__ void merge_row_warp(const MergeParts& p, int64_t rows
       for (int j2 = 0; j2 < nseg && rank < k; ++j2) {
         if (j2 == j) continue;
         int lo = 0, hi = part_cnt[base + j2];  // list[0..lo) > key, list[hi..) < key
+        hi = hi < 0 ? 0 : hi;
         while (lo < hi) {
           const int mid = (lo + hi) >> 1;
           if (make_key(part_val[(base + j2) * k + mid], part_idx[(base + j2) * k + mid]) > key) lo = mid + 1;
@@ -114,14 +121,21 @@ __device__ __forceinline__ void merge_row_warp(const MergeParts& p, int64_t rows
       }
     }
   }
-  for (int j = lane; j < nseg; j += 32) found += part_cnt[base + j];
+  int gave_up = 0;
+  for (int j = lane; j < nseg; j += 32) {
+    const int c = part_cnt[base + j];
+    gave_up |= c < 0;
+    found += c < 0 ? 0 : c;
+  }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) found += __shfl_xor_sync(FULL, found, o);
+  gave_up = __any_sync(FULL, gave_up);
   for (int r = found + lane; r < k; r += 32) {  // fewer than k entries above -inf: documented as unsupported
     cand_ids[row * k + r] = -1;
     cand_lp[row * k + r] = -INFINITY;
     if (sm_ids) { sm_ids[r] = -1; sm_lp[r] = -INFINITY; }
   }
+  return ((lse == lse && lse < INFINITY) ? 0 : kStatusNonFinite) | (gave_up ? kStatusWaitGaveUp : 0);
 }
 
 }  // namespace ubt

@@ -63,7 +63,7 @@ extern "C" int ubt_verify_tree_static(const ubt_tree* tree, const void* target_l
   if (launch_row_argmax(target_logits, dtype, rows, V, w, tree_smem_bytes(tree->L, tree->k, tree->N), false, st) !=
       cudaSuccess)
     return UBT_ERR_CUDA;
-  if (launch_walk(*tree, UBT_VERIFY_GREEDY, w, V, nullptr, node_pick, *out, st) != cudaSuccess) return UBT_ERR_CUDA;
+  if (launch_walk(*tree, UBT_VERIFY_GREEDY, w, V, nullptr, node_pick, *out, nullptr, st) != cudaSuccess) return UBT_ERR_CUDA;
   return UBT_OK;
 }
 

@@ -577,7 +577,17 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
     pos += sg.len;
   }
   __syncthreads();
-  if (tid == 0 && *reinterpret_cast<volatile int*>(&sh.fail)) prod.drain(consumed > 0 ? consumed - 1 : 0, full);
+  if (tid == 0 && *reinterpret_cast<volatile int*>(&sh.fail)) {
+    prod.drain(consumed > 0 ? consumed - 1 : 0, full);
+    // a wait gave up: mark every segment of this span (written or not) so that the merge reports it
+    for (int64_t pos = lo; pos < hi;) {
+      Segment sg;
+      sg.at(pos, hi, V);
+      const int64_t c_first = (sg.row * (int64_t)V) / plan.span;
+      g_cnt[sg.row * plan.smax + ((int64_t)blockIdx.x - c_first)] = -1;
+      pos += sg.len;
+    }
+  }
 }
 
 // One warp per row: combine the partials of the row's segments (see merge_row_warp in ubt_merge.cuh).

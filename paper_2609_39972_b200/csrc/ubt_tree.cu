@@ -46,7 +46,7 @@ struct TreeSmem {
   Span<int> depth_off;      // [L+2]
   Span<int> x_fill;         // [L+2] fill counters of the grouping by depth
   Span<uint32_t> maskrow;   // [N, mask_words]
-  Span<int> scalars;        // [0] = accepted count, [1] = threshold key of a round, [2] = flags
+  Span<int> scalars;        // [0] accepted count, [1]-[3] scratch of the expansion, [4] status bits of the sequence
   // Nodes enumerated by the parallel expansion (resident table only; see expand_rounds): node 0 is the root.
   int xcap;                 // capacity (0 in lazy mode)
   Span<short> x_parent;     // [xcap] enumerated parent, -1 for the root
@@ -95,7 +95,7 @@ inline TreeLayout tree_layout(int L, int k, int N) {
   o.nd_pk = take(sizeof(unsigned long long) * 2 * N); o.kk = take(sizeof(int) * N);
   o.depth_cnt = take(sizeof(int) * (L + 2)); o.depth_off = take(sizeof(int) * (L + 2));
   o.x_fill = take(sizeof(int) * (L + 2));
-  o.maskrow = take(sizeof(uint32_t) * N * mw); o.scalars = take(sizeof(int) * 4);
+  o.maskrow = take(sizeof(uint32_t) * N * mw); o.scalars = take(sizeof(int) * 8);
   const int xcap = lazy ? 0 : expand_capacity(N);
   o.xcap = xcap;
   o.x_parent = take(sizeof(short) * xcap); o.x_depth = take(xcap); o.x_rank = take(xcap); o.x_next = take(xcap);
@@ -141,7 +141,7 @@ __device__ __forceinline__ void tree_bind(TreeSmem* s, unsigned char* base, cons
   s->depth_off = Span<int>((int*)(base + o.depth_off), L + 2, 117);
   s->x_fill = Span<int>((int*)(base + o.x_fill), L + 2, 131);
   s->maskrow = Span<uint32_t>((uint32_t*)(base + o.maskrow), (long long)N * mw, 118);
-  s->scalars = Span<int>((int*)(base + o.scalars), 4, 119);
+  s->scalars = Span<int>((int*)(base + o.scalars), 8, 119);
 }
 
 size_t tree_smem_bytes(int L, int k, int N) { return tree_layout(L, k, N).total; }
@@ -873,7 +873,7 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
              const float* __restrict__ alpha, const float* __restrict__ lambda,
              const float* __restrict__ anchor_bigram, const int32_t* __restrict__ anchor_tokens,
              const int32_t* __restrict__ pos_offset, ubt_tree out, MergeParts parts, int V,
-             const __grid_constant__ TreeLayout lay) {
+             int32_t* __restrict__ status, const __grid_constant__ TreeLayout lay) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   TreeSmem s;
   tree_bind(&s, smem_raw, lay, L, k, N);
@@ -901,6 +901,7 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
     s.al[i] = alpha ? alpha[i] : 1.f;
     s.la[i] = lambda ? lambda[i] : 1.f;
   }
+  if (tid == 0) s.scalars[4] = 0;
   if constexpr (lazy) {
     for (int i = tid; i < L * k + 1; i += G2_T) s.rowmap[i] = (short)-1;
   } else {
@@ -927,13 +928,17 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   // ---- step a1's last part when fused: merge the row partials of this sequence's L rows (one warp per row; the
   // candidates go to global memory and to the shared-memory staging at once); otherwise stage the candidates
   if (parts.part_ms != nullptr) {
-    for (int i = tid >> 5; i < L; i += G2_T / 32)
-      merge_row_warp(parts, nB * L, (int64_t)b * L + i, V, k, out.cand_ids, out.cand_logprob, lane,
-                     s.tok.ptr((long long)i * k, k), s.lp.ptr((long long)i * k, k));
+    for (int i = tid >> 5; i < L; i += G2_T / 32) {
+      const int bits = merge_row_warp(parts, nB * L, (int64_t)b * L + i, V, k, out.cand_ids, out.cand_logprob, lane,
+                                      s.tok.ptr((long long)i * k, k), s.lp.ptr((long long)i * k, k));
+      if (bits && lane == 0) atomicOr(&s.scalars[4], bits);
+    }
   } else {
     for (int i = tid; i < L * k; i += G2_T) {
-      s.lp[i] = g_lp[(int64_t)b * L * k + i];
+      const float lpv = g_lp[(int64_t)b * L * k + i];
+      s.lp[i] = lpv;
       s.tok[i] = g_ids[(int64_t)b * L * k + i];
+      if (!(lpv <= 0.f || lpv > 0.f) || lpv == INFINITY) atomicOr(&s.scalars[4], kStatusNonFinite);
     }
   }
   int kp = 1;
@@ -1172,6 +1177,7 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
     g_par[o] = -1; g_dep[o] = 0; g_rk[o] = -1; g_pos[o] = poff;
     g_sc[o] = 0.f; g_nn[b] = n_acc + 1;
     s.maskrow[0] = 1u;
+    if (status) status[b] = s.scalars[4];
   }
   if (tid < n_acc) {
     const int sl = s.nd_slot[tid], p = s.nd_parent[tid], d = s.nd_depth[tid], r = s.nd_rank[tid];
@@ -1224,7 +1230,7 @@ k_build_mask(ubt_tree tree, const int32_t* __restrict__ pos_offset) {
 cudaError_t launch_build_tree(const float* bigram, int B, int L, int k, int N, int W, float zeta,
                               const float* alpha, const float* lambda, const float* anchor_bigram,
                               const int32_t* anchor_tokens, const int32_t* pos_offset,
-                              const ubt_tree& out, const MergeParts& parts, int V, cudaStream_t st) {
+                              const ubt_tree& out, const MergeParts& parts, int V, int32_t* status, cudaStream_t st) {
   if (B == 0) return cudaSuccess;
   const TreeLayout lay = tree_layout(L, k, N);
   const size_t smem = lay.total;
@@ -1234,7 +1240,7 @@ cudaError_t launch_build_tree(const float* bigram, int B, int L, int k, int N, i
   if (e != cudaSuccess) return e;
   // programmatic launch only when the kernel before it is this library's own streaming kernel
   return launch_kernel(kern, dim3(B), dim3(G2_T), smem, st, parts.part_ms != nullptr, bigram, L, k, N, W,
-                       zeta, alpha, lambda, anchor_bigram, anchor_tokens, pos_offset, out, parts, V, lay);
+                       zeta, alpha, lambda, anchor_bigram, anchor_tokens, pos_offset, out, parts, V, status, lay);
 }
 
 cudaError_t launch_build_mask(const ubt_tree& tree, const int32_t* pos_offset, cudaStream_t st) {

@@ -21,6 +21,21 @@ namespace ubt {
 constexpr int G4_T = 512;
 constexpr int G4_U = 4;
 
+// A NaN among the logits must not go unnoticed, so the maxima below let NaN win: a fragment that holds one has
+// the maximum NaN, fails every "<=" and ">" test, and is reported through a marker key instead of a pick.
+__device__ __forceinline__ float max_nan(float a, float b) {
+  float d;
+  asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+  return d;
+}
+// Keys above the key of +inf never stand for a value: the first marks a row segment that holds a NaN, the
+// second a segment whose CTA gave up a bounded wait.  The walk kernel turns them into status bits; the token
+// they decode to is in range, so whatever follows stays memory-safe.
+constexpr unsigned long long kKeyPlusInf = 0xff800000ull << 32;
+constexpr unsigned long long kKeyNaNSeen = (0xffc00000ull << 32) | 0xffffffffull;
+constexpr unsigned long long kKeyGaveUp = ~0ull;
+
+
 template <typename T, int VEC>
 __device__ __forceinline__ void load_row_frag(const T* seg, int nfrag, int i, uint4& raw, float& sc) {
   if constexpr (VEC == 1) {
@@ -69,6 +84,7 @@ k_row_argmax(const T* __restrict__ logits, int64_t total, int V, SpanPlan plan,
     // Baseline (-inf, the thread's first column): true if all its elements are -inf, replaced otherwise.
     float best = -INFINITY;
     int bcol = c0 + tid * VEC;
+    bool saw_nan = false;
     const bool has = tid < nfrag;
     uint4 cur[G4_U], nxt[G4_U];
     float curs[G4_U], nxts[G4_U];
@@ -86,7 +102,8 @@ k_row_argmax(const T* __restrict__ logits, int64_t total, int V, SpanPlan plan,
         frag_values<T, VEC>(cur[u], curs[u], x);
         float vmax = x[0];
 #pragma unroll
-        for (int j = 1; j < VEC; ++j) vmax = fmaxf(vmax, x[j]);
+        for (int j = 1; j < VEC; ++j) vmax = max_nan(vmax, x[j]);
+        saw_nan = saw_nan || vmax != vmax;
         if (vmax > best) {  // columns ascend within a thread: strict > keeps the lowest token
           const int col0 = c0 + (base + u * G4_T + tid) * VEC;
 #pragma unroll
@@ -98,6 +115,7 @@ k_row_argmax(const T* __restrict__ logits, int64_t total, int V, SpanPlan plan,
       for (int u = 0; u < G4_U; ++u) { cur[u] = nxt[u]; curs[u] = nxts[u]; }
     }
     unsigned long long key = has ? make_key(best, bcol) : 0ull;
+    key = saw_nan ? kKeyNaNSeen : key;
     key = warp_max_u64(key);
     __syncthreads();
     if (lane == 0) red[tid >> 5] = key;
@@ -114,16 +132,16 @@ k_row_argmax(const T* __restrict__ logits, int64_t total, int V, SpanPlan plan,
 // ---------------------------------------------------------------------------- greedy picks, ring-fed
 // Fragment maximum without widening: packed bf16 max of the four words, then the two halves.
 __device__ __forceinline__ float frag_max(const uint4& v, const __nv_bfloat16*) {
-  const __nv_bfloat162 a = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&v.x),
-                                   *reinterpret_cast<const __nv_bfloat162*>(&v.y));
-  const __nv_bfloat162 b = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&v.z),
-                                   *reinterpret_cast<const __nv_bfloat162*>(&v.w));
-  const __nv_bfloat162 c = __hmax2(a, b);
+  const __nv_bfloat162 a = __hmax2_nan(*reinterpret_cast<const __nv_bfloat162*>(&v.x),
+                                       *reinterpret_cast<const __nv_bfloat162*>(&v.y));
+  const __nv_bfloat162 b = __hmax2_nan(*reinterpret_cast<const __nv_bfloat162*>(&v.z),
+                                       *reinterpret_cast<const __nv_bfloat162*>(&v.w));
+  const __nv_bfloat162 c = __hmax2_nan(a, b);
   const uint32_t w = *reinterpret_cast<const uint32_t*>(&c);
-  return fmaxf(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+  return max_nan(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
 }
 __device__ __forceinline__ float frag_max(const uint4& v, const float*) {
-  return fmaxf(fmaxf(__uint_as_float(v.x), __uint_as_float(v.y)), fmaxf(__uint_as_float(v.z), __uint_as_float(v.w)));
+  return max_nan(max_nan(__uint_as_float(v.x), __uint_as_float(v.y)), max_nan(__uint_as_float(v.z), __uint_as_float(v.w)));
 }
 
 // One CTA per SM; the span's chunks arrive through the shared-memory ring (ubt_ring.cuh).
@@ -182,9 +200,11 @@ k_row_argmax_ring(const T* __restrict__ logits, int64_t total, int V, SpanPlan p
     sg.at(pos, hi, V);
     float best = -INFINITY, wthr = -INFINITY;  // wthr: warp-uniform threshold, -inf = none yet
     int bcol = -1;
+    bool saw_nan = false;
     // One fragment against the threshold; every lane of the warp must call it (it votes).
     auto visit = [&](const uint4& v, float fm, int col) {
       const bool beat = fm > wthr;
+      saw_nan = saw_nan || fm != fm;
       if (__any_sync(FULL, beat)) {
         if (beat) {
           Frag<T> x;
@@ -217,7 +237,7 @@ k_row_argmax_ring(const T* __restrict__ logits, int64_t total, int V, SpanPlan p
           for (int u = 0; u < 4; ++u) v[u] = stage[f0 + u * THREADS];
 #pragma unroll
           for (int u = 0; u < 4; ++u) fm[u] = frag_max(v[u], (const T*)nullptr);
-          if (__any_sync(FULL, fmaxf(fmaxf(fm[0], fm[1]), fmaxf(fm[2], fm[3])) > wthr)) {
+          if (__any_sync(FULL, !(max_nan(max_nan(fm[0], fm[1]), max_nan(fm[2], fm[3])) <= wthr))) {
 #pragma unroll
             for (int u = 0; u < 4; ++u) visit(v[u], fm[u], colbase + (f0 + u * THREADS) * VEC);
           }
@@ -238,6 +258,7 @@ k_row_argmax_ring(const T* __restrict__ logits, int64_t total, int V, SpanPlan p
     }
     if (failed) break;
     unsigned long long key = bcol >= 0 ? make_key(best, bcol) : 0ull;
+    key = saw_nan ? kKeyNaNSeen : key;
     key = warp_max_u64(key);
     if (lane == 0) red[tid >> 5] = key;
     if (tid == 0) s_thr[0] = s_thr[1] = 0u;  // nobody touches them between the two barriers
@@ -251,7 +272,16 @@ k_row_argmax_ring(const T* __restrict__ logits, int64_t total, int V, SpanPlan p
     pos += sg.len;
   }
   __syncthreads();
-  if (tid == 0 && *reinterpret_cast<volatile int*>(&s_fail)) prod.drain(consumed > 0 ? consumed - 1 : 0, full);
+  if (tid == 0 && *reinterpret_cast<volatile int*>(&s_fail)) {
+    prod.drain(consumed > 0 ? consumed - 1 : 0, full);
+    for (int64_t pos = lo; pos < hi;) {  // a wait gave up: mark every segment of this span for the walk
+      Segment sg;
+      sg.at(pos, hi, V);
+      const int64_t c_first = (sg.row * (int64_t)V) / plan.span;
+      part_key[sg.row * plan.smax + ((int64_t)blockIdx.x - c_first)] = kKeyGaveUp;
+      pos += sg.len;
+    }
+  }
   // An early start must not become an early finish: the walk behind this kernel waits for THIS grid only, so
   // this grid may not complete before the kernel in front of it (the tree builder) has.
   if (early && tid == 0) pdl_wait();
@@ -479,7 +509,7 @@ k_row_weights_ring(const T* __restrict__ logits, int64_t rows, int V, float temp
         const uint4* stage = reinterpret_cast<const uint4*>(ring + (size_t)rp.stage * G5R_STAGE_BYTES);
         const int nfrag = l / VEC;
 #pragma unroll 4
-        for (int f = tid; f < nfrag; f += G5R_T) m = fmaxf(m, frag_max(stage[f], (const T*)nullptr));
+        for (int f = tid; f < nfrag; f += G5R_T) m = max_nan(m, frag_max(stage[f], (const T*)nullptr));
       } else {
         s_fail = 1;
       }
@@ -489,12 +519,12 @@ k_row_weights_ring(const T* __restrict__ logits, int64_t rows, int V, float temp
     }
     if (failed) break;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(FULL, m, o));
+    for (int o = 16; o > 0; o >>= 1) m = max_nan(m, __shfl_xor_sync(FULL, m, o));
     if (lane == 0) redf[warp] = m;
     __syncthreads();
     m = redf[0];
-    for (int w = 1; w < G5R_T / 32; ++w) m = fmaxf(m, redf[w]);
-    const float c = -__fmul_rn(m, a);
+    for (int w = 1; w < G5R_T / 32; ++w) m = max_nan(m, redf[w]);
+    const float c = -__fmul_rn(m, a);  // NaN / -inf for a row that holds a NaN / +inf: the pick kernel reports it
     if (tid == 0) { row_ac[row * 2] = a; row_ac[row * 2 + 1] = c; }
     WeightConsts2 wc;
     wc.init(a, c);
@@ -541,7 +571,10 @@ k_row_weights_ring(const T* __restrict__ logits, int64_t rows, int V, float temp
     }
   }
   __syncthreads();
-  if (tid == 0 && *reinterpret_cast<volatile int*>(&s_fail)) prod.drain(consumed > 0 ? consumed - 1 : 0, full);
+  if (tid == 0 && *reinterpret_cast<volatile int*>(&s_fail)) {
+    prod.drain(consumed > 0 ? consumed - 1 : 0, full);
+    for (int64_t row = r0; row < r1; ++row) row_ac[row * 2] = -1.0f;  // a wait gave up: no scale is negative
+  }
   if (early && tid == 0) pdl_wait();  // started early: do not complete before the kernel in front
 }
 
@@ -556,8 +589,12 @@ k_row_pick(const T* __restrict__ logits, int64_t rows, int N, int V, uint64_t se
   pdl_wait();
   pdl_launch_dependents();
   if (row >= rows) return;
-  const int ans = locate_pick<T>(logits + row * V, V, row_ac[row * 2], row_ac[row * 2 + 1],
-                                 block_sum + row * nblocks, nblocks, seed, (uint32_t)(row / N), (uint32_t)(row % N), lane);
+  const float a = row_ac[row * 2], c = row_ac[row * 2 + 1];
+  int ans;
+  if (a < 0.f) ans = -2;                                   // the weights kernel gave up a wait on this row
+  else if (!(c == c) || c == INFINITY || c == -INFINITY) ans = -1;  // row maximum NaN or +inf (c = -max * a)
+  else ans = locate_pick<T>(logits + row * V, V, a, c, block_sum + row * nblocks, nblocks, seed, (uint32_t)(row / N),
+                            (uint32_t)(row % N), lane);
   if (lane == 0) pick[row] = ans;
 }
 
@@ -587,15 +624,20 @@ k_row_sample(const T* __restrict__ logits, int64_t rows, int N, int V, uint64_t 
       float x[VEC];
       frag_values<T, VEC>(raw, sc, x);
 #pragma unroll
-      for (int j = 0; j < VEC; ++j) m = fmaxf(m, x[j]);
+      for (int j = 0; j < VEC; ++j) m = max_nan(m, x[j]);
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(FULL, m, o));
+    for (int o = 16; o > 0; o >>= 1) m = max_nan(m, __shfl_xor_sync(FULL, m, o));
     __syncthreads();
     if (lane == 0) redf[warp] = m;
     __syncthreads();
     m = redf[0];
-    for (int w = 1; w < G5_T / 32; ++w) m = fmaxf(m, redf[w]);
+    for (int w = 1; w < G5_T / 32; ++w) m = max_nan(m, redf[w]);
+    if (!(m == m) || m == INFINITY) {  // a NaN or +inf in the row: no pick, reported by the walk
+      if (tid == 0) pick[row] = -1;
+      __syncthreads();
+      continue;
+    }
     const float inv_t = __fdiv_rn(1.0f, temperature);
     const float a = __fmul_rn(0x1.715476p+0f, inv_t);
     const float c = -__fmul_rn(m, a);
@@ -632,13 +674,17 @@ k_row_sample(const T* __restrict__ logits, int64_t rows, int N, int V, uint64_t 
 // One CTA per sequence: gather the picks of its N slots, then warp 0 walks from the root.
 __global__ void __launch_bounds__(128)
 k_walk(ubt_tree tree, int mode, SpanPlan plan, const unsigned long long* __restrict__ part_key, int V,
-       const int32_t* __restrict__ sampled_pick, int32_t* __restrict__ node_pick, ubt_verify_result out) {
+       const int32_t* __restrict__ sampled_pick, int32_t* __restrict__ node_pick, ubt_verify_result out,
+       int32_t* __restrict__ status) {
   __shared__ int s_pick[kMaxN], s_tok[kMaxN], s_par[kMaxN];
+  __shared__ int s_bits;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, N = tree.N, L = tree.L;
   const int64_t o = (int64_t)b * N;
+  if (tid == 0) s_bits = 0;
   pdl_wait();  // picks and tree come from the kernels before this one
+  __syncthreads();
   for (int n = tid; n < N; n += blockDim.x) {
-    int p;
+    int p, bits = 0;
     if (mode == UBT_VERIFY_GREEDY) {
       const int64_t row = o + n;
       const int64_t c_first = (row * (int64_t)V) / plan.span;
@@ -648,10 +694,14 @@ k_walk(ubt_tree tree, int mode, SpanPlan plan, const unsigned long long* __restr
         const unsigned long long key = part_key[row * plan.smax + j];
         best = key > best ? key : best;
       }
-      p = best ? key_idx(best) : 0;  // a row without any comparable value (all NaN) falls back to token 0
+      p = best ? key_idx(best) : 0;  // a row without any comparable value falls back to token 0
+      if (best == kKeyGaveUp) bits = kStatusWaitGaveUp;
+      else if (best >= kKeyPlusInf) bits = kStatusNonFinite;  // +inf as the maximum, or the NaN marker
     } else {
       p = sampled_pick[o + n];
+      if (p < 0) { bits = p == -2 ? kStatusWaitGaveUp : kStatusNonFinite; p = 0; }
     }
+    if (bits) atomicOr(&s_bits, bits);
     s_pick[n] = p;
     s_tok[n] = tree.token_ids[o + n];
     s_par[n] = tree.parents[o + n];
@@ -661,6 +711,7 @@ k_walk(ubt_tree tree, int mode, SpanPlan plan, const unsigned long long* __restr
   // Only now may a kernel behind this one become resident: the scratch (row keys / picks) has been read for the
   // last time, so an early-started pass of a following verify call cannot overwrite anything still needed here.
   pdl_launch_dependents();
+  if (tid == 0 && status) status[b] = s_bits;
   if (tid >= 32) return;
   const int n_nodes = tree.n_nodes[b];
   int32_t* an = out.accepted_nodes + (int64_t)b * (L + 1);
@@ -820,10 +871,10 @@ cudaError_t launch_row_sample(const void* logits, int dtype, int B, int N, int V
 
 cudaError_t launch_walk(const ubt_tree& tree, int mode, const VerifyWorkspace& w, int V,
                         const int32_t* sampled_pick, int32_t* node_pick, const ubt_verify_result& out,
-                        cudaStream_t st) {
+                        int32_t* status, cudaStream_t st) {
   if (tree.B == 0) return cudaSuccess;
   return launch_kernel(k_walk, dim3(tree.B), dim3(128), 0, st, true, tree, mode, w.plan,
-                       (const unsigned long long*)w.part_key, V, sampled_pick, node_pick, out);
+                       (const unsigned long long*)w.part_key, V, sampled_pick, node_pick, out, status);
 }
 
 // Number of bounded waits that gave up in this file's kernels (0 in a healthy run).

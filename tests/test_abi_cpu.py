@@ -105,3 +105,35 @@ def test_binding_refuses_cpu_tensors():
     x = torch.zeros((1, 4, 1000), dtype=torch.bfloat16)
     with pytest.raises(ValueError, match="CUDA tensor"):
         u.ubt_draft_tree(x, torch.zeros((1, 3, 4, 4)), 4, 16)
+
+
+def test_struct_layouts_match_the_header(tmp_path):
+    """The ctypes mirrors of the option / result structs must have the size and field offsets the C compiler
+    gives the declarations of include/ubt.h."""
+    import subprocess
+    structs = {"ubt_tree": binding._Tree, "ubt_draft_opts": binding._DraftOpts, "ubt_verify_opts": binding._VerifyOpts,
+               "ubt_verify_result": binding._VerifyResult}
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "ubt.h"', 'int main(void) {']
+    for cname, ct in structs.items():
+        lines.append(f'  printf("{cname} size %zu\\n", sizeof({cname}));')
+        for fname, _ in ct._fields_:
+            cfield = fname.rstrip("_")                      # lambda_ in Python, lambda in C
+            lines.append(f'  printf("{cname} {fname} %zu\\n", offsetof({cname}, {cfield}));')
+    lines += ['  return 0;', '}']
+    src = tmp_path / "layout.c"
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.check_call(["gcc", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)])
+    out = subprocess.check_output([str(exe)], text=True)
+    for line in out.splitlines():
+        cname, field, value = line.split()
+        ct = structs[cname]
+        if field == "size":
+            assert C.sizeof(ct) == int(value), line
+        else:
+            assert getattr(ct, field).offset == int(value), line
+
+
+def test_status_strings_cover_every_code():
+    assert "NaN" in u.status_string(6)
+    assert u.status_string(99) == "unknown status"
