@@ -216,7 +216,7 @@ def measure_workload(ubt, args, cfg, paper_flow, world, rank, dev, stream, headl
 
     sel = {}
     if paper_flow:
-        R, W = synth.SELECTOR_RANK, synth.PAPER_SEARCH_WIDTH
+        R, W = synth.SELECTOR_RANK, synth.search_width(cfg)
         phi, psi, gate, anchor = synth.device_selector_tables(cfg.V, R, cfg.B, cfg.L, input_seed(rank, 99), dev)
         sel = dict(phi=phi, psi=psi, gate=gate, anchor=anchor, W=W,
                    big=torch.empty((cfg.B, cfg.L - 1, cfg.k, cfg.k), dtype=torch.float32, device=dev),
@@ -279,6 +279,15 @@ def measure_workload(ubt, args, cfg, paper_flow, world, rank, dev, stream, headl
         step(args.warmup + i, early=True)
     e3.record(stream)
     torch.cuda.synchronize()
+    # ---- the verify call in its path-only form (reads only the target rows a walk visits), timed alone
+    e4, e5 = mk(), mk()
+    e4.record(stream)
+    for i in range(K):
+        ubt.ubt_verify_tree(tree, sets[(args.warmup + i) % n_sets][2], cfg.mode, seed=i, result=res, ws=ws_v,
+                            stream=stream, path_only=True)
+    e5.record(stream)
+    torch.cuda.synchronize()
+    path_ms = max_over_ranks(e4.elapsed_time(e5), world, dev) / K
     t_wall1 = time.time()
     barrier(world)
     clocks = sampler.stop(t_wall0, t_wall1)
@@ -333,6 +342,10 @@ def measure_workload(ubt, args, cfg, paper_flow, world, rank, dev, stream, headl
         "chained_early_start": {"ms_per_step": chained_ms / K, "trees_per_s": cfg.B * K * world / (chained_ms * 1e-3),
                                 "note": "verify pass started while the draft call still ran (ubt_verify_opts.early_start);"
                                         " not reachable when the target logits depend on the tree"},
+        "verify_path_only": {"ms_per_call": path_ms, "mean_accepted_len": float(res.accepted_len.float().mean()),
+                             "note": "ubt_verify_opts.path_only: evaluates at most L+1 of the N target rows of a "
+                                     "sequence; its time grows with the accepted length (synthetic targets here "
+                                     "accept almost nothing)"},
         "kernels": kernels, "gpu_launches": launches_per_step * K, "clocks": clocks,
     }
     state = dict(sets=sets, tree=tree, res=res, ws_d=ws_d, ws_v=ws_v, draft=draft, sel=sel, dominant=dominant,
@@ -352,7 +365,7 @@ def live_parity(ubt, cfg, paper_flow, st, dev, stream, sample, timed_seconds=0.0
     if paper_flow:
         kw = dict(phi=synth.to_host_bits(sel["phi"]), psi=synth.to_host_bits(sel["psi"]),
                   gate=sel["gate"][:sample].cpu().numpy(), anchor=sel["anchor"][:sample].cpu().numpy(),
-                  W=synth.PAPER_SEARCH_WIDTH)
+                  W=synth.search_width(cfg))
     done, spent = 0, 0.0
     while True:
         tr, ov, dt = oracle_pass(cfg, uh, bh, zh, 0, **kw)
@@ -365,7 +378,7 @@ def live_parity(ubt, cfg, paper_flow, st, dev, stream, sample, timed_seconds=0.0
     torch.cuda.synchronize()
     try:
         g = tree_to_numpy(st["tree"])
-        swaps = compare_draft(g, tr, cfg.L, cfg.k, cfg.N, synth.PAPER_SEARCH_WIDTH if paper_flow else 0, 0.0,
+        swaps = compare_draft(g, tr, cfg.L, cfg.k, cfg.N, synth.search_width(cfg) if paper_flow else 0, 0.0,
                               kw.get("anchor"), None, rows=list(range(sample)))
         if not swaps:
             compare_verify(st["res"], ov, pick, rows=slice(0, sample))
@@ -467,7 +480,7 @@ def main():
         "config": {"workload": cfg.name, "B": cfg.B, "L": cfg.L, "V": cfg.V, "k": cfg.k, "node_budget": cfg.N,
                    "verify": cfg.mode, "logits": cfg.dtype, "input_sets": n_sets,
                    "order": "plain stream order: draft call, then verify call, nothing overlapped",
-                   **({"search_width": synth.PAPER_SEARCH_WIDTH, "selector_rank": synth.SELECTOR_RANK,
+                   **({"search_width": synth.search_width(cfg), "selector_rank": synth.SELECTOR_RANK,
                        "flow": "ubt_topk_logprob -> ubt_selector_scores -> ubt_build_tree -> ubt_verify_tree"}
                       if paper_flow else {}),
                    "l2": "inputs larger than L2 (rotation of %d MB)" % (batch_bytes * n_sets // 1_000_000)},

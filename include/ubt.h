@@ -119,6 +119,12 @@ typedef struct ubt_verify_opts {
   int32_t *status;     /* optional [B] device words, written for every sequence: 0, or UBT_STATUS_* bits (a NaN
                           or +inf in one of the sequence's N target rows, used slot or not) */
   int32_t validate_finite; /* host-buffer form only: return UBT_ERR_NONFINITE if any sequence was flagged */
+  int32_t path_only;   /* 1: evaluate only the target rows the walk visits (at most L + 1 of the N rows of a
+                          sequence) instead of all of them: the same verdict from a fraction of the bytes, as a
+                          chain of at most L + 1 dependent steps inside one cooperative launch (needs B <= 1024,
+                          else UBT_ERR_UNSUPPORTED).  node_pick then receives the picks of the visited slots and
+                          -1 elsewhere; early_start is ignored.  Worth it when B * N is large (most rows are never
+                          visited); for a single small tree the all-rows pass is as fast. */
 } ubt_verify_opts;
 
 typedef struct ubt_verify_result {

@@ -45,7 +45,7 @@ class _DraftOpts(C.Structure):
 class _VerifyOpts(C.Structure):
     _fields_ = [("seed", C.c_uint64), ("temperature", C.c_float), ("node_pick", C.c_void_p),
                 ("event_before", C.c_void_p), ("event_after", C.c_void_p), ("early_start", C.c_int32),
-                ("status", C.c_void_p), ("validate_finite", C.c_int32)]
+                ("status", C.c_void_p), ("validate_finite", C.c_int32), ("path_only", C.c_int32)]
 
 
 class _VerifyResult(C.Structure):
@@ -283,8 +283,10 @@ def ubt_draft_tree(unigram_logits: torch.Tensor, bigram_scores: Optional[torch.T
 def ubt_verify_tree(tree: Tree, target_logits: torch.Tensor, mode="greedy", seed: int = 0, temperature: float = 1.0,
                     node_pick: Optional[torch.Tensor] = None, result: Optional[VerifyResult] = None,
                     ws: Optional[torch.Tensor] = None, stream=None, event_before=None,
-                    event_after=None, early_start: bool = False, status: Optional[torch.Tensor] = None) -> VerifyResult:
-    """Walk ``tree`` against ``target_logits[B,N,V]`` (step a4).  ``early_start``: see ``ubt_verify_opts``."""
+                    event_after=None, early_start: bool = False, status: Optional[torch.Tensor] = None,
+                    path_only: bool = False) -> VerifyResult:
+    """Walk ``tree`` against ``target_logits[B,N,V]`` (step a4).  ``early_start``, ``path_only``: see
+    ``ubt_verify_opts``."""
     _need(target_logits, "target_logits")
     B, N, V = target_logits.shape
     m = _MODES.get(mode, mode)
@@ -295,7 +297,7 @@ def ubt_verify_tree(tree: Tree, target_logits: torch.Tensor, mode="greedy", seed
     ev = lambda e: None if e is None else C.c_void_p(e.cuda_event)
     o = _VerifyOpts(int(seed), float(temperature), None if node_pick is None else node_pick.data_ptr(),
                     ev(event_before), ev(event_after), int(bool(early_start)),
-                    None if status is None else status.data_ptr(), 0)
+                    None if status is None else status.data_ptr(), 0, int(bool(path_only)))
     t = tree.c_struct()
     r = result.c_struct()
     _check(load().ubt_verify_tree(C.byref(t), _ptr(target_logits), _dtype_code(target_logits), V, m, C.byref(o),
@@ -332,7 +334,7 @@ def ubt_verify_tree_host(tree: Tree, target_logits: torch.Tensor, result: Verify
     _need(target_logits, "target_logits", cuda=False)
     B, N, V = target_logits.shape
     o = _VerifyOpts(int(seed), float(temperature), None if node_pick is None else node_pick.data_ptr(), None, None, 0,
-                    None if status is None else status.data_ptr(), int(bool(validate_finite)))
+                    None if status is None else status.data_ptr(), int(bool(validate_finite)), 0)
     t = tree.c_struct()
     r = result.c_struct()
     _check(load().ubt_verify_tree_host(C.byref(t), _ptr(target_logits), _dtype_code(target_logits), V,

@@ -151,7 +151,8 @@ size_t ubt_draft_workspace_bytes(int B, int L, int V, int k, int N) {
 
 size_t ubt_verify_workspace_bytes(int B, int N, int V, int mode) {
   if (B < 0 || N < 1 || V < 1 || (mode != UBT_VERIFY_GREEDY && mode != UBT_VERIFY_SAMPLE)) return 0;
-  return verify_workspace_bytes((int64_t)B * N, V, mode) + 256;
+  const size_t all_rows = verify_workspace_bytes((int64_t)B * N, V, mode), path = verify_path_workspace_bytes(B, N, mode);
+  return (all_rows > path ? all_rows : path) + 256;  // either form of the call fits
 }
 
 int ubt_topk_logprob(const void* logits, int dtype, int64_t rows, int V, int k, int32_t* cand_ids,
@@ -262,17 +263,32 @@ int ubt_verify_tree(const ubt_tree* tree, const void* target_logits, int dtype, 
   const int B = tree->B, N = tree->N, L = tree->L;
   if (B < 0 || N < 1 || L < 1) return UBT_ERR_INVALID_ARG;
   if (N > kMaxN || L > kMaxL) return UBT_ERR_UNSUPPORTED;
-  const ubt_verify_opts d{0, 1.0f, nullptr, nullptr, nullptr, 0, nullptr, 0};
+  const ubt_verify_opts d{0, 1.0f, nullptr, nullptr, nullptr, 0, nullptr, 0, 0};
   const ubt_verify_opts* o = opts ? opts : &d;
   if (mode == UBT_VERIFY_SAMPLE) {
     if (!(o->temperature > 0.0f)) return UBT_ERR_INVALID_ARG;
     if (V > 2048 * 1024) return UBT_ERR_UNSUPPORTED;
   }
+  if (o->path_only && B > verify_path_max_batch()) return UBT_ERR_UNSUPPORTED;
   if (B == 0) return UBT_OK;
   const int64_t rows = (int64_t)B * N;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (o->path_only) {
+    if (!workspace || !aligned16(workspace) || workspace_bytes < verify_path_workspace_bytes(B, N, mode))
+      return UBT_ERR_WORKSPACE;
+    if (o->event_before && cudaEventRecord(static_cast<cudaEvent_t>(o->event_before), st) != cudaSuccess)
+      return UBT_ERR_CUDA;
+    if (launch_verify_path(*tree, target_logits, dtype, V, mode, o->seed, o->temperature, workspace, o->node_pick, *out,
+                           o->status, st) != cudaSuccess) {
+      cudaGetLastError();
+      return UBT_ERR_CUDA;
+    }
+    if (o->event_after && cudaEventRecord(static_cast<cudaEvent_t>(o->event_after), st) != cudaSuccess)
+      return UBT_ERR_CUDA;
+    return UBT_OK;
+  }
   if (!workspace || !aligned16(workspace) || workspace_bytes < verify_workspace_bytes(rows, V, mode))
     return UBT_ERR_WORKSPACE;
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   VerifyWorkspace w = carve_verify_workspace(workspace, rows, V, mode);
   const int32_t* sampled = nullptr;
   if (o->event_before && cudaEventRecord(static_cast<cudaEvent_t>(o->event_before), st) != cudaSuccess)
@@ -468,7 +484,7 @@ int ubt_verify_tree_host(const ubt_tree* tree, const void* target_logits, int dt
   UBT_CUDA_OK(cudaMemcpyAsync(d.tree.t.token_ids, tree->token_ids, bn * 4, cudaMemcpyHostToDevice, st));
   UBT_CUDA_OK(cudaMemcpyAsync(d.tree.t.parents, tree->parents, bn * 4, cudaMemcpyHostToDevice, st));
   UBT_CUDA_OK(cudaMemcpyAsync(d.tree.t.n_nodes, tree->n_nodes, (size_t)B * 4, cudaMemcpyHostToDevice, st));
-  ubt_verify_opts dev_opts{0, 1.0f, nullptr, nullptr, nullptr, 0, nullptr, 0};
+  ubt_verify_opts dev_opts{0, 1.0f, nullptr, nullptr, nullptr, 0, nullptr, 0, 0};
   if (opts) { dev_opts = *opts; }
   dev_opts.early_start = 0;  // the logits are copied in just before: nothing to start ahead of
   int32_t* host_status = dev_opts.status;  // a HOST array in this form
@@ -491,12 +507,15 @@ int ubt_verify_tree_host(const ubt_tree* tree, const void* target_logits, int dt
 namespace ubt {
 cudaError_t ring_timeouts_verify(unsigned int* out);
 cudaError_t ring_timeouts_topk(unsigned int* out);
+cudaError_t ring_timeouts_path(unsigned int* out);
 }  // namespace ubt
 extern "C" {
 long long ubt_debug_ring_timeouts(void) {
-  unsigned int a = 0, b = 0;
-  if (ring_timeouts_verify(&a) != cudaSuccess || ring_timeouts_topk(&b) != cudaSuccess) return -1;
-  return (long long)a + b;
+  unsigned int a = 0, b = 0, c = 0;
+  if (ring_timeouts_verify(&a) != cudaSuccess || ring_timeouts_topk(&b) != cudaSuccess ||
+      ring_timeouts_path(&c) != cudaSuccess)
+    return -1;
+  return (long long)a + b + c;
 }
 
 #ifdef UBT_BOUNDS_CHECK

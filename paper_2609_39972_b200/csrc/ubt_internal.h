@@ -123,4 +123,11 @@ cudaError_t launch_walk(const ubt_tree& tree, int mode, const VerifyWorkspace& w
                         const int32_t* sampled_pick, int32_t* node_pick,
                         const ubt_verify_result& out, int32_t* status, cudaStream_t st);
 
+// ---- a4, path-only form: evaluates only the target rows the walk visits (ubt_verify_path.cu)
+size_t verify_path_workspace_bytes(int B, int N, int mode);
+int verify_path_max_batch();
+cudaError_t launch_verify_path(const ubt_tree& tree, const void* logits, int dtype, int V, int mode, uint64_t seed,
+                               float temperature, void* ws, int32_t* node_pick, const ubt_verify_result& out,
+                               int32_t* status, cudaStream_t st);
+
 }  // namespace ubt

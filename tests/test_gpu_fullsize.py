@@ -40,6 +40,9 @@ def _run_full(name, pick_rows, seeds=(0,)):
         # the oracle numbers sequences by their place in the arrays it is given: the whole batch keeps b true
         ov = oracle.verify(g.token_ids, g.parents, g.n_nodes, cfg.L, zh, cfg.mode, seed=s, all_nodes=False)
         compare_verify(res, ov)
+        res_p = u.ubt_verify_tree(gtree, zd, cfg.mode, seed=s, path_only=True)     # visits the walk's rows only
+        torch.cuda.synchronize()
+        compare_verify(res_p, ov)
         if cfg.mode == "greedy":
             sub = lambda a: a[rows]
             ov8 = oracle.verify(sub(g.token_ids), sub(g.parents), sub(g.n_nodes), cfg.L, zr, "greedy")

@@ -54,12 +54,28 @@ def run_case(cfg, seed, targets="plant", W=0, zeta=0.0, use_opts=False, seeds_sa
         res2 = u.ubt_verify_tree(gtree, zd, "greedy")          # without node_pick
         torch.cuda.synchronize()
         compare_verify(res2, ov)
+        _check_path_only(u, gtree, zd, "greedy", 0, ov, g, cfg)
     for s in (seeds_sample if cfg.mode == "sample" else ()):
         res = u.ubt_verify_tree(gtree, zd, "sample", seed=s, temperature=1.0, node_pick=pick)
         torch.cuda.synchronize()
         ov = oracle.verify(g.token_ids, g.parents, g.n_nodes, cfg.L, z, "sample", seed=s, temperature=1.0)
         compare_verify(res, ov, pick)
+        _check_path_only(u, gtree, zd, "sample", s, ov, g, cfg)
     return swaps
+
+
+def _check_path_only(u, gtree, zd, mode, seed, ov, g, cfg):
+    """The path-only form of the verify call: the same verdict, picks reported at the visited slots only."""
+    pick = torch.full((cfg.B, cfg.N), -7, dtype=torch.int32, device=DEV)
+    res = u.ubt_verify_tree(gtree, zd, mode, seed=seed, temperature=1.0, node_pick=pick, path_only=True)
+    torch.cuda.synchronize()
+    compare_verify(res, ov)
+    pk = pick.cpu().numpy()
+    nodes = res.accepted_nodes.cpu().numpy()
+    for b in range(cfg.B):
+        visited = [int(n) for n in nodes[b] if n >= 0]
+        for n in range(cfg.N):
+            assert pk[b, n] == (ov.node_pick[b, n] if n in visited else -1), (b, n)
 
 
 @pytest.mark.parametrize("seed", range(6))

@@ -74,7 +74,17 @@ PAPER_SEARCH_WIDTH = 12
 NEXT_CONFIGS = {
     "p1": Config("p1", 32, 15, V_QWEN3, 64, 65, "bf16", "pos_uniform:0.5,8", 1.0, 4.0, "greedy"),
     "p1-b1": Config("p1-b1", 1, 15, V_QWEN3, 64, 65, "bf16", "pos_uniform:0.5,8", 1.0, 4.0, "greedy"),
+    # The smaller (budget / width) pairs of the paper's load-adaptive serving setup ("Academic-scale
+    # Experiment", concurrent serving): 32 / 8 and 16 / 3 non-root nodes / search width.
+    "p2": Config("p2", 32, 15, V_QWEN3, 64, 33, "bf16", "pos_uniform:0.5,8", 1.0, 4.0, "greedy"),
+    "p3": Config("p3", 32, 15, V_QWEN3, 64, 17, "bf16", "pos_uniform:0.5,8", 1.0, 4.0, "greedy"),
 }
+SEARCH_WIDTH = {"p1": 12, "p1-b1": 12, "p2": 8, "p3": 3}
+
+
+def search_width(cfg: "Config") -> int:
+    """Search width the paper pairs with a next-row configuration (0 = unbounded for the others)."""
+    return SEARCH_WIDTH.get(cfg.name.split("-B")[0], 0)
 
 
 # --------------------------------------------------------------------------
