@@ -288,6 +288,20 @@ def measure_workload(ubt, args, cfg, paper_flow, world, rank, dev, stream, headl
     e5.record(stream)
     torch.cuda.synchronize()
     path_ms = max_over_ranks(e4.elapsed_time(e5), world, dev) / K
+    path_len = float(res.accepted_len.float().mean())
+    # ... and on targets that agree with the drafted tree (each child's token boosted in its parent's row), so
+    # that the walks are several steps long.  Done last: it edits input set 0 in place.
+    draft(sets[0][0], sets[0][1])
+    torch.cuda.synchronize()
+    synth.boost_children_on_device(sets[0][2], tree.token_ids, tree.parents, tree.n_nodes, boost=14.0)
+    e6, e7 = mk(), mk()
+    e6.record(stream)
+    for i in range(K):
+        ubt.ubt_verify_tree(tree, sets[0][2], cfg.mode, seed=i, result=res, ws=ws_v, stream=stream, path_only=True)
+    e7.record(stream)
+    torch.cuda.synchronize()
+    path_agree_ms = max_over_ranks(e6.elapsed_time(e7), world, dev) / K
+    path_agree_len = float(res.accepted_len.float().mean())
     t_wall1 = time.time()
     barrier(world)
     clocks = sampler.stop(t_wall0, t_wall1)
@@ -342,10 +356,11 @@ def measure_workload(ubt, args, cfg, paper_flow, world, rank, dev, stream, headl
         "chained_early_start": {"ms_per_step": chained_ms / K, "trees_per_s": cfg.B * K * world / (chained_ms * 1e-3),
                                 "note": "verify pass started while the draft call still ran (ubt_verify_opts.early_start);"
                                         " not reachable when the target logits depend on the tree"},
-        "verify_path_only": {"ms_per_call": path_ms, "mean_accepted_len": float(res.accepted_len.float().mean()),
+        "verify_path_only": {"ms_per_call": path_ms, "mean_accepted_len": path_len,
+                             "agreeing_targets": {"ms_per_call": path_agree_ms, "mean_accepted_len": path_agree_len},
                              "note": "ubt_verify_opts.path_only: evaluates at most L+1 of the N target rows of a "
-                                     "sequence; its time grows with the accepted length (synthetic targets here "
-                                     "accept almost nothing)"},
+                                     "sequence; its time grows with the accepted length (noise targets accept almost "
+                                     "nothing; the second figure is on targets boosted towards the drafted tree)"},
         "kernels": kernels, "gpu_launches": launches_per_step * K, "clocks": clocks,
     }
     state = dict(sets=sets, tree=tree, res=res, ws_d=ws_d, ws_v=ws_v, draft=draft, sel=sel, dominant=dominant,

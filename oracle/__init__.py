@@ -52,6 +52,8 @@ def lib() -> C.CDLL:
         _lib.ubt_oracle_walks_from_cdf.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p,
                                                    C.c_uint32, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         _lib.ubt_oracle_weight_consts.argtypes = [C.c_float, C.c_float, C.c_void_p, C.c_void_p]
+        _lib.ubt_oracle_lm_head_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int, C.c_int, C.c_int,
+                                                 C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         _lib.ubt_oracle_selector_scores.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int, C.c_void_p,
                                                     C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p,
                                                     C.c_void_p]
@@ -94,6 +96,27 @@ def topk_logprob(logits: np.ndarray, k: int):
     if rc:
         raise ValueError("oracle topk_logprob rejected its arguments")
     return ids, lp, lse
+
+
+def lm_head_topk(hidden: np.ndarray, weight: np.ndarray, k: int, want_logits: bool = False):
+    """Unigram logits ``hidden[rows, d] @ weight[V, d].T`` in double, then step 1 on them (Section 3.1.1, eq. 3).
+
+    ``hidden`` and ``weight`` are fp32, or bf16 bit patterns as uint16.  Returns ``(cand_ids[rows, k] i32,
+    cand_lp[rows, k] f64, lse[rows] f64, logits[rows, V] f64 or None)``.
+    """
+    hidden = np.ascontiguousarray(hidden); weight = np.ascontiguousarray(weight)
+    rows, d = hidden.shape
+    V, d2 = weight.shape
+    assert d == d2 and hidden.dtype == weight.dtype
+    ids = np.empty((rows, k), np.int32)
+    lp = np.empty((rows, k), np.float64)
+    lse = np.empty(rows, np.float64)
+    logits = np.empty((rows, V), np.float64) if want_logits else None
+    rc = lib().ubt_oracle_lm_head_topk(_p(hidden), _p(weight), _dtype_code(hidden), rows, d, V, k, _p(ids), _p(lp),
+                                       _p(lse), _p(logits) if want_logits else None)
+    if rc:
+        raise ValueError("oracle lm_head_topk rejected its arguments")
+    return ids, lp, lse, logits
 
 
 def selector_scores(phi: np.ndarray, psi: np.ndarray, gate: np.ndarray, cand_ids: np.ndarray,

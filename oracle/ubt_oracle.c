@@ -94,6 +94,54 @@ int ubt_oracle_topk_logprob(const void *logits, int dtype, int64_t rows, int V, 
 }
 
 /* ---------------------------------------------------------------------- */
+/* Unigram logits from the proposer state (Section 3.1.1, eq. 3: the logit   */
+/* vector of a position is the frozen LM head applied to the position's       */
+/* hidden state), followed by the candidate selection above:                  */
+/*   u[row][v] = sum_j h[row][j] * W[v][j]      (double; inputs bf16 or fp32) */
+/* then the k best under (logit descending, token id ascending) and           */
+/*   cand_lp[r] = u[C_r] - log sum_v exp u[v].                                 */
+/* W is [V, d] row-major (one row of d weights per token), h is [rows, d].    */
+/* row_logits (optional, [rows, V] double) receives u for tests.              */
+/* ---------------------------------------------------------------------- */
+int ubt_oracle_lm_head_topk(const void *h, const void *W, int dtype, int64_t rows, int d, int V, int k,
+                            int32_t *cand_ids, double *cand_lp, double *row_lse, double *row_logits) {
+  if (!h || !W || rows < 0 || d < 1 || V < 1 || k < 1 || k > V) return 1;
+  int bad = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t row = 0; row < rows; ++row) {
+    double *x = (double *)malloc(sizeof(double) * (size_t)V);
+    double *hr = (double *)malloc(sizeof(double) * (size_t)d);
+    char *taken = (char *)calloc((size_t)V, 1);
+    if (!x || !hr || !taken) { bad = 1; free(x); free(hr); free(taken); continue; }
+    for (int j = 0; j < d; ++j) hr[j] = (double)load_f32(h, dtype, row * (int64_t)d + j);
+    for (int v = 0; v < V; ++v) {
+      double acc = 0.0;
+      for (int j = 0; j < d; ++j) acc += hr[j] * (double)load_f32(W, dtype, (int64_t)v * d + j);
+      x[v] = acc;
+    }
+    if (row_logits) memcpy(row_logits + row * (int64_t)V, x, sizeof(double) * (size_t)V);
+    double m = x[0];
+    for (int v = 1; v < V; ++v) if (x[v] > m) m = x[v];
+    double sum = 0.0;
+    for (int v = 0; v < V; ++v) sum += exp(x[v] - m);
+    double lse = m + log(sum);
+    if (row_lse) row_lse[row] = lse;
+    for (int r = 0; r < k; ++r) {
+      int best = -1;
+      for (int v = 0; v < V; ++v) {
+        if (taken[v]) continue;
+        if (best < 0 || x[v] > x[best]) best = v; /* strict >: lower id wins ties */
+      }
+      taken[best] = 1;
+      cand_ids[row * k + r] = best;
+      cand_lp[row * k + r] = x[best] - lse;
+    }
+    free(x); free(hr); free(taken);
+  }
+  return bad;
+}
+
+/* ---------------------------------------------------------------------- */
 /* Selector scores (Section 3.1.2, "Parallel Computation", the edge-matrix   */
 /* equation; the score of one pair is the low-rank bigram selector of        */
 /* Section 2): for predecessor token a and successor token b at position i,  */

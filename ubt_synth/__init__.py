@@ -329,6 +329,34 @@ def selector_tables(V: int, R: int, B: int, L: int, seed: int, dtype: str = "bf1
     return phi, psi, gate
 
 
+def lm_head_inputs(rows: int, d: int, V: int, seed: int, scale: float = 2.0, dtype: str = "bf16"):
+    """Synthetic stand-ins for the proposer's hidden states and the frozen LM head: ``hidden[rows, d]`` N(0,1) and
+    ``weight[V, d]`` N(0, scale^2 / d), so that a logit (a sum of d products) is N(0, scale^2) like the
+    configurations' unigram logits.  bf16 as bit patterns (uint16), or fp32."""
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence([seed, 0x11EAD])))
+    h = rng.standard_normal((rows, d), dtype=np.float32)
+    w = (rng.standard_normal((V, d), dtype=np.float32) * np.float32(scale / np.sqrt(d))).astype(np.float32)
+    if dtype == "bf16":
+        h, w = f32_to_bf16_bits(h), f32_to_bf16_bits(w)
+    return h, w
+
+
+def device_lm_head_inputs(rows: int, d: int, V: int, seed: int, device, scale: float = 2.0):
+    """Device-resident ``(hidden[rows, d] bf16, weight[V, d] bf16)`` with the distributions of ``lm_head_inputs``."""
+    import torch
+
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed) * 1_000_003 + 0x11E)
+    h = torch.randn((rows, d), generator=g, device=device, dtype=torch.float32).to(torch.bfloat16)
+    w = torch.empty((V, d), dtype=torch.bfloat16, device=device)
+    step = max(1, (1 << 26) // d)
+    for v0 in range(0, V, step):
+        v1 = min(V, v0 + step)
+        w[v0:v1] = (torch.randn((v1 - v0, d), generator=g, device=device, dtype=torch.float32)
+                    * float(scale / np.sqrt(d))).to(torch.bfloat16)
+    return h, w
+
+
 def device_selector_tables(V: int, R: int, B: int, L: int, seed: int, device):
     """Device-resident stand-ins for the selector's tables: ``(phi[V,R] bf16, psi[V,R] bf16, gate[B,L,R] fp32,
     anchor_tokens[B] i32)``, same distributions as ``selector_tables``, drawn with a seeded torch generator."""
