@@ -156,6 +156,23 @@ int ubt_topk_logprob(const void *logits, int dtype, int64_t rows, int V, int k, 
                      float *cand_logprob, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * The proposer's LM head fused with step a1 (Section 3.1.1, eq. 3: the unigram logits of a position are the
+ * frozen LM head applied to the position's hidden state; the paper times this projection inside its draft
+ * post-processing stage, appendix "Drafting Latency Analysis").  For each of `rows` hidden states:
+ *   u[v] = sum_j hidden[row, j] * weight[v, j]          (bf16 inputs, fp32 accumulation on the tensor cores)
+ * then the k largest u ordered (value descending, token id ascending) and cand_logprob[r] = u[cand_ids[r]] -
+ * log(sum_v exp u[v]) -- the [rows, V] logits are never written to memory.  hidden: [rows, d] bf16 row-major;
+ * weight: [V, d] bf16 row-major (one row of d weights per token); both 16-byte aligned, d a multiple of 64,
+ * k <= 16 (else UBT_ERR_UNSUPPORTED: keep the logits and call ubt_topk_logprob).  The logits carry the
+ * rounding of an fp32 accumulation in the tensor cores' order, so candidates whose logits differ by less than
+ * about 1e-5 * sqrt(d) relative may come out in either order.  Workspace: ubt_lm_head_workspace_bytes().
+ * A device-side wait that gives up (counted by ubt_debug_ring_timeouts) leaves the outputs undefined.
+ */
+size_t ubt_lm_head_workspace_bytes(int64_t rows, int d, int V, int k);
+int ubt_lm_head_topk(const void *hidden, const void *weight, int64_t rows, int d, int V, int k, int32_t *cand_ids,
+                     float *cand_logprob, void *workspace, size_t workspace_bytes, void *cuda_stream);
+
+/*
  * Steps a2, a3, a3b from candidates that are already in out->cand_ids / out->cand_logprob
  * (eq. 5, eq. 9-12, Algorithm 1).  bigram_scores[b,j,ra,rb] is the selector score delta of the
  * transition from the rank-ra candidate of position j to the rank-rb candidate of position j+1.

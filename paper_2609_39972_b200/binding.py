@@ -56,7 +56,8 @@ class _VerifyResult(C.Structure):
 EXPORTS = ["ubt_version", "ubt_status_string", "ubt_debug_ring_timeouts", "ubt_draft_workspace_bytes", "ubt_verify_workspace_bytes",
            "ubt_topk_logprob", "ubt_selector_scores", "ubt_build_tree", "ubt_build_mask", "ubt_draft_tree", "ubt_verify_tree",
            "ubt_draft_host_buffer_bytes", "ubt_verify_host_buffer_bytes", "ubt_draft_tree_host",
-           "ubt_verify_tree_host", "ubt_verify_tree_static", "ubt_verify_static_capacity"]
+           "ubt_verify_tree_host", "ubt_verify_tree_static", "ubt_verify_static_capacity", "ubt_lm_head_workspace_bytes",
+           "ubt_lm_head_topk"]
 
 _lib = None
 
@@ -98,6 +99,10 @@ def load() -> C.CDLL:
                                   C.c_void_p, C.c_size_t, C.c_void_p]
     L.ubt_verify_tree_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
     L.ubt_verify_static_capacity.restype = C.c_longlong
+    L.ubt_lm_head_workspace_bytes.restype = C.c_size_t
+    L.ubt_lm_head_workspace_bytes.argtypes = [C.c_int64, C.c_int, C.c_int, C.c_int]
+    L.ubt_lm_head_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
+                                   C.c_void_p, C.c_size_t, C.c_void_p]
     L.ubt_debug_ring_timeouts.restype = C.c_longlong
     L.ubt_draft_tree_host.argtypes = L.ubt_draft_tree.argtypes
     L.ubt_verify_tree_host.argtypes = L.ubt_verify_tree.argtypes
@@ -227,6 +232,31 @@ def ubt_topk_logprob(logits: torch.Tensor, k: int, cand_ids: torch.Tensor, cand_
     _check(load().ubt_topk_logprob(_ptr(logits), _dtype_code(logits), rows, V, k, _ptr(_need(cand_ids, "cand_ids")),
                                    _ptr(_need(cand_logprob, "cand_logprob")), _ptr(ws), ws.numel(), _stream(stream)),
            "ubt_topk_logprob")
+
+
+def ubt_lm_head_workspace_bytes(rows: int, d: int, V: int, k: int) -> int:
+    return int(load().ubt_lm_head_workspace_bytes(rows, d, V, k))
+
+
+def ubt_lm_head_topk(hidden: torch.Tensor, weight: torch.Tensor, k: int, cand_ids: Optional[torch.Tensor] = None,
+                     cand_logprob: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None, stream=None):
+    """LM head fused with step a1: ``hidden[..., d]`` (bf16) x ``weight[V, d]`` (bf16) -> ``(cand_ids[..., k],
+    cand_logprob[..., k])``; the logits themselves are never stored."""
+    _need(hidden, "hidden"); _need(weight, "weight")
+    if hidden.dtype != torch.bfloat16 or weight.dtype != torch.bfloat16:
+        raise TypeError("hidden and weight must be torch.bfloat16")
+    d = hidden.shape[-1]
+    V = weight.shape[0]
+    rows = hidden.numel() // d
+    if cand_ids is None:
+        cand_ids = torch.empty(hidden.shape[:-1] + (k,), dtype=torch.int32, device=hidden.device)
+    if cand_logprob is None:
+        cand_logprob = torch.empty(hidden.shape[:-1] + (k,), dtype=torch.float32, device=hidden.device)
+    if ws is None:
+        ws = workspace(ubt_lm_head_workspace_bytes(rows, d, V, k), hidden.device)
+    _check(load().ubt_lm_head_topk(_ptr(hidden), _ptr(weight), rows, d, V, k, _ptr(cand_ids), _ptr(cand_logprob),
+                                   _ptr(ws), ws.numel(), _stream(stream)), "ubt_lm_head_topk")
+    return cand_ids, cand_logprob
 
 
 def ubt_build_tree(bigram_scores: Optional[torch.Tensor], tree: Tree, stream=None, **opts) -> None:

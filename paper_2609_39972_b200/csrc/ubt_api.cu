@@ -171,6 +171,26 @@ int ubt_topk_logprob(const void* logits, int dtype, int64_t rows, int V, int k, 
   return UBT_OK;
 }
 
+size_t ubt_lm_head_workspace_bytes(int64_t rows, int d, int V, int k) {
+  if (rows < 0 || d < 1 || V < 1 || k < 1 || k > V || k > lm_head_max_k() || d % 64 != 0) return 0;
+  return lm_head_workspace_bytes(rows, k);
+}
+
+int ubt_lm_head_topk(const void* hidden, const void* weight, int64_t rows, int d, int V, int k, int32_t* cand_ids,
+                     float* cand_logprob, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!hidden || !weight || !cand_ids || !cand_logprob || rows < 0 || d < 1 || V < 1 || k < 1 || k > V)
+    return UBT_ERR_INVALID_ARG;
+  if (!aligned16(hidden) || !aligned16(weight) || !aligned16(cand_ids) || !aligned16(cand_logprob))
+    return UBT_ERR_INVALID_ARG;
+  if (d % 64 != 0 || k > lm_head_max_k() || device_info().sm_count > 256) return UBT_ERR_UNSUPPORTED;
+  if (rows == 0) return UBT_OK;
+  if (!workspace || !aligned16(workspace) || workspace_bytes < lm_head_workspace_bytes(rows, k)) return UBT_ERR_WORKSPACE;
+  cudaError_t e = launch_lm_head_topk(hidden, weight, rows, d, V, k, cand_ids, cand_logprob, workspace,
+                                      static_cast<cudaStream_t>(cuda_stream));
+  if (e != cudaSuccess) { cudaGetLastError(); return e == cudaErrorNotSupported ? UBT_ERR_UNSUPPORTED : UBT_ERR_CUDA; }
+  return UBT_OK;
+}
+
 static int check_draft_opts(const ubt_draft_opts* o) {
   if (!o) return UBT_OK;
   if (o->search_width < 0 || !(o->depth_bonus <= 0.0f)) return UBT_ERR_INVALID_ARG;
@@ -508,14 +528,15 @@ namespace ubt {
 cudaError_t ring_timeouts_verify(unsigned int* out);
 cudaError_t ring_timeouts_topk(unsigned int* out);
 cudaError_t ring_timeouts_path(unsigned int* out);
+cudaError_t lm_head_timeouts(unsigned int* out);
 }  // namespace ubt
 extern "C" {
 long long ubt_debug_ring_timeouts(void) {
-  unsigned int a = 0, b = 0, c = 0;
+  unsigned int a = 0, b = 0, c = 0, d = 0;
   if (ring_timeouts_verify(&a) != cudaSuccess || ring_timeouts_topk(&b) != cudaSuccess ||
-      ring_timeouts_path(&c) != cudaSuccess)
+      ring_timeouts_path(&c) != cudaSuccess || lm_head_timeouts(&d) != cudaSuccess)
     return -1;
-  return (long long)a + b + c;
+  return (long long)a + b + c + d;
 }
 
 #ifdef UBT_BOUNDS_CHECK

@@ -123,6 +123,12 @@ cudaError_t launch_walk(const ubt_tree& tree, int mode, const VerifyWorkspace& w
                         const int32_t* sampled_pick, int32_t* node_pick,
                         const ubt_verify_result& out, int32_t* status, cudaStream_t st);
 
+// ---- LM head fused with a1 (ubt_lmhead.cu): tcgen05 GEMM whose epilogue keeps (max, sum exp, top-k) per row
+int lm_head_max_k();
+size_t lm_head_workspace_bytes(int64_t rows, int k);
+cudaError_t launch_lm_head_topk(const void* hidden, const void* weight, int64_t rows, int d, int V, int k,
+                                int32_t* cand_ids, float* cand_lp, void* ws, cudaStream_t st);
+
 // ---- a4, path-only form: evaluates only the target rows the walk visits (ubt_verify_path.cu)
 size_t verify_path_workspace_bytes(int B, int N, int mode);
 int verify_path_max_batch();
