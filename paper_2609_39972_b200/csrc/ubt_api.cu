@@ -172,7 +172,8 @@ int ubt_topk_logprob(const void* logits, int dtype, int64_t rows, int V, int k, 
 }
 
 size_t ubt_lm_head_workspace_bytes(int64_t rows, int d, int V, int k) {
-  if (rows < 0 || d < 1 || V < 1 || k < 1 || k > V || k > lm_head_max_k() || d % 64 != 0) return 0;
+  if (rows < 0 || d < 1 || V < 1 || k < 1 || k > V || k > lm_head_max_k() || d % 64 != 0 || rows > lm_head_max_rows())
+    return 0;
   return lm_head_workspace_bytes(rows, k);
 }
 
@@ -182,7 +183,8 @@ int ubt_lm_head_topk(const void* hidden, const void* weight, int64_t rows, int d
     return UBT_ERR_INVALID_ARG;
   if (!aligned16(hidden) || !aligned16(weight) || !aligned16(cand_ids) || !aligned16(cand_logprob))
     return UBT_ERR_INVALID_ARG;
-  if (d % 64 != 0 || k > lm_head_max_k() || device_info().sm_count > 256) return UBT_ERR_UNSUPPORTED;
+  if (d % 64 != 0 || k > lm_head_max_k() || rows > lm_head_max_rows() || device_info().sm_count > 256)
+    return UBT_ERR_UNSUPPORTED;
   if (rows == 0) return UBT_OK;
   if (!workspace || !aligned16(workspace) || workspace_bytes < lm_head_workspace_bytes(rows, k)) return UBT_ERR_WORKSPACE;
   cudaError_t e = launch_lm_head_topk(hidden, weight, rows, d, V, k, cand_ids, cand_logprob, workspace,

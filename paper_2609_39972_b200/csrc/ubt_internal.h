@@ -125,6 +125,7 @@ cudaError_t launch_walk(const ubt_tree& tree, int mode, const VerifyWorkspace& w
 
 // ---- LM head fused with a1 (ubt_lmhead.cu): tcgen05 GEMM whose epilogue keeps (max, sum exp, top-k) per row
 int lm_head_max_k();
+int lm_head_max_rows();
 size_t lm_head_workspace_bytes(int64_t rows, int k);
 cudaError_t launch_lm_head_topk(const void* hidden, const void* weight, int64_t rows, int d, int V, int k,
                                 int32_t* cand_ids, float* cand_lp, void* ws, cudaStream_t st);

@@ -3,17 +3,22 @@
 // vocabulary log-sum-exp and the k best logits of step a1 -- the [rows, V] logits never reach HBM.
 //
 // One persistent CTA per SM, warp-specialised, on the fifth-generation tensor cores:
-//   warp 0  (one lane)  TMA producer: 128 x 64 tiles of hidden and 256 x 64 tiles of weight (bf16, 128-byte
-//                       swizzle, no multicast) into a four-stage shared-memory ring
-//   warp 1  (one lane)  issues tcgen05.mma (M = 128, N = 256, K = 16, bf16 -> fp32) into one of two 256-column
-//                       accumulators in tensor memory; tcgen05.commit frees ring stages and hands accumulators over
-//   warps 2-5           epilogue: thread = row of the tile; reads its row of the accumulator with tcgen05.ld,
-//                       folds the 256 logits into a running (max, sum exp) and tests them against the row's
-//                       exclusive top-k threshold; the few that pass are inserted into the row's sorted list
-// A CTA takes vocabulary tiles c, c + grid, ... and, for each, every row tile, so a row's list and (max, sum) are
-// carried across all the CTA's vocabulary tiles; one partial per (CTA, row) goes to the workspace and a small
-// kernel merges the partials of a row.  The epilogue of one tile runs while the next tile's products accumulate
-// in the other half of tensor memory.
+//   warp 0  (one lane)  TMA producer: a stage of the shared-memory ring holds a 256 x 64 tile of hidden and a
+//                       256 x 64 tile of weight (bf16, 128-byte swizzle, no multicast), so every weight tile
+//                       serves two accumulators; three stages (four of 128 + 256 rows when there are at most
+//                       128 rows in all)
+//   warp 1  (one lane)  issues tcgen05.mma (M = 128, N = 256, K = 16, bf16 -> fp32): rows 0-127 of the item
+//                       into the first 256 columns of tensor memory, rows 128-255 into the other 256;
+//                       tcgen05.commit frees ring stages and hands the accumulators over
+//   warps 2-5, 6-9      epilogue of the first / second accumulator: thread = row; reads its row with tcgen05.ld
+//                       32 columns at a time, folds them into a running (max, sum exp) and, when the largest of
+//                       the 32 beats the row's exclusive top-k threshold (or the list is short), extracts the
+//                       qualifying logits best first and inserts them into the row's sorted list
+// Work items are (vocabulary tile, block of 256 rows) pairs dealt round-robin to the CTAs; a row's list and
+// (max, sum) are carried across all the items a CTA gets for it (parked in the workspace between visits), so one
+// partial per (CTA, row) is left for a small kernel that merges the partials of a row.  Tensor memory holds
+// exactly one item, so the epilogue is not hidden behind the next item's products: it is kept short instead
+// (both accumulators drained at once, one row per thread), while the producer refills the ring.
 //
 // Every wait (on a ring stage, on an accumulator) is bounded: a wait that gives up raises a flag, the roles leave
 // their loops, the producer waits (bounded again) for the copies still landing, the CTA meets at its last barrier,
@@ -27,21 +32,25 @@
 
 namespace ubt {
 
-constexpr int LM_BM = 128, LM_BN = 256, LM_BK = 64, LM_STAGES = 4;
-constexpr int LM_THREADS = 192;              // warp 0 producer, warp 1 MMA, warps 2-5 epilogue
-constexpr int LM_MAX_RT = 16;                // row tiles per launch (2048 rows); more rows take more launches
+constexpr int LM_BM = 128, LM_BN = 256, LM_BK = 64;
+constexpr int LM_RB = 2 * LM_BM;             // rows of a work item: two accumulators share every weight tile
+constexpr int LM_MAX_STAGES = 4;
+constexpr int LM_RING_BYTES = 192 * 1024;    // three stages of 64 KB or four of 48 KB
+constexpr int LM_THREADS = 320;              // warp 0 producer, warp 1 MMA, warps 2-5 and 6-9 epilogue
 constexpr int LM_MAX_K = 16;                 // candidates per row the fused epilogue keeps
-constexpr int LM_A_BYTES = LM_BM * LM_BK * 2, LM_B_BYTES = LM_BN * LM_BK * 2, LM_STAGE_BYTES = LM_A_BYTES + LM_B_BYTES;
+constexpr int LM_MAX_ROWS = 64 * LM_RB;      // rows per call (one bit per row block in a CTA's visited mask)
+constexpr int LM_B_BYTES = LM_BN * LM_BK * 2;
 constexpr int LM_SPIN_LIMIT = 1 << 22;
 
 static __device__ unsigned int g_lm_timeouts;
 
 struct LmShared {  // behind the ring in dynamic shared memory
-  uint64_t full[LM_STAGES], empty[LM_STAGES], acc_full[2], acc_empty[2];
+  uint64_t full[LM_MAX_STAGES], empty[LM_MAX_STAGES], acc_full[2], acc_empty[2];
   uint32_t tmem_base;
   int fail;
-  float m[LM_MAX_RT][LM_BM], s[LM_MAX_RT][LM_BM], thr[LM_MAX_RT][LM_BM];
-  unsigned char cnt[LM_MAX_RT][LM_BM];
+  // the sorted candidate lists of the rows being finished, entry i of all rows side by side (a warp touching
+  // entry i of its 32 rows touches 32 different banks); between two visits a row's list lives in the workspace
+  unsigned long long list[2][LM_MAX_K][LM_BM];
 };
 
 __device__ __forceinline__ uint32_t lm_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -123,27 +132,36 @@ struct LmParts {                   // one partial per (CTA, row of the launch's 
   int rpad;                        // rows of the block rounded up to whole row tiles
 };
 
+// Entry `key` into the row's sorted list (column r of `list`); a full list drops its last entry.
+__device__ __forceinline__ void lm_list_insert(unsigned long long (*list)[LM_BM], int r, int k, int& cnt, float& thr,
+                                               unsigned long long key) {
+  int pos = cnt < k ? cnt : k - 1;
+  while (pos > 0 && list[pos - 1][r] < key) { list[pos][r] = list[pos - 1][r]; --pos; }
+  list[pos][r] = key;
+  cnt = cnt < k ? cnt + 1 : k;
+  if (cnt == k) thr = key_val(list[k - 1][r]);
+}
+
 __global__ void __launch_bounds__(LM_THREADS, 1)
 k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w, int rows, int d,
-               int V, int k, LmParts parts, int* __restrict__ fail_flag) {
+               int V, int k, int a_rows, int n_stages, LmParts parts, int* __restrict__ fail_flag) {
   extern __shared__ __align__(1024) unsigned char lm_smem_raw[];
   unsigned char* ring = lm_smem_raw;
-  LmShared& sh = *reinterpret_cast<LmShared*>(lm_smem_raw + LM_STAGES * LM_STAGE_BYTES);
+  LmShared& sh = *reinterpret_cast<LmShared*>(lm_smem_raw + LM_RING_BYTES);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = gridDim.x, cta = blockIdx.x;
-  const int n_rt = (rows + LM_BM - 1) / LM_BM, n_vt = (V + LM_BN - 1) / LM_BN, n_kb = d / LM_BK;
-  const int my_vt = cta < n_vt ? (n_vt - cta + G - 1) / G : 0;   // vocabulary tiles cta, cta + G, ...
-  const int n_items = my_vt * n_rt;
+  const int n_rb = (rows + LM_RB - 1) / LM_RB, n_vt = (V + LM_BN - 1) / LM_BN, n_kb = d / LM_BK;
+  const int a_bytes = a_rows * LM_BK * 2, stage_bytes = a_bytes + LM_B_BYTES;
+  // work items: (vocabulary tile, row block) pairs, row block fastest, dealt round-robin: cta, cta + G, ...
+  const int n_all = n_vt * n_rb;
+  const int n_items = cta < n_all ? (n_all - cta + G - 1) / G : 0;
   volatile int* fail = &sh.fail;
 
   if (tid == 0) {
-    for (int s = 0; s < LM_STAGES; ++s) { lm_bar_init(&sh.full[s], 1); lm_bar_init(&sh.empty[s], 1); }
+    for (int s = 0; s < LM_MAX_STAGES; ++s) { lm_bar_init(&sh.full[s], 1); lm_bar_init(&sh.empty[s], 1); }
     for (int a = 0; a < 2; ++a) { lm_bar_init(&sh.acc_full[a], 1); lm_bar_init(&sh.acc_empty[a], 4); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     sh.fail = 0;
-  }
-  for (int i = tid; i < LM_MAX_RT * LM_BM; i += LM_THREADS) {
-    (&sh.m[0][0])[i] = -1.0e30f; (&sh.s[0][0])[i] = 0.f; (&sh.thr[0][0])[i] = -INFINITY; (&sh.cnt[0][0])[i] = 0;
   }
   if (warp == 1) {  // tensor memory: both accumulators (512 columns), allocated by one warp
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(lm_smem(&sh.tmem_base)), "r"(512u) : "memory");
@@ -159,116 +177,153 @@ k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant_
     if (lane == 0) {
       int it = 0;
       for (int item = 0; item < n_items && !*fail; ++item) {
-        const int vt = cta + (item / n_rt) * G, rt = item % n_rt;
+        const int g = cta + item * G, vt = g / n_rb, rb = g % n_rb;
         for (int kb = 0; kb < n_kb; ++kb, ++it) {
-          const int s = it % LM_STAGES;
-          const uint32_t ph = (uint32_t)(it / LM_STAGES) & 1u;
+          const int s = it % n_stages;
+          const uint32_t ph = (uint32_t)(it / n_stages) & 1u;
           if (!lm_bar_wait(&sh.empty[s], ph ^ 1u, fail)) break;
-          lm_bar_expect(&sh.full[s], LM_STAGE_BYTES);
-          unsigned char* a = ring + (size_t)s * LM_STAGE_BYTES;
-          lm_tma_load(a, &map_h, kb * LM_BK, rt * LM_BM, &sh.full[s]);
-          lm_tma_load(a + LM_A_BYTES, &map_w, kb * LM_BK, vt * LM_BN, &sh.full[s]);
+          lm_bar_expect(&sh.full[s], (uint32_t)stage_bytes);
+          unsigned char* a = ring + (size_t)s * stage_bytes;
+          lm_tma_load(a, &map_h, kb * LM_BK, rb * LM_RB, &sh.full[s]);
+          lm_tma_load(a + a_bytes, &map_w, kb * LM_BK, vt * LM_BN, &sh.full[s]);
         }
       }
       if (*fail)  // gave up: before the CTA leaves, wait (bounded) for the copies still landing in its ring
-        for (int i = it > LM_STAGES ? it - LM_STAGES : 0; i < it; ++i)
-          lm_bar_wait(&sh.full[i % LM_STAGES], (uint32_t)(i / LM_STAGES) & 1u, fail);
+        for (int i = it > n_stages ? it - n_stages : 0; i < it; ++i)
+          lm_bar_wait(&sh.full[i % n_stages], (uint32_t)(i / n_stages) & 1u, fail);
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
       int it = 0;
+      uint32_t use[2] = {0u, 0u};  // how often each accumulator has been handed over
       for (int item = 0; item < n_items && !*fail; ++item) {
-        const int ab = item & 1;
-        const uint32_t aph = (uint32_t)(item >> 1) & 1u;
-        if (!lm_bar_wait(&sh.acc_empty[ab], aph ^ 1u, fail)) break;  // the epilogue has drained this accumulator
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t d_tmem = tmem + (uint32_t)(ab * LM_BN);
+        const int rb = (cta + item * G) % n_rb;
+        const int n_half = rows - rb * LM_RB > LM_BM ? 2 : 1;  // a row block of at most 128 rows fills one accumulator
         bool ok = true;
         for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
-          const int s = it % LM_STAGES;
-          const uint32_t ph = (uint32_t)(it / LM_STAGES) & 1u;
+          const int s = it % n_stages;
+          const uint32_t ph = (uint32_t)(it / n_stages) & 1u;
           ok = lm_bar_wait(&sh.full[s], ph, fail);
           if (!ok) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t a_addr = lm_smem(ring + (size_t)s * LM_STAGE_BYTES), b_addr = a_addr + LM_A_BYTES;
+          const uint32_t a_addr = lm_smem(ring + (size_t)s * stage_bytes), b_addr = a_addr + (uint32_t)a_bytes;
 #pragma unroll
-          for (int kk = 0; kk < LM_BK / 16; ++kk)  // 16 bf16 = 32 bytes along K inside the swizzled row
-            lm_mma(d_tmem, lm_desc(a_addr + kk * 32), lm_desc(b_addr + kk * 32), (kb | kk) != 0 ? 1u : 0u);
+          for (int half = 0; half < 2; ++half) {  // rows 0-127 -> accumulator 0, rows 128-255 -> accumulator 1
+            if (half >= n_half) break;
+            if (kb == 0) {  // the epilogue has drained this accumulator
+              ok = lm_bar_wait(&sh.acc_empty[half], (use[half] & 1u) ^ 1u, fail);
+              if (!ok) break;
+              asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            }
+            const uint32_t d_tmem = tmem + (uint32_t)(half * LM_BN);
+            const uint32_t ah = a_addr + (uint32_t)(half * LM_BM * LM_BK * 2);
+#pragma unroll
+            for (int kk = 0; kk < LM_BK / 16; ++kk)  // 16 bf16 = 32 bytes along K inside the swizzled row
+              lm_mma(d_tmem, lm_desc(ah + kk * 32), lm_desc(b_addr + kk * 32), (kb | kk) != 0 ? 1u : 0u);
+          }
+          if (!ok) break;
           lm_commit(&sh.empty[s]);  // the stage may be refilled once these MMAs have read it
         }
         if (!ok) break;
-        lm_commit(&sh.acc_full[ab]);  // the accumulator is complete once every MMA above is
+        for (int half = 0; half < n_half; ++half) {  // complete once every MMA above is
+          lm_commit(&sh.acc_full[half]);
+          use[half] += 1u;
+        }
       }
     }
   } else {
-    // ---------------------------------------------------------------- epilogue: thread = row of the tile
+    // ---------------------------------------------------------------- epilogue: thread = row of one accumulator
+    const int half = (warp - 2) >> 2;
     const int lg = warp & 3;                      // the TMEM lanes this warp may read: 32 * (warp % 4) ...
     const int r_in_tile = lg * 32 + lane;
+    unsigned long long(*list)[LM_BM] = sh.list[half];  // list[i][r_in_tile] = i-th best of this thread's row
+    const uint32_t taddr = tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)(half * LM_BN);
+    unsigned long long visited = 0ull;            // row blocks this CTA has a partial for already
+    uint32_t use = 0u;
+    bool ok = true;
     for (int item = 0; item < n_items && !*fail; ++item) {
-      const int vt = cta + (item / n_rt) * G, rt = item % n_rt;
-      const int ab = item & 1;
-      const uint32_t aph = (uint32_t)(item >> 1) & 1u;
-      if (!lm_bar_wait(&sh.acc_full[ab], aph, fail)) break;
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int row = rt * LM_BM + r_in_tile;
-      float m = sh.m[rt][r_in_tile], ssum = sh.s[rt][r_in_tile], thr = sh.thr[rt][r_in_tile];
-      int cnt = sh.cnt[rt][r_in_tile];
-      unsigned long long* list = parts.list + ((size_t)cta * parts.rpad + row) * k;
-      const uint32_t taddr = tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)(ab * LM_BN);
+      const int g = cta + item * G, vt = g / n_rb, rb = g % n_rb;
+      if (half == 1 && rows - rb * LM_RB <= LM_BM) continue;  // this item leaves the second accumulator unused
+      const uint32_t aph = use & 1u;
+      use += 1u;
+      const bool first = !((visited >> rb) & 1ull);
+      visited |= 1ull << rb;
       const int col_base = vt * LM_BN;
+      const int row = rb * LM_RB + half * LM_BM + r_in_tile;
+      const bool valid = row < rows;
+      const size_t slot = (size_t)cta * parts.rpad + row;
+      // the row's running state: from the workspace unless this is the CTA's first visit of the row block
+      float m = -1.0e30f, ssum = 0.f;
+      int cnt = 0;
+      if (!first && valid) {
+        m = parts.ms[slot * 2]; ssum = parts.ms[slot * 2 + 1]; cnt = parts.cnt[slot];
+        for (int i = 0; i < cnt; ++i) list[i][r_in_tile] = parts.list[slot * k + i];
+      }
+      float thr = cnt == k ? key_val(list[k - 1][r_in_tile]) : -INFINITY;
+      ok = lm_bar_wait(&sh.acc_full[half], aph, fail);
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll 1
       for (int c0 = 0; c0 < LM_BN; c0 += 32) {
         uint32_t r[32];
         lm_tmem_ld32(taddr + (uint32_t)c0, r);
         const int ncol = V - (col_base + c0);     // columns of this chunk that exist (the last tile is ragged)
-        if (ncol <= 0 || row >= rows) continue;   // (every lane still took part in the load above)
-        float cm = -INFINITY;
+        if (ncol <= 0 || !valid) continue;        // (every lane still took part in the load above)
+        if (ncol < 32) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float x = __uint_as_float(r[j]);
-          if (j < ncol) cm = fmaxf(cm, x);
+          for (int j = 0; j < 32; ++j)
+            if (j >= ncol) r[j] = 0xff800000u;    // -inf: adds nothing to the sum, never chosen
         }
+        float cm = __uint_as_float(r[0]);
+#pragma unroll
+        for (int j = 1; j < 32; ++j) cm = fmaxf(cm, __uint_as_float(r[j]));
         if (cm > m) {  // online log-sum-exp: move the running maximum up
-          ssum *= exp2f((m - cm) * kLog2e);
+          ssum *= ex2_approx((m - cm) * kLog2e);
           m = cm;
         }
         const float negm = -m * kLog2e;
+        float s0 = 0.f, s1 = 0.f;
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const float x = __uint_as_float(r[j]);
-          if (j < ncol) ssum += exp2f(fmaf(x, kLog2e, negm));
+        for (int j = 0; j < 32; j += 2) {
+          s0 += ex2_approx(fmaf(__uint_as_float(r[j]), kLog2e, negm));
+          s1 += ex2_approx(fmaf(__uint_as_float(r[j + 1]), kLog2e, negm));
         }
-        if (cm > thr || cnt < k) {  // some logit of the chunk enters the row's list
-#pragma unroll 1
-          for (int j = 0; j < 32 && j < ncol; ++j) {
-            const float x = __uint_as_float(r[j]);
-            if (!(x > thr) && cnt >= k) continue;   // columns ascend: an equal value loses to the one already kept
-            const unsigned long long key = make_key(x, col_base + c0 + j);
-            int pos = cnt < k ? cnt : k - 1;        // a full list drops its last entry
-            while (pos > 0 && list[pos - 1] < key) { list[pos] = list[pos - 1]; --pos; }
-            list[pos] = key;
-            cnt = cnt < k ? cnt + 1 : k;
-            if (cnt == k) thr = key_val(list[k - 1]);
-          }
+        ssum += s0 + s1;
+        if (cm > thr || cnt < k) {  // some logit of the chunk enters the row's list: take them best first
+          uint32_t avail = ncol < 32 ? (1u << ncol) - 1u : 0xffffffffu;
+          do {
+            float best = -INFINITY;
+            int bj = -1;
+#pragma unroll
+            for (int j = 31; j >= 0; --j) {  // ">=" on the way down: of equal values the lowest column wins
+              const float x = __uint_as_float(r[j]);
+              if (((avail >> j) & 1u) && x >= best) { best = x; bj = j; }
+            }
+            // an equal value loses to the one already kept: columns ascend over a CTA's visits of a row
+            if (bj < 0 || (cnt >= k && !(best > thr))) break;
+            lm_list_insert(list, r_in_tile, k, cnt, thr, make_key(best, col_base + c0 + bj));
+            avail &= ~(1u << bj);
+          } while (avail);
         }
-      }
-      if (row < rows) {
-        sh.m[rt][r_in_tile] = m; sh.s[rt][r_in_tile] = ssum; sh.thr[rt][r_in_tile] = thr;
-        sh.cnt[rt][r_in_tile] = (unsigned char)cnt;
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
-      if (lane == 0) lm_bar_arrive(&sh.acc_empty[ab]);  // this warp's quarter of the accumulator is drained
+      if (lane == 0) lm_bar_arrive(&sh.acc_empty[half]);  // this warp's quarter of the accumulator is drained
+      if (valid) {  // the row's state goes back to the workspace (the merge reads it from there, too)
+        parts.ms[slot * 2] = m; parts.ms[slot * 2 + 1] = ssum; parts.cnt[slot] = cnt;
+        for (int i = 0; i < cnt; ++i) parts.list[slot * k + i] = list[i][r_in_tile];
+      }
     }
-    // partial of every row this thread owns (all row tiles), for the merge
-    for (int rt = 0; rt < n_rt; ++rt) {
-      const int row = rt * LM_BM + r_in_tile;
+    // rows this CTA never visited (more CTAs than work items) and, after a give-up, every row: empty / marked
+    for (int rb = 0; rb < n_rb; ++rb) {
+      const bool seen = (visited >> rb) & 1ull;
+      if (seen && !*fail) continue;
+      const int row = rb * LM_RB + half * LM_BM + r_in_tile;
       if (row >= rows) continue;
       const size_t slot = (size_t)cta * parts.rpad + row;
-      parts.ms[slot * 2] = sh.m[rt][r_in_tile];
-      parts.ms[slot * 2 + 1] = sh.s[rt][r_in_tile];
-      parts.cnt[slot] = *fail ? -1 : (int)sh.cnt[rt][r_in_tile];
+      if (!seen) { parts.ms[slot * 2] = -1.0e30f; parts.ms[slot * 2 + 1] = 0.f; }
+      parts.cnt[slot] = *fail ? -1 : 0;
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -371,10 +426,11 @@ size_t lm_align(size_t x) { return (x + 255) / 256 * 256; }
 
 int lm_head_max_k() { return LM_MAX_K; }
 
+int lm_head_max_rows() { return LM_MAX_ROWS; }
+
 size_t lm_head_workspace_bytes(int64_t rows, int k) {
   const size_t grid = (size_t)device_info().sm_count;
-  const size_t blk = (size_t)(rows < LM_MAX_RT * LM_BM ? rows : LM_MAX_RT * LM_BM);
-  const size_t rpad = (blk + LM_BM - 1) / LM_BM * LM_BM;
+  const size_t rpad = ((size_t)rows + LM_RB - 1) / LM_RB * LM_RB;
   return 256 + lm_align(grid * rpad * 2 * sizeof(float)) + lm_align(grid * rpad * (size_t)k * 8) +
          lm_align(grid * rpad * sizeof(int32_t));
 }
@@ -384,13 +440,13 @@ cudaError_t launch_lm_head_topk(const void* hidden, const void* weight, int64_t 
                                 int32_t* cand_ids, float* cand_lp, void* ws, cudaStream_t st) {
   if (rows == 0) return cudaSuccess;
   const int grid = device_info().sm_count;
-  const size_t smem = (size_t)LM_STAGES * LM_STAGE_BYTES + sizeof(LmShared);
+  const size_t smem = (size_t)LM_RING_BYTES + sizeof(LmShared);
+  const int a_rows = rows <= LM_BM ? LM_BM : LM_RB, n_stages = rows <= LM_BM ? 4 : 3;
   cudaError_t e = allow_max_dynamic_smem<k_lm_head_topk>();
   if (e != cudaSuccess) return e;
   unsigned char* p = static_cast<unsigned char*>(ws);
   int* fail_flag = reinterpret_cast<int*>(p); p += 256;
-  const int64_t blk_rows = LM_MAX_RT * LM_BM;
-  const size_t rpad = (size_t)((rows < blk_rows ? rows : blk_rows) + LM_BM - 1) / LM_BM * LM_BM;
+  const size_t rpad = ((size_t)rows + LM_RB - 1) / LM_RB * LM_RB;
   LmParts parts{};
   parts.rpad = (int)rpad;
   parts.ms = reinterpret_cast<float*>(p); p += lm_align((size_t)grid * rpad * 2 * sizeof(float));
@@ -398,21 +454,14 @@ cudaError_t launch_lm_head_topk(const void* hidden, const void* weight, int64_t 
   parts.cnt = reinterpret_cast<int32_t*>(p);
   e = cudaMemsetAsync(fail_flag, 0, 256, st);
   if (e != cudaSuccess) return e;
-  CUtensorMap map_w;
+  CUtensorMap map_w, map_h;
   if (!make_map(&map_w, weight, (uint64_t)d, (uint64_t)V, LM_BN)) return cudaErrorNotSupported;
-  for (int64_t r0 = 0; r0 < rows; r0 += blk_rows) {  // blocks of at most 2048 rows (the weight table is re-read per block)
-    const int nr = (int)(rows - r0 < blk_rows ? rows - r0 : blk_rows);
-    CUtensorMap map_h;
-    if (!make_map(&map_h, static_cast<const unsigned char*>(hidden) + (size_t)r0 * d * 2, (uint64_t)d, (uint64_t)nr, LM_BM))
-      return cudaErrorNotSupported;
-    k_lm_head_topk<<<grid, LM_THREADS, smem, st>>>(map_h, map_w, nr, d, V, k, parts, fail_flag);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    k_lm_head_merge<<<(nr + 3) / 4, 128, 0, st>>>(parts, grid, nr, k, cand_ids + (size_t)r0 * k, cand_lp + (size_t)r0 * k);
-    e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-  }
-  return cudaSuccess;
+  if (!make_map(&map_h, hidden, (uint64_t)d, (uint64_t)rows, (uint32_t)a_rows)) return cudaErrorNotSupported;
+  k_lm_head_topk<<<grid, LM_THREADS, smem, st>>>(map_h, map_w, (int)rows, d, V, k, a_rows, n_stages, parts, fail_flag);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  k_lm_head_merge<<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(parts, grid, (int)rows, k, cand_ids, cand_lp);
+  return cudaGetLastError();
 }
 
 cudaError_t lm_head_timeouts(unsigned int* out) { return cudaMemcpyFromSymbol(out, g_lm_timeouts, sizeof *out); }
