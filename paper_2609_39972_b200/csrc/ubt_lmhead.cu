@@ -48,9 +48,6 @@ struct LmShared {  // behind the ring in dynamic shared memory
   uint64_t full[LM_MAX_STAGES], empty[LM_MAX_STAGES], acc_full[2], acc_empty[2];
   uint32_t tmem_base;
   int fail;
-  // the sorted candidate lists of the rows being finished, entry i of all rows side by side (a warp touching
-  // entry i of its 32 rows touches 32 different banks); between two visits a row's list lives in the workspace
-  unsigned long long list[2][LM_MAX_K][LM_BM];
 };
 
 __device__ __forceinline__ uint32_t lm_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -132,16 +129,28 @@ struct LmParts {                   // one partial per (CTA, row of the launch's 
   int rpad;                        // rows of the block rounded up to whole row tiles
 };
 
-// Entry `key` into the row's sorted list (column r of `list`); a full list drops its last entry.
-__device__ __forceinline__ void lm_list_insert(unsigned long long (*list)[LM_BM], int r, int k, int& cnt, float& thr,
-                                               unsigned long long key) {
-  int pos = cnt < k ? cnt : k - 1;
-  while (pos > 0 && list[pos - 1][r] < key) { list[pos][r] = list[pos - 1][r]; --pos; }
-  list[pos][r] = key;
-  cnt = cnt < k ? cnt + 1 : k;
-  if (cnt == k) thr = key_val(list[k - 1][r]);
+// The row's candidate list lives in registers, best first, 0 = no entry (below every key); only its first k
+// entries count.  Every new entry depends on the old list alone, so the KR updates are independent instructions.
+template <int KR>
+__device__ __forceinline__ void lm_list_insert(unsigned long long (&L)[KR], unsigned long long key) {
+#pragma unroll
+  for (int i = KR - 1; i > 0; --i) L[i] = key > L[i] ? (key > L[i - 1] ? L[i - 1] : key) : L[i];
+  L[0] = key > L[0] ? key : L[0];
+}
+// (number of entries among the first k, exclusive threshold = value of the k-th entry or -inf)
+template <int KR>
+__device__ __forceinline__ void lm_list_state(const unsigned long long (&L)[KR], int k, int& cnt, float& thr) {
+  unsigned long long kth = 0ull;
+  cnt = 0;
+#pragma unroll
+  for (int i = 0; i < KR; ++i) {
+    if (i == k - 1) kth = L[i];
+    cnt += (i < k && L[i] != 0ull) ? 1 : 0;
+  }
+  thr = kth != 0ull ? key_val(kth) : -INFINITY;
 }
 
+template <int KR>
 __global__ void __launch_bounds__(LM_THREADS, 1)
 k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w, int rows, int d,
                int V, int k, int a_rows, int n_stages, LmParts parts, int* __restrict__ fail_flag) {
@@ -237,7 +246,6 @@ k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant_
     const int half = (warp - 2) >> 2;
     const int lg = warp & 3;                      // the TMEM lanes this warp may read: 32 * (warp % 4) ...
     const int r_in_tile = lg * 32 + lane;
-    unsigned long long(*list)[LM_BM] = sh.list[half];  // list[i][r_in_tile] = i-th best of this thread's row
     const uint32_t taddr = tmem + ((uint32_t)(lg * 32) << 16) + (uint32_t)(half * LM_BN);
     unsigned long long visited = 0ull;            // row blocks this CTA has a partial for already
     uint32_t use = 0u;
@@ -254,13 +262,13 @@ k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant_
       const bool valid = row < rows;
       const size_t slot = (size_t)cta * parts.rpad + row;
       // the row's running state: from the workspace unless this is the CTA's first visit of the row block
-      float m = -1.0e30f, ssum = 0.f;
+      float m = -1.0e30f, ssum = 0.f, thr;
       int cnt = 0;
-      if (!first && valid) {
-        m = parts.ms[slot * 2]; ssum = parts.ms[slot * 2 + 1]; cnt = parts.cnt[slot];
-        for (int i = 0; i < cnt; ++i) list[i][r_in_tile] = parts.list[slot * k + i];
-      }
-      float thr = cnt == k ? key_val(list[k - 1][r_in_tile]) : -INFINITY;
+      unsigned long long L[KR];
+      if (!first && valid) { m = parts.ms[slot * 2]; ssum = parts.ms[slot * 2 + 1]; cnt = parts.cnt[slot]; }
+#pragma unroll
+      for (int i = 0; i < KR; ++i) L[i] = i < cnt ? parts.list[slot * k + i] : 0ull;
+      lm_list_state(L, k, cnt, thr);
       ok = lm_bar_wait(&sh.acc_full[half], aph, fail);
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -290,9 +298,9 @@ k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant_
           s1 += ex2_approx(fmaf(__uint_as_float(r[j + 1]), kLog2e, negm));
         }
         ssum += s0 + s1;
-        if (cm > thr || cnt < k) {  // some logit of the chunk enters the row's list: take them best first
+        if (cm > thr || cnt < k) {  // some logit of the chunk enters the row's list
           uint32_t avail = ncol < 32 ? (1u << ncol) - 1u : 0xffffffffu;
-          do {
+          while (cnt < k && avail) {  // a short list (the CTA's first columns of the row): fill it best first
             float best = -INFINITY;
             int bj = -1;
 #pragma unroll
@@ -300,11 +308,36 @@ k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant_
               const float x = __uint_as_float(r[j]);
               if (((avail >> j) & 1u) && x >= best) { best = x; bj = j; }
             }
-            // an equal value loses to the one already kept: columns ascend over a CTA's visits of a row
-            if (bj < 0 || (cnt >= k && !(best > thr))) break;
-            lm_list_insert(list, r_in_tile, k, cnt, thr, make_key(best, col_base + c0 + bj));
+            if (bj < 0) break;
+            lm_list_insert(L, make_key(best, col_base + c0 + bj));
+            cnt += 1;
             avail &= ~(1u << bj);
-          } while (avail);
+          }
+          lm_list_state(L, k, cnt, thr);
+          // a full list: the columns above the threshold, in ascending order (an equal value loses to the one
+          // already kept: columns ascend over a CTA's visits of a row, and within this loop)
+          uint32_t q = 0u;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) q |= (__uint_as_float(r[j]) > thr ? 1u : 0u) << j;
+          q &= avail;
+          while (q) {
+            const int j = __ffs((int)q) - 1;
+            q &= q - 1u;
+            uint32_t t16[16], t8[8], t4[4], t2[2];  // r[j] by a tree of selects (the registers cannot be indexed)
+#pragma unroll
+            for (int i = 0; i < 16; ++i) t16[i] = (j & 1) ? r[2 * i + 1] : r[2 * i];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) t8[i] = (j & 2) ? t16[2 * i + 1] : t16[2 * i];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) t4[i] = (j & 4) ? t8[2 * i + 1] : t8[2 * i];
+#pragma unroll
+            for (int i = 0; i < 2; ++i) t2[i] = (j & 8) ? t4[2 * i + 1] : t4[2 * i];
+            const float x = __uint_as_float((j & 16) ? t2[1] : t2[0]);
+            if (x > thr) {
+              lm_list_insert(L, make_key(x, col_base + c0 + j));
+              lm_list_state(L, k, cnt, thr);
+            }
+          }
         }
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -312,7 +345,9 @@ k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant_
       if (lane == 0) lm_bar_arrive(&sh.acc_empty[half]);  // this warp's quarter of the accumulator is drained
       if (valid) {  // the row's state goes back to the workspace (the merge reads it from there, too)
         parts.ms[slot * 2] = m; parts.ms[slot * 2 + 1] = ssum; parts.cnt[slot] = cnt;
-        for (int i = 0; i < cnt; ++i) parts.list[slot * k + i] = list[i][r_in_tile];
+#pragma unroll
+        for (int i = 0; i < KR; ++i)
+          if (i < cnt) parts.list[slot * k + i] = L[i];
       }
     }
     // rows this CTA never visited (more CTAs than work items) and, after a give-up, every row: empty / marked
@@ -442,7 +477,9 @@ cudaError_t launch_lm_head_topk(const void* hidden, const void* weight, int64_t 
   const int grid = device_info().sm_count;
   const size_t smem = (size_t)LM_RING_BYTES + sizeof(LmShared);
   const int a_rows = rows <= LM_BM ? LM_BM : LM_RB, n_stages = rows <= LM_BM ? 4 : 3;
-  cudaError_t e = allow_max_dynamic_smem<k_lm_head_topk>();
+  cudaError_t e = allow_max_dynamic_smem<k_lm_head_topk<4>>();
+  if (e == cudaSuccess) e = allow_max_dynamic_smem<k_lm_head_topk<8>>();
+  if (e == cudaSuccess) e = allow_max_dynamic_smem<k_lm_head_topk<16>>();
   if (e != cudaSuccess) return e;
   unsigned char* p = static_cast<unsigned char*>(ws);
   int* fail_flag = reinterpret_cast<int*>(p); p += 256;
@@ -457,7 +494,12 @@ cudaError_t launch_lm_head_topk(const void* hidden, const void* weight, int64_t 
   CUtensorMap map_w, map_h;
   if (!make_map(&map_w, weight, (uint64_t)d, (uint64_t)V, LM_BN)) return cudaErrorNotSupported;
   if (!make_map(&map_h, hidden, (uint64_t)d, (uint64_t)rows, (uint32_t)a_rows)) return cudaErrorNotSupported;
-  k_lm_head_topk<<<grid, LM_THREADS, smem, st>>>(map_h, map_w, (int)rows, d, V, k, a_rows, n_stages, parts, fail_flag);
+  if (k <= 4)
+    k_lm_head_topk<4><<<grid, LM_THREADS, smem, st>>>(map_h, map_w, (int)rows, d, V, k, a_rows, n_stages, parts, fail_flag);
+  else if (k <= 8)
+    k_lm_head_topk<8><<<grid, LM_THREADS, smem, st>>>(map_h, map_w, (int)rows, d, V, k, a_rows, n_stages, parts, fail_flag);
+  else
+    k_lm_head_topk<16><<<grid, LM_THREADS, smem, st>>>(map_h, map_w, (int)rows, d, V, k, a_rows, n_stages, parts, fail_flag);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   k_lm_head_merge<<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(parts, grid, (int)rows, k, cand_ids, cand_lp);

@@ -32,7 +32,9 @@ def check_rows(ids_g, lp_g, o_ids, o_lp, o_lse, o_logits, k):
     return swaps
 
 
-@pytest.mark.parametrize("rows,d,V,k", [(200, 128, 1000, 8), (300, 256, 5000, 16), (1, 64, 300, 4), (129, 512, 2049, 1)])
+# the last two have more work items than CTAs: a CTA comes back to a row block whose state it parked before
+@pytest.mark.parametrize("rows,d,V,k", [(200, 128, 1000, 8), (300, 256, 5000, 16), (1, 64, 300, 4), (129, 512, 2049, 1),
+                                        (300, 64, 51237, 5), (520, 64, 40000, 16)])
 def test_small_shapes_every_row(rows, d, V, k):
     import paper_2609_39972_b200 as u
     h, w = synth.lm_head_inputs(rows, d, V, seed=rows + d, scale=3.0)
