@@ -55,6 +55,54 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+def measured_tensor_peak():
+    """Dense bf16 TFLOP/s of a library product on this machine: the burst figure, for a kernel timed alone."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured (burst)"
+    except Exception:
+        return 1590.0, "fallback"
+
+
+def measure_lm_head(ubt, dev, rows=512, d=4096, V=151936, k=8, reps=10):
+    """The LM head fused with step a1 (one tensor-core kernel, logits never stored), timed alone with CUDA events,
+    and next to it the unfused route on the same inputs: a library bf16 product that stores the logits, then
+    ubt_topk_logprob.  L2: the weight matrix (1.2 GB) is larger than L2 and every launch reads all of it."""
+    hd, wd = synth.device_lm_head_inputs(rows, d, V, seed=5, device=dev)
+    ids = torch.empty((rows, k), dtype=torch.int32, device=dev)
+    lp = torch.empty((rows, k), dtype=torch.float32, device=dev)
+    ws = ubt.workspace(ubt.ubt_lm_head_workspace_bytes(rows, d, V, k), dev)
+    logits = torch.empty((rows, V), dtype=torch.bfloat16, device=dev)
+    ws_t = ubt.workspace(ubt.ubt_draft_workspace_bytes(rows, 1, V, k, 1), dev)
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    def unfused():
+        torch.matmul(hd, wd.T, out=logits)
+        ubt.ubt_topk_logprob(logits, k, ids, lp, ws_t)
+
+    t_f = timed(lambda: ubt.ubt_lm_head_topk(hd, wd, k, ids, lp, ws))
+    t_u = timed(unfused)
+    flops = 2.0 * rows * d * V
+    peak, kind = measured_tensor_peak()
+    return {"kernel": "k_lm_head_topk", "bound": "tensor", "rows": rows, "d": d, "V": V, "k": k, "dtype": "bf16",
+            "avg_ms": t_f, "achieved": flops / (t_f * 1e-3) / 1e12, "unit": "TFLOP/s", "peak": peak,
+            "peak_source": f"of {kind}", "frac": flops / (t_f * 1e-3) / 1e12 / peak,
+            "unfused_ms": t_u, "unfused": "library bf16 product storing the logits + ubt_topk_logprob",
+            "launches_per_call": 2, "timeouts": ubt.ubt_debug_ring_timeouts()}
+
+
 def recorded_traffic(kernel: str, workload: str):
     """DRAM bytes per launch of `kernel` from the committed ncu summary, if one exists (else None)."""
     path = os.path.join(ROOT, "profiles", "dram_traffic.json")
@@ -433,6 +481,7 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time budget of the oracle baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-lm-head", action="store_true", help="skip the fused LM head measurement (a 'next' row)")
     ap.add_argument("--batch", type=int, default=0, help="override B of the workload (profiling captures only)")
     args = ap.parse_args()
     if args.warmup < 3:
@@ -508,6 +557,11 @@ def main():
         "clocks": st["clocks"],
         "gpu_launches": head["gpu_launches"],
     }
+
+    # ---- a row beyond the timed path: the LM head fused with step a1, timed alone (default run only)
+    if rank == 0 and not args.no_lm_head and args.workload is None and args.batch == 0:
+        line["next_rows"] = {"lm_head_topk": measure_lm_head(ubt, dev)}
+        torch.cuda.empty_cache()
 
     # ---- end to end through the host-buffer entry points (pinned host inputs, results read back)
     if not args.no_e2e:
