@@ -482,6 +482,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-lm-head", action="store_true", help="skip the fused LM head measurement (a 'next' row)")
+    ap.add_argument("--lm-head-only", action="store_true", help="only that measurement (profiling captures)")
     ap.add_argument("--batch", type=int, default=0, help="override B of the workload (profiling captures only)")
     args = ap.parse_args()
     if args.warmup < 3:
@@ -512,6 +513,10 @@ def main():
     dev = torch.device("cuda", local)
     ubt.load()
     stream = torch.cuda.current_stream()
+    if args.lm_head_only:
+        if rank == 0:
+            print(json.dumps({"next_rows": {"lm_head_topk": measure_lm_head(ubt, dev, reps=max(1, args.steps))}}), flush=True)
+        return
 
     # the other workloads first, so that the headline's buffers are the ones kept for the end-to-end legs
     per_workload = {}

@@ -1,20 +1,20 @@
 // Steps a2, a3, a3b: candidate-pair log-probabilities, budgeted tree expansion, tree-attention inputs.
 //
 // One CTA per sequence.  The pair table t[i][ra][.] = log q^bi (eq. 5 + eq. 9) lives in shared memory,
-// every row sorted best first, next to the permutation that sorted it.  Algorithm 1 is run as a best-first
-// search: the frontier holds, per expanded node, its best not-yet-taken child; a pop takes the best
-// frontier entry under the total order (score desc, depth asc, token asc, rank path asc), replaces it by its
-// next sibling and adds its own first child.  Because every pair log-probability is <= 0 and zeta <= 0,
-// scores never increase along a path, so pops come out in the global order; a node popped when its depth
-// already holds W nodes is outside Top_W(E_d) and is dropped with its later siblings.  N-1 accepted pops
-// give Top_B of the supertree (eq. 11-12).
-//
-// The search is a chain of N-1 dependent pops by one warp, so its latency is what counts: the ordering keys of
-// the frontier live in registers (entry i in lane i&31, slot i>>5), the 16-byte records in shared memory; a pop
-// is a register scan, three warp reductions, one 16-byte and four scalar shared-memory loads, and stores that all
-// lanes execute alike (see expand_tree).  Everything around it -- merging the top-k partials, eq. 5 / eq. 9 and
-// the row sorts, slot assignment, masks -- is spread over the CTA's 16 warps.  When the pair table does not fit
-// in shared memory its rows are prepared on demand (k_build_tree<true>, see TreeSmem and lazy_row).
+// every row sorted best first, next to the permutation that sorted it.  Every pair log-probability is <= 0 and
+// zeta <= 0, so scores never increase from a node to its children or to its later siblings; Algorithm 1 (Top_W per
+// depth, eq. 11, then the global Top_B, eq. 12) is evaluated in two equivalent ways that both rest on that:
+//   * threshold rounds (the whole table resident): the nodes that reach a threshold form a set closed under
+//     "parent" and "earlier sibling" that is enumerated in parallel, wave by wave; the threshold falls from round
+//     to round until the set covers the budget, and the budget's best nodes of the last round are chosen under the
+//     total order (score desc, depth asc, token asc, rank path asc).  See expand_rounds_warp / expand_rounds_cta.
+//   * best-first search by one warp (pair table too large for shared memory, rows prepared on demand; also the
+//     fallback when masses of exactly tied scores outgrow the rounds' node arrays): the frontier holds, per
+//     expanded node, its best not-yet-taken child; a pop takes the best entry, replaces it by its next sibling
+//     and adds its own first child, so pops come out in the global order; a node popped when its depth already
+//     holds W nodes is outside Top_W(E_d) and is dropped with its later siblings.  See expand_tree.
+// Everything around the search -- merging the top-k partials, eq. 5 / eq. 9 and the row sorts, slot assignment,
+// masks -- is spread over the CTA's 16 warps.
 #include "ubt_internal.h"
 
 namespace ubt {
