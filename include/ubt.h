@@ -156,6 +156,28 @@ int ubt_topk_logprob(const void *logits, int dtype, int64_t rows, int V, int k, 
                      float *cand_logprob, void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Step a1 with the vocabulary split over the ranks of a tensor-parallel group (the paper serves with the LM
+ * head, and so every logits row, sharded over the vocabulary; Section 3.1.1 defines the candidates on the whole
+ * row).  Rank r holds the columns [v0, v0 + Vs) of every row as a dense [rows, Vs] tensor and calls
+ * ubt_topk_shard, which writes its per-row partial: (max, sum of exp relative to it), the k best values of the
+ * slice (raw logits, best first) with their token ids in the WHOLE vocabulary (column + v0), and how many there
+ * are.  The partial is one buffer of ubt_topk_shard_bytes(rows, k) bytes (the same for every rank; four arrays,
+ * each 256-byte aligned: float[rows,2], float[rows,k], int32[rows,k], int32[rows]).  The caller gathers the
+ * partials of all ranks back to back in rank order -- one all-gather of rows * (8k + 12) bytes, padding aside --
+ * and every rank calls ubt_topk_merge_shards on the gathered buffer, which gives cand_ids / cand_logprob exactly
+ * as ubt_topk_logprob would on the whole rows (same ordering, ties to the lower token id; the log-sum-exp is
+ * summed in a different order, so log-probabilities agree to fp32 rounding).  Slices may differ in width; every
+ * slice needs Vs >= k.  A slice whose streaming kernel gave up a wait has count -1 for the rows concerned; the
+ * merge then treats its list as empty (ubt_debug_ring_timeouts tells).  No collective is issued by the library.
+ * Workspace of ubt_topk_shard: ubt_draft_workspace_bytes(rows, 1, Vs, k, 1).
+ */
+size_t ubt_topk_shard_bytes(int64_t rows, int k);
+int ubt_topk_shard(const void *logits_shard, int dtype, int64_t rows, int Vs, int k, int v0, void *partial,
+                   void *workspace, size_t workspace_bytes, void *cuda_stream);
+int ubt_topk_merge_shards(const void *gathered, int shards, int64_t rows, int k, int32_t *cand_ids,
+                          float *cand_logprob, void *cuda_stream);
+
+/*
  * The proposer's LM head fused with step a1 (Section 3.1.1, eq. 3: the unigram logits of a position are the
  * frozen LM head applied to the position's hidden state; the paper times this projection inside its draft
  * post-processing stage, appendix "Drafting Latency Analysis").  For each of `rows` hidden states:

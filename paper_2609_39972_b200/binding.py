@@ -57,7 +57,8 @@ EXPORTS = ["ubt_version", "ubt_status_string", "ubt_debug_ring_timeouts", "ubt_d
            "ubt_topk_logprob", "ubt_selector_scores", "ubt_build_tree", "ubt_build_mask", "ubt_draft_tree", "ubt_verify_tree",
            "ubt_draft_host_buffer_bytes", "ubt_verify_host_buffer_bytes", "ubt_draft_tree_host",
            "ubt_verify_tree_host", "ubt_verify_tree_static", "ubt_verify_static_capacity", "ubt_lm_head_workspace_bytes",
-           "ubt_lm_head_topk"]
+           "ubt_lm_head_topk", "ubt_topk_shard_bytes", "ubt_topk_shard", "ubt_topk_merge_shards",
+           "gather_shard_partials", "topk_logprob_vocab_parallel"]
 
 _lib = None
 
@@ -103,6 +104,11 @@ def load() -> C.CDLL:
     L.ubt_lm_head_workspace_bytes.argtypes = [C.c_int64, C.c_int, C.c_int, C.c_int]
     L.ubt_lm_head_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
                                    C.c_void_p, C.c_size_t, C.c_void_p]
+    L.ubt_topk_shard_bytes.restype = C.c_size_t
+    L.ubt_topk_shard_bytes.argtypes = [C.c_int64, C.c_int]
+    L.ubt_topk_shard.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
+                                 C.c_size_t, C.c_void_p]
+    L.ubt_topk_merge_shards.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
     L.ubt_debug_ring_timeouts.restype = C.c_longlong
     L.ubt_draft_tree_host.argtypes = L.ubt_draft_tree.argtypes
     L.ubt_verify_tree_host.argtypes = L.ubt_verify_tree.argtypes
@@ -232,6 +238,66 @@ def ubt_topk_logprob(logits: torch.Tensor, k: int, cand_ids: torch.Tensor, cand_
     _check(load().ubt_topk_logprob(_ptr(logits), _dtype_code(logits), rows, V, k, _ptr(_need(cand_ids, "cand_ids")),
                                    _ptr(_need(cand_logprob, "cand_logprob")), _ptr(ws), ws.numel(), _stream(stream)),
            "ubt_topk_logprob")
+
+
+def ubt_topk_shard_bytes(rows: int, k: int) -> int:
+    return int(load().ubt_topk_shard_bytes(rows, k))
+
+
+def ubt_topk_shard(logits_shard: torch.Tensor, k: int, v0: int, partial: Optional[torch.Tensor] = None,
+                   ws: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Step a1 on this rank's slice of the vocabulary (columns ``v0 ...`` of every row, dense ``[..., Vs]``):
+    returns the rank's per-row partial, a uint8 buffer of ``ubt_topk_shard_bytes(rows, k)`` bytes."""
+    _need(logits_shard, "logits_shard")
+    Vs = logits_shard.shape[-1]
+    rows = logits_shard.numel() // Vs
+    if partial is None:
+        partial = workspace(ubt_topk_shard_bytes(rows, k), logits_shard.device)
+    if ws is None:
+        ws = workspace(ubt_draft_workspace_bytes(rows, 1, Vs, k, 1), logits_shard.device)
+    _check(load().ubt_topk_shard(_ptr(logits_shard), _dtype_code(logits_shard), rows, Vs, k, int(v0), _ptr(partial),
+                                 _ptr(ws), ws.numel(), _stream(stream)), "ubt_topk_shard")
+    return partial
+
+
+def ubt_topk_merge_shards(gathered: torch.Tensor, shards: int, rows: int, k: int,
+                          cand_ids: Optional[torch.Tensor] = None, cand_logprob: Optional[torch.Tensor] = None,
+                          stream=None):
+    """Candidates of the whole rows from the partials of all ranks, back to back in rank order."""
+    _need(gathered, "gathered")
+    if gathered.numel() * gathered.element_size() < shards * ubt_topk_shard_bytes(rows, k):
+        raise ValueError("gathered buffer is smaller than shards * ubt_topk_shard_bytes(rows, k)")
+    if cand_ids is None:
+        cand_ids = torch.empty((rows, k), dtype=torch.int32, device=gathered.device)
+    if cand_logprob is None:
+        cand_logprob = torch.empty((rows, k), dtype=torch.float32, device=gathered.device)
+    _check(load().ubt_topk_merge_shards(_ptr(gathered), shards, rows, k, _ptr(_need(cand_ids, "cand_ids")),
+                                        _ptr(_need(cand_logprob, "cand_logprob")), _stream(stream)),
+           "ubt_topk_merge_shards")
+    return cand_ids, cand_logprob
+
+
+def gather_shard_partials(partial: torch.Tensor, group=None) -> tuple:
+    """All-gather of the ranks' partials in rank order (NCCL for device buffers): ``(gathered, shards)``.  Without
+    an initialised process group the single partial is the gathered buffer."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return partial, 1
+    shards = dist.get_world_size(group)
+    gathered = torch.empty((shards * partial.numel(),), dtype=partial.dtype, device=partial.device)
+    dist.all_gather_into_tensor(gathered, partial.contiguous().view(-1), group=group)
+    return gathered, shards
+
+
+def topk_logprob_vocab_parallel(logits_shard: torch.Tensor, k: int, v0: int, group=None):
+    """Step a1 of rows whose vocabulary is split over the ranks of ``group``: local partial, one all-gather,
+    merge, all on torch's current stream.  Every rank returns the same ``(cand_ids[rows, k],
+    cand_logprob[rows, k])``."""
+    Vs = logits_shard.shape[-1]
+    rows = logits_shard.numel() // Vs
+    partial = ubt_topk_shard(logits_shard, k, v0)
+    gathered, shards = gather_shard_partials(partial, group)
+    return ubt_topk_merge_shards(gathered, shards, rows, k)
 
 
 def ubt_lm_head_workspace_bytes(rows: int, d: int, V: int, k: int) -> int:

@@ -171,6 +171,40 @@ int ubt_topk_logprob(const void* logits, int dtype, int64_t rows, int V, int k, 
   return UBT_OK;
 }
 
+size_t ubt_topk_shard_bytes(int64_t rows, int k) {
+  if (rows < 0 || k < 1 || k > kMaxK) return 0;
+  return shard_partial_bytes(rows, k);
+}
+
+int ubt_topk_shard(const void* logits_shard, int dtype, int64_t rows, int Vs, int k, int v0, void* partial,
+                   void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!logits_shard || !partial || rows < 0 || Vs < 1 || k < 1 || k > Vs || v0 < 0) return UBT_ERR_INVALID_ARG;
+  if (dtype != UBT_F32 && dtype != UBT_BF16) return UBT_ERR_INVALID_ARG;
+  if (!aligned16(logits_shard) || !aligned16(partial)) return UBT_ERR_INVALID_ARG;
+  if (k > kMaxK || (int64_t)v0 + Vs > 0x7fffffffll) return UBT_ERR_UNSUPPORTED;
+  if (rows == 0) return UBT_OK;
+  if (!workspace || !aligned16(workspace) || workspace_bytes < topk_workspace_bytes(rows, Vs, k))
+    return UBT_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  TopkWorkspace w = carve_topk_workspace(workspace, rows, Vs, k);
+  if (launch_lse_topk(logits_shard, dtype, rows, Vs, k, w, st) != cudaSuccess) return UBT_ERR_CUDA;
+  const cudaError_t e = launch_merge_topk_shard(rows, Vs, k, w, partial, v0, st);
+  if (e != cudaSuccess) { cudaGetLastError(); return e == cudaErrorNotSupported ? UBT_ERR_UNSUPPORTED : UBT_ERR_CUDA; }
+  return UBT_OK;
+}
+
+int ubt_topk_merge_shards(const void* gathered, int shards, int64_t rows, int k, int32_t* cand_ids,
+                          float* cand_logprob, void* cuda_stream) {
+  if (!gathered || !cand_ids || !cand_logprob || shards < 1 || rows < 0 || k < 1) return UBT_ERR_INVALID_ARG;
+  if (!aligned16(gathered) || !aligned16(cand_ids) || !aligned16(cand_logprob)) return UBT_ERR_INVALID_ARG;
+  if (k > kMaxK) return UBT_ERR_UNSUPPORTED;
+  if (rows == 0) return UBT_OK;
+  const cudaError_t e = launch_merge_shards(gathered, shards, rows, k, cand_ids, cand_logprob,
+                                            static_cast<cudaStream_t>(cuda_stream));
+  if (e != cudaSuccess) { cudaGetLastError(); return e == cudaErrorNotSupported ? UBT_ERR_UNSUPPORTED : UBT_ERR_CUDA; }
+  return UBT_OK;
+}
+
 size_t ubt_lm_head_workspace_bytes(int64_t rows, int d, int V, int k) {
   if (rows < 0 || d < 1 || V < 1 || k < 1 || k > V || k > lm_head_max_k() || d % 64 != 0 || rows > lm_head_max_rows())
     return 0;

@@ -78,6 +78,12 @@ cudaError_t launch_lse_topk(const void* logits, int dtype, int64_t rows, int V, 
                             const TopkWorkspace& w, cudaStream_t st);
 cudaError_t launch_merge_topk(int64_t rows, int V, int k, const TopkWorkspace& w, int32_t* cand_ids,
                               float* cand_lp, cudaStream_t st);
+// Vocabulary-parallel a1: this rank's per-row partial from its slice, and the merge of the gathered partials.
+size_t shard_partial_bytes(int64_t rows, int k);
+cudaError_t launch_merge_topk_shard(int64_t rows, int V, int k, const TopkWorkspace& w, void* partial, int v0,
+                                    cudaStream_t st);
+cudaError_t launch_merge_shards(const void* gathered, int shards, int64_t rows, int k, int32_t* cand_ids,
+                                float* cand_lp, cudaStream_t st);
 inline MergeParts merge_parts(const TopkWorkspace& w) {
   return MergeParts{w.plan, w.part_ms, w.part_val, w.part_idx, w.part_cnt};
 }

@@ -138,4 +138,119 @@ __device__ __forceinline__ int merge_row_warp(const MergeParts& p, int64_t rows,
   return ((lse == lse && lse < INFINITY) ? 0 : kStatusNonFinite) | (gave_up ? kStatusWaitGaveUp : 0);
 }
 
+// ---------------------------------------------------------------------------------------- one CTA per row
+// The same merge by a whole CTA with the lists staged in shared memory, for rows with many entries (large k, many
+// segments) and for the two ends of a vocabulary-parallel a1:
+//   * source: the segment partials of this GPU's streaming kernel (`shards` == 0), or `shards` per-row partials
+//     gathered from the ranks of a vocabulary-parallel group, rank r's arrays `shard_bytes` * r bytes behind rank
+//     0's ([rows,2] (max, sum exp), [rows,k] values, [rows,k] token ids of the whole vocabulary, [rows] counts);
+//   * result: the row's candidates (ids, value - log-sum-exp of the row), or, with MergeShardOut::ms set, this
+//     rank's per-row partial in that format: raw values, ids moved by `id_offset` (the first column of the rank's
+//     slice), (max, sum exp) and the count (-1 if a streaming CTA of the row gave up a wait).
+struct MergeSource {
+  MergeParts parts;
+  int shards;
+  int64_t shard_bytes;
+};
+struct MergeShardOut {
+  float* ms;
+  float* val;
+  int32_t* idx;
+  int32_t* cnt;
+  int id_offset;
+};
+
+// s_key: [lists * k] keys, s_cnt: [lists], s_red: [2]; every thread of the CTA calls this for the same row.
+template <int THREADS>
+__device__ __forceinline__ void merge_row_cta(const MergeSource& src, int64_t rows, int64_t row, int V, int k,
+                                              int32_t* __restrict__ cand_ids, float* __restrict__ cand_lp,
+                                              const MergeShardOut& so, unsigned long long* s_key, int* s_cnt,
+                                              float* s_red) {
+  const MergeParts& p = src.parts;
+  const int tid = threadIdx.x, lane = tid & 31;
+  int nseg;
+  int64_t base = 0;
+  if (src.shards) {
+    nseg = src.shards;
+  } else {
+    const int64_t c_first = (row * (int64_t)V) / p.plan.span;
+    const int64_t c_last = ((row + 1) * (int64_t)V - 1) / p.plan.span;
+    nseg = (int)(c_last - c_first + 1);
+    base = row * p.plan.smax;
+  }
+  auto shard = [&](const void* a, int j) { return static_cast<const char*>(a) + (int64_t)j * src.shard_bytes; };
+  auto ms_of = [&](int j) {
+    return src.shards ? reinterpret_cast<const float*>(shard(p.part_ms, j)) + row * 2 : p.part_ms + (base + j) * 2;
+  };
+  auto val_of = [&](int j) {
+    return src.shards ? reinterpret_cast<const float*>(shard(p.part_val, j)) + row * k : p.part_val + (base + j) * k;
+  };
+  auto idx_of = [&](int j) {
+    return src.shards ? reinterpret_cast<const int32_t*>(shard(p.part_idx, j)) + row * k : p.part_idx + (base + j) * k;
+  };
+  auto cnt_of = [&](int j) {
+    return src.shards ? reinterpret_cast<const int32_t*>(shard(p.part_cnt, j))[row] : p.part_cnt[base + j];
+  };
+
+  for (int j = tid; j < nseg; j += THREADS) s_cnt[j] = cnt_of(j);
+  __syncthreads();
+  const int nq = nseg * k;
+  for (int q = tid; q < nq; q += THREADS) {
+    const int j = q / k, i = q - j * k;
+    s_key[q] = i < s_cnt[j] ? make_key(val_of(j)[i], idx_of(j)[i]) : 0ull;  // slots beyond the count hold stale data
+  }
+  if (tid < 32) {
+    float M = -1.0e30f;
+    for (int j = lane; j < nseg; j += 32) M = fmaxf(M, ms_of(j)[0]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(FULL, M, o));
+    float S = 0.f;
+    for (int j = lane; j < nseg; j += 32) S += ms_of(j)[1] * exp2f((ms_of(j)[0] - M) * kLog2e);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) S += __shfl_xor_sync(FULL, S, o);
+    if (lane == 0) { s_red[0] = M; s_red[1] = S; }
+  }
+  __syncthreads();
+  const float M = s_red[0], S = s_red[1];
+  const float sub = so.ms ? 0.f : M + logf(S);
+  int32_t* ids_out = so.ms ? so.idx : cand_ids;
+  float* val_out = so.ms ? so.val : cand_lp;
+  // every list is sorted best first: an entry's rank is its place in its own list plus, per other list, the
+  // number of better keys there (binary search); keys are unique, so ranks are
+  for (int q = tid; q < nq; q += THREADS) {
+    const unsigned long long key = s_key[q];
+    if (key == 0ull) continue;
+    const int j = q / k;
+    int rank = q - j * k;
+    for (int j2 = 0; j2 < nseg && rank < k; ++j2) {
+      if (j2 == j) continue;
+      int lo = 0, hi = s_cnt[j2] < 0 ? 0 : s_cnt[j2];  // list[0..lo) > key, list[hi..) < key
+      while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (s_key[j2 * k + mid] > key) lo = mid + 1;
+        else hi = mid;
+      }
+      rank += lo;
+    }
+    if (rank < k) {
+      ids_out[row * k + rank] = key_idx(key) + so.id_offset;
+      val_out[row * k + rank] = key_val(key) - sub;
+    }
+  }
+  int found = 0, gave_up = 0;
+  for (int j = 0; j < nseg; ++j) {
+    gave_up |= s_cnt[j] < 0;
+    found += s_cnt[j] < 0 ? 0 : s_cnt[j];
+  }
+  for (int r = found + tid; r < k; r += THREADS) {  // fewer than k entries in the whole row
+    ids_out[row * k + r] = -1;
+    val_out[row * k + r] = -INFINITY;
+  }
+  if (so.ms && tid == 0) {
+    so.ms[row * 2] = M;
+    so.ms[row * 2 + 1] = S;
+    so.cnt[row] = gave_up ? -1 : (found < k ? found : k);
+  }
+}
+
 }  // namespace ubt

@@ -599,6 +599,19 @@ k_merge_topk(MergeParts parts, int64_t rows, int V, int k, int32_t* __restrict__
   merge_row_warp(parts, rows, row, V, k, cand_ids, cand_lp, threadIdx.x & 31);
 }
 
+// One CTA per row, lists staged in shared memory (see merge_row_cta in ubt_merge.cuh).
+constexpr int MERGE_CTA_T = 128;
+__global__ void __launch_bounds__(MERGE_CTA_T)
+k_merge_topk_cta(MergeSource src, int64_t rows, int V, int k, int32_t* __restrict__ cand_ids,
+                 float* __restrict__ cand_lp, MergeShardOut so) {
+  extern __shared__ __align__(16) unsigned char merge_smem[];
+  const int lists = src.shards ? src.shards : src.parts.plan.smax;
+  unsigned long long* s_key = reinterpret_cast<unsigned long long*>(merge_smem);
+  int* s_cnt = reinterpret_cast<int*>(s_key + (size_t)lists * k);
+  float* s_red = reinterpret_cast<float*>(s_cnt + lists);
+  merge_row_cta<MERGE_CTA_T>(src, rows, blockIdx.x, V, k, cand_ids, cand_lp, so, s_key, s_cnt, s_red);
+}
+
 // ------------------------------------------------------------------------------------ host side
 SpanPlan make_span_plan(int64_t rows, int V, int ctas, int64_t min_span) {
   SpanPlan p;
@@ -672,8 +685,58 @@ cudaError_t launch_lse_topk(const void* logits, int dtype, int64_t rows, int V, 
   return launch_lse_topk_t<float, 1>(logits, rows, V, k, w, st);
 }
 
+static cudaError_t launch_merge_cta(const MergeSource& src, int64_t rows, int V, int k, int32_t* cand_ids,
+                                    float* cand_lp, const MergeShardOut& so, cudaStream_t st) {
+  if (rows == 0) return cudaSuccess;
+  const int lists = src.shards ? src.shards : src.parts.plan.smax;
+  const size_t smem = (size_t)lists * k * 8 + (size_t)lists * 4 + 16;
+  if (smem > (size_t)device_info().max_smem_optin) return cudaErrorNotSupported;
+  cudaError_t e = allow_max_dynamic_smem<k_merge_topk_cta>();
+  if (e != cudaSuccess) return e;
+  k_merge_topk_cta<<<(unsigned)rows, MERGE_CTA_T, smem, st>>>(src, rows, V, k, cand_ids, cand_lp, so);
+  return cudaGetLastError();
+}
+
+size_t shard_partial_bytes(int64_t rows, int k) {
+  return align_up((size_t)rows * 2 * sizeof(float), 256) + 2 * align_up((size_t)rows * k * 4, 256) +
+         align_up((size_t)rows * sizeof(int32_t), 256);
+}
+// The four arrays of one rank's partial: (max, sum exp) [rows,2], values [rows,k], ids [rows,k], counts [rows].
+static MergeShardOut carve_shard_partial(void* partial, int64_t rows, int k, int id_offset) {
+  unsigned char* p = static_cast<unsigned char*>(partial);
+  MergeShardOut so{};
+  so.ms = reinterpret_cast<float*>(p); p += align_up((size_t)rows * 2 * sizeof(float), 256);
+  so.val = reinterpret_cast<float*>(p); p += align_up((size_t)rows * k * 4, 256);
+  so.idx = reinterpret_cast<int32_t*>(p); p += align_up((size_t)rows * k * 4, 256);
+  so.cnt = reinterpret_cast<int32_t*>(p);
+  so.id_offset = id_offset;
+  return so;
+}
+
+cudaError_t launch_merge_topk_shard(int64_t rows, int V, int k, const TopkWorkspace& w, void* partial, int v0,
+                                    cudaStream_t st) {
+  const MergeSource src{merge_parts(w), 0, 0};
+  return launch_merge_cta(src, rows, V, k, nullptr, nullptr, carve_shard_partial(partial, rows, k, v0), st);
+}
+
+cudaError_t launch_merge_shards(const void* gathered, int shards, int64_t rows, int k, int32_t* cand_ids,
+                                float* cand_lp, cudaStream_t st) {
+  const MergeShardOut a = carve_shard_partial(const_cast<void*>(gathered), rows, k, 0);
+  MergeSource src{};
+  src.parts = MergeParts{SpanPlan{}, a.ms, a.val, a.idx, a.cnt};
+  src.shards = shards;
+  src.shard_bytes = (int64_t)shard_partial_bytes(rows, k);
+  return launch_merge_cta(src, rows, shards, k, cand_ids, cand_lp, MergeShardOut{}, st);
+}
+
 cudaError_t launch_merge_topk(int64_t rows, int V, int k, const TopkWorkspace& w, int32_t* cand_ids,
                               float* cand_lp, cudaStream_t st) {
+  // many entries per row (large k): a CTA per row ranks them out of shared memory
+  if ((int64_t)w.plan.smax * k > 64) {
+    const MergeSource src{merge_parts(w), 0, 0};
+    const cudaError_t e = launch_merge_cta(src, rows, V, k, cand_ids, cand_lp, MergeShardOut{}, st);
+    if (e != cudaErrorNotSupported) return e;
+  }
   const int warps = 4;
   const int grid = (int)((rows + warps - 1) / warps);
   k_merge_topk<<<grid, warps * 32, 0, st>>>(merge_parts(w), rows, V, k, cand_ids, cand_lp);

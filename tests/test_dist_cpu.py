@@ -95,3 +95,45 @@ def test_ranks_draw_different_batches():
     import bench
     seeds = {bench.input_seed(r, s) for r in range(8) for s in range(16)}
     assert len(seeds) == 8 * 16
+
+
+# ---- vocabulary-parallel step a1: the all-gather of the ranks' partials (layout and rank order)
+def _shard_rank_main(rank: int, world: int, port: int, out_dir: str):
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world),
+                      MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    sys.path.insert(0, ROOT); sys.path.insert(0, os.path.join(ROOT, "tests"))
+    import numpy as np
+    import torch.distributed as dist
+    import oracle
+    import shard_layout
+    import paper_2609_39972_b200 as u
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    rows, V, k = 9, 600, 5
+    rng = np.random.Generator(np.random.PCG64(11))           # the same rows on every rank
+    x = np.round(rng.standard_normal((rows, V)).astype(np.float32) * 4.0) / 4.0     # with ties across slices
+    cuts = [0, 248, V]
+    v0, v1 = cuts[rank], cuts[rank + 1]
+    # this rank's partial from the oracle on its slice, packed as the header documents it
+    ids, lp, lse = oracle.topk_logprob(np.ascontiguousarray(x[:, v0:v1]), k)
+    val = np.take_along_axis(x[:, v0:v1], ids.astype(np.int64), axis=1)
+    m = x[:, v0:v1].max(axis=1)
+    s = np.exp(x[:, v0:v1].astype(np.float64) - m[:, None]).sum(axis=1)
+    part = shard_layout.pack(np.stack([m, s], axis=1), val, ids + v0, np.full(rows, k, np.int32))
+    assert part.size == u.ubt_topk_shard_bytes(rows, k)      # host-side query of the library
+    gathered, shards = u.gather_shard_partials(torch.from_numpy(part))
+    assert shards == world and gathered.numel() == world * part.size
+    g_ids, g_lp = shard_layout.merge(gathered.numpy(), shards, rows, k)
+    o_ids, o_lp, _ = oracle.topk_logprob(x, k)
+    np.testing.assert_array_equal(g_ids, o_ids)
+    np.testing.assert_allclose(g_lp, o_lp, rtol=1e-6, atol=1e-6)
+    with open(os.path.join(out_dir, f"shard{rank}.ok"), "w") as f:
+        f.write("ok")
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+@pytest.mark.timeout(180)
+def test_shard_partials_gathered_in_rank_order_two_gloo_ranks(tmp_path):
+    port = _free_port()
+    mp.spawn(_shard_rank_main, args=(2, port, str(tmp_path)), nprocs=2, join=True)
+    assert all((tmp_path / f"shard{r}.ok").exists() for r in range(2))

@@ -1,0 +1,116 @@
+"""Step a1 with the vocabulary split over ranks (ubt_topk_shard, ubt_topk_merge_shards) against the oracle on the
+whole rows.  The ranks are emulated one after the other on one GPU: each slice is copied into a dense tensor of
+its own, its partial is computed, the partials are laid back to back in rank order (what an all-gather gives)
+and merged.  Nothing waits on anything else, so no second GPU is needed for the arithmetic; the collective
+itself is plain torch.distributed and is covered by the two-rank CPU test."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import shard_layout
+import ubt_synth as synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _logits(rows, V, dtype, seed, quantise=False):
+    rng = np.random.Generator(np.random.PCG64(seed))
+    x = (rng.standard_normal((rows, V)) * rng.uniform(0.5, 6.0, size=(rows, 1))).astype(np.float32)
+    if quantise:                       # a handful of distinct values: ties inside and across slices
+        x = np.round(x * 2.0) / 2.0
+    return synth.f32_to_bf16_bits(x) if dtype == "bf16" else x
+
+
+def _cuts(V, shards, even, align):
+    """Slice boundaries: equal widths, or ragged ones (multiples of `align`, the last slice takes the rest)."""
+    if even:
+        assert V % shards == 0
+        return [V // shards * r for r in range(shards + 1)]
+    w = V // shards
+    cuts = [0]
+    for r in range(1, shards):
+        cuts.append(max(cuts[-1] + align, (w * r + (37 * r) % w // 3) // align * align))
+    return cuts + [V]
+
+
+@pytest.mark.parametrize("rows,V,k,shards,dtype,even,align,quantise", [
+    (37, 8192, 8, 4, "bf16", True, 8, False),        # ring path in every slice
+    (37, 8192, 8, 4, "bf16", False, 1, False),       # ragged widths: plain-load kernels
+    (5, 151936, 16, 8, "bf16", True, 8, False),      # the Qwen3 vocabulary over eight ranks
+    (64, 40000, 64, 8, "bf16", True, 8, False),      # k = 64: many long lists per row
+    (19, 4096, 4, 2, "f32", True, 4, False),
+    (23, 6000, 8, 3, "bf16", True, 8, True),         # ties across slices go to the lower token id
+    (3, 1000, 8, 1, "f32", True, 4, False),          # one rank: the partial alone
+])
+def test_sharded_topk_equals_the_oracle_on_whole_rows(rows, V, k, shards, dtype, even, align, quantise):
+    import paper_2609_39972_b200 as u
+    x = _logits(rows, V, dtype, seed=rows * 1000 + shards, quantise=quantise)
+    o_ids, o_lp, o_lse = oracle.topk_logprob(x, k)
+    cuts = _cuts(V, shards, even, align)
+    xd = synth.to_device(x, dtype, DEV)
+    nbytes = u.ubt_topk_shard_bytes(rows, k)
+    assert nbytes == shard_layout.offsets(rows, k)[4]
+    gathered = torch.empty(shards * nbytes, dtype=torch.uint8, device=DEV)
+    for r in range(shards):
+        v0, v1 = cuts[r], cuts[r + 1]
+        assert v1 - v0 >= k
+        part = u.ubt_topk_shard(xd[:, v0:v1].contiguous(), k, v0)
+        gathered[r * nbytes:(r + 1) * nbytes] = part[:nbytes]
+        # the partial itself, against the oracle on the slice
+        ms, val, idx, cnt = shard_layout.unpack(part.cpu().numpy(), rows, k)
+        s_ids, s_lp, s_lse = oracle.topk_logprob(np.ascontiguousarray(x[:, v0:v1]), k)
+        assert (cnt == k).all()
+        np.testing.assert_array_equal(idx, s_ids + v0)
+        np.testing.assert_allclose(ms[:, 0].astype(np.float64) + np.log(ms[:, 1].astype(np.float64)), s_lse,
+                                   rtol=1e-5, atol=1e-5)
+        np.testing.assert_allclose(val.astype(np.float64) - s_lse[:, None], s_lp, rtol=1e-5, atol=1e-5)
+    ids, lp = u.ubt_topk_merge_shards(gathered, shards, rows, k)
+    torch.cuda.synchronize()
+    assert u.ubt_debug_ring_timeouts() == 0
+    np.testing.assert_array_equal(ids.cpu().numpy(), o_ids)
+    np.testing.assert_allclose(lp.cpu().numpy().astype(np.float64), o_lp, rtol=1e-5, atol=1e-5)
+    # the same through the one-GPU entry point, and the host restatement of the merge
+    ids1 = torch.empty((rows, k), dtype=torch.int32, device=DEV)
+    lp1 = torch.empty((rows, k), dtype=torch.float32, device=DEV)
+    u.ubt_topk_logprob(xd, k, ids1, lp1, u.workspace(u.ubt_draft_workspace_bytes(rows, 1, V, k, 1), DEV))
+    torch.cuda.synchronize()
+    assert torch.equal(ids1, ids)
+    assert float((lp1 - lp).abs().max()) <= 1e-5 * max(1.0, float(lp.abs().max()))
+    h_ids, h_lp = shard_layout.merge(gathered.cpu().numpy(), shards, rows, k)
+    np.testing.assert_array_equal(h_ids, o_ids)
+    np.testing.assert_allclose(h_lp, o_lp, rtol=1e-5, atol=1e-5)
+
+
+def test_sharded_candidates_build_the_same_tree():
+    """draft = sharded a1 + ubt_build_tree equals ubt_draft_tree on the whole rows (c2 shapes, four ranks)."""
+    import paper_2609_39972_b200 as u
+    cfg = synth.CONFIGS["c2"].replace(B=3)
+    di = synth.draft_inputs(cfg, 77)
+    ud = synth.to_device(di.unigram_logits, cfg.dtype, DEV)
+    bd = torch.from_numpy(di.bigram_scores).to(DEV)
+    whole = u.ubt_draft_tree(ud, bd, cfg.k, cfg.N)
+    shards, rows = 4, cfg.B * cfg.L
+    nbytes = u.ubt_topk_shard_bytes(rows, cfg.k)
+    gathered = torch.empty(shards * nbytes, dtype=torch.uint8, device=DEV)
+    w = cfg.V // shards
+    for r in range(shards):
+        gathered[r * nbytes:(r + 1) * nbytes] = u.ubt_topk_shard(ud[..., r * w:(r + 1) * w].contiguous(), cfg.k, r * w)[:nbytes]
+    split = u.Tree.empty(cfg.B, cfg.N, cfg.L, cfg.k, DEV)
+    u.ubt_topk_merge_shards(gathered, shards, rows, cfg.k, split.cand_ids, split.cand_logprob)
+    u.ubt_build_tree(bd, split)
+    torch.cuda.synchronize()
+    for name in ("cand_ids", "token_ids", "parents", "depths", "position_ids", "cand_rank", "mask", "n_nodes"):
+        assert torch.equal(getattr(whole, name), getattr(split, name)), name
+
+
+def test_argument_checks():
+    import paper_2609_39972_b200 as u
+    x = torch.zeros((4, 64), dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(u.UbtError):
+        u.ubt_topk_shard(x, 128, 0)              # k > Vs
+    with pytest.raises(u.UbtError):
+        u.ubt_topk_shard(x, 8, -1)               # negative first column
+    with pytest.raises(ValueError):
+        u.ubt_topk_merge_shards(torch.zeros(16, dtype=torch.uint8, device=DEV), 2, 4, 8)
