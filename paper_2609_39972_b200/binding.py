@@ -57,8 +57,7 @@ EXPORTS = ["ubt_version", "ubt_status_string", "ubt_debug_ring_timeouts", "ubt_d
            "ubt_topk_logprob", "ubt_selector_scores", "ubt_build_tree", "ubt_build_mask", "ubt_draft_tree", "ubt_verify_tree",
            "ubt_draft_host_buffer_bytes", "ubt_verify_host_buffer_bytes", "ubt_draft_tree_host",
            "ubt_verify_tree_host", "ubt_verify_tree_static", "ubt_verify_static_capacity", "ubt_lm_head_workspace_bytes",
-           "ubt_lm_head_topk", "ubt_topk_shard_bytes", "ubt_topk_shard", "ubt_topk_merge_shards",
-           "gather_shard_partials", "topk_logprob_vocab_parallel"]
+           "ubt_lm_head_topk", "ubt_topk_shard_bytes", "ubt_topk_shard", "ubt_topk_merge_shards"]
 
 _lib = None
 
