@@ -259,6 +259,26 @@ int ubt_verify_tree(const ubt_tree *tree, const void *target_logits, int dtype, 
                     size_t workspace_bytes, void *cuda_stream);
 
 /*
+ * Greedy step a4 with the vocabulary of the target logits split over the ranks of a tensor-parallel group
+ * (appendix "Verification via Tree-attention": the pick of a slot is the arg max over the whole vocabulary).
+ * Rank r holds the columns [v0, v0 + Vs) of every target row as a dense [B, node_budget, Vs] tensor and calls
+ * ubt_verify_keys_shard, which writes one 8-byte ordering key per row into row_keys[B * node_budget]: the best
+ * (value, token) of the slice with the token counted in the WHOLE vocabulary; a larger key is a better pick
+ * (higher value, then lower token id), so the pick of a row is the maximum of the ranks' keys.  The caller
+ * gathers the ranks' key arrays back to back in rank order (one all-gather of B * node_budget * 8 bytes) and
+ * every rank calls ubt_verify_tree_keys, which takes the maximum per slot and walks the tree exactly as
+ * ubt_verify_tree does in greedy mode: identical accepted_len, accepted_nodes, out_tokens, bonus_token,
+ * node_pick and status words (a NaN, +inf or an abandoned wait in any slice is reported).  Of `opts` only
+ * node_pick and status are read.  Workspace of ubt_verify_keys_shard: ubt_verify_workspace_bytes(B,
+ * node_budget, Vs, UBT_VERIFY_GREEDY).  No collective is issued by the library.  Sampling is not split this way.
+ */
+int ubt_verify_keys_shard(const void *target_shard, int dtype, int B, int node_budget, int Vs, int v0,
+                          unsigned long long *row_keys, void *workspace, size_t workspace_bytes,
+                          void *cuda_stream);
+int ubt_verify_tree_keys(const ubt_tree *tree, const unsigned long long *gathered_keys, int shards,
+                         ubt_verify_result *out, const ubt_verify_opts *opts, void *cuda_stream);
+
+/*
  * Host-buffer forms.  Every pointer inside `tree`, `opts` (alpha ... pos_offset, node_pick) and
  * `out`, and the logits / bigram arguments, are HOST pointers (pinned memory makes the copies
  * asynchronous).  `device_buffer` is caller-owned DEVICE memory of at least

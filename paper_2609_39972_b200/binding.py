@@ -57,7 +57,8 @@ EXPORTS = ["ubt_version", "ubt_status_string", "ubt_debug_ring_timeouts", "ubt_d
            "ubt_topk_logprob", "ubt_selector_scores", "ubt_build_tree", "ubt_build_mask", "ubt_draft_tree", "ubt_verify_tree",
            "ubt_draft_host_buffer_bytes", "ubt_verify_host_buffer_bytes", "ubt_draft_tree_host",
            "ubt_verify_tree_host", "ubt_verify_tree_static", "ubt_verify_static_capacity", "ubt_lm_head_workspace_bytes",
-           "ubt_lm_head_topk", "ubt_topk_shard_bytes", "ubt_topk_shard", "ubt_topk_merge_shards"]
+           "ubt_lm_head_topk", "ubt_topk_shard_bytes", "ubt_topk_shard", "ubt_topk_merge_shards", "ubt_verify_keys_shard",
+           "ubt_verify_tree_keys"]
 
 _lib = None
 
@@ -108,6 +109,9 @@ def load() -> C.CDLL:
     L.ubt_topk_shard.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
                                  C.c_size_t, C.c_void_p]
     L.ubt_topk_merge_shards.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.ubt_verify_keys_shard.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
+                                        C.c_size_t, C.c_void_p]
+    L.ubt_verify_tree_keys.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
     L.ubt_debug_ring_timeouts.restype = C.c_longlong
     L.ubt_draft_tree_host.argtypes = L.ubt_draft_tree.argtypes
     L.ubt_verify_tree_host.argtypes = L.ubt_verify_tree.argtypes
@@ -399,6 +403,49 @@ def ubt_verify_tree(tree: Tree, target_logits: torch.Tensor, mode="greedy", seed
                                   C.byref(r), _ptr(ws), ws.numel(), _stream(stream)), "ubt_verify_tree")
     result.node_pick = node_pick
     return result
+
+
+def ubt_verify_keys_shard(target_shard: torch.Tensor, v0: int, row_keys: Optional[torch.Tensor] = None,
+                          ws: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Greedy step a4 on this rank's slice of the vocabulary (``target_shard[B, N, Vs]``, first column ``v0``): one
+    8-byte ordering key per row, ``int64[B * N]`` (opaque; larger = better pick)."""
+    _need(target_shard, "target_shard")
+    B, N, Vs = target_shard.shape
+    if row_keys is None:
+        row_keys = torch.empty((B * N,), dtype=torch.int64, device=target_shard.device)
+    if ws is None:
+        ws = workspace(ubt_verify_workspace_bytes(B, N, Vs, UBT_VERIFY_GREEDY), target_shard.device)
+    _check(load().ubt_verify_keys_shard(_ptr(target_shard), _dtype_code(target_shard), B, N, Vs, int(v0),
+                                        _ptr(_need(row_keys, "row_keys")), _ptr(ws), ws.numel(), _stream(stream)),
+           "ubt_verify_keys_shard")
+    return row_keys
+
+
+def ubt_verify_tree_keys(tree: Tree, gathered_keys: torch.Tensor, shards: int,
+                         node_pick: Optional[torch.Tensor] = None, result: Optional[VerifyResult] = None,
+                         status: Optional[torch.Tensor] = None, stream=None) -> VerifyResult:
+    """The greedy walk on the ranks' keys, back to back in rank order (``int64[shards * B * N]``)."""
+    _need(gathered_keys, "gathered_keys")
+    if gathered_keys.numel() < shards * tree.B * tree.N:
+        raise ValueError("gathered_keys is smaller than shards * B * N")
+    if result is None:
+        result = VerifyResult.empty(tree.B, tree.L, gathered_keys.device)
+    o = _VerifyOpts(0, 1.0, None if node_pick is None else node_pick.data_ptr(), None, None, 0,
+                    None if status is None else status.data_ptr(), 0, 0)
+    t = tree.c_struct()
+    r = result.c_struct()
+    _check(load().ubt_verify_tree_keys(C.byref(t), _ptr(gathered_keys), shards, C.byref(r), C.byref(o),
+                                       _stream(stream)), "ubt_verify_tree_keys")
+    result.node_pick = node_pick
+    return result
+
+
+def verify_tree_vocab_parallel(tree: Tree, target_shard: torch.Tensor, v0: int, group=None, **kw) -> VerifyResult:
+    """Greedy verification of target logits whose vocabulary is split over the ranks of ``group``: local keys, one
+    all-gather, walk; all on torch's current stream.  Every rank returns the same verdict."""
+    keys = ubt_verify_keys_shard(target_shard, v0)
+    gathered, shards = gather_shard_partials(keys, group)
+    return ubt_verify_tree_keys(tree, gathered, shards, **kw)
 
 
 def ubt_draft_host_buffer_bytes(B, L, V, k, node_budget, dtype) -> int:

@@ -590,4 +590,37 @@ int ubt_debug_bounds_report(int which, long long out[4]) {
 }
 #endif
 
+int ubt_verify_keys_shard(const void* target_shard, int dtype, int B, int N, int Vs, int v0,
+                          unsigned long long* row_keys, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!target_shard || !row_keys || B < 0 || N < 1 || Vs < 1 || v0 < 0) return UBT_ERR_INVALID_ARG;
+  if (dtype != UBT_F32 && dtype != UBT_BF16) return UBT_ERR_INVALID_ARG;
+  if (!aligned16(target_shard) || !aligned16(row_keys)) return UBT_ERR_INVALID_ARG;
+  if (N > kMaxN || (int64_t)v0 + Vs > 0x7fffffffll) return UBT_ERR_UNSUPPORTED;
+  if (B == 0) return UBT_OK;
+  const int64_t rows = (int64_t)B * N;
+  if (!workspace || !aligned16(workspace) || workspace_bytes < verify_workspace_bytes(rows, Vs, UBT_VERIFY_GREEDY))
+    return UBT_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  VerifyWorkspace w = carve_verify_workspace(workspace, rows, Vs, UBT_VERIFY_GREEDY);
+  if (launch_row_argmax(target_shard, dtype, rows, Vs, w, 0, false, st) != cudaSuccess) return UBT_ERR_CUDA;
+  if (launch_row_keys_shard(w, rows, Vs, v0, row_keys, st) != cudaSuccess) return UBT_ERR_CUDA;
+  return UBT_OK;
+}
+
+int ubt_verify_tree_keys(const ubt_tree* tree, const unsigned long long* gathered_keys, int shards,
+                         ubt_verify_result* out, const ubt_verify_opts* opts, void* cuda_stream) {
+  if (!tree || !out || !gathered_keys || shards < 1) return UBT_ERR_INVALID_ARG;
+  if (!tree->token_ids || !tree->parents || !tree->n_nodes) return UBT_ERR_INVALID_ARG;
+  if (!out->accepted_len || !out->bonus_token || !out->accepted_nodes || !out->out_tokens) return UBT_ERR_INVALID_ARG;
+  if (!aligned16(gathered_keys)) return UBT_ERR_INVALID_ARG;
+  const int B = tree->B, N = tree->N, L = tree->L;
+  if (B < 0 || N < 1 || L < 1) return UBT_ERR_INVALID_ARG;
+  if (N > kMaxN || L > kMaxL) return UBT_ERR_UNSUPPORTED;
+  if (B == 0) return UBT_OK;
+  if (launch_walk_keys(*tree, gathered_keys, shards, opts ? opts->node_pick : nullptr, *out,
+                       opts ? opts->status : nullptr, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    return UBT_ERR_CUDA;
+  return UBT_OK;
+}
+
 }  // extern "C"

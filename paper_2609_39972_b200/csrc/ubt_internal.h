@@ -129,6 +129,12 @@ cudaError_t launch_walk(const ubt_tree& tree, int mode, const VerifyWorkspace& w
                         const int32_t* sampled_pick, int32_t* node_pick,
                         const ubt_verify_result& out, int32_t* status, cudaStream_t st);
 
+// vocabulary-parallel greedy a4: one key per row of this rank's slice; the walk on the gathered keys
+cudaError_t launch_row_keys_shard(const VerifyWorkspace& w, int64_t rows, int V, int v0, unsigned long long* row_keys,
+                                  cudaStream_t st);
+cudaError_t launch_walk_keys(const ubt_tree& tree, const unsigned long long* gathered_keys, int shards,
+                             int32_t* node_pick, const ubt_verify_result& out, int32_t* status, cudaStream_t st);
+
 // ---- LM head fused with a1 (ubt_lmhead.cu): tcgen05 GEMM whose epilogue keeps (max, sum exp, top-k) per row
 int lm_head_max_k();
 int lm_head_max_rows();

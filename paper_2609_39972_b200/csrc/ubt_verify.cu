@@ -613,7 +613,7 @@ k_row_sample(const T* __restrict__ logits, int64_t rows, int N, int V, uint64_t 
 __global__ void __launch_bounds__(128)
 k_walk(ubt_tree tree, int mode, SpanPlan plan, const unsigned long long* __restrict__ part_key, int V,
        const int32_t* __restrict__ sampled_pick, int32_t* __restrict__ node_pick, ubt_verify_result out,
-       int32_t* __restrict__ status) {
+       int32_t* __restrict__ status, int shards, int64_t shard_stride) {
   __shared__ int s_pick[kMaxN], s_tok[kMaxN], s_par[kMaxN];
   __shared__ int s_bits;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, N = tree.N, L = tree.L;
@@ -625,11 +625,19 @@ k_walk(ubt_tree tree, int mode, SpanPlan plan, const unsigned long long* __restr
     int p, bits = 0;
     if (mode == UBT_VERIFY_GREEDY) {
       const int64_t row = o + n;
-      const int64_t c_first = (row * (int64_t)V) / plan.span;
-      const int64_t c_last = ((row + 1) * (int64_t)V - 1) / plan.span;
+      // the keys of the row: one per segment of this GPU's row-argmax pass, or (shards > 0) one per rank of a
+      // vocabulary-parallel group, rank r's keys `shard_stride` * r entries behind rank 0's
+      int64_t nseg = shards, base = row, stride = shard_stride;
+      if (shards == 0) {
+        const int64_t c_first = (row * (int64_t)V) / plan.span;
+        const int64_t c_last = ((row + 1) * (int64_t)V - 1) / plan.span;
+        nseg = c_last - c_first + 1;
+        base = row * plan.smax;
+        stride = 1;
+      }
       unsigned long long best = 0;
-      for (int64_t j = 0; j <= c_last - c_first; ++j) {
-        const unsigned long long key = part_key[row * plan.smax + j];
+      for (int64_t j = 0; j < nseg; ++j) {
+        const unsigned long long key = part_key[base + j * stride];
         best = key > best ? key : best;
       }
       p = best ? key_idx(best) : 0;  // a row without any comparable value falls back to token 0
@@ -812,7 +820,44 @@ cudaError_t launch_walk(const ubt_tree& tree, int mode, const VerifyWorkspace& w
                         int32_t* status, cudaStream_t st) {
   if (tree.B == 0) return cudaSuccess;
   return launch_kernel(k_walk, dim3(tree.B), dim3(128), 0, st, true, tree, mode, w.plan,
-                       (const unsigned long long*)w.part_key, V, sampled_pick, node_pick, out, status);
+                       (const unsigned long long*)w.part_key, V, sampled_pick, node_pick, out, status, 0,
+                       (int64_t)0);
+}
+
+// Vocabulary-parallel greedy a4, first half: one key per row of this rank's slice -- the best key of the row's
+// segments with its token moved by the slice's first column (the low word of a key is ~token; the marker keys of
+// a non-finite or abandoned segment are kept as they are).
+__global__ void __launch_bounds__(128)
+k_row_keys_shard(SpanPlan plan, const unsigned long long* __restrict__ part_key, int64_t rows, int V, int v0,
+                 unsigned long long* __restrict__ row_keys) {
+  const int64_t row = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (row >= rows) return;
+  const int64_t c_first = (row * (int64_t)V) / plan.span;
+  const int64_t c_last = ((row + 1) * (int64_t)V - 1) / plan.span;
+  unsigned long long best = 0;
+  for (int64_t j = 0; j <= c_last - c_first; ++j) {
+    const unsigned long long key = part_key[row * plan.smax + j];
+    best = key > best ? key : best;
+  }
+  if (best != 0ull && (best >> 32) <= (kKeyPlusInf >> 32))  // the key of a value (+inf included), not a marker
+    best = (best & 0xffffffff00000000ull) | (unsigned long long)((uint32_t)best - (uint32_t)v0);
+  row_keys[row] = best;
+}
+
+cudaError_t launch_row_keys_shard(const VerifyWorkspace& w, int64_t rows, int V, int v0, unsigned long long* row_keys,
+                                  cudaStream_t st) {
+  if (rows == 0) return cudaSuccess;
+  k_row_keys_shard<<<(unsigned)((rows + 127) / 128), 128, 0, st>>>(w.plan, w.part_key, rows, V, v0, row_keys);
+  return cudaGetLastError();
+}
+
+// Second half: the walk on the gathered keys ([shards, B*N], rank order).
+cudaError_t launch_walk_keys(const ubt_tree& tree, const unsigned long long* gathered_keys, int shards,
+                             int32_t* node_pick, const ubt_verify_result& out, int32_t* status, cudaStream_t st) {
+  if (tree.B == 0) return cudaSuccess;
+  return launch_kernel(k_walk, dim3(tree.B), dim3(128), 0, st, true, tree, (int)UBT_VERIFY_GREEDY, SpanPlan{},
+                       gathered_keys, 1, (const int32_t*)nullptr, node_pick, out, status, shards,
+                       (int64_t)tree.B * tree.N);
 }
 
 // Number of bounded waits that gave up in this file's kernels (0 in a healthy run).

@@ -114,3 +114,66 @@ def test_argument_checks():
         u.ubt_topk_shard(x, 8, -1)               # negative first column
     with pytest.raises(ValueError):
         u.ubt_topk_merge_shards(torch.zeros(16, dtype=torch.uint8, device=DEV), 2, 4, 8)
+
+
+# ---- greedy verification with the target logits' vocabulary split over ranks
+def _drafted(cfg, seed):
+    import paper_2609_39972_b200 as u
+    from parity import tree_to_numpy
+    di = synth.draft_inputs(cfg, seed)
+    tree = u.ubt_draft_tree(synth.to_device(di.unigram_logits, cfg.dtype, DEV),
+                            torch.from_numpy(di.bigram_scores).to(DEV), cfg.k, cfg.N)
+    torch.cuda.synchronize()
+    return tree, tree_to_numpy(tree)
+
+
+@pytest.mark.parametrize("V,shards,even", [(8192, 4, True), (8192, 3, False), (151936, 8, True)])
+def test_sharded_greedy_verify_equals_the_oracle(V, shards, even):
+    import paper_2609_39972_b200 as u
+    from parity import compare_verify
+    cfg = synth.CONFIGS["c2"].replace(B=3, L=6, N=24, k=4, V=V)
+    tree, g = _drafted(cfg, 5)
+    z = synth.target_logits(cfg, 5)
+    synth.plant_path(z, cfg.dtype, g.token_ids, g.parents, g.n_nodes, 5)
+    # a tie between two slices: the lower token id must win in every row of sequence 0
+    zf = synth.as_f32(z, cfg.dtype)
+    top = zf[0].max(axis=1) + 1.0
+    for n in range(cfg.N):
+        for col in (V - 3, 5):
+            z[0, n, col] = synth.f32_to_bf16_bits(np.float32([top[n]]))[0]
+    want = oracle.verify(g.token_ids, g.parents, g.n_nodes, cfg.L, z, "greedy")
+    zd = synth.to_device(z, cfg.dtype, DEV)
+    cuts = _cuts(V, shards, even, 1 if not even else 8)
+    rows = cfg.B * cfg.N
+    gathered = torch.empty(shards * rows, dtype=torch.int64, device=DEV)
+    for r in range(shards):
+        u.ubt_verify_keys_shard(zd[..., cuts[r]:cuts[r + 1]].contiguous(), cuts[r], gathered[r * rows:(r + 1) * rows])
+    pick = torch.full((cfg.B, cfg.N), -9, dtype=torch.int32, device=DEV)
+    status = torch.full((cfg.B,), -1, dtype=torch.int32, device=DEV)
+    res = u.ubt_verify_tree_keys(tree, gathered, shards, node_pick=pick, status=status)
+    torch.cuda.synchronize()
+    compare_verify(res, want, pick)
+    assert (pick[0] == 5).all()
+    assert status.tolist() == [0] * cfg.B
+    # and bit for bit what the one-GPU call gives
+    one = u.ubt_verify_tree(tree, zd, "greedy")
+    torch.cuda.synchronize()
+    for name in ("accepted_len", "bonus_token", "accepted_nodes", "out_tokens"):
+        assert torch.equal(getattr(one, name), getattr(res, name)), name
+
+
+def test_sharded_greedy_verify_reports_a_nan_in_any_slice():
+    import paper_2609_39972_b200 as u
+    cfg = synth.CONFIGS["c2"].replace(B=2, L=6, N=24, k=4, V=8192)
+    tree, g = _drafted(cfg, 9)
+    z = synth.target_logits(cfg, 9)
+    z[1, 3, 6000] = 0x7FC0                     # a bf16 NaN in the third slice of sequence 1
+    zd = synth.to_device(z, cfg.dtype, DEV)
+    shards, rows, w = 4, cfg.B * cfg.N, cfg.V // 4
+    gathered = torch.empty(shards * rows, dtype=torch.int64, device=DEV)
+    for r in range(shards):
+        u.ubt_verify_keys_shard(zd[..., r * w:(r + 1) * w].contiguous(), r * w, gathered[r * rows:(r + 1) * rows])
+    status = torch.zeros((cfg.B,), dtype=torch.int32, device=DEV)
+    u.ubt_verify_tree_keys(tree, gathered, shards, status=status)
+    torch.cuda.synchronize()
+    assert status.tolist() == [0, 1]
