@@ -121,10 +121,11 @@ typedef struct ubt_verify_opts {
   int32_t validate_finite; /* host-buffer form only: return UBT_ERR_NONFINITE if any sequence was flagged */
   int32_t path_only;   /* 1: evaluate only the target rows the walk visits (at most L + 1 of the N rows of a
                           sequence) instead of all of them: the same verdict from a fraction of the bytes, as a
-                          chain of at most L + 1 dependent steps inside one cooperative launch (needs B <= 1024,
-                          else UBT_ERR_UNSUPPORTED).  node_pick then receives the picks of the visited slots and
-                          -1 elsewhere; early_start is ignored.  Worth it when B * N is large (most rows are never
-                          visited); for a single small tree the all-rows pass is as fast. */
+                          chain of at most L + 1 dependent steps inside one launch (a thread-block cluster per
+                          sequence; no workspace is used, any B).  node_pick then receives the picks of the
+                          visited slots and -1 elsewhere, status flags a NaN or +inf in a VISITED row only;
+                          early_start is ignored.  Worth it when B * N is large (most rows are never visited);
+                          for a single small tree the all-rows pass is as fast. */
 } ubt_verify_opts;
 
 typedef struct ubt_verify_result {
