@@ -48,7 +48,7 @@ struct TreeSmem {
   Span<uint32_t> maskrow;   // [N, mask_words]
   Span<int> scalars;        // [0] accepted count, [1]-[3] scratch of the expansion, [4] status bits of the sequence
   // Nodes enumerated by the parallel expansion (resident table only; see expand_rounds): node 0 is the root.
-  int xcap;                 // capacity (0 in lazy mode)
+  int xcap;                 // capacity (lazy mode: 0, or that of the depth-by-depth expansion)
   Span<short> x_parent;     // [xcap] enumerated parent, -1 for the root
   Span<unsigned char> x_depth, x_rank, x_next, x_bak;  // [xcap] depth, candidate rank, next child to enumerate (+ its backup)
   Span<float> x_score;      // [xcap]
@@ -56,12 +56,20 @@ struct TreeSmem {
   Span<short> x_aux;        // [xcap] per-round scratch
   Span<unsigned long long> x_key64;  // [xcap] ordering keys of the final choice
   Span<int> x_wsum;         // [32] warp totals of the block scans
+  Span<unsigned long long> dw_row;  // depth-by-depth expansion: [warps, k] ordering keys of the row a warp has open
 };
 
 // Rows of the pair table are computed on demand when the whole table would not fit.
 __host__ __device__ inline bool tree_lazy(int L, int k) { return (size_t)L * k * k * 5 > kTreeTableBytes; }
 // Nodes the parallel expansion may enumerate before it picks the N - 1 best (root included).
 __host__ __device__ inline int expand_capacity(int N) { return 4 * N < 128 ? 128 : (4 * N > 1024 ? 1024 : 4 * N); }
+// Lazy mode with a small finite width runs eq. 11 depth by depth (expand_depthwise): the node arrays then hold the
+// root and W nodes per depth, followed by a scratch area for the W * min(W, k) candidates of one depth.
+constexpr int kDepthwiseMaxW = 16;
+__host__ __device__ inline int depthwise_capacity(int L, int k, int N, int W) {
+  if (!tree_lazy(L, k) || W <= 0 || W >= N - 1 || W > kDepthwiseMaxW) return 0;
+  return 1 + W * L + W * (W < k ? W : k);
+}
 
 // Byte offsets of the arrays above inside the CTA's dynamic shared memory.  They depend on L, k, N only, so
 // the host computes them once per launch and passes them as a kernel argument: the kernel then forms every
@@ -69,12 +77,13 @@ __host__ __device__ inline int expand_capacity(int N) { return 4 * N < 128 ? 128
 struct TreeLayout {
   uint32_t t, ord, rowmap, la, pre, lp, tok, al, ent, nd_parent, nd_depth, nd_rank, nd_score, nd_slot, nd_pk, kk,
       depth_cnt, depth_off, x_fill, maskrow, scalars, x_parent, x_depth, x_rank, x_next, x_bak, x_score, x_key, x_aux,
-      x_wsum, x_key64;
+      x_wsum, x_key64, dw_row;
   uint32_t total;
   int xcap;
+  int lazy;
 };
 
-inline TreeLayout tree_layout(int L, int k, int N) {
+inline TreeLayout tree_layout(int L, int k, int N, int W = 0) {
   TreeLayout o{};
   size_t off = 0;
   auto take = [&](size_t bytes) {
@@ -96,19 +105,21 @@ inline TreeLayout tree_layout(int L, int k, int N) {
   o.depth_cnt = take(sizeof(int) * (L + 2)); o.depth_off = take(sizeof(int) * (L + 2));
   o.x_fill = take(sizeof(int) * (L + 2));
   o.maskrow = take(sizeof(uint32_t) * N * mw); o.scalars = take(sizeof(int) * 8);
-  const int xcap = lazy ? 0 : expand_capacity(N);
+  const int xcap = lazy ? depthwise_capacity(L, k, N, W) : expand_capacity(N);
   o.xcap = xcap;
+  o.lazy = lazy ? 1 : 0;
   o.x_parent = take(sizeof(short) * xcap); o.x_depth = take(xcap); o.x_rank = take(xcap); o.x_next = take(xcap);
   o.x_bak = take(xcap); o.x_score = take(sizeof(float) * xcap); o.x_key = take(sizeof(uint32_t) * xcap);
   o.x_aux = take(sizeof(short) * xcap); o.x_wsum = take(sizeof(int) * 32);
   o.x_key64 = take(sizeof(unsigned long long) * xcap);
+  o.dw_row = take(lazy && xcap > 0 ? sizeof(unsigned long long) * (G2_T / 32) * k : 0);
   o.total = (uint32_t)off;
   return o;
 }
 
 __device__ __forceinline__ void tree_bind(TreeSmem* s, unsigned char* base, const TreeLayout& o, int L, int k, int N) {
   const int mw = (N + 31) / 32, xcap = o.xcap;
-  const bool lazy = xcap == 0;
+  const bool lazy = o.lazy != 0;
   const long long lkk = lazy ? (long long)N * k : (long long)L * k * k, lk = (long long)L * k;
   s->xcap = xcap;
   s->x_parent = Span<short>((short*)(base + o.x_parent), xcap, 121);
@@ -121,6 +132,7 @@ __device__ __forceinline__ void tree_bind(TreeSmem* s, unsigned char* base, cons
   s->x_aux = Span<short>((short*)(base + o.x_aux), xcap, 128);
   s->x_wsum = Span<int>((int*)(base + o.x_wsum), 32, 129);
   s->x_key64 = Span<unsigned long long>((unsigned long long*)(base + o.x_key64), xcap, 130);
+  s->dw_row = Span<unsigned long long>((unsigned long long*)(base + o.dw_row), lazy && xcap > 0 ? (long long)(G2_T / 32) * k : 0, 131);
   s->t = Span<float>((float*)(base + o.t), lkk, 101);
   s->ord = Span<unsigned char>(base + o.ord, lkk, 102);
   s->rowmap = Span<short>((short*)(base + o.rowmap), lazy ? lk + 1 : 0, 107);
@@ -814,6 +826,138 @@ __device__ __forceinline__ int select_enumerated(TreeSmem& s, int n, int n_sure,
   return n_sel;
 }
 
+// Eq. 11 as it stands, for the case the other forms serve badly: the pair table does not fit in shared memory
+// (k = 64) and the width is small (W <= 16).  Depth by depth: one warp per node of F_{d-1} fetches the raw selector
+// scores of the node's row from global memory, applies eq. 5 and eq. 9 with the row in registers (two successors
+// per lane) and extracts the row's min(W, k) best children under (score desc, token asc) -- no other child of
+// that node can be among the W best of the depth; then all threads rank the at most W * W candidates of the depth
+// under the total order, and the W best become F_d.  The node arrays end up holding S = F_1 u ... u F_L (root at
+// 0); the caller picks the budget's best of them (eq. 12).  Two CTA barriers per depth, and the only dependent
+// global access per depth is one 4 k-byte row per node, so the chain is L short steps instead of N - 1 pops that
+// each prepare a row.  Every thread of the CTA calls this; returns the number of enumerated nodes, root included.
+__device__ __forceinline__ int expand_depthwise(TreeSmem& s, const RowSource& src, int L, int k, int W, float zeta) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int NW = G2_T / 32;
+  const int m = W < k ? W : k;      // children a node can contribute to its depth
+  const int cbase = 1 + W * L;      // candidates of the current depth live behind the nodes
+  if (tid == 0) { s.x_parent[0] = -1; s.x_depth[0] = 0; s.x_rank[0] = 0; s.x_score[0] = 0.f; }
+  __syncthreads();
+  int lo = 0, hi = 1;               // F_{d-1} = nodes [lo, hi)
+  for (int d = 1; d <= L; ++d) {
+    const int np = hi - lo, i = d - 1;  // i: position of the children
+    const float al = s.al[i], la = s.la[i];
+    for (int p = warp; p < np; p += NW) {
+      const int node = lo + p, ra = d == 1 ? 0 : (int)s.x_rank[node];
+      const float sc = s.x_score[node];
+      const float* row = i == 0 ? src.anchor_bigram : src.bigram + ((size_t)(i - 1) * k + ra) * k;
+      float v[2];
+      uint32_t ntok[2];
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int rb = lane + 32 * h;
+        v[h] = -INFINITY;
+        ntok[h] = 0u;
+        if (rb < k) {
+          v[h] = fmaf(al, s.lp[i * k + rb], la * (row ? __ldg(row + rb) : 0.f));
+          ntok[h] = ~(uint32_t)s.tok[i * k + rb];
+        }
+      }
+      float mx = fmaxf(v[0], v[1]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, o));
+      float sum = (lane < k ? expf(v[0] - mx) : 0.f) + (lane + 32 < k ? expf(v[1] - mx) : 0.f);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(FULL, sum, o);
+      const float lse = mx + logf(sum);
+      // the row's ordering keys (score, ~token) meet in shared memory; every lane then counts, for its two
+      // children, the keys in front of them (64 independent loads: no warp-wide reductions, no rounds) and the
+      // children with fewer than m in front write their records to the candidate place of that rank
+      unsigned long long k64[2];
+      unsigned long long* rowkeys = s.dw_row.ptr((long long)warp * k, k);
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int rb = lane + 32 * h;
+        v[h] = sc + (v[h] - lse) + zeta;  // the child's score
+        uint32_t kh = f2key(v[h]);
+        kh = kh == 0u ? 1u : kh;
+        k64[h] = ((unsigned long long)kh << 32) | ntok[h];
+        if (rb < k) rowkeys[rb] = k64[h];
+      }
+      __syncwarp();
+      int r0 = 0, r1 = 0;
+#pragma unroll 16
+      for (int j = 0; j < k; ++j) {  // (unrolled: sixteen loads in flight; the loop is latency otherwise)
+        const unsigned long long kj = rowkeys[j];
+        r0 += kj > k64[0];
+        r1 += kj > k64[1];
+      }
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int rb = lane + 32 * h, r = h == 0 ? r0 : r1;
+        if (rb < k && r < m) {  // tokens of a position are distinct, so the keys of a row are
+          const int c = cbase + p * m + r;
+          s.x_parent[c] = (short)node;
+          s.x_rank[c] = (unsigned char)rb;
+          s.x_score[c] = v[h];
+          s.x_key64[c] = k64[h];
+        }
+      }
+      __syncwarp();
+    }
+    __syncthreads();
+    // the W best of the depth's candidates under (score desc, token asc, rank path asc): `sp` threads share the
+    // count of one candidate; the loop is branch-free, exact ties (rare) are settled behind it
+    const int nc = np * m;
+    int sp = 1;
+    while (sp < 8 && sp * 2 * nc <= G2_T) sp <<= 1;
+    const int cand = tid / sp, q = tid & (sp - 1);
+    int r = 0, same = 0;
+    unsigned long long kc = 0ull;
+    if (cand < nc) {
+      kc = s.x_key64[cbase + cand];
+#pragma unroll 16
+      for (int j = q; j < nc; j += sp) {
+        const unsigned long long kj = s.x_key64[cbase + j];
+        r += kj > kc;
+        same += kj == kc;
+      }
+    }
+    for (int o = sp >> 1; o > 0; o >>= 1) {
+      r += __shfl_xor_sync(FULL, r, o);
+      same += __shfl_xor_sync(FULL, same, o);
+    }
+    if (cand < nc && q == 0) {
+      if (same > 1) {  // same score and token under other parents: the parents' rank paths decide
+        for (int j = 0; j < nc; ++j) {
+          if (j == cand || s.x_key64[cbase + j] != kc) continue;
+          int a = s.x_parent[cbase + j], bnode = s.x_parent[cbase + cand], ra2 = 0, rb2 = 0;
+          while (a != bnode) {
+            ra2 = s.x_rank[a]; rb2 = s.x_rank[bnode];
+            a = s.x_parent[a]; bnode = s.x_parent[bnode];
+          }
+          r += ra2 < rb2;
+        }
+      }
+      if (r < W) {
+        const int at = hi + r, rk = s.x_rank[cbase + cand];
+        s.x_parent[at] = s.x_parent[cbase + cand];
+        s.x_depth[at] = (unsigned char)d;
+        s.x_rank[at] = (unsigned char)rk;
+        s.x_score[at] = s.x_score[cbase + cand];
+        if (d < L && src.bigram) {  // the row this node opens at the next depth: start fetching it now
+          const float* nxt = src.bigram + ((size_t)(d - 1) * k + rk) * k;
+          asm volatile("prefetch.global.L1 [%0];" ::"l"(nxt));
+          if (k > 32) asm volatile("prefetch.global.L1 [%0];" ::"l"(nxt + 32));
+        }
+      }
+    }
+    __syncthreads();
+    lo = hi;
+    hi += nc < W ? nc : W;
+  }
+  return hi;
+}
+
 // eq. 5 and eq. 9, then the sort by (t desc, token asc), one THREAD per (position, predecessor) row, for k <= KP
 // <= 16: the row lives in registers, nothing is exchanged between lanes and the k^2 comparisons are independent
 // of one another.  Element e of the row is visited in an order that starts at tid % k, so that the lanes of a
@@ -1057,6 +1201,17 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   while ((1 << bits) < k) ++bits;
   const bool use_pk = bits * L <= 128;
   bool sequential = LAZY;
+  RowSource src;
+  src.bigram = L > 1 ? bigram + (size_t)b * (L - 1) * kk2 : nullptr;
+  src.anchor_bigram = anchor_bigram ? anchor_bigram + (size_t)b * k : nullptr;
+  if constexpr (LAZY) {
+    if (s.xcap > 0) {  // a small finite width: eq. 11 depth by depth, then eq. 12 on the union
+      const int n = expand_depthwise(s, src, L, k, W, zeta);
+      const int n_sel = select_enumerated<G2_T>(s, n, 1, budget, k);
+      if (tid == 0) s.scalars[0] = n_sel;
+      sequential = false;
+    }
+  }
   if constexpr (!LAZY) {
     int n;
     if (W > 0 && W < budget) {  // a finite width closes depths in order: one warp
@@ -1087,9 +1242,6 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
   }
   if (sequential && tid < 32) {
     int n;
-    RowSource src;
-    src.bigram = L > 1 ? bigram + (size_t)b * (L - 1) * kk2 : nullptr;
-    src.anchor_bigram = anchor_bigram ? anchor_bigram + (size_t)b * k : nullptr;
     if (N <= 64) n = expand_tree<2, LAZY>(s, src, L, k, budget, W, zeta, lane);
     else if (N <= 128) n = expand_tree<4, LAZY>(s, src, L, k, budget, W, zeta, lane);
     else n = expand_tree<8, LAZY>(s, src, L, k, budget, W, zeta, lane);
@@ -1232,7 +1384,8 @@ cudaError_t launch_build_tree(const float* bigram, int B, int L, int k, int N, i
                               const int32_t* anchor_tokens, const int32_t* pos_offset,
                               const ubt_tree& out, const MergeParts& parts, int V, int32_t* status, cudaStream_t st) {
   if (B == 0) return cudaSuccess;
-  const TreeLayout lay = tree_layout(L, k, N);
+  TreeLayout lay = tree_layout(L, k, N, W);
+  if (lay.total > (size_t)device_info().max_smem_optin) lay = tree_layout(L, k, N);  // without the depth-by-depth arrays
   const size_t smem = lay.total;
   const bool lazy = tree_lazy(L, k);
   auto kern = lazy ? k_build_tree<true> : k_build_tree<false>;
