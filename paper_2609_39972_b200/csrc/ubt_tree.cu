@@ -63,11 +63,14 @@ struct TreeSmem {
 __host__ __device__ inline bool tree_lazy(int L, int k) { return (size_t)L * k * k * 5 > kTreeTableBytes; }
 // Nodes the parallel expansion may enumerate before it picks the N - 1 best (root included).
 __host__ __device__ inline int expand_capacity(int N) { return 4 * N < 128 ? 128 : (4 * N > 1024 ? 1024 : 4 * N); }
-// Lazy mode with a small finite width runs eq. 11 depth by depth (expand_depthwise): the node arrays then hold the
-// root and W nodes per depth, followed by a scratch area for the W * min(W, k) candidates of one depth.
-constexpr int kDepthwiseMaxW = 16;
+// Many candidates per position and a small finite width: eq. 11 runs depth by depth (expand_depthwise) on rows
+// normalised on demand, whether or not the pair table would fit (preparing and sorting all L k rows of k = 64
+// entries costs far more than the W rows per depth the search opens).  The node arrays then hold the root and W
+// nodes per depth, followed by a scratch area for the W * min(W, k) candidates of one depth.
+constexpr int kDepthwiseMaxW = 16, kDepthwiseMinK = 17;
 __host__ __device__ inline int depthwise_capacity(int L, int k, int N, int W) {
-  if (!tree_lazy(L, k) || W <= 0 || W >= N - 1 || W > kDepthwiseMaxW) return 0;
+  if (W <= 0 || W >= N - 1 || W > kDepthwiseMaxW) return 0;
+  if (!tree_lazy(L, k) && k < kDepthwiseMinK) return 0;
   return 1 + W * L + W * (W < k ? W : k);
 }
 
@@ -92,7 +95,7 @@ inline TreeLayout tree_layout(int L, int k, int N, int W = 0) {
     return (uint32_t)at;
   };
   const int mw = (N + 31) / 32;
-  const bool lazy = tree_lazy(L, k);
+  const bool lazy = tree_lazy(L, k) || depthwise_capacity(L, k, N, W) > 0;  // rows on demand
   const long long lkk = lazy ? (long long)N * k : (long long)L * k * k, lk = (long long)L * k;
   o.t = take(sizeof(float) * lkk); o.ord = take((size_t)lkk);
   o.rowmap = take(lazy ? sizeof(short) * (lk + 1) : 0); o.la = take(sizeof(float) * L);
@@ -900,6 +903,11 @@ __device__ __forceinline__ int expand_depthwise(TreeSmem& s, const RowSource& sr
           s.x_rank[c] = (unsigned char)rb;
           s.x_score[c] = v[h];
           s.x_key64[c] = k64[h];
+          if (d < L && src.bigram) {  // the row this child would open at the next depth: start fetching it now, the
+            const float* nxt = src.bigram + ((size_t)(d - 1) * k + rb) * k;  // ranking below covers the latency
+            asm volatile("prefetch.global.L1 [%0];" ::"l"(nxt));
+            if (k > 32) asm volatile("prefetch.global.L1 [%0];" ::"l"(nxt + 32));
+          }
         }
       }
       __syncwarp();
@@ -915,11 +923,13 @@ __device__ __forceinline__ int expand_depthwise(TreeSmem& s, const RowSource& sr
     unsigned long long kc = 0ull;
     if (cand < nc) {
       kc = s.x_key64[cbase + cand];
+      const uint32_t sc32 = (uint32_t)(kc >> 32);  // the loop compares score keys only: one load, two operations
+      const uint32_t* hi32 = reinterpret_cast<const uint32_t*>(s.x_key64.ptr(cbase, nc)) + 1;
 #pragma unroll 16
       for (int j = q; j < nc; j += sp) {
-        const unsigned long long kj = s.x_key64[cbase + j];
-        r += kj > kc;
-        same += kj == kc;
+        const uint32_t kj = hi32[2 * j];
+        r += kj > sc32;
+        same += kj == sc32;
       }
     }
     for (int o = sp >> 1; o > 0; o >>= 1) {
@@ -927,9 +937,11 @@ __device__ __forceinline__ int expand_depthwise(TreeSmem& s, const RowSource& sr
       same += __shfl_xor_sync(FULL, same, o);
     }
     if (cand < nc && q == 0) {
-      if (same > 1) {  // same score and token under other parents: the parents' rank paths decide
+      if (same > 1) {  // equal scores (rare): the token decides, then the parents' rank paths
         for (int j = 0; j < nc; ++j) {
-          if (j == cand || s.x_key64[cbase + j] != kc) continue;
+          const unsigned long long kj = s.x_key64[cbase + j];
+          if (j == cand || (uint32_t)(kj >> 32) != (uint32_t)(kc >> 32)) continue;
+          if (kj != kc) { r += kj > kc; continue; }
           int a = s.x_parent[cbase + j], bnode = s.x_parent[cbase + cand], ra2 = 0, rb2 = 0;
           while (a != bnode) {
             ra2 = s.x_rank[a]; rb2 = s.x_rank[bnode];
@@ -944,11 +956,6 @@ __device__ __forceinline__ int expand_depthwise(TreeSmem& s, const RowSource& sr
         s.x_depth[at] = (unsigned char)d;
         s.x_rank[at] = (unsigned char)rk;
         s.x_score[at] = s.x_score[cbase + cand];
-        if (d < L && src.bigram) {  // the row this node opens at the next depth: start fetching it now
-          const float* nxt = src.bigram + ((size_t)(d - 1) * k + rk) * k;
-          asm volatile("prefetch.global.L1 [%0];" ::"l"(nxt));
-          if (k > 32) asm volatile("prefetch.global.L1 [%0];" ::"l"(nxt + 32));
-        }
       }
     }
     __syncthreads();
@@ -1387,7 +1394,7 @@ cudaError_t launch_build_tree(const float* bigram, int B, int L, int k, int N, i
   TreeLayout lay = tree_layout(L, k, N, W);
   if (lay.total > (size_t)device_info().max_smem_optin) lay = tree_layout(L, k, N);  // without the depth-by-depth arrays
   const size_t smem = lay.total;
-  const bool lazy = tree_lazy(L, k);
+  const bool lazy = lay.lazy != 0;
   auto kern = lazy ? k_build_tree<true> : k_build_tree<false>;
   cudaError_t e = lazy ? allow_max_dynamic_smem<k_build_tree<true>>() : allow_max_dynamic_smem<k_build_tree<false>>();
   if (e != cudaSuccess) return e;
