@@ -63,14 +63,13 @@ struct TreeSmem {
 __host__ __device__ inline bool tree_lazy(int L, int k) { return (size_t)L * k * k * 5 > kTreeTableBytes; }
 // Nodes the parallel expansion may enumerate before it picks the N - 1 best (root included).
 __host__ __device__ inline int expand_capacity(int N) { return 4 * N < 128 ? 128 : (4 * N > 1024 ? 1024 : 4 * N); }
-// Many candidates per position and a small finite width: eq. 11 runs depth by depth (expand_depthwise) on rows
-// normalised on demand, whether or not the pair table would fit (preparing and sorting all L k rows of k = 64
-// entries costs far more than the W rows per depth the search opens).  The node arrays then hold the root and W
-// nodes per depth, followed by a scratch area for the W * min(W, k) candidates of one depth.
-constexpr int kDepthwiseMaxW = 16, kDepthwiseMinK = 17;
+// A small finite width: eq. 11 runs depth by depth (expand_depthwise) on rows normalised on demand, whether or not
+// the pair table would fit -- the search opens W rows per depth, and preparing just those is cheaper than the
+// whole table.  The node arrays then hold the root and W nodes per depth, followed by a scratch area for the
+// W * min(W, k) candidates of one depth.
+constexpr int kDepthwiseMaxW = 16;
 __host__ __device__ inline int depthwise_capacity(int L, int k, int N, int W) {
   if (W <= 0 || W >= N - 1 || W > kDepthwiseMaxW) return 0;
-  if (!tree_lazy(L, k) && k < kDepthwiseMinK) return 0;
   return 1 + W * L + W * (W < k ? W : k);
 }
 
