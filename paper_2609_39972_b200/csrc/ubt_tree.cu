@@ -56,7 +56,7 @@ struct TreeSmem {
   Span<short> x_aux;        // [xcap] per-round scratch
   Span<unsigned long long> x_key64;  // [xcap] ordering keys of the final choice
   Span<int> x_wsum;         // [32] warp totals of the block scans
-  Span<unsigned long long> dw_row;  // depth-by-depth expansion: [warps, k] ordering keys of the row a warp has open
+  Span<unsigned long long> dw_row;  // [warps, k] ordering keys of the row a warp is ranking
 };
 
 // Rows of the pair table are computed on demand when the whole table would not fit.
@@ -114,7 +114,7 @@ inline TreeLayout tree_layout(int L, int k, int N, int W = 0) {
   o.x_bak = take(xcap); o.x_score = take(sizeof(float) * xcap); o.x_key = take(sizeof(uint32_t) * xcap);
   o.x_aux = take(sizeof(short) * xcap); o.x_wsum = take(sizeof(int) * 32);
   o.x_key64 = take(sizeof(unsigned long long) * xcap);
-  o.dw_row = take(lazy && xcap > 0 ? sizeof(unsigned long long) * (G2_T / 32) * k : 0);
+  o.dw_row = take(sizeof(unsigned long long) * (G2_T / 32) * k);
   o.total = (uint32_t)off;
   return o;
 }
@@ -134,7 +134,7 @@ __device__ __forceinline__ void tree_bind(TreeSmem* s, unsigned char* base, cons
   s->x_aux = Span<short>((short*)(base + o.x_aux), xcap, 128);
   s->x_wsum = Span<int>((int*)(base + o.x_wsum), 32, 129);
   s->x_key64 = Span<unsigned long long>((unsigned long long*)(base + o.x_key64), xcap, 130);
-  s->dw_row = Span<unsigned long long>((unsigned long long*)(base + o.dw_row), lazy && xcap > 0 ? (long long)(G2_T / 32) * k : 0, 131);
+  s->dw_row = Span<unsigned long long>((unsigned long long*)(base + o.dw_row), (long long)(G2_T / 32) * k, 131);
   s->t = Span<float>((float*)(base + o.t), lkk, 101);
   s->ord = Span<unsigned char>(base + o.ord, lkk, 102);
   s->rowmap = Span<short>((short*)(base + o.rowmap), lazy ? lk + 1 : 0, 107);
@@ -197,10 +197,35 @@ __device__ __forceinline__ void prefetch_row(TreeSmem& s, const RowSource& src, 
     }
   }
 }
+// One warp ranks the k <= 64 entries of a row (two per lane: lane and lane + 32) under (value desc, token asc): the
+// (value key, ~token) keys meet in the warp's scratch and every lane counts the keys in front of its two entries
+// -- k independent shared-memory loads, no warp-wide reductions, no extraction rounds.  The candidates of a
+// position are distinct tokens, so the keys are distinct and the ranks a permutation.  k64[h] receives the keys.
+__device__ __forceinline__ void rank_row_warp(TreeSmem& s, const float (&v)[2], const uint32_t (&ntok)[2], int k, int lane,
+                                              unsigned long long (&k64)[2], int& r0, int& r1) {
+  unsigned long long* rowkeys = s.dw_row.ptr((long long)(threadIdx.x >> 5) * k, k);
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    uint32_t kh = f2key(v[h]);
+    kh = kh == 0u ? 1u : kh;
+    k64[h] = ((unsigned long long)kh << 32) | ntok[h];
+    if (lane + 32 * h < k) rowkeys[lane + 32 * h] = k64[h];
+  }
+  __syncwarp();
+  r0 = 0; r1 = 0;
+#pragma unroll 16
+  for (int j = 0; j < k; ++j) {  // (unrolled: sixteen loads in flight; the loop is latency otherwise)
+    const unsigned long long kj = rowkeys[j];
+    r0 += kj > k64[0];
+    r1 += kj > k64[1];
+  }
+  __syncwarp();  // the scratch may be overwritten by the warp's next row
+}
+
 // One warp: eq. 5 and eq. 9 for row q from the raw scores in prefetch slot e, then its `m` best successors under
 // (t desc, token asc) into cache slot `slot` (the search never looks further down a row: at most W, or the whole
-// budget, of its entries can be accepted, plus one that is dropped).  Successors are extracted one per round by
-// a warp maximum over (score key, ~token); the candidates of a position are distinct tokens.
+// budget, of its entries can be accepted, plus one that is dropped).  The candidates of a position are distinct
+// tokens, so (value key, ~token) orders a row strictly.
 __device__ __forceinline__ void lazy_row(TreeSmem& s, int q, int e, int slot, int k, int m, int lane) {
   const int i = q / k;
   const float al = s.al[i], la = s.la[i];
@@ -225,22 +250,16 @@ __device__ __forceinline__ void lazy_row(TreeSmem& s, int q, int e, int slot, in
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(FULL, sum, o);
   const float lse = mx + logf(sum);
-  uint32_t key[2];
+  v[0] -= lse; v[1] -= lse;
+  unsigned long long k64[2];
+  int r0, r1;
+  rank_row_warp(s, v, ntok, k, lane, k64, r0, r1);
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
-    v[h] -= lse;
-    key[h] = lane + 32 * h < k ? f2key(v[h]) : 0u;  // 0: not a successor / already taken
-  }
-  for (int j = 0; j < m; ++j) {
-    const bool first = key[0] > key[1] || (key[0] == key[1] && ntok[0] >= ntok[1]);
-    const uint32_t bk = first ? key[0] : key[1], bt = first ? ntok[0] : ntok[1];
-    const uint32_t mk = __reduce_max_sync(FULL, bk);
-    const uint32_t mt = __reduce_max_sync(FULL, bk == mk ? bt : 0u);
-    const unsigned holders = __ballot_sync(FULL, bk == mk && bt == mt);
-    if (lane == __ffs(holders) - 1) {
-      s.t[(long long)slot * k + j] = first ? v[0] : v[1];
-      s.ord[(long long)slot * k + j] = (unsigned char)(first ? lane : lane + 32);
-      if (first) key[0] = 0u; else key[1] = 0u;
+    const int rb = lane + 32 * h, r = h == 0 ? r0 : r1;
+    if (rb < k && r < m) {
+      s.t[(long long)slot * k + r] = v[h];
+      s.ord[(long long)slot * k + r] = (unsigned char)rb;
     }
   }
   __syncwarp();
@@ -871,32 +890,17 @@ __device__ __forceinline__ int expand_depthwise(TreeSmem& s, const RowSource& sr
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(FULL, sum, o);
       const float lse = mx + logf(sum);
-      // the row's ordering keys (score, ~token) meet in shared memory; every lane then counts, for its two
-      // children, the keys in front of them (64 independent loads: no warp-wide reductions, no rounds) and the
-      // children with fewer than m in front write their records to the candidate place of that rank
-      unsigned long long k64[2];
-      unsigned long long* rowkeys = s.dw_row.ptr((long long)warp * k, k);
+      // the children's scores, ranked within the row; those with fewer than m in front become candidates of the
+      // depth at the place of that rank
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        const int rb = lane + 32 * h;
-        v[h] = sc + (v[h] - lse) + zeta;  // the child's score
-        uint32_t kh = f2key(v[h]);
-        kh = kh == 0u ? 1u : kh;
-        k64[h] = ((unsigned long long)kh << 32) | ntok[h];
-        if (rb < k) rowkeys[rb] = k64[h];
-      }
-      __syncwarp();
-      int r0 = 0, r1 = 0;
-#pragma unroll 16
-      for (int j = 0; j < k; ++j) {  // (unrolled: sixteen loads in flight; the loop is latency otherwise)
-        const unsigned long long kj = rowkeys[j];
-        r0 += kj > k64[0];
-        r1 += kj > k64[1];
-      }
+      for (int h = 0; h < 2; ++h) v[h] = sc + (v[h] - lse) + zeta;
+      unsigned long long k64[2];
+      int r0, r1;
+      rank_row_warp(s, v, ntok, k, lane, k64, r0, r1);
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         const int rb = lane + 32 * h, r = h == 0 ? r0 : r1;
-        if (rb < k && r < m) {  // tokens of a position are distinct, so the keys of a row are
+        if (rb < k && r < m) {
           const int c = cbase + p * m + r;
           s.x_parent[c] = (short)node;
           s.x_rank[c] = (unsigned char)rb;
@@ -1102,99 +1106,45 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
     else if (kp == 4) prepare_rows_by_thread<4>(s, k, nrows, tid);
     else if (kp == 8) prepare_rows_by_thread<8>(s, k, nrows, tid);
     else prepare_rows_by_thread<16>(s, k, nrows, tid);
-  } else if (k <= 32) {
-    // ---- eq. 5 and eq. 9, then every row sorted by (t desc, token asc): a group of kp = 2^ceil(log2 k)
-    // lanes per (position, predecessor) row, the row's values in registers, reductions and exact ranks by
-    // shuffles inside the group; integer keys and a final index tie-break keep the ranks a permutation
-    // whatever the values are (even NaN).  Several rows are in flight per warp and no CTA barrier is needed.
-    __syncthreads();  // s.lp, s.tok
-    const int gpw = 32 / kp, rb = lane & (kp - 1);
-    const int gid = (tid >> 5) * gpw + lane / kp, ngroups = (G2_T / 32) * gpw;
-    for (int r0 = 0; r0 < nrows; r0 += ngroups) {
-      const int r = r0 + gid;
-      const bool active = r < nrows && rb < k;
-      const int i = r <= 0 ? 0 : 1 + (r - 1) / k;
-      const int ra = r <= 0 ? 0 : (r - 1) % k;
-      float v = -INFINITY;
-      int tk = 0;
-      const int at = (i * k + ra) * k;
-      if (active) {
-        v = fmaf(s.al[i], s.lp[i * k + rb], s.t[at + rb]);
-        tk = s.tok[i * k + rb];
-      }
-      float mx = v;
-      for (int o = kp >> 1; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, o));
-      float sum = active ? expf(v - mx) : 0.f;
-      for (int o = kp >> 1; o > 0; o >>= 1) sum += __shfl_xor_sync(FULL, sum, o);
-      const float tv = v - (mx + logf(sum));
-      const uint32_t kv = f2key(tv);
-      int rank = 0;
-      bool tie = false;
-#pragma unroll 4
-      for (int j = 0; j < k; ++j) {
-        const uint32_t kj = __shfl_sync(FULL, kv, j, kp);
-        rank += kj > kv;
-        tie |= kj == kv && j != rb;
-      }
-      if (__any_sync(FULL, tie && active)) {  // equal values in one row (rare): token, then index, decide
-        rank = 0;
-        for (int j = 0; j < k; ++j) {
-          const uint32_t kj = __shfl_sync(FULL, kv, j, kp);
-          const int tj = __shfl_sync(FULL, tk, j, kp);
-          rank += (kj > kv) || (kj == kv && (tj < tk || (tj == tk && j < rb)));
-        }
-      }
-      if (active) {
-        s.t[at + rank] = tv;
-        s.ord[at + rank] = (unsigned char)rb;
-      }
-    }
   } else {
-    __syncthreads();
-    // eq. 5 and eq. 9: one thread per (position, predecessor) row
-    for (int r = tid; r < nrows; r += G2_T) {
+    // 16 < k <= 64: one warp per (position, predecessor) row, two entries per lane; eq. 5, eq. 9, ranks by counting
+    __syncthreads();  // s.lp, s.tok
+    for (int r = tid >> 5; r < nrows; r += G2_T / 32) {
       const int i = r == 0 ? 0 : 1 + (r - 1) / k;
       const int ra = r == 0 ? 0 : (r - 1) % k;
-      float* row = s.t.ptr(((long long)i * k + ra) * k, k);
+      const int at = (i * k + ra) * k;
       const float al = s.al[i];
-      float mx = -INFINITY;
-      for (int rb = 0; rb < k; ++rb) {
-        float v = fmaf(al, s.lp[i * k + rb], row[rb]);
-        row[rb] = v;
-        mx = fmaxf(mx, v);
-      }
-      float sum = 0.f;
-      for (int rb = 0; rb < k; ++rb) sum += expf(row[rb] - mx);
-      const float lse = mx + logf(sum);
-      for (int rb = 0; rb < k; ++rb) row[rb] -= lse;
-    }
-    __syncthreads();
-    // in-place sort, whole rows per batch: a row is read completely before it is rewritten
-    const int rows_per_batch = G2_T / k;
-    for (int row0 = 0; row0 < nrows; row0 += rows_per_batch) {
-      const int r = row0 + tid / k, rb = tid % k;
-      const bool active = tid < rows_per_batch * k && r < nrows;
-      float v = 0.f;
-      int rank = 0, at = 0;
-      if (active) {
-        const int i = r == 0 ? 0 : 1 + (r - 1) / k;
-        const int ra = r == 0 ? 0 : (r - 1) % k;
-        at = (i * k + ra) * k;
-        const float* row = s.t.ptr(at, k);
-        const int* tk = s.tok.ptr((long long)i * k, k);
-        v = row[rb];
-        const uint32_t kv = f2key(v);
-        for (int j = 0; j < k; ++j) {
-          const uint32_t kj = f2key(row[j]);
-          rank += (kj > kv) || (kj == kv && (tk[j] < tk[rb] || (tk[j] == tk[rb] && j < rb)));
+      float v[2];
+      uint32_t ntok[2];
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int rb = lane + 32 * h;
+        v[h] = -INFINITY;
+        ntok[h] = 0u;
+        if (rb < k) {
+          v[h] = fmaf(al, s.lp[i * k + rb], s.t[at + rb]);
+          ntok[h] = ~(uint32_t)s.tok[i * k + rb];
         }
       }
-      __syncthreads();  // all reads of this batch of rows precede the in-place writes
-      if (active) {
-        s.t[at + rank] = v;
-        s.ord[at + rank] = (unsigned char)rb;
+      float mx = fmaxf(v[0], v[1]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, o));
+      float sum = (lane < k ? expf(v[0] - mx) : 0.f) + (lane + 32 < k ? expf(v[1] - mx) : 0.f);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(FULL, sum, o);
+      const float lse = mx + logf(sum);
+      v[0] -= lse; v[1] -= lse;
+      unsigned long long k64[2];
+      int r0, r1;
+      rank_row_warp(s, v, ntok, k, lane, k64, r0, r1);  // (every lane has read its raw entries: the row may be rewritten)
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int rb = lane + 32 * h, rk = h == 0 ? r0 : r1;
+        if (rb < k) {
+          s.t[at + rk] = v[h];
+          s.ord[at + rk] = (unsigned char)rb;
+        }
       }
-      __syncthreads();
     }
   }
   __syncthreads();
