@@ -11,7 +11,7 @@ LIB = os.path.join(HERE, "libubt.so")
 CHECKED_LIB = os.path.join(HERE, "libubt_checked.so")   # -DUBT_BOUNDS_CHECK debug build
 SOURCES = ["ubt_api.cu", "ubt_topk.cu", "ubt_tree.cu", "ubt_verify.cu", "ubt_verify_path.cu", "ubt_noalloc.cu",
            "ubt_selector.cu", "ubt_lmhead.cu"]
-HEADERS = ["ubt_common.cuh", "ubt_internal.h", "ubt_merge.cuh", "ubt_ring.cuh", "ubt_pick.cuh", os.path.join("..", "..", "include", "ubt.h")]
+HEADERS = ["ubt_common.cuh", "ubt_internal.h", "ubt_merge.cuh", "ubt_ring.cuh", "ubt_pick.cuh", "ubt_tc.cuh", os.path.join("..", "..", "include", "ubt.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

@@ -568,11 +568,12 @@ cudaError_t lm_head_timeouts(unsigned int* out);
 }  // namespace ubt
 extern "C" {
 long long ubt_debug_ring_timeouts(void) {
-  unsigned int a = 0, b = 0, c = 0, d = 0;
+  unsigned int a = 0, b = 0, c = 0, d = 0, e = 0;
   if (ring_timeouts_verify(&a) != cudaSuccess || ring_timeouts_topk(&b) != cudaSuccess ||
-      ring_timeouts_path(&c) != cudaSuccess || lm_head_timeouts(&d) != cudaSuccess)
+      ring_timeouts_path(&c) != cudaSuccess || lm_head_timeouts(&d) != cudaSuccess ||
+      selector_timeouts(&e) != cudaSuccess)
     return -1;
-  return (long long)a + b + c + d;
+  return (long long)a + b + c + d + e;
 }
 
 #ifdef UBT_BOUNDS_CHECK

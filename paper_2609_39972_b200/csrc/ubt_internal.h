@@ -135,6 +135,8 @@ cudaError_t launch_row_keys_shard(const VerifyWorkspace& w, int64_t rows, int V,
 cudaError_t launch_walk_keys(const ubt_tree& tree, const unsigned long long* gathered_keys, int shards,
                              int32_t* node_pick, const ubt_verify_result& out, int32_t* status, cudaStream_t st);
 
+cudaError_t selector_timeouts(unsigned int* out);
+
 // ---- LM head fused with a1 (ubt_lmhead.cu): tcgen05 GEMM whose epilogue keeps (max, sum exp, top-k) per row
 int lm_head_max_k();
 int lm_head_max_rows();

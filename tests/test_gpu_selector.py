@@ -18,7 +18,8 @@ def _dev_table(a, dtype):
 
 @pytest.mark.parametrize("dtype,V,R,B,L,k", [("f32", 3000, 64, 3, 5, 6), ("bf16", 3000, 64, 3, 5, 6),
                                              ("bf16", 5000, 256, 2, 4, 64), ("f32", 700, 1024, 2, 3, 8), ("bf16", 900, 1000, 2, 3, 64),
-                                             ("bf16", 900, 8, 1, 1, 4)])
+                                             ("bf16", 900, 8, 1, 1, 4), ("bf16", 2000, 128, 2, 3, 33),
+                                             ("bf16", 2000, 192, 1, 2, 17)])
 def test_scores_match_the_oracle(dtype, V, R, B, L, k):
     import paper_2609_39972_b200 as u
     phi, psi, gate = synth.selector_tables(V, R, B, L, 7, dtype)
