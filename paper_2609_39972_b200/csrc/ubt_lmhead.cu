@@ -29,6 +29,7 @@
 #include <mutex>
 
 #include "ubt_internal.h"
+#include "ubt_tc.cuh"
 
 namespace ubt {
 
@@ -50,15 +51,14 @@ struct LmShared {  // behind the ring in dynamic shared memory
   int fail;
 };
 
-__device__ __forceinline__ uint32_t lm_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void lm_bar_init(uint64_t* bar, int count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(lm_smem(bar)), "r"(count));
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(tc_smem(bar)), "r"(count));
 }
 __device__ __forceinline__ void lm_bar_expect(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(lm_smem(bar)), "r"(bytes) : "memory");
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(tc_smem(bar)), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void lm_bar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(lm_smem(bar)) : "memory");
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(tc_smem(bar)) : "memory");
 }
 // Bounded wait for the phase with the given parity; false = gave up (counted).
 __device__ __forceinline__ bool lm_bar_wait(uint64_t* bar, uint32_t parity, volatile int* fail) {
@@ -66,7 +66,7 @@ __device__ __forceinline__ bool lm_bar_wait(uint64_t* bar, uint32_t parity, vola
     uint32_t ok;
     asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
                  : "=r"(ok)
-                 : "r"(lm_smem(bar)), "r"(parity)
+                 : "r"(tc_smem(bar)), "r"(parity)
                  : "memory");
     if (ok) return true;
     if ((spins & 1023) == 1023 && *fail) return false;  // another role already gave up
@@ -78,49 +78,12 @@ __device__ __forceinline__ bool lm_bar_wait(uint64_t* bar, uint32_t parity, vola
 // 2-D tiled bulk load (TMA) of this GPU's own memory; completes on the mbarrier with its byte count.
 __device__ __forceinline__ void lm_tma_load(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
   asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
-                   lm_smem(dst)),
-               "l"(map), "r"(x), "r"(y), "r"(lm_smem(bar))
+                   tc_smem(dst)),
+               "l"(map), "r"(x), "r"(y), "r"(tc_smem(bar))
                : "memory");
 }
-// Shared-memory matrix descriptor of a K-major bf16 tile stored as rows of 128 bytes under the 128-byte swizzle:
-// start address, stride between groups of eight rows (1024 bytes), descriptor version 1, swizzle mode 2.
-__device__ __forceinline__ uint64_t lm_desc(uint32_t smem_addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((smem_addr & 0x3ffffu) >> 4);        // [0,14)  start address >> 4
-  d |= (uint64_t)1 << 16;                              // [16,30) leading byte offset >> 4 (unused with this swizzle)
-  d |= (uint64_t)(1024 >> 4) << 32;                    // [32,46) stride byte offset >> 4
-  d |= (uint64_t)1 << 46;                              // [46,48) descriptor version
-  d |= (uint64_t)2 << 61;                              // [61,64) 128-byte swizzle
-  return d;
-}
 // Instruction descriptor: fp32 accumulator, bf16 x bf16, both operands K-major, N = 256, M = 128.
-constexpr uint32_t kLmIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(LM_BN >> 3) << 17) | ((uint32_t)(LM_BM >> 4) << 24);
-
-__device__ __forceinline__ void lm_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t"
-      ".reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t"
-      "}\n" ::"r"(d_tmem),
-      "l"(adesc), "l"(bdesc), "r"(kLmIdesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
-      : "memory");
-}
-__device__ __forceinline__ void lm_commit(uint64_t* bar) {  // arrives on the barrier when the MMAs issued so far are done
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(lm_smem(bar)) : "memory");
-}
-__device__ __forceinline__ void lm_tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
+constexpr uint32_t kLmIdesc = tc_idesc_bf16(LM_BM, LM_BN);
 
 struct LmParts {                   // one partial per (CTA, row of the launch's row block)
   float* ms;                       // [grid, rpad, 2] (max, sum exp relative to it)
@@ -173,7 +136,7 @@ k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant_
     sh.fail = 0;
   }
   if (warp == 1) {  // tensor memory: both accumulators (512 columns), allocated by one warp
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(lm_smem(&sh.tmem_base)), "r"(512u) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc_smem(&sh.tmem_base)), "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -216,7 +179,7 @@ k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant_
           ok = lm_bar_wait(&sh.full[s], ph, fail);
           if (!ok) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t a_addr = lm_smem(ring + (size_t)s * stage_bytes), b_addr = a_addr + (uint32_t)a_bytes;
+          const uint32_t a_addr = tc_smem(ring + (size_t)s * stage_bytes), b_addr = a_addr + (uint32_t)a_bytes;
 #pragma unroll
           for (int half = 0; half < 2; ++half) {  // rows 0-127 -> accumulator 0, rows 128-255 -> accumulator 1
             if (half >= n_half) break;
@@ -229,14 +192,14 @@ k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant_
             const uint32_t ah = a_addr + (uint32_t)(half * LM_BM * LM_BK * 2);
 #pragma unroll
             for (int kk = 0; kk < LM_BK / 16; ++kk)  // 16 bf16 = 32 bytes along K inside the swizzled row
-              lm_mma(d_tmem, lm_desc(ah + kk * 32), lm_desc(b_addr + kk * 32), (kb | kk) != 0 ? 1u : 0u);
+              tc_mma(d_tmem, tc_desc(ah + kk * 32), tc_desc(b_addr + kk * 32), kLmIdesc, (kb | kk) != 0 ? 1u : 0u);
           }
           if (!ok) break;
-          lm_commit(&sh.empty[s]);  // the stage may be refilled once these MMAs have read it
+          tc_commit(&sh.empty[s]);  // the stage may be refilled once these MMAs have read it
         }
         if (!ok) break;
         for (int half = 0; half < n_half; ++half) {  // complete once every MMA above is
-          lm_commit(&sh.acc_full[half]);
+          tc_commit(&sh.acc_full[half]);
           use[half] += 1u;
         }
       }
@@ -275,7 +238,7 @@ k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant_
 #pragma unroll 1
       for (int c0 = 0; c0 < LM_BN; c0 += 32) {
         uint32_t r[32];
-        lm_tmem_ld32(taddr + (uint32_t)c0, r);
+        tc_tmem_ld32(taddr + (uint32_t)c0, r);
         const int ncol = V - (col_base + c0);     // columns of this chunk that exist (the last tile is ragged)
         if (ncol <= 0 || !valid) continue;        // (every lane still took part in the load above)
         if (ncol < 32) {
