@@ -198,26 +198,48 @@ __device__ __forceinline__ void prefetch_row(TreeSmem& s, const RowSource& src, 
   }
 }
 // One warp ranks the k <= 64 entries of a row (two per lane: lane and lane + 32) under (value desc, token asc): the
-// (value key, ~token) keys meet in the warp's scratch and every lane counts the keys in front of its two entries
-// -- k independent shared-memory loads, no warp-wide reductions, no extraction rounds.  The candidates of a
-// position are distinct tokens, so the keys are distinct and the ranks a permutation.  k64[h] receives the keys.
+// 32-bit value keys meet in the warp's scratch and every lane counts the keys in front of its two entries -- k
+// independent shared-memory loads and 2 k compares, no warp-wide reductions, no extraction rounds.  Equal values
+// (rare) would give two entries the same rank: every entry marks the place of its rank with its index, an entry
+// that finds another index there was tied, and the warp then counts again with the full (value key, ~token) keys,
+// which are distinct because the candidates of a position are distinct tokens.  k64[h] receives the full keys.
 __device__ __forceinline__ void rank_row_warp(TreeSmem& s, const float (&v)[2], const uint32_t (&ntok)[2], int k, int lane,
                                               unsigned long long (&k64)[2], int& r0, int& r1) {
   unsigned long long* rowkeys = s.dw_row.ptr((long long)(threadIdx.x >> 5) * k, k);
+  uint32_t* key32 = reinterpret_cast<uint32_t*>(rowkeys);      // [k] value keys, then [k] marks
+  uint32_t kv[2];
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
-    uint32_t kh = f2key(v[h]);
-    kh = kh == 0u ? 1u : kh;
-    k64[h] = ((unsigned long long)kh << 32) | ntok[h];
-    if (lane + 32 * h < k) rowkeys[lane + 32 * h] = k64[h];
+    kv[h] = f2key(v[h]);
+    kv[h] = kv[h] == 0u ? 1u : kv[h];
+    k64[h] = ((unsigned long long)kv[h] << 32) | ntok[h];
+    if (lane + 32 * h < k) key32[lane + 32 * h] = kv[h];
   }
   __syncwarp();
   r0 = 0; r1 = 0;
 #pragma unroll 16
   for (int j = 0; j < k; ++j) {  // (unrolled: sixteen loads in flight; the loop is latency otherwise)
-    const unsigned long long kj = rowkeys[j];
-    r0 += kj > k64[0];
-    r1 += kj > k64[1];
+    const uint32_t kj = key32[j];
+    r0 += kj > kv[0];
+    r1 += kj > kv[1];
+  }
+  // a place per rank: ties collide
+  if (lane < k) key32[k + r0] = (uint32_t)lane;
+  if (lane + 32 < k) key32[k + r1] = (uint32_t)(lane + 32);
+  __syncwarp();
+  const bool clash = (lane < k && key32[k + r0] != (uint32_t)lane) || (lane + 32 < k && key32[k + r1] != (uint32_t)(lane + 32));
+  if (__any_sync(FULL, clash)) {  // equal values in the row: rank again on (value key, ~token)
+    __syncwarp();
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+      if (lane + 32 * h < k) rowkeys[lane + 32 * h] = k64[h];
+    __syncwarp();
+    r0 = 0; r1 = 0;
+    for (int j = 0; j < k; ++j) {
+      const unsigned long long kj = rowkeys[j];
+      r0 += kj > k64[0];
+      r1 += kj > k64[1];
+    }
   }
   __syncwarp();  // the scratch may be overwritten by the warp's next row
 }
