@@ -56,7 +56,8 @@ struct TreeSmem {
   Span<short> x_aux;        // [xcap] per-round scratch
   Span<unsigned long long> x_key64;  // [xcap] ordering keys of the final choice
   Span<int> x_wsum;         // [32] warp totals of the block scans
-  Span<unsigned long long> dw_row;  // [warps, k] ordering keys of the row a warp is ranking
+  Span<unsigned long long> dw_row;  // [warps, k rounded up to 4] ordering keys of the row a warp is ranking
+  Span<uint32_t> dw_ckey;           // depth-by-depth expansion: score keys of a depth's candidates, packed
 };
 
 // Rows of the pair table are computed on demand when the whole table would not fit.
@@ -79,7 +80,7 @@ __host__ __device__ inline int depthwise_capacity(int L, int k, int N, int W) {
 struct TreeLayout {
   uint32_t t, ord, rowmap, la, pre, lp, tok, al, ent, nd_parent, nd_depth, nd_rank, nd_score, nd_slot, nd_pk, kk,
       depth_cnt, depth_off, x_fill, maskrow, scalars, x_parent, x_depth, x_rank, x_next, x_bak, x_score, x_key, x_aux,
-      x_wsum, x_key64, dw_row;
+      x_wsum, x_key64, dw_row, dw_ckey;
   uint32_t total;
   int xcap;
   int lazy;
@@ -114,7 +115,8 @@ inline TreeLayout tree_layout(int L, int k, int N, int W = 0) {
   o.x_bak = take(xcap); o.x_score = take(sizeof(float) * xcap); o.x_key = take(sizeof(uint32_t) * xcap);
   o.x_aux = take(sizeof(short) * xcap); o.x_wsum = take(sizeof(int) * 32);
   o.x_key64 = take(sizeof(unsigned long long) * xcap);
-  o.dw_row = take(sizeof(unsigned long long) * (G2_T / 32) * k);
+  o.dw_row = take(sizeof(unsigned long long) * (G2_T / 32) * ((k + 3) & ~3));
+  o.dw_ckey = take(sizeof(uint32_t) * kDepthwiseMaxW * kDepthwiseMaxW);
   o.total = (uint32_t)off;
   return o;
 }
@@ -134,7 +136,8 @@ __device__ __forceinline__ void tree_bind(TreeSmem* s, unsigned char* base, cons
   s->x_aux = Span<short>((short*)(base + o.x_aux), xcap, 128);
   s->x_wsum = Span<int>((int*)(base + o.x_wsum), 32, 129);
   s->x_key64 = Span<unsigned long long>((unsigned long long*)(base + o.x_key64), xcap, 130);
-  s->dw_row = Span<unsigned long long>((unsigned long long*)(base + o.dw_row), (long long)(G2_T / 32) * k, 131);
+  s->dw_row = Span<unsigned long long>((unsigned long long*)(base + o.dw_row), (long long)(G2_T / 32) * ((k + 3) & ~3), 131);
+  s->dw_ckey = Span<uint32_t>((uint32_t*)(base + o.dw_ckey), kDepthwiseMaxW * kDepthwiseMaxW, 132);
   s->t = Span<float>((float*)(base + o.t), lkk, 101);
   s->ord = Span<unsigned char>(base + o.ord, lkk, 102);
   s->rowmap = Span<short>((short*)(base + o.rowmap), lazy ? lk + 1 : 0, 107);
@@ -205,29 +208,36 @@ __device__ __forceinline__ void prefetch_row(TreeSmem& s, const RowSource& src, 
 // which are distinct because the candidates of a position are distinct tokens.  k64[h] receives the full keys.
 __device__ __forceinline__ void rank_row_warp(TreeSmem& s, const float (&v)[2], const uint32_t (&ntok)[2], int k, int lane,
                                               unsigned long long (&k64)[2], int& r0, int& r1) {
-  unsigned long long* rowkeys = s.dw_row.ptr((long long)(threadIdx.x >> 5) * k, k);
-  uint32_t* key32 = reinterpret_cast<uint32_t*>(rowkeys);      // [k] value keys, then [k] marks
+  const int kpad = (k + 3) & ~3;
+  unsigned long long* rowkeys = s.dw_row.ptr((long long)(threadIdx.x >> 5) * kpad, kpad);
+  uint32_t* key32 = reinterpret_cast<uint32_t*>(rowkeys);      // [kpad] value keys (0 = none), then [kpad] marks
   uint32_t kv[2];
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
+    const int rb = lane + 32 * h;
     kv[h] = f2key(v[h]);
     kv[h] = kv[h] == 0u ? 1u : kv[h];
     k64[h] = ((unsigned long long)kv[h] << 32) | ntok[h];
-    if (lane + 32 * h < k) key32[lane + 32 * h] = kv[h];
+    if (rb < kpad) key32[rb] = rb < k ? kv[h] : 0u;
   }
   __syncwarp();
-  r0 = 0; r1 = 0;
-#pragma unroll 16
-  for (int j = 0; j < k; ++j) {  // (unrolled: sixteen loads in flight; the loop is latency otherwise)
-    const uint32_t kj = key32[j];
-    r0 += kj > kv[0];
-    r1 += kj > kv[1];
+  // four keys per load and eight independent counters: a single warp issues a dependent instruction only every
+  // few cycles, so the loop is a matter of keeping independent work in flight
+  const uint4* key128 = reinterpret_cast<const uint4*>(key32);
+  int a0 = 0, a1 = 0, a2 = 0, a3 = 0, b0 = 0, b1 = 0, b2 = 0, b3 = 0;
+#pragma unroll 4
+  for (int j = 0; j < kpad / 4; ++j) {
+    const uint4 q = key128[j];
+    a0 += q.x > kv[0]; a1 += q.y > kv[0]; a2 += q.z > kv[0]; a3 += q.w > kv[0];
+    b0 += q.x > kv[1]; b1 += q.y > kv[1]; b2 += q.z > kv[1]; b3 += q.w > kv[1];
   }
+  r0 = (a0 + a1) + (a2 + a3);
+  r1 = (b0 + b1) + (b2 + b3);
   // a place per rank: ties collide
-  if (lane < k) key32[k + r0] = (uint32_t)lane;
-  if (lane + 32 < k) key32[k + r1] = (uint32_t)(lane + 32);
+  if (lane < k) key32[kpad + r0] = (uint32_t)lane;
+  if (lane + 32 < k) key32[kpad + r1] = (uint32_t)(lane + 32);
   __syncwarp();
-  const bool clash = (lane < k && key32[k + r0] != (uint32_t)lane) || (lane + 32 < k && key32[k + r1] != (uint32_t)(lane + 32));
+  const bool clash = (lane < k && key32[kpad + r0] != (uint32_t)lane) || (lane + 32 < k && key32[kpad + r1] != (uint32_t)(lane + 32));
   if (__any_sync(FULL, clash)) {  // equal values in the row: rank again on (value key, ~token)
     __syncwarp();
 #pragma unroll
@@ -928,6 +938,7 @@ __device__ __forceinline__ int expand_depthwise(TreeSmem& s, const RowSource& sr
           s.x_rank[c] = (unsigned char)rb;
           s.x_score[c] = v[h];
           s.x_key64[c] = k64[h];
+          s.dw_ckey[p * m + r] = (uint32_t)(k64[h] >> 32);
           if (d < L && src.bigram) {  // the row this child would open at the next depth: start fetching it now, the
             const float* nxt = src.bigram + ((size_t)(d - 1) * k + rb) * k;  // ranking below covers the latency
             asm volatile("prefetch.global.L1 [%0];" ::"l"(nxt));
@@ -948,14 +959,24 @@ __device__ __forceinline__ int expand_depthwise(TreeSmem& s, const RowSource& sr
     unsigned long long kc = 0ull;
     if (cand < nc) {
       kc = s.x_key64[cbase + cand];
-      const uint32_t sc32 = (uint32_t)(kc >> 32);  // the loop compares score keys only: one load, two operations
-      const uint32_t* hi32 = reinterpret_cast<const uint32_t*>(s.x_key64.ptr(cbase, nc)) + 1;
-#pragma unroll 16
-      for (int j = q; j < nc; j += sp) {
-        const uint32_t kj = hi32[2 * j];
-        r += kj > sc32;
-        same += kj == sc32;
+      const uint32_t sc32 = (uint32_t)(kc >> 32);  // the loop compares score keys only, four per load
+      const uint4* ck = reinterpret_cast<const uint4*>(s.dw_ckey.ptr(0, (nc + 3) & ~3));
+      const int n4 = nc >> 2;
+      int c0 = 0, c1 = 0, c2 = 0, c3 = 0, e0 = 0, e1 = 0, e2 = 0, e3 = 0;  // independent counters (see rank_row_warp)
+#pragma unroll 4
+      for (int j = q; j < n4; j += sp) {
+        const uint4 w = ck[j];
+        c0 += w.x > sc32; c1 += w.y > sc32; c2 += w.z > sc32; c3 += w.w > sc32;
+        e0 += w.x == sc32; e1 += w.y == sc32; e2 += w.z == sc32; e3 += w.w == sc32;
       }
+      r = (c0 + c1) + (c2 + c3);
+      same = (e0 + e1) + (e2 + e3);
+      if (q == 0)
+        for (int j = n4 * 4; j < nc; ++j) {  // the last one to three
+          const uint32_t kj = s.dw_ckey[j];
+          r += kj > sc32;
+          same += kj == sc32;
+        }
     }
     for (int o = sp >> 1; o > 0; o >>= 1) {
       r += __shfl_xor_sync(FULL, r, o);
