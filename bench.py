@@ -56,7 +56,7 @@ def measured_peak():
 
 
 def measured_tensor_peak():
-    """Dense bf16 TFLOP/s of a library product on this machine: the burst figure, for a kernel timed alone."""
+    """Dense bf16 TFLOP/s of a library product measured on this kind of GPU: the burst figure, for a kernel timed alone."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
         with open(path) as f:
