@@ -252,6 +252,31 @@ def test_exact_score_ties_follow_total_order():
     compare_draft(tree_to_numpy(gtree), otree, L, k, N)
 
 
+@pytest.mark.parametrize("L,V,k,N,W", [(4, 64, 4, 12, 0), (4, 64, 4, 12, 2), (4, 64, 4, 12, 5), (5, 128, 20, 40, 0),
+                                       (5, 128, 20, 40, 4), (6, 128, 40, 60, 6), (15, 256, 64, 65, 12),
+                                       (15, 256, 64, 65, 0), (6, 64, 8, 30, 3), (8, 128, 16, 100, 16)])
+def test_duplicated_values_tie_exactly_in_every_form_of_the_expansion(L, V, k, N, W):
+    """Every logit value occurs twice (tokens 2j and 2j + 1) and lambda = 0, so that the rows of a position do not
+    depend on the predecessor: the two tokens of a pair tie inside every row, sibling nodes of a pair have equal
+    scores, and so have their children of equal rank under either of them -- ties inside a row, across parents
+    and across the final cut, all exact in double and in fp32 alike because the tied values come from identical
+    operations.  Values that are not duplicates differ by O(1).  Every form of the expansion (threshold rounds,
+    depth by depth, best-first on rows prepared on demand) and of the row ranking has to settle the ties by token
+    and rank path as the oracle does."""
+    u = ubt()
+    rng = np.random.default_rng(30 + k + W)
+    B = 3
+    y = (rng.standard_normal((B, L, V // 2)) * 3).astype(np.float32)
+    x = np.repeat(y, 2, axis=2)
+    big = np.zeros((B, L - 1, k, k), np.float32)
+    lam = np.zeros(L, np.float32)
+    otree = oracle.draft_tree(x, big, k, N, lam=lam, W=W)
+    gtree = u.ubt_draft_tree(torch.from_numpy(x).to(DEV), torch.from_numpy(big).to(DEV), k, N,
+                             lam=torch.from_numpy(lam).to(DEV), search_width=W)
+    torch.cuda.synchronize()
+    compare_draft(tree_to_numpy(gtree), otree, L, k, N)
+
+
 def test_split_entry_points_match_fused_call():
     u = ubt()
     cfg = synth.CONFIGS["c2"].replace(V=20000)
