@@ -82,8 +82,6 @@ __device__ __forceinline__ void lm_tma_load(void* dst, const CUtensorMap* map, i
                "l"(map), "r"(x), "r"(y), "r"(tc_smem(bar))
                : "memory");
 }
-// Instruction descriptor: fp32 accumulator, bf16 x bf16, both operands K-major, N = 256, M = 128.
-constexpr uint32_t kLmIdesc = tc_idesc_bf16(LM_BM, LM_BN);
 
 struct LmParts {                   // one partial per (CTA, row of the launch's row block)
   float* ms;                       // [grid, rpad, 2] (max, sum exp relative to it)
@@ -116,14 +114,18 @@ __device__ __forceinline__ void lm_list_state(const unsigned long long (&L)[KR],
 template <int KR>
 __global__ void __launch_bounds__(LM_THREADS, 1)
 k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w, int rows, int d,
-               int V, int k, int a_rows, int n_stages, LmParts parts, int* __restrict__ fail_flag) {
+               int V, int k, int a_rows, int n_stages, int bn, LmParts parts, int* __restrict__ fail_flag) {
   extern __shared__ __align__(1024) unsigned char lm_smem_raw[];
   unsigned char* ring = lm_smem_raw;
   LmShared& sh = *reinterpret_cast<LmShared*>(lm_smem_raw + LM_RING_BYTES);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = gridDim.x, cta = blockIdx.x;
-  const int n_rb = (rows + LM_RB - 1) / LM_RB, n_vt = (V + LM_BN - 1) / LM_BN, n_kb = d / LM_BK;
+  // bn: vocabulary columns of a work item (a multiple of 16, at most LM_BN), chosen on the host so that the items
+  // spread evenly over the CTAs; a stage keeps room for LM_BN weight rows whatever bn is
+  const int n_rb = (rows + LM_RB - 1) / LM_RB, n_vt = (V + bn - 1) / bn, n_kb = d / LM_BK;
   const int a_bytes = a_rows * LM_BK * 2, stage_bytes = a_bytes + LM_B_BYTES;
+  const uint32_t tx_bytes = (uint32_t)(a_bytes + bn * LM_BK * 2);
+  const uint32_t idesc = tc_idesc_bf16(LM_BM, bn);
   // work items: (vocabulary tile, row block) pairs, row block fastest, dealt round-robin: cta, cta + G, ...
   const int n_all = n_vt * n_rb;
   const int n_items = cta < n_all ? (n_all - cta + G - 1) / G : 0;
@@ -154,10 +156,10 @@ k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant_
           const int s = it % n_stages;
           const uint32_t ph = (uint32_t)(it / n_stages) & 1u;
           if (!lm_bar_wait(&sh.empty[s], ph ^ 1u, fail)) break;
-          lm_bar_expect(&sh.full[s], (uint32_t)stage_bytes);
+          lm_bar_expect(&sh.full[s], tx_bytes);
           unsigned char* a = ring + (size_t)s * stage_bytes;
           lm_tma_load(a, &map_h, kb * LM_BK, rb * LM_RB, &sh.full[s]);
-          lm_tma_load(a + a_bytes, &map_w, kb * LM_BK, vt * LM_BN, &sh.full[s]);
+          lm_tma_load(a + a_bytes, &map_w, kb * LM_BK, vt * bn, &sh.full[s]);
         }
       }
       if (*fail)  // gave up: before the CTA leaves, wait (bounded) for the copies still landing in its ring
@@ -192,7 +194,7 @@ k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant_
             const uint32_t ah = a_addr + (uint32_t)(half * LM_BM * LM_BK * 2);
 #pragma unroll
             for (int kk = 0; kk < LM_BK / 16; ++kk)  // 16 bf16 = 32 bytes along K inside the swizzled row
-              tc_mma(d_tmem, tc_desc(ah + kk * 32), tc_desc(b_addr + kk * 32), kLmIdesc, (kb | kk) != 0 ? 1u : 0u);
+              tc_mma(d_tmem, tc_desc(ah + kk * 32), tc_desc(b_addr + kk * 32), idesc, (kb | kk) != 0 ? 1u : 0u);
           }
           if (!ok) break;
           tc_commit(&sh.empty[s]);  // the stage may be refilled once these MMAs have read it
@@ -220,7 +222,7 @@ k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant_
       use += 1u;
       const bool first = !((visited >> rb) & 1ull);
       visited |= 1ull << rb;
-      const int col_base = vt * LM_BN;
+      const int col_base = vt * bn;
       const int row = rb * LM_RB + half * LM_BM + r_in_tile;
       const bool valid = row < rows;
       const size_t slot = (size_t)cta * parts.rpad + row;
@@ -236,10 +238,11 @@ k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant_
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll 1
-      for (int c0 = 0; c0 < LM_BN; c0 += 32) {
+      for (int c0 = 0; c0 < bn; c0 += 32) {
         uint32_t r[32];
         tc_tmem_ld32(taddr + (uint32_t)c0, r);
-        const int ncol = V - (col_base + c0);     // columns of this chunk that exist (the last tile is ragged)
+        // columns of this chunk that belong to the item and exist (the last tile of the vocabulary is ragged)
+        const int ncol = min(V - (col_base + c0), bn - c0);
         if (ncol <= 0 || !valid) continue;        // (every lane still took part in the load above)
         if (ncol < 32) {
 #pragma unroll
@@ -440,6 +443,20 @@ cudaError_t launch_lm_head_topk(const void* hidden, const void* weight, int64_t 
   const int grid = device_info().sm_count;
   const size_t smem = (size_t)LM_RING_BYTES + sizeof(LmShared);
   const int a_rows = rows <= LM_BM ? LM_BM : LM_RB, n_stages = rows <= LM_BM ? 4 : 3;
+  // Width of a work item along the vocabulary: the widest tile is the most efficient one, but the items are dealt
+  // in whole rounds over the CTAs, and 594 tiles of 256 columns over 148 CTAs is four rounds and a fifth for two
+  // CTAs.  Take the width (a multiple of 16) with the shortest schedule: rounds x (width + the fixed cost of an
+  // item in columns' worth).  Measured at d = 4096: an item takes 10 us + 0.17 us per column when one block of
+  // rows streams the weights (bound by their bandwidth), and 27 us + 0.12 us per column with two accumulators.
+  const int n_rb = (int)((rows + LM_RB - 1) / LM_RB);
+  const int fixed_cols = rows <= LM_RB ? 60 : 224;
+  int bn = LM_BN;
+  long long best_cost = -1;
+  for (int w = LM_BN; w >= 128; w -= 16) {
+    const long long items = (long long)((V + w - 1) / w) * n_rb;
+    const long long cost = ((items + grid - 1) / grid) * (w + fixed_cols);
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; bn = w; }
+  }
   cudaError_t e = allow_max_dynamic_smem<k_lm_head_topk<4>>();
   if (e == cudaSuccess) e = allow_max_dynamic_smem<k_lm_head_topk<8>>();
   if (e == cudaSuccess) e = allow_max_dynamic_smem<k_lm_head_topk<16>>();
@@ -455,14 +472,14 @@ cudaError_t launch_lm_head_topk(const void* hidden, const void* weight, int64_t 
   e = cudaMemsetAsync(fail_flag, 0, 256, st);
   if (e != cudaSuccess) return e;
   CUtensorMap map_w, map_h;
-  if (!make_map(&map_w, weight, (uint64_t)d, (uint64_t)V, LM_BN)) return cudaErrorNotSupported;
+  if (!make_map(&map_w, weight, (uint64_t)d, (uint64_t)V, (uint32_t)bn)) return cudaErrorNotSupported;
   if (!make_map(&map_h, hidden, (uint64_t)d, (uint64_t)rows, (uint32_t)a_rows)) return cudaErrorNotSupported;
   if (k <= 4)
-    k_lm_head_topk<4><<<grid, LM_THREADS, smem, st>>>(map_h, map_w, (int)rows, d, V, k, a_rows, n_stages, parts, fail_flag);
+    k_lm_head_topk<4><<<grid, LM_THREADS, smem, st>>>(map_h, map_w, (int)rows, d, V, k, a_rows, n_stages, bn, parts, fail_flag);
   else if (k <= 8)
-    k_lm_head_topk<8><<<grid, LM_THREADS, smem, st>>>(map_h, map_w, (int)rows, d, V, k, a_rows, n_stages, parts, fail_flag);
+    k_lm_head_topk<8><<<grid, LM_THREADS, smem, st>>>(map_h, map_w, (int)rows, d, V, k, a_rows, n_stages, bn, parts, fail_flag);
   else
-    k_lm_head_topk<16><<<grid, LM_THREADS, smem, st>>>(map_h, map_w, (int)rows, d, V, k, a_rows, n_stages, parts, fail_flag);
+    k_lm_head_topk<16><<<grid, LM_THREADS, smem, st>>>(map_h, map_w, (int)rows, d, V, k, a_rows, n_stages, bn, parts, fail_flag);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   k_lm_head_merge<<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(parts, grid, (int)rows, k, cand_ids, cand_lp);
