@@ -56,7 +56,7 @@ struct TreeSmem {
   Span<short> x_aux;        // [xcap] per-round scratch
   Span<unsigned long long> x_key64;  // [xcap] ordering keys of the final choice
   Span<int> x_wsum;         // [32] warp totals of the block scans
-  Span<unsigned long long> dw_row;  // [warps, k rounded up to 4] ordering keys of the row a warp is ranking
+  Span<unsigned long long> dw_row;  // [warps, max(32, k rounded up to 4)] ordering keys of the rows a warp is ranking
   Span<uint32_t> dw_ckey;           // depth-by-depth expansion: score keys of a depth's candidates, packed
 };
 
@@ -115,7 +115,7 @@ inline TreeLayout tree_layout(int L, int k, int N, int W = 0) {
   o.x_bak = take(xcap); o.x_score = take(sizeof(float) * xcap); o.x_key = take(sizeof(uint32_t) * xcap);
   o.x_aux = take(sizeof(short) * xcap); o.x_wsum = take(sizeof(int) * 32);
   o.x_key64 = take(sizeof(unsigned long long) * xcap);
-  o.dw_row = take(sizeof(unsigned long long) * (G2_T / 32) * ((k + 3) & ~3));
+  o.dw_row = take(sizeof(unsigned long long) * (G2_T / 32) * (((k + 3) & ~3) < 32 ? 32 : ((k + 3) & ~3)));
   o.dw_ckey = take(sizeof(uint32_t) * kDepthwiseMaxW * kDepthwiseMaxW);
   o.total = (uint32_t)off;
   return o;
@@ -136,7 +136,7 @@ __device__ __forceinline__ void tree_bind(TreeSmem* s, unsigned char* base, cons
   s->x_aux = Span<short>((short*)(base + o.x_aux), xcap, 128);
   s->x_wsum = Span<int>((int*)(base + o.x_wsum), 32, 129);
   s->x_key64 = Span<unsigned long long>((unsigned long long*)(base + o.x_key64), xcap, 130);
-  s->dw_row = Span<unsigned long long>((unsigned long long*)(base + o.dw_row), (long long)(G2_T / 32) * ((k + 3) & ~3), 131);
+  s->dw_row = Span<unsigned long long>((unsigned long long*)(base + o.dw_row), (long long)(G2_T / 32) * (((k + 3) & ~3) < 32 ? 32 : ((k + 3) & ~3)), 131);
   s->dw_ckey = Span<uint32_t>((uint32_t*)(base + o.dw_ckey), kDepthwiseMaxW * kDepthwiseMaxW, 132);
   s->t = Span<float>((float*)(base + o.t), lkk, 101);
   s->ord = Span<unsigned char>(base + o.ord, lkk, 102);
@@ -1012,7 +1012,7 @@ __device__ __forceinline__ int expand_depthwise(TreeSmem& s, const RowSource& sr
 }
 
 // eq. 5 and eq. 9, then the sort by (t desc, token asc), one THREAD per (position, predecessor) row, for k <= KP
-// <= 16: the row lives in registers, nothing is exchanged between lanes and the k^2 comparisons are independent
+// <= 4: the row lives in registers, nothing is exchanged between lanes and the k^2 comparisons are independent
 // of one another.  Element e of the row is visited in an order that starts at tid % k, so that the lanes of a
 // warp spread over the shared-memory banks.  In place: a thread reads its whole row before it rewrites it.
 template <int KP>
@@ -1058,6 +1058,67 @@ __device__ __forceinline__ void prepare_rows_by_thread(TreeSmem& s, int k, int n
       int e = start + a;
       e = e >= k ? e - k : e;
       s.t[at + rank] = v[a];
+      s.ord[at + rank] = (unsigned char)e;
+    }
+  }
+}
+
+// The same for 8 <= KP <= 16 (KP a power of two, k <= KP): KP lanes per row, 32 / KP rows per warp at a time, one entry
+// per lane.  The log-sum-exp is a butterfly inside the lane group; the ranks come from counting the group's 32-bit
+// value keys out of the warp's scratch (KP / 4 vector loads per lane), with the same collision check and 64-bit
+// recount for equal values as rank_row_warp.  A thread that holds a whole row of 16 in registers spends a thousand
+// dependent instructions on it while most of the CTA's issue slots stay empty; here a row costs a few dozen.
+template <int KP>
+__device__ __forceinline__ void prepare_rows_by_group(TreeSmem& s, int k, int nrows, int tid) {
+  constexpr int RPW = 32 / KP;
+  const int lane = tid & 31, warp = tid >> 5, g = lane / KP, e = lane % KP;
+  unsigned long long* scratch64 = s.dw_row.ptr((long long)warp * 32, 32);
+  uint32_t* key32 = reinterpret_cast<uint32_t*>(scratch64);  // [32] value keys (0 = none), then [32] marks
+  for (int rbase = warp * RPW; rbase < nrows; rbase += (G2_T / 32) * RPW) {
+    const int r = rbase + g;
+    const bool on = r < nrows && e < k;
+    const int i = r == 0 ? 0 : 1 + (r - 1) / k;
+    const int ra = r == 0 ? 0 : (r - 1) % k;
+    const int at = (i * k + ra) * k;
+    float v = -INFINITY;
+    uint32_t ntok = 0u;
+    if (on) {
+      v = fmaf(s.al[i], s.lp[i * k + e], s.t[at + e]);
+      ntok = ~(uint32_t)s.tok[i * k + e];
+    }
+    float mx = v;
+#pragma unroll
+    for (int o = KP / 2; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, o));
+    float sum = on ? expf(v - mx) : 0.f;
+#pragma unroll
+    for (int o = KP / 2; o > 0; o >>= 1) sum += __shfl_xor_sync(FULL, sum, o);
+    v -= mx + logf(sum);
+    uint32_t kv = f2key(v);
+    kv = kv == 0u ? 1u : kv;
+    key32[lane] = on ? kv : 0u;
+    __syncwarp();
+    const uint4* grp = reinterpret_cast<const uint4*>(key32 + g * KP);
+    int c0 = 0, c1 = 0, c2 = 0, c3 = 0;
+#pragma unroll
+    for (int j = 0; j < KP / 4; ++j) {
+      const uint4 q = grp[j];
+      c0 += q.x > kv; c1 += q.y > kv; c2 += q.z > kv; c3 += q.w > kv;
+    }
+    int rank = (c0 + c1) + (c2 + c3);
+    if (on) key32[32 + g * KP + rank] = (uint32_t)e;
+    __syncwarp();
+    const bool clash = on && key32[32 + g * KP + rank] != (uint32_t)e;
+    if (__any_sync(FULL, clash)) {  // equal values in a row: rank again on (value key, ~token)
+      __syncwarp();
+      const unsigned long long k64 = ((unsigned long long)kv << 32) | ntok;
+      scratch64[lane] = on ? k64 : 0ull;
+      __syncwarp();
+      rank = 0;
+      for (int j = 0; j < k; ++j) rank += scratch64[g * KP + j] > k64;
+    }
+    __syncwarp();  // every lane has read its raw entry and the scratch: both may be rewritten
+    if (on) {
+      s.t[at + rank] = v;
       s.ord[at + rank] = (unsigned char)e;
     }
   }
@@ -1147,8 +1208,8 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
     if (kp == 1) prepare_rows_by_thread<1>(s, k, nrows, tid);
     else if (kp == 2) prepare_rows_by_thread<2>(s, k, nrows, tid);
     else if (kp == 4) prepare_rows_by_thread<4>(s, k, nrows, tid);
-    else if (kp == 8) prepare_rows_by_thread<8>(s, k, nrows, tid);
-    else prepare_rows_by_thread<16>(s, k, nrows, tid);
+    else if (kp == 8) prepare_rows_by_group<8>(s, k, nrows, tid);
+    else prepare_rows_by_group<16>(s, k, nrows, tid);
   } else {
     // 16 < k <= 64: one warp per (position, predecessor) row, two entries per lane; eq. 5, eq. 9, ranks by counting
     __syncthreads();  // s.lp, s.tok
