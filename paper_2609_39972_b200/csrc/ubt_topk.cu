@@ -590,6 +590,318 @@ k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanP
   }
 }
 
+// ------------------------------------------------------------------------------- deferred candidates
+// The streaming loop of this form touches no candidate at all.  Per chunk a thread keeps the maximum of its own
+// fragments (8 slots of shared memory per thread, a chunk uses slot chunk % 8, stored rounded up to bf16); per
+// segment it keeps the exact maximum of all its elements.  When the segment has streamed past:
+//   * the k-th largest of the 256 per-thread maxima is a lower bound of the k-th largest element (the maxima are
+//     256 distinct elements); it is bisected on the leading key bits with CTA-wide counts;
+//   * a thread whose slot maximum reaches the bound reads the fragments of that slot's chunks again -- from L2,
+//     where the segment still sits -- and appends the elements that reach the bound to the pool; on ordinary
+//     rows that is about k + k^2 / 512 elements in as many (thread, chunk) groups of 8 fragments;
+//   * the pool is ranked once.
+// A pool that overflows (a row with hundreds of elements equal to its maximum) is handled by walking the segment
+// again in column order in slices that cannot overflow, ranking after each slice that produced a hit.
+constexpr int G1D_SLOTS = 8;
+constexpr int G1D_POOL = 512;
+static_assert(G1D_POOL <= G1R_POOL, "the deferred form shares the pool and its ranking with the ring form");
+
+struct G1DShared : G1RShared {
+  // pool[] of the base is used up to G1D_POOL entries only; what follows overlays its upper half
+};
+constexpr size_t kG1DGmaxOffset = offsetof(G1RShared, pool) + sizeof(unsigned long long) * G1D_POOL;
+static_assert(sizeof(unsigned short) * G1D_SLOTS * G1R_T <= sizeof(unsigned long long) * (G1R_POOL - G1D_POOL),
+              "the slot maxima live in the unused upper half of the pool");
+
+__device__ __forceinline__ unsigned short bf16_bits_round_up(float x) {
+  const uint32_t u = __float_as_uint(x);
+  uint32_t h = u >> 16;
+  if (!(u >> 31) && (u & 0xffffu)) h += 1;  // positive: magnitude up; negative: truncation already rounds up
+  return (unsigned short)h;
+}
+
+template <int VEC>
+__device__ __forceinline__ void append_hits_d(G1RShared& sh, const float (&x)[VEC], float taux, int col0) {
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) {
+    if (x[j] > taux) {
+      const int at = atomicAdd(&sh.cnt, 1);
+      if (at < G1D_POOL) sh.pool[at] = make_key(x[j], col0 + j);
+    }
+  }
+}
+
+// flush_keyed for a pool of at most G1D_POOL entries
+__device__ void flush_keyed_d(G1RShared& sh, int k) {
+  const int tid = threadIdx.x;
+  const int M = sh.cnt < G1D_POOL ? sh.cnt : G1D_POOL, nt = sh.ntop, total = M + nt;
+  const int newn = total < k ? total : k;
+  for (int i = tid; i < total; i += G1R_T) {
+    const unsigned long long ki = i < M ? sh.pool[i] : sh.top[i - M];
+    int rank = 0;
+    for (int j = 0; j < M; ++j) rank += sh.pool[j] > ki;
+    for (int j = 0; j < nt; ++j) rank += sh.top[j] > ki;
+    if (rank < k) sh.topn[rank] = ki;
+  }
+  __syncthreads();
+  if (tid < newn) sh.top[tid] = sh.topn[tid];
+  if (tid == 0) {
+    sh.ntop = newn;
+    sh.cnt = 0;
+    if (newn == k) sh.taux = key_val(sh.topn[k - 1]);
+  }
+  __syncthreads();
+}
+
+template <typename T>
+__global__ void __launch_bounds__(G1R_T, G1R_CTAS)
+k_lse_topk_defer(const T* __restrict__ logits, int64_t total, int V, int k, SpanPlan plan,
+                 float* __restrict__ part_ms, float* __restrict__ part_val, int32_t* __restrict__ part_idx,
+                 int32_t* __restrict__ part_cnt) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  constexpr int VEC = 16 / (int)sizeof(T);
+  constexpr int STAGE_ELEMS = G1R_STAGE_BYTES / (int)sizeof(T);
+  constexpr int CHUNK_FRAGS = STAGE_ELEMS / VEC / G1R_T;  // fragments of a full chunk per thread
+  constexpr int RING_BYTES = G1R_STAGES * G1R_STAGE_BYTES;
+  constexpr int NW = G1R_T / 32;
+  constexpr int LOW_BIT = sizeof(T) == 2 ? 16 : 12;  // bf16 values have no key bits below 16
+  unsigned char* ring = smem_raw;
+  G1RShared& sh = *reinterpret_cast<G1RShared*>(smem_raw + RING_BYTES);
+  unsigned short* gmax = reinterpret_cast<unsigned short*>(smem_raw + RING_BYTES + kG1DGmaxOffset);  // [slot][thread]
+  __shared__ uint64_t full[G1R_STAGES];
+
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int64_t lo = (int64_t)blockIdx.x * plan.span;
+  const int64_t hi = lo + plan.span < total ? lo + plan.span : total;
+  pdl_wait();  // nothing is read or written before the kernel in front has completed
+  pdl_launch_dependents();
+  if (lo >= hi) return;
+  const long long nslots = (total / V) * plan.smax;
+  const Span<float> g_ms(part_ms, nslots * 2, 341), g_val(part_val, nslots * k, 342);
+  const Span<int32_t> g_idx(part_idx, nslots * k, 343), g_cnt(part_cnt, nslots, 344);
+
+  if (tid == 0) {
+    for (int s = 0; s < G1R_STAGES; ++s) mbar_init(&full[s], 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    sh.fail = 0;
+  }
+  __syncthreads();
+  RingProducer<T, G1R_STAGES, G1R_STAGE_BYTES> prod;
+  if (tid == 0) {
+    prod.init(lo, hi, V);
+    for (int i = 0; i < G1R_STAGES - 1; ++i) prod.issue_one(logits, ring, full);
+  }
+  RingPos<G1R_STAGES> rp;
+  rp.init();
+  int consumed = 0;
+  bool failed = false;
+  const unsigned long long l2e2 = pack2(kLog2e, kLog2e);
+
+  for (int64_t pos = lo; pos < hi && !failed;) {
+    Segment sg;
+    sg.at(pos, hi, V);
+    if (tid == 0) { sh.cnt = 0; sh.ntop = 0; sh.taux = -INFINITY; }
+    float ref = -1.0e30f, negref = 1.0e30f * kLog2e;  // ref = -1e30: not fixed yet
+    float segmax = -INFINITY;
+    unsigned long long acc[G1R_GROUP];  // packed pairs of partial sums (one FADD2 adds two exponentials)
+#pragma unroll
+    for (int u = 0; u < G1R_GROUP; ++u) acc[u] = 0ull;
+
+    int chunk = 0;
+    for (int c = 0; c < sg.len; c += STAGE_ELEMS, ++chunk) {
+      const int l = sg.len - c < STAGE_ELEMS ? sg.len - c : STAGE_ELEMS;
+      if (*reinterpret_cast<volatile int*>(&sh.fail)) { failed = true; break; }
+      if (tid == 0) prod.issue_one(logits, ring, full);
+      const bool ok = mbar_wait(&full[rp.stage], rp.parity);
+      if (!ok) sh.fail = 1;
+      const uint4* stage = reinterpret_cast<const uint4*>(ring + (size_t)rp.stage * G1R_STAGE_BYTES) + tid;
+      const int nfrag = ok ? l / VEC : 0;
+      float cmax = -INFINITY;
+      int f0 = 0;
+      for (; f0 + G1R_GROUP * G1R_T <= nfrag; f0 += G1R_GROUP * G1R_T) {  // full groups: no bounds checks
+        float x[G1R_GROUP][VEC];
+        float vmax[G1R_GROUP];
+#pragma unroll
+        for (int u = 0; u < G1R_GROUP; ++u) {
+          Frag<T> fr;
+          fr.unpack(stage[f0 + u * G1R_T]);
+          vmax[u] = fr.x[0];
+#pragma unroll
+          for (int j = 0; j < VEC; ++j) { x[u][j] = fr.x[j]; vmax[u] = fmaxf(vmax[u], fr.x[j]); }
+        }
+        const float gm = fmaxf(fmaxf(vmax[0], vmax[1]), fmaxf(vmax[2], vmax[3]));
+        cmax = fmaxf(cmax, gm);
+        if (gm > ref + 60.f) {  // rare: the first elements of a segment, or an element far above the reference
+          const float sc = ex2_approx(fmaf(ref, kLog2e, -gm * kLog2e));
+#pragma unroll
+          for (int u = 0; u < G1R_GROUP; ++u) acc[u] = fma2(acc[u], pack2(sc, sc), 0ull);
+          ref = gm;
+          negref = -gm * kLog2e;
+        }
+#pragma unroll
+        for (int u = 0; u < G1R_GROUP; ++u) {
+#pragma unroll
+          for (int j = 0; j < VEC; j += 2) {
+            float y0, y1;
+            unpack2(fma2(pack2(x[u][j], x[u][j + 1]), l2e2, pack2(negref, negref)), y0, y1);
+            acc[u] = add2(acc[u], pack2(ex2_approx(y0), ex2_approx(y1)));
+          }
+        }
+      }
+      for (; f0 + tid < nfrag; f0 += G1R_T) {  // ragged end of a chunk
+        Frag<T> fr;
+        fr.unpack(stage[f0]);
+        float vm = fr.x[0];
+#pragma unroll
+        for (int j = 1; j < VEC; ++j) vm = fmaxf(vm, fr.x[j]);
+        cmax = fmaxf(cmax, vm);
+        if (vm > ref + 60.f) {
+          const float sc = ex2_approx(fmaf(ref, kLog2e, -vm * kLog2e));
+#pragma unroll
+          for (int u = 0; u < G1R_GROUP; ++u) acc[u] = fma2(acc[u], pack2(sc, sc), 0ull);
+          ref = vm;
+          negref = -vm * kLog2e;
+        }
+#pragma unroll
+        for (int j = 0; j < VEC; j += 2) {
+          float y0, y1;
+          unpack2(fma2(pack2(fr.x[j], fr.x[j + 1]), l2e2, pack2(negref, negref)), y0, y1);
+          acc[0] = add2(acc[0], pack2(ex2_approx(y0), ex2_approx(y1)));
+        }
+      }
+      {
+        const int slot = chunk & (G1D_SLOTS - 1);
+        float m = cmax;
+        if (chunk >= G1D_SLOTS) m = fmaxf(m, __uint_as_float((uint32_t)gmax[slot * G1R_T + tid] << 16));
+        gmax[slot * G1R_T + tid] = bf16_bits_round_up(m);
+        segmax = fmaxf(segmax, cmax);
+      }
+      __syncthreads();  // the stage is free for the copy after next
+      rp.next();
+      ++consumed;
+    }
+    if (failed) break;
+
+    // ---- the candidates of the segment
+    const T* seg = logits + sg.row * (int64_t)V + sg.col0;
+    const uint32_t mykey = segmax > -INFINITY ? f2key(segmax) : 0u;
+    uint32_t lob = 0;
+    for (int bit = 31; bit >= LOW_BIT; --bit) {
+      const uint32_t cand = lob | (1u << bit);
+      if (__syncthreads_count(mykey >= cand) >= k) lob = cand;
+    }
+    float taux = -INFINITY;  // exclusive bound: an element is a candidate iff it is > taux
+    if (lob != 0u) {
+      uint32_t below = lob - 1;
+      if (below == 0x7fffffffu) below = 0x7ffffffeu;  // skip -0: it equals +0
+      const float t = key2f(below), t0 = key2f(lob);
+      if (t == t && t0 == t0) taux = t;
+    }
+    const int nchunks = chunk;
+    // Which of its (thread, chunk) groups can hold a candidate: a thread knows from its slot maxima.  The warp then
+    // reads the groups again together: up to four groups per round, eight lanes per group and one fragment per
+    // lane, so that the loads of a round -- typically all the warp has -- are in flight at the same time (the
+    // latency of a load is microseconds while every SM is streaming).
+    uint32_t qm = 0;
+#pragma unroll
+    for (int slot = 0; slot < G1D_SLOTS; ++slot)
+      if (slot < nchunks && __uint_as_float((uint32_t)gmax[slot * G1R_T + tid] << 16) > taux) qm |= 1u << slot;
+    static_assert(CHUNK_FRAGS == 8 && G1D_SLOTS == 8, "eight lanes read the eight fragments of a group");
+    for (int base = 0; base < nchunks; base += 32) {
+      uint32_t rem = qm | (qm << 8) | (qm << 16) | (qm << 24);  // bit i: chunk base + i (slot i % 8)
+      if (nchunks - base < 32) rem &= (1u << (nchunks - base)) - 1u;
+      for (;;) {
+        const uint32_t has = __ballot_sync(FULL, rem != 0u);
+        if (has == 0u) break;
+        const uint32_t src = __fns(has, 0, (lane >> 3) + 1);  // the lane whose group this lane helps to read
+        const int mine = rem ? __ffs(rem) - 1 : 0;
+        const int ch = base + __shfl_sync(FULL, mine, src & 31);
+        if (src < 32u) {
+          const int c = ch * STAGE_ELEMS;
+          const int nfrag = (sg.len - c < STAGE_ELEMS ? sg.len - c : STAGE_ELEMS) / VEC;
+          const int f = (lane & 7) * G1R_T + (tid & ~31) + (int)src;
+          if (f < nfrag) {
+            Frag<T> fr;
+            fr.unpack(__ldg(reinterpret_cast<const uint4*>(seg + c) + f));
+            append_hits_d<VEC>(sh, fr.x, taux, sg.col0 + c + f * VEC);
+          }
+        }
+        if (rem != 0u && __popc(has & ((1u << lane) - 1u)) < 4) rem &= rem - 1u;
+      }
+    }
+    __syncthreads();
+    if (sh.cnt > G1D_POOL) {
+      // more candidates than the pool holds: walk the segment in column order, a slice of G1D_POOL elements at a
+      // time; once k entries stand, only a strictly larger element can still enter (an equal one has the
+      // higher column)
+      __syncthreads();
+      if (tid == 0) { sh.cnt = 0; sh.ntop = 0; sh.taux = taux; }
+      __syncthreads();
+      constexpr int SLICE = G1D_POOL / VEC;  // fragments per slice
+      const int nfrag_seg = sg.len / VEC;
+      for (int g0 = 0; g0 < nfrag_seg; g0 += SLICE) {
+        const float tx = sh.taux;
+        const int f = g0 + tid;
+        if (tid < SLICE && f < nfrag_seg) {
+          Frag<T> fr;
+          fr.unpack(__ldg(reinterpret_cast<const uint4*>(seg) + f));
+          append_hits_d<VEC>(sh, fr.x, tx, sg.col0 + f * VEC);
+        }
+        if (__syncthreads_or(*reinterpret_cast<volatile int*>(&sh.cnt) > 0)) flush_keyed_d(sh, k);
+      }
+    } else {
+      flush_keyed_d(sh, k);
+    }
+
+    // partial (max, sum exp) of the segment from the per-thread (reference, sum) pairs
+    float s_t;
+    {
+      float a0, a1;
+      unpack2(add2(add2(acc[0], acc[1]), add2(acc[2], acc[3])), a0, a1);
+      s_t = a0 + a1;
+    }
+    float mw = ref;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mw = fmaxf(mw, __shfl_xor_sync(FULL, mw, o));
+    if (lane == 0) sh.redf[tid >> 5] = mw;
+    __syncthreads();
+    float M = sh.redf[0];
+    for (int w = 1; w < NW; ++w) M = fmaxf(M, sh.redf[w]);
+    float sw = s_t * ex2_approx((ref - M) * kLog2e);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sw += __shfl_xor_sync(FULL, sw, o);
+    if (lane == 0) sh.redf[NW + (tid >> 5)] = sw;
+    __syncthreads();
+    const int64_t c_first = (sg.row * (int64_t)V) / plan.span;
+    const int64_t slot = sg.row * plan.smax + ((int64_t)blockIdx.x - c_first);
+    if (tid == 0) {
+      float S = 0.f;
+      for (int w = 0; w < NW; ++w) S += sh.redf[NW + w];
+      g_ms[slot * 2] = M;
+      g_ms[slot * 2 + 1] = S;
+      g_cnt[slot] = sh.ntop;
+    }
+    if (tid < sh.ntop) {
+      g_val[slot * k + tid] = key_val(sh.top[tid]);
+      g_idx[slot * k + tid] = key_idx(sh.top[tid]);
+    }
+    __syncthreads();
+    pos += sg.len;
+  }
+  __syncthreads();
+  if (tid == 0 && *reinterpret_cast<volatile int*>(&sh.fail)) {
+    prod.drain(consumed > 0 ? consumed - 1 : 0, full);
+    // a wait gave up: mark every segment of this span (written or not) so that the merge reports it
+    for (int64_t pos = lo; pos < hi;) {
+      Segment sg;
+      sg.at(pos, hi, V);
+      const int64_t c_first = (sg.row * (int64_t)V) / plan.span;
+      g_cnt[sg.row * plan.smax + ((int64_t)blockIdx.x - c_first)] = -1;
+      pos += sg.len;
+    }
+  }
+}
+
 // One warp per row: combine the partials of the row's segments (see merge_row_warp in ubt_merge.cuh).
 __global__ void __launch_bounds__(128)
 k_merge_topk(MergeParts parts, int64_t rows, int V, int k, int32_t* __restrict__ cand_ids,
@@ -667,8 +979,13 @@ template <typename T>
 static cudaError_t launch_lse_topk_ring_t(const void* logits, int64_t rows, int V, int k, const TopkWorkspace& w,
                                           cudaStream_t st) {
   const size_t smem = (size_t)G1R_STAGES * G1R_STAGE_BYTES + sizeof(G1RShared);
+#ifdef UBT_TOPK_LOCKSTEP
   auto kern = k_lse_topk_ring<T>;
   cudaError_t e = allow_max_dynamic_smem<k_lse_topk_ring<T>>();
+#else
+  auto kern = k_lse_topk_defer<T>;
+  cudaError_t e = allow_max_dynamic_smem<k_lse_topk_defer<T>>();
+#endif
   if (e != cudaSuccess) return e;
   return launch_kernel(kern, dim3(w.plan.grid), dim3(G1R_T), smem, st, true, static_cast<const T*>(logits),
                        rows * (int64_t)V, V, k, w.plan, w.part_ms, w.part_val, w.part_idx, w.part_cnt);
