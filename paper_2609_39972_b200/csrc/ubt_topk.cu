@@ -6,12 +6,12 @@
 //
 // Streaming one segment (k_lse_topk_ring, rows made of whole 16-byte fragments): chunks of the span arrive in a
 // shared-memory ring through bulk asynchronous copies; every thread sums 2^((x - ref) log2 e) relative to a
-// reference of its own that moves up when an element exceeds it by 60, and a group of four fragments per lane is
-// tested against a CTA-wide exclusive threshold by one warp vote; elements above it are appended as 64-bit
-// (value, ~column) keys to a shared pool.  The threshold starts at the k-th largest per-thread maximum of the
-// first chunk (bisection with CTA-wide counts) and becomes exact whenever the pool holds k entries and is
-// ranked ("flush").  k_lse_topk is the plain-load form for other vocabularies (online max per thread, columns
-// in the pool, the next tile prefetched into registers).
+// reference of its own and keeps the maximum of its fragments per chunk.  The candidates are found when the
+// segment has streamed past: the k-th largest per-thread maximum bounds the k-th largest element from below, the
+// few (thread, chunk) groups whose maximum reaches the bound are read again from L2, and their elements above
+// the bound are ranked once as 64-bit (value, ~column) keys.  k_lse_topk is the plain-load form for other
+// vocabularies (online max per thread, columns in a pool that is ranked whenever it fills, the next tile
+// prefetched into registers).
 #include "ubt_internal.h"
 #include "ubt_merge.cuh"
 #include "ubt_ring.cuh"
@@ -267,31 +267,80 @@ k_lse_topk(const T* __restrict__ logits, int64_t total, int V, int k, SpanPlan p
 }
 
 // ------------------------------------------------------------------------------- ring-fed version
-// Same algorithm with the logits arriving through the bulk-copy ring (ubt_ring.cuh), three CTAs per SM so
-// that one CTA's barriers (threshold bisection, pool ranking) overlap the others' streaming.
+// The logits arrive through the bulk-copy ring (ubt_ring.cuh), three CTAs per SM.
 //
-// Log-sum-exp without a running maximum in the common path: every thread fixes a reference ref >= tau0 (the
-// bisected bound, which the exclusive threshold taux never falls below) and accumulates 2^((x-ref)*log2 e).
-// An element <= taux cannot overflow that; an element > taux takes the rare hit path anyway, where the
-// thread moves its reference up if the element is more than 60 above it.
+// Log-sum-exp without a running maximum in the common path: every thread sums 2^((x - ref) log2 e) relative to a
+// reference of its own, the largest element of the first group it sees; an element more than 60 above the
+// reference (rare) moves the reference up and rescales the sum.
 //
-// Hits go to a small pool of (value, column) keys, so ranking the pool touches shared memory only.  A chunk
-// that overflows the pool (possible only for pathological rows, e.g. long runs of equal values before the
-// threshold turns strict) has its hits discarded and is walked again in slices that cannot overflow.
+// Top-k with deferred candidates: the streaming loop touches no candidate at all.  Per chunk a thread keeps the
+// maximum of its own fragments (8 slots of shared memory per thread, a chunk uses slot chunk % 8, stored rounded
+// up to bf16); per segment it keeps the exact maximum of all its elements so far.
+//   * The k-th largest of the 256 per-thread maxima is a lower bound of the k-th largest element (the maxima are
+//     256 distinct elements), and it only grows as more of the segment is seen.  It is bisected on the leading
+//     key bits with CTA-wide counts BEFORE the segment's last chunk is processed.
+//   * A thread whose slot maximum reaches the bound holds a possible candidate in that (thread, chunk) group of 8
+//     fragments; on ordinary rows about k + k^2 / 512 groups qualify.  The threads list their groups, and the CTA
+//     copies the listed groups again from global memory (L2) into a side buffer with asynchronous 16-byte
+//     copies, 32 groups per round, one fragment per thread; the copies of the last round stay in flight while
+//     the last chunk streams through the arithmetic (a load takes microseconds while every SM is streaming).
+//   * After the last chunk every thread whose maximum of that chunk reaches the bound scans its fragments of it
+//     once more in the stage, the side buffer is scanned, and the pool of (value, ~column) keys is ranked once.
+// A pool that overflows (a row with hundreds of elements equal to its maximum) is handled by walking the segment
+// again in column order, ranking after each step that produced a hit.
 constexpr int G1R_T = 256, G1R_STAGES = 2, G1R_STAGE_BYTES = 32768, G1R_CTAS = 3;
-constexpr int G1R_POOL = 1024;  // hit pool entries
-constexpr int G1R_GROUP = 4;    // fragments per vote
+constexpr int G1R_GROUP = 4;                                     // fragments per thread and loop iteration
+constexpr int G1R_CHUNK_FRAGS = G1R_STAGE_BYTES / 16 / G1R_T;    // fragments of a full chunk per thread
+constexpr int G1R_SLOTS = 8;                                     // chunk maxima a thread keeps
+constexpr int G1R_POOL = 192;                                    // candidate pool entries
+constexpr int G1R_ROUND = G1R_T / G1R_CHUNK_FRAGS;               // groups the CTA copies per round
+constexpr int G1R_ITEMS = 128;  // groups a segment may list; more send it down the slow path
 
-struct G1RShared {
-  int cnt;     // pool entries (may exceed G1R_POOL while a chunk overflows)
+struct alignas(16) G1RShared {
+  int cnt;     // pool entries (may exceed G1R_POOL: the surplus is dropped and the segment walked again)
   int ntop;    // entries of top[]
-  float taux;  // exclusive threshold: x enters the pool iff x > taux
+  float taux;  // slow path: exclusive threshold, x enters the pool iff x > taux
   int fail;    // a bounded wait gave up
+  int nlist;   // entries of list[] (may exceed G1R_ITEMS)
+  int pad[3];
   float redf[2 * (G1R_T / 32)];
   unsigned long long top[kMaxK];
   unsigned long long topn[kMaxK];
   unsigned long long pool[G1R_POOL];
+  unsigned short gmax[G1R_SLOTS * G1R_T];  // [slot][thread] chunk maxima, bf16 bits rounded up
+  uint4 side[G1R_T];                        // fragments read again, one per thread
+  unsigned short list[G1R_ITEMS];           // thread << 8 | chunk of the groups to read again
 };
+static_assert(offsetof(G1RShared, side) % 16 == 0, "the side buffer receives 16-byte copies");
+// three CTAs per SM: ring + this struct + the static barriers + 1 KiB the system reserves, times three, in 228 KiB
+static_assert(3 * (G1R_STAGES * G1R_STAGE_BYTES + sizeof(G1RShared) + 128 + 1024) <= 233472, "three CTAs per SM");
+
+__device__ __forceinline__ unsigned short bf16_bits_round_up(float x) {
+  const uint32_t u = __float_as_uint(x);
+  uint32_t h = u >> 16;
+  if (!(u >> 31) && (u & 0xffffu)) h += 1;  // positive: magnitude up; negative: truncation already rounds up
+  return (unsigned short)h;
+}
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
+               : "memory");
+}
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// Returns the number of elements appended (or dropped because the pool was full).
+template <int VEC>
+__device__ __forceinline__ int append_hits(G1RShared& sh, const float (&x)[VEC], float taux, int col0) {
+  int hits = 0;
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) {
+    if (x[j] > taux) {
+      const int at = atomicAdd(&sh.cnt, 1);
+      if (at < G1R_POOL) sh.pool[at] = make_key(x[j], col0 + j);
+      ++hits;
+    }
+  }
+  return hits;
+}
 
 // Rank pool + carried list exactly (keys are unique); afterwards top[0..ntop) is sorted best first, the
 // pool is empty and, when k entries exist, taux is the k-th best value (strict from then on).
@@ -316,361 +365,27 @@ __device__ void flush_keyed(G1RShared& sh, int k) {
   __syncthreads();
 }
 
-// Append the elements of one fragment that beat the threshold.  Hits are rare, so each hit lane reserves its
-// own pool entry; the other lanes fall through.
-template <int VEC>
-__device__ __forceinline__ void append_hits(G1RShared& sh, const float (&x)[VEC], float taux, int col0) {
-#pragma unroll
-  for (int j = 0; j < VEC; ++j) {
-    if (x[j] > taux) {
-      const int at = atomicAdd(&sh.cnt, 1);
-      if (at < G1R_POOL) sh.pool[at] = make_key(x[j], col0 + j);
-    }
-  }
-}
-
 template <typename T>
 __global__ void __launch_bounds__(G1R_T, G1R_CTAS)
 k_lse_topk_ring(const T* __restrict__ logits, int64_t total, int V, int k, SpanPlan plan,
-                float* __restrict__ part_ms, float* __restrict__ part_val, int32_t* __restrict__ part_idx,
-                int32_t* __restrict__ part_cnt) {
-  extern __shared__ __align__(128) unsigned char smem_raw[];
-  constexpr int VEC = 16 / (int)sizeof(T);
-  constexpr int STAGE_ELEMS = G1R_STAGE_BYTES / (int)sizeof(T);
-  constexpr int RING_BYTES = G1R_STAGES * G1R_STAGE_BYTES;
-  constexpr int NW = G1R_T / 32;
-  unsigned char* ring = smem_raw;
-  G1RShared& sh = *reinterpret_cast<G1RShared*>(smem_raw + RING_BYTES);
-  __shared__ uint64_t full[G1R_STAGES];
-
-  const int tid = threadIdx.x, lane = tid & 31;
-  const int64_t lo = (int64_t)blockIdx.x * plan.span;
-  const int64_t hi = lo + plan.span < total ? lo + plan.span : total;
-  // Launched programmatically: the CTAs may become resident while the kernel in front is still running.  Nothing
-  // is read or written before that kernel has completed; only then may the tree kernel behind this one be
-  // scheduled (it waits for this grid before it reads the partials).
-  pdl_wait();
-  pdl_launch_dependents();
-  if (lo >= hi) return;
-  const long long nslots = (total / V) * plan.smax;
-  const Span<float> g_ms(part_ms, nslots * 2, 341), g_val(part_val, nslots * k, 342);
-  const Span<int32_t> g_idx(part_idx, nslots * k, 343), g_cnt(part_cnt, nslots, 344);
-
-  if (tid == 0) {
-    for (int s = 0; s < G1R_STAGES; ++s) mbar_init(&full[s], 1);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    sh.fail = 0;
-  }
-  __syncthreads();
-  RingProducer<T, G1R_STAGES, G1R_STAGE_BYTES> prod;
-  if (tid == 0) {
-    prod.init(lo, hi, V);
-    for (int i = 0; i < G1R_STAGES - 1; ++i) prod.issue_one(logits, ring, full);
-  }
-  RingPos<G1R_STAGES> rp;
-  rp.init();
-  int consumed = 0;
-  bool failed = false;
-
-  for (int64_t pos = lo; pos < hi && !failed;) {
-    Segment sg;
-    sg.at(pos, hi, V);
-    if (tid == 0) { sh.cnt = 0; sh.ntop = 0; sh.taux = -INFINITY; }
-    float ref = -1.0e30f, negref = 1.0e30f * kLog2e;  // ref = -1e30: not fixed yet
-    unsigned long long acc[G1R_GROUP];  // packed pairs of partial sums (one FADD2 adds two exponentials)
-#pragma unroll
-    for (int u = 0; u < G1R_GROUP; ++u) acc[u] = 0ull;
-    const unsigned long long l2e2 = pack2(kLog2e, kLog2e);
-
-    for (int c = 0; c < sg.len; c += STAGE_ELEMS) {
-      const int l = sg.len - c < STAGE_ELEMS ? sg.len - c : STAGE_ELEMS;
-      if (*reinterpret_cast<volatile int*>(&sh.fail)) { failed = true; break; }
-      if (tid == 0) prod.issue_one(logits, ring, full);
-      const bool ok = mbar_wait(&full[rp.stage], rp.parity);
-      if (!ok) sh.fail = 1;
-      const uint4* stage = reinterpret_cast<const uint4*>(ring + (size_t)rp.stage * G1R_STAGE_BYTES) + tid;
-      const int nfrag = ok ? l / VEC : 0;
-      const int colbase = sg.col0 + c + tid * VEC;
-
-      if (c == 0) {
-        // Bound for the k-th largest element: bisect the top 16 key bits of the per-thread maxima of the
-        // first chunk with CTA-wide counts; the result never exceeds the k-th largest maximum.
-        float tmax = -INFINITY;
-        bool has = false;
-        for (int f0 = 0; f0 + tid < nfrag; f0 += G1R_T) {
-          Frag<T> x;
-          x.unpack(stage[f0]);
-#pragma unroll
-          for (int j = 0; j < VEC; ++j) tmax = fmaxf(tmax, x.x[j]);
-          has = true;
-        }
-        const uint32_t mykey = has ? f2key(tmax) : 0u;
-        uint32_t lob = 0;
-        for (int bit = 31; bit >= 16; --bit) {
-          const uint32_t cand = lob | (1u << bit);
-          if (__syncthreads_count(mykey >= cand) >= k) lob = cand;
-        }
-        float tau0 = -INFINITY;
-        if (lob != 0u) {
-          uint32_t below = lob - 1;
-          if (below == 0x7fffffffu) below = 0x7ffffffeu;  // skip -0: it equals +0
-          const float t = key2f(below), t0 = key2f(lob);
-          if (t == t && t0 == t0) {
-            tau0 = t0;
-            if (tid == 0) sh.taux = t;
-          }
-        }
-        const float r0 = fmaxf(tau0, has ? tmax : -INFINITY);
-        if (r0 > -1.0e29f && r0 < 1.0e30f) { ref = r0; negref = -r0 * kLog2e; }
-        __syncthreads();
-      }
-      const float taux = sh.taux;
-      int f0 = 0;
-      for (; f0 + G1R_GROUP * G1R_T <= nfrag; f0 += G1R_GROUP * G1R_T) {  // full groups: no bounds checks
-        float x[G1R_GROUP][VEC];
-        float vmax[G1R_GROUP];
-#pragma unroll
-        for (int u = 0; u < G1R_GROUP; ++u) {
-          Frag<T> fr;
-          fr.unpack(stage[f0 + u * G1R_T]);
-          vmax[u] = fr.x[0];
-#pragma unroll
-          for (int j = 0; j < VEC; ++j) { x[u][j] = fr.x[j]; vmax[u] = fmaxf(vmax[u], fr.x[j]); }
-        }
-        const float gmax = fmaxf(fmaxf(vmax[0], vmax[1]), fmaxf(vmax[2], vmax[3]));
-        // rare: a candidate somewhere in the warp's 4 fragments, or an element far above a lane's reference (the
-        // bound rises with what OTHER warps have seen, so a non-candidate can still overflow 2^((x - ref) log2 e))
-        if (__any_sync(FULL, gmax > fminf(taux, ref + 60.f))) {
-          if (gmax > ref + 60.f || (ref < -1.0e29f && gmax > -INFINITY)) {  // move the reference up
-            const float sc = ex2_approx(fmaf(ref, kLog2e, -gmax * kLog2e));
-#pragma unroll
-            for (int u = 0; u < G1R_GROUP; ++u) acc[u] = fma2(acc[u], pack2(sc, sc), 0ull);
-            ref = gmax;
-            negref = -gmax * kLog2e;
-          }
-#pragma unroll
-          for (int u = 0; u < G1R_GROUP; ++u)
-            if (vmax[u] > taux) append_hits<VEC>(sh, x[u], taux, colbase + (f0 + u * G1R_T) * VEC);
-        }
-#pragma unroll
-        for (int u = 0; u < G1R_GROUP; ++u) {
-#pragma unroll
-          for (int j = 0; j < VEC; j += 2) {
-            float y0, y1;
-            unpack2(fma2(pack2(x[u][j], x[u][j + 1]), l2e2, pack2(negref, negref)), y0, y1);
-            acc[u] = add2(acc[u], pack2(ex2_approx(y0), ex2_approx(y1)));
-          }
-        }
-      }
-      for (; f0 < nfrag; f0 += G1R_T) {  // ragged end of a chunk, one fragment per vote
-        float x[VEC];
-        if (f0 + tid < nfrag) {
-          Frag<T> fr;
-          fr.unpack(stage[f0]);
-#pragma unroll
-          for (int j = 0; j < VEC; ++j) x[j] = fr.x[j];
-        } else {
-#pragma unroll
-          for (int j = 0; j < VEC; ++j) x[j] = -INFINITY;
-        }
-        float vm = x[0];
-#pragma unroll
-        for (int j = 1; j < VEC; ++j) vm = fmaxf(vm, x[j]);
-        if (__any_sync(FULL, vm > fminf(taux, ref + 60.f))) {
-          if (vm > ref + 60.f || (ref < -1.0e29f && vm > -INFINITY)) {
-            const float sc = ex2_approx(fmaf(ref, kLog2e, -vm * kLog2e));
-#pragma unroll
-            for (int u = 0; u < G1R_GROUP; ++u) acc[u] = fma2(acc[u], pack2(sc, sc), 0ull);
-            ref = vm;
-            negref = -vm * kLog2e;
-          }
-          if (vm > taux) append_hits<VEC>(sh, x, taux, colbase + f0 * VEC);
-        }
-#pragma unroll
-        for (int j = 0; j < VEC; j += 2) {
-          float y0, y1;
-          unpack2(fma2(pack2(x[j], x[j + 1]), l2e2, pack2(negref, negref)), y0, y1);
-          acc[0] = add2(acc[0], pack2(ex2_approx(y0), ex2_approx(y1)));
-        }
-      }
-      // One barrier takes the decision on the final hit count (see the comment in k_lse_topk): rank the pool
-      // now?  Inside the branch nobody is ahead in the next chunk, so the counter can be read plainly.
-      if (__syncthreads_or(*reinterpret_cast<volatile int*>(&sh.cnt) >= k)) {
-        const bool overflow = sh.cnt > G1R_POOL;
-        flush_keyed(sh, k);  // ranks what the pool holds; tightens the threshold
-        if (overflow) {
-          // The chunk produced more hits than the pool holds and the surplus was dropped.  Walk the chunk
-          // again in slices of 64 fragments, ranking after each slice so that the pool cannot overflow; a
-          // hit that already sits in the carried list (it was ranked above) is not added twice.  The walk
-          // admits elements EQUAL to the current k-th value too: a dropped one may have the lower column.
-          const uint4* st0 = stage - tid;
-          for (int g0 = 0; g0 < nfrag; g0 += 64) {
-            const float tx = next_below(sh.taux);
-            if (tid < 64) {  // two whole warps
-              float x[VEC];
-              const int f = g0 + tid;
-              if (f < nfrag) {
-                Frag<T> fr;
-                fr.unpack(st0[f]);
-#pragma unroll
-                for (int j = 0; j < VEC; ++j) x[j] = fr.x[j];
-              } else {
-#pragma unroll
-                for (int j = 0; j < VEC; ++j) x[j] = -INFINITY;
-              }
-              const int col0 = sg.col0 + c + f * VEC;
-              const int nt = sh.ntop;
-#pragma unroll
-              for (int j = 0; j < VEC; ++j) {
-                if (x[j] > tx) {
-                  const unsigned long long key = make_key(x[j], col0 + j);
-                  for (int q = 0; q < nt; ++q)
-                    if (sh.top[q] == key) x[j] = -INFINITY;  // already ranked
-                }
-              }
-              append_hits<VEC>(sh, x, tx, col0);
-            }
-            __syncthreads();
-            flush_keyed(sh, k);
-          }
-        }
-      }
-      rp.next();
-      ++consumed;
-    }
-    if (failed) break;
-    flush_keyed(sh, k);
-
-    // partial (max, sum exp) of the segment from the per-thread (reference, sum) pairs
-    float s_t;
-    {
-      float a0, a1;
-      unpack2(add2(add2(acc[0], acc[1]), add2(acc[2], acc[3])), a0, a1);
-      s_t = a0 + a1;
-    }
-    float mw = ref;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) mw = fmaxf(mw, __shfl_xor_sync(FULL, mw, o));
-    if (lane == 0) sh.redf[tid >> 5] = mw;
-    __syncthreads();
-    float M = sh.redf[0];
-    for (int w = 1; w < NW; ++w) M = fmaxf(M, sh.redf[w]);
-    float sw = s_t * ex2_approx((ref - M) * kLog2e);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) sw += __shfl_xor_sync(FULL, sw, o);
-    if (lane == 0) sh.redf[NW + (tid >> 5)] = sw;
-    __syncthreads();
-    const int64_t c_first = (sg.row * (int64_t)V) / plan.span;
-    const int64_t slot = sg.row * plan.smax + ((int64_t)blockIdx.x - c_first);
-    if (tid == 0) {
-      float S = 0.f;
-      for (int w = 0; w < NW; ++w) S += sh.redf[NW + w];
-      g_ms[slot * 2] = M;
-      g_ms[slot * 2 + 1] = S;
-      g_cnt[slot] = sh.ntop;
-    }
-    if (tid < sh.ntop) {
-      g_val[slot * k + tid] = key_val(sh.top[tid]);
-      g_idx[slot * k + tid] = key_idx(sh.top[tid]);
-    }
-    __syncthreads();
-    pos += sg.len;
-  }
-  __syncthreads();
-  if (tid == 0 && *reinterpret_cast<volatile int*>(&sh.fail)) {
-    prod.drain(consumed > 0 ? consumed - 1 : 0, full);
-    // a wait gave up: mark every segment of this span (written or not) so that the merge reports it
-    for (int64_t pos = lo; pos < hi;) {
-      Segment sg;
-      sg.at(pos, hi, V);
-      const int64_t c_first = (sg.row * (int64_t)V) / plan.span;
-      g_cnt[sg.row * plan.smax + ((int64_t)blockIdx.x - c_first)] = -1;
-      pos += sg.len;
-    }
-  }
-}
-
-// ------------------------------------------------------------------------------- deferred candidates
-// The streaming loop of this form touches no candidate at all.  Per chunk a thread keeps the maximum of its own
-// fragments (8 slots of shared memory per thread, a chunk uses slot chunk % 8, stored rounded up to bf16); per
-// segment it keeps the exact maximum of all its elements.  When the segment has streamed past:
-//   * the k-th largest of the 256 per-thread maxima is a lower bound of the k-th largest element (the maxima are
-//     256 distinct elements); it is bisected on the leading key bits with CTA-wide counts;
-//   * a thread whose slot maximum reaches the bound reads the fragments of that slot's chunks again -- from L2,
-//     where the segment still sits -- and appends the elements that reach the bound to the pool; on ordinary
-//     rows that is about k + k^2 / 512 elements in as many (thread, chunk) groups of 8 fragments;
-//   * the pool is ranked once.
-// A pool that overflows (a row with hundreds of elements equal to its maximum) is handled by walking the segment
-// again in column order in slices that cannot overflow, ranking after each slice that produced a hit.
-constexpr int G1D_SLOTS = 8;
-constexpr int G1D_POOL = 512;
-static_assert(G1D_POOL <= G1R_POOL, "the deferred form shares the pool and its ranking with the ring form");
-
-struct G1DShared : G1RShared {
-  // pool[] of the base is used up to G1D_POOL entries only; what follows overlays its upper half
-};
-constexpr size_t kG1DGmaxOffset = offsetof(G1RShared, pool) + sizeof(unsigned long long) * G1D_POOL;
-static_assert(sizeof(unsigned short) * G1D_SLOTS * G1R_T <= sizeof(unsigned long long) * (G1R_POOL - G1D_POOL),
-              "the slot maxima live in the unused upper half of the pool");
-
-__device__ __forceinline__ unsigned short bf16_bits_round_up(float x) {
-  const uint32_t u = __float_as_uint(x);
-  uint32_t h = u >> 16;
-  if (!(u >> 31) && (u & 0xffffu)) h += 1;  // positive: magnitude up; negative: truncation already rounds up
-  return (unsigned short)h;
-}
-
-template <int VEC>
-__device__ __forceinline__ void append_hits_d(G1RShared& sh, const float (&x)[VEC], float taux, int col0) {
-#pragma unroll
-  for (int j = 0; j < VEC; ++j) {
-    if (x[j] > taux) {
-      const int at = atomicAdd(&sh.cnt, 1);
-      if (at < G1D_POOL) sh.pool[at] = make_key(x[j], col0 + j);
-    }
-  }
-}
-
-// flush_keyed for a pool of at most G1D_POOL entries
-__device__ void flush_keyed_d(G1RShared& sh, int k) {
-  const int tid = threadIdx.x;
-  const int M = sh.cnt < G1D_POOL ? sh.cnt : G1D_POOL, nt = sh.ntop, total = M + nt;
-  const int newn = total < k ? total : k;
-  for (int i = tid; i < total; i += G1R_T) {
-    const unsigned long long ki = i < M ? sh.pool[i] : sh.top[i - M];
-    int rank = 0;
-    for (int j = 0; j < M; ++j) rank += sh.pool[j] > ki;
-    for (int j = 0; j < nt; ++j) rank += sh.top[j] > ki;
-    if (rank < k) sh.topn[rank] = ki;
-  }
-  __syncthreads();
-  if (tid < newn) sh.top[tid] = sh.topn[tid];
-  if (tid == 0) {
-    sh.ntop = newn;
-    sh.cnt = 0;
-    if (newn == k) sh.taux = key_val(sh.topn[k - 1]);
-  }
-  __syncthreads();
-}
-
-template <typename T>
-__global__ void __launch_bounds__(G1R_T, G1R_CTAS)
-k_lse_topk_defer(const T* __restrict__ logits, int64_t total, int V, int k, SpanPlan plan,
                  float* __restrict__ part_ms, float* __restrict__ part_val, int32_t* __restrict__ part_idx,
                  int32_t* __restrict__ part_cnt) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   constexpr int VEC = 16 / (int)sizeof(T);
   constexpr int STAGE_ELEMS = G1R_STAGE_BYTES / (int)sizeof(T);
-  constexpr int CHUNK_FRAGS = STAGE_ELEMS / VEC / G1R_T;  // fragments of a full chunk per thread
+  constexpr int CHUNK_FRAGS = G1R_CHUNK_FRAGS;
   constexpr int RING_BYTES = G1R_STAGES * G1R_STAGE_BYTES;
   constexpr int NW = G1R_T / 32;
   constexpr int LOW_BIT = sizeof(T) == 2 ? 16 : 12;  // bf16 values have no key bits below 16
   unsigned char* ring = smem_raw;
   G1RShared& sh = *reinterpret_cast<G1RShared*>(smem_raw + RING_BYTES);
-  unsigned short* gmax = reinterpret_cast<unsigned short*>(smem_raw + RING_BYTES + kG1DGmaxOffset);  // [slot][thread]
+  unsigned short* gmax = sh.gmax;
   __shared__ uint64_t full[G1R_STAGES];
 
   const int tid = threadIdx.x, lane = tid & 31;
+  uint4* side = sh.side + tid;
+  unsigned short* list = sh.list;
+  int* nlist = &sh.nlist;
   const int64_t lo = (int64_t)blockIdx.x * plan.span;
   const int64_t hi = lo + plan.span < total ? lo + plan.span : total;
   pdl_wait();  // nothing is read or written before the kernel in front has completed
@@ -695,23 +410,81 @@ k_lse_topk_defer(const T* __restrict__ logits, int64_t total, int V, int k, Span
   rp.init();
   int consumed = 0;
   bool failed = false;
+  bool ahead = false;  // the copy that the next chunk would issue is already on its way
   const unsigned long long l2e2 = pack2(kLog2e, kLog2e);
 
   for (int64_t pos = lo; pos < hi && !failed;) {
     Segment sg;
     sg.at(pos, hi, V);
-    if (tid == 0) { sh.cnt = 0; sh.ntop = 0; sh.taux = -INFINITY; }
+    const T* seg = logits + sg.row * (int64_t)V + sg.col0;
+    if (tid == 0) { sh.cnt = 0; sh.ntop = 0; sh.taux = -INFINITY; *nlist = 0; }
     float ref = -1.0e30f, negref = 1.0e30f * kLog2e;  // ref = -1e30: not fixed yet
     float segmax = -INFINITY;
+    float taux = -INFINITY;  // exclusive bound: an element is a candidate iff it is > taux
+    int side_col = -1;       // column of the fragment this lane has in flight to the side buffer
     unsigned long long acc[G1R_GROUP];  // packed pairs of partial sums (one FADD2 adds two exponentials)
 #pragma unroll
     for (int u = 0; u < G1R_GROUP; ++u) acc[u] = 0ull;
 
+    // the bound from the per-thread maxima seen so far
+    auto bisect = [&]() {
+      const uint32_t mykey = segmax > -INFINITY ? f2key(segmax) : 0u;
+      uint32_t lob = 0;
+      for (int bit = 31; bit >= LOW_BIT; --bit) {
+        const uint32_t cand = lob | (1u << bit);
+        if (__syncthreads_count(mykey >= cand) >= k) lob = cand;
+      }
+      if (lob != 0u) {
+        uint32_t below = lob - 1;
+        if (below == 0x7fffffffu) below = 0x7ffffffeu;  // skip -0: it equals +0
+        const float t = key2f(below), t0 = key2f(lob);
+        if (t == t && t0 == t0) taux = t;
+      }
+    };
+    // what this thread copied to the side buffer
+    auto scan_side = [&]() {
+      cp_async_wait();
+      if (side_col >= 0) {
+        Frag<T> fr;
+        fr.unpack(*side);
+        append_hits<VEC>(sh, fr.x, taux, side_col);
+      }
+      side_col = -1;
+    };
+
     int chunk = 0;
     for (int c = 0; c < sg.len; c += STAGE_ELEMS, ++chunk) {
       const int l = sg.len - c < STAGE_ELEMS ? sg.len - c : STAGE_ELEMS;
+      const bool last = c + STAGE_ELEMS >= sg.len;
       if (*reinterpret_cast<volatile int*>(&sh.fail)) { failed = true; break; }
-      if (tid == 0) prod.issue_one(logits, ring, full);
+      if (tid == 0 && !ahead) prod.issue_one(logits, ring, full);
+      ahead = false;
+      if (last && chunk > 0) {
+        // the chunks before the last: bound, then the groups that may hold a candidate, read again
+        bisect();
+#pragma unroll
+        for (int slot = 0; slot < G1R_SLOTS; ++slot) {
+          if (slot < chunk && __uint_as_float((uint32_t)gmax[slot * G1R_T + tid] << 16) > taux) {
+            for (int ch = slot; ch < chunk; ch += G1R_SLOTS) {
+              const int at = atomicAdd(nlist, 1);
+              if (at < G1R_ITEMS && ch < 256) list[at] = (unsigned short)((tid << 8) | ch);
+              else atomicAdd(&sh.cnt, G1R_POOL + 1);  // the list is full: this segment takes the slow path
+            }
+          }
+        }
+        __syncthreads();
+        const int n_items = *nlist < G1R_ITEMS ? *nlist : G1R_ITEMS;
+        for (int i0 = 0; i0 < n_items; i0 += G1R_ROUND) {
+          const int it = i0 + tid / CHUNK_FRAGS;
+          if (it < n_items) {
+            const int owner = list[it] >> 8, cc = (list[it] & 255) * STAGE_ELEMS;
+            const int f = (tid % CHUNK_FRAGS) * G1R_T + owner;  // a chunk before the last is full
+            cp_async_16(side, reinterpret_cast<const uint4*>(seg + cc) + f);
+            side_col = sg.col0 + cc + f * VEC;
+          }
+          if (i0 + G1R_ROUND < n_items) scan_side();  // more rounds follow: take this one in first
+        }
+      }
       const bool ok = mbar_wait(&full[rp.stage], rp.parity);
       if (!ok) sh.fail = 1;
       const uint4* stage = reinterpret_cast<const uint4*>(ring + (size_t)rp.stage * G1R_STAGE_BYTES) + tid;
@@ -769,88 +542,68 @@ k_lse_topk_defer(const T* __restrict__ logits, int64_t total, int V, int k, Span
           acc[0] = add2(acc[0], pack2(ex2_approx(y0), ex2_approx(y1)));
         }
       }
-      {
-        const int slot = chunk & (G1D_SLOTS - 1);
+      segmax = fmaxf(segmax, cmax);
+      if (!last) {
+        const int slot = chunk & (G1R_SLOTS - 1);
         float m = cmax;
-        if (chunk >= G1D_SLOTS) m = fmaxf(m, __uint_as_float((uint32_t)gmax[slot * G1R_T + tid] << 16));
+        if (chunk >= G1R_SLOTS) m = fmaxf(m, __uint_as_float((uint32_t)gmax[slot * G1R_T + tid] << 16));
         gmax[slot * G1R_T + tid] = bf16_bits_round_up(m);
-        segmax = fmaxf(segmax, cmax);
+      } else {
+        // the last chunk is still in its stage: a thread whose maximum of it reaches the bound scans its fragments
+        // once more (a segment of one chunk gets its bound only now)
+        if (chunk == 0) bisect();
+        if (cmax > taux) {
+          for (int f = 0; f + tid < nfrag; f += G1R_T) {
+            Frag<T> fr;
+            fr.unpack(stage[f]);
+            append_hits<VEC>(sh, fr.x, taux, sg.col0 + c + (f + tid) * VEC);
+          }
+        }
+        scan_side();
       }
-      __syncthreads();  // the stage is free for the copy after next
+      __syncthreads();  // the stage is free for the copy after next; after the last chunk: the pool is complete
       rp.next();
       ++consumed;
     }
     if (failed) break;
+    // the stage of the last chunk is free: keep the ring full while the candidates are ranked
+    if (tid == 0) prod.issue_one(logits, ring, full);
+    ahead = true;
 
-    // ---- the candidates of the segment
-    const T* seg = logits + sg.row * (int64_t)V + sg.col0;
-    const uint32_t mykey = segmax > -INFINITY ? f2key(segmax) : 0u;
-    uint32_t lob = 0;
-    for (int bit = 31; bit >= LOW_BIT; --bit) {
-      const uint32_t cand = lob | (1u << bit);
-      if (__syncthreads_count(mykey >= cand) >= k) lob = cand;
-    }
-    float taux = -INFINITY;  // exclusive bound: an element is a candidate iff it is > taux
-    if (lob != 0u) {
-      uint32_t below = lob - 1;
-      if (below == 0x7fffffffu) below = 0x7ffffffeu;  // skip -0: it equals +0
-      const float t = key2f(below), t0 = key2f(lob);
-      if (t == t && t0 == t0) taux = t;
-    }
-    const int nchunks = chunk;
-    // Which of its (thread, chunk) groups can hold a candidate: a thread knows from its slot maxima.  The warp then
-    // reads the groups again together: up to four groups per round, eight lanes per group and one fragment per
-    // lane, so that the loads of a round -- typically all the warp has -- are in flight at the same time (the
-    // latency of a load is microseconds while every SM is streaming).
-    uint32_t qm = 0;
-#pragma unroll
-    for (int slot = 0; slot < G1D_SLOTS; ++slot)
-      if (slot < nchunks && __uint_as_float((uint32_t)gmax[slot * G1R_T + tid] << 16) > taux) qm |= 1u << slot;
-    static_assert(CHUNK_FRAGS == 8 && G1D_SLOTS == 8, "eight lanes read the eight fragments of a group");
-    for (int base = 0; base < nchunks; base += 32) {
-      uint32_t rem = qm | (qm << 8) | (qm << 16) | (qm << 24);  // bit i: chunk base + i (slot i % 8)
-      if (nchunks - base < 32) rem &= (1u << (nchunks - base)) - 1u;
-      for (;;) {
-        const uint32_t has = __ballot_sync(FULL, rem != 0u);
-        if (has == 0u) break;
-        const uint32_t src = __fns(has, 0, (lane >> 3) + 1);  // the lane whose group this lane helps to read
-        const int mine = rem ? __ffs(rem) - 1 : 0;
-        const int ch = base + __shfl_sync(FULL, mine, src & 31);
-        if (src < 32u) {
-          const int c = ch * STAGE_ELEMS;
-          const int nfrag = (sg.len - c < STAGE_ELEMS ? sg.len - c : STAGE_ELEMS) / VEC;
-          const int f = (lane & 7) * G1R_T + (tid & ~31) + (int)src;
-          if (f < nfrag) {
-            Frag<T> fr;
-            fr.unpack(__ldg(reinterpret_cast<const uint4*>(seg + c) + f));
-            append_hits_d<VEC>(sh, fr.x, taux, sg.col0 + c + f * VEC);
-          }
-        }
-        if (rem != 0u && __popc(has & ((1u << lane) - 1u)) < 4) rem &= rem - 1u;
-      }
-    }
-    __syncthreads();
-    if (sh.cnt > G1D_POOL) {
-      // more candidates than the pool holds: walk the segment in column order, a slice of G1D_POOL elements at a
-      // time; once k entries stand, only a strictly larger element can still enter (an equal one has the
-      // higher column)
+    if (sh.cnt > G1R_POOL) {
+      // more candidates than the pool holds: walk the segment in column order, 256 fragments at a time; once k
+      // entries stand, only a strictly larger element can still enter (an equal one has the higher column)
       __syncthreads();
       if (tid == 0) { sh.cnt = 0; sh.ntop = 0; sh.taux = taux; }
       __syncthreads();
-      constexpr int SLICE = G1D_POOL / VEC;  // fragments per slice
+      constexpr int SLICE = G1R_POOL / VEC;  // fragments whose elements fit the pool in any case
       const int nfrag_seg = sg.len / VEC;
-      for (int g0 = 0; g0 < nfrag_seg; g0 += SLICE) {
+      for (int g0 = 0; g0 < nfrag_seg; g0 += G1R_T) {
         const float tx = sh.taux;
         const int f = g0 + tid;
-        if (tid < SLICE && f < nfrag_seg) {
-          Frag<T> fr;
+        Frag<T> fr;
+        int hits = 0;
+        if (f < nfrag_seg) {
           fr.unpack(__ldg(reinterpret_cast<const uint4*>(seg) + f));
-          append_hits_d<VEC>(sh, fr.x, tx, sg.col0 + f * VEC);
+          hits = append_hits<VEC>(sh, fr.x, tx, sg.col0 + f * VEC);
         }
-        if (__syncthreads_or(*reinterpret_cast<volatile int*>(&sh.cnt) > 0)) flush_keyed_d(sh, k);
+        if (!__syncthreads_or(hits > 0)) continue;
+        if (sh.cnt <= G1R_POOL) {
+          flush_keyed(sh, k);
+          continue;
+        }
+        __syncthreads();  // too many for one ranking: the same fragments again, a pool's worth at a time
+        if (tid == 0) sh.cnt = 0;
+        __syncthreads();
+        for (int s0 = 0; s0 < G1R_T; s0 += SLICE) {
+          const float tx2 = sh.taux;
+          int h2 = 0;
+          if (f < nfrag_seg && tid >= s0 && tid < s0 + SLICE) h2 = append_hits<VEC>(sh, fr.x, tx2, sg.col0 + f * VEC);
+          if (__syncthreads_or(h2 > 0)) flush_keyed(sh, k);
+        }
       }
     } else {
-      flush_keyed_d(sh, k);
+      flush_keyed(sh, k);
     }
 
     // partial (max, sum exp) of the segment from the per-thread (reference, sum) pairs
@@ -888,6 +641,7 @@ k_lse_topk_defer(const T* __restrict__ logits, int64_t total, int V, int k, Span
     __syncthreads();
     pos += sg.len;
   }
+  cp_async_wait();
   __syncthreads();
   if (tid == 0 && *reinterpret_cast<volatile int*>(&sh.fail)) {
     prod.drain(consumed > 0 ? consumed - 1 : 0, full);
@@ -979,13 +733,8 @@ template <typename T>
 static cudaError_t launch_lse_topk_ring_t(const void* logits, int64_t rows, int V, int k, const TopkWorkspace& w,
                                           cudaStream_t st) {
   const size_t smem = (size_t)G1R_STAGES * G1R_STAGE_BYTES + sizeof(G1RShared);
-#ifdef UBT_TOPK_LOCKSTEP
   auto kern = k_lse_topk_ring<T>;
   cudaError_t e = allow_max_dynamic_smem<k_lse_topk_ring<T>>();
-#else
-  auto kern = k_lse_topk_defer<T>;
-  cudaError_t e = allow_max_dynamic_smem<k_lse_topk_defer<T>>();
-#endif
   if (e != cudaSuccess) return e;
   return launch_kernel(kern, dim3(w.plan.grid), dim3(G1R_T), smem, st, true, static_cast<const T*>(logits),
                        rows * (int64_t)V, V, k, w.plan, w.part_ms, w.part_val, w.part_idx, w.part_cnt);

@@ -237,6 +237,37 @@ def test_rows_whose_level_jumps_inside_one_warps_share():
     np.testing.assert_allclose(clp.cpu().numpy(), lp, rtol=1e-5, atol=1e-5)
 
 
+@pytest.mark.parametrize("rows,V,k,dtype,kind", [
+    (8, 98304, 64, "bf16", "levels"),      # every (thread, chunk) group holds the maximum: the group list overflows
+    (3, 98304, 16, "bf16", "plateau"),     # 300 elements equal to the maximum: the candidate pool overflows
+    (4, 300000, 16, "f32", "normal"),      # 37 chunks per row: the eight maxima slots of a thread wrap four times
+    (2, 2200000, 8, "f32", "normal"),      # more than 256 chunks per row: beyond what a list entry can name
+    (40, 30000, 64, "bf16", "normal"),     # k = 64: several groups per warp, short segments at the span borders
+    (5, 16392, 16, "bf16", "normal"),      # a second chunk of one fragment
+])
+def test_topk_rows_that_leave_the_streaming_kernels_common_path(rows, V, k, dtype, kind):
+    u = ubt()
+    rng = np.random.default_rng(rows * 7 + k)
+    if kind == "levels":
+        x = rng.integers(0, 4, (rows, V)).astype(np.float32)
+    elif kind == "plateau":
+        x = rng.standard_normal((rows, V)).astype(np.float32)
+        for r in range(rows):
+            x[r, rng.choice(V, 300, replace=False)] = 9.0
+    else:
+        x = (rng.standard_normal((rows, V)) * 2.5).astype(np.float32)
+    host = synth.f32_to_bf16_bits(x) if dtype == "bf16" else x
+    ids, lp, _ = oracle.topk_logprob(host, k)
+    d = synth.to_device(host, dtype, DEV)
+    cid = torch.empty((rows, k), dtype=torch.int32, device=DEV)
+    clp = torch.empty((rows, k), dtype=torch.float32, device=DEV)
+    ws = u.workspace(u.ubt_draft_workspace_bytes(rows, 1, V, k, 1), DEV)
+    u.ubt_topk_logprob(d, k, cid, clp, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(cid.cpu().numpy(), ids)
+    np.testing.assert_allclose(clp.cpu().numpy(), lp, rtol=1e-5, atol=2e-5)
+
+
 def test_exact_score_ties_follow_total_order():
     # integer-valued inputs with lambda = 0: many node scores are exactly equal in fp32 and in double
     u = ubt()
