@@ -313,7 +313,7 @@ struct alignas(16) G1RShared {
 };
 static_assert(offsetof(G1RShared, side) % 16 == 0, "the side buffer receives 16-byte copies");
 // three CTAs per SM: ring + this struct + the static barriers + 1 KiB the system reserves, times three, in 228 KiB
-static_assert(3 * (G1R_STAGES * G1R_STAGE_BYTES + sizeof(G1RShared) + 128 + 1024) <= 233472, "three CTAs per SM");
+static_assert(G1R_CTAS * (G1R_STAGES * G1R_STAGE_BYTES + sizeof(G1RShared) + 128 + 1024) <= 233472, "three CTAs per SM");
 
 __device__ __forceinline__ unsigned short bf16_bits_round_up(float x) {
   const uint32_t u = __float_as_uint(x);
