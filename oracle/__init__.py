@@ -52,6 +52,7 @@ def lib() -> C.CDLL:
         _lib.ubt_oracle_walks_from_cdf.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p,
                                                    C.c_uint32, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p]
         _lib.ubt_oracle_weight_consts.argtypes = [C.c_float, C.c_float, C.c_void_p, C.c_void_p]
+        _lib.ubt_oracle_walk_picks.argtypes = [C.c_void_p] * 3 + [C.c_int] * 3 + [C.c_void_p] * 5
         _lib.ubt_oracle_lm_head_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int, C.c_int, C.c_int,
                                                  C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         _lib.ubt_oracle_selector_scores.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int64, C.c_int, C.c_void_p,
@@ -219,6 +220,24 @@ def verify(token_ids, parents, n_nodes, L: int, target_logits, mode: str = "gree
                                  _p(out.bonus_token), _p(out.node_pick))
     if rc:
         raise ValueError("oracle verify rejected its arguments")
+    return out
+
+
+def verify_picks(token_ids, parents, n_nodes, L: int, picks) -> Verdict:
+    """The walk of step 4 alone on given per-slot picks ``picks[B,N]`` (Appendix A, verification)."""
+    token_ids = np.ascontiguousarray(token_ids, np.int32)
+    parents = np.ascontiguousarray(parents, np.int32)
+    n_nodes = np.ascontiguousarray(n_nodes, np.int32)
+    picks = np.ascontiguousarray(picks, np.int32)
+    B, N = token_ids.shape
+    assert picks.shape == (B, N)
+    out = Verdict(np.empty(B, np.int32), np.empty((B, L + 1), np.int32), np.empty((B, L + 1), np.int32),
+                  np.empty(B, np.int32), picks)
+    rc = lib().ubt_oracle_walk_picks(_p(token_ids), _p(parents), _p(n_nodes), B, N, L, _p(picks),
+                                     _p(out.accepted_len), _p(out.accepted_nodes), _p(out.out_tokens),
+                                     _p(out.bonus_token))
+    if rc:
+        raise ValueError("oracle walk rejected its arguments")
     return out
 
 

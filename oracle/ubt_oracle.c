@@ -598,6 +598,37 @@ int ubt_oracle_verify(const int32_t *token_ids, const int32_t *parents, const in
 }
 
 /*
+ * The walk alone, for picks that come from elsewhere (Appendix A, verification: "the walk stops at the first pick
+ * that no child carries and keeps that pick as the bonus token").  picks[B,N] holds the target's token at every
+ * slot; only the slots the walk visits are read.  Outputs as ubt_oracle_verify.
+ */
+int ubt_oracle_walk_picks(const int32_t *token_ids, const int32_t *parents, const int32_t *n_nodes,
+                          int B, int N, int L, const int32_t *picks, int32_t *accepted_len,
+                          int32_t *accepted_nodes, int32_t *out_tokens, int32_t *bonus_token) {
+  if (B < 0 || N < 1 || L < 1) return 1;
+  for (int b = 0; b < B; ++b) {
+    const int32_t *tok = token_ids + (int64_t)b * N, *par = parents + (int64_t)b * N;
+    int32_t *an = accepted_nodes + (int64_t)b * (L + 1), *ot = out_tokens + (int64_t)b * (L + 1);
+    for (int j = 0; j <= L; ++j) an[j] = ot[j] = -1;
+    int cur = 0, acc = 0;
+    an[0] = 0;
+    for (;;) {
+      const int32_t x = picks[(int64_t)b * N + cur];
+      ot[acc] = x;
+      int child = -1;
+      for (int c = 1; c < n_nodes[b]; ++c)
+        if (par[c] == cur && tok[c] == x) { child = c; break; }
+      if (child < 0) { bonus_token[b] = x; break; }
+      ++acc;
+      an[acc] = child;
+      cur = child;
+    }
+    accepted_len[b] = acc;
+  }
+  return 0;
+}
+
+/*
  * Many sampling walks over one sequence's tree from precomputed row CDFs
  * (cdf[n] = inclusive prefix sums of row n, as ubt_oracle_row_cdf writes them).
  * Same definition as above with the prefix sums looked up instead of summed

@@ -345,6 +345,39 @@ def test_greedy_pick_is_library_argmax_and_planted_path_is_found():
         assert lazy.out_tokens.tolist() == v.out_tokens.tolist()
 
 
+def test_walk_on_given_picks_hand_worked_and_consistent_with_verify():
+    # (a) the hand-worked fixture
+    par = np.array([[-1, 0, 0, 1, 1, 3]], np.int32)
+    tok = np.array([[-1, 5, 7, 9, 2, 4]], np.int32)
+    nn = np.array([6], np.int32)
+    with open(os.path.join(GOLDEN, "walk_worked_example.txt")) as f:
+        rows = [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 6
+    for r in rows:
+        picks = np.array([[int(x) for x in r[:6]]], np.int32)
+        want_len, want_slots, want_tok = int(r[6]), [int(x) for x in r[7].split(",")], [int(x) for x in r[8].split(",")]
+        v = oracle.verify_picks(tok, par, nn, 3, picks)
+        assert v.accepted_len[0] == want_len
+        assert v.accepted_nodes[0].tolist() == want_slots + [-1] * (4 - len(want_slots))
+        assert v.out_tokens[0].tolist() == want_tok + [-1] * (4 - len(want_tok))
+        assert v.bonus_token[0] == want_tok[-1]
+    # a slot beyond n_nodes never matches, whatever it holds
+    v = oracle.verify_picks(tok, par, np.array([3], np.int32), 3, np.array([[5, 9, 0, 4, 0, 8]], np.int32))
+    assert v.accepted_len[0] == 1 and v.bonus_token[0] == 9
+    # (b) on drafted trees: the walk on the picks of the full verification is that verification
+    cfg = synth.CONFIGS["c1"]
+    for seed in range(4):
+        di = synth.draft_inputs(cfg, seed)
+        tr = oracle.draft_tree(di.unigram_logits, di.bigram_scores, cfg.k, cfg.N)
+        z = synth.target_logits(cfg, seed)
+        synth.plant_path(z, cfg.dtype, tr.token_ids, tr.parents, tr.n_nodes, seed)
+        for mode in ("greedy", "sample"):
+            full = oracle.verify(tr.token_ids, tr.parents, tr.n_nodes, cfg.L, z, mode, seed=seed)
+            w = oracle.verify_picks(tr.token_ids, tr.parents, tr.n_nodes, cfg.L, full.node_pick)
+            for name in ("accepted_len", "accepted_nodes", "out_tokens", "bonus_token"):
+                assert getattr(w, name).tolist() == getattr(full, name).tolist()
+
+
 def test_weight_routine_against_double_exp():
     rng = np.random.default_rng(2)
     for T in (1.0, 0.7, 2.5):
