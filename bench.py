@@ -103,6 +103,49 @@ def measure_lm_head(ubt, dev, rows=512, d=4096, V=151936, k=8, reps=10):
             "launches_per_call": 2, "timeouts": ubt.ubt_debug_ring_timeouts()}
 
 
+def measure_lm_head_verify(ubt, dev, d=4096, reps=5):
+    """Greedy verification straight from the target's hidden states of the tree slots (c3's trees: 32 x 64 slots):
+    the LM head fused with the row arg max (ubt_lm_head_topk, k = 1), then the walk on the picks
+    (ubt_verify_tree_picks); next to it the unfused route, a library bf16 product that stores the [B, N, V] target
+    logits followed by ubt_verify_tree."""
+    cfg = synth.CONFIGS["c3"]
+    ud, bd, _ = synth.device_inputs(cfg, 1, dev, want_target=False)
+    tree = ubt.ubt_draft_tree(ud, bd, cfg.k, cfg.N)
+    rows = cfg.B * cfg.N
+    hd, wd = synth.device_lm_head_inputs(rows, d, cfg.V, seed=6, device=dev)
+    hidden = hd.view(cfg.B, cfg.N, d)
+    logits = torch.empty((cfg.B, cfg.N, cfg.V), dtype=torch.bfloat16, device=dev)
+    res = ubt.VerifyResult.empty(cfg.B, cfg.L, dev)
+    ws_v = ubt.workspace(ubt.ubt_verify_workspace_bytes(cfg.B, cfg.N, cfg.V, "greedy"), dev)
+
+    def timed(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+
+    def unfused():
+        torch.matmul(hd, wd.T, out=logits.view(rows, cfg.V))
+        ubt.ubt_verify_tree(tree, logits, "greedy", result=res, ws=ws_v)
+
+    t_f = timed(lambda: ubt.verify_tree_from_hidden(tree, hidden, wd, result=res))
+    t_u = timed(unfused)
+    flops = 2.0 * rows * d * cfg.V
+    peak, kind = measured_tensor_peak()
+    return {"kernels": "k_lm_head_topk + k_lm_head_merge + k_walk", "bound": "tensor", "workload": "c3 trees",
+            "rows": rows, "d": d, "V": cfg.V, "dtype": "bf16", "avg_ms": t_f,
+            "achieved": flops / (t_f * 1e-3) / 1e12, "unit": "TFLOP/s", "peak": peak, "peak_source": f"of {kind}",
+            "frac": flops / (t_f * 1e-3) / 1e12 / peak, "unfused_ms": t_u,
+            "unfused": "library bf16 product storing the target logits + ubt_verify_tree",
+            "logits_bytes_not_written": rows * cfg.V * 2, "timeouts": ubt.ubt_debug_ring_timeouts()}
+
+
 def recorded_traffic(kernel: str, workload: str):
     """DRAM bytes per launch of `kernel` from the committed ncu summary, if one exists (else None)."""
     path = os.path.join(ROOT, "profiles", "dram_traffic.json")
@@ -519,7 +562,8 @@ def main():
     stream = torch.cuda.current_stream()
     if args.lm_head_only:
         if rank == 0:
-            print(json.dumps({"next_rows": {"lm_head_topk": measure_lm_head(ubt, dev, reps=max(1, args.steps))}}), flush=True)
+            print(json.dumps({"next_rows": {"lm_head_topk": measure_lm_head(ubt, dev, reps=max(1, args.steps)),
+                                            "lm_head_verify": measure_lm_head_verify(ubt, dev)}}), flush=True)
         return
 
     # the other workloads first, so that the headline's buffers are the ones kept for the end-to-end legs
@@ -569,7 +613,8 @@ def main():
 
     # ---- a row beyond the timed path: the LM head fused with step a1, timed alone (default run only)
     if rank == 0 and not args.no_lm_head and args.workload is None and args.batch == 0:
-        line["next_rows"] = {"lm_head_topk": measure_lm_head(ubt, dev)}
+        line["next_rows"] = {"lm_head_topk": measure_lm_head(ubt, dev),
+                             "lm_head_verify": measure_lm_head_verify(ubt, dev)}
         torch.cuda.empty_cache()
 
     # ---- end to end through the host-buffer entry points (pinned host inputs, results read back)

@@ -280,6 +280,20 @@ int ubt_verify_tree_keys(const ubt_tree *tree, const unsigned long long *gathere
                          ubt_verify_result *out, const ubt_verify_opts *opts, void *cuda_stream);
 
 /*
+ * The walk of step a4 alone (Appendix A, "Verification via Tree-attention"), for callers that already hold the
+ * target's pick of every slot.  node_pick[B, node_budget] (DEVICE, int32, read only) is the token the target
+ * chose at each slot: from ubt_lm_head_topk with k = 1 on the target's hidden states of the tree slots (greedy
+ * verification with the target logits never written to memory: cand_ids[B * node_budget, 1] IS this array), from
+ * a sampler of the caller's, or gathered from other ranks.  From the root the walk follows the child whose token
+ * equals the pick of the current slot until none matches; that pick is the bonus token.  *out is written as
+ * ubt_verify_tree writes it.  Every entry must be a token id >= 0 or negative for "no valid pick": a sequence
+ * with a negative entry at any of its node_budget slots gets UBT_STATUS_NONFINITE in status[b] (DEVICE, B words,
+ * may be NULL), and the entry counts as token 0.  No workspace.  Stream-ordered like every other call.
+ */
+int ubt_verify_tree_picks(const ubt_tree *tree, const int32_t *node_pick, ubt_verify_result *out,
+                          int32_t *status, void *cuda_stream);
+
+/*
  * Host-buffer forms.  Every pointer inside `tree`, `opts` (alpha ... pos_offset, node_pick) and
  * `out`, and the logits / bigram arguments, are HOST pointers (pinned memory makes the copies
  * asynchronous).  `device_buffer` is caller-owned DEVICE memory of at least

@@ -58,7 +58,7 @@ EXPORTS = ["ubt_version", "ubt_status_string", "ubt_debug_ring_timeouts", "ubt_d
            "ubt_draft_host_buffer_bytes", "ubt_verify_host_buffer_bytes", "ubt_draft_tree_host",
            "ubt_verify_tree_host", "ubt_verify_tree_static", "ubt_verify_static_capacity", "ubt_lm_head_workspace_bytes",
            "ubt_lm_head_topk", "ubt_topk_shard_bytes", "ubt_topk_shard", "ubt_topk_merge_shards", "ubt_verify_keys_shard",
-           "ubt_verify_tree_keys"]
+           "ubt_verify_tree_keys", "ubt_verify_tree_picks"]
 
 _lib = None
 
@@ -112,6 +112,7 @@ def load() -> C.CDLL:
     L.ubt_verify_keys_shard.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
                                         C.c_size_t, C.c_void_p]
     L.ubt_verify_tree_keys.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.ubt_verify_tree_picks.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
     L.ubt_debug_ring_timeouts.restype = C.c_longlong
     L.ubt_draft_tree_host.argtypes = L.ubt_draft_tree.argtypes
     L.ubt_verify_tree_host.argtypes = L.ubt_verify_tree.argtypes
@@ -438,6 +439,31 @@ def ubt_verify_tree_keys(tree: Tree, gathered_keys: torch.Tensor, shards: int,
                                        _stream(stream)), "ubt_verify_tree_keys")
     result.node_pick = node_pick
     return result
+
+
+def ubt_verify_tree_picks(tree: Tree, node_pick: torch.Tensor, result: Optional[VerifyResult] = None,
+                          status: Optional[torch.Tensor] = None, stream=None) -> VerifyResult:
+    """The walk alone on given per-slot picks ``node_pick`` (``int32[B, N]``, or ``[B * N, 1]`` as
+    ``ubt_lm_head_topk`` with ``k = 1`` returns them)."""
+    _need(node_pick, "node_pick")
+    if node_pick.dtype != torch.int32 or node_pick.numel() != tree.B * tree.N or not node_pick.is_contiguous():
+        raise ValueError("node_pick must be a contiguous int32 tensor of B * N entries")
+    if result is None:
+        result = VerifyResult.empty(tree.B, tree.L, node_pick.device)
+    t = tree.c_struct()
+    r = result.c_struct()
+    _check(load().ubt_verify_tree_picks(C.byref(t), _ptr(node_pick), C.byref(r), _ptr(status), _stream(stream)),
+           "ubt_verify_tree_picks")
+    result.node_pick = node_pick.view(tree.B, tree.N)
+    return result
+
+
+def verify_tree_from_hidden(tree: Tree, target_hidden: torch.Tensor, weight: torch.Tensor, **kw) -> VerifyResult:
+    """Greedy verification from the target's hidden states of the tree slots (``bf16[B, N, d]``) and its LM head
+    (``bf16[V, d]``): the head fused with the row arg max (``ubt_lm_head_topk``, k = 1), then the walk; the
+    ``[B, N, V]`` target logits are never written to memory."""
+    picks, _ = ubt_lm_head_topk(target_hidden.reshape(tree.B * tree.N, -1), weight, 1)
+    return ubt_verify_tree_picks(tree, picks, **kw)
 
 
 def verify_tree_vocab_parallel(tree: Tree, target_shard: torch.Tensor, v0: int, group=None, **kw) -> VerifyResult:

@@ -369,6 +369,22 @@ int ubt_verify_tree(const ubt_tree* tree, const void* target_logits, int dtype, 
   return UBT_OK;
 }
 
+int ubt_verify_tree_picks(const ubt_tree* tree, const int32_t* node_pick, ubt_verify_result* out, int32_t* status,
+                          void* cuda_stream) {
+  if (!tree || !out || !node_pick) return UBT_ERR_INVALID_ARG;
+  if (!tree->token_ids || !tree->parents || !tree->n_nodes) return UBT_ERR_INVALID_ARG;
+  if (!out->accepted_len || !out->bonus_token || !out->accepted_nodes || !out->out_tokens) return UBT_ERR_INVALID_ARG;
+  const int B = tree->B, N = tree->N, L = tree->L;
+  if (B < 0 || N < 1 || L < 1) return UBT_ERR_INVALID_ARG;
+  if (N > kMaxN || L > kMaxL) return UBT_ERR_UNSUPPORTED;
+  if (B == 0) return UBT_OK;
+  // the walk kernel in the mode that takes the picks as given (the sampling mode's second half)
+  if (launch_walk(*tree, UBT_VERIFY_SAMPLE, VerifyWorkspace{}, 0, node_pick, nullptr, *out, status,
+                  static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    return UBT_ERR_CUDA;
+  return UBT_OK;
+}
+
 }  // extern "C"
 
 // ------------------------------------------------------------------------- host-buffer forms
