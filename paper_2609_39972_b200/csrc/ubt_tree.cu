@@ -692,7 +692,9 @@ __device__ __forceinline__ int expand_rounds_warp(TreeSmem& s, int L, int k, int
 constexpr int EX_T = 128;
 __device__ __forceinline__ void ex_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(EX_T) : "memory"); }
 
-__device__ __forceinline__ int expand_rounds_cta(TreeSmem& s, int L, int k, int budget, float zeta, int& n_sure) {
+__device__ __forceinline__ void prepare_rows(TreeSmem& s, int k, int row0, int nrows, int tid, int nthreads);
+__device__ __forceinline__ int expand_rounds_cta(TreeSmem& s, int L, int k, int budget, float zeta, int& n_sure,
+                                                 int& d_ready) {
   const int tid = threadIdx.x, lane = tid & 31;
   const int cap = s.xcap;
   if (tid == 0) {
@@ -791,6 +793,10 @@ __device__ __forceinline__ int expand_rounds_cta(TreeSmem& s, int L, int k, int 
           s.x_next[idx] = 0;
         }
         s.x_next[par] = (unsigned char)(j0 + c);
+        if (d + 1 >= d_ready && d_ready < L) {  // the children just appended open rows that are not prepared yet
+          atomicOr(&s.scalars[3], 8);
+          break;
+        }
         sc = sc + s.t[base + j0] + zeta; r = s.ord[base + j0];
         par = at; d += 1; j0 = 0;
       }
@@ -805,7 +811,13 @@ __device__ __forceinline__ int expand_rounds_cta(TreeSmem& s, int L, int k, int 
       ex_barrier();  // the appended nodes and the counter are final for this wave
       const int n_now = s.scalars[1];
       overflow = (s.scalars[3] & 2) != 0;
+      const bool deeper = (s.scalars[3] & 8) != 0;
       ex_barrier();  // ... and every thread has read them before the next wave moves them on
+      if (deeper && d_ready < L) {  // a node beyond the prepared positions: prepare the rest of the table now
+        prepare_rows(s, k, 1 + (d_ready - 1) * k, 1 + (L - 1) * k, tid, EX_T);
+        d_ready = L;
+        ex_barrier();
+      }
       if (overflow || n_now == hi) { n = n_now; break; }
       lo = hi; hi = n_now; first = false;
       n = n_now;
@@ -1016,9 +1028,9 @@ __device__ __forceinline__ int expand_depthwise(TreeSmem& s, const RowSource& sr
 // of one another.  Element e of the row is visited in an order that starts at tid % k, so that the lanes of a
 // warp spread over the shared-memory banks.  In place: a thread reads its whole row before it rewrites it.
 template <int KP>
-__device__ __forceinline__ void prepare_rows_by_thread(TreeSmem& s, int k, int nrows, int tid) {
+__device__ __forceinline__ void prepare_rows_by_thread(TreeSmem& s, int k, int row0, int nrows, int tid, int nthreads) {
   const int start = tid % k;
-  for (int r = tid; r < nrows; r += G2_T) {
+  for (int r = row0 + tid; r < nrows; r += nthreads) {
     const int i = r == 0 ? 0 : 1 + (r - 1) / k;
     const int ra = r == 0 ? 0 : (r - 1) % k;
     const int at = (i * k + ra) * k;
@@ -1069,12 +1081,12 @@ __device__ __forceinline__ void prepare_rows_by_thread(TreeSmem& s, int k, int n
 // recount for equal values as rank_row_warp.  A thread that holds a whole row of 16 in registers spends a thousand
 // dependent instructions on it while most of the CTA's issue slots stay empty; here a row costs a few dozen.
 template <int KP>
-__device__ __forceinline__ void prepare_rows_by_group(TreeSmem& s, int k, int nrows, int tid) {
+__device__ __forceinline__ void prepare_rows_by_group(TreeSmem& s, int k, int row0, int nrows, int tid, int nthreads) {
   constexpr int RPW = 32 / KP;
   const int lane = tid & 31, warp = tid >> 5, g = lane / KP, e = lane % KP;
   unsigned long long* scratch64 = s.dw_row.ptr((long long)warp * 32, 32);
   uint32_t* key32 = reinterpret_cast<uint32_t*>(scratch64);  // [32] value keys (0 = none), then [32] marks
-  for (int rbase = warp * RPW; rbase < nrows; rbase += (G2_T / 32) * RPW) {
+  for (int rbase = row0 + warp * RPW; rbase < nrows; rbase += (nthreads / 32) * RPW) {
     const int r = rbase + g;
     const bool on = r < nrows && e < k;
     const int i = r == 0 ? 0 : 1 + (r - 1) / k;
@@ -1123,6 +1135,20 @@ __device__ __forceinline__ void prepare_rows_by_group(TreeSmem& s, int k, int nr
     }
   }
 }
+
+// Rows [row0, nrows) of a table of k <= 16 successors per row, by the first `nthreads` threads of the CTA (a
+// multiple of 32; all of them call).
+__device__ __forceinline__ void prepare_rows(TreeSmem& s, int k, int row0, int nrows, int tid, int nthreads) {
+  if (k <= 1) prepare_rows_by_thread<1>(s, k, row0, nrows, tid, nthreads);
+  else if (k <= 2) prepare_rows_by_thread<2>(s, k, row0, nrows, tid, nthreads);
+  else if (k <= 4) prepare_rows_by_thread<4>(s, k, row0, nrows, tid, nthreads);
+  else if (k <= 8) prepare_rows_by_group<8>(s, k, row0, nrows, tid, nthreads);
+  else prepare_rows_by_group<16>(s, k, row0, nrows, tid, nthreads);
+}
+// With k <= 16 and unbounded width the rows of the first kEagerDepths positions are prepared up front and the
+// rest only if the expansion appends a node that deep: a budget of a few hundred nodes rarely reaches beyond
+// depth 12, while the positions go up to L = 32.
+constexpr int kEagerDepths = 16;
 
 // LAZY: the rows of the pair table are computed on demand (see TreeSmem).
 template <bool LAZY>
@@ -1199,17 +1225,14 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
       if (!(lpv <= 0.f || lpv > 0.f) || lpv == INFINITY) atomicOr(&s.scalars[4], kStatusNonFinite);
     }
   }
-  int kp = 1;
-  while (kp < k) kp <<= 1;
+  // positions whose rows are prepared before the expansion starts (all of them unless the threshold rounds run)
+  const bool rounds_cta = !LAZY && !(W > 0 && W < budget);
+  int d_ready = rounds_cta && k <= 16 && L > kEagerDepths ? kEagerDepths : L;
   if constexpr (lazy) {
     // rows are normalised and sorted by the expanding warp, one at a time, when the search first needs them
   } else if (k <= 16) {
     __syncthreads();  // s.lp, s.tok
-    if (kp == 1) prepare_rows_by_thread<1>(s, k, nrows, tid);
-    else if (kp == 2) prepare_rows_by_thread<2>(s, k, nrows, tid);
-    else if (kp == 4) prepare_rows_by_thread<4>(s, k, nrows, tid);
-    else if (kp == 8) prepare_rows_by_group<8>(s, k, nrows, tid);
-    else prepare_rows_by_group<16>(s, k, nrows, tid);
+    prepare_rows(s, k, 0, 1 + (d_ready - 1) * k, tid, G2_T);
   } else {
     // 16 < k <= 64: one warp per (position, predecessor) row, two entries per lane; eq. 5, eq. 9, ranks by counting
     __syncthreads();  // s.lp, s.tok
@@ -1285,13 +1308,18 @@ k_build_tree(const float* __restrict__ bigram, int L, int k, int N, int W, float
     } else {
       if (tid < EX_T) {
         int n_sure = 1;
-        const int nn = expand_rounds_cta(s, L, k, budget, zeta, n_sure);
-        if (tid == 0) { s.scalars[1] = nn; s.scalars[2] = n_sure; }
+        const int nn = expand_rounds_cta(s, L, k, budget, zeta, n_sure, d_ready);
+        if (tid == 0) { s.scalars[1] = nn; s.scalars[2] = n_sure; s.scalars[5] = d_ready; }
       }
       __syncthreads();
       n = s.scalars[1];
+      d_ready = s.scalars[5];
     }
     if (n < 0) {
+      if (d_ready < L) {  // the sequential search may open any row
+        prepare_rows(s, k, 1 + (d_ready - 1) * k, 1 + (L - 1) * k, tid, G2_T);
+        d_ready = L;
+      }
       sequential = true;
       for (int i = tid; i < L + 2; i += G2_T) s.depth_cnt[i] = 0;
       __syncthreads();

@@ -179,6 +179,19 @@ def test_random_shapes_both_table_modes(block):
             raise AssertionError(f"shape k={k} L={L} N={N} W={W} V={V} {dtype} zeta={zeta} {cfg.mode}: {e}") from e
 
 
+@pytest.mark.parametrize("k,N,seed", [(8, 48, 0), (16, 96, 1), (6, 40, 2)])
+def test_deep_chains_open_rows_beyond_the_positions_prepared_up_front(k, N, seed):
+    """L = 28 positions with one dominant token per position: the tree is a few long chains, so the expansion
+    appends nodes deeper than the positions whose rows the tree kernel prepares before it starts."""
+    cfg = synth.CONFIGS["c2"].replace(name="deep", B=3, L=28, N=N, k=k, V=4096, scale="fixed:0.5", spike=12.0,
+                                      bigram_std=0.3)
+    di = synth.draft_inputs(cfg, seed)
+    otree = oracle.draft_tree(di.unigram_logits, di.bigram_scores, cfg.k, cfg.N)
+    assert int(otree.depths.max()) >= 20
+    run_case(cfg, seed, targets="agree")
+    run_case(cfg, seed, targets="plant", use_opts=True)
+
+
 def test_rows_full_of_ties():
     # bf16 rows quantised to a handful of values, rows with +-0 at the top, a constant row
     u = ubt()
