@@ -111,21 +111,28 @@ __device__ __forceinline__ void lm_list_state(const unsigned long long (&L)[KR],
   thr = kth != 0ull ? key_val(kth) : -INFINITY;
 }
 
+// How the vocabulary is cut into the tiles of the work items: n1 tiles of bn1 columns, then n2 tiles of bn2.
+struct LmTiling {
+  int bn1, n1, bn2, n2;
+  __host__ __device__ int width(int vt) const { return vt < n1 ? bn1 : bn2; }
+  __host__ __device__ int col_base(int vt) const { return vt < n1 ? vt * bn1 : n1 * bn1 + (vt - n1) * bn2; }
+};
+
 template <int KR>
 __global__ void __launch_bounds__(LM_THREADS, 1)
-k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w, int rows, int d,
-               int V, int k, int a_rows, int n_stages, int bn, LmParts parts, int* __restrict__ fail_flag) {
+k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_w,
+               const __grid_constant__ CUtensorMap map_w2, int rows, int d, int V, int k, int a_rows, int n_stages,
+               LmTiling tl, LmParts parts, int* __restrict__ fail_flag) {
   extern __shared__ __align__(1024) unsigned char lm_smem_raw[];
   unsigned char* ring = lm_smem_raw;
   LmShared& sh = *reinterpret_cast<LmShared*>(lm_smem_raw + LM_RING_BYTES);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int G = gridDim.x, cta = blockIdx.x;
-  // bn: vocabulary columns of a work item (a multiple of 16, at most LM_BN), chosen on the host so that the items
-  // spread evenly over the CTAs; a stage keeps room for LM_BN weight rows whatever bn is
-  const int n_rb = (rows + LM_RB - 1) / LM_RB, n_vt = (V + bn - 1) / bn, n_kb = d / LM_BK;
+  // The vocabulary is cut into tl.n1 tiles of tl.bn1 columns followed by tl.n2 tiles of tl.bn2 columns (multiples
+  // of 16, at most LM_BN), chosen on the host so that the work items fill whole rounds over the CTAs; a stage keeps
+  // room for LM_BN weight rows whatever the width is.
+  const int n_rb = (rows + LM_RB - 1) / LM_RB, n_vt = tl.n1 + tl.n2, n_kb = d / LM_BK;
   const int a_bytes = a_rows * LM_BK * 2, stage_bytes = a_bytes + LM_B_BYTES;
-  const uint32_t tx_bytes = (uint32_t)(a_bytes + bn * LM_BK * 2);
-  const uint32_t idesc = tc_idesc_bf16(LM_BM, bn);
   // work items: (vocabulary tile, row block) pairs, row block fastest, dealt round-robin: cta, cta + G, ...
   const int n_all = n_vt * n_rb;
   const int n_items = cta < n_all ? (n_all - cta + G - 1) / G : 0;
@@ -152,6 +159,9 @@ k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant_
       int it = 0;
       for (int item = 0; item < n_items && !*fail; ++item) {
         const int g = cta + item * G, vt = g / n_rb, rb = g % n_rb;
+        const bool wide = vt < tl.n1;
+        const uint32_t tx_bytes = (uint32_t)(a_bytes + tl.width(vt) * LM_BK * 2);
+        const int col_base = tl.col_base(vt);
         for (int kb = 0; kb < n_kb; ++kb, ++it) {
           const int s = it % n_stages;
           const uint32_t ph = (uint32_t)(it / n_stages) & 1u;
@@ -159,7 +169,7 @@ k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant_
           lm_bar_expect(&sh.full[s], tx_bytes);
           unsigned char* a = ring + (size_t)s * stage_bytes;
           lm_tma_load(a, &map_h, kb * LM_BK, rb * LM_RB, &sh.full[s]);
-          lm_tma_load(a + a_bytes, &map_w, kb * LM_BK, vt * bn, &sh.full[s]);
+          lm_tma_load(a + a_bytes, wide ? &map_w : &map_w2, kb * LM_BK, col_base, &sh.full[s]);
         }
       }
       if (*fail)  // gave up: before the CTA leaves, wait (bounded) for the copies still landing in its ring
@@ -173,6 +183,7 @@ k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant_
       uint32_t use[2] = {0u, 0u};  // how often each accumulator has been handed over
       for (int item = 0; item < n_items && !*fail; ++item) {
         const int rb = (cta + item * G) % n_rb;
+        const uint32_t idesc = tc_idesc_bf16(LM_BM, tl.width((cta + item * G) / n_rb));
         const int n_half = rows - rb * LM_RB > LM_BM ? 2 : 1;  // a row block of at most 128 rows fills one accumulator
         bool ok = true;
         for (int kb = 0; kb < n_kb && ok; ++kb, ++it) {
@@ -222,7 +233,7 @@ k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant_
       use += 1u;
       const bool first = !((visited >> rb) & 1ull);
       visited |= 1ull << rb;
-      const int col_base = vt * bn;
+      const int col_base = tl.col_base(vt), bn = tl.width(vt);
       const int row = rb * LM_RB + half * LM_BM + r_in_tile;
       const bool valid = row < rows;
       const size_t slot = (size_t)cta * parts.rpad + row;
@@ -450,12 +461,30 @@ cudaError_t launch_lm_head_topk(const void* hidden, const void* weight, int64_t 
   // rows streams the weights (bound by their bandwidth), and 27 us + 0.12 us per column with two accumulators.
   const int n_rb = (int)((rows + LM_RB - 1) / LM_RB);
   const int fixed_cols = rows <= LM_RB ? 60 : 224;
-  int bn = LM_BN;
+  LmTiling tl{LM_BN, (V + LM_BN - 1) / LM_BN, LM_BN, 0};
   long long best_cost = -1;
   for (int w = LM_BN; w >= 128; w -= 16) {
     const long long items = (long long)((V + w - 1) / w) * n_rb;
     const long long cost = ((items + grid - 1) / grid) * (w + fixed_cols);
-    if (best_cost < 0 || cost < best_cost) { best_cost = cost; bn = w; }
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; tl = LmTiling{w, (V + w - 1) / w, w, 0}; }
+  }
+  // Two widths 16 apart let the number of tiles be chosen freely, so that the items are exactly `rounds` per CTA:
+  // 666 tiles of 240 and 224 columns are nine full rounds for two row blocks over 148 CTAs, against nine rounds
+  // (the last nearly empty) of 256-column tiles.
+  for (long long rounds = 1; rounds <= 4096; ++rounds) {
+    const long long n_tiles = rounds * grid / n_rb;
+    if (n_tiles < 1 || n_tiles * LM_BN < V) continue;
+    const int lo = (int)(V / n_tiles) / 16 * 16;  // the narrower width
+    if (lo < 128) break;                          // narrower tiles than the uniform search considers
+    const int hi = lo + 16 <= LM_BN ? lo + 16 : LM_BN;
+    const long long n_hi = hi > lo ? (V - n_tiles * lo + 15) / 16 : 0;  // tiles that must be 16 columns wider
+    if (n_hi > n_tiles) continue;
+    const long long cost = rounds * (long long)((V + n_tiles - 1) / n_tiles + fixed_cols);
+    if (cost < best_cost) {
+      best_cost = cost;
+      tl = n_hi > 0 ? LmTiling{hi, (int)n_hi, lo, (int)(n_tiles - n_hi)} : LmTiling{lo, (int)n_tiles, lo, 0};
+    }
+    break;  // more rounds of narrower tiles only cost more
   }
   cudaError_t e = allow_max_dynamic_smem<k_lm_head_topk<4>>();
   if (e == cudaSuccess) e = allow_max_dynamic_smem<k_lm_head_topk<8>>();
@@ -471,15 +500,16 @@ cudaError_t launch_lm_head_topk(const void* hidden, const void* weight, int64_t 
   parts.cnt = reinterpret_cast<int32_t*>(p);
   e = cudaMemsetAsync(fail_flag, 0, 256, st);
   if (e != cudaSuccess) return e;
-  CUtensorMap map_w, map_h;
-  if (!make_map(&map_w, weight, (uint64_t)d, (uint64_t)V, (uint32_t)bn)) return cudaErrorNotSupported;
+  CUtensorMap map_w, map_w2, map_h;
+  if (!make_map(&map_w, weight, (uint64_t)d, (uint64_t)V, (uint32_t)tl.bn1)) return cudaErrorNotSupported;
+  if (!make_map(&map_w2, weight, (uint64_t)d, (uint64_t)V, (uint32_t)tl.bn2)) return cudaErrorNotSupported;
   if (!make_map(&map_h, hidden, (uint64_t)d, (uint64_t)rows, (uint32_t)a_rows)) return cudaErrorNotSupported;
   if (k <= 4)
-    k_lm_head_topk<4><<<grid, LM_THREADS, smem, st>>>(map_h, map_w, (int)rows, d, V, k, a_rows, n_stages, bn, parts, fail_flag);
+    k_lm_head_topk<4><<<grid, LM_THREADS, smem, st>>>(map_h, map_w, map_w2, (int)rows, d, V, k, a_rows, n_stages, tl, parts, fail_flag);
   else if (k <= 8)
-    k_lm_head_topk<8><<<grid, LM_THREADS, smem, st>>>(map_h, map_w, (int)rows, d, V, k, a_rows, n_stages, bn, parts, fail_flag);
+    k_lm_head_topk<8><<<grid, LM_THREADS, smem, st>>>(map_h, map_w, map_w2, (int)rows, d, V, k, a_rows, n_stages, tl, parts, fail_flag);
   else
-    k_lm_head_topk<16><<<grid, LM_THREADS, smem, st>>>(map_h, map_w, (int)rows, d, V, k, a_rows, n_stages, bn, parts, fail_flag);
+    k_lm_head_topk<16><<<grid, LM_THREADS, smem, st>>>(map_h, map_w, map_w2, (int)rows, d, V, k, a_rows, n_stages, tl, parts, fail_flag);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   k_lm_head_merge<<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(parts, grid, (int)rows, k, cand_ids, cand_lp);
