@@ -284,14 +284,45 @@ int ubt_verify_tree_keys(const ubt_tree *tree, const unsigned long long *gathere
  * target's pick of every slot.  node_pick[B, node_budget] (DEVICE, int32, read only) is the token the target
  * chose at each slot: from ubt_lm_head_topk with k = 1 on the target's hidden states of the tree slots (greedy
  * verification with the target logits never written to memory: cand_ids[B * node_budget, 1] IS this array), from
- * a sampler of the caller's, or gathered from other ranks.  From the root the walk follows the child whose token
- * equals the pick of the current slot until none matches; that pick is the bonus token.  *out is written as
- * ubt_verify_tree writes it.  Every entry must be a token id >= 0 or negative for "no valid pick": a sequence
- * with a negative entry at any of its node_budget slots gets UBT_STATUS_NONFINITE in status[b] (DEVICE, B words,
- * may be NULL), and the entry counts as token 0.  No workspace.  Stream-ordered like every other call.
+ * a sampler of the caller's, or gathered from the ranks of a vocabulary-parallel group: with shards > 1 node_pick
+ * is [shards, B, node_budget] and the pick of a slot is the largest of the shards' entries (the rank that owns the
+ * pick holds a token, the others -1; if all are negative the smallest is taken); shards = 1 otherwise.  From the
+ * root the walk follows the child whose token equals the pick of the current slot until none matches; that pick is
+ * the bonus token.  *out is written as ubt_verify_tree writes it.  Every entry must be a token id >= 0 or negative
+ * for "no valid pick": a sequence with a negative pick at any of its node_budget slots gets UBT_STATUS_NONFINITE
+ * (UBT_STATUS_WAIT_GAVE_UP for -2) in status[b] (DEVICE, B words, may be NULL), and the pick counts as token 0.
+ * No workspace.  Stream-ordered like every other call.
  */
-int ubt_verify_tree_picks(const ubt_tree *tree, const int32_t *node_pick, ubt_verify_result *out,
+int ubt_verify_tree_picks(const ubt_tree *tree, const int32_t *node_pick, int shards, ubt_verify_result *out,
                           int32_t *status, void *cuda_stream);
+
+/*
+ * Sampling step a4 with the vocabulary of the target logits split over the ranks of a tensor-parallel group.  The
+ * integer weights of ubt_verify_tree's sampling mode make the split exact -- the picks are bit-identical to those
+ * of one GPU holding whole rows.  Rank r holds the columns [v0, v0 + Vs) of every target row as a dense
+ * [B, node_budget, Vs] tensor; ranks are numbered in the order of their columns.  Per call of the verifier:
+ *   1. ubt_verify_keys_shard (above) -> row_keys; all-gather -> gathered_keys[shards, B * node_budget]: the row
+ *      maximum over the whole vocabulary is the value of the largest key;
+ *   2. ubt_sample_totals_shard: the weights w_v = trunc(2^(40 + fma(z_v, a, c))) of this rank's columns with
+ *      a = log2(e)/temperature, c = -max * a, summed per row into totals[B * node_budget] (DEVICE, uint64); the
+ *      per-1024-token sums stay in `workspace` for step 3; all-gather -> gathered_totals[shards, B * node_budget];
+ *   3. ubt_sample_picks_shard: theta = floor(R * sum of the ranks' totals / 2^64) as in ubt_verify_tree; the one
+ *      rank whose share of the running sum over ranks holds theta writes the token (counted in the WHOLE
+ *      vocabulary) to picks[B * node_budget] (DEVICE, int32), every other rank -1; a row whose maximum is NaN or
+ *      +inf on any rank gets -1 from every rank (-2 after an abandoned device-side wait);
+ *      all-gather -> gathered_picks[shards, B * node_budget];
+ *   4. ubt_verify_tree_picks with that array and `shards`.
+ * `workspace` (steps 2 and 3, the same buffer, untouched in between): ubt_verify_workspace_bytes(B, node_budget, Vs,
+ * UBT_VERIFY_SAMPLE).  `rank` is this rank's position in the gathered arrays.  No collective is issued by the
+ * library: three all-gathers of 8, 8 and 4 bytes per tree slot.
+ */
+int ubt_sample_totals_shard(const void *target_shard, int dtype, int B, int node_budget, int Vs,
+                            const unsigned long long *gathered_keys, int shards, float temperature,
+                            unsigned long long *totals, void *workspace, size_t workspace_bytes,
+                            void *cuda_stream);
+int ubt_sample_picks_shard(const void *target_shard, int dtype, int B, int node_budget, int Vs, int v0, int rank,
+                           const unsigned long long *gathered_totals, int shards, uint64_t seed, int32_t *picks,
+                           void *workspace, size_t workspace_bytes, void *cuda_stream);
 
 /*
  * Host-buffer forms.  Every pointer inside `tree`, `opts` (alpha ... pos_offset, node_pick) and

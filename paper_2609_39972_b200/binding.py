@@ -58,7 +58,7 @@ EXPORTS = ["ubt_version", "ubt_status_string", "ubt_debug_ring_timeouts", "ubt_d
            "ubt_draft_host_buffer_bytes", "ubt_verify_host_buffer_bytes", "ubt_draft_tree_host",
            "ubt_verify_tree_host", "ubt_verify_tree_static", "ubt_verify_static_capacity", "ubt_lm_head_workspace_bytes",
            "ubt_lm_head_topk", "ubt_topk_shard_bytes", "ubt_topk_shard", "ubt_topk_merge_shards", "ubt_verify_keys_shard",
-           "ubt_verify_tree_keys", "ubt_verify_tree_picks"]
+           "ubt_verify_tree_keys", "ubt_verify_tree_picks", "ubt_sample_totals_shard", "ubt_sample_picks_shard"]
 
 _lib = None
 
@@ -112,7 +112,11 @@ def load() -> C.CDLL:
     L.ubt_verify_keys_shard.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
                                         C.c_size_t, C.c_void_p]
     L.ubt_verify_tree_keys.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
-    L.ubt_verify_tree_picks.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.ubt_verify_tree_picks.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
+    L.ubt_sample_totals_shard.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_int,
+                                          C.c_float, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    L.ubt_sample_picks_shard.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_void_p,
+                                         C.c_int, C.c_uint64, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
     L.ubt_debug_ring_timeouts.restype = C.c_longlong
     L.ubt_draft_tree_host.argtypes = L.ubt_draft_tree.argtypes
     L.ubt_verify_tree_host.argtypes = L.ubt_verify_tree.argtypes
@@ -441,21 +445,71 @@ def ubt_verify_tree_keys(tree: Tree, gathered_keys: torch.Tensor, shards: int,
     return result
 
 
-def ubt_verify_tree_picks(tree: Tree, node_pick: torch.Tensor, result: Optional[VerifyResult] = None,
-                          status: Optional[torch.Tensor] = None, stream=None) -> VerifyResult:
+def ubt_verify_tree_picks(tree: Tree, node_pick: torch.Tensor, shards: int = 1,
+                          result: Optional[VerifyResult] = None, status: Optional[torch.Tensor] = None,
+                          stream=None) -> VerifyResult:
     """The walk alone on given per-slot picks ``node_pick`` (``int32[B, N]``, or ``[B * N, 1]`` as
-    ``ubt_lm_head_topk`` with ``k = 1`` returns them)."""
+    ``ubt_lm_head_topk`` with ``k = 1`` returns them; with ``shards > 1`` the ranks' picks back to back,
+    ``[shards, B, N]``)."""
     _need(node_pick, "node_pick")
-    if node_pick.dtype != torch.int32 or node_pick.numel() != tree.B * tree.N or not node_pick.is_contiguous():
-        raise ValueError("node_pick must be a contiguous int32 tensor of B * N entries")
+    if (node_pick.dtype != torch.int32 or node_pick.numel() != shards * tree.B * tree.N
+            or not node_pick.is_contiguous()):
+        raise ValueError("node_pick must be a contiguous int32 tensor of shards * B * N entries")
     if result is None:
         result = VerifyResult.empty(tree.B, tree.L, node_pick.device)
     t = tree.c_struct()
     r = result.c_struct()
-    _check(load().ubt_verify_tree_picks(C.byref(t), _ptr(node_pick), C.byref(r), _ptr(status), _stream(stream)),
-           "ubt_verify_tree_picks")
-    result.node_pick = node_pick.view(tree.B, tree.N)
+    _check(load().ubt_verify_tree_picks(C.byref(t), _ptr(node_pick), shards, C.byref(r), _ptr(status),
+                                        _stream(stream)), "ubt_verify_tree_picks")
+    result.node_pick = node_pick.view(tree.B, tree.N) if shards == 1 else None
     return result
+
+
+def ubt_sample_totals_shard(target_shard: torch.Tensor, gathered_keys: torch.Tensor, shards: int,
+                            temperature: float = 1.0, totals: Optional[torch.Tensor] = None,
+                            ws: Optional[torch.Tensor] = None, stream=None):
+    """Sampling a4 over a vocabulary-parallel group, second step: the integer weights of this rank's columns summed
+    per row (``int64[B * N]``), with the row maximum taken from the gathered keys.  Returns ``(totals, ws)``; pass
+    the same ``ws`` to ``ubt_sample_picks_shard``."""
+    _need(target_shard, "target_shard"); _need(gathered_keys, "gathered_keys")
+    B, N, Vs = target_shard.shape
+    if totals is None:
+        totals = torch.empty((B * N,), dtype=torch.int64, device=target_shard.device)
+    if ws is None:
+        ws = workspace(ubt_verify_workspace_bytes(B, N, Vs, "sample"), target_shard.device)
+    _check(load().ubt_sample_totals_shard(_ptr(target_shard), _dtype_code(target_shard), B, N, Vs, _ptr(gathered_keys),
+                                          shards, float(temperature), _ptr(totals), _ptr(ws), ws.numel(),
+                                          _stream(stream)), "ubt_sample_totals_shard")
+    return totals, ws
+
+
+def ubt_sample_picks_shard(target_shard: torch.Tensor, v0: int, rank: int, gathered_totals: torch.Tensor, shards: int,
+                           seed: int, ws: torch.Tensor, picks: Optional[torch.Tensor] = None, stream=None):
+    """Third step: this rank's picks (``int32[B * N]``: a token where the rank owns the slot's pick, else -1)."""
+    _need(target_shard, "target_shard"); _need(gathered_totals, "gathered_totals")
+    B, N, Vs = target_shard.shape
+    if picks is None:
+        picks = torch.empty((B * N,), dtype=torch.int32, device=target_shard.device)
+    _check(load().ubt_sample_picks_shard(_ptr(target_shard), _dtype_code(target_shard), B, N, Vs, int(v0), int(rank),
+                                         _ptr(gathered_totals), shards, int(seed) & 0xFFFFFFFFFFFFFFFF, _ptr(picks),
+                                         _ptr(ws), ws.numel(), _stream(stream)), "ubt_sample_picks_shard")
+    return picks
+
+
+def sample_tree_vocab_parallel(tree: Tree, target_shard: torch.Tensor, v0: int, seed: int, temperature: float = 1.0,
+                               group=None, **kw) -> VerifyResult:
+    """Sampling verification of target logits whose vocabulary is split over the ranks of ``group`` (ranks in the
+    order of their columns): keys, totals and picks with one all-gather each, then the walk; all on torch's current
+    stream.  Every rank returns the verdict that one GPU holding whole rows would."""
+    import torch.distributed as dist
+    rank = dist.get_rank(group) if dist.is_available() and dist.is_initialized() else 0
+    keys = ubt_verify_keys_shard(target_shard, v0)
+    g_keys, shards = gather_shard_partials(keys, group)
+    totals, ws = ubt_sample_totals_shard(target_shard, g_keys, shards, temperature)
+    g_tot, _ = gather_shard_partials(totals, group)
+    picks = ubt_sample_picks_shard(target_shard, v0, rank, g_tot, shards, seed, ws)
+    g_picks, _ = gather_shard_partials(picks, group)
+    return ubt_verify_tree_picks(tree, g_picks, shards, **kw)
 
 
 def verify_tree_from_hidden(tree: Tree, target_hidden: torch.Tensor, weight: torch.Tensor, **kw) -> VerifyResult:

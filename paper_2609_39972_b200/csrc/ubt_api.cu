@@ -369,9 +369,9 @@ int ubt_verify_tree(const ubt_tree* tree, const void* target_logits, int dtype, 
   return UBT_OK;
 }
 
-int ubt_verify_tree_picks(const ubt_tree* tree, const int32_t* node_pick, ubt_verify_result* out, int32_t* status,
-                          void* cuda_stream) {
-  if (!tree || !out || !node_pick) return UBT_ERR_INVALID_ARG;
+int ubt_verify_tree_picks(const ubt_tree* tree, const int32_t* node_pick, int shards, ubt_verify_result* out,
+                          int32_t* status, void* cuda_stream) {
+  if (!tree || !out || !node_pick || shards < 1) return UBT_ERR_INVALID_ARG;
   if (!tree->token_ids || !tree->parents || !tree->n_nodes) return UBT_ERR_INVALID_ARG;
   if (!out->accepted_len || !out->bonus_token || !out->accepted_nodes || !out->out_tokens) return UBT_ERR_INVALID_ARG;
   const int B = tree->B, N = tree->N, L = tree->L;
@@ -380,7 +380,50 @@ int ubt_verify_tree_picks(const ubt_tree* tree, const int32_t* node_pick, ubt_ve
   if (B == 0) return UBT_OK;
   // the walk kernel in the mode that takes the picks as given (the sampling mode's second half)
   if (launch_walk(*tree, UBT_VERIFY_SAMPLE, VerifyWorkspace{}, 0, node_pick, nullptr, *out, status,
-                  static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+                  static_cast<cudaStream_t>(cuda_stream), shards) != cudaSuccess)
+    return UBT_ERR_CUDA;
+  return UBT_OK;
+}
+
+static int check_sample_shard(const void* target_shard, int dtype, int B, int N, int Vs, const void* gathered, int shards,
+                              void* workspace, size_t workspace_bytes) {
+  if (!target_shard || !gathered || B < 0 || N < 1 || Vs < 1 || shards < 1) return UBT_ERR_INVALID_ARG;
+  if (dtype != UBT_F32 && dtype != UBT_BF16) return UBT_ERR_INVALID_ARG;
+  if (!aligned16(target_shard) || !aligned16(gathered)) return UBT_ERR_INVALID_ARG;
+  if (N > kMaxN) return UBT_ERR_UNSUPPORTED;
+  if (B > 0 && (!workspace || !aligned16(workspace) ||
+                workspace_bytes < verify_workspace_bytes((int64_t)B * N, Vs, UBT_VERIFY_SAMPLE)))
+    return UBT_ERR_WORKSPACE;
+  return UBT_OK;
+}
+
+int ubt_sample_totals_shard(const void* target_shard, int dtype, int B, int N, int Vs,
+                            const unsigned long long* gathered_keys, int shards, float temperature,
+                            unsigned long long* totals, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  const int rc = check_sample_shard(target_shard, dtype, B, N, Vs, gathered_keys, shards, workspace, workspace_bytes);
+  if (rc != UBT_OK) return rc;
+  if (!totals || !(temperature > 0.f)) return UBT_ERR_INVALID_ARG;
+  if (B == 0) return UBT_OK;
+  const int64_t rows = (int64_t)B * N;
+  const VerifyWorkspace w = carve_verify_workspace(workspace, rows, Vs, UBT_VERIFY_SAMPLE);
+  if (launch_row_totals_shard(target_shard, dtype, rows, Vs, gathered_keys, shards, temperature, w, totals,
+                              static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    return UBT_ERR_CUDA;
+  return UBT_OK;
+}
+
+int ubt_sample_picks_shard(const void* target_shard, int dtype, int B, int N, int Vs, int v0, int rank,
+                           const unsigned long long* gathered_totals, int shards, uint64_t seed, int32_t* picks,
+                           void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  const int rc = check_sample_shard(target_shard, dtype, B, N, Vs, gathered_totals, shards, workspace, workspace_bytes);
+  if (rc != UBT_OK) return rc;
+  if (!picks || v0 < 0 || rank < 0 || rank >= shards) return UBT_ERR_INVALID_ARG;
+  if ((int64_t)v0 + Vs > 0x7fffffffll) return UBT_ERR_UNSUPPORTED;
+  if (B == 0) return UBT_OK;
+  const int64_t rows = (int64_t)B * N;
+  const VerifyWorkspace w = carve_verify_workspace(workspace, rows, Vs, UBT_VERIFY_SAMPLE);
+  if (launch_row_pick_shard(target_shard, dtype, rows, N, Vs, v0, rank, shards, gathered_totals, seed, w, picks,
+                            static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
     return UBT_ERR_CUDA;
   return UBT_OK;
 }

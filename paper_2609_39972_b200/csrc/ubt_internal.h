@@ -127,7 +127,14 @@ cudaError_t launch_row_sample(const void* logits, int dtype, int B, int N, int V
                               cudaStream_t st);
 cudaError_t launch_walk(const ubt_tree& tree, int mode, const VerifyWorkspace& w, int V,
                         const int32_t* sampled_pick, int32_t* node_pick,
-                        const ubt_verify_result& out, int32_t* status, cudaStream_t st);
+                        const ubt_verify_result& out, int32_t* status, cudaStream_t st, int pick_shards = 1);
+// sampling a4 over a vocabulary-parallel group (see ubt_verify.cu)
+cudaError_t launch_row_totals_shard(const void* logits, int dtype, int64_t rows, int Vs,
+                                    const unsigned long long* gathered_keys, int shards, float temperature,
+                                    const VerifyWorkspace& w, unsigned long long* totals, cudaStream_t st);
+cudaError_t launch_row_pick_shard(const void* logits, int dtype, int64_t rows, int N, int Vs, int v0, int rank, int shards,
+                                  const unsigned long long* gathered_totals, uint64_t seed, const VerifyWorkspace& w,
+                                  int32_t* pick, cudaStream_t st);
 
 // vocabulary-parallel greedy a4: one key per row of this rank's slice; the walk on the gathered keys
 cudaError_t launch_row_keys_shard(const VerifyWorkspace& w, int64_t rows, int V, int v0, unsigned long long* row_keys,

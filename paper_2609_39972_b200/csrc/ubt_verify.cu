@@ -308,16 +308,20 @@ constexpr int G5_CHUNK = 1024;  // tokens per partial sum
 // One warp: from the per-1024-token sums of a row's integer weights to the sampled token.  total = sum of
 // the sums; theta = floor(R * total / 2^64) with R from Philox4x32-10(counter = (slot, b, 0, 0), key = seed);
 // the pick is the first token whose inclusive prefix sum exceeds theta.  All lanes return the pick.
-template <typename T>
-__device__ int locate_pick(const T* rowp, int V, float a, float c, const unsigned long long* csum, int nchunks,
-                           uint64_t seed, uint32_t b, uint32_t slot, int lane) {
-  unsigned long long run = 0;
-  for (int ch = lane; ch < nchunks; ch += 32) run += csum[ch];
-  const unsigned long long total = warp_sum_u64(run);
+// theta = floor(R * total / 2^64), R the first two words of Philox4x32-10(counter = (slot, b, 0, 0), key = seed)
+__device__ __forceinline__ unsigned long long sample_threshold(uint64_t seed, uint32_t b, uint32_t slot,
+                                                               unsigned long long total) {
   uint32_t x[4];
   philox4x32_10(slot, b, 0u, 0u, (uint32_t)seed, (uint32_t)(seed >> 32), x);
   const unsigned long long R = (unsigned long long)x[0] | ((unsigned long long)x[1] << 32);
-  unsigned long long theta = __umul64hi(R, total);
+  return __umul64hi(R, total);
+}
+
+// One warp: the first token of rowp[0, V) whose inclusive prefix sum of weights exceeds theta (theta below the sum
+// of all of them), from the per-1024-token sums csum.  All lanes return it.
+template <typename T>
+__device__ int locate_theta(const T* rowp, int V, float a, float c, const unsigned long long* csum, int nchunks,
+                            unsigned long long theta, int lane) {
   // sequential over groups of 32 chunks, warp scan inside a group
   int found_chunk = nchunks - 1;
   unsigned long long before = 0;
@@ -367,6 +371,15 @@ __device__ int locate_pick(const T* rowp, int V, float a, float c, const unsigne
     ans = ans < V ? ans : V - 1;
   }
   return __shfl_sync(FULL, ans, l);
+}
+
+template <typename T>
+__device__ int locate_pick(const T* rowp, int V, float a, float c, const unsigned long long* csum, int nchunks,
+                           uint64_t seed, uint32_t b, uint32_t slot, int lane) {
+  unsigned long long run = 0;
+  for (int ch = lane; ch < nchunks; ch += 32) run += csum[ch];
+  const unsigned long long total = warp_sum_u64(run);
+  return locate_theta<T>(rowp, V, a, c, csum, nchunks, sample_threshold(seed, b, slot, total), lane);
 }
 
 // ---------------------------------------------------------------------------- sampling picks, ring-fed
@@ -651,6 +664,15 @@ k_walk(ubt_tree tree, int mode, SpanPlan plan, const unsigned long long* __restr
       else if (best >= kKeyPlusInf) bits = kStatusNonFinite;  // +inf as the maximum, or the NaN marker
     } else {
       p = sampled_pick[o + n];
+      // picks gathered from the ranks of a vocabulary-parallel group: the one rank that owns the slot's pick has a
+      // token there, the others -1; no owner at all = no valid pick (the most severe marker is kept)
+      int worst = p;
+      for (int r = 1; r < shards; ++r) {
+        const int q = sampled_pick[(int64_t)r * shard_stride + o + n];
+        p = q > p ? q : p;
+        worst = q < worst ? q : worst;
+      }
+      if (p < 0) p = worst;
       if (p < 0) { bits = p == -2 ? kStatusWaitGaveUp : kStatusNonFinite; p = 0; }
     }
     if (bits) atomicOr(&s_bits, bits);
@@ -823,11 +845,11 @@ cudaError_t launch_row_sample(const void* logits, int dtype, int B, int N, int V
 
 cudaError_t launch_walk(const ubt_tree& tree, int mode, const VerifyWorkspace& w, int V,
                         const int32_t* sampled_pick, int32_t* node_pick, const ubt_verify_result& out,
-                        int32_t* status, cudaStream_t st) {
+                        int32_t* status, cudaStream_t st, int pick_shards) {
   if (tree.B == 0) return cudaSuccess;
   return launch_kernel(k_walk, dim3(tree.B), dim3(128), 0, st, true, tree, mode, w.plan,
-                       (const unsigned long long*)w.part_key, V, sampled_pick, node_pick, out, status, 0,
-                       (int64_t)0);
+                       (const unsigned long long*)w.part_key, V, sampled_pick, node_pick, out, status,
+                       mode == UBT_VERIFY_GREEDY ? 0 : pick_shards, (int64_t)tree.B * tree.N);
 }
 
 // Vocabulary-parallel greedy a4, first half: one key per row of this rank's slice -- the best key of the row's
@@ -864,6 +886,135 @@ cudaError_t launch_walk_keys(const ubt_tree& tree, const unsigned long long* gat
   return launch_kernel(k_walk, dim3(tree.B), dim3(128), 0, st, true, tree, (int)UBT_VERIFY_GREEDY, SpanPlan{},
                        gathered_keys, 1, (const int32_t*)nullptr, node_pick, out, status, shards,
                        (int64_t)tree.B * tree.N);
+}
+
+// ------------------------------------------------------- sampling a4 with the vocabulary split over ranks
+// The integer weights make the split exact: with the row maximum taken over ALL ranks' slices (from the gathered
+// keys of the greedy pass), every rank computes the weights of its own columns with the same (a, c) as one GPU
+// would, the row total is the sum of the ranks' totals, theta follows from it, and the rank whose share of the
+// running sum holds theta finds the token in its slice.
+//
+// First half: per row the global maximum from the gathered keys, (a, c), the per-1024-token sums of this slice's
+// weights (kept in the workspace for the second half) and their total.
+template <typename T, int VEC>
+__global__ void __launch_bounds__(G5_T, 2)
+k_row_totals_shard(const T* __restrict__ logits, int64_t rows, int Vs, const unsigned long long* __restrict__ gathered_keys,
+                   int shards, float temperature, float* __restrict__ row_ac, unsigned long long* __restrict__ block_sum,
+                   int nblocks, unsigned long long* __restrict__ totals) {
+  __shared__ unsigned long long wsum[G5_T / 32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int CF = G5_CHUNK / VEC;  // fragments per chunk
+  const float inv_t = __fdiv_rn(1.0f, temperature);
+  const float a = __fmul_rn(0x1.715476p+0f, inv_t);
+  for (int64_t row = blockIdx.x; row < rows; row += gridDim.x) {
+    unsigned long long best = 0;
+    for (int r = 0; r < shards; ++r) {
+      const unsigned long long key = gathered_keys[(int64_t)r * rows + row];
+      best = key > best ? key : best;
+    }
+    // a marker key (a NaN or +inf somewhere in the row, an abandoned wait) or no key at all: no pick for this row
+    float a_row = a, c = __uint_as_float(0x7fc00000u);
+    if (best == kKeyGaveUp) a_row = -1.0f;
+    else if (best != 0ull && best < kKeyPlusInf) c = -__fmul_rn(key_val(best), a);
+    const bool live = a_row >= 0.f && c == c && c != INFINITY && c != -INFINITY;
+    if (tid == 0) { row_ac[row * 2] = a_row; row_ac[row * 2 + 1] = c; }
+    unsigned long long wtot = 0;
+    if (live) {
+      const T* rowp = logits + row * Vs;
+      const int nfrag = Vs / VEC;  // Vs % VEC == 0 on the vector path; VEC == 1 otherwise
+      for (int ch = warp; ch < nblocks; ch += G5_T / 32) {
+        unsigned long long acc = 0;
+        for (int fi = lane; fi < CF; fi += 32) {
+          const int f = ch * CF + fi;
+          if (f < nfrag) {
+            uint4 raw; float sc = 0.f;
+            load_row_frag<T, VEC>(rowp, nfrag, f, raw, sc);
+            float x[VEC];
+            frag_values<T, VEC>(raw, sc, x);
+#pragma unroll
+            for (int j = 0; j < VEC; ++j) acc += weight_of(x[j], a, c);
+          }
+        }
+        acc = warp_sum_u64(acc);
+        if (lane == 0) block_sum[row * nblocks + ch] = acc;
+        wtot += acc;
+      }
+    }
+    if (lane == 0) wsum[warp] = wtot;
+    __syncthreads();
+    if (tid == 0) {
+      unsigned long long t = 0;
+      for (int w = 0; w < G5_T / 32; ++w) t += wsum[w];
+      totals[row] = t;
+    }
+    __syncthreads();
+  }
+}
+
+// Second half, one warp per row: theta from the sum of the ranks' totals; the rank whose share [before, before +
+// own total) holds theta writes the token (counted in the whole vocabulary), every other rank -1.  A row without a
+// valid maximum gets -1 (-2 after an abandoned wait) from every rank.
+template <typename T>
+__global__ void __launch_bounds__(128)
+k_row_pick_shard(const T* __restrict__ logits, int64_t rows, int N, int Vs, int v0, int rank, int shards,
+                 const unsigned long long* __restrict__ gathered_totals, uint64_t seed, const float* __restrict__ row_ac,
+                 const unsigned long long* __restrict__ block_sum, int nblocks, int32_t* __restrict__ pick) {
+  const int lane = threadIdx.x & 31;
+  const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const float a = row_ac[row * 2], c = row_ac[row * 2 + 1];
+  int ans = -1;
+  if (a < 0.f) {
+    ans = -2;
+  } else if (c == c && c != INFINITY && c != -INFINITY) {
+    unsigned long long total = 0, before = 0;
+    for (int r = 0; r < shards; ++r) {
+      const unsigned long long t = gathered_totals[(int64_t)r * rows + row];
+      if (r < rank) before += t;
+      total += t;
+    }
+    const unsigned long long mine = gathered_totals[(int64_t)rank * rows + row];
+    const unsigned long long theta = sample_threshold(seed, (uint32_t)(row / N), (uint32_t)(row % N), total);
+    if (theta >= before && theta - before < mine)
+      ans = v0 + locate_theta<T>(logits + row * Vs, Vs, a, c, block_sum + row * nblocks, nblocks, theta - before, lane);
+  }
+  if (lane == 0) pick[row] = ans;
+}
+
+cudaError_t launch_row_totals_shard(const void* logits, int dtype, int64_t rows, int Vs,
+                                    const unsigned long long* gathered_keys, int shards, float temperature,
+                                    const VerifyWorkspace& w, unsigned long long* totals, cudaStream_t st) {
+  if (rows == 0) return cudaSuccess;
+  const int grid = (int)(rows < 4096 ? rows : 4096);
+  if (dtype == UBT_BF16) {
+    if (Vs % 8 == 0)
+      k_row_totals_shard<__nv_bfloat16, 8><<<grid, G5_T, 0, st>>>(static_cast<const __nv_bfloat16*>(logits), rows, Vs, gathered_keys,
+                                                                   shards, temperature, w.row_ac, w.block_sum, w.nblocks, totals);
+    else
+      k_row_totals_shard<__nv_bfloat16, 1><<<grid, G5_T, 0, st>>>(static_cast<const __nv_bfloat16*>(logits), rows, Vs, gathered_keys,
+                                                                   shards, temperature, w.row_ac, w.block_sum, w.nblocks, totals);
+  } else if (Vs % 4 == 0) {
+    k_row_totals_shard<float, 4><<<grid, G5_T, 0, st>>>(static_cast<const float*>(logits), rows, Vs, gathered_keys, shards,
+                                                        temperature, w.row_ac, w.block_sum, w.nblocks, totals);
+  } else {
+    k_row_totals_shard<float, 1><<<grid, G5_T, 0, st>>>(static_cast<const float*>(logits), rows, Vs, gathered_keys, shards,
+                                                        temperature, w.row_ac, w.block_sum, w.nblocks, totals);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_row_pick_shard(const void* logits, int dtype, int64_t rows, int N, int Vs, int v0, int rank, int shards,
+                                  const unsigned long long* gathered_totals, uint64_t seed, const VerifyWorkspace& w,
+                                  int32_t* pick, cudaStream_t st) {
+  if (rows == 0) return cudaSuccess;
+  const unsigned grid = (unsigned)((rows + 3) / 4);
+  if (dtype == UBT_BF16)
+    k_row_pick_shard<__nv_bfloat16><<<grid, 128, 0, st>>>(static_cast<const __nv_bfloat16*>(logits), rows, N, Vs, v0, rank, shards,
+                                                          gathered_totals, seed, w.row_ac, w.block_sum, w.nblocks, pick);
+  else
+    k_row_pick_shard<float><<<grid, 128, 0, st>>>(static_cast<const float*>(logits), rows, N, Vs, v0, rank, shards,
+                                                  gathered_totals, seed, w.row_ac, w.block_sum, w.nblocks, pick);
+  return cudaGetLastError();
 }
 
 // Number of bounded waits that gave up in this file's kernels (0 in a healthy run).

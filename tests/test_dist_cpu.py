@@ -126,6 +126,36 @@ def _shard_rank_main(rank: int, world: int, port: int, out_dir: str):
     o_ids, o_lp, _ = oracle.topk_logprob(x, k)
     np.testing.assert_array_equal(g_ids, o_ids)
     np.testing.assert_allclose(g_lp, o_lp, rtol=1e-6, atol=1e-6)
+    # ---- sampling a4 over the same split, on the host with the oracle's integer weights: maxima, totals and picks
+    # travel through the same gather (8-, 8- and 4-byte entries per tree slot, rank order), and the picks are those
+    # of whole rows
+    B, N, seed, temp = 1, rows, 77, 0.9
+    z = x.reshape(B, N, V)
+    want = oracle.verify(np.full((B, N), -1, np.int32), np.full((B, N), -1, np.int32), np.ones(B, np.int32), 3, z,
+                         "sample", seed=seed, temperature=temp).node_pick
+    local_max = torch.from_numpy(x[:, v0:v1].max(axis=1).astype(np.float32))
+    g_max, _ = u.gather_shard_partials(local_max)
+    row_max = g_max.view(world, rows).max(dim=0).values.numpy()
+    totals = np.zeros(rows, np.int64)
+    cums = []
+    for r_ in range(rows):
+        a, c = oracle.weight_consts(float(row_max[r_]), temp)
+        w = np.array([oracle.weight(float(zv), a, c) for zv in x[r_, v0:v1]], dtype=np.uint64)
+        cums.append(np.cumsum(w))
+        totals[r_] = int(cums[-1][-1])
+    g_tot, _ = u.gather_shard_partials(torch.from_numpy(totals))
+    g_tot = g_tot.view(world, rows).numpy().astype(np.uint64)
+    picks = np.full(rows, -1, np.int32)
+    for r_ in range(rows):
+        total = int(g_tot[:, r_].sum())
+        theta = oracle.threshold(seed, 0, r_, total)
+        before = int(g_tot[:rank, r_].sum())
+        if before <= theta < before + int(g_tot[rank, r_]):
+            picks[r_] = v0 + int(np.searchsorted(cums[r_], np.uint64(theta - before), side="right"))
+    g_picks, _ = u.gather_shard_partials(torch.from_numpy(picks))
+    g_picks = g_picks.view(world, rows).numpy()
+    assert ((g_picks >= 0).sum(axis=0) == 1).all()
+    np.testing.assert_array_equal(g_picks.max(axis=0), want[0])
     with open(os.path.join(out_dir, f"shard{rank}.ok"), "w") as f:
         f.write("ok")
     dist.barrier()

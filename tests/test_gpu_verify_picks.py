@@ -82,7 +82,7 @@ def test_argument_checks():
         u.ubt_verify_tree_picks(gtree, torch.zeros((cfg.B, cfg.N), dtype=torch.int64, device=DEV))
     res = binding.VerifyResult.empty(cfg.B, cfg.L, DEV)
     t, r = gtree.c_struct(), res.c_struct()
-    rc = binding.load().ubt_verify_tree_picks(C.byref(t), None, C.byref(r), None, None)
+    rc = binding.load().ubt_verify_tree_picks(C.byref(t), None, 1, C.byref(r), None, None)
     assert rc == 1                                  # UBT_ERR_INVALID_ARG
 
 

@@ -177,3 +177,92 @@ def test_sharded_greedy_verify_reports_a_nan_in_any_slice():
     u.ubt_verify_tree_keys(tree, gathered, shards, status=status)
     torch.cuda.synchronize()
     assert status.tolist() == [0, 1]
+
+
+def _sharded_sampling(u, tree, zd, cuts, seed, temperature, status=None):
+    """The four steps of sampling verification over a vocabulary-parallel group, the ranks run one after the other
+    on this GPU; the buffers that an all-gather would fill are written slice by slice."""
+    shards = len(cuts) - 1
+    B, N, _ = zd.shape
+    rows = B * N
+    shard = [zd[..., cuts[r]:cuts[r + 1]].contiguous() for r in range(shards)]
+    g_keys = torch.empty(shards * rows, dtype=torch.int64, device=DEV)
+    for r in range(shards):
+        u.ubt_verify_keys_shard(shard[r], cuts[r], g_keys[r * rows:(r + 1) * rows])
+    g_tot = torch.empty(shards * rows, dtype=torch.int64, device=DEV)
+    ws = []
+    for r in range(shards):
+        _, w = u.ubt_sample_totals_shard(shard[r], g_keys, shards, temperature, totals=g_tot[r * rows:(r + 1) * rows])
+        ws.append(w)
+    g_picks = torch.empty(shards * rows, dtype=torch.int32, device=DEV)
+    for r in range(shards):
+        u.ubt_sample_picks_shard(shard[r], cuts[r], r, g_tot, shards, seed, ws[r], picks=g_picks[r * rows:(r + 1) * rows])
+    res = u.ubt_verify_tree_picks(tree, g_picks, shards, status=status)
+    torch.cuda.synchronize()
+    return res, g_picks.view(shards, B, N)
+
+
+@pytest.mark.parametrize("V,shards,even,dtype,temperature", [
+    (8192, 4, True, "bf16", 1.0), (8192, 3, False, "bf16", 0.7), (4001, 2, False, "f32", 1.3),
+    (151936, 8, True, "bf16", 1.0), (40000, 5, False, "f32", 1.0)])
+def test_sharded_sampling_verify_equals_the_oracle(V, shards, even, dtype, temperature):
+    import paper_2609_39972_b200 as u
+    from parity import compare_verify
+    cfg = synth.CONFIGS["c2"].replace(B=3, L=6, N=24, k=4, V=V, dtype=dtype, mode="sample")
+    tree, g = _drafted(cfg, 11)
+    z = synth.agree_targets(cfg, synth.draft_inputs(cfg, 11).unigram_logits, g.token_ids, g.parents, g.depths,
+                            g.n_nodes, 11)
+    zd = synth.to_device(z, cfg.dtype, DEV)
+    cuts = _cuts(V, shards, even, 1 if not even else 8)
+    walked = 0
+    for seed in (0, 1, 12345678901234567):
+        want = oracle.verify(g.token_ids, g.parents, g.n_nodes, cfg.L, z, "sample", seed=seed, temperature=temperature)
+        status = torch.full((cfg.B,), -1, dtype=torch.int32, device=DEV)
+        res, picks = _sharded_sampling(u, tree, zd, cuts, seed, temperature, status)
+        compare_verify(res, want)
+        assert status.tolist() == [0] * cfg.B
+        # every slot has exactly one owner, and it holds the oracle's pick
+        p = picks.cpu().numpy()
+        assert ((p >= 0).sum(axis=0) == 1).all()
+        assert (p.max(axis=0) == want.node_pick).all()
+        walked += int(want.accepted_len.sum())
+        # and bit for bit what the one-GPU call gives
+        one = u.ubt_verify_tree(tree, zd, "sample", seed=seed, temperature=temperature)
+        torch.cuda.synchronize()
+        for name in ("accepted_len", "bonus_token", "accepted_nodes", "out_tokens"):
+            assert torch.equal(getattr(one, name), getattr(res, name)), name
+    assert walked > 0
+
+
+def test_sharded_sampling_reports_a_nan_or_inf_in_any_slice():
+    import paper_2609_39972_b200 as u
+    from parity import compare_verify
+    cfg = synth.CONFIGS["c2"].replace(B=3, L=6, N=24, k=4, V=8192, mode="sample")
+    tree, g = _drafted(cfg, 9)
+    z = synth.target_logits(cfg, 9)
+    clean = z.copy()
+    z[1, 3, 6000] = 0x7FC0                     # a bf16 NaN in the third slice of sequence 1
+    z[2, 0, 100] = 0x7F80                      # +inf in the first slice of sequence 2
+    zd = synth.to_device(z, cfg.dtype, DEV)
+    status = torch.zeros((cfg.B,), dtype=torch.int32, device=DEV)
+    res, picks = _sharded_sampling(u, tree, zd, [0, 2048, 4096, 6144, 8192], 3, 1.0, status)
+    assert status.tolist() == [0, 1, 1]
+    p = picks.cpu().numpy()
+    assert (p[:, 1, 3] == -1).all() and (p[:, 2, 0] == -1).all()
+    want = oracle.verify(g.token_ids[:1], g.parents[:1], g.n_nodes[:1], cfg.L, clean[:1], "sample", seed=3)
+    compare_verify(res, want, rows=[0])
+
+
+def test_sharded_sampling_argument_checks():
+    import paper_2609_39972_b200 as u
+    cfg = synth.CONFIGS["c2"].replace(B=1, L=4, N=8, k=4, V=4096)
+    zd = synth.to_device(synth.target_logits(cfg, 1), cfg.dtype, DEV)
+    keys = u.ubt_verify_keys_shard(zd, 0)
+    small = torch.empty(16, dtype=torch.uint8, device=DEV)
+    with pytest.raises(u.UbtError):
+        u.ubt_sample_totals_shard(zd, keys, 1, ws=small)                       # workspace too small
+    with pytest.raises(u.UbtError):
+        u.ubt_sample_totals_shard(zd, keys, 1, temperature=0.0)
+    totals, ws = u.ubt_sample_totals_shard(zd, keys, 1)
+    with pytest.raises(u.UbtError):
+        u.ubt_sample_picks_shard(zd, 0, 1, totals, 1, 0, ws)                   # rank outside the group
