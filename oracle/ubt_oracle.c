@@ -598,9 +598,10 @@ int ubt_oracle_verify(const int32_t *token_ids, const int32_t *parents, const in
 }
 
 /*
- * The walk alone, for picks that come from elsewhere (Appendix A, verification: "the walk stops at the first pick
- * that no child carries and keeps that pick as the bonus token").  picks[B,N] holds the target's token at every
- * slot; only the slots the walk visits are read.  Outputs as ubt_oracle_verify.
+ * The walk alone, for picks that come from elsewhere (Appendix A, verification): from the root, move to the child
+ * that carries the pick of the current slot; the first pick that no child carries ends the walk and is the bonus
+ * token.  picks[B,N] holds the target's token at every slot; only the slots the walk visits are read.  Outputs as
+ * ubt_oracle_verify.
  */
 int ubt_oracle_walk_picks(const int32_t *token_ids, const int32_t *parents, const int32_t *n_nodes,
                           int B, int N, int L, const int32_t *picks, int32_t *accepted_len,
