@@ -281,6 +281,28 @@ def test_topk_rows_that_leave_the_streaming_kernels_common_path(rows, V, k, dtyp
     np.testing.assert_allclose(clp.cpu().numpy(), lp, rtol=1e-5, atol=2e-5)
 
 
+@pytest.mark.parametrize("rows,V,k,dtype", [
+    (700, 16384, 16, "bf16"), (700, 16376, 7, "bf16"), (333, 32776, 33, "bf16"), (97, 49152, 64, "bf16"),
+    (1200, 8200, 1, "bf16"), (450, 16388, 16, "f32"), (130, 40964, 64, "f32"), (64, 151936, 50, "bf16"),
+    (9, 151936, 3, "f32")])
+def test_topk_rows_cut_at_chunk_and_span_borders(rows, V, k, dtype):
+    """Vocabularies one fragment off a multiple of the 32 KiB chunk, row counts that put the span borders (and
+    with them very short row segments) at ever different columns."""
+    u = ubt()
+    rng = np.random.default_rng(rows + V + k)
+    x = (rng.standard_normal((rows, V)) * rng.uniform(0.3, 6.0, (rows, 1))).astype(np.float32)
+    host = synth.f32_to_bf16_bits(x) if dtype == "bf16" else x
+    ids, lp, _ = oracle.topk_logprob(host, k)
+    d = synth.to_device(host, dtype, DEV)
+    cid = torch.empty((rows, k), dtype=torch.int32, device=DEV)
+    clp = torch.empty((rows, k), dtype=torch.float32, device=DEV)
+    ws = u.workspace(u.ubt_draft_workspace_bytes(rows, 1, V, k, 1), DEV)
+    u.ubt_topk_logprob(d, k, cid, clp, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(cid.cpu().numpy(), ids)
+    np.testing.assert_allclose(clp.cpu().numpy(), lp, rtol=1e-5, atol=2e-5)
+
+
 def test_exact_score_ties_follow_total_order():
     # integer-valued inputs with lambda = 0: many node scores are exactly equal in fp32 and in double
     u = ubt()
