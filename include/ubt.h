@@ -192,6 +192,16 @@ int ubt_topk_merge_shards(const void *gathered, int shards, int64_t rows, int k,
  * A device-side wait that gives up (counted by ubt_debug_ring_timeouts) leaves the outputs undefined.
  */
 size_t ubt_lm_head_workspace_bytes(int64_t rows, int d, int V, int k);
+/*
+ * The same with the head split over the ranks of a tensor-parallel group along the vocabulary, as the paper serves
+ * it: weight_shard is this rank's [Vs, d] rows of the head (tokens v0 ... v0 + Vs - 1).  Writes this rank's per-row
+ * partial in the format of ubt_topk_shard (ubt_topk_shard_bytes(rows, k) bytes: (max, sum exp), the k best raw
+ * logits of the slice with token ids of the whole vocabulary, the count; k <= Vs); after one all-gather
+ * ubt_topk_merge_shards gives every rank the candidates of the whole vocabulary.  Workspace:
+ * ubt_lm_head_workspace_bytes(rows, d, Vs, k).
+ */
+int ubt_lm_head_topk_shard(const void *hidden, const void *weight_shard, int64_t rows, int d, int Vs, int k, int v0,
+                           void *partial, void *workspace, size_t workspace_bytes, void *cuda_stream);
 int ubt_lm_head_topk(const void *hidden, const void *weight, int64_t rows, int d, int V, int k, int32_t *cand_ids,
                      float *cand_logprob, void *workspace, size_t workspace_bytes, void *cuda_stream);
 

@@ -58,7 +58,7 @@ EXPORTS = ["ubt_version", "ubt_status_string", "ubt_debug_ring_timeouts", "ubt_d
            "ubt_draft_host_buffer_bytes", "ubt_verify_host_buffer_bytes", "ubt_draft_tree_host",
            "ubt_verify_tree_host", "ubt_verify_tree_static", "ubt_verify_static_capacity", "ubt_lm_head_workspace_bytes",
            "ubt_lm_head_topk", "ubt_topk_shard_bytes", "ubt_topk_shard", "ubt_topk_merge_shards", "ubt_verify_keys_shard",
-           "ubt_verify_tree_keys", "ubt_verify_tree_picks", "ubt_sample_totals_shard", "ubt_sample_picks_shard"]
+           "ubt_verify_tree_keys", "ubt_verify_tree_picks", "ubt_sample_totals_shard", "ubt_sample_picks_shard", "ubt_lm_head_topk_shard"]
 
 _lib = None
 
@@ -104,6 +104,8 @@ def load() -> C.CDLL:
     L.ubt_lm_head_workspace_bytes.argtypes = [C.c_int64, C.c_int, C.c_int, C.c_int]
     L.ubt_lm_head_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
                                    C.c_void_p, C.c_size_t, C.c_void_p]
+    L.ubt_lm_head_topk_shard.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_int,
+                                         C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
     L.ubt_topk_shard_bytes.restype = C.c_size_t
     L.ubt_topk_shard_bytes.argtypes = [C.c_int64, C.c_int]
     L.ubt_topk_shard.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
@@ -331,6 +333,36 @@ def ubt_lm_head_topk(hidden: torch.Tensor, weight: torch.Tensor, k: int, cand_id
     _check(load().ubt_lm_head_topk(_ptr(hidden), _ptr(weight), rows, d, V, k, _ptr(cand_ids), _ptr(cand_logprob),
                                    _ptr(ws), ws.numel(), _stream(stream)), "ubt_lm_head_topk")
     return cand_ids, cand_logprob
+
+
+def ubt_lm_head_topk_shard(hidden: torch.Tensor, weight_shard: torch.Tensor, k: int, v0: int,
+                           partial: Optional[torch.Tensor] = None, ws: Optional[torch.Tensor] = None,
+                           stream=None) -> torch.Tensor:
+    """The fused LM head on this rank's ``[Vs, d]`` slice of a vocabulary-parallel head (tokens ``v0 ...``): the
+    rank's per-row partial (``ubt_topk_shard``'s format); gather and ``ubt_topk_merge_shards`` as for
+    ``ubt_topk_shard``."""
+    _need(hidden, "hidden"); _need(weight_shard, "weight_shard")
+    if hidden.dtype != torch.bfloat16 or weight_shard.dtype != torch.bfloat16:
+        raise TypeError("hidden and weight_shard must be torch.bfloat16")
+    d = hidden.shape[-1]
+    Vs = weight_shard.shape[0]
+    rows = hidden.numel() // d
+    if partial is None:
+        partial = workspace(ubt_topk_shard_bytes(rows, k), hidden.device)
+    if ws is None:
+        ws = workspace(ubt_lm_head_workspace_bytes(rows, d, Vs, k), hidden.device)
+    _check(load().ubt_lm_head_topk_shard(_ptr(hidden), _ptr(weight_shard), rows, d, Vs, k, int(v0), _ptr(partial),
+                                         _ptr(ws), ws.numel(), _stream(stream)), "ubt_lm_head_topk_shard")
+    return partial
+
+
+def lm_head_topk_vocab_parallel(hidden: torch.Tensor, weight_shard: torch.Tensor, k: int, v0: int, group=None):
+    """LM head + step a1 with the head split along the vocabulary over the ranks of ``group``: fused head on the
+    slice, one all-gather of the partials, merge.  Every rank returns the same ``(cand_ids, cand_logprob)``."""
+    rows = hidden.numel() // hidden.shape[-1]
+    partial = ubt_lm_head_topk_shard(hidden, weight_shard, k, v0)
+    gathered, shards = gather_shard_partials(partial, group)
+    return ubt_topk_merge_shards(gathered, shards, rows, k)
 
 
 def ubt_build_tree(bigram_scores: Optional[torch.Tensor], tree: Tree, stream=None, **opts) -> None:

@@ -227,6 +227,22 @@ int ubt_lm_head_topk(const void* hidden, const void* weight, int64_t rows, int d
   return UBT_OK;
 }
 
+int ubt_lm_head_topk_shard(const void* hidden, const void* weight_shard, int64_t rows, int d, int Vs, int k, int v0,
+                           void* partial, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!hidden || !weight_shard || !partial || rows < 0 || d < 1 || Vs < 1 || k < 1 || k > Vs || v0 < 0)
+    return UBT_ERR_INVALID_ARG;
+  if (!aligned16(hidden) || !aligned16(weight_shard) || !aligned16(partial)) return UBT_ERR_INVALID_ARG;
+  if (d % 64 != 0 || k > lm_head_max_k() || rows > lm_head_max_rows() || device_info().sm_count > 256 ||
+      (int64_t)v0 + Vs > 0x7fffffffll)
+    return UBT_ERR_UNSUPPORTED;
+  if (rows == 0) return UBT_OK;
+  if (!workspace || !aligned16(workspace) || workspace_bytes < lm_head_workspace_bytes(rows, k)) return UBT_ERR_WORKSPACE;
+  cudaError_t e = launch_lm_head_topk(hidden, weight_shard, rows, d, Vs, k, nullptr, nullptr, workspace,
+                                      static_cast<cudaStream_t>(cuda_stream), partial, v0);
+  if (e != cudaSuccess) { cudaGetLastError(); return e == cudaErrorNotSupported ? UBT_ERR_UNSUPPORTED : UBT_ERR_CUDA; }
+  return UBT_OK;
+}
+
 static int check_draft_opts(const ubt_draft_opts* o) {
   if (!o) return UBT_OK;
   if (o->search_width < 0 || !(o->depth_bonus <= 0.0f)) return UBT_ERR_INVALID_ARG;

@@ -80,6 +80,8 @@ cudaError_t launch_merge_topk(int64_t rows, int V, int k, const TopkWorkspace& w
                               float* cand_lp, cudaStream_t st);
 // Vocabulary-parallel a1: this rank's per-row partial from its slice, and the merge of the gathered partials.
 size_t shard_partial_bytes(int64_t rows, int k);
+// The four arrays of one rank's partial inside its buffer, ids to be moved by id_offset when written.
+MergeShardOut carve_shard_partial(void* partial, int64_t rows, int k, int id_offset);
 cudaError_t launch_merge_topk_shard(int64_t rows, int V, int k, const TopkWorkspace& w, void* partial, int v0,
                                     cudaStream_t st);
 cudaError_t launch_merge_shards(const void* gathered, int shards, int64_t rows, int k, int32_t* cand_ids,
@@ -148,8 +150,11 @@ cudaError_t selector_timeouts(unsigned int* out);
 int lm_head_max_k();
 int lm_head_max_rows();
 size_t lm_head_workspace_bytes(int64_t rows, int k);
+// shard_partial != nullptr: `weight` is the slice [V, d] of a vocabulary-parallel head that starts at column v0 of
+// the whole vocabulary, and the result is this rank's partial (ubt_topk_shard's format) instead of candidates
 cudaError_t launch_lm_head_topk(const void* hidden, const void* weight, int64_t rows, int d, int V, int k,
-                                int32_t* cand_ids, float* cand_lp, void* ws, cudaStream_t st);
+                                int32_t* cand_ids, float* cand_lp, void* ws, cudaStream_t st,
+                                void* shard_partial = nullptr, int v0 = 0);
 
 // ---- a4, path-only form: evaluates only the target rows the walk visits (ubt_verify_path.cu)
 size_t verify_path_workspace_bytes(int B, int N, int mode);

@@ -29,6 +29,7 @@
 #include <mutex>
 
 #include "ubt_internal.h"
+#include "ubt_merge.cuh"
 #include "ubt_tc.cuh"
 
 namespace ubt {
@@ -349,7 +350,10 @@ k_lm_head_topk(const __grid_constant__ CUtensorMap map_h, const __grid_constant_
 // One warp per row: (max, sum) over the CTAs' partials, then the k best of their sorted lists by k rounds of
 // "best head"; cand_lp = value - log-sum-exp.
 __global__ void __launch_bounds__(128)
-k_lm_head_merge(LmParts parts, int grid, int rows, int k, int32_t* __restrict__ cand_ids, float* __restrict__ cand_lp) {
+k_lm_head_merge(LmParts parts, int grid, int rows, int k, int32_t* __restrict__ cand_ids, float* __restrict__ cand_lp,
+                MergeShardOut so) {
+  // so.ms set: this GPU holds a slice of the vocabulary; the row's result is written as the rank's partial of a
+  // vocabulary-parallel a1 (raw values, ids moved by the slice's first column, (max, sum exp), count) instead
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (row >= rows) return;
@@ -372,6 +376,7 @@ k_lm_head_merge(LmParts parts, int grid, int rows, int k, int32_t* __restrict__ 
   int head[8];
 #pragma unroll
   for (int q = 0; q < 8; ++q) head[q] = 0;
+  int found = 0;
   for (int r = 0; r < k; ++r) {
     unsigned long long best = 0ull;
     int bq = -1;
@@ -388,17 +393,28 @@ k_lm_head_merge(LmParts parts, int grid, int rows, int k, int32_t* __restrict__ 
     }
     const unsigned long long win = warp_max_u64(best);
     if (win == 0ull) {  // fewer than k entries in the whole row
-      if (lane == 0) { cand_ids[(size_t)row * k + r] = -1; cand_lp[(size_t)row * k + r] = -INFINITY; }
+      if (lane == 0 && !so.ms) { cand_ids[(size_t)row * k + r] = -1; cand_lp[(size_t)row * k + r] = -INFINITY; }
       continue;
     }
+    ++found;
     const unsigned holders = __ballot_sync(FULL, best == win);  // keys are unique: one lane holds it
     if (lane == __ffs(holders) - 1) {
 #pragma unroll
       for (int q = 0; q < 8; ++q)
         if (q == bq) head[q] += 1;
-      cand_ids[(size_t)row * k + r] = key_idx(win);
-      cand_lp[(size_t)row * k + r] = key_val(win) - lse;
+      if (so.ms) {
+        so.idx[(size_t)row * k + r] = key_idx(win) + so.id_offset;
+        so.val[(size_t)row * k + r] = key_val(win);
+      } else {
+        cand_ids[(size_t)row * k + r] = key_idx(win);
+        cand_lp[(size_t)row * k + r] = key_val(win) - lse;
+      }
     }
+  }
+  if (so.ms && lane == 0) {
+    so.ms[(size_t)row * 2] = M;
+    so.ms[(size_t)row * 2 + 1] = S;
+    so.cnt[row] = found;
   }
 }
 
@@ -449,7 +465,8 @@ size_t lm_head_workspace_bytes(int64_t rows, int k) {
 
 // Returns cudaSuccess, or an error; *device_failed (host) is set if a bounded wait gave up on the device.
 cudaError_t launch_lm_head_topk(const void* hidden, const void* weight, int64_t rows, int d, int V, int k,
-                                int32_t* cand_ids, float* cand_lp, void* ws, cudaStream_t st) {
+                                int32_t* cand_ids, float* cand_lp, void* ws, cudaStream_t st, void* shard_partial,
+                                int v0) {
   if (rows == 0) return cudaSuccess;
   const int grid = device_info().sm_count;
   const size_t smem = (size_t)LM_RING_BYTES + sizeof(LmShared);
@@ -512,7 +529,9 @@ cudaError_t launch_lm_head_topk(const void* hidden, const void* weight, int64_t 
     k_lm_head_topk<16><<<grid, LM_THREADS, smem, st>>>(map_h, map_w, map_w2, (int)rows, d, V, k, a_rows, n_stages, tl, parts, fail_flag);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  k_lm_head_merge<<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(parts, grid, (int)rows, k, cand_ids, cand_lp);
+  MergeShardOut so{};
+  if (shard_partial) so = carve_shard_partial(shard_partial, rows, k, v0);
+  k_lm_head_merge<<<(unsigned)((rows + 3) / 4), 128, 0, st>>>(parts, grid, (int)rows, k, cand_ids, cand_lp, so);
   return cudaGetLastError();
 }
 

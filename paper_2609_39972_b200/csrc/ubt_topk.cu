@@ -768,7 +768,7 @@ size_t shard_partial_bytes(int64_t rows, int k) {
          align_up((size_t)rows * sizeof(int32_t), 256);
 }
 // The four arrays of one rank's partial: (max, sum exp) [rows,2], values [rows,k], ids [rows,k], counts [rows].
-static MergeShardOut carve_shard_partial(void* partial, int64_t rows, int k, int id_offset) {
+MergeShardOut carve_shard_partial(void* partial, int64_t rows, int k, int id_offset) {
   unsigned char* p = static_cast<unsigned char*>(partial);
   MergeShardOut so{};
   so.ms = reinterpret_cast<float*>(p); p += align_up((size_t)rows * 2 * sizeof(float), 256);

@@ -87,3 +87,30 @@ def test_argument_checks():
     with pytest.raises(u.UbtError) as ei:
         u.ubt_lm_head_topk(h, w, 17, ws=u.workspace(1 << 20, DEV))      # beyond the fused epilogue's k
     assert ei.value.status == 2
+
+
+@pytest.mark.parametrize("rows,d,V,k,cuts", [(200, 128, 5000, 8, [0, 1200, 2608, 5000]),
+                                              (300, 256, 20011, 16, [0, 5003, 10006, 15009, 20011]),
+                                              (64, 64, 4096, 1, [0, 2048, 4096])])
+def test_head_split_along_the_vocabulary_matches_the_whole_head(rows, d, V, k, cuts):
+    """The ranks of a tensor-parallel group, one after the other on this GPU: fused head on each slice of the head
+    matrix, the partials laid out as an all-gather would, merge; against the oracle on the whole head and against
+    the one-GPU fused call."""
+    import paper_2609_39972_b200 as u
+    h, w = synth.lm_head_inputs(rows, d, V, seed=rows + V, scale=3.0)
+    hd, wd = synth.to_device(h, "bf16", DEV), synth.to_device(w, "bf16", DEV)
+    shards = len(cuts) - 1
+    nbytes = u.ubt_topk_shard_bytes(rows, k)
+    gathered = torch.empty(shards * nbytes, dtype=torch.uint8, device=DEV)
+    for r in range(shards):
+        u.ubt_lm_head_topk_shard(hd, wd[cuts[r]:cuts[r + 1]].contiguous(), k, cuts[r],
+                                 partial=gathered[r * nbytes:(r + 1) * nbytes])
+    ids_g, lp_g = u.ubt_topk_merge_shards(gathered, shards, rows, k)
+    torch.cuda.synchronize()
+    assert u.ubt_debug_ring_timeouts() == 0
+    o_ids, o_lp, o_lse, o_logits = oracle.lm_head_topk(h, w, k, want_logits=True)
+    check_rows(ids_g.cpu().numpy(), lp_g.cpu().numpy().astype(np.float64), o_ids, o_lp, o_lse, o_logits, k)
+    ids_1, lp_1 = u.ubt_lm_head_topk(hd, wd, k)
+    torch.cuda.synchronize()
+    assert float((ids_1 == ids_g).float().mean()) > 0.99          # the same up to near-ties
+    assert float((lp_1 - lp_g).abs().max()) < 2e-4
