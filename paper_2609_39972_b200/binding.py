@@ -552,6 +552,14 @@ def verify_tree_from_hidden(tree: Tree, target_hidden: torch.Tensor, weight: tor
     return ubt_verify_tree_picks(tree, picks, **kw)
 
 
+def verify_tree_from_hidden_vocab_parallel(tree: Tree, target_hidden: torch.Tensor, weight_shard: torch.Tensor,
+                                           v0: int, group=None, **kw) -> VerifyResult:
+    """Greedy verification from the target's hidden states with the head split along the vocabulary over the ranks
+    of ``group``: fused head + arg max on the slice (k = 1), one all-gather of ``20 B`` per tree slot, merge, walk."""
+    picks, _ = lm_head_topk_vocab_parallel(target_hidden.reshape(tree.B * tree.N, -1), weight_shard, 1, v0, group)
+    return ubt_verify_tree_picks(tree, picks, **kw)
+
+
 def verify_tree_vocab_parallel(tree: Tree, target_shard: torch.Tensor, v0: int, group=None, **kw) -> VerifyResult:
     """Greedy verification of target logits whose vocabulary is split over the ranks of ``group``: local keys, one
     all-gather, walk; all on torch's current stream.  Every rank returns the same verdict."""

@@ -107,3 +107,30 @@ def test_greedy_verification_from_hidden_states(B, N, L, k, d, V, seed):
     torch.cuda.synchronize()
     assert u.ubt_debug_ring_timeouts() == 0
     compare_verify(res, ov, res.node_pick)
+
+
+def test_greedy_verification_from_hidden_states_with_a_split_head():
+    """The head cut into three vocabulary slices (ranks emulated one after the other): k = 1 partial per slice, merge,
+    walk; the same verdict as the whole head."""
+    import paper_2609_39972_b200 as u
+    B, N, L, k, d, V = 3, 32, 6, 4, 128, 6000
+    cfg = synth.CONFIGS["c1"].replace(name="h", B=B, L=L, V=V, k=k, N=N)
+    gtree, g = drafted_tree(u, cfg, 3)
+    want = picks_that_walk(g, cfg, 103)
+    _, w = synth.lm_head_inputs(1, d, V, seed=10, scale=8.0)
+    hidden = synth.f32_to_bf16_bits(synth.as_f32(w, "bf16")[want.reshape(-1)] * 4.0)
+    ov = oracle.verify_picks(g.token_ids, g.parents, g.n_nodes, L, oracle.lm_head_topk(hidden, w, 1)[0].reshape(B, N))
+    hd, wd = synth.to_device(hidden, "bf16", DEV), synth.to_device(w, "bf16", DEV)
+    cuts, rows = [0, 1808, 4000, V], B * N
+    nbytes = u.ubt_topk_shard_bytes(rows, 1)
+    gathered = torch.empty(3 * nbytes, dtype=torch.uint8, device=DEV)
+    for r in range(3):
+        u.ubt_lm_head_topk_shard(hd, wd[cuts[r]:cuts[r + 1]].contiguous(), 1, cuts[r],
+                                 partial=gathered[r * nbytes:(r + 1) * nbytes])
+    picks, _ = u.ubt_topk_merge_shards(gathered, 3, rows, 1)
+    res = u.ubt_verify_tree_picks(gtree, picks)
+    torch.cuda.synchronize()
+    compare_verify(res, ov, res.node_pick)
+    one = u.verify_tree_from_hidden_vocab_parallel(gtree, hd.view(B, N, d), wd, 0)     # a group of one
+    torch.cuda.synchronize()
+    compare_verify(one, ov, one.node_pick)
