@@ -690,6 +690,7 @@ __device__ __forceinline__ int expand_rounds_warp(TreeSmem& s, int L, int k, int
 // scalars[1] = node count, scalars[2] = threshold key, scalars[3] = flags (1: nothing left, 2: out of room,
 // 4: smallest step).
 constexpr int EX_T = 128;
+constexpr float kFirstShare = 3.0f;  // first threshold of the rounds: path probability kFirstShare / budget
 __device__ __forceinline__ void ex_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(EX_T) : "memory"); }
 
 __device__ __forceinline__ void prepare_rows(TreeSmem& s, int k, int row0, int nrows, int tid, int nthreads);
@@ -762,6 +763,14 @@ __device__ __forceinline__ int expand_rounds_cta(TreeSmem& s, int L, int k, int 
           ks = ks < tau_full ? tau_full : ks;
           tau = ks < tau ? ks : tau;
         }
+      }
+      if (guard == 0) {
+        // First round: the successor scores of a row are normalised (eq. 9), so a node's score is the logarithm of
+        // a path probability (plus depth * zeta <= 0) and at most 1 / theta nodes of a depth reach ln theta: start
+        // at theta = kFirstShare / budget instead of at the best child of the root.
+        uint32_t k1 = f2key(-__logf((float)budget * (1.0f / kFirstShare)));
+        k1 = k1 == 0u ? 1u : k1;
+        tau = k1 < tau ? k1 : tau;
       }
       if (tau > kmax) tau = kmax;  // a round must add at least the best open child
       if (lane == 0) {
