@@ -690,7 +690,7 @@ __device__ __forceinline__ int expand_rounds_warp(TreeSmem& s, int L, int k, int
 // scalars[1] = node count, scalars[2] = threshold key, scalars[3] = flags (1: nothing left, 2: out of room,
 // 4: smallest step).
 constexpr int EX_T = 128;
-constexpr float kFirstShare = 3.0f;  // first threshold of the rounds: path probability kFirstShare / budget
+constexpr float kFirstShare = 1.5f;  // first threshold of the rounds: path probability kFirstShare / budget
 __device__ __forceinline__ void ex_barrier() { asm volatile("bar.sync 1, %0;" ::"n"(EX_T) : "memory"); }
 
 __device__ __forceinline__ void prepare_rows(TreeSmem& s, int k, int row0, int nrows, int tid, int nthreads);
