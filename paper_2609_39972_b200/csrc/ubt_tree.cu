@@ -783,32 +783,29 @@ __device__ __forceinline__ int expand_rounds_cta(TreeSmem& s, int L, int k, int 
     const bool smallest_step = (s.scalars[3] & 4) != 0;
     const uint32_t tau = (uint32_t)s.scalars[2];
     const int n_before = n;
-    // The qualifying children of node i, then those of the first child appended, and so on down (a chain of
-    // best children costs one wave); every level reserves its places with the shared counter.
+    // The children of node i that reach the threshold (a row is sorted: they are the next ones in it); they
+    // reserve their places with the shared counter and are visited themselves in the next wave.  (Walking on down
+    // the first child in the same wave was measured: the long serial chains cost more than the waves they save
+    // once a round adds dozens of nodes.)
     auto chain = [&](int i) {
-      int d = s.x_depth[i], r = s.x_rank[i], j0 = s.x_next[i], par = i;
-      float sc = s.x_score[i];
-      while (d < L) {
-        const int base = (d * k + r) * k;
-        int c = 0;
-        while (j0 + c < k && f2key(sc + s.t[base + j0 + c] + zeta) >= tau) ++c;
-        if (c == 0) break;
-        const int at = atomicAdd(&s.scalars[1], c);
-        if (at + c > cap) { atomicOr(&s.scalars[3], 2); break; }
-        for (int q = 0; q < c; ++q) {
-          const int idx = at + q;
-          s.x_parent[idx] = (short)par; s.x_depth[idx] = (unsigned char)(d + 1);
-          s.x_rank[idx] = s.ord[base + j0 + q]; s.x_score[idx] = sc + s.t[base + j0 + q] + zeta;
-          s.x_next[idx] = 0;
-        }
-        s.x_next[par] = (unsigned char)(j0 + c);
-        if (d + 1 >= d_ready && d_ready < L) {  // the children just appended open rows that are not prepared yet
-          atomicOr(&s.scalars[3], 8);
-          break;
-        }
-        sc = sc + s.t[base + j0] + zeta; r = s.ord[base + j0];
-        par = at; d += 1; j0 = 0;
+      const int d = s.x_depth[i];
+      if (d >= L) return;
+      const int j0 = s.x_next[i], base = (d * k + (int)s.x_rank[i]) * k;
+      const float sc = s.x_score[i];
+      int c = 0;
+      while (j0 + c < k && f2key(sc + s.t[base + j0 + c] + zeta) >= tau) ++c;
+      if (c == 0) return;
+      const int at = atomicAdd(&s.scalars[1], c);
+      if (at + c > cap) { atomicOr(&s.scalars[3], 2); return; }
+      for (int q = 0; q < c; ++q) {
+        const int idx = at + q;
+        s.x_parent[idx] = (short)i; s.x_depth[idx] = (unsigned char)(d + 1);
+        s.x_rank[idx] = s.ord[base + j0 + q]; s.x_score[idx] = sc + s.t[base + j0 + q] + zeta;
+        s.x_next[idx] = 0;
       }
+      s.x_next[i] = (unsigned char)(j0 + c);
+      // the children just appended open rows that are not prepared yet
+      if (d + 1 >= d_ready && d_ready < L) atomicOr(&s.scalars[3], 8);
     };
     int lo = 0, hi = n;
     bool first = true, overflow = false;
