@@ -718,70 +718,76 @@ __device__ __forceinline__ int expand_rounds_cta(TreeSmem& s, int L, int k, int 
   for (int guard = 0; budget - (n - 1) > 0; ++guard) {
     if (guard > 16 * (budget + 16)) return -1;
     const int remaining = budget - (n - 1);
-    if (tid < 32) {
-      const int idx = n <= 32 ? lane : (lane * n) >> 5;
-      const uint32_t mine = idx < n ? open_key(idx) : 0u;
-      int ls = __popc(__ballot_sync(FULL, mine != 0u));
-      uint32_t kmax = __reduce_max_sync(FULL, mine);
-      int live = n <= 32 ? ls : (ls * n + 31) >> 5;  // beyond 32 nodes an estimate is all the rule needs
-      if (ls == 0 && n > 32) {                       // none in the sample: look at every node
-        int cnt = 0;
-        for (int i = lane; i < n; i += 32) {
-          const uint32_t key = open_key(i);
-          cnt += key != 0u;
-          kmax = key > kmax ? key : kmax;
+    uint32_t tau = 0u;
+    bool smallest_step = false;
+    if (guard == 0) {
+      // First round (only the root is there): the successor scores of a row are normalised (eq. 9), so a node's
+      // score is the logarithm of a path probability (plus depth * zeta <= 0) and at most 1 / theta nodes of a depth
+      // reach ln theta: start at theta = kFirstShare / budget instead of at the best child of the root.  Every
+      // thread computes it; no barrier.
+      const uint32_t kbest = open_key(0);
+      if (kbest == 0u) break;
+      uint32_t k1 = f2key(-__logf((float)budget * (1.0f / kFirstShare)));
+      k1 = k1 == 0u ? 1u : k1;
+      tau = k1 < kbest ? k1 : kbest;  // a round must add at least the best open child
+    } else {
+      if (tid < 32) {
+        const int idx = n <= 32 ? lane : (lane * n) >> 5;
+        const uint32_t mine = idx < n ? open_key(idx) : 0u;
+        int ls = __popc(__ballot_sync(FULL, mine != 0u));
+        uint32_t kmax = __reduce_max_sync(FULL, mine);
+        int live = n <= 32 ? ls : (ls * n + 31) >> 5;  // beyond 32 nodes an estimate is all the rule needs
+        if (ls == 0 && n > 32) {                       // none in the sample: look at every node
+          int cnt = 0;
+          for (int i = lane; i < n; i += 32) {
+            const uint32_t key = open_key(i);
+            cnt += key != 0u;
+            kmax = key > kmax ? key : kmax;
+          }
+          live = __reduce_add_sync(FULL, cnt);
+          kmax = __reduce_max_sync(FULL, kmax);
         }
-        live = __reduce_add_sync(FULL, cnt);
-        kmax = __reduce_max_sync(FULL, kmax);
-      }
-      const int half = (live + 1) >> 1;
-      int m = (remaining < half ? remaining : half) >> (2 * shrink);
-      m = m < 1 ? 1 : m;
-      int r = 0;
-#pragma unroll 8
-      for (int j = 0; j < 32; ++j) {
-        const uint32_t kj = __shfl_sync(FULL, mine, j);
-        r += (kj > mine) || (kj == mine && j < lane);
-      }
-      int want = ls > 0 ? (m * ls + live - 1) / (live > 0 ? live : 1) - 1 : 0;
-      want = want < 0 ? 0 : (want > ls - 1 ? ls - 1 : want);
-      const unsigned holder = __ballot_sync(FULL, mine != 0u && r == want);
-      uint32_t tau = holder ? __shfl_sync(FULL, mine, __ffs(holder) - 1) : kmax;
-      if (shrink == 0 && n_prev2 >= 8 && n_prev > n_prev2 && t_prev < t_prev2) {
-        // secant step, never below the key that the rank rule gives for the whole open budget
-        int mf = remaining < live ? remaining : live;
-        int wf = ls > 0 ? (mf * ls + live - 1) / (live > 0 ? live : 1) - 1 : 0;
-        wf = wf < 0 ? 0 : (wf > ls - 1 ? ls - 1 : wf);
-        const unsigned hf = __ballot_sync(FULL, mine != 0u && r == wf);
-        const uint32_t tau_full = hf ? __shfl_sync(FULL, mine, __ffs(hf) - 1) : tau;
-        const float ln1 = __logf((float)n_prev2), ln2 = __logf((float)n_prev);
-        const float slope = (ln2 - ln1) / (t_prev2 - t_prev);
-        const float ts = t_prev - (__logf((float)(budget + 1)) - ln2) / slope;
-        if (ts == ts && ts < 0.f) {
-          uint32_t ks = f2key(ts);
-          ks = ks == 0u ? 1u : ks;
-          ks = ks < tau_full ? tau_full : ks;
-          tau = ks < tau ? ks : tau;
+        const int half = (live + 1) >> 1;
+        int m = (remaining < half ? remaining : half) >> (2 * shrink);
+        m = m < 1 ? 1 : m;
+        int r = 0;
+  #pragma unroll 8
+        for (int j = 0; j < 32; ++j) {
+          const uint32_t kj = __shfl_sync(FULL, mine, j);
+          r += (kj > mine) || (kj == mine && j < lane);
+        }
+        int want = ls > 0 ? (m * ls + live - 1) / (live > 0 ? live : 1) - 1 : 0;
+        want = want < 0 ? 0 : (want > ls - 1 ? ls - 1 : want);
+        const unsigned holder = __ballot_sync(FULL, mine != 0u && r == want);
+        tau = holder ? __shfl_sync(FULL, mine, __ffs(holder) - 1) : kmax;
+        if (shrink == 0 && n_prev2 >= 8 && n_prev > n_prev2 && t_prev < t_prev2) {
+          // secant step, never below the key that the rank rule gives for the whole open budget
+          int mf = remaining < live ? remaining : live;
+          int wf = ls > 0 ? (mf * ls + live - 1) / (live > 0 ? live : 1) - 1 : 0;
+          wf = wf < 0 ? 0 : (wf > ls - 1 ? ls - 1 : wf);
+          const unsigned hf = __ballot_sync(FULL, mine != 0u && r == wf);
+          const uint32_t tau_full = hf ? __shfl_sync(FULL, mine, __ffs(hf) - 1) : tau;
+          const float ln1 = __logf((float)n_prev2), ln2 = __logf((float)n_prev);
+          const float slope = (ln2 - ln1) / (t_prev2 - t_prev);
+          const float ts = t_prev - (__logf((float)(budget + 1)) - ln2) / slope;
+          if (ts == ts && ts < 0.f) {
+            uint32_t ks = f2key(ts);
+            ks = ks == 0u ? 1u : ks;
+            ks = ks < tau_full ? tau_full : ks;
+            tau = ks < tau ? ks : tau;
+          }
+        }
+        if (tau > kmax) tau = kmax;  // a round must add at least the best open child
+        if (lane == 0) {
+          s.scalars[2] = (int)tau;
+          s.scalars[3] = (live == 0 || kmax == 0u ? 1 : 0) | (m == 1 && shrink > 0 ? 4 : 0);
         }
       }
-      if (guard == 0) {
-        // First round: the successor scores of a row are normalised (eq. 9), so a node's score is the logarithm of
-        // a path probability (plus depth * zeta <= 0) and at most 1 / theta nodes of a depth reach ln theta: start
-        // at theta = kFirstShare / budget instead of at the best child of the root.
-        uint32_t k1 = f2key(-__logf((float)budget * (1.0f / kFirstShare)));
-        k1 = k1 == 0u ? 1u : k1;
-        tau = k1 < tau ? k1 : tau;
-      }
-      if (tau > kmax) tau = kmax;  // a round must add at least the best open child
-      if (lane == 0) {
-        s.scalars[2] = (int)tau;
-        s.scalars[3] = (live == 0 || kmax == 0u ? 1 : 0) | (m == 1 && shrink > 0 ? 4 : 0);
-      }
+      ex_barrier();
+      if (s.scalars[3] & 1) break;
+      smallest_step = (s.scalars[3] & 4) != 0;
+      tau = (uint32_t)s.scalars[2];
     }
-    ex_barrier();
-    if (s.scalars[3] & 1) break;
-    const bool smallest_step = (s.scalars[3] & 4) != 0;
-    const uint32_t tau = (uint32_t)s.scalars[2];
     const int n_before = n;
     // The children of node i that reach the threshold (a row is sorted: they are the next ones in it); they
     // reserve their places with the shared counter and are visited themselves in the next wave.  (Walking on down
